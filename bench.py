@@ -1,0 +1,264 @@
+#!/usr/bin/env python
+"""Benchmark of the batch-1 decode step: ms/token and achieved fraction of the HBM roofline.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+One "step" is one decode step (one token) of the named decoder shape over its pre-filled KV cache,
+i.e. one replay of the step graph.  The default workload is the Qwen2.5-1.5B-shaped decoder with a
+2048-position cache.  With N > 1 (torchrun) every rank runs an independent replica of the same
+request (the step does not shard; there is no collective on the data path).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+import numpy as np
+
+from edgefm_synth import CONFIGS, GLOBAL_SEED, first_token, make_kv, make_weights
+
+METRIC = "batch1_decode_ms_per_token"
+UNIT = "ms/token"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            return float(json.loads(p.read_text())["hbm_gbs"]), "measured (MEASURED_PEAKS.json, torch copy read+write)"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """nvidia-smi sampled every 200 ms while the timed region runs (read-only queries)."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            f = tempfile.NamedTemporaryFile("w", suffix=".csv", delete=False)
+            self.path = f.name
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "200", "-i", str(self.gpu)], stdout=f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in Path(self.path).read_text().splitlines():
+                c = [x.strip() for x in line.split(",")]
+                if len(c) < 9:
+                    continue
+                try:
+                    sm.append(float(c[1])); mx.append(float(c[2]))
+                except ValueError:
+                    continue
+                for n, val in zip(names, c[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(n)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def time_oracle(cfg, weights, k, v, steps: int, warmup: int):
+    """The CPU oracle as it stands, on the host cores: `steps` decode steps from the configured cache."""
+    from oracle import OracleModel
+    m = OracleModel(cfg, weights, cfg.cache_len + steps + warmup)
+    m.load_kv(k, v)
+    tok, pos = first_token(cfg), cfg.first_position
+    for _ in range(warmup):
+        _, tok = m.step(tok, pos); pos += 1
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        _, tok = m.step(tok, pos); pos += 1
+    dt = time.perf_counter() - t0
+    m.close()
+    return dt / steps * 1e3
+
+
+def run_reference(args, cfg, rank):
+    if rank != 0:
+        return
+    cores = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
+    os.environ["OMP_NUM_THREADS"] = str(cores)
+    weights = make_weights(cfg)
+    k, v = make_kv(cfg)
+    ms = time_oracle(cfg, weights, k, v, args.steps, args.warmup)
+    sample = f"{args.steps} full oracle decode steps of {cfg.name} from a {cfg.cache_len}-position cache (fp64 accumulation)"
+    line = {"impl": "reference", "metric": METRIC, "value": ms, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64 accumulate over bf16 weights", "data": "synthetic",
+            "config": {"workload": workload_name(cfg)},
+            "cpu_baseline": {"value": ms, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": ms, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def workload_name(cfg):
+    return (f"{cfg.name}-shaped decoder, batch 1, {cfg.cache_len}-position bf16 KV cache, greedy decode steps "
+            f"(L={cfg.n_layers} H={cfg.hidden} heads={cfg.n_q_heads}/{cfg.n_kv_heads} d={cfg.head_dim} F={cfg.ffn} V={cfg.vocab})")
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=128)
+    ap.add_argument("--warmup", type=int, default=16)
+    ap.add_argument("--config", default="qwen2.5-1.5b", choices=sorted(CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU-oracle timing leg")
+    ap.add_argument("--cpu-steps", type=int, default=3)
+    args = ap.parse_args()
+    cfg = CONFIGS[args.config]
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, cfg, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2604_27476_b200 import DecodeContext, build as cuda_build, edgefm_decode_step, upload_weights
+
+    if rank == 0:
+        cuda_build.build()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the decode step has no CPU path")
+    dev = f"cuda:{local_rank}"
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+        dist.barrier()
+
+    steps, warmup = args.steps, max(args.warmup, 0)
+    weights = make_weights(cfg)
+    k, v = make_kv(cfg)
+    ptrs, keep = upload_weights(weights, dev)
+    span = max(steps, warmup, 1)
+    ctx = DecodeContext(cfg, ptrs, cfg.cache_len + span, dev)
+    kd = torch.from_numpy(k.view(np.int16)).to(dev)
+    vd = torch.from_numpy(v.view(np.int16)).to(dev)
+    stream = torch.cuda.current_stream().cuda_stream
+    tok0, pos0 = first_token(cfg), cfg.first_position
+    handle = ctx.handle
+
+    def free_run(n):
+        """n chained greedy steps, token and position carried on the device (one graph launch per token)."""
+        ctx.prefill_kv(kd, vd)
+        edgefm_decode_step(handle, tok0, pos0, stream, None, None)
+        for _ in range(n - 1):
+            edgefm_decode_step(handle, -1, -1, stream, None, None)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- device-resident timing (inputs in HBM; weights 3 GB >> L2, so no flush between steps) ---------
+    if warmup:
+        free_run(warmup)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ctx.prefill_kv(kd, vd)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    edgefm_decode_step(handle, tok0, pos0, stream, None, None)
+    for _ in range(steps - 1):
+        edgefm_decode_step(handle, -1, -1, stream, None, None)
+    e1.record()
+    barrier()
+    dev_ms = e0.elapsed_time(e1)
+
+    # ---- end to end through the C ABI with host buffers: the token crosses PCIe both ways every step ----
+    host_tok = torch.zeros(1, dtype=torch.int32).pin_memory()
+    ctx.prefill_kv(kd, vd)
+    barrier()
+    t0 = time.perf_counter()
+    tok, pos = tok0, pos0
+    for _ in range(steps):
+        edgefm_decode_step(handle, tok, pos, stream, None, ctx.next_token.data_ptr())   # request block: host -> device
+        host_tok.copy_(ctx.next_token, non_blocking=True)                                # result: device -> host
+        torch.cuda.current_stream().synchronize()
+        tok, pos = int(host_tok[0]), pos + 1
+    e2e_ms = (time.perf_counter() - t0) * 1e3
+    clocks = sampler.stop()
+
+    times = torch.tensor([dev_ms, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    dev_ms, e2e_ms = float(times[0]), float(times[1])
+    launches = ctx.launches_per_step
+
+    if rank == 0:
+        tokens = steps * world
+        ms_per_token = dev_ms / tokens
+        bytes_per_step = float(np.mean([cfg.step_bytes(cfg.cache_len + i) for i in range(steps)]))
+        gbs = bytes_per_step / (dev_ms / steps * 1e-3) / 1e9          # per GPU
+        peak, peak_src = measured_peak()
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            cores = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
+            cpu_ms = time_oracle(cfg, weights, k, v, args.cpu_steps, 1)
+            cpu = {"value": cpu_ms, "unit": UNIT, "cores": cores, "kind": "oracle",
+                   "sample": f"{args.cpu_steps} full oracle decode steps at context {cfg.cache_len} (after 1 warm-up step)"}
+        line = {
+            "metric": METRIC, "value": ms_per_token, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+            "ms_per_step": dev_ms / steps, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16 weights/KV, fp32 accumulate", "data": "synthetic",
+            "config": {"workload": workload_name(cfg), "replicas": world, "l2": "working set 3 GB per step exceeds L2; no flush",
+                       "seed": GLOBAL_SEED},
+            "tokens_per_s": tokens / (dev_ms * 1e-3),
+            "roofline": {"bound": "hbm", "kernel": f"whole decode step ({launches} kernels in one CUDA graph)",
+                         "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak, "peak_source": peak_src,
+                         "bytes_per_launch": bytes_per_step, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS, "traffic": None},
+            "e2e": {"value": e2e_ms / tokens, "unit": UNIT, "h2d_bytes_per_step": 24, "d2h_bytes_per_step": 4},
+            "gpu_launches": launches * steps,
+            "clocks": clocks,
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

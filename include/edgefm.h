@@ -1,0 +1,146 @@
+/*
+ * edgefm.h -- C ABI of the batch-1 decode step of a Qwen2.5-style decoder on one NVIDIA B200.
+ *
+ * The library implements the decode phase of Eq. 4 of the paper,
+ *     y_t <- DecodeStep(y_{t-1}, KV; theta_d),   KV <- UpdateKV(KV, y_t),
+ * for one request slot (Sec. 3.7, 3.9: a slot owns a pre-allocated KV cache) with greedy sampling
+ * (Sec. 4.2: temperature 0, top_k = 1), replayed as one fixed CUDA graph per token whose dynamic
+ * parameters (token, position, cache length) live in device memory (Sec. 3.10).
+ *
+ * Conventions
+ *   - "device" pointers are CUDA device pointers on the device that was current at edgefm_create;
+ *     "host" pointers are ordinary host memory.  All bf16 data is raw 16-bit patterns.
+ *   - Weights are BORROWED: the caller allocates them, keeps them alive and unmodified until
+ *     edgefm_destroy.  The context OWNS its KV cache, work buffers, device state and CUDA graph.
+ *   - edgefm_prefill_kv and edgefm_decode_step only enqueue work on `stream` (a cudaStream_t passed
+ *     as void*; NULL = the legacy default stream) and return without synchronising.  All calls on
+ *     one context must be issued on one stream or be externally ordered; a context is not
+ *     thread-safe; distinct contexts are independent.
+ *   - Every call returns an edgefm_status; nothing throws or aborts.  Arguments are validated on the
+ *     host before anything is launched; a call that returns an error has launched nothing and
+ *     changed no state (except edgefm_last_error's message).
+ *   - There is no CPU fallback: without a CUDA device every call that needs one returns
+ *     EDGEFM_ERR_CUDA.
+ */
+#ifndef EDGEFM_H_
+#define EDGEFM_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct edgefm_ctx edgefm_ctx; /* opaque: one request slot */
+
+typedef enum {
+    EDGEFM_OK = 0,
+    EDGEFM_ERR_INVALID_ARG = 1,   /* null pointer, token out of range, negative size ...            */
+    EDGEFM_ERR_BAD_SHAPE = 2,     /* model shape the kernels do not support (see edgefm_create)      */
+    EDGEFM_ERR_CONTEXT_FULL = 3,  /* the KV cache has no free slot / prefill longer than max_context */
+    EDGEFM_ERR_OUT_OF_MEMORY = 4, /* device or host allocation failed                                */
+    EDGEFM_ERR_CUDA = 5,          /* a CUDA runtime call failed; see edgefm_last_error               */
+    EDGEFM_ERR_TIMEOUT = 6        /* reserved: a bounded device-side wait expired                     */
+} edgefm_status;
+
+/* Model shape (the public Qwen2.5 decoder block). */
+typedef struct {
+    int32_t n_layers;
+    int32_t hidden;      /* H, multiple of 8                                        */
+    int32_t n_q_heads;   /* multiple of n_kv_heads, group size n_q/n_kv in 1..8     */
+    int32_t n_kv_heads;
+    int32_t head_dim;    /* d: 64 or 128                                            */
+    int32_t ffn;         /* F, multiple of 8                                        */
+    int32_t vocab;       /* V                                                       */
+    float rms_eps;       /* RMSNorm epsilon (inside the square root)                */
+    float rope_theta;    /* RoPE base; rotate-half pairs (i, i+d/2)                 */
+    int32_t qkv_bias;    /* 1: bqkv is used; 0: it is ignored                       */
+} edgefm_shape;
+
+/* Per-layer DEVICE pointers, bf16, row-major [out][in]. */
+typedef struct {
+    const void *input_norm; /* [H]                                                        */
+    const void *wqkv;       /* [(n_q + 2 n_kv) d][H]; rows: q heads, then k heads, then v */
+    const void *bqkv;       /* [(n_q + 2 n_kv) d], or NULL when qkv_bias == 0              */
+    const void *wo;         /* [H][n_q d]                                                 */
+    const void *post_norm;  /* [H]                                                        */
+    const void *w_gate_up;  /* [2F][H]; rows 0..F-1 gate, F..2F-1 up                      */
+    const void *w_down;     /* [H][F]                                                     */
+} edgefm_layer_weights;
+
+typedef struct {
+    const void *embed;                  /* device bf16 [V][H]                                  */
+    const void *final_norm;             /* device bf16 [H]                                     */
+    const void *lm_head;                /* device bf16 [V][H]; may equal embed (tied)          */
+    const edgefm_layer_weights *layers; /* HOST array [n_layers] of structs of device pointers */
+} edgefm_weights;
+
+/*
+ * edgefm_create -- build a context for one request slot (Sec. 3.7 step 1, Sec. 3.9 pre-allocation).
+ * Allocates the KV cache K,V : bf16 [n_layers][n_kv_heads][max_context][head_dim] (cache length 0),
+ * the work buffers and the device state, and records the step as a CUDA graph.
+ * All matrix base pointers must be 16-byte aligned.  `shape` and `weights` (and the `layers` array)
+ * are read during the call only; the device buffers they point to are borrowed until destroy.
+ * Errors: INVALID_ARG (null pointers, max_context < 1), BAD_SHAPE, OUT_OF_MEMORY, CUDA.
+ * On error *out is set to NULL.
+ */
+edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *weights, int32_t max_context,
+                            edgefm_ctx **out);
+
+/*
+ * edgefm_prefill_kv -- load an already computed KV cache (Eq. 3: KV <- Prefill(x_1:T); here the
+ * result of the prefill is given, vision-token positions included; Sec. 3.9 Eq. 5 prefix reuse).
+ * k, v: DEVICE bf16; element (layer l, kv head g, position t, j) is read at
+ *       l*stride_layer + g*stride_head + t*stride_pos + j  (strides in elements; the last
+ *       dimension is contiguous).  Keys must already carry their rotary embedding.
+ * Copies positions 0 .. n_positions-1 into cache slots 0 .. n_positions-1 and sets the cache
+ * length to n_positions (n_positions = 0 empties the cache; k, v may then be NULL).
+ * The copy is asynchronous on `stream`; k and v must stay valid until it has run.
+ * Errors: INVALID_ARG, CONTEXT_FULL (n_positions > max_context; nothing is written), CUDA.
+ */
+edgefm_status edgefm_prefill_kv(edgefm_ctx *ctx, const void *k, const void *v, int32_t n_positions,
+                                int64_t stride_layer, int64_t stride_head, int64_t stride_pos, void *stream);
+
+/*
+ * edgefm_decode_step -- one decode step (Eq. 4): consume one token, append its K/V at cache slot
+ * cur_len, attend over slots 0 .. cur_len, produce the logits and the greedy next token.
+ *   token_id  >= 0 : the input token.  -1 : the token the previous step on this context produced
+ *                    (kept on the device, no host round trip).
+ *   position  >= 0 : rotary position of the input token (it may differ from the cache slot, e.g.
+ *                    after vision tokens).  -1 : previous step's position + 1 (cache length for the
+ *                    first step after prefill).
+ *   logits_out      : DEVICE fp32 [vocab] or NULL.
+ *   next_token_out  : DEVICE int32 [1] or NULL (lowest index among the maxima of the logits).
+ * Outputs are valid once `stream` has executed the step.  The cache length grows by one.
+ * Errors: INVALID_ARG (token_id >= vocab or < -1, position < -1, token_id == -1 before any step),
+ * CONTEXT_FULL (cache length == max_context; nothing is launched), CUDA.
+ */
+edgefm_status edgefm_decode_step(edgefm_ctx *ctx, int32_t token_id, int32_t position, void *stream,
+                                 float *logits_out, int32_t *next_token_out);
+
+/* edgefm_destroy -- synchronise the device, then free everything the context owns (Sec. 3.7 step 4). NULL is a no-op. */
+edgefm_status edgefm_destroy(edgefm_ctx *ctx);
+
+/* ---- small helpers (tests, benchmarks) ---------------------------------------------------------- */
+
+/* Host-side cache length (number of filled slots) after all calls enqueued so far; no sync. */
+edgefm_status edgefm_get_length(const edgefm_ctx *ctx, int32_t *cur_len_host);
+
+/* Copy the whole cache, internal layout bf16 [n_layers][n_kv_heads][max_context][head_dim], to the
+ * DEVICE buffers k_out / v_out (asynchronous on `stream`). */
+edgefm_status edgefm_export_kv(edgefm_ctx *ctx, void *k_out, void *v_out, void *stream);
+
+/* Number of kernel launches one decode step performs (nodes of the step graph). */
+edgefm_status edgefm_get_launches_per_step(const edgefm_ctx *ctx, int32_t *n_launches_host);
+
+/* Message of the last error on this context ("" if none); ctx == NULL: last error of edgefm_create
+ * on the calling thread. The string is owned by the library. */
+const char *edgefm_last_error(const edgefm_ctx *ctx);
+
+/* Library version string. */
+const char *edgefm_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EDGEFM_H_ */

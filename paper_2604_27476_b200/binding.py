@@ -1,0 +1,230 @@
+"""ctypes binding of include/edgefm.h: same names, argument marshalling only.
+
+There is no fallback: if libedgefm.so is missing or cannot be loaded, load_library raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import enum
+from pathlib import Path
+
+_PKG = Path(__file__).resolve().parent
+_LIB_PATH = _PKG / "libedgefm.so"
+_lib = None
+
+
+class Status(enum.IntEnum):
+    OK = 0
+    ERR_INVALID_ARG = 1
+    ERR_BAD_SHAPE = 2
+    ERR_CONTEXT_FULL = 3
+    ERR_OUT_OF_MEMORY = 4
+    ERR_CUDA = 5
+    ERR_TIMEOUT = 6
+
+
+class EdgefmError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"{Status(status).name}: {message}")
+        self.status = Status(status)
+
+
+class _Shape(ctypes.Structure):
+    _fields_ = [("n_layers", ctypes.c_int32), ("hidden", ctypes.c_int32), ("n_q_heads", ctypes.c_int32),
+                ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("ffn", ctypes.c_int32),
+                ("vocab", ctypes.c_int32), ("rms_eps", ctypes.c_float), ("rope_theta", ctypes.c_float),
+                ("qkv_bias", ctypes.c_int32)]
+
+
+class _LayerWeights(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in ("input_norm", "wqkv", "bqkv", "wo", "post_norm", "w_gate_up", "w_down")]
+
+
+class _Weights(ctypes.Structure):
+    _fields_ = [("embed", ctypes.c_void_p), ("final_norm", ctypes.c_void_p), ("lm_head", ctypes.c_void_p),
+                ("layers", ctypes.POINTER(_LayerWeights))]
+
+
+EXPORTS = ("edgefm_create", "edgefm_prefill_kv", "edgefm_decode_step", "edgefm_destroy", "edgefm_get_length",
+           "edgefm_export_kv", "edgefm_get_launches_per_step", "edgefm_last_error", "edgefm_version")
+
+
+def library_path() -> Path:
+    return _LIB_PATH
+
+
+def load_library():
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not _LIB_PATH.exists():
+        raise FileNotFoundError(f"{_LIB_PATH} is missing: build it with `python -m paper_2604_27476_b200.build` "
+                                "(there is no CPU fallback)")
+    L = ctypes.CDLL(str(_LIB_PATH))
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    L.edgefm_create.restype = ctypes.c_int
+    L.edgefm_create.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Weights), i32, ctypes.POINTER(vp)]
+    L.edgefm_prefill_kv.restype = ctypes.c_int
+    L.edgefm_prefill_kv.argtypes = [vp, vp, vp, i32, i64, i64, i64, vp]
+    L.edgefm_decode_step.restype = ctypes.c_int
+    L.edgefm_decode_step.argtypes = [vp, i32, i32, vp, vp, vp]
+    L.edgefm_destroy.restype = ctypes.c_int
+    L.edgefm_destroy.argtypes = [vp]
+    L.edgefm_get_length.restype = ctypes.c_int
+    L.edgefm_get_length.argtypes = [vp, ctypes.POINTER(i32)]
+    L.edgefm_export_kv.restype = ctypes.c_int
+    L.edgefm_export_kv.argtypes = [vp, vp, vp, vp]
+    L.edgefm_get_launches_per_step.restype = ctypes.c_int
+    L.edgefm_get_launches_per_step.argtypes = [vp, ctypes.POINTER(i32)]
+    L.edgefm_last_error.restype = ctypes.c_char_p
+    L.edgefm_last_error.argtypes = [vp]
+    L.edgefm_version.restype = ctypes.c_char_p
+    L.edgefm_version.argtypes = []
+    _lib = L
+    return L
+
+
+def _check(status: int, ctx=None):
+    if status != 0:
+        raise EdgefmError(status, edgefm_last_error(ctx))
+
+
+# ---- the C calls, one Python function each -------------------------------------------------------
+def edgefm_version() -> str:
+    return load_library().edgefm_version().decode()
+
+
+def edgefm_last_error(ctx=None) -> str:
+    return load_library().edgefm_last_error(ctx).decode()
+
+
+def edgefm_create(shape: dict, weights: dict, max_context: int):
+    """shape: dict with the fields of edgefm_shape; weights: {"embed", "final_norm", "lm_head": device
+    pointers (int), "layers": [ {field: device pointer or None} ]}.  Returns the opaque context handle."""
+    L = load_library()
+    sh = _Shape(**shape)
+    layers = weights["layers"]
+    arr = (_LayerWeights * max(1, len(layers)))()
+    for i, lw in enumerate(layers):
+        for name, _ in _LayerWeights._fields_:
+            setattr(arr[i], name, lw.get(name))
+    w = _Weights(weights["embed"], weights["final_norm"], weights["lm_head"], arr)
+    out = ctypes.c_void_p()
+    _check(L.edgefm_create(ctypes.byref(sh), ctypes.byref(w), max_context, ctypes.byref(out)))
+    return out
+
+
+def edgefm_prefill_kv(ctx, k_ptr, v_ptr, n_positions, stride_layer, stride_head, stride_pos, stream=None):
+    _check(load_library().edgefm_prefill_kv(ctx, k_ptr, v_ptr, n_positions, stride_layer, stride_head, stride_pos, stream), ctx)
+
+
+def edgefm_decode_step(ctx, token_id, position, stream=None, logits_out=None, next_token_out=None):
+    _check(load_library().edgefm_decode_step(ctx, token_id, position, stream, logits_out, next_token_out), ctx)
+
+
+def edgefm_destroy(ctx):
+    _check(load_library().edgefm_destroy(ctx))
+
+
+def edgefm_get_length(ctx) -> int:
+    n = ctypes.c_int32()
+    _check(load_library().edgefm_get_length(ctx, ctypes.byref(n)), ctx)
+    return n.value
+
+
+def edgefm_get_launches_per_step(ctx) -> int:
+    n = ctypes.c_int32()
+    _check(load_library().edgefm_get_launches_per_step(ctx, ctypes.byref(n)), ctx)
+    return n.value
+
+
+def edgefm_export_kv(ctx, k_out_ptr, v_out_ptr, stream=None):
+    _check(load_library().edgefm_export_kv(ctx, k_out_ptr, v_out_ptr, stream), ctx)
+
+
+# ---- convenience for tests and the benchmark: torch owns the device memory ------------------------
+def upload_weights(host_weights: dict, device="cuda:0"):
+    """Copy a dict of numpy uint16 (bf16 bits) arrays (layout of edgefm_weights) to the device.
+    Returns (pointer dict for edgefm_create, list of torch tensors that must be kept alive)."""
+    import numpy as np
+    import torch
+
+    keep = []
+
+    def up(a):
+        if a is None:
+            return None
+        t = torch.from_numpy(a.view(np.int16)).to(device)
+        keep.append(t)
+        return t.data_ptr()
+
+    embed = up(host_weights["embed"])
+    lm = embed if host_weights["lm_head"] is host_weights["embed"] else up(host_weights["lm_head"])
+    ptrs = {"embed": embed, "final_norm": up(host_weights["final_norm"]), "lm_head": lm,
+            "layers": [{k: up(v) for k, v in lw.items()} for lw in host_weights["layers"]]}
+    return ptrs, keep
+
+
+class DecodeContext:
+    """RAII wrapper of one edgefm context with torch-allocated I/O buffers."""
+
+    def __init__(self, cfg, device_weight_ptrs: dict, max_context: int, device="cuda:0"):
+        import torch
+
+        self.cfg = cfg
+        self.device = torch.device(device)
+        self.max_context = max_context
+        shape = dict(n_layers=cfg.n_layers, hidden=cfg.hidden, n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads,
+                     head_dim=cfg.head_dim, ffn=cfg.ffn, vocab=cfg.vocab, rms_eps=cfg.rms_eps,
+                     rope_theta=cfg.rope_theta, qkv_bias=int(cfg.qkv_bias))
+        with torch.cuda.device(self.device):
+            self.handle = edgefm_create(shape, device_weight_ptrs, max_context)
+        self.logits = torch.empty(cfg.vocab, dtype=torch.float32, device=self.device)
+        self.next_token = torch.zeros(1, dtype=torch.int32, device=self.device)
+
+    def _stream(self):
+        import torch
+        return torch.cuda.current_stream(self.device).cuda_stream
+
+    def prefill_kv(self, k, v):
+        """k, v: torch int16/bf16 tensors [L][n_kv][n][d] on the device (any strides with contiguous last dim)."""
+        n = k.shape[2]
+        assert k.stride() == v.stride() and k.stride(3) == 1
+        edgefm_prefill_kv(self.handle, k.data_ptr(), v.data_ptr(), n, k.stride(0), k.stride(1), k.stride(2), self._stream())
+
+    def reset(self):
+        """Empty the cache (cache length 0)."""
+        edgefm_prefill_kv(self.handle, None, None, 0, 0, 0, 0, self._stream())
+
+    def step(self, token_id=-1, position=-1, want_logits=True, want_token=True):
+        edgefm_decode_step(self.handle, token_id, position, self._stream(),
+                           self.logits.data_ptr() if want_logits else None,
+                           self.next_token.data_ptr() if want_token else None)
+
+    def export_kv(self):
+        import torch
+        c = self.cfg
+        shape = (c.n_layers, c.n_kv_heads, self.max_context, c.head_dim)
+        k = torch.empty(shape, dtype=torch.int16, device=self.device)
+        v = torch.empty(shape, dtype=torch.int16, device=self.device)
+        edgefm_export_kv(self.handle, k.data_ptr(), v.data_ptr(), self._stream())
+        return k, v
+
+    @property
+    def cur_len(self) -> int:
+        return edgefm_get_length(self.handle)
+
+    @property
+    def launches_per_step(self) -> int:
+        return edgefm_get_launches_per_step(self.handle)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            edgefm_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,83 @@
+// Shared device helpers of the decode-step kernels (sm_100a).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace edgefm {
+
+// Device-resident dynamic parameters of the step graph (Sec. 3.10 of the paper: dynamic
+// parameters live in GPU buffers so that one fixed graph serves every decode iteration).
+struct StepState {
+    int token;          // input token of the step in flight (resolved by step_begin_kernel)
+    int position;       // its rotary position
+    int cur_len;        // filled cache slots before the step == slot the step writes
+    int next_token;     // greedy result of the last finished step
+    int next_position;  // position the next step uses when the caller passes -1
+    int status;         // 0 = ok (reserved for bounded-wait failures)
+    int pad[2];
+};
+
+// What the host asks of the next step; uploaded only when it differs from the previous request.
+struct StepRequest {
+    int token;          // >= 0 explicit, -1 = StepState::next_token
+    int position;       // >= 0 explicit, -1 = StepState::next_position
+    float *logits_out;  // device fp32[V] or null
+    int *next_token_out;  // device int32[1] or null
+};
+
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// 128-bit streaming load of read-only data that is used once: bypass L1, prefetch the L2 sector pair.
+__device__ __forceinline__ uint4 ldg_stream16(const void *p) {
+    uint4 v;
+    asm("ld.global.nc.L1::no_allocate.L2::256B.v4.u32 {%0,%1,%2,%3}, [%4];"
+        : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+        : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint2 ldg_stream8(const void *p) {
+    uint2 v;
+    asm("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint32_t ldg_stream4(const void *p) {
+    uint32_t v;
+    asm("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+__device__ __forceinline__ float bf16_bits_to_f32(uint16_t b) { return __uint_as_float(static_cast<uint32_t>(b) << 16); }
+__device__ __forceinline__ uint16_t f32_to_bf16_bits(float f) { return __bfloat16_as_ushort(__float2bfloat16_rn(f)); }
+
+// acc += <8 bf16 weights, 8 fp32 activations>
+__device__ __forceinline__ float dot8(uint4 w, float4 x0, float4 x1, float acc) {
+    acc = fmaf(bf16lo(w.x), x0.x, acc);
+    acc = fmaf(bf16hi(w.x), x0.y, acc);
+    acc = fmaf(bf16lo(w.y), x0.z, acc);
+    acc = fmaf(bf16hi(w.y), x0.w, acc);
+    acc = fmaf(bf16lo(w.z), x1.x, acc);
+    acc = fmaf(bf16hi(w.z), x1.y, acc);
+    acc = fmaf(bf16lo(w.w), x1.z, acc);
+    acc = fmaf(bf16hi(w.w), x1.w, acc);
+    return acc;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+// (value, index) ordering of the greedy sampler: larger value wins, equal values -> lower index.
+__device__ __forceinline__ bool arg_better(float v, int i, float bv, int bi) { return v > bv || (v == bv && i < bi); }
+
+}  // namespace edgefm

@@ -1,0 +1,549 @@
+// C ABI of the batch-1 decode step (see include/edgefm.h) and the assembly of the step as a CUDA graph.
+#include "../../include/edgefm.h"
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "attention.cuh"
+#include "common.cuh"
+#include "gemv.cuh"
+
+namespace edgefm {
+
+// ---- small kernels -------------------------------------------------------------------------------
+
+// First node of the step graph: resolve the request into (token, position), gather the embedding
+// row into the fp32 residual stream and build the cos/sin table of the rotary position.  The
+// angle is evaluated in fp64 (position up to ~33k times the fastest frequency needs more than
+// fp32's 24 bits to stay accurate), rounded to fp32 once.
+__global__ void __launch_bounds__(256) step_begin_kernel(const StepRequest *req, StepState *st, const uint16_t *embed,
+                                                         const double *inv_freq, float *x, float *rope_cs, int H,
+                                                         int half_d) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int rt = req->token, rp = req->position;
+    const int token = rt >= 0 ? rt : st->next_token;
+    const int pos = rp >= 0 ? rp : st->next_position;
+    __syncthreads();  // every thread has read the previous state before it is overwritten
+    if (threadIdx.x == 0) { st->token = token; st->position = pos; }
+    const uint16_t *row = embed + static_cast<size_t>(token) * H;
+    for (int i = threadIdx.x; i < H; i += blockDim.x) x[i] = bf16_bits_to_f32(row[i]);
+    for (int i = threadIdx.x; i < half_d; i += blockDim.x) {
+        double s, c;
+        sincos(static_cast<double>(pos) * inv_freq[i], &s, &c);
+        rope_cs[i] = static_cast<float>(c);
+        rope_cs[half_d + i] = static_cast<float>(s);
+    }
+}
+
+// Strided copy of a caller-provided KV prefix into the cache; also sets the device state.
+__global__ void __launch_bounds__(256) prefill_copy_kernel(const uint16_t *k, const uint16_t *v, uint16_t *kc, uint16_t *vc,
+                                                           int L, int nkv, int n, int d, int max_context, long long s_layer,
+                                                           long long s_head, long long s_pos, int vec_ok, StepState *st) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        st->cur_len = n;
+        st->next_position = n;
+        st->status = 0;
+    }
+    const long long total = static_cast<long long>(L) * nkv * n * d;
+    const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
+    if (vec_ok) {  // 16-byte pieces: d % 8 == 0, all strides % 8 == 0, bases 16-byte aligned
+        const int dp = d >> 3;
+        for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total >> 3; i += stride) {
+            const int j = static_cast<int>(i % dp);
+            long long r = i / dp;
+            const int t = static_cast<int>(r % n); r /= n;
+            const int g = static_cast<int>(r % nkv);
+            const int l = static_cast<int>(r / nkv);
+            const long long src = l * s_layer + g * s_head + t * s_pos + j * 8;
+            const long long dst = ((static_cast<long long>(l) * nkv + g) * max_context + t) * d + j * 8;
+            *reinterpret_cast<uint4 *>(kc + dst) = *reinterpret_cast<const uint4 *>(k + src);
+            *reinterpret_cast<uint4 *>(vc + dst) = *reinterpret_cast<const uint4 *>(v + src);
+        }
+    } else {
+        for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total; i += stride) {
+            const int j = static_cast<int>(i % d);
+            long long r = i / d;
+            const int t = static_cast<int>(r % n); r /= n;
+            const int g = static_cast<int>(r % nkv);
+            const int l = static_cast<int>(r / nkv);
+            const long long src = l * s_layer + g * s_head + t * s_pos + j;
+            const long long dst = ((static_cast<long long>(l) * nkv + g) * max_context + t) * d + j;
+            kc[dst] = k[src];
+            vc[dst] = v[src];
+        }
+    }
+}
+
+// ---- launch helpers ------------------------------------------------------------------------------
+
+template <typename Kern, typename... Args>
+cudaError_t launch(Kern kern, dim3 grid, dim3 block, size_t smem, cudaStream_t s, bool pdl, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+
+using GemvKernel = void (*)(const GemvArgs);
+using AttnKernel = void (*)(const AttnArgs);
+
+struct GemvPlan {
+    GemvKernel kern = nullptr;
+    int threads = 0, tile_rows = 0, wk = 0;
+    int grid = 0;
+    size_t smem = 0;
+};
+
+struct AttnPlan {
+    AttnKernel kern = nullptr;
+    int threads = 0;
+    size_t smem = 0;
+    int max_chunks = 0, min_chunk = 0;
+};
+
+template <int PRO, int EPI, int RW, int WR, int WK, int U>
+GemvPlan make_gemv_plan(int units, int K, int num_sms, cudaError_t *err) {
+    GemvPlan p;
+    p.kern = gemv_kernel<PRO, EPI, RW, WR, WK, U>;
+    p.threads = WR * WK * 32;
+    p.tile_rows = RW * WR;
+    p.wk = WK;
+    p.smem = (static_cast<size_t>(K) + (WK + 1) * RW * WR) * sizeof(float);
+    *err = cudaFuncSetAttribute(p.kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(p.smem));
+    if (*err != cudaSuccess) return p;
+    int per_sm = 0;
+    *err = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, p.kern, p.threads, p.smem);
+    if (*err != cudaSuccess) return p;
+    if (per_sm < 1) per_sm = 1;
+    const int paired = (EPI == EPI_QKV || EPI == EPI_SWIGLU) ? 2 : 1;
+    const int per_tile = p.tile_rows / paired;
+    const int ntiles = (units + per_tile - 1) / per_tile;
+    const int cap = num_sms * per_sm;
+    p.grid = ntiles < cap ? ntiles : cap;
+    if (p.grid < 1) p.grid = 1;
+    return p;
+}
+
+template <int D, int G, int LPP, int NW>
+AttnPlan make_attn_plan_t(cudaError_t *err) {
+    AttnPlan p;
+    p.kern = attn_kernel<D, G, LPP, NW>;
+    p.threads = NW * 32;
+    p.smem = AttnSmem<D, G, LPP, NW>::TOTAL;
+    *err = cudaFuncSetAttribute(p.kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(p.smem));
+    return p;
+}
+
+template <int D, int LPP, int NW>
+AttnPlan make_attn_plan_g(int G, cudaError_t *err) {
+    switch (G) {
+        case 1: return make_attn_plan_t<D, 1, LPP, NW>(err);
+        case 2: return make_attn_plan_t<D, 2, LPP, NW>(err);
+        case 3: return make_attn_plan_t<D, 3, LPP, NW>(err);
+        case 4: return make_attn_plan_t<D, 4, LPP, NW>(err);
+        case 5: return make_attn_plan_t<D, 5, LPP, NW>(err);
+        case 6: return make_attn_plan_t<D, 6, LPP, NW>(err);
+        case 7: return make_attn_plan_t<D, 7, LPP, NW>(err);
+        case 8: return make_attn_plan_t<D, 8, LPP, NW>(err);
+    }
+    *err = cudaErrorInvalidValue;
+    return AttnPlan();
+}
+
+}  // namespace edgefm
+
+using namespace edgefm;
+
+// ---- the context -----------------------------------------------------------------------------------
+
+struct edgefm_ctx {
+    edgefm_shape shape{};
+    int max_context = 0;
+    int device = -1;
+    int num_sms = 0;
+    bool use_pdl = true;
+    std::vector<edgefm_layer_weights> layers;
+    const void *embed = nullptr, *final_norm = nullptr, *lm_head = nullptr;
+
+    // owned device memory
+    uint16_t *k_cache = nullptr, *v_cache = nullptr;  // [L][nkv][max_context][d]
+    float *x = nullptr;          // residual stream [H]
+    float *q = nullptr;          // rotated queries [nq*d]
+    float *attn = nullptr;       // attention output [nq*d]
+    float *act = nullptr;        // SwiGLU output [F]
+    float *rope_cs = nullptr;    // [d]
+    double *inv_freq = nullptr;  // [d/2]
+    float *part_m = nullptr, *part_l = nullptr, *part_o = nullptr;
+    float *lm_part_val = nullptr;
+    int *lm_part_idx = nullptr;
+    unsigned *tickets = nullptr;  // [nkv] attention + [1] lm_head
+    StepState *state = nullptr;
+    StepRequest *req = nullptr;
+
+    GemvPlan p_qkv, p_o, p_gu, p_down, p_lm;
+    AttnPlan p_attn;
+
+    cudaStream_t build_stream = nullptr;
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t exec = nullptr;
+    int launches_per_step = 0;
+
+    // host mirrors
+    int cur_len = 0;
+    bool have_token = false;
+    bool req_valid = false;
+    StepRequest last_req{};
+    std::string err;
+};
+
+namespace {
+
+thread_local std::string g_create_error;
+
+edgefm_status fail(edgefm_ctx *ctx, edgefm_status st, const char *fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    if (ctx) ctx->err = buf; else g_create_error = buf;
+    return st;
+}
+
+#define CUDA_TRY(ctx, call)                                                                                   \
+    do {                                                                                                      \
+        cudaError_t e_ = (call);                                                                              \
+        if (e_ != cudaSuccess)                                                                                \
+            return fail(ctx, e_ == cudaErrorMemoryAllocation ? EDGEFM_ERR_OUT_OF_MEMORY : EDGEFM_ERR_CUDA,    \
+                        "%s failed: %s", #call, cudaGetErrorString(e_));                                      \
+    } while (0)
+
+struct DeviceGuard {
+    int prev = -1;
+    bool active = false;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) { cudaSetDevice(dev); active = true; }
+    }
+    ~DeviceGuard() { if (active) cudaSetDevice(prev); }
+};
+
+template <typename T>
+cudaError_t dev_alloc(T **p, size_t count) {
+    return cudaMalloc(reinterpret_cast<void **>(p), count * sizeof(T) + 256);  // + guard bytes behind every buffer
+}
+
+void free_all(edgefm_ctx *c) {
+    if (c->exec) cudaGraphExecDestroy(c->exec);
+    if (c->graph) cudaGraphDestroy(c->graph);
+    if (c->build_stream) cudaStreamDestroy(c->build_stream);
+    void *bufs[] = {c->k_cache, c->v_cache, c->x, c->q, c->attn, c->act, c->rope_cs, c->inv_freq, c->part_m, c->part_l,
+                    c->part_o, c->lm_part_val, c->lm_part_idx, c->tickets, c->state, c->req};
+    for (void *b : bufs) if (b) cudaFree(b);
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Enqueue the kernels of one decode step (used once, under stream capture).
+cudaError_t enqueue_step(edgefm_ctx *c, cudaStream_t s, int *n_launches) {
+    const edgefm_shape &sh = c->shape;
+    const int H = sh.hidden, d = sh.head_dim, nq = sh.n_q_heads, nkv = sh.n_kv_heads, F = sh.ffn;
+    const int R = (nq + 2 * nkv) * d;
+    const bool pdl = c->use_pdl;
+    int n = 0;
+    cudaError_t e;
+    // The first node follows the previous graph launch by ordinary stream order.
+    e = launch(step_begin_kernel, dim3(1), dim3(256), 0, s, false, (const StepRequest *)c->req, c->state,
+               (const uint16_t *)c->embed, (const double *)c->inv_freq, c->x, c->rope_cs, H, d / 2);
+    if (e != cudaSuccess) return e;
+    ++n;
+    const size_t kv_layer = static_cast<size_t>(nkv) * c->max_context * d;
+    for (int l = 0; l < sh.n_layers; ++l) {
+        const edgefm_layer_weights &w = c->layers[l];
+        GemvArgs a{};
+        a.W = (const uint16_t *)w.wqkv; a.rows = R; a.K = H; a.x_in = c->x; a.norm_w = (const uint16_t *)w.input_norm;
+        a.eps = sh.rms_eps; a.bias = sh.qkv_bias ? (const uint16_t *)w.bqkv : nullptr; a.out = c->q;
+        a.k_cache = c->k_cache + l * kv_layer; a.v_cache = c->v_cache + l * kv_layer; a.max_context = c->max_context;
+        a.nq = nq; a.nkv = nkv; a.d = d; a.rope_cs = c->rope_cs; a.state = c->state;
+        e = launch(c->p_qkv.kern, dim3(c->p_qkv.grid), dim3(c->p_qkv.threads), c->p_qkv.smem, s, pdl, a);
+        if (e != cudaSuccess) return e;
+        ++n;
+
+        AttnArgs t{};
+        t.q = c->q; t.k_cache = a.k_cache; t.v_cache = a.v_cache; t.out = c->attn; t.part_m = c->part_m;
+        t.part_l = c->part_l; t.part_o = c->part_o; t.tickets = c->tickets; t.state = c->state;
+        t.max_context = c->max_context; t.max_chunks = c->p_attn.max_chunks; t.min_chunk = c->p_attn.min_chunk;
+        t.scale = static_cast<float>(1.0 / std::sqrt(static_cast<double>(d)));
+        e = launch(c->p_attn.kern, dim3(c->p_attn.max_chunks, nkv), dim3(c->p_attn.threads), c->p_attn.smem, s, pdl, t);
+        if (e != cudaSuccess) return e;
+        ++n;
+
+        GemvArgs o{};
+        o.W = (const uint16_t *)w.wo; o.rows = H; o.K = nq * d; o.x_in = c->attn; o.out = c->x;
+        e = launch(c->p_o.kern, dim3(c->p_o.grid), dim3(c->p_o.threads), c->p_o.smem, s, pdl, o);
+        if (e != cudaSuccess) return e;
+        ++n;
+
+        GemvArgs gu{};
+        gu.W = (const uint16_t *)w.w_gate_up; gu.rows = 2 * F; gu.K = H; gu.x_in = c->x;
+        gu.norm_w = (const uint16_t *)w.post_norm; gu.eps = sh.rms_eps; gu.out = c->act; gu.F = F;
+        e = launch(c->p_gu.kern, dim3(c->p_gu.grid), dim3(c->p_gu.threads), c->p_gu.smem, s, pdl, gu);
+        if (e != cudaSuccess) return e;
+        ++n;
+
+        GemvArgs dn{};
+        dn.W = (const uint16_t *)w.w_down; dn.rows = H; dn.K = F; dn.x_in = c->act; dn.out = c->x;
+        e = launch(c->p_down.kern, dim3(c->p_down.grid), dim3(c->p_down.threads), c->p_down.smem, s, pdl, dn);
+        if (e != cudaSuccess) return e;
+        ++n;
+    }
+    GemvArgs lm{};
+    lm.W = (const uint16_t *)c->lm_head; lm.rows = sh.vocab; lm.K = H; lm.x_in = c->x;
+    lm.norm_w = (const uint16_t *)c->final_norm; lm.eps = sh.rms_eps; lm.state = c->state; lm.req = c->req;
+    lm.part_val = c->lm_part_val; lm.part_idx = c->lm_part_idx; lm.ticket = c->tickets + nkv;
+    e = launch(c->p_lm.kern, dim3(c->p_lm.grid), dim3(c->p_lm.threads), c->p_lm.smem, s, pdl, lm);
+    if (e != cudaSuccess) return e;
+    ++n;
+    *n_launches = n;
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *edgefm_version(void) { return "edgefm-b200 0.1 (sm_100a)"; }
+
+const char *edgefm_last_error(const edgefm_ctx *ctx) { return ctx ? ctx->err.c_str() : g_create_error.c_str(); }
+
+edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *weights, int32_t max_context,
+                            edgefm_ctx **out) {
+    if (out) *out = nullptr;
+    if (!shape || !weights || !out) return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "null argument");
+    if (max_context < 1) return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "max_context must be >= 1");
+    const edgefm_shape &sh = *shape;
+    if (sh.n_layers < 1 || sh.hidden < 8 || sh.n_q_heads < 1 || sh.n_kv_heads < 1 || sh.ffn < 8 || sh.vocab < 1)
+        return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "non-positive dimension");
+    if (sh.hidden % 8 || sh.ffn % 8) return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "hidden and ffn must be multiples of 8");
+    if (sh.head_dim != 64 && sh.head_dim != 128) return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "head_dim must be 64 or 128");
+    if (sh.n_q_heads % sh.n_kv_heads) return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "n_q_heads must be a multiple of n_kv_heads");
+    const int G = sh.n_q_heads / sh.n_kv_heads;
+    if (G > 8) return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "group size n_q/n_kv must be <= 8");
+    if (!(sh.rms_eps >= 0.f) || !(sh.rope_theta > 0.f)) return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "bad rms_eps / rope_theta");
+    if (static_cast<long long>(sh.vocab) * sh.hidden > (1LL << 40)) return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "model too large");
+    if (!weights->embed || !weights->final_norm || !weights->lm_head || !weights->layers)
+        return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "null weight pointer");
+    if (!aligned16(weights->embed) || !aligned16(weights->lm_head) || !aligned16(weights->final_norm))
+        return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "weight pointers must be 16-byte aligned");
+    for (int l = 0; l < sh.n_layers; ++l) {
+        const edgefm_layer_weights &w = weights->layers[l];
+        if (!w.input_norm || !w.wqkv || !w.wo || !w.post_norm || !w.w_gate_up || !w.w_down || (sh.qkv_bias && !w.bqkv))
+            return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "null weight pointer in layer %d", l);
+        if (!aligned16(w.input_norm) || !aligned16(w.wqkv) || !aligned16(w.wo) || !aligned16(w.post_norm) ||
+            !aligned16(w.w_gate_up) || !aligned16(w.w_down))
+            return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "weight pointers must be 16-byte aligned (layer %d)", l);
+    }
+
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(nullptr, EDGEFM_ERR_CUDA, "no CUDA device available (this library has no CPU path)");
+    }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(nullptr, EDGEFM_ERR_CUDA, "cudaGetDeviceProperties failed");
+    }
+    if (prop.major < 10) return fail(nullptr, EDGEFM_ERR_CUDA, "device sm_%d%d is not supported (built for sm_100a)", prop.major, prop.minor);
+
+    edgefm_ctx *c = new (std::nothrow) edgefm_ctx();
+    if (!c) return fail(nullptr, EDGEFM_ERR_OUT_OF_MEMORY, "host allocation failed");
+    c->shape = sh;
+    c->max_context = max_context;
+    c->device = dev;
+    c->num_sms = prop.multiProcessorCount;
+    const char *env = getenv("EDGEFM_PDL");
+    c->use_pdl = !(env && env[0] == '0');
+    c->layers.assign(weights->layers, weights->layers + sh.n_layers);
+    c->embed = weights->embed; c->final_norm = weights->final_norm; c->lm_head = weights->lm_head;
+
+    auto bail = [&](edgefm_status st, const char *what, cudaError_t e) {
+        g_create_error = std::string(what) + ": " + cudaGetErrorString(e);
+        cudaGetLastError();
+        free_all(c);
+        delete c;
+        return st;
+    };
+#define CREATE_TRY(call)                                                                                            \
+    do {                                                                                                            \
+        cudaError_t e_ = (call);                                                                                    \
+        if (e_ != cudaSuccess) return bail(e_ == cudaErrorMemoryAllocation ? EDGEFM_ERR_OUT_OF_MEMORY : EDGEFM_ERR_CUDA, #call, e_); \
+    } while (0)
+
+    const int H = sh.hidden, d = sh.head_dim, nq = sh.n_q_heads, nkv = sh.n_kv_heads, F = sh.ffn;
+    const int R = (nq + 2 * nkv) * d;
+    cudaError_t pe = cudaSuccess;
+
+    // kernel variants per operator (tile rows x split-K chosen for the operator's aspect ratio)
+    c->p_qkv = make_gemv_plan<PRO_RMSNORM, EPI_QKV, 2, 8, 1, 4>(R / 2, H, c->num_sms, &pe);
+    CREATE_TRY(pe);
+    c->p_o = make_gemv_plan<PRO_PLAIN, EPI_RESIDUAL, 1, 8, 1, 6>(H, nq * d, c->num_sms, &pe);
+    CREATE_TRY(pe);
+    c->p_gu = make_gemv_plan<PRO_RMSNORM, EPI_SWIGLU, 2, 8, 1, 4>(F, H, c->num_sms, &pe);
+    CREATE_TRY(pe);
+    c->p_down = make_gemv_plan<PRO_PLAIN, EPI_RESIDUAL, 4, 1, 8, 2>(H, F, c->num_sms, &pe);
+    CREATE_TRY(pe);
+    c->p_lm = make_gemv_plan<PRO_RMSNORM, EPI_LMHEAD, 2, 8, 1, 4>(sh.vocab, H, c->num_sms, &pe);
+    CREATE_TRY(pe);
+    if (d == 64) c->p_attn = make_attn_plan_g<64, 2, 4>(G, &pe); else c->p_attn = make_attn_plan_g<128, 2, 4>(G, &pe);
+    CREATE_TRY(pe);
+    c->p_attn.min_chunk = 64;
+    {
+        int per_head = (2 * c->num_sms + nkv - 1) / nkv;
+        const int need = (max_context + c->p_attn.min_chunk - 1) / c->p_attn.min_chunk;
+        if (per_head > need) per_head = need;
+        if (per_head < 1) per_head = 1;
+        c->p_attn.max_chunks = per_head;
+    }
+
+    const size_t kv_elems = static_cast<size_t>(sh.n_layers) * nkv * max_context * d;
+    CREATE_TRY(dev_alloc(&c->k_cache, kv_elems));
+    CREATE_TRY(dev_alloc(&c->v_cache, kv_elems));
+    CREATE_TRY(dev_alloc(&c->x, H));
+    CREATE_TRY(dev_alloc(&c->q, nq * d));
+    CREATE_TRY(dev_alloc(&c->attn, nq * d));
+    CREATE_TRY(dev_alloc(&c->act, F));
+    CREATE_TRY(dev_alloc(&c->rope_cs, d));
+    CREATE_TRY(dev_alloc(&c->inv_freq, d / 2));
+    CREATE_TRY(dev_alloc(&c->part_m, static_cast<size_t>(nq) * c->p_attn.max_chunks));
+    CREATE_TRY(dev_alloc(&c->part_l, static_cast<size_t>(nq) * c->p_attn.max_chunks));
+    CREATE_TRY(dev_alloc(&c->part_o, static_cast<size_t>(nq) * c->p_attn.max_chunks * d));
+    CREATE_TRY(dev_alloc(&c->lm_part_val, c->p_lm.grid));
+    CREATE_TRY(dev_alloc(&c->lm_part_idx, c->p_lm.grid));
+    CREATE_TRY(dev_alloc(&c->tickets, nkv + 1));
+    CREATE_TRY(dev_alloc(&c->state, 1));
+    CREATE_TRY(dev_alloc(&c->req, 1));
+    CREATE_TRY(cudaMemset(c->k_cache, 0, kv_elems * 2));
+    CREATE_TRY(cudaMemset(c->v_cache, 0, kv_elems * 2));
+    CREATE_TRY(cudaMemset(c->tickets, 0, (nkv + 1) * sizeof(unsigned)));
+    CREATE_TRY(cudaMemset(c->state, 0, sizeof(StepState)));
+    {
+        StepRequest r{-1, -1, nullptr, nullptr};
+        CREATE_TRY(cudaMemcpy(c->req, &r, sizeof r, cudaMemcpyHostToDevice));
+        std::vector<double> inv(d / 2);
+        for (int i = 0; i < d / 2; ++i) inv[i] = std::pow(static_cast<double>(sh.rope_theta), -2.0 * i / d);
+        CREATE_TRY(cudaMemcpy(c->inv_freq, inv.data(), inv.size() * sizeof(double), cudaMemcpyHostToDevice));
+    }
+
+    // record the step once; every decode step replays this graph
+    CREATE_TRY(cudaStreamCreateWithFlags(&c->build_stream, cudaStreamNonBlocking));
+    CREATE_TRY(cudaStreamBeginCapture(c->build_stream, cudaStreamCaptureModeThreadLocal));
+    cudaError_t le = enqueue_step(c, c->build_stream, &c->launches_per_step);
+    cudaError_t ce = cudaStreamEndCapture(c->build_stream, &c->graph);
+    if (le != cudaSuccess) return bail(EDGEFM_ERR_CUDA, "kernel launch during graph capture", le);
+    CREATE_TRY(ce);
+    CREATE_TRY(cudaGraphInstantiate(&c->exec, c->graph, 0));
+    CREATE_TRY(cudaDeviceSynchronize());
+#undef CREATE_TRY
+    g_create_error.clear();
+    *out = c;
+    return EDGEFM_OK;
+}
+
+edgefm_status edgefm_prefill_kv(edgefm_ctx *ctx, const void *k, const void *v, int32_t n_positions, int64_t stride_layer,
+                                int64_t stride_head, int64_t stride_pos, void *stream) {
+    if (!ctx) return EDGEFM_ERR_INVALID_ARG;
+    if (n_positions < 0) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "n_positions < 0");
+    if (n_positions > ctx->max_context)
+        return fail(ctx, EDGEFM_ERR_CONTEXT_FULL, "n_positions %d exceeds max_context %d", n_positions, ctx->max_context);
+    if (n_positions > 0 && (!k || !v)) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "null k or v");
+    if (n_positions > 0 && (stride_layer < 0 || stride_head < 0 || stride_pos < ctx->shape.head_dim))
+        return fail(ctx, EDGEFM_ERR_INVALID_ARG, "bad strides");
+    DeviceGuard guard(ctx->device);
+    const edgefm_shape &sh = ctx->shape;
+    const int vec_ok = n_positions > 0 && aligned16(k) && aligned16(v) && stride_layer % 8 == 0 && stride_head % 8 == 0 &&
+                       stride_pos % 8 == 0;
+    const long long total = static_cast<long long>(sh.n_layers) * sh.n_kv_heads * n_positions * sh.head_dim;
+    long long blocks = (total / (vec_ok ? 8 : 1) + 255) / 256;
+    if (blocks < 1) blocks = 1;
+    if (blocks > ctx->num_sms * 16) blocks = ctx->num_sms * 16;
+    prefill_copy_kernel<<<static_cast<unsigned>(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint16_t *>(k), static_cast<const uint16_t *>(v), ctx->k_cache, ctx->v_cache, sh.n_layers,
+        sh.n_kv_heads, n_positions, sh.head_dim, ctx->max_context, stride_layer, stride_head, stride_pos, vec_ok, ctx->state);
+    CUDA_TRY(ctx, cudaGetLastError());
+    ctx->cur_len = n_positions;
+    ctx->err.clear();
+    return EDGEFM_OK;
+}
+
+edgefm_status edgefm_decode_step(edgefm_ctx *ctx, int32_t token_id, int32_t position, void *stream, float *logits_out,
+                                 int32_t *next_token_out) {
+    if (!ctx) return EDGEFM_ERR_INVALID_ARG;
+    if (token_id < -1 || token_id >= ctx->shape.vocab) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "token_id %d out of range", token_id);
+    if (position < -1) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "position %d out of range", position);
+    if (token_id == -1 && !ctx->have_token)
+        return fail(ctx, EDGEFM_ERR_INVALID_ARG, "token_id -1 needs a previous step on this context");
+    if (ctx->cur_len >= ctx->max_context)
+        return fail(ctx, EDGEFM_ERR_CONTEXT_FULL, "KV cache is full (%d slots)", ctx->max_context);
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    StepRequest r{token_id, position, logits_out, next_token_out};
+    if (!ctx->req_valid || std::memcmp(&r, &ctx->last_req, sizeof r) != 0) {
+        // small pageable copy: the runtime stages the bytes before returning, so `r` may live on the stack
+        CUDA_TRY(ctx, cudaMemcpyAsync(ctx->req, &r, sizeof r, cudaMemcpyHostToDevice, s));
+        ctx->last_req = r;
+        ctx->req_valid = true;
+    }
+    CUDA_TRY(ctx, cudaGraphLaunch(ctx->exec, s));
+    ctx->cur_len += 1;
+    ctx->have_token = true;
+    ctx->err.clear();
+    return EDGEFM_OK;
+}
+
+edgefm_status edgefm_destroy(edgefm_ctx *ctx) {
+    if (!ctx) return EDGEFM_OK;
+    DeviceGuard guard(ctx->device);
+    cudaError_t e = cudaDeviceSynchronize();
+    free_all(ctx);
+    delete ctx;
+    return e == cudaSuccess ? EDGEFM_OK : EDGEFM_ERR_CUDA;
+}
+
+edgefm_status edgefm_get_length(const edgefm_ctx *ctx, int32_t *cur_len_host) {
+    if (!ctx || !cur_len_host) return EDGEFM_ERR_INVALID_ARG;
+    *cur_len_host = ctx->cur_len;
+    return EDGEFM_OK;
+}
+
+edgefm_status edgefm_get_launches_per_step(const edgefm_ctx *ctx, int32_t *n) {
+    if (!ctx || !n) return EDGEFM_ERR_INVALID_ARG;
+    *n = ctx->launches_per_step;
+    return EDGEFM_OK;
+}
+
+edgefm_status edgefm_export_kv(edgefm_ctx *ctx, void *k_out, void *v_out, void *stream) {
+    if (!ctx) return EDGEFM_ERR_INVALID_ARG;
+    if (!k_out || !v_out) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "null output");
+    DeviceGuard guard(ctx->device);
+    const edgefm_shape &sh = ctx->shape;
+    const size_t bytes = static_cast<size_t>(sh.n_layers) * sh.n_kv_heads * ctx->max_context * sh.head_dim * 2;
+    CUDA_TRY(ctx, cudaMemcpyAsync(k_out, ctx->k_cache, bytes, cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(stream)));
+    CUDA_TRY(ctx, cudaMemcpyAsync(v_out, ctx->v_cache, bytes, cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(stream)));
+    return EDGEFM_OK;
+}
+
+}  // extern "C"
