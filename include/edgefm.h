@@ -133,6 +133,18 @@ edgefm_status edgefm_export_kv(edgefm_ctx *ctx, void *k_out, void *v_out, void *
 /* Number of kernel launches one decode step performs (nodes of the step graph). */
 edgefm_status edgefm_get_launches_per_step(const edgefm_ctx *ctx, int32_t *n_launches_host);
 
+/* Synchronise `stream`, then report whether a bounded device-side wait of the persistent step kernel
+ * expired (EDGEFM_ERR_TIMEOUT; the context is then unusable and must be destroyed) or all is well. */
+edgefm_status edgefm_sync_status(edgefm_ctx *ctx, void *stream);
+
+/* Diagnostics.  When the environment variable EDGEFM_PROFILE=1 was set at edgefm_create, every CTA of
+ * the persistent step kernel records device timestamps (ns) at fixed points of the last step: start,
+ * then per layer {QKV: staged, done, released; attention: done, released; O, gate/up, down: staged,
+ * done, released}, then lm_head staged, done.  Synchronises the device and copies the
+ * [n_ctas][stride] table to out_host (capacity in elements).  n_ctas = 0 when profiling is off;
+ * out_host may be NULL to query the sizes. */
+edgefm_status edgefm_debug_profile(edgefm_ctx *ctx, uint64_t *out_host, int64_t capacity, int32_t *n_ctas, int32_t *stride);
+
 /* Message of the last error on this context ("" if none); ctx == NULL: last error of edgefm_create
  * on the calling thread. The string is owned by the library. */
 const char *edgefm_last_error(const edgefm_ctx *ctx);

@@ -46,7 +46,8 @@ class _Weights(ctypes.Structure):
 
 
 EXPORTS = ("edgefm_create", "edgefm_prefill_kv", "edgefm_decode_step", "edgefm_destroy", "edgefm_get_length",
-           "edgefm_export_kv", "edgefm_get_launches_per_step", "edgefm_last_error", "edgefm_version")
+           "edgefm_export_kv", "edgefm_get_launches_per_step", "edgefm_last_error", "edgefm_version",
+           "edgefm_sync_status", "edgefm_debug_profile")
 
 
 def library_path() -> Path:
@@ -76,6 +77,10 @@ def load_library():
     L.edgefm_export_kv.argtypes = [vp, vp, vp, vp]
     L.edgefm_get_launches_per_step.restype = ctypes.c_int
     L.edgefm_get_launches_per_step.argtypes = [vp, ctypes.POINTER(i32)]
+    L.edgefm_sync_status.restype = ctypes.c_int
+    L.edgefm_sync_status.argtypes = [vp, vp]
+    L.edgefm_debug_profile.restype = ctypes.c_int
+    L.edgefm_debug_profile.argtypes = [vp, vp, i64, ctypes.POINTER(i32), ctypes.POINTER(i32)]
     L.edgefm_last_error.restype = ctypes.c_char_p
     L.edgefm_last_error.argtypes = [vp]
     L.edgefm_version.restype = ctypes.c_char_p
@@ -136,6 +141,23 @@ def edgefm_get_launches_per_step(ctx) -> int:
     n = ctypes.c_int32()
     _check(load_library().edgefm_get_launches_per_step(ctx, ctypes.byref(n)), ctx)
     return n.value
+
+
+def edgefm_sync_status(ctx, stream=None):
+    _check(load_library().edgefm_sync_status(ctx, stream), ctx)
+
+
+def edgefm_debug_profile(ctx):
+    """-> numpy uint64 [n_ctas][stride] of device timestamps (ns) of the last step, or None when profiling is off."""
+    import numpy as np
+    L = load_library()
+    n, st = ctypes.c_int32(), ctypes.c_int32()
+    _check(L.edgefm_debug_profile(ctx, None, 0, ctypes.byref(n), ctypes.byref(st)), ctx)
+    if n.value == 0:
+        return None
+    out = np.zeros((n.value, st.value), np.uint64)
+    _check(L.edgefm_debug_profile(ctx, out.ctypes.data, out.size, ctypes.byref(n), ctypes.byref(st)), ctx)
+    return out
 
 
 def edgefm_export_kv(ctx, k_out_ptr, v_out_ptr, stream=None):

@@ -13,6 +13,7 @@
 #include "attention.cuh"
 #include "common.cuh"
 #include "gemv.cuh"
+#include "megakernel.cuh"
 
 namespace edgefm {
 
@@ -164,6 +165,42 @@ AttnPlan make_attn_plan_g(int G, cudaError_t *err) {
     return AttnPlan();
 }
 
+using MegaKernel = void (*)(const MkParams);
+
+template <int D>
+MegaKernel mega_kernel_g(int G) {
+    switch (G) {
+        case 1: return decode_megakernel<D, 1>;
+        case 2: return decode_megakernel<D, 2>;
+        case 3: return decode_megakernel<D, 3>;
+        case 4: return decode_megakernel<D, 4>;
+        case 5: return decode_megakernel<D, 5>;
+        case 6: return decode_megakernel<D, 6>;
+        case 7: return decode_megakernel<D, 7>;
+        case 8: return decode_megakernel<D, 8>;
+    }
+    return nullptr;
+}
+
+// Tile geometry of one weight-streaming operator: as many rows (or row pairs) per tile as fit the
+// slot budget; rows longer than the budget are cut into K slices that divide the row evenly.
+inline void choose_tile(int K, bool paired, int pair_align, int budget_bytes, int *rw, int *ksplit) {
+    const int kc = K / 8;
+    const int mult = paired ? 2 : 1;
+    const long long row_bytes = static_cast<long long>(K) * 2;
+    if (row_bytes * mult <= budget_bytes) {
+        int r = paired ? 4 : 8;
+        while (r > 1 && (row_bytes * mult * r > budget_bytes || (paired && pair_align % r != 0))) r >>= 1;
+        *rw = r;
+        *ksplit = 1;
+        return;
+    }
+    *rw = 1;
+    int s = 2;
+    while (s < kc && (kc % s != 0 || static_cast<long long>(kc / s) * 16 * mult > budget_bytes)) ++s;
+    *ksplit = s;
+}
+
 }  // namespace edgefm
 
 using namespace edgefm;
@@ -196,6 +233,17 @@ struct edgefm_ctx {
 
     GemvPlan p_qkv, p_o, p_gu, p_down, p_lm;
     AttnPlan p_attn;
+
+    // persistent-kernel path
+    bool use_mega = true;
+    MegaKernel mega = nullptr;
+    MkPhase *d_phases = nullptr;
+    unsigned *grid_bar = nullptr;
+    unsigned long long *prof = nullptr;
+    int prof_stride = 0;
+    MkParams mk{};
+    size_t mega_smem = 0;
+    int mega_grid = 0;
 
     cudaStream_t build_stream = nullptr;
     cudaGraph_t graph = nullptr;
@@ -251,7 +299,7 @@ void free_all(edgefm_ctx *c) {
     if (c->graph) cudaGraphDestroy(c->graph);
     if (c->build_stream) cudaStreamDestroy(c->build_stream);
     void *bufs[] = {c->k_cache, c->v_cache, c->x, c->q, c->attn, c->act, c->rope_cs, c->inv_freq, c->part_m, c->part_l,
-                    c->part_o, c->lm_part_val, c->lm_part_idx, c->tickets, c->state, c->req};
+                    c->part_o, c->lm_part_val, c->lm_part_idx, c->tickets, c->state, c->req, c->d_phases, c->grid_bar, c->prof};
     for (void *b : bufs) if (b) cudaFree(b);
 }
 
@@ -265,6 +313,23 @@ cudaError_t enqueue_step(edgefm_ctx *c, cudaStream_t s, int *n_launches) {
     const bool pdl = c->use_pdl;
     int n = 0;
     cudaError_t e;
+    if (c->use_mega) {
+        // one cooperative launch: all CTAs are co-resident, which the grid barriers rely on
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(c->mega_grid);
+        cfg.blockDim = dim3(MK_THREADS);
+        cfg.dynamicSmemBytes = c->mega_smem;
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeCooperative;
+        attr[0].val.cooperative = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, c->mega, c->mk);
+        if (e != cudaSuccess) return e;
+        *n_launches = 1;
+        return cudaSuccess;
+    }
     // The first node follows the previous graph launch by ordinary stream order.
     e = launch(step_begin_kernel, dim3(1), dim3(256), 0, s, false, (const StepRequest *)c->req, c->state,
                (const uint16_t *)c->embed, (const double *)c->inv_freq, c->x, c->rope_cs, H, d / 2);
@@ -419,6 +484,79 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
         c->p_attn.max_chunks = per_head;
     }
 
+    {
+        const char *impl = getenv("EDGEFM_IMPL");
+        c->use_mega = !(impl && std::strcmp(impl, "kernels") == 0);
+    }
+    std::vector<MkPhase> phases;
+    if (c->use_mega) {
+        c->mega = d == 64 ? mega_kernel_g<64>(G) : mega_kernel_g<128>(G);
+        int smem_optin = 0, coop = 0;
+        CREATE_TRY(cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+        CREATE_TRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
+        if (!coop) return bail(EDGEFM_ERR_CUDA, "device lacks cooperative launch", cudaErrorNotSupported);
+        c->mega_grid = c->num_sms;
+        // shared-memory plan: activation / attention scratch, the schedule, then the weight ring split
+        // into one private sub-ring of `depth` slots per consumer warp
+        const int max_chunks = c->mega_grid / nkv > 0 ? c->mega_grid / nkv : 1;
+        c->mk.max_chunks = max_chunks;
+        int max_k = H;
+        if (nq * d > max_k) max_k = nq * d;
+        if (F > max_k) max_k = F;
+        const size_t att_bytes = (static_cast<size_t>(G) * d + MK_NWC * G * MK_ATT_TILE + 2 * MK_ATT_MW * G +
+                                  static_cast<size_t>(MK_ATT_MW) * G * d + 2 * static_cast<size_t>(G) * max_chunks) * 4;
+        size_t xbuf = static_cast<size_t>(max_k) * 4;
+        if (att_bytes > xbuf) xbuf = att_bytes;
+        xbuf = (xbuf + 255) / 256 * 256;
+        const size_t static_smem = 2048;  // mbarriers, rotary table, reduction scratch
+        const size_t n_phases = 4 * static_cast<size_t>(sh.n_layers) + 1;
+        const size_t sched = (n_phases * sizeof(MkPhase) + 127) / 128 * 128;
+        if (xbuf + sched + static_smem + static_cast<size_t>(MK_NWC) * 1024 > static_cast<size_t>(smem_optin))
+            return bail(EDGEFM_ERR_CUDA, "model shape does not fit the shared-memory plan", cudaErrorInvalidValue);
+        const size_t avail = smem_optin - static_smem - xbuf - sched;
+        int depth = avail / (2 * MK_NWC) >= 4096 ? 2 : 1;
+        if (const char *dp = getenv("EDGEFM_RING_DEPTH")) { const int v = atoi(dp); if (v == 1 || v == 2) depth = v; }
+        int budget = 8192;   // upper bound of one tile = one ring slot
+        if (const char *tb = getenv("EDGEFM_TILE_BYTES")) { const int v = atoi(tb); if (v >= 1024 && v <= 65536) budget = v; }
+        const int fit = static_cast<int>(avail / (static_cast<size_t>(depth) * MK_NWC) / 128 * 128);
+        if (budget > fit) budget = fit;
+        int max_tile = 0;
+        auto add = [&](int kind, const void *W, int K, int units, const void *bias, const void *norm, const float *xsrc,
+                       float *out, int layer) {
+            MkPhase ph{};
+            const bool paired = kind == PH_QKV || kind == PH_SWIGLU;
+            choose_tile(K, paired, kind == PH_QKV ? d / 2 : 4, budget, &ph.rw, &ph.ksplit);
+            ph.W = (const uint16_t *)W; ph.bias = (const uint16_t *)bias; ph.norm_w = (const uint16_t *)norm;
+            ph.x_src = xsrc; ph.out = out; ph.K = K; ph.kind = kind; ph.kcs = K / 8 / ph.ksplit;
+            ph.units_total = units; ph.items_total = (units + ph.rw - 1) / ph.rw; ph.layer = layer;
+            const int tile = ph.rw * (paired ? 2 : 1) * ph.kcs * 16;
+            if (tile > max_tile) max_tile = tile;
+            phases.push_back(ph);
+        };
+        // buffers are allocated below; the descriptors' buffer pointers are filled after allocation
+        for (int l = 0; l < sh.n_layers; ++l) {
+            const edgefm_layer_weights &w = c->layers[l];
+            add(PH_QKV, w.wqkv, H, R / 2, sh.qkv_bias ? w.bqkv : nullptr, w.input_norm, nullptr, nullptr, l);
+            add(PH_RESID, w.wo, nq * d, H, nullptr, nullptr, nullptr, nullptr, l);
+            add(PH_SWIGLU, w.w_gate_up, H, F, nullptr, w.post_norm, nullptr, nullptr, l);
+            add(PH_RESID, w.w_down, F, H, nullptr, nullptr, nullptr, nullptr, l);
+        }
+        add(PH_LMHEAD, c->lm_head, H, sh.vocab, nullptr, c->final_norm, nullptr, nullptr, sh.n_layers);
+        const int slot_bytes = (max_tile + 127) / 128 * 128;
+        if (static_cast<size_t>(slot_bytes) * depth * MK_NWC > avail)
+            return bail(EDGEFM_ERR_CUDA, "weight rows do not fit the shared-memory ring", cudaErrorInvalidValue);
+        const int nslot = depth * MK_NWC;
+        c->mk.nslot = nslot; c->mk.slot_bytes = slot_bytes; c->mk.xbuf_bytes = static_cast<int>(xbuf);
+        c->mk.sched_bytes = static_cast<int>(sched);
+        c->mega_smem = xbuf + sched + static_cast<size_t>(nslot) * slot_bytes;
+        CREATE_TRY(cudaFuncSetAttribute(c->mega, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(c->mega_smem)));
+        int per_sm = 0;
+        CREATE_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, c->mega, MK_THREADS, c->mega_smem));
+        if (per_sm < 1) return bail(EDGEFM_ERR_CUDA, "persistent kernel does not fit one CTA per SM", cudaErrorInvalidValue);
+        c->p_attn.max_chunks = max_chunks;  // sizes the partial buffers below
+        c->p_lm.grid = c->mega_grid;
+    }
+
     const size_t kv_elems = static_cast<size_t>(sh.n_layers) * nkv * max_context * d;
     CREATE_TRY(dev_alloc(&c->k_cache, kv_elems));
     CREATE_TRY(dev_alloc(&c->v_cache, kv_elems));
@@ -446,6 +584,38 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
         std::vector<double> inv(d / 2);
         for (int i = 0; i < d / 2; ++i) inv[i] = std::pow(static_cast<double>(sh.rope_theta), -2.0 * i / d);
         CREATE_TRY(cudaMemcpy(c->inv_freq, inv.data(), inv.size() * sizeof(double), cudaMemcpyHostToDevice));
+    }
+
+    if (c->use_mega) {
+        CREATE_TRY(dev_alloc(&c->d_phases, phases.size()));
+        CREATE_TRY(dev_alloc(&c->grid_bar, 1));
+        CREATE_TRY(cudaMemset(c->grid_bar, 0, sizeof(unsigned)));
+        for (size_t i = 0; i < phases.size(); ++i) {
+            MkPhase &ph = phases[i];
+            const int k = static_cast<int>(i % 4);
+            if (i + 1 == phases.size()) { ph.x_src = c->x; ph.out = nullptr; }
+            else if (k == 0) { ph.x_src = ph.layer == 0 ? nullptr : c->x; ph.out = c->q; }
+            else if (k == 1) { ph.x_src = c->attn; ph.out = c->x; }
+            else if (k == 2) { ph.x_src = c->x; ph.out = c->act; }
+            else { ph.x_src = c->act; ph.out = c->x; }
+        }
+        CREATE_TRY(cudaMemcpy(c->d_phases, phases.data(), phases.size() * sizeof(MkPhase), cudaMemcpyHostToDevice));
+        MkParams &m = c->mk;
+        m.phases = c->d_phases; m.n_layers = sh.n_layers; m.H = H; m.nq = nq; m.nkv = nkv; m.d = d; m.F = F; m.V = sh.vocab;
+        m.eps = sh.rms_eps; m.scale = static_cast<float>(1.0 / std::sqrt(static_cast<double>(d)));
+        m.max_context = max_context; m.k_cache = c->k_cache; m.v_cache = c->v_cache; m.embed = (const uint16_t *)c->embed;
+        m.inv_freq = c->inv_freq; m.x = c->x; m.q = c->q; m.attn = c->attn; m.part_m = c->part_m; m.part_l = c->part_l;
+        m.part_o = c->part_o; m.att_min_chunk = 256;
+        if (const char *ac = getenv("EDGEFM_ATT_CHUNK")) { const int v = atoi(ac); if (v >= 8) m.att_min_chunk = v; } m.tickets = c->tickets; m.barrier = c->grid_bar;
+        m.lm_part_val = c->lm_part_val; m.lm_part_idx = c->lm_part_idx; m.state = c->state; m.req = c->req;
+        m.spin_limit = 1000000000u;  // 1 s
+        const char *pe_ = getenv("EDGEFM_PROFILE");
+        if (pe_ && pe_[0] == '1') {
+            c->prof_stride = 3 + 14 * sh.n_layers;
+            CREATE_TRY(dev_alloc(&c->prof, static_cast<size_t>(c->mega_grid) * c->prof_stride));
+            CREATE_TRY(cudaMemset(c->prof, 0, static_cast<size_t>(c->mega_grid) * c->prof_stride * 8));
+            m.prof = c->prof; m.prof_stride = c->prof_stride;
+        }
     }
 
     // record the step once; every decode step replays this graph
@@ -532,6 +702,31 @@ edgefm_status edgefm_get_length(const edgefm_ctx *ctx, int32_t *cur_len_host) {
 edgefm_status edgefm_get_launches_per_step(const edgefm_ctx *ctx, int32_t *n) {
     if (!ctx || !n) return EDGEFM_ERR_INVALID_ARG;
     *n = ctx->launches_per_step;
+    return EDGEFM_OK;
+}
+
+edgefm_status edgefm_debug_profile(edgefm_ctx *ctx, uint64_t *out_host, int64_t capacity, int32_t *n_ctas, int32_t *stride) {
+    if (!ctx || !n_ctas || !stride) return EDGEFM_ERR_INVALID_ARG;
+    *n_ctas = ctx->prof ? ctx->mega_grid : 0;
+    *stride = ctx->prof_stride;
+    if (!ctx->prof || !out_host) return EDGEFM_OK;
+    const int64_t n = static_cast<int64_t>(ctx->mega_grid) * ctx->prof_stride;
+    if (capacity < n) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "profile buffer too small");
+    DeviceGuard guard(ctx->device);
+    CUDA_TRY(ctx, cudaDeviceSynchronize());
+    CUDA_TRY(ctx, cudaMemcpy(out_host, ctx->prof, static_cast<size_t>(n) * 8, cudaMemcpyDeviceToHost));
+    return EDGEFM_OK;
+}
+
+edgefm_status edgefm_sync_status(edgefm_ctx *ctx, void *stream) {
+    if (!ctx) return EDGEFM_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    CUDA_TRY(ctx, cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    StepState st;
+    CUDA_TRY(ctx, cudaMemcpy(&st, ctx->state, sizeof st, cudaMemcpyDeviceToHost));
+    if (st.status != 0)
+        return fail(ctx, EDGEFM_ERR_TIMEOUT, "device status %d (6 = a bounded wait expired, 100+ = self-check code) operands %d %d; "
+                    "the context must be destroyed", st.status, st.pad[0], st.pad[1]);
     return EDGEFM_OK;
 }
 

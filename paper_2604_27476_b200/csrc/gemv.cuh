@@ -80,7 +80,8 @@ __global__ void __launch_bounds__(WR *WK * 32) gemv_kernel(const GemvArgs a) {
     constexpr int TR = RW * WR;
     constexpr int NT = WR * WK * 32;
     static_assert(TR % 2 == 0 || (EPI != EPI_QKV && EPI != EPI_SWIGLU), "paired epilogues need an even tile");
-    extern __shared__ __align__(16) float smem[];
+    extern __shared__ __align__(16) float gemv_smem[];
+    float *smem = gemv_smem;
     float *xs = smem;                 // [K]
     float *red = smem + a.K;          // [WK][TR]
     float *yt = red + WK * TR;        // [TR]

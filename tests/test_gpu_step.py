@@ -92,6 +92,8 @@ VARIANTS = {
     "g3_d128": dict(n_q_heads=6, n_kv_heads=2, head_dim=128, hidden=264),
     "g8": dict(n_q_heads=8, n_kv_heads=1, hidden=200, ffn=72, vocab=1000),
     "g7_odd": dict(n_q_heads=7, n_kv_heads=1, hidden=136, ffn=8, vocab=33, n_layers=3, qkv_bias=True),
+    # long rows (K slices per work item) and enough tiles per warp to wrap the shared-memory ring many times
+    "ring_wrap_ksplit": dict(hidden=512, ffn=6144, vocab=50000, n_layers=3, qkv_bias=True),
     "g5_kv3": dict(n_q_heads=15, n_kv_heads=3, head_dim=128, hidden=512, ffn=1000, vocab=777),
 }
 
@@ -130,7 +132,7 @@ def test_free_run_matches_teacher_forced_and_device_chaining():
     """token = -1 / position = -1 chain the previous step's result on the device."""
     import torch
     cfg = TINY
-    pair = Pair(cfg)
+    pair = Pair(cfg, max_context=cfg.cache_len + 20)
     try:
         tok, pos = first_token(cfg), cfg.first_position
         toks_ref, margins = [], []
