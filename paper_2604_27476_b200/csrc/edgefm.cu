@@ -182,23 +182,31 @@ MegaKernel mega_kernel_g(int G) {
     return nullptr;
 }
 
-// Tile geometry of one weight-streaming operator: as many rows (or row pairs) per tile as fit the
-// slot budget; rows longer than the budget are cut into K slices that divide the row evenly.
-inline void choose_tile(int K, bool paired, int pair_align, int budget_bytes, int *rw, int *ksplit) {
+// Tile geometry of one weight-streaming operator.
+//  * long operators (many rows per CTA): whole rows, as many per tile (rw rows or row pairs) as fit the
+//    slot budget while every warp keeps about two tiles;
+//  * short operators, and rows longer than a slot: one row (pair) per item, cut into `ksplit` K slices
+//    (a power of two dividing the row) that go to different warps, so that all warps of a CTA share the
+//    latency of the operator; their partial sums meet in shared memory.
+inline void choose_tile(int K, bool paired, int pair_align, int units, int ncta, int budget_bytes, int *rw, int *ksplit, int *split) {
     const int kc = K / 8;
     const int mult = paired ? 2 : 1;
-    const long long row_bytes = static_cast<long long>(K) * 2;
-    if (row_bytes * mult <= budget_bytes) {
+    const long long row_bytes = static_cast<long long>(K) * 2 * mult;
+    const double per_cta = static_cast<double>(units) / ncta;
+    *rw = 1; *ksplit = 1; *split = 0;
+    if (row_bytes <= budget_bytes && per_cta >= 2.0 * MK_NW) {
         int r = paired ? 4 : 8;
-        while (r > 1 && (row_bytes * mult * r > budget_bytes || (paired && pair_align % r != 0))) r >>= 1;
+        while (r > 1 && (row_bytes * r > budget_bytes || (paired && pair_align % r != 0) || per_cta / r < 2.0 * MK_NW)) r >>= 1;
         *rw = r;
-        *ksplit = 1;
         return;
     }
-    *rw = 1;
-    int s = 2;
-    while (s < kc && (kc % s != 0 || static_cast<long long>(kc / s) * 16 * mult > budget_bytes)) ++s;
+    int s = 1;
+    auto can_double = [&](int min_kcs) { return kc % (2 * s) == 0 && kc / (2 * s) >= min_kcs && 2 * s <= 16; };
+    while (row_bytes / s > budget_bytes && kc % (2 * s) == 0) s *= 2;           // must fit a slot
+    while (per_cta * s < MK_NW && can_double(64)) s *= 2;                       // at least one tile per warp
+    while (per_cta * s < 2.0 * MK_NW && can_double(256)) s *= 2;                // two per warp while slices stay long
     *ksplit = s;
+    *split = s > 1 ? 1 : 0;
 }
 
 }  // namespace edgefm
@@ -317,7 +325,7 @@ cudaError_t enqueue_step(edgefm_ctx *c, cudaStream_t s, int *n_launches) {
         // one cooperative launch: all CTAs are co-resident, which the grid barriers rely on
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(c->mega_grid);
-        cfg.blockDim = dim3(MK_THREADS);
+        cfg.blockDim = dim3(MK_NT);
         cfg.dynamicSmemBytes = c->mega_smem;
         cfg.stream = s;
         cudaLaunchAttribute attr[1];
@@ -503,34 +511,44 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
         int max_k = H;
         if (nq * d > max_k) max_k = nq * d;
         if (F > max_k) max_k = F;
-        const size_t att_bytes = (static_cast<size_t>(G) * d + MK_NWC * G * MK_ATT_TILE + 2 * MK_ATT_MW * G +
+        const size_t att_bytes = (static_cast<size_t>(G) * d + MK_NW * G * MK_ATT_TILE + 2 * MK_ATT_MW * G +
                                   static_cast<size_t>(MK_ATT_MW) * G * d + 2 * static_cast<size_t>(G) * max_chunks) * 4;
         size_t xbuf = static_cast<size_t>(max_k) * 4;
         if (att_bytes > xbuf) xbuf = att_bytes;
         xbuf = (xbuf + 255) / 256 * 256;
-        const size_t static_smem = 2048;  // mbarriers, rotary table, reduction scratch
+        cudaFuncAttributes fa{};
+        CREATE_TRY(cudaFuncGetAttributes(&fa, c->mega));
+        const size_t static_smem = fa.sharedSizeBytes + 1024;  // the kernel's static shared memory (mbarriers, tables, scratch) + margin
         const size_t n_phases = 4 * static_cast<size_t>(sh.n_layers) + 1;
-        const size_t sched = (n_phases * sizeof(MkPhase) + 127) / 128 * 128;
-        if (xbuf + sched + static_smem + static_cast<size_t>(MK_NWC) * 1024 > static_cast<size_t>(smem_optin))
+        const size_t sched = (n_phases * (sizeof(MkPhase) + sizeof(int2)) + 127) / 128 * 128;
+        if (xbuf + sched + static_smem + static_cast<size_t>(MK_NW) * 1024 > static_cast<size_t>(smem_optin))
             return bail(EDGEFM_ERR_CUDA, "model shape does not fit the shared-memory plan", cudaErrorInvalidValue);
         const size_t avail = smem_optin - static_smem - xbuf - sched;
-        int depth = avail / (2 * MK_NWC) >= 4096 ? 2 : 1;
-        if (const char *dp = getenv("EDGEFM_RING_DEPTH")) { const int v = atoi(dp); if (v == 1 || v == 2) depth = v; }
-        int budget = 8192;   // upper bound of one tile = one ring slot
+        // ring: `depth` slots per warp; prefer two slots of a natural tile size, deeper rings for small tiles
+        int budget = 12288;  // upper bound of one tile = one ring slot
         if (const char *tb = getenv("EDGEFM_TILE_BYTES")) { const int v = atoi(tb); if (v >= 1024 && v <= 65536) budget = v; }
-        const int fit = static_cast<int>(avail / (static_cast<size_t>(depth) * MK_NWC) / 128 * 128);
-        if (budget > fit) budget = fit;
+        {
+            const int fit1 = static_cast<int>(avail / MK_NW / 128 * 128);
+            if (budget > fit1) budget = fit1;
+        }
         int max_tile = 0;
+        bool split_overflow = false;
         auto add = [&](int kind, const void *W, int K, int units, const void *bias, const void *norm, const float *xsrc,
                        float *out, int layer) {
             MkPhase ph{};
             const bool paired = kind == PH_QKV || kind == PH_SWIGLU;
-            choose_tile(K, paired, kind == PH_QKV ? d / 2 : 4, budget, &ph.rw, &ph.ksplit);
+            choose_tile(K, paired, kind == PH_QKV ? d / 2 : 4, units, c->mega_grid, budget, &ph.rw, &ph.ksplit, &ph.split);
+            ph.s_shift = 0;
+            while ((1 << ph.s_shift) < ph.ksplit) ++ph.s_shift;
             ph.W = (const uint16_t *)W; ph.bias = (const uint16_t *)bias; ph.norm_w = (const uint16_t *)norm;
             ph.x_src = xsrc; ph.out = out; ph.K = K; ph.kind = kind; ph.kcs = K / 8 / ph.ksplit;
             ph.units_total = units; ph.items_total = (units + ph.rw - 1) / ph.rw; ph.layer = layer;
             const int tile = ph.rw * (paired ? 2 : 1) * ph.kcs * 16;
             if (tile > max_tile) max_tile = tile;
+            if (ph.split) {  // partial sums of one CTA's share must fit the shared-memory scratch
+                const long long per_cta = (ph.items_total + c->mega_grid - 1) / c->mega_grid + 1;
+                if (per_cta * ph.ksplit * (paired ? 2 : 1) > MK_PARTIAL_FLOATS) split_overflow = true;
+            }
             phases.push_back(ph);
         };
         // buffers are allocated below; the descriptors' buffer pointers are filled after allocation
@@ -542,16 +560,20 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
             add(PH_RESID, w.w_down, F, H, nullptr, nullptr, nullptr, nullptr, l);
         }
         add(PH_LMHEAD, c->lm_head, H, sh.vocab, nullptr, c->final_norm, nullptr, nullptr, sh.n_layers);
+        if (split_overflow || max_tile > budget)
+            return bail(EDGEFM_ERR_CUDA, "model shape does not fit the tile plan", cudaErrorInvalidValue);
         const int slot_bytes = (max_tile + 127) / 128 * 128;
-        if (static_cast<size_t>(slot_bytes) * depth * MK_NWC > avail)
-            return bail(EDGEFM_ERR_CUDA, "weight rows do not fit the shared-memory ring", cudaErrorInvalidValue);
-        const int nslot = depth * MK_NWC;
-        c->mk.nslot = nslot; c->mk.slot_bytes = slot_bytes; c->mk.xbuf_bytes = static_cast<int>(xbuf);
+        int depth = static_cast<int>(avail / (static_cast<size_t>(slot_bytes) * MK_NW));
+        if (const char *dp = getenv("EDGEFM_RING_DEPTH")) { const int v = atoi(dp); if (v >= 1 && v < depth) depth = v; }
+        if (depth < 1) return bail(EDGEFM_ERR_CUDA, "weight rows do not fit the shared-memory ring", cudaErrorInvalidValue);
+        depth = depth >= 4 ? 4 : (depth >= 2 ? 2 : 1);   // power of two
+        c->mk.depth = depth; c->mk.depth_shift = depth == 4 ? 2 : (depth == 2 ? 1 : 0);
+        c->mk.slot_bytes = slot_bytes; c->mk.xbuf_bytes = static_cast<int>(xbuf);
         c->mk.sched_bytes = static_cast<int>(sched);
-        c->mega_smem = xbuf + sched + static_cast<size_t>(nslot) * slot_bytes;
+        c->mega_smem = xbuf + sched + static_cast<size_t>(depth) * MK_NW * slot_bytes;
         CREATE_TRY(cudaFuncSetAttribute(c->mega, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(c->mega_smem)));
         int per_sm = 0;
-        CREATE_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, c->mega, MK_THREADS, c->mega_smem));
+        CREATE_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, c->mega, MK_NT, c->mega_smem));
         if (per_sm < 1) return bail(EDGEFM_ERR_CUDA, "persistent kernel does not fit one CTA per SM", cudaErrorInvalidValue);
         c->p_attn.max_chunks = max_chunks;  // sizes the partial buffers below
         c->p_lm.grid = c->mega_grid;
@@ -571,12 +593,12 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
     CREATE_TRY(dev_alloc(&c->part_o, static_cast<size_t>(nq) * c->p_attn.max_chunks * d));
     CREATE_TRY(dev_alloc(&c->lm_part_val, c->p_lm.grid));
     CREATE_TRY(dev_alloc(&c->lm_part_idx, c->p_lm.grid));
-    CREATE_TRY(dev_alloc(&c->tickets, nkv + 1));
+    CREATE_TRY(dev_alloc(&c->tickets, nq + nkv + 2));
     CREATE_TRY(dev_alloc(&c->state, 1));
     CREATE_TRY(dev_alloc(&c->req, 1));
     CREATE_TRY(cudaMemset(c->k_cache, 0, kv_elems * 2));
     CREATE_TRY(cudaMemset(c->v_cache, 0, kv_elems * 2));
-    CREATE_TRY(cudaMemset(c->tickets, 0, (nkv + 1) * sizeof(unsigned)));
+    CREATE_TRY(cudaMemset(c->tickets, 0, (nq + nkv + 2) * sizeof(unsigned)));
     CREATE_TRY(cudaMemset(c->state, 0, sizeof(StepState)));
     {
         StepRequest r{-1, -1, nullptr, nullptr};
@@ -605,8 +627,12 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
         m.eps = sh.rms_eps; m.scale = static_cast<float>(1.0 / std::sqrt(static_cast<double>(d)));
         m.max_context = max_context; m.k_cache = c->k_cache; m.v_cache = c->v_cache; m.embed = (const uint16_t *)c->embed;
         m.inv_freq = c->inv_freq; m.x = c->x; m.q = c->q; m.attn = c->attn; m.part_m = c->part_m; m.part_l = c->part_l;
-        m.part_o = c->part_o; m.att_min_chunk = 256;
-        if (const char *ac = getenv("EDGEFM_ATT_CHUNK")) { const int v = atoi(ac); if (v >= 8) m.att_min_chunk = v; } m.tickets = c->tickets; m.barrier = c->grid_bar;
+        m.part_o = c->part_o; m.tickets = c->tickets; m.barrier = c->grid_bar;
+        m.nph = static_cast<int>(phases.size());
+        m.half_shift = d == 64 ? 5 : 6;
+        m.att_chunk_shared = 256; m.att_chunk_split = 64; m.att_split_max_n = 8192;
+        if (const char *ac = getenv("EDGEFM_ATT_SPLIT_MAX")) { const int v = atoi(ac); if (v >= 0) m.att_split_max_n = v; }
+        if (const char *ac = getenv("EDGEFM_ATT_CHUNK")) { const int v = atoi(ac); if (v >= 8) { m.att_chunk_shared = v; m.att_chunk_split = v; } }
         m.lm_part_val = c->lm_part_val; m.lm_part_idx = c->lm_part_idx; m.state = c->state; m.req = c->req;
         m.spin_limit = 1000000000u;  // 1 s
         const char *pe_ = getenv("EDGEFM_PROFILE");

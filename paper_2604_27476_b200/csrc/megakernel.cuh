@@ -4,16 +4,22 @@
 // split over five operators that depend on one another.  Separate kernels drain and refill the memory
 // pipeline at every boundary.  Here the weight stream is decoupled from the dependency chain:
 //
-//   * a PRODUCER warp per CTA walks the step's static schedule (QKV, O, gate/up, down of every layer,
-//     then lm_head) and keeps a ring of shared-memory slots full with bulk async copies (TMA,
-//     cp.async.bulk + mbarrier complete_tx) of this CTA's weight tiles.  It never waits for the
-//     arithmetic, only for a free slot, so HBM stays busy across operator boundaries and grid barriers;
-//   * CONSUMER warps take tiles from the ring (one warp per work item, no intra-tile cross-warp sync),
-//     multiply them with the activation vector staged in shared memory, and run the fused epilogues
-//     (bias + RoPE + KV append, residual add, SwiGLU, logits + argmax);
-//   * between dependent operators the consumers meet at a grid barrier (monotonic counter in global
-//     memory, release/acquire, bounded spin).  Attention (split-KV with an exact log-sum-exp merge) runs
-//     on the consumer warps between two barriers while the producer prefetches the next operators.
+//   * The step's weight traffic is a static schedule (QKV, O, gate/up, down of every layer, then
+//     lm_head).  Every CTA owns a fixed share of each operator's rows, and every warp of the CTA a fixed
+//     sequence of tiles (a few rows, or one K slice of a long row) across the WHOLE step.
+//   * Each warp keeps a private ring of `depth` shared-memory slots filled with its next tiles by bulk
+//     async copies (TMA: cp.async.bulk + mbarrier complete_tx).  When it has consumed a tile it
+//     immediately re-arms the slot with the tile `depth` ahead -- regardless of operator boundaries.
+//     So HBM keeps streaming while the arithmetic waits at a grid barrier, stages an activation vector
+//     or runs attention.
+//     A slot is armed and drained by the same warp, in program order, so the one-bit mbarrier phase
+//     parity cannot alias and no "empty" barrier is needed (a proxy fence orders the warp's reads before
+//     the next asynchronous write).
+//   * A tile is multiplied with the activation vector staged in shared memory; the fused epilogues
+//     (bias + RoPE + KV append, residual add, SwiGLU, logits + argmax) run in the warp that owns the rows.
+//   * Between dependent operators all CTAs meet at a grid barrier (monotonic counter in global memory,
+//     release/acquire, bounded spin).  Attention (split-KV, exact log-sum-exp merge) runs between two
+//     barriers.
 //
 // Every wait is bounded: on expiry the CTA records EDGEFM_ERR_TIMEOUT in the device state, stops
 // issuing copies, waits (bounded) for the copies it has in flight and returns.
@@ -22,15 +28,14 @@
 
 namespace edgefm {
 
-constexpr int MK_NWC = 15;                       // consumer warps per CTA
-constexpr int MK_NTC = MK_NWC * 32;              // consumer threads
-constexpr int MK_THREADS = MK_NTC + 32;          // + one producer warp
-constexpr int MK_MAX_SLOTS = 32;
+constexpr int MK_NW = 12;                        // warps per CTA (each streams and consumes its own tiles)
+constexpr int MK_NT = MK_NW * 32;
+constexpr int MK_MAX_DEPTH = 4;                  // ring slots per warp
 constexpr int MK_ATT_LPP = 4;                    // lanes per cached position in the score phase
 constexpr int MK_ATT_TILE = 32 / MK_ATT_LPP;     // positions per warp iteration
-constexpr int MK_ATT_MW = (MK_NWC + 1) / 2;      // warps whose partials fit the merge area at once
-
-static_assert(2 * MK_NWC <= MK_MAX_SLOTS && MK_MAX_SLOTS <= 32, "one producer lane per ring slot");
+constexpr int MK_ATT_MW = (MK_NW + 1) / 2;       // warps whose partials fit the merge area at once
+constexpr int MK_ATT_SPLIT_MAXC = 12;            // chunks per head when every query head has its own CTAs
+constexpr int MK_PARTIAL_FLOATS = 2048;          // shared-memory scratch: split-K partial sums / chunk statistics
 
 enum { PH_QKV = 0, PH_RESID = 1, PH_SWIGLU = 2, PH_LMHEAD = 3 };
 
@@ -43,19 +48,23 @@ struct alignas(16) MkPhase {
     float *out;              // PH_QKV: q fp32; PH_RESID: x (+=); PH_SWIGLU: act; PH_LMHEAD: unused
     int K;                   // columns (multiple of 8)
     int kind;
-    int rw;                  // units per work item (rows, or row pairs for PH_QKV / PH_SWIGLU)
+    int rw;                  // units per work item (rows, or row pairs for PH_QKV / PH_SWIGLU); 1 when split
     int ksplit;              // K slices per item (tiles per item)
     int kcs;                 // 16-byte pieces per row slice = K / 8 / ksplit
     int units_total;         // rows (PH_RESID, PH_LMHEAD), pairs (PH_QKV: rows/2, PH_SWIGLU: F)
     int items_total;         // ceil(units_total / rw)
     int layer;
-    int pad_[3];
+    int s_shift;             // log2(ksplit); ksplit is a power of two
+    int split;               // 1: the tiles of an item go to different warps, partial sums meet in shared memory
+    int pad_;
 };
 static_assert(sizeof(MkPhase) % 16 == 0, "descriptor is copied in 16-byte pieces");
 
 struct MkParams {
-    const MkPhase *phases;   // [4 * n_layers + 1]
+    const MkPhase *phases;   // [nph]
+    int nph;                 // 4 * n_layers + 1
     int n_layers, H, nq, nkv, d, F, V;
+    int half_shift;          // log2(d / 2)
     float eps, scale;
     int max_context;
     uint16_t *k_cache, *v_cache;   // [L][nkv][max_context][d]
@@ -63,15 +72,18 @@ struct MkParams {
     const double *inv_freq;        // [d/2]
     float *x, *q, *attn;
     float *part_m, *part_l, *part_o;
-    int max_chunks;                // attention chunks per kv head (<= gridDim.x / nkv)
-    int att_min_chunk;
-    unsigned *tickets;             // [nkv] attention, [nkv] lm_head
+    int max_chunks;                // row stride of the attention partial buffers (>= any chunk count)
+    int att_chunk_shared;          // smallest chunk (positions) when one CTA serves a whole GQA group
+    int att_chunk_split;           // smallest chunk when every query head has its own CTAs
+    int att_split_max_n;           // contexts up to this length use one-head-per-CTA attention
+    unsigned *tickets;             // [nq] attention, [nq] = lm_head
     unsigned *barrier;             // grid barrier counter (0 between launches)
     float *lm_part_val;
     int *lm_part_idx;
     StepState *state;
     const StepRequest *req;
-    int nslot, slot_bytes, xbuf_bytes, sched_bytes;
+    int depth, depth_shift;        // ring slots per warp (1, 2 or 4) and its log2
+    int slot_bytes, xbuf_bytes, sched_bytes;
     unsigned spin_limit;           // upper bound of every device-side wait, nanoseconds
     unsigned long long *prof;      // optional timestamps [gridDim.x][prof_stride] (diagnostics), or null
     int prof_stride;
@@ -81,9 +93,6 @@ struct MkParams {
 __device__ __forceinline__ unsigned smem_u32(const void *p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
 __device__ __forceinline__ void mbar_init(unsigned long long *b, unsigned count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(b)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(unsigned long long *b) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(b)) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long *b, unsigned bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(bytes) : "memory");
@@ -125,7 +134,10 @@ __device__ __forceinline__ void bulk_copy_g2s(void *dst, const void *src, unsign
         ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
         : "memory");
 }
-__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(MK_NTC) : "memory"); }
+__device__ __forceinline__ void bulk_prefetch_l2(const void *src, unsigned bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cta_sync() { __syncthreads(); }
 
 __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned *p) {
     unsigned v;
@@ -133,9 +145,9 @@ __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned *p) {
     return v;
 }
 
-// Diagnostics: consumer thread 0 of every CTA records %globaltimer at fixed points of the step.
-__device__ __forceinline__ void prof_stamp(const MkParams &p, int tidc, int &idx) {
-    if (p.prof && tidc == 0) {
+// Diagnostics: thread 0 of every CTA records %globaltimer at fixed points of the step.
+__device__ __forceinline__ void prof_stamp(const MkParams &p, int tid, int &idx) {
+    if (p.prof && tid == 0) {
         if (idx < p.prof_stride) p.prof[static_cast<size_t>(blockIdx.x) * p.prof_stride + idx] = global_ns();
         ++idx;
     }
@@ -151,11 +163,11 @@ __device__ __forceinline__ bool diag_fail(const MkParams &p, volatile int *abort
     return false;
 }
 
-// All consumer threads of all CTAs meet here.  Returns false when the wait expired (step aborted).
-__device__ __forceinline__ bool grid_barrier(const MkParams &p, unsigned target, volatile int *abort_flag, int tidc, int &prof_idx) {
-    consumer_sync();
-    prof_stamp(p, tidc, prof_idx);   // this CTA's share of the operator is done
-    if (tidc == 0 && !*abort_flag) {
+// All threads of all CTAs meet here.  Returns false when the wait expired (step aborted).
+__device__ __forceinline__ bool grid_barrier(const MkParams &p, unsigned target, volatile int *abort_flag, int tid, int &prof_idx) {
+    cta_sync();
+    prof_stamp(p, tid, prof_idx);   // this CTA's share of the operator is done
+    if (tid == 0 && !*abort_flag) {
         asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.barrier) : "memory");
         unsigned it = 0;
         unsigned long long t0 = 0;
@@ -167,8 +179,8 @@ __device__ __forceinline__ bool grid_barrier(const MkParams &p, unsigned target,
             }
         }
     }
-    consumer_sync();
-    prof_stamp(p, tidc, prof_idx);   // released by the slowest CTA
+    cta_sync();
+    prof_stamp(p, tid, prof_idx);   // released by the slowest CTA
     return !*abort_flag;
 }
 
@@ -184,90 +196,78 @@ __device__ __forceinline__ int item_rows(const MkPhase &P, const MkParams &p, in
     cnt = min(P.rw, P.units_total - u0);
     if (P.kind == PH_QKV) {
         const int half = p.d >> 1;
-        const int head = u0 / half, i0 = u0 - head * half;
+        const int head = u0 >> p.half_shift, i0 = u0 & (half - 1);
         return head * p.d + i0 + blk * half;
     }
     if (P.kind == PH_SWIGLU) return u0 + blk * p.F;
     return u0;
 }
 
-// ---- producer: keep the ring full -----------------------------------------------------------------------
-// Every consumer warp w has a private sub-ring of `depth` slots (slot = w * depth + q).  Warp w consumes
-// its own tiles strictly in order, so a slot is always filled and drained by the same pair of threads
-// in alternation: the one-bit mbarrier phase parity can never alias (a warp cannot run a whole ring
-// round ahead of a slot it does not own), and a slow warp never blocks the supply of the others.
-// Lane (w, q) of the producer warp issues the tiles k = q, q + depth, ... of warp w's tile sequence over
-// the whole step; the lanes work independently, so their address arithmetic overlaps.
-__device__ __noinline__ void producer_loop(const MkParams &p, const MkPhase *s_ph, unsigned char *ring,
-                                           unsigned long long *full_bar, unsigned long long *empty_bar,
-                                           volatile int *abort_flag, int lane) {
-    if (lane >= p.nslot) return;
-    unsigned long long policy;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-    const int cta = blockIdx.x, ncta = gridDim.x;
-    const int nph = 4 * p.n_layers + 1;
-    const int depth = p.nslot / MK_NWC;
-    const int w = lane / depth;          // consumer warp served by this lane
-    unsigned char *dst = ring + static_cast<size_t>(lane) * p.slot_bytes;
-    unsigned long long *fb = &full_bar[lane], *eb = &empty_bar[lane];
-    int ph = 0, it0 = 0, ntiles = 0;
-    int local = lane - w * depth;  // index in warp w's tile sequence of the current phase
-    unsigned round = 0;            // how often this slot has been filled
-    bool ok = true;
-    bool fresh = true;             // phase changed: recompute the warp's share
-    while (ok) {
-        if (fresh) {
-            if (ph >= nph) break;
-            int it1;
-            item_range(s_ph[ph].items_total, cta, ncta, it0, it1);
-            const int n_items = it1 - it0;
-            const int mine = n_items > w ? (n_items - w + MK_NWC - 1) / MK_NWC : 0;   // items i = w, w + NWC, ...
-            ntiles = mine * s_ph[ph].ksplit;
-            fresh = false;
-        }
-        if (local >= ntiles) { local -= ntiles; ++ph; fresh = true; continue; }
-        const MkPhase &P = s_ph[ph];
-        const int S = P.ksplit;
-        const int it = it0 + w + (S == 1 ? local : local / S) * MK_NWC;
-        const int sl = S == 1 ? 0 : local % S;
-        const int nblk = (P.kind == PH_QKV || P.kind == PH_SWIGLU) ? 2 : 1;
-        const unsigned seg_bytes = static_cast<unsigned>(P.kcs) * 16u;
-        int cnt;
-        const int row_lo = item_rows(P, p, it, 0, cnt);
-        {   // bounds of the tile about to be fetched (rows inside the matrix, bytes inside the slot, 16-byte rule)
-            const long long rows_total = P.kind == PH_QKV ? 2LL * P.units_total : (P.kind == PH_SWIGLU ? 2LL * p.F : P.units_total);
-            const int row_hi_chk = nblk == 2 ? item_rows(P, p, it, 1, cnt) : row_lo;
-            const bool bad = cnt < 1 || seg_bytes == 0 || (seg_bytes & 15u) || row_lo < 0 || row_lo + cnt > rows_total ||
-                             row_hi_chk + cnt > rows_total || static_cast<long long>(nblk - 1) * P.rw * seg_bytes + static_cast<long long>(cnt) * seg_bytes > p.slot_bytes ||
-                             (sl + 1) * P.kcs * 8 > P.K || (reinterpret_cast<unsigned long long>(P.W) & 15ull) || (smem_u32(dst) & 15u);
-            if (bad) { ok = diag_fail(p, abort_flag, 1, ph, it); break; }
-        }
-        if (!mbar_wait(eb, (round & 1u) ^ 1u, abort_flag, p.spin_limit)) { ok = false; break; }
-        mbar_arrive_expect_tx(fb, static_cast<unsigned>(cnt * nblk) * seg_bytes);
-        for (int b = 0; b < nblk; ++b) {
-            const int row0 = b ? item_rows(P, p, it, 1, cnt) : row_lo;
-            unsigned char *d = dst + static_cast<size_t>(b * P.rw) * seg_bytes;
-            if (S == 1) {  // whole rows are contiguous: one copy per block
-                bulk_copy_g2s(d, P.W + static_cast<size_t>(row0) * P.K, static_cast<unsigned>(cnt) * seg_bytes, fb, policy);
-            } else {
-                for (int r = 0; r < cnt; ++r)
-                    bulk_copy_g2s(d + static_cast<size_t>(r) * seg_bytes,
-                                  P.W + static_cast<size_t>(row0 + r) * P.K + static_cast<size_t>(sl) * P.kcs * 8, seg_bytes, fb, policy);
-            }
-        }
-        ++round;
-        local += depth;
-    }
-    if (!ok && round > 0) {
-        // aborted: wait (bounded) until the last copy this lane issued has landed before the CTA may exit
-        if (p.state->status == 0) p.state->status = 6;
-        const unsigned long long t0 = global_ns();
-        while (!mbar_try_wait(fb, (round - 1u) & 1u))
-            if (global_ns() - t0 > p.spin_limit) break;
+// ---- a warp's position in its tile sequence over the whole step ----------------------------------------
+// Tile j of a CTA's share of an operator is slice (j & (ksplit-1)) of item (j >> s_shift); warp w owns the
+// tiles j = w, w + NW, ...  The CTA's item range of every operator is tabulated once per launch (s_rng).
+struct TileCursor {
+    int ph;        // operator index (nph = past the end)
+    int j;         // tile index inside this CTA's share of the operator
+    int it0;       // first item of this CTA in operator ph
+    int n_tiles;   // tiles of this CTA in operator ph
+};
+__device__ __forceinline__ void cursor_enter_phase(TileCursor &c, const MkParams &p, const MkPhase *s_ph, const int2 *s_rng, int warp) {
+    while (c.ph < p.nph) {  // skip operators in which this warp owns no tile
+        const int2 r = s_rng[c.ph];
+        c.it0 = r.x;
+        c.n_tiles = (r.y - r.x) << s_ph[c.ph].s_shift;
+        if (warp < c.n_tiles) { c.j = warp; return; }
+        ++c.ph;
     }
 }
+__device__ __forceinline__ void cursor_advance(TileCursor &c, const MkParams &p, const MkPhase *s_ph, const int2 *s_rng, int warp) {
+    c.j += MK_NW;
+    if (c.j < c.n_tiles) return;
+    ++c.ph;
+    cursor_enter_phase(c, p, s_ph, s_rng, warp);
+}
 
-// ---- consumer: one work item (rw rows or row pairs, all K slices) by one warp -----------------------------
+// Fetch the tile under cursor `c` into a ring slot.  Called by a whole warp after __syncwarp(); lane 0 issues.
+__device__ __forceinline__ bool issue_tile(const MkParams &p, const MkPhase *s_ph, const TileCursor &c, unsigned char *dst,
+                                           unsigned long long *bar, unsigned long long policy, volatile int *abort_flag, int lane) {
+    const MkPhase &P = s_ph[c.ph];
+    const int it = c.it0 + (c.j >> P.s_shift);
+    const int sl = c.j & (P.ksplit - 1);
+    const int nblk = (P.kind == PH_QKV || P.kind == PH_SWIGLU) ? 2 : 1;
+    const unsigned seg_bytes = static_cast<unsigned>(P.kcs) * 16u;
+    int cnt;
+    const int row_lo = item_rows(P, p, it, 0, cnt);
+    const unsigned bytes = static_cast<unsigned>(cnt) * seg_bytes;   // one contiguous run per block
+    // bounds of the tile: at least one row, inside the slot, inside the matrix (16-byte rule holds by construction:
+    // K % 8 == 0, kcs * 16-byte slices, 16-byte aligned bases and slots, all checked on the host)
+    if (cnt < 1 || static_cast<unsigned>(nblk - 1) * P.rw * seg_bytes + bytes > static_cast<unsigned>(p.slot_bytes) ||
+        it >= P.items_total || (sl + 1) * P.kcs * 8 > P.K)
+        return diag_fail(p, abort_flag, 1, c.ph, it);
+    if (lane == 0) {
+        const uint16_t *src = P.W + static_cast<size_t>(row_lo) * P.K + static_cast<size_t>(sl) * P.kcs * 8;
+        // the slot was read through the generic proxy by this warp: order those reads before the async write
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive_expect_tx(bar, bytes * nblk);
+        bulk_copy_g2s(dst, src, bytes, bar, policy);
+        if (nblk == 2) {
+            const size_t partner = P.kind == PH_QKV ? static_cast<size_t>(p.d >> 1) : static_cast<size_t>(p.F);   // rows between the blocks
+            bulk_copy_g2s(dst + static_cast<size_t>(P.rw) * seg_bytes, src + partner * P.K, bytes, bar, policy);
+        }
+    }
+    return true;
+}
+
+// Per-warp streaming state.
+struct WarpStream {
+    TileCursor pf;          // next tile to fetch into shared memory (depth tiles ahead of consumption)
+    unsigned consumed;      // tiles consumed so far by this warp
+    unsigned issued;        // tiles fetched so far
+    unsigned char *slots;   // this warp's `depth` ring slots
+    unsigned long long *bars;
+    unsigned long long policy;
+};
+
 struct ItemCtx {
     float rscale;          // deferred RMSNorm factor (1 for plain prologues)
     int slot_row;          // cache slot written by this step
@@ -275,132 +275,225 @@ struct ItemCtx {
     float best_v;          // PH_LMHEAD running argmax of this lane
     int best_i;
     float *logits_out;
-    unsigned warp;         // consumer warp index
 };
 
+// ---- fused epilogue of one output unit (a row, or a row pair) ------------------------------------------------
+__device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkPhase &P, ItemCtx &cx, int u, float lo, float hi) {
+    if (P.kind == PH_RESID) {
+        P.out[u] = __ldcg(P.out + u) + lo;
+    } else if (P.kind == PH_LMHEAD) {
+        if (cx.logits_out) cx.logits_out[u] = lo;
+        if (arg_better(lo, u, cx.best_v, cx.best_i)) { cx.best_v = lo; cx.best_i = u; }
+    } else if (P.kind == PH_SWIGLU) {
+        P.out[u] = lo / (1.f + expf(-lo)) * hi;
+    } else {  // PH_QKV: bias, rotate-half RoPE of q and k, q to the work buffer, k and v to the cache row of this step
+        const int half = p.d >> 1;
+        const int head = u >> p.half_shift, i = u & (half - 1);
+        const int row_lo = head * p.d + i, row_hi = row_lo + half;
+        if (P.bias) { lo += bf16_bits_to_f32(P.bias[row_lo]); hi += bf16_bits_to_f32(P.bias[row_hi]); }
+        const size_t layer_off = static_cast<size_t>(P.layer) * p.nkv * p.max_context * p.d;
+        if (head < p.nq + p.nkv) {
+            const float c = cx.rope[i], sn = cx.rope[half + i];
+            const float rlo = lo * c - hi * sn, rhi = hi * c + lo * sn;
+            if (head < p.nq) {
+                P.out[row_lo] = rlo;
+                P.out[row_hi] = rhi;
+            } else {
+                uint16_t *dst = p.k_cache + layer_off + (static_cast<size_t>(head - p.nq) * p.max_context + cx.slot_row) * p.d;
+                dst[i] = f32_to_bf16_bits(rlo);
+                dst[i + half] = f32_to_bf16_bits(rhi);
+            }
+        } else {
+            uint16_t *dst = p.v_cache + layer_off + (static_cast<size_t>(head - p.nq - p.nkv) * p.max_context + cx.slot_row) * p.d;
+            dst[i] = f32_to_bf16_bits(lo);
+            dst[i + half] = f32_to_bf16_bits(hi);
+        }
+    }
+}
+
+// ---- one tile (NR row slices of kcs 16-byte pieces) by one warp: wait, multiply, re-arm the slot ------------
 template <int NR>
-__device__ __forceinline__ bool consume_item(const MkParams &p, const MkPhase &P, int it, unsigned &tile_no, const float4 *xsA,
-                                             const float4 *xsB, const unsigned char *ring, unsigned long long *full_bar,
-                                             unsigned long long *empty_bar, volatile int *abort_flag, ItemCtx &cx, int lane) {
+__device__ __forceinline__ bool consume_tile(const MkParams &p, const MkPhase *s_ph, const int2 *s_rng, const MkPhase &P, int slice,
+                                             WarpStream &ws, const float4 *xsA, const float4 *xsB, volatile int *abort_flag,
+                                             float (&out)[NR], int warp, int lane) {
     float acc[NR], acc2[NR];   // two chains per row halve the dependent-FMA latency
 #pragma unroll
     for (int r = 0; r < NR; ++r) { acc[r] = 0.f; acc2[r] = 0.f; }
     const int kcs = P.kcs;
-    for (int s = 0; s < P.ksplit; ++s) {
-        const unsigned depth = static_cast<unsigned>(p.nslot) / MK_NWC;       // this warp's private sub-ring
-        const unsigned slot = cx.warp * depth + tile_no % depth;
-        const unsigned par = (tile_no / depth) & 1u;
-        ++tile_no;
-        if (NR * kcs * 16 > p.slot_bytes || (s + 1) * kcs * 32 > p.xbuf_bytes) return diag_fail(p, abort_flag, 2, kcs, NR);
-        if (!mbar_wait(&full_bar[slot], par, abort_flag, p.spin_limit)) return false;
-        const uint4 *t = reinterpret_cast<const uint4 *>(ring + static_cast<size_t>(slot) * p.slot_bytes);
-        const float4 *a = xsA + s * kcs, *b = xsB + s * kcs;
-#pragma unroll 2
-        for (int c = lane; c < kcs; c += 32) {
-            const float4 x0 = a[c], x1 = b[c];
+    if (NR * kcs * 16 > p.slot_bytes || P.ksplit * kcs * 32 > p.xbuf_bytes) return diag_fail(p, abort_flag, 2, kcs, NR);
+    const unsigned q = ws.consumed & static_cast<unsigned>(p.depth - 1);             // depth is a power of two
+    const unsigned par = (ws.consumed >> p.depth_shift) & 1u;
+    if (!mbar_wait(&ws.bars[q], par, abort_flag, p.spin_limit)) return false;
+    unsigned char *slot = ws.slots + static_cast<size_t>(q) * p.slot_bytes;
+    const uint4 *t = reinterpret_cast<const uint4 *>(slot);
+    const float4 *a = xsA + slice * kcs, *b = xsB + slice * kcs;
+    auto fma_chunk = [&](const uint4 &w, const float4 &x0, const float4 &x1, int r) {
+        acc[r] = fmaf(bf16lo(w.x), x0.x, acc[r]);  acc2[r] = fmaf(bf16hi(w.x), x0.y, acc2[r]);
+        acc[r] = fmaf(bf16lo(w.y), x0.z, acc[r]);  acc2[r] = fmaf(bf16hi(w.y), x0.w, acc2[r]);
+        acc[r] = fmaf(bf16lo(w.z), x1.x, acc[r]);  acc2[r] = fmaf(bf16hi(w.z), x1.y, acc2[r]);
+        acc[r] = fmaf(bf16lo(w.w), x1.z, acc[r]);  acc2[r] = fmaf(bf16hi(w.w), x1.w, acc2[r]);
+    };
+    constexpr int UN = NR >= 8 ? 1 : (NR == 4 ? 2 : 3);   // lane-chunks whose loads are issued together
+    int c = lane;
+    for (; c + 32 * (UN - 1) < kcs; c += 32 * UN) {
+        float4 x0[UN], x1[UN];
+        uint4 w[UN][NR];
 #pragma unroll
-            for (int r = 0; r < NR; ++r) {
-                const uint4 w = t[r * kcs + c];
-                acc[r] = fmaf(bf16lo(w.x), x0.x, acc[r]);  acc2[r] = fmaf(bf16hi(w.x), x0.y, acc2[r]);
-                acc[r] = fmaf(bf16lo(w.y), x0.z, acc[r]);  acc2[r] = fmaf(bf16hi(w.y), x0.w, acc2[r]);
-                acc[r] = fmaf(bf16lo(w.z), x1.x, acc[r]);  acc2[r] = fmaf(bf16hi(w.z), x1.y, acc2[r]);
-                acc[r] = fmaf(bf16lo(w.w), x1.z, acc[r]);  acc2[r] = fmaf(bf16hi(w.w), x1.w, acc2[r]);
-            }
+        for (int u = 0; u < UN; ++u) {
+            x0[u] = a[c + 32 * u]; x1[u] = b[c + 32 * u];
+#pragma unroll
+            for (int r = 0; r < NR; ++r) w[u][r] = t[r * kcs + c + 32 * u];
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&empty_bar[slot]);
+#pragma unroll
+        for (int u = 0; u < UN; ++u)
+#pragma unroll
+            for (int r = 0; r < NR; ++r) fma_chunk(w[u][r], x0[u], x1[u], r);
+    }
+    for (; c < kcs; c += 32) {
+        const float4 x0 = a[c], x1 = b[c];
+#pragma unroll
+        for (int r = 0; r < NR; ++r) fma_chunk(t[r * kcs + c], x0, x1, r);
+    }
+    ++ws.consumed;
+    __syncwarp();
+    // re-arm the slot with the tile `depth` ahead in this warp's sequence
+    if (ws.pf.ph < p.nph) {
+        if (!issue_tile(p, s_ph, ws.pf, slot, &ws.bars[q], ws.policy, abort_flag, lane)) return false;
+        ++ws.issued;
+        cursor_advance(ws.pf, p, s_ph, s_rng, warp);
     }
 #pragma unroll
-    for (int r = 0; r < NR; ++r) acc[r] = warp_sum(acc[r] + acc2[r]) * cx.rscale;
+    for (int r = 0; r < NR; ++r) out[r] = warp_sum(acc[r] + acc2[r]);
+    return true;
+}
 
-    // ---- fused epilogue: lane r finishes unit r of the item ---------------------------------------------
-    const int u0 = it * P.rw;
-    if (P.kind == PH_RESID) {
+// Tiles of this warp in one operator.  Whole items (ksplit == 1): the warp that owns the rows finishes
+// them (lane r = unit r).  Split items: the partial sum of every tile goes to shared memory.
+template <int NR>
+__device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkPhase *s_ph, const int2 *s_rng, const MkPhase &P, int it0,
+                                              int n_tiles, WarpStream &ws, const float4 *xsA, const float4 *xsB,
+                                              volatile int *abort_flag, ItemCtx &cx, float *s_partial, int warp, int lane) {
+    for (int j = warp; j < n_tiles; j += MK_NW) {
+        float y[NR];
+        if (!consume_tile<NR>(p, s_ph, s_rng, P, j & (P.ksplit - 1), ws, xsA, xsB, abort_flag, y, warp, lane)) return false;
+        if (P.split) {
 #pragma unroll
-        for (int r = 0; r < NR; ++r)
-            if (lane == r && u0 + r < P.units_total) P.out[u0 + r] = __ldcg(P.out + u0 + r) + acc[r];
-    } else if (P.kind == PH_LMHEAD) {
+            for (int r = 0; r < NR; ++r)
+                if (lane == r) s_partial[j * NR + r] = y[r];
+        } else {
+            const int u0 = (it0 + j) * P.rw;
+            constexpr int NU = NR >= 2 ? NR / 2 : 1;
+            if (P.kind == PH_QKV || P.kind == PH_SWIGLU) {
+                if constexpr (NR >= 2) {
 #pragma unroll
-        for (int r = 0; r < NR; ++r)
-            if (lane == r && u0 + r < P.units_total) {
-                if (cx.logits_out) cx.logits_out[u0 + r] = acc[r];
-                if (arg_better(acc[r], u0 + r, cx.best_v, cx.best_i)) { cx.best_v = acc[r]; cx.best_i = u0 + r; }
-            }
-    } else if constexpr (NR >= 2) {
-        constexpr int RWP = NR / 2;  // pairs in the tile: low rows [0, RWP), partner rows [RWP, NR)
-#pragma unroll
-        for (int r = 0; r < RWP; ++r) {
-            if (lane == r && u0 + r < P.units_total) {
-                float lo = acc[r], hi = acc[r + RWP];
-                if (P.kind == PH_SWIGLU) {
-                    P.out[u0 + r] = lo / (1.f + expf(-lo)) * hi;
-                } else {  // PH_QKV
-                    const int half = p.d >> 1;
-                    const int u = u0 + r;
-                    const int head = u / half, i = u - head * half;
-                    const int row_lo = head * p.d + i, row_hi = row_lo + half;
-                    if (P.bias) { lo += bf16_bits_to_f32(P.bias[row_lo]); hi += bf16_bits_to_f32(P.bias[row_hi]); }
-                    const size_t layer_off = static_cast<size_t>(P.layer) * p.nkv * p.max_context * p.d;
-                    if (head < p.nq + p.nkv) {
-                        const float c = cx.rope[i], sn = cx.rope[half + i];
-                        const float rlo = lo * c - hi * sn, rhi = hi * c + lo * sn;
-                        if (head < p.nq) {
-                            P.out[row_lo] = rlo;
-                            P.out[row_hi] = rhi;
-                        } else {
-                            uint16_t *dst = p.k_cache + layer_off + (static_cast<size_t>(head - p.nq) * p.max_context + cx.slot_row) * p.d;
-                            dst[i] = f32_to_bf16_bits(rlo);
-                            dst[i + half] = f32_to_bf16_bits(rhi);
-                        }
-                    } else {
-                        uint16_t *dst = p.v_cache + layer_off + (static_cast<size_t>(head - p.nq - p.nkv) * p.max_context + cx.slot_row) * p.d;
-                        dst[i] = f32_to_bf16_bits(lo);
-                        dst[i + half] = f32_to_bf16_bits(hi);
-                    }
+                    for (int r = 0; r < NU; ++r)
+                        if (lane == r && u0 + r < P.units_total) apply_epilogue(p, P, cx, u0 + r, y[r] * cx.rscale, y[r + NU] * cx.rscale);
                 }
+            } else {
+#pragma unroll
+                for (int r = 0; r < NR; ++r)
+                    if (lane == r && u0 + r < P.units_total) apply_epilogue(p, P, cx, u0 + r, y[r] * cx.rscale, 0.f);
             }
         }
     }
     return true;
 }
 
-// One weight-streaming operator on the consumer warps: prologue (stage the activation vector, RMSNorm
-// folded in: x*w is staged and the scalar rsqrt(mean x^2 + eps) is applied to the dot products), items.
-__device__ __forceinline__ bool gemv_phase(const MkParams &p, const MkPhase &P, unsigned &tile_no, float4 *xsA, float4 *xsB,
-                                           const unsigned char *ring, unsigned long long *full_bar, unsigned long long *empty_bar,
-                                           volatile int *abort_flag, float *s_part, ItemCtx &cx, int token, int tidc, int &prof_idx) {
-    const int lane = tidc & 31, warp = tidc >> 5;
-    const int cta = blockIdx.x, ncta = gridDim.x;
+// Attention chunking shared by the attention phase and by the consumer of its partial results.
+__device__ __forceinline__ void att_chunking(const MkParams &p, int n, int hg, int min_chunk, int ncta, int &nch, int &chunk_len) {
+    const int groups = p.nq / hg;
+    nch = (n + min_chunk - 1) / min_chunk;
+    nch = min(nch, min(ncta / groups, p.max_chunks));
+    if (hg == 1) nch = min(nch, MK_ATT_SPLIT_MAXC);
+    nch = max(nch, 1);
+    chunk_len = (n + nch - 1) / nch;
+    chunk_len = (chunk_len + MK_ATT_TILE - 1) / MK_ATT_TILE * MK_ATT_TILE;
+    nch = (n + chunk_len - 1) / chunk_len;
+}
+
+// One weight-streaming operator: prologue (stage the activation vector, RMSNorm folded in: x*w is staged
+// and the scalar rsqrt(mean x^2 + eps) is applied to the dot products), then this warp's tiles.
+// merge_attn > 0: the input is the attention output, still split into merge_attn chunk partials per head
+// (m, l, unnormalised o); the exact log-sum-exp merge is done here, in chunk order, by every CTA.
+__device__ __forceinline__ bool gemv_phase(const MkParams &p, const MkPhase *s_ph, const int2 *s_rng, int ph, WarpStream &ws, float4 *xsA,
+                                           float4 *xsB, volatile int *abort_flag, float *s_part, float *s_partial, ItemCtx &cx, int token,
+                                           int merge_attn, int tid, int &prof_idx) {
+    const MkPhase &P = s_ph[ph];
+    const int lane = tid & 31, warp = tid >> 5;
+    const int cta = blockIdx.x;
     const int n4 = P.K >> 2;
     float ss = 0.f;
-    constexpr int PU = 4;  // loads in flight per thread
-    for (int base = tidc; base < n4; base += MK_NTC * PU) {
-        float4 v[PU];
-        uint2 w[PU];
+    if (merge_attn > 0) {
+        const int nch = merge_attn;
+        const int d4 = p.d >> 2;
+        float *sm_m = s_partial;                 // [nq][nch] chunk maxima
+        float *sm_l = s_partial + p.nq * nch;    // [nq][nch] chunk denominators
+        float4 ob[MK_ATT_SPLIT_MAXC];
+        auto load_partials = [&](int o4) {
+            const int h = o4 / d4, j4 = o4 - h * d4;
+            const float4 *po = reinterpret_cast<const float4 *>(p.part_o + static_cast<size_t>(h) * p.max_chunks * p.d) + j4;
 #pragma unroll
-        for (int u = 0; u < PU; ++u) {
-            const int i4 = base + u * MK_NTC;
-            if (i4 < n4) {
-                if (P.x_src) {
-                    v[u] = __ldcg(reinterpret_cast<const float4 *>(P.x_src) + i4);
-                } else {  // first operator of the step: the embedding row is the residual stream
-                    const uint2 e = *reinterpret_cast<const uint2 *>(p.embed + static_cast<size_t>(token) * p.H + i4 * 4);
-                    v[u] = make_float4(bf16lo(e.x), bf16hi(e.x), bf16lo(e.y), bf16hi(e.y));
-                }
-                if (P.norm_w) w[u] = *reinterpret_cast<const uint2 *>(P.norm_w + i4 * 4);
-            }
+            for (int c = 0; c < MK_ATT_SPLIT_MAXC; ++c)
+                if (c < nch) ob[c] = __ldcg(po + static_cast<size_t>(c) * d4);
+        };
+        if (tid < n4) load_partials(tid);        // issued before the statistics are waited for
+        for (int i = tid; i < p.nq * nch; i += MK_NT) {
+            const int h = i / nch, c = i - h * nch;
+            sm_m[i] = __ldcg(p.part_m + h * p.max_chunks + c);
+            sm_l[i] = __ldcg(p.part_l + h * p.max_chunks + c);
         }
+        cta_sync();
+        for (int o4 = tid; o4 < n4; o4 += MK_NT) {
+            if (o4 != tid) load_partials(o4);
+            const int h = o4 / d4;
+            const float *hm = sm_m + h * nch, *hl = sm_l + h * nch;
+            float mm = -INFINITY;
+            for (int c = 0; c < nch; ++c) mm = fmaxf(mm, hm[c]);
+            float ll = 0.f;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int u = 0; u < PU; ++u) {
-            const int i4 = base + u * MK_NTC;
-            if (i4 < n4) {
-                float4 t = v[u];
-                if (!P.x_src && cta == 0) reinterpret_cast<float4 *>(p.x)[i4] = t;
-                if (P.norm_w) {
-                    ss = fmaf(t.x, t.x, ss); ss = fmaf(t.y, t.y, ss); ss = fmaf(t.z, t.z, ss); ss = fmaf(t.w, t.w, ss);
-                    t.x *= bf16lo(w[u].x); t.y *= bf16hi(w[u].x); t.z *= bf16lo(w[u].y); t.w *= bf16hi(w[u].y);
+            for (int c = 0; c < MK_ATT_SPLIT_MAXC; ++c) {
+                if (c < nch) {
+                    const float e = __expf(hm[c] - mm);
+                    ll = fmaf(hl[c], e, ll);
+                    acc.x = fmaf(ob[c].x, e, acc.x); acc.y = fmaf(ob[c].y, e, acc.y);
+                    acc.z = fmaf(ob[c].z, e, acc.z); acc.w = fmaf(ob[c].w, e, acc.w);
                 }
-                if (i4 & 1) xsB[i4 >> 1] = t; else xsA[i4 >> 1] = t;
+            }
+            const float inv = 1.f / ll;
+            acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+            if (o4 & 1) xsB[o4 >> 1] = acc; else xsA[o4 >> 1] = acc;
+        }
+    } else {
+        constexpr int PU = 4;  // loads in flight per thread
+        for (int base = tid; base < n4; base += MK_NT * PU) {
+            float4 v[PU];
+            uint2 w[PU];
+#pragma unroll
+            for (int u = 0; u < PU; ++u) {
+                const int i4 = base + u * MK_NT;
+                if (i4 < n4) {
+                    if (P.x_src) {
+                        v[u] = __ldcg(reinterpret_cast<const float4 *>(P.x_src) + i4);
+                    } else {  // first operator of the step: the embedding row is the residual stream
+                        const uint2 e = *reinterpret_cast<const uint2 *>(p.embed + static_cast<size_t>(token) * p.H + i4 * 4);
+                        v[u] = make_float4(bf16lo(e.x), bf16hi(e.x), bf16lo(e.y), bf16hi(e.y));
+                    }
+                    if (P.norm_w) w[u] = *reinterpret_cast<const uint2 *>(P.norm_w + i4 * 4);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < PU; ++u) {
+                const int i4 = base + u * MK_NT;
+                if (i4 < n4) {
+                    float4 t = v[u];
+                    if (!P.x_src && cta == 0) reinterpret_cast<float4 *>(p.x)[i4] = t;
+                    if (P.norm_w) {
+                        ss = fmaf(t.x, t.x, ss); ss = fmaf(t.y, t.y, ss); ss = fmaf(t.z, t.z, ss); ss = fmaf(t.w, t.w, ss);
+                        t.x *= bf16lo(w[u].x); t.y *= bf16hi(w[u].x); t.z *= bf16lo(w[u].y); t.w *= bf16hi(w[u].y);
+                    }
+                    if (i4 & 1) xsB[i4 >> 1] = t; else xsA[i4 >> 1] = t;
+                }
             }
         }
     }
@@ -408,77 +501,97 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, const MkPhase &P, 
         ss = warp_sum(ss);
         if (lane == 0) s_part[warp] = ss;
     }
-    consumer_sync();
-    prof_stamp(p, tidc, prof_idx);   // activation vector staged
+    cta_sync();
+    prof_stamp(p, tid, prof_idx);   // activation vector staged
     cx.rscale = 1.f;
     if (P.norm_w) {
         float tot = 0.f;
 #pragma unroll
-        for (int w = 0; w < MK_NWC; ++w) tot += s_part[w];
+        for (int w = 0; w < MK_NW; ++w) tot += s_part[w];
         cx.rscale = rsqrtf(tot / static_cast<float>(P.K) + p.eps);
     }
-    int it0, it1;
-    item_range(P.items_total, cta, ncta, it0, it1);
-    const int nr = (P.kind == PH_QKV || P.kind == PH_SWIGLU) ? 2 * P.rw : P.rw;
-    bool ok = true;
-    for (int i = warp; i < it1 - it0 && ok; i += MK_NWC) {
-        switch (nr) {
-            case 1: ok = consume_item<1>(p, P, it0 + i, tile_no, xsA, xsB, ring, full_bar, empty_bar, abort_flag, cx, lane); break;
-            case 2: ok = consume_item<2>(p, P, it0 + i, tile_no, xsA, xsB, ring, full_bar, empty_bar, abort_flag, cx, lane); break;
-            case 4: ok = consume_item<4>(p, P, it0 + i, tile_no, xsA, xsB, ring, full_bar, empty_bar, abort_flag, cx, lane); break;
-            default: ok = consume_item<8>(p, P, it0 + i, tile_no, xsA, xsB, ring, full_bar, empty_bar, abort_flag, cx, lane); break;
+    const int2 rng = s_rng[ph];
+    const int n_items = rng.y - rng.x;
+    const int n_tiles = n_items << P.s_shift;
+    const bool paired = P.kind == PH_QKV || P.kind == PH_SWIGLU;
+    const int nr = paired ? 2 * P.rw : P.rw;
+    bool ok;
+    switch (nr) {
+        case 1: ok = consume_tiles<1>(p, s_ph, s_rng, P, rng.x, n_tiles, ws, xsA, xsB, abort_flag, cx, s_partial, warp, lane); break;
+        case 2: ok = consume_tiles<2>(p, s_ph, s_rng, P, rng.x, n_tiles, ws, xsA, xsB, abort_flag, cx, s_partial, warp, lane); break;
+        case 4: ok = consume_tiles<4>(p, s_ph, s_rng, P, rng.x, n_tiles, ws, xsA, xsB, abort_flag, cx, s_partial, warp, lane); break;
+        default: ok = consume_tiles<8>(p, s_ph, s_rng, P, rng.x, n_tiles, ws, xsA, xsB, abort_flag, cx, s_partial, warp, lane); break;
+    }
+    if (P.split) {
+        // partial sums of the K slices meet here; thread u finishes unit u of this CTA (rw == 1), slices in order
+        cta_sync();
+        if (!*abort_flag) {
+            for (int u = tid; u < n_items; u += MK_NT) {
+                float lo = 0.f, hi = 0.f;
+                for (int sl = 0; sl < P.ksplit; ++sl) {
+                    const int j = (u << P.s_shift) + sl;
+                    if (paired) { lo += s_partial[2 * j]; hi += s_partial[2 * j + 1]; } else { lo += s_partial[j]; }
+                }
+                apply_epilogue(p, P, cx, rng.x + u, lo * cx.rscale, hi * cx.rscale);
+            }
         }
     }
     return ok;
 }
 
-// ---- attention on the consumer warps ------------------------------------------------------------------
-// CTA (g, c) = chunk c of kv head g; all G query heads of the group share each K/V row read.
+// ---- attention -----------------------------------------------------------------------------------------------
+// A CTA serves HG query heads of one GQA group over one chunk of the cached positions: HG = G (the whole
+// group shares every K/V row read: least traffic, for long contexts) or HG = 1 (every query head has
+// its own CTAs: G times more parallelism for short, latency-bound contexts; K/V re-reads hit L2).
 // Scores: MK_ATT_LPP lanes per position, each lane reads interleaved 16-byte pieces of the K row from
 // global memory; P V: every lane owns d/32 dims.  Shared memory (the idle activation buffer): q,
-// probabilities, warp merge area, chunk statistics.
-template <int D, int G>
-__device__ __forceinline__ void attention_phase(const MkParams &p, int layer, int n, unsigned char *xbuf, int tidc, int *s_flag) {
+// probabilities, warp merge area, chunk statistics.  The CTA that arrives last for its head group
+// (atomic ticket, no waiting) merges the chunks exactly:  m = max m_c, l = sum l_c e^{m_c - m},
+// o = sum o_c e^{m_c - m} / l, in index order.
+template <int D, int HG>
+__device__ __forceinline__ void attention_phase(const MkParams &p, int layer, int n, int min_chunk, bool defer_merge,
+                                                unsigned char *xbuf, int tid, int *s_flag) {
     constexpr int TILE = MK_ATT_TILE, LPP = MK_ATT_LPP;
     constexpr int DV = D / 32, CPR = D / 8, CPL = CPR / LPP;
-    const int lane = tidc & 31, warp = tidc >> 5;
-    const int cta = blockIdx.x;
-    int nch = (n + p.att_min_chunk - 1) / p.att_min_chunk;
-    nch = min(nch, p.max_chunks);
-    int chunk_len = (n + nch - 1) / nch;
-    chunk_len = (chunk_len + TILE - 1) / TILE * TILE;
-    nch = (n + chunk_len - 1) / chunk_len;
-    if (cta >= nch * p.nkv) return;
-    const int g = cta / nch, c = cta - g * nch;
+    constexpr int MW = MK_ATT_MW;
+    const int lane = tid & 31, warp = tid >> 5;
+    const int cta = blockIdx.x, ncta = gridDim.x;
+    const int G = p.nq / p.nkv;
+    const int groups = p.nq / HG;                       // head groups served by separate CTAs
+    int nch, chunk_len;
+    att_chunking(p, n, HG, min_chunk, ncta, nch, chunk_len);
+    if (cta >= nch * groups) return;
+    const int grp = cta / nch, c = cta - grp * nch;
+    const int qh0 = grp * HG;                            // first query head of this CTA
+    const int g = qh0 / G;                               // its kv head
     const int t0 = c * chunk_len, t1 = min(n, t0 + chunk_len);
 
-    float *qs = reinterpret_cast<float *>(xbuf);               // [G][D]
-    float *ps = qs + G * D;                                     // [NWC][G][TILE]
-    constexpr int MW = MK_ATT_MW;
-    float *mg_m = ps + MK_NWC * G * TILE;                       // [MW][G]
-    float *mg_l = mg_m + MW * G;                                // [MW][G]
-    float *mg_o = mg_l + MW * G;                                // [MW][G][D]
-    float *cm = mg_o + MW * G * D;                              // [G][max_chunks] chunk maxima
-    float *cl = cm + G * p.max_chunks;                          // [G][max_chunks] chunk denominators
+    float *qs = reinterpret_cast<float *>(xbuf);               // [HG][D]
+    float *ps = qs + HG * D;                                    // [NW][HG][TILE]
+    float *mg_m = ps + MK_NW * HG * TILE;                       // [MW][HG]
+    float *mg_l = mg_m + MW * HG;                               // [MW][HG]
+    float *mg_o = mg_l + MW * HG;                               // [MW][HG][D]
+    float *cm = mg_o + MW * HG * D;                             // [HG][max_chunks] chunk maxima
+    float *cl = cm + HG * p.max_chunks;                         // [HG][max_chunks] chunk denominators
 
-    for (int i = tidc; i < G * D; i += MK_NTC) qs[i] = __ldcg(p.q + static_cast<size_t>(g) * G * D + i) * p.scale;
-    consumer_sync();
+    for (int i = tid; i < HG * D; i += MK_NT) qs[i] = __ldcg(p.q + static_cast<size_t>(qh0) * D + i) * p.scale;
+    cta_sync();
 
     const size_t head_off = (static_cast<size_t>(layer) * p.nkv + g) * p.max_context * D;
     const uint16_t *kg = p.k_cache + head_off;
     const uint16_t *vg = p.v_cache + head_off;
-    float *pw = ps + warp * (G * TILE);
+    float *pw = ps + warp * (HG * TILE);
     const int pi = lane / LPP, part = lane % LPP;
 
-    float m[G], l[G], o[G][DV];
+    float m[HG], l[HG], o[HG][DV];
 #pragma unroll
-    for (int h = 0; h < G; ++h) {
+    for (int h = 0; h < HG; ++h) {
         m[h] = -INFINITY; l[h] = 0.f;
 #pragma unroll
         for (int e = 0; e < DV; ++e) o[h][e] = 0.f;
     }
 
-    for (int tt = t0 + warp * TILE; tt < t1; tt += MK_NWC * TILE) {
+    for (int tt = t0 + warp * TILE; tt < t1; tt += MK_NW * TILE) {
         const bool pvalid = tt + pi < t1;
         uint4 kk[CPL];
 #pragma unroll
@@ -498,21 +611,21 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
                 vraw[x][0] = t < t1 ? __ldcg(reinterpret_cast<const unsigned *>(vp)) : 0u;
             }
         }
-        float s[G];
+        float s[HG];
 #pragma unroll
-        for (int h = 0; h < G; ++h) s[h] = 0.f;
+        for (int h = 0; h < HG; ++h) s[h] = 0.f;
 #pragma unroll
         for (int j = 0; j < CPL; ++j) {
             const int cc = j * LPP + part;
 #pragma unroll
-            for (int h = 0; h < G; ++h) {
+            for (int h = 0; h < HG; ++h) {
                 const float4 q0 = *reinterpret_cast<const float4 *>(qs + h * D + cc * 8);
                 const float4 q1 = *reinterpret_cast<const float4 *>(qs + h * D + cc * 8 + 4);
                 s[h] = dot8(kk[j], q0, q1, s[h]);
             }
         }
 #pragma unroll
-        for (int h = 0; h < G; ++h) {
+        for (int h = 0; h < HG; ++h) {
 #pragma unroll
             for (int x = 1; x < LPP; x <<= 1) s[h] += __shfl_xor_sync(0xffffffffu, s[h], x);
             if (!pvalid) s[h] = -INFINITY;
@@ -538,7 +651,7 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
                 }
             }
 #pragma unroll
-            for (int h = 0; h < G; ++h) {
+            for (int h = 0; h < HG; ++h) {
                 const float4 p4 = *reinterpret_cast<const float4 *>(pw + h * TILE + tb);
 #pragma unroll
                 for (int e = 0; e < DV; ++e) {
@@ -554,87 +667,86 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
 
     // merge the warps of the CTA in two passes through a merge area of MW entries (idle warps carry
     // m = -inf and weigh 0): upper warps publish, lower warps fold them in, then publish themselves.
-    float lt[G];
+    float lt[HG];
 #pragma unroll
-    for (int h = 0; h < G; ++h) lt[h] = warp_sum(l[h]);
+    for (int h = 0; h < HG; ++h) lt[h] = warp_sum(l[h]);
     if (warp >= MW) {
         const int u = warp - MW;
 #pragma unroll
-        for (int h = 0; h < G; ++h) {
-            if (lane == 0) { mg_m[u * G + h] = m[h]; mg_l[u * G + h] = lt[h]; }
+        for (int h = 0; h < HG; ++h) {
+            if (lane == 0) { mg_m[u * HG + h] = m[h]; mg_l[u * HG + h] = lt[h]; }
 #pragma unroll
-            for (int e = 0; e < DV; ++e) mg_o[(u * G + h) * D + lane * DV + e] = o[h][e];
+            for (int e = 0; e < DV; ++e) mg_o[(u * HG + h) * D + lane * DV + e] = o[h][e];
         }
     }
-    consumer_sync();
-    if (warp < MK_NWC - MW) {
+    cta_sync();
+    if (warp < MK_NW - MW) {
 #pragma unroll
-        for (int h = 0; h < G; ++h) {
-            const float m2 = mg_m[warp * G + h], l2 = mg_l[warp * G + h];
+        for (int h = 0; h < HG; ++h) {
+            const float m2 = mg_m[warp * HG + h], l2 = mg_l[warp * HG + h];
             const float mn = fmaxf(m[h], m2);
             const float e1 = m[h] == mn ? 1.f : __expf(m[h] - mn);
             const float e2 = m2 == mn ? 1.f : __expf(m2 - mn);
             lt[h] = lt[h] * e1 + l2 * e2;
 #pragma unroll
-            for (int e = 0; e < DV; ++e) o[h][e] = o[h][e] * e1 + mg_o[(warp * G + h) * D + lane * DV + e] * e2;
+            for (int e = 0; e < DV; ++e) o[h][e] = o[h][e] * e1 + mg_o[(warp * HG + h) * D + lane * DV + e] * e2;
             m[h] = mn;
         }
     }
-    consumer_sync();
+    cta_sync();
     if (warp < MW) {
 #pragma unroll
-        for (int h = 0; h < G; ++h) {
-            if (lane == 0) { mg_m[warp * G + h] = m[h]; mg_l[warp * G + h] = lt[h]; }
+        for (int h = 0; h < HG; ++h) {
+            if (lane == 0) { mg_m[warp * HG + h] = m[h]; mg_l[warp * HG + h] = lt[h]; }
 #pragma unroll
-            for (int e = 0; e < DV; ++e) mg_o[(warp * G + h) * D + lane * DV + e] = o[h][e];
+            for (int e = 0; e < DV; ++e) mg_o[(warp * HG + h) * D + lane * DV + e] = o[h][e];
         }
     }
-    consumer_sync();
-    for (int i = tidc; i < G * D; i += MK_NTC) {
+    cta_sync();
+    for (int i = tid; i < HG * D; i += MK_NT) {
         const int h = i / D, j = i - h * D;
         float mm = -INFINITY;
 #pragma unroll
-        for (int w = 0; w < MW; ++w) mm = fmaxf(mm, mg_m[w * G + h]);
+        for (int w = 0; w < MW; ++w) mm = fmaxf(mm, mg_m[w * HG + h]);
         float ll = 0.f, oo = 0.f;
 #pragma unroll
         for (int w = 0; w < MW; ++w) {
-            const float e = __expf(mg_m[w * G + h] - mm);
-            ll = fmaf(mg_l[w * G + h], e, ll);
-            oo = fmaf(mg_o[(w * G + h) * D + j], e, oo);
+            const float e = __expf(mg_m[w * HG + h] - mm);
+            ll = fmaf(mg_l[w * HG + h], e, ll);
+            oo = fmaf(mg_o[(w * HG + h) * D + j], e, oo);
         }
-        const int qh = g * G + h;
-        if (nch == 1) {  // nothing to merge across CTAs
+        const int qh = qh0 + h;
+        if (nch == 1 && !defer_merge) {  // nothing to merge across CTAs
             p.attn[qh * D + j] = oo / ll;
         } else {
             p.part_o[(static_cast<size_t>(qh) * p.max_chunks + c) * D + j] = oo;
             if (j == 0) { p.part_m[qh * p.max_chunks + c] = mm; p.part_l[qh * p.max_chunks + c] = ll; }
         }
     }
-    if (nch == 1) return;
+    if (nch == 1 || defer_merge) return;   // deferred: the next operator's prologue merges the chunks
     __threadfence();
-    consumer_sync();
-    if (tidc == 0) *s_flag = (atomicAdd(p.tickets + g, 1u) == static_cast<unsigned>(nch - 1)) ? 1 : 0;
-    consumer_sync();
+    cta_sync();
+    if (tid == 0) *s_flag = (atomicAdd(p.tickets + grp, 1u) == static_cast<unsigned>(nch - 1)) ? 1 : 0;
+    cta_sync();
     if (!*s_flag) return;
 
-    // Last CTA of this kv head: exact log-sum-exp merge of the chunks, in index order.  All loads of a
-    // batch (chunk statistics and up to CB partial vectors per thread) are issued before any is used.
+    // Last CTA of this head group: merge the chunks.  All loads of a batch (chunk statistics and up to
+    // CB partial vectors per thread) are issued before any is used.
     __threadfence();
     constexpr int CB = 8;
-    const int i0 = tidc;                       // output (h, j4) of this thread, if any
-    const bool has_out = i0 < G * D / 4;
-    const int oh = has_out ? i0 / (D / 4) : 0, oj4 = has_out ? i0 - oh * (D / 4) : 0;
-    const float4 *po = reinterpret_cast<const float4 *>(p.part_o + static_cast<size_t>(g * G + oh) * p.max_chunks * D) + oj4;
+    const bool has_out = tid < HG * D / 4;       // output (h, j4) of this thread, if any
+    const int oh = has_out ? tid / (D / 4) : 0, oj4 = has_out ? tid - oh * (D / 4) : 0;
+    const float4 *po = reinterpret_cast<const float4 *>(p.part_o + static_cast<size_t>(qh0 + oh) * p.max_chunks * D) + oj4;
     float4 ob[CB];
 #pragma unroll
     for (int u = 0; u < CB; ++u)
         ob[u] = (has_out && u < nch) ? __ldcg(po + static_cast<size_t>(u) * (D / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int i = tidc; i < G * nch; i += MK_NTC) {
+    for (int i = tid; i < HG * nch; i += MK_NT) {
         const int h = i / nch, cc = i - h * nch;
-        cm[h * p.max_chunks + cc] = __ldcg(p.part_m + (g * G + h) * p.max_chunks + cc);
-        cl[h * p.max_chunks + cc] = __ldcg(p.part_l + (g * G + h) * p.max_chunks + cc);
+        cm[h * p.max_chunks + cc] = __ldcg(p.part_m + (qh0 + h) * p.max_chunks + cc);
+        cl[h * p.max_chunks + cc] = __ldcg(p.part_l + (qh0 + h) * p.max_chunks + cc);
     }
-    consumer_sync();
+    cta_sync();
     if (has_out) {
         const float *hm = cm + oh * p.max_chunks, *hl = cl + oh * p.max_chunks;
         float mm = -INFINITY;
@@ -659,93 +771,120 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
         }
         const float inv = 1.f / ll;
         acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-        reinterpret_cast<float4 *>(p.attn + (g * G + oh) * D)[oj4] = acc;
+        reinterpret_cast<float4 *>(p.attn + (qh0 + oh) * D)[oj4] = acc;
     }
-    if (tidc == 0) p.tickets[g] = 0u;
+    if (tid == 0) p.tickets[grp] = 0u;
 }
 
 // ---- the kernel -----------------------------------------------------------------------------------------------
 template <int D, int G>
-__global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParams p) {
+__global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) {
     extern __shared__ __align__(128) unsigned char mk_smem[];
     unsigned char *smem = mk_smem;
     float4 *xsA = reinterpret_cast<float4 *>(smem);
     float4 *xsB = reinterpret_cast<float4 *>(smem + p.xbuf_bytes / 2);
     MkPhase *s_ph = reinterpret_cast<MkPhase *>(smem + p.xbuf_bytes);          // the step's schedule
+    int2 *s_rng = reinterpret_cast<int2 *>(s_ph + p.nph);                      // this CTA's item range per operator
     unsigned char *ring = smem + p.xbuf_bytes + p.sched_bytes;
-    __shared__ __align__(8) unsigned long long full_bar[MK_MAX_SLOTS];
-    __shared__ __align__(8) unsigned long long empty_bar[MK_MAX_SLOTS];
+    __shared__ __align__(8) unsigned long long full_bar[MK_NW * MK_MAX_DEPTH];
     __shared__ float s_rope[128];
-    __shared__ float s_part[MK_NWC];
-    __shared__ float s_bv[MK_NWC];
-    __shared__ int s_bi[MK_NWC];
+    __shared__ float s_part[MK_NW];
+    __shared__ float s_partial[MK_PARTIAL_FLOATS];
+    __shared__ float s_bv[MK_NW];
+    __shared__ int s_bi[MK_NW];
     __shared__ int s_flag;
     __shared__ int s_abort;
 
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int cta = blockIdx.x, ncta = gridDim.x;
     if (tid == 0) {
-        for (int i = 0; i < p.nslot; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], 1); }
+        for (int i = 0; i < MK_NW * p.depth; ++i) mbar_init(&full_bar[i], 1);
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     {
-        const int n16 = (4 * p.n_layers + 1) * static_cast<int>(sizeof(MkPhase) / 16);
+        const int n16 = p.nph * static_cast<int>(sizeof(MkPhase) / 16);
         const uint4 *src = reinterpret_cast<const uint4 *>(p.phases);
         uint4 *dst = reinterpret_cast<uint4 *>(s_ph);
-        for (int i = tid; i < n16; i += MK_THREADS) dst[i] = src[i];
+        for (int i = tid; i < n16; i += MK_NT) dst[i] = src[i];
+        for (int i = tid; i < p.nph; i += MK_NT) {
+            int it0, it1;
+            item_range(p.phases[i].items_total, cta, ncta, it0, it1);
+            s_rng[i] = make_int2(it0, it1);
+        }
     }
     __syncthreads();
     volatile int *abort_flag = &s_abort;
 
-    if (tid >= MK_NTC) {  // ---- producer warp ----
-        producer_loop(p, s_ph, ring, full_bar, empty_bar, abort_flag, tid - MK_NTC);
-        return;
+    // ---- start this warp's weight stream: fill its ring, then run the L2 prefetch ahead ---------------
+    WarpStream ws;
+    ws.consumed = 0; ws.issued = 0;
+    ws.slots = ring + static_cast<size_t>(warp) * p.depth * p.slot_bytes;
+    ws.bars = &full_bar[warp * p.depth];
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(ws.policy));
+    ws.pf.ph = 0;
+    cursor_enter_phase(ws.pf, p, s_ph, s_rng, warp);
+    bool ok = true;
+    for (int q = 0; q < p.depth && ok && ws.pf.ph < p.nph; ++q) {
+        ok = issue_tile(p, s_ph, ws.pf, ws.slots + static_cast<size_t>(q) * p.slot_bytes, &ws.bars[q], ws.policy, abort_flag, lane);
+        ++ws.issued;
+        cursor_advance(ws.pf, p, s_ph, s_rng, warp);
     }
-
-    // ---- consumer warps ----
-    const int tidc = tid, lane = tid & 31, warp = tid >> 5;
-    const int cta = blockIdx.x, ncta = gridDim.x;
     const int rt = p.req->token, rp = p.req->position;
     const int token = rt >= 0 ? rt : p.state->next_token;
     const int pos = rp >= 0 ? rp : p.state->next_position;
     const int slot_row = p.state->cur_len;
     const int half = p.d >> 1;
-    if (tidc < half) {  // rotary table of this step's position; fp64 angle, rounded once
-        double sn, cs;
-        sincos(static_cast<double>(pos) * p.inv_freq[tidc], &sn, &cs);
-        s_rope[tidc] = static_cast<float>(cs);
-        s_rope[half + tidc] = static_cast<float>(sn);
-    }
     if (token < 0 || token >= p.V || slot_row < 0 || slot_row >= p.max_context || pos < 0) {
-        if (tidc == 0) diag_fail(p, abort_flag, 3, token, slot_row);   // corrupt request/state: touch nothing
-        return;
+        if (tid == 0) diag_fail(p, abort_flag, 3, token, slot_row);   // corrupt request/state: compute nothing
+        ok = false;
     }
-    if (cta == 0 && tidc == 0) { p.state->token = token; p.state->position = pos; }
-    // (s_rope is published by the consumer_sync of the first prologue)
+    if (ok && tid < half) {  // rotary table of this step's position; fp64 angle, rounded once
+        double sn, cs;
+        sincos(static_cast<double>(pos) * p.inv_freq[tid], &sn, &cs);
+        s_rope[tid] = static_cast<float>(cs);
+        s_rope[half + tid] = static_cast<float>(sn);
+    }
+    if (ok && cta == 0 && tid == 0) { p.state->token = token; p.state->position = pos; }
+    // (s_rope is published by the __syncthreads of the first prologue)
 
     ItemCtx cx;
     cx.rscale = 1.f; cx.slot_row = slot_row; cx.rope = s_rope; cx.best_v = -INFINITY; cx.best_i = 0x7fffffff;
     cx.logits_out = p.req->logits_out;
-    cx.warp = static_cast<unsigned>(warp);
 
-    unsigned tile_no = 0, bar_no = 0;   // tile_no: tiles this warp has consumed so far
+    unsigned bar_no = 0;
     int prof_idx = 0;
-    prof_stamp(p, tidc, prof_idx);
-    bool ok = true;
+    prof_stamp(p, tid, prof_idx);
+    const int n_att = slot_row + 1;
+    const bool att_split = n_att <= p.att_split_max_n && static_cast<long long>(p.nq) * MK_ATT_SPLIT_MAXC * 2 <= MK_PARTIAL_FLOATS;
+    int merge_chunks = 0;   // chunks per head the O-projection prologue has to merge (split mode)
+    if (att_split) { int cl; att_chunking(p, n_att, 1, p.att_chunk_split, ncta, merge_chunks, cl); }
     for (int l = 0; l < p.n_layers && ok; ++l) {
-        ok = gemv_phase(p, s_ph[4 * l], tile_no, xsA, xsB, ring, full_bar, empty_bar, abort_flag, s_part, cx, token, tidc, prof_idx);
-        ok = grid_barrier(p, ++bar_no * ncta, abort_flag, tidc, prof_idx) && ok;
-        if (ok) attention_phase<D, G>(p, l, slot_row + 1, smem, tidc, &s_flag);
-        ok = grid_barrier(p, ++bar_no * ncta, abort_flag, tidc, prof_idx) && ok;
+        ok = gemv_phase(p, s_ph, s_rng, 4 * l, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token, 0, tid, prof_idx);
+        ok = grid_barrier(p, ++bar_no * ncta, abort_flag, tid, prof_idx) && ok;
+        if (ok) {
+            if (att_split) attention_phase<D, 1>(p, l, n_att, p.att_chunk_split, true, smem, tid, &s_flag);
+            else attention_phase<D, G>(p, l, n_att, p.att_chunk_shared, false, smem, tid, &s_flag);
+        }
+        ok = grid_barrier(p, ++bar_no * ncta, abort_flag, tid, prof_idx) && ok;
         for (int k = 1; k < 4 && ok; ++k) {
-            ok = gemv_phase(p, s_ph[4 * l + k], tile_no, xsA, xsB, ring, full_bar, empty_bar, abort_flag, s_part, cx, token, tidc, prof_idx);
-            ok = grid_barrier(p, ++bar_no * ncta, abort_flag, tidc, prof_idx) && ok;
+            ok = gemv_phase(p, s_ph, s_rng, 4 * l + k, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token,
+                            k == 1 ? merge_chunks : 0, tid, prof_idx);
+            ok = grid_barrier(p, ++bar_no * ncta, abort_flag, tid, prof_idx) && ok;
         }
     }
-    if (ok) ok = gemv_phase(p, s_ph[4 * p.n_layers], tile_no, xsA, xsB, ring, full_bar, empty_bar, abort_flag, s_part, cx, token, tidc, prof_idx);
-    prof_stamp(p, tidc, prof_idx);
-    if (!ok) {
-        if (tidc == 0) p.state->status = 6;
+    if (ok) ok = gemv_phase(p, s_ph, s_rng, 4 * p.n_layers, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token, 0, tid, prof_idx);
+    prof_stamp(p, tid, prof_idx);
+    if (!ok || *abort_flag) {
+        // aborted: wait (bounded) for the copies this warp still has in flight, then leave
+        if (tid == 0 && p.state->status == 0) p.state->status = 6;
+        for (unsigned k = ws.consumed; k < ws.issued; ++k) {
+            const unsigned q = k & static_cast<unsigned>(p.depth - 1);
+            const unsigned par = (k >> p.depth_shift) & 1u;
+            const unsigned long long t0 = global_ns();
+            while (!mbar_try_wait(&ws.bars[q], par))
+                if (global_ns() - t0 > p.spin_limit) break;
+        }
         return;
     }
 
@@ -759,16 +898,16 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
         if (arg_better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
     }
     if (lane == 0) { s_bv[warp] = bv; s_bi[warp] = bi; }
-    consumer_sync();
-    if (tidc == 0) {
-        for (int w = 1; w < MK_NWC; ++w)
+    cta_sync();
+    if (tid == 0) {
+        for (int w = 1; w < MK_NW; ++w)
             if (arg_better(s_bv[w], s_bi[w], bv, bi)) { bv = s_bv[w]; bi = s_bi[w]; }
         p.lm_part_val[cta] = bv;
         p.lm_part_idx[cta] = bi;
         __threadfence();
-        s_flag = (atomicAdd(p.tickets + p.nkv, 1u) == static_cast<unsigned>(ncta - 1)) ? 1 : 0;
+        s_flag = (atomicAdd(p.tickets + p.nq, 1u) == static_cast<unsigned>(ncta - 1)) ? 1 : 0;
     }
-    consumer_sync();
+    cta_sync();
     if (!s_flag) return;
     __threadfence();
     if (warp == 0) {
@@ -791,7 +930,7 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
             p.state->next_token = bi;
             p.state->next_position = pos + 1;
             p.state->cur_len = slot_row + 1;
-            p.tickets[p.nkv] = 0u;
+            p.tickets[p.nq] = 0u;
             *p.barrier = 0u;  // every CTA has passed the last grid barrier
         }
     }
