@@ -525,10 +525,10 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
             return bail(EDGEFM_ERR_CUDA, "model shape does not fit the shared-memory plan", cudaErrorInvalidValue);
         const size_t avail = smem_optin - static_smem - xbuf - sched;
         // ring: `depth` slots per warp; prefer two slots of a natural tile size, deeper rings for small tiles
-        int budget = 12288;  // upper bound of one tile = one ring slot
+        int budget = 8192;   // upper bound of one tile
         if (const char *tb = getenv("EDGEFM_TILE_BYTES")) { const int v = atoi(tb); if (v >= 1024 && v <= 65536) budget = v; }
         {
-            const int fit1 = static_cast<int>(avail / MK_NW / 128 * 128);
+            const int fit1 = static_cast<int>(avail / MK_NW / 128 * 128);   // a tile must fit a warp's ring
             if (budget > fit1) budget = fit1;
         }
         int max_tile = 0;
@@ -563,14 +563,12 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
         if (split_overflow || max_tile > budget)
             return bail(EDGEFM_ERR_CUDA, "model shape does not fit the tile plan", cudaErrorInvalidValue);
         const int slot_bytes = (max_tile + 127) / 128 * 128;
-        int depth = static_cast<int>(avail / (static_cast<size_t>(slot_bytes) * MK_NW));
-        if (const char *dp = getenv("EDGEFM_RING_DEPTH")) { const int v = atoi(dp); if (v >= 1 && v < depth) depth = v; }
-        if (depth < 1) return bail(EDGEFM_ERR_CUDA, "weight rows do not fit the shared-memory ring", cudaErrorInvalidValue);
-        depth = depth >= 4 ? 4 : (depth >= 2 ? 2 : 1);   // power of two
-        c->mk.depth = depth; c->mk.depth_shift = depth == 4 ? 2 : (depth == 2 ? 1 : 0);
-        c->mk.slot_bytes = slot_bytes; c->mk.xbuf_bytes = static_cast<int>(xbuf);
+        const int ring_bytes = static_cast<int>(avail / MK_NW / 128 * 128);
+        if (slot_bytes > ring_bytes || ring_bytes > (0xffff << 4))
+            return bail(EDGEFM_ERR_CUDA, "weight rows do not fit the shared-memory ring", cudaErrorInvalidValue);
+        c->mk.ring_bytes = ring_bytes; c->mk.slot_bytes = slot_bytes; c->mk.xbuf_bytes = static_cast<int>(xbuf);
         c->mk.sched_bytes = static_cast<int>(sched);
-        c->mega_smem = xbuf + sched + static_cast<size_t>(depth) * MK_NW * slot_bytes;
+        c->mega_smem = xbuf + sched + static_cast<size_t>(ring_bytes) * MK_NW;
         CREATE_TRY(cudaFuncSetAttribute(c->mega, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(c->mega_smem)));
         int per_sm = 0;
         CREATE_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, c->mega, MK_NT, c->mega_smem));
@@ -638,8 +636,8 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
         const char *pe_ = getenv("EDGEFM_PROFILE");
         if (pe_ && pe_[0] == '1') {
             c->prof_stride = 3 + 14 * sh.n_layers;
-            CREATE_TRY(dev_alloc(&c->prof, static_cast<size_t>(c->mega_grid) * c->prof_stride));
-            CREATE_TRY(cudaMemset(c->prof, 0, static_cast<size_t>(c->mega_grid) * c->prof_stride * 8));
+            CREATE_TRY(dev_alloc(&c->prof, static_cast<size_t>(c->mega_grid + 1) * c->prof_stride + MK_NW * 16));
+            CREATE_TRY(cudaMemset(c->prof, 0, (static_cast<size_t>(c->mega_grid + 1) * c->prof_stride + MK_NW * 16) * 8));
             m.prof = c->prof; m.prof_stride = c->prof_stride;
         }
     }
@@ -736,7 +734,8 @@ edgefm_status edgefm_debug_profile(edgefm_ctx *ctx, uint64_t *out_host, int64_t 
     *n_ctas = ctx->prof ? ctx->mega_grid : 0;
     *stride = ctx->prof_stride;
     if (!ctx->prof || !out_host) return EDGEFM_OK;
-    const int64_t n = static_cast<int64_t>(ctx->mega_grid) * ctx->prof_stride;
+    int64_t n = static_cast<int64_t>(ctx->mega_grid) * ctx->prof_stride;
+    if (capacity >= n + MK_NW * 16) n += MK_NW * 16;   // optional per-warp trace behind the table
     if (capacity < n) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "profile buffer too small");
     DeviceGuard guard(ctx->device);
     CUDA_TRY(ctx, cudaDeviceSynchronize());

@@ -7,14 +7,15 @@
 //   * The step's weight traffic is a static schedule (QKV, O, gate/up, down of every layer, then
 //     lm_head).  Every CTA owns a fixed share of each operator's rows, and every warp of the CTA a fixed
 //     sequence of tiles (a few rows, or one K slice of a long row) across the WHOLE step.
-//   * Each warp keeps a private ring of `depth` shared-memory slots filled with its next tiles by bulk
-//     async copies (TMA: cp.async.bulk + mbarrier complete_tx).  When it has consumed a tile it
-//     immediately re-arms the slot with the tile `depth` ahead -- regardless of operator boundaries.
-//     So HBM keeps streaming while the arithmetic waits at a grid barrier, stages an activation vector
-//     or runs attention.
-//     A slot is armed and drained by the same warp, in program order, so the one-bit mbarrier phase
-//     parity cannot alias and no "empty" barrier is needed (a proxy fence orders the warp's reads before
-//     the next asynchronous write).
+//   * Each warp keeps a private byte ring in shared memory filled with its next tiles (up to MK_MAXF in
+//     flight, variable size, allocated first-in first-out) by bulk async copies (TMA: cp.async.bulk +
+//     mbarrier complete_tx).  When it has consumed a tile it immediately fetches as many further tiles
+//     as now fit -- regardless of operator boundaries -- so the short operators of a layer are already
+//     on chip when their turn comes, and HBM keeps streaming while the arithmetic waits at a grid
+//     barrier, stages an activation vector or runs attention.
+//     Ring space and mbarriers are armed and drained by the same warp, in program order, so the one-bit
+//     mbarrier phase parity cannot alias and no "empty" barrier is needed (a proxy fence orders the
+//     warp's reads before the next asynchronous write).
 //   * A tile is multiplied with the activation vector staged in shared memory; the fused epilogues
 //     (bias + RoPE + KV append, residual add, SwiGLU, logits + argmax) run in the warp that owns the rows.
 //   * Between dependent operators all CTAs meet at a grid barrier (monotonic counter in global memory,
@@ -30,7 +31,7 @@ namespace edgefm {
 
 constexpr int MK_NW = 12;                        // warps per CTA (each streams and consumes its own tiles)
 constexpr int MK_NT = MK_NW * 32;
-constexpr int MK_MAX_DEPTH = 4;                  // ring slots per warp
+constexpr int MK_MAXF = 4;                       // tiles in flight per warp (one mbarrier each)
 constexpr int MK_ATT_LPP = 4;                    // lanes per cached position in the score phase
 constexpr int MK_ATT_TILE = 32 / MK_ATT_LPP;     // positions per warp iteration
 constexpr int MK_ATT_MW = (MK_NW + 1) / 2;       // warps whose partials fit the merge area at once
@@ -82,12 +83,30 @@ struct MkParams {
     int *lm_part_idx;
     StepState *state;
     const StepRequest *req;
-    int depth, depth_shift;        // ring slots per warp (1, 2 or 4) and its log2
-    int slot_bytes, xbuf_bytes, sched_bytes;
+    int ring_bytes;                // shared-memory ring of one warp
+    int slot_bytes;                // largest tile (checked against ring_bytes on the host)
+    int xbuf_bytes, sched_bytes;
     unsigned spin_limit;           // upper bound of every device-side wait, nanoseconds
     unsigned long long *prof;      // optional timestamps [gridDim.x][prof_stride] (diagnostics), or null
     int prof_stride;
 };
+
+// Optional fine-grained trace of one operator in CTA 0 (compile with -DEDGEFM_TRACE_PHASE=<operator index>):
+// lane 0 of every warp appends %globaltimer stamps behind the regular profile table.
+#ifdef EDGEFM_TRACE_PHASE
+#define MK_TRACE(p, ph, warp, lane, slot)                                                                          \
+    do {                                                                                                           \
+        if ((p).prof && (ph) == EDGEFM_TRACE_PHASE && blockIdx.x == 0 && (lane) == 0 && (slot) < 16)               \
+            (p).prof[static_cast<size_t>(gridDim.x) * (p).prof_stride + (warp) * 16 + (slot)] = global_ns_();        \
+    } while (0)
+__device__ __forceinline__ unsigned long long global_ns_() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+#else
+#define MK_TRACE(p, ph, warp, lane, slot) do {} while (0)
+#endif
 
 // ---- mbarrier / bulk copy primitives -----------------------------------------------------------------
 __device__ __forceinline__ unsigned smem_u32(const void *p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
@@ -164,11 +183,15 @@ __device__ __forceinline__ bool diag_fail(const MkParams &p, volatile int *abort
 }
 
 // All threads of all CTAs meet here.  Returns false when the wait expired (step aborted).
-__device__ __forceinline__ bool grid_barrier(const MkParams &p, unsigned target, volatile int *abort_flag, int tid, int &prof_idx) {
+// While the CTA waits, every warp tops up its weight ring (the fetches short operators skipped).
+template <typename Refill>
+__device__ __forceinline__ bool grid_barrier(const MkParams &p, unsigned target, volatile int *abort_flag, int tid, int &prof_idx,
+                                             Refill &&refill_fn) {
     cta_sync();
     prof_stamp(p, tid, prof_idx);   // this CTA's share of the operator is done
+    if (tid == 0 && !*abort_flag) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.barrier) : "memory");
+    refill_fn();
     if (tid == 0 && !*abort_flag) {
-        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.barrier) : "memory");
         unsigned it = 0;
         unsigned long long t0 = 0;
         while (ld_acquire_gpu(p.barrier) < target) {
@@ -206,18 +229,36 @@ __device__ __forceinline__ int item_rows(const MkPhase &P, const MkParams &p, in
 // ---- a warp's position in its tile sequence over the whole step ----------------------------------------
 // Tile j of a CTA's share of an operator is slice (j & (ksplit-1)) of item (j >> s_shift); warp w owns the
 // tiles j = w, w + NW, ...  The CTA's item range of every operator is tabulated once per launch (s_rng).
+// The cursor keeps the constants of its operator in registers so that issuing a tile costs no shared-memory
+// round trips.
 struct TileCursor {
     int ph;        // operator index (nph = past the end)
     int j;         // tile index inside this CTA's share of the operator
     int it0;       // first item of this CTA in operator ph
     int n_tiles;   // tiles of this CTA in operator ph
+    // cached from s_ph[ph]
+    const uint16_t *W;
+    int K, rw, s_shift, smask, units_total, kind;
+    unsigned seg_bytes;      // bytes of one row slice
+    unsigned alloc_bytes;    // ring bytes of one tile
+    unsigned partner_elems;  // elements between the two blocks of a paired tile (0: single block)
 };
 __device__ __forceinline__ void cursor_enter_phase(TileCursor &c, const MkParams &p, const MkPhase *s_ph, const int2 *s_rng, int warp) {
     while (c.ph < p.nph) {  // skip operators in which this warp owns no tile
+        const MkPhase &P = s_ph[c.ph];
         const int2 r = s_rng[c.ph];
         c.it0 = r.x;
-        c.n_tiles = (r.y - r.x) << s_ph[c.ph].s_shift;
-        if (warp < c.n_tiles) { c.j = warp; return; }
+        c.n_tiles = (r.y - r.x) << P.s_shift;
+        if (warp < c.n_tiles) {
+            c.j = warp;
+            c.W = P.W; c.K = P.K; c.rw = P.rw; c.s_shift = P.s_shift; c.smask = P.ksplit - 1; c.units_total = P.units_total;
+            c.kind = P.kind;
+            c.seg_bytes = static_cast<unsigned>(P.kcs) * 16u;
+            const bool paired = P.kind == PH_QKV || P.kind == PH_SWIGLU;
+            c.alloc_bytes = (paired ? 2u : 1u) * P.rw * c.seg_bytes;
+            c.partner_elems = !paired ? 0u : static_cast<unsigned>(P.kind == PH_QKV ? (p.d >> 1) : p.F) * static_cast<unsigned>(P.K);
+            return;
+        }
         ++c.ph;
     }
 }
@@ -228,31 +269,31 @@ __device__ __forceinline__ void cursor_advance(TileCursor &c, const MkParams &p,
     cursor_enter_phase(c, p, s_ph, s_rng, warp);
 }
 
-// Fetch the tile under cursor `c` into a ring slot.  Called by a whole warp after __syncwarp(); lane 0 issues.
-__device__ __forceinline__ bool issue_tile(const MkParams &p, const MkPhase *s_ph, const TileCursor &c, unsigned char *dst,
-                                           unsigned long long *bar, unsigned long long policy, volatile int *abort_flag, int lane) {
-    const MkPhase &P = s_ph[c.ph];
-    const int it = c.it0 + (c.j >> P.s_shift);
-    const int sl = c.j & (P.ksplit - 1);
-    const int nblk = (P.kind == PH_QKV || P.kind == PH_SWIGLU) ? 2 : 1;
-    const unsigned seg_bytes = static_cast<unsigned>(P.kcs) * 16u;
-    int cnt;
-    const int row_lo = item_rows(P, p, it, 0, cnt);
-    const unsigned bytes = static_cast<unsigned>(cnt) * seg_bytes;   // one contiguous run per block
-    // bounds of the tile: at least one row, inside the slot, inside the matrix (16-byte rule holds by construction:
-    // K % 8 == 0, kcs * 16-byte slices, 16-byte aligned bases and slots, all checked on the host)
-    if (cnt < 1 || static_cast<unsigned>(nblk - 1) * P.rw * seg_bytes + bytes > static_cast<unsigned>(p.slot_bytes) ||
-        it >= P.items_total || (sl + 1) * P.kcs * 8 > P.K)
-        return diag_fail(p, abort_flag, 1, c.ph, it);
+// Fetch the tile under cursor `c` into ring space.  Called by a whole warp after __syncwarp(); lane 0 issues.
+__device__ __forceinline__ bool issue_tile(const MkParams &p, const TileCursor &c, unsigned char *dst, unsigned long long *bar,
+                                           unsigned long long policy, volatile int *abort_flag, int lane) {
+    const int it = c.it0 + (c.j >> c.s_shift);
+    const int sl = c.j & c.smask;
+    const int u0 = it * c.rw;
+    const int cnt = min(c.rw, c.units_total - u0);
+    int row_lo = u0;
+    if (c.kind == PH_QKV) {
+        const int half = p.d >> 1;
+        row_lo = (u0 >> p.half_shift) * p.d + (u0 & (half - 1));
+    }
+    const unsigned bytes = static_cast<unsigned>(cnt) * c.seg_bytes;   // one contiguous run per block
+    // bounds: at least one row, inside the matrix (16-byte rule holds by construction: K % 8 == 0, slices of
+    // kcs 16-byte pieces, 16-byte aligned bases and ring offsets, all checked on the host)
+    if (cnt < 1 || (sl + 1) * static_cast<int>(c.seg_bytes >> 1) > c.K) return diag_fail(p, abort_flag, 1, c.ph, it);
     if (lane == 0) {
-        const uint16_t *src = P.W + static_cast<size_t>(row_lo) * P.K + static_cast<size_t>(sl) * P.kcs * 8;
-        // the slot was read through the generic proxy by this warp: order those reads before the async write
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive_expect_tx(bar, bytes * nblk);
-        bulk_copy_g2s(dst, src, bytes, bar, policy);
-        if (nblk == 2) {
-            const size_t partner = P.kind == PH_QKV ? static_cast<size_t>(p.d >> 1) : static_cast<size_t>(p.F);   // rows between the blocks
-            bulk_copy_g2s(dst + static_cast<size_t>(P.rw) * seg_bytes, src + partner * P.K, bytes, bar, policy);
+        const uint16_t *src = c.W + static_cast<size_t>(row_lo) * c.K + static_cast<size_t>(sl) * (c.seg_bytes >> 1);
+        if (c.partner_elems) {
+            mbar_arrive_expect_tx(bar, bytes * 2u);
+            bulk_copy_g2s(dst, src, bytes, bar, policy);
+            bulk_copy_g2s(dst + static_cast<size_t>(c.rw) * c.seg_bytes, src + c.partner_elems, bytes, bar, policy);
+        } else {
+            mbar_arrive_expect_tx(bar, bytes);
+            bulk_copy_g2s(dst, src, bytes, bar, policy);
         }
     }
     return true;
@@ -260,13 +301,54 @@ __device__ __forceinline__ bool issue_tile(const MkParams &p, const MkPhase *s_p
 
 // Per-warp streaming state.
 struct WarpStream {
-    TileCursor pf;          // next tile to fetch into shared memory (depth tiles ahead of consumption)
-    unsigned consumed;      // tiles consumed so far by this warp
-    unsigned issued;        // tiles fetched so far
-    unsigned char *slots;   // this warp's `depth` ring slots
-    unsigned long long *bars;
+    TileCursor pf;            // next tile to fetch into shared memory
+    unsigned consumed;        // tiles consumed so far by this warp
+    unsigned issued;          // tiles fetched so far (issued - consumed <= MK_MAXF)
+    unsigned char *ring;      // this warp's byte ring
+    int head, tail;           // ring offsets: [head, tail) (cyclically) holds the tiles in flight
+    unsigned long long fifo;  // ring offset / 16 of tile k in the 16-bit field k % MK_MAXF
+    unsigned long long *bars; // [MK_MAXF]
     unsigned long long policy;
 };
+static_assert(MK_MAXF == 4, "fifo packs four 16-bit offsets into one register");
+__device__ __forceinline__ int fifo_get(const WarpStream &ws, unsigned k) {
+    return static_cast<int>((ws.fifo >> ((k & 3u) * 16u)) & 0xffffull) << 4;
+}
+__device__ __forceinline__ void fifo_set(WarpStream &ws, unsigned k, int off) {
+    const unsigned sh = (k & 3u) * 16u;
+    ws.fifo = (ws.fifo & ~(0xffffull << sh)) | (static_cast<unsigned long long>(off >> 4) << sh);
+}
+
+// Fetch as many of this warp's next tiles as fit its ring (first-in first-out space, at most MK_MAXF in
+// flight).  Whole warp, after __syncwarp() when ring space has just been read.
+__device__ __forceinline__ bool refill(const MkParams &p, const MkPhase *s_ph, const int2 *s_rng, WarpStream &ws,
+                                       volatile int *abort_flag, int warp, int lane) {
+    bool fenced = false;
+    while (ws.issued - ws.consumed < MK_MAXF && ws.pf.ph < p.nph) {
+        const int sz = static_cast<int>(ws.pf.alloc_bytes);
+        if (ws.issued == ws.consumed) { ws.head = 0; ws.tail = 0; }   // empty: restart at the base
+        int off;
+        if (ws.head <= ws.tail) {            // in flight: [head, tail); free: [tail, R) and [0, head)
+            if (ws.tail + sz <= p.ring_bytes) off = ws.tail;
+            else if (sz < ws.head) off = 0;  // wrap (the bytes behind tail stay unused this round)
+            else break;
+        } else {                              // wrapped: free is [tail, head)
+            if (ws.tail + sz < ws.head) off = ws.tail;
+            else break;
+        }
+        if (!fenced) {
+            // ring space was read through the generic proxy by this warp: order those reads before async writes
+            if (lane == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            fenced = true;
+        }
+        if (!issue_tile(p, ws.pf, ws.ring + off, &ws.bars[ws.issued & (MK_MAXF - 1)], ws.policy, abort_flag, lane)) return false;
+        fifo_set(ws, ws.issued, off);
+        ws.tail = off + sz;
+        ++ws.issued;
+        cursor_advance(ws.pf, p, s_ph, s_rng, warp);
+    }
+    return true;
+}
 
 struct ItemCtx {
     float rscale;          // deferred RMSNorm factor (1 for plain prologues)
@@ -278,9 +360,11 @@ struct ItemCtx {
 };
 
 // ---- fused epilogue of one output unit (a row, or a row pair) ------------------------------------------------
-__device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkPhase &P, ItemCtx &cx, int u, float lo, float hi) {
+// pre: the value the epilogue adds (old residual / the two biases) was fetched ahead into pre_lo, pre_hi.
+__device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkPhase &P, ItemCtx &cx, int u, float lo, float hi,
+                                               bool pre = false, float pre_lo = 0.f, float pre_hi = 0.f) {
     if (P.kind == PH_RESID) {
-        P.out[u] = __ldcg(P.out + u) + lo;
+        P.out[u] = (pre ? pre_lo : __ldcg(P.out + u)) + lo;
     } else if (P.kind == PH_LMHEAD) {
         if (cx.logits_out) cx.logits_out[u] = lo;
         if (arg_better(lo, u, cx.best_v, cx.best_i)) { cx.best_v = lo; cx.best_i = u; }
@@ -290,7 +374,10 @@ __device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkPhase 
         const int half = p.d >> 1;
         const int head = u >> p.half_shift, i = u & (half - 1);
         const int row_lo = head * p.d + i, row_hi = row_lo + half;
-        if (P.bias) { lo += bf16_bits_to_f32(P.bias[row_lo]); hi += bf16_bits_to_f32(P.bias[row_hi]); }
+        if (P.bias) {
+            lo += pre ? pre_lo : bf16_bits_to_f32(P.bias[row_lo]);
+            hi += pre ? pre_hi : bf16_bits_to_f32(P.bias[row_hi]);
+        }
         const size_t layer_off = static_cast<size_t>(P.layer) * p.nkv * p.max_context * p.d;
         if (head < p.nq + p.nkv) {
             const float c = cx.rope[i], sn = cx.rope[half + i];
@@ -313,19 +400,21 @@ __device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkPhase 
 
 // ---- one tile (NR row slices of kcs 16-byte pieces) by one warp: wait, multiply, re-arm the slot ------------
 template <int NR>
-__device__ __forceinline__ bool consume_tile(const MkParams &p, const MkPhase *s_ph, const int2 *s_rng, const MkPhase &P, int slice,
+__device__ __forceinline__ bool consume_tile(const MkParams &p, const MkPhase *s_ph, const int2 *s_rng, int kcs, int slice, bool do_refill,
                                              WarpStream &ws, const float4 *xsA, const float4 *xsB, volatile int *abort_flag,
                                              float (&out)[NR], int warp, int lane) {
     float acc[NR], acc2[NR];   // two chains per row halve the dependent-FMA latency
 #pragma unroll
     for (int r = 0; r < NR; ++r) { acc[r] = 0.f; acc2[r] = 0.f; }
-    const int kcs = P.kcs;
-    if (NR * kcs * 16 > p.slot_bytes || P.ksplit * kcs * 32 > p.xbuf_bytes) return diag_fail(p, abort_flag, 2, kcs, NR);
-    const unsigned q = ws.consumed & static_cast<unsigned>(p.depth - 1);             // depth is a power of two
-    const unsigned par = (ws.consumed >> p.depth_shift) & 1u;
+    if (ws.consumed == ws.issued) {   // not fetched yet (short operator whose tiles exceed the ring): fetch on demand
+        __syncwarp();
+        if (!refill(p, s_ph, s_rng, ws, abort_flag, warp, lane)) return false;
+        if (ws.consumed == ws.issued) return diag_fail(p, abort_flag, 2, kcs, NR);
+    }
+    const unsigned q = ws.consumed & (MK_MAXF - 1);
+    const unsigned par = (ws.consumed / MK_MAXF) & 1u;
     if (!mbar_wait(&ws.bars[q], par, abort_flag, p.spin_limit)) return false;
-    unsigned char *slot = ws.slots + static_cast<size_t>(q) * p.slot_bytes;
-    const uint4 *t = reinterpret_cast<const uint4 *>(slot);
+    const uint4 *t = reinterpret_cast<const uint4 *>(ws.ring + fifo_get(ws, ws.consumed));
     const float4 *a = xsA + slice * kcs, *b = xsB + slice * kcs;
     auto fma_chunk = [&](const uint4 &w, const float4 &x0, const float4 &x1, int r) {
         acc[r] = fmaf(bf16lo(w.x), x0.x, acc[r]);  acc2[r] = fmaf(bf16hi(w.x), x0.y, acc2[r]);
@@ -355,13 +444,9 @@ __device__ __forceinline__ bool consume_tile(const MkParams &p, const MkPhase *s
         for (int r = 0; r < NR; ++r) fma_chunk(t[r * kcs + c], x0, x1, r);
     }
     ++ws.consumed;
+    ws.head = ws.consumed < ws.issued ? fifo_get(ws, ws.consumed) : ws.tail;   // free the tile's bytes
     __syncwarp();
-    // re-arm the slot with the tile `depth` ahead in this warp's sequence
-    if (ws.pf.ph < p.nph) {
-        if (!issue_tile(p, s_ph, ws.pf, slot, &ws.bars[q], ws.policy, abort_flag, lane)) return false;
-        ++ws.issued;
-        cursor_advance(ws.pf, p, s_ph, s_rng, warp);
-    }
+    if (do_refill && !refill(p, s_ph, s_rng, ws, abort_flag, warp, lane)) return false;
 #pragma unroll
     for (int r = 0; r < NR; ++r) out[r] = warp_sum(acc[r] + acc2[r]);
     return true;
@@ -372,27 +457,38 @@ __device__ __forceinline__ bool consume_tile(const MkParams &p, const MkPhase *s
 template <int NR>
 __device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkPhase *s_ph, const int2 *s_rng, const MkPhase &P, int it0,
                                               int n_tiles, WarpStream &ws, const float4 *xsA, const float4 *xsB,
-                                              volatile int *abort_flag, ItemCtx &cx, float *s_partial, int warp, int lane) {
+                                              volatile int *abort_flag, ItemCtx &cx, float *s_partial, int warp, int lane,
+                                              int ph_index) {
+    int trace_slot = 1;
+    // operator constants in registers (the asm memory clobbers would otherwise force shared-memory reloads)
+    const int kcs = P.kcs, smask = P.ksplit - 1, rw = P.rw, kind = P.kind, units_total = P.units_total;
+    const bool split = P.split != 0;
+    if (NR * kcs * 16 > p.slot_bytes || P.ksplit * kcs * 32 > p.xbuf_bytes) return diag_fail(p, abort_flag, 2, kcs, NR);
+    // short operators leave the ring alone (it is topped up while the CTA waits at the grid barrier), so that
+    // nothing but the arithmetic sits on their critical path; streaming operators refill after every tile
+    const bool do_refill = n_tiles > 2 * MK_NW;
     for (int j = warp; j < n_tiles; j += MK_NW) {
         float y[NR];
-        if (!consume_tile<NR>(p, s_ph, s_rng, P, j & (P.ksplit - 1), ws, xsA, xsB, abort_flag, y, warp, lane)) return false;
-        if (P.split) {
+        MK_TRACE(p, ph_index, warp, lane, trace_slot); ++trace_slot;
+        if (!consume_tile<NR>(p, s_ph, s_rng, kcs, j & smask, do_refill, ws, xsA, xsB, abort_flag, y, warp, lane)) return false;
+        MK_TRACE(p, ph_index, warp, lane, trace_slot); ++trace_slot;
+        if (split) {
 #pragma unroll
             for (int r = 0; r < NR; ++r)
                 if (lane == r) s_partial[j * NR + r] = y[r];
         } else {
-            const int u0 = (it0 + j) * P.rw;
+            const int u0 = (it0 + j) * rw;
             constexpr int NU = NR >= 2 ? NR / 2 : 1;
-            if (P.kind == PH_QKV || P.kind == PH_SWIGLU) {
+            if (kind == PH_QKV || kind == PH_SWIGLU) {
                 if constexpr (NR >= 2) {
 #pragma unroll
                     for (int r = 0; r < NU; ++r)
-                        if (lane == r && u0 + r < P.units_total) apply_epilogue(p, P, cx, u0 + r, y[r] * cx.rscale, y[r + NU] * cx.rscale);
+                        if (lane == r && u0 + r < units_total) apply_epilogue(p, P, cx, u0 + r, y[r] * cx.rscale, y[r + NU] * cx.rscale);
                 }
             } else {
 #pragma unroll
                 for (int r = 0; r < NR; ++r)
-                    if (lane == r && u0 + r < P.units_total) apply_epilogue(p, P, cx, u0 + r, y[r] * cx.rscale, 0.f);
+                    if (lane == r && u0 + r < units_total) apply_epilogue(p, P, cx, u0 + r, y[r] * cx.rscale, 0.f);
             }
         }
     }
@@ -510,21 +606,38 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, const MkPhase *s_p
         for (int w = 0; w < MK_NW; ++w) tot += s_part[w];
         cx.rscale = rsqrtf(tot / static_cast<float>(P.K) + p.eps);
     }
+    MK_TRACE(p, ph, warp, lane, 0);
     const int2 rng = s_rng[ph];
     const int n_items = rng.y - rng.x;
     const int n_tiles = n_items << P.s_shift;
     const bool paired = P.kind == PH_QKV || P.kind == PH_SWIGLU;
+    // split operators: thread u finishes unit u after the tiles; fetch what its epilogue adds (old residual
+    // value, bias) now, so that the load latency overlaps the arithmetic
+    float pre_lo = 0.f, pre_hi = 0.f;
+    if (P.split && tid < n_items) {
+        const int u = rng.x + tid;
+        if (P.kind == PH_RESID) {
+            pre_lo = __ldcg(P.out + u);
+        } else if (P.kind == PH_QKV && P.bias) {
+            const int half = p.d >> 1;
+            const int row_lo = (u >> p.half_shift) * p.d + (u & (half - 1));
+            pre_lo = bf16_bits_to_f32(P.bias[row_lo]);
+            pre_hi = bf16_bits_to_f32(P.bias[row_lo + half]);
+        }
+    }
     const int nr = paired ? 2 * P.rw : P.rw;
     bool ok;
     switch (nr) {
-        case 1: ok = consume_tiles<1>(p, s_ph, s_rng, P, rng.x, n_tiles, ws, xsA, xsB, abort_flag, cx, s_partial, warp, lane); break;
-        case 2: ok = consume_tiles<2>(p, s_ph, s_rng, P, rng.x, n_tiles, ws, xsA, xsB, abort_flag, cx, s_partial, warp, lane); break;
-        case 4: ok = consume_tiles<4>(p, s_ph, s_rng, P, rng.x, n_tiles, ws, xsA, xsB, abort_flag, cx, s_partial, warp, lane); break;
-        default: ok = consume_tiles<8>(p, s_ph, s_rng, P, rng.x, n_tiles, ws, xsA, xsB, abort_flag, cx, s_partial, warp, lane); break;
+        case 1: ok = consume_tiles<1>(p, s_ph, s_rng, P, rng.x, n_tiles, ws, xsA, xsB, abort_flag, cx, s_partial, warp, lane, ph); break;
+        case 2: ok = consume_tiles<2>(p, s_ph, s_rng, P, rng.x, n_tiles, ws, xsA, xsB, abort_flag, cx, s_partial, warp, lane, ph); break;
+        case 4: ok = consume_tiles<4>(p, s_ph, s_rng, P, rng.x, n_tiles, ws, xsA, xsB, abort_flag, cx, s_partial, warp, lane, ph); break;
+        default: ok = consume_tiles<8>(p, s_ph, s_rng, P, rng.x, n_tiles, ws, xsA, xsB, abort_flag, cx, s_partial, warp, lane, ph); break;
     }
+    MK_TRACE(p, ph, warp, lane, 12);
     if (P.split) {
         // partial sums of the K slices meet here; thread u finishes unit u of this CTA (rw == 1), slices in order
         cta_sync();
+        MK_TRACE(p, ph, warp, lane, 13);
         if (!*abort_flag) {
             for (int u = tid; u < n_items; u += MK_NT) {
                 float lo = 0.f, hi = 0.f;
@@ -532,9 +645,11 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, const MkPhase *s_p
                     const int j = (u << P.s_shift) + sl;
                     if (paired) { lo += s_partial[2 * j]; hi += s_partial[2 * j + 1]; } else { lo += s_partial[j]; }
                 }
-                apply_epilogue(p, P, cx, rng.x + u, lo * cx.rscale, hi * cx.rscale);
+                const bool pre = u == tid;   // operands fetched ahead (first MK_NT units)
+                apply_epilogue(p, P, cx, rng.x + u, lo * cx.rscale, hi * cx.rscale, pre, pre_lo, pre_hi);
             }
         }
+        MK_TRACE(p, ph, warp, lane, 14);
     }
     return ok;
 }
@@ -786,7 +901,7 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
     MkPhase *s_ph = reinterpret_cast<MkPhase *>(smem + p.xbuf_bytes);          // the step's schedule
     int2 *s_rng = reinterpret_cast<int2 *>(s_ph + p.nph);                      // this CTA's item range per operator
     unsigned char *ring = smem + p.xbuf_bytes + p.sched_bytes;
-    __shared__ __align__(8) unsigned long long full_bar[MK_NW * MK_MAX_DEPTH];
+    __shared__ __align__(8) unsigned long long full_bar[MK_NW * MK_MAXF];
     __shared__ float s_rope[128];
     __shared__ float s_part[MK_NW];
     __shared__ float s_partial[MK_PARTIAL_FLOATS];
@@ -798,7 +913,7 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int cta = blockIdx.x, ncta = gridDim.x;
     if (tid == 0) {
-        for (int i = 0; i < MK_NW * p.depth; ++i) mbar_init(&full_bar[i], 1);
+        for (int i = 0; i < MK_NW * MK_MAXF; ++i) mbar_init(&full_bar[i], 1);
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -818,18 +933,13 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
 
     // ---- start this warp's weight stream: fill its ring, then run the L2 prefetch ahead ---------------
     WarpStream ws;
-    ws.consumed = 0; ws.issued = 0;
-    ws.slots = ring + static_cast<size_t>(warp) * p.depth * p.slot_bytes;
-    ws.bars = &full_bar[warp * p.depth];
+    ws.consumed = 0; ws.issued = 0; ws.head = 0; ws.tail = 0; ws.fifo = 0;
+    ws.ring = ring + static_cast<size_t>(warp) * p.ring_bytes;
+    ws.bars = &full_bar[warp * MK_MAXF];
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(ws.policy));
     ws.pf.ph = 0;
     cursor_enter_phase(ws.pf, p, s_ph, s_rng, warp);
-    bool ok = true;
-    for (int q = 0; q < p.depth && ok && ws.pf.ph < p.nph; ++q) {
-        ok = issue_tile(p, s_ph, ws.pf, ws.slots + static_cast<size_t>(q) * p.slot_bytes, &ws.bars[q], ws.policy, abort_flag, lane);
-        ++ws.issued;
-        cursor_advance(ws.pf, p, s_ph, s_rng, warp);
-    }
+    bool ok = refill(p, s_ph, s_rng, ws, abort_flag, warp, lane);
     const int rt = p.req->token, rp = p.req->position;
     const int token = rt >= 0 ? rt : p.state->next_token;
     const int pos = rp >= 0 ? rp : p.state->next_position;
@@ -855,22 +965,23 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
     unsigned bar_no = 0;
     int prof_idx = 0;
     prof_stamp(p, tid, prof_idx);
+    auto top_up = [&]() { __syncwarp(); if (ok && !*abort_flag) refill(p, s_ph, s_rng, ws, abort_flag, warp, lane); };
     const int n_att = slot_row + 1;
     const bool att_split = n_att <= p.att_split_max_n && static_cast<long long>(p.nq) * MK_ATT_SPLIT_MAXC * 2 <= MK_PARTIAL_FLOATS;
     int merge_chunks = 0;   // chunks per head the O-projection prologue has to merge (split mode)
     if (att_split) { int cl; att_chunking(p, n_att, 1, p.att_chunk_split, ncta, merge_chunks, cl); }
     for (int l = 0; l < p.n_layers && ok; ++l) {
         ok = gemv_phase(p, s_ph, s_rng, 4 * l, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token, 0, tid, prof_idx);
-        ok = grid_barrier(p, ++bar_no * ncta, abort_flag, tid, prof_idx) && ok;
+        ok = grid_barrier(p, ++bar_no * ncta, abort_flag, tid, prof_idx, top_up) && ok;
         if (ok) {
             if (att_split) attention_phase<D, 1>(p, l, n_att, p.att_chunk_split, true, smem, tid, &s_flag);
             else attention_phase<D, G>(p, l, n_att, p.att_chunk_shared, false, smem, tid, &s_flag);
         }
-        ok = grid_barrier(p, ++bar_no * ncta, abort_flag, tid, prof_idx) && ok;
+        ok = grid_barrier(p, ++bar_no * ncta, abort_flag, tid, prof_idx, top_up) && ok;
         for (int k = 1; k < 4 && ok; ++k) {
             ok = gemv_phase(p, s_ph, s_rng, 4 * l + k, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token,
                             k == 1 ? merge_chunks : 0, tid, prof_idx);
-            ok = grid_barrier(p, ++bar_no * ncta, abort_flag, tid, prof_idx) && ok;
+            ok = grid_barrier(p, ++bar_no * ncta, abort_flag, tid, prof_idx, top_up) && ok;
         }
     }
     if (ok) ok = gemv_phase(p, s_ph, s_rng, 4 * p.n_layers, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token, 0, tid, prof_idx);
@@ -879,8 +990,8 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
         // aborted: wait (bounded) for the copies this warp still has in flight, then leave
         if (tid == 0 && p.state->status == 0) p.state->status = 6;
         for (unsigned k = ws.consumed; k < ws.issued; ++k) {
-            const unsigned q = k & static_cast<unsigned>(p.depth - 1);
-            const unsigned par = (k >> p.depth_shift) & 1u;
+            const unsigned q = k & (MK_MAXF - 1);
+            const unsigned par = (k / MK_MAXF) & 1u;
             const unsigned long long t0 = global_ns();
             while (!mbar_try_wait(&ws.bars[q], par))
                 if (global_ns() - t0 > p.spin_limit) break;
