@@ -32,6 +32,7 @@ namespace edgefm {
 constexpr int MK_NW = 12;                        // warps per CTA (each streams and consumes its own tiles)
 constexpr int MK_NT = MK_NW * 32;
 constexpr int MK_MAXF = 4;                       // tiles in flight per warp (one mbarrier each)
+constexpr int MK_BAR_POLLERS = 1;                // warps whose lane 0 polls the grid barrier counter
 constexpr int MK_ATT_LPP = 4;                    // lanes per cached position in the score phase
 constexpr int MK_ATT_TILE = 32 / MK_ATT_LPP;     // positions per warp iteration
 constexpr int MK_ATT_MW = (MK_NW + 1) / 2;       // warps whose partials fit the merge area at once
@@ -185,22 +186,29 @@ __device__ __forceinline__ bool diag_fail(const MkParams &p, volatile int *abort
 // All threads of all CTAs meet here.  Returns false when the wait expired (step aborted).
 // While the CTA waits, every warp tops up its weight ring (the fetches short operators skipped).
 template <typename Refill>
-__device__ __forceinline__ bool grid_barrier(const MkParams &p, unsigned target, volatile int *abort_flag, int tid, int &prof_idx,
-                                             Refill &&refill_fn) {
+__device__ __forceinline__ bool grid_barrier(const MkParams &p, unsigned target, volatile int *abort_flag, volatile int *s_released,
+                                             int tid, int &prof_idx, Refill &&refill_fn) {
     cta_sync();
     prof_stamp(p, tid, prof_idx);   // this CTA's share of the operator is done
-    if (tid == 0 && !*abort_flag) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.barrier) : "memory");
-    refill_fn();
     if (tid == 0 && !*abort_flag) {
+        *s_released = 0;
+        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.barrier) : "memory");
+    }
+    refill_fn();
+    // lane 0 of the first MK_BAR_POLLERS warps polls the counter; their polls interleave in time, which shortens the
+    // delay between the last arrival and its detection; whoever sees it first releases the others
+    if ((tid & 31) == 0 && (tid >> 5) < MK_BAR_POLLERS && !*abort_flag) {
         unsigned it = 0;
         unsigned long long t0 = 0;
         while (ld_acquire_gpu(p.barrier) < target) {
+            if (*s_released) break;
             if ((++it & 63u) == 0u) {
                 const unsigned long long now = global_ns();
                 if (t0 == 0) t0 = now;
                 else if (now - t0 > p.spin_limit) { *abort_flag = 1; p.state->status = 6; break; }
             }
         }
+        *s_released = 1;
     }
     cta_sync();
     prof_stamp(p, tid, prof_idx);   // released by the slowest CTA
@@ -306,6 +314,7 @@ struct WarpStream {
     unsigned issued;          // tiles fetched so far (issued - consumed <= MK_MAXF)
     unsigned char *ring;      // this warp's byte ring
     int head, tail;           // ring offsets: [head, tail) (cyclically) holds the tiles in flight
+    bool wrapped;             // tail has wrapped around the ring end and head has not yet
     unsigned long long fifo;  // ring offset / 16 of tile k in the 16-bit field k % MK_MAXF
     unsigned long long *bars; // [MK_MAXF]
     unsigned long long policy;
@@ -326,14 +335,14 @@ __device__ __forceinline__ bool refill(const MkParams &p, const MkPhase *s_ph, c
     bool fenced = false;
     while (ws.issued - ws.consumed < MK_MAXF && ws.pf.ph < p.nph) {
         const int sz = static_cast<int>(ws.pf.alloc_bytes);
-        if (ws.issued == ws.consumed) { ws.head = 0; ws.tail = 0; }   // empty: restart at the base
+        if (ws.issued == ws.consumed) { ws.head = 0; ws.tail = 0; ws.wrapped = false; }   // empty: restart at the base
         int off;
-        if (ws.head <= ws.tail) {            // in flight: [head, tail); free: [tail, R) and [0, head)
+        if (!ws.wrapped) {                   // in flight: [head, tail); free: [tail, R) and [0, head)
             if (ws.tail + sz <= p.ring_bytes) off = ws.tail;
-            else if (sz < ws.head) off = 0;  // wrap (the bytes behind tail stay unused this round)
+            else if (sz <= ws.head) { off = 0; ws.wrapped = true; }   // wrap (the bytes behind tail stay unused this round)
             else break;
-        } else {                              // wrapped: free is [tail, head)
-            if (ws.tail + sz < ws.head) off = ws.tail;
+        } else {                              // in flight: [head, R) and [0, tail); free: [tail, head)
+            if (ws.tail + sz <= ws.head) off = ws.tail;
             else break;
         }
         if (!fenced) {
@@ -444,7 +453,11 @@ __device__ __forceinline__ bool consume_tile(const MkParams &p, const MkPhase *s
         for (int r = 0; r < NR; ++r) fma_chunk(t[r * kcs + c], x0, x1, r);
     }
     ++ws.consumed;
-    ws.head = ws.consumed < ws.issued ? fifo_get(ws, ws.consumed) : ws.tail;   // free the tile's bytes
+    {   // free the tile's bytes: head moves to the next tile in flight (back to the ring start once it passes the wrap)
+        const int nh = ws.consumed < ws.issued ? fifo_get(ws, ws.consumed) : ws.tail;
+        if (nh < ws.head) ws.wrapped = false;
+        ws.head = nh;
+    }
     __syncwarp();
     if (do_refill && !refill(p, s_ph, s_rng, ws, abort_flag, warp, lane)) return false;
 #pragma unroll
@@ -909,6 +922,7 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
     __shared__ int s_bi[MK_NW];
     __shared__ int s_flag;
     __shared__ int s_abort;
+    __shared__ int s_released;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int cta = blockIdx.x, ncta = gridDim.x;
@@ -931,9 +945,18 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
     __syncthreads();
     volatile int *abort_flag = &s_abort;
 
+    // The small per-layer vectors (norm weights, biases) are read on the critical path right after a grid barrier;
+    // ask L2 for all of them now (they stay: the weight stream is evict-first).
+    for (int i = cta * MK_NT + tid; i < p.nph * 64; i += ncta * MK_NT) {
+        const MkPhase &P = s_ph[i >> 6];
+        const int line = i & 63;   // 128-byte line of the vector
+        if (P.norm_w && line * 64 < P.K) asm volatile("prefetch.global.L2 [%0];" ::"l"(P.norm_w + line * 64));
+        if (P.bias && P.kind == PH_QKV && line * 64 < 2 * P.units_total) asm volatile("prefetch.global.L2 [%0];" ::"l"(P.bias + line * 64));
+    }
+
     // ---- start this warp's weight stream: fill its ring, then run the L2 prefetch ahead ---------------
     WarpStream ws;
-    ws.consumed = 0; ws.issued = 0; ws.head = 0; ws.tail = 0; ws.fifo = 0;
+    ws.consumed = 0; ws.issued = 0; ws.head = 0; ws.tail = 0; ws.wrapped = false; ws.fifo = 0;
     ws.ring = ring + static_cast<size_t>(warp) * p.ring_bytes;
     ws.bars = &full_bar[warp * MK_MAXF];
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(ws.policy));
@@ -972,16 +995,16 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
     if (att_split) { int cl; att_chunking(p, n_att, 1, p.att_chunk_split, ncta, merge_chunks, cl); }
     for (int l = 0; l < p.n_layers && ok; ++l) {
         ok = gemv_phase(p, s_ph, s_rng, 4 * l, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token, 0, tid, prof_idx);
-        ok = grid_barrier(p, ++bar_no * ncta, abort_flag, tid, prof_idx, top_up) && ok;
+        ok = grid_barrier(p, ++bar_no * ncta, abort_flag, &s_released, tid, prof_idx, top_up) && ok;
         if (ok) {
             if (att_split) attention_phase<D, 1>(p, l, n_att, p.att_chunk_split, true, smem, tid, &s_flag);
             else attention_phase<D, G>(p, l, n_att, p.att_chunk_shared, false, smem, tid, &s_flag);
         }
-        ok = grid_barrier(p, ++bar_no * ncta, abort_flag, tid, prof_idx, top_up) && ok;
+        ok = grid_barrier(p, ++bar_no * ncta, abort_flag, &s_released, tid, prof_idx, top_up) && ok;
         for (int k = 1; k < 4 && ok; ++k) {
             ok = gemv_phase(p, s_ph, s_rng, 4 * l + k, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token,
                             k == 1 ? merge_chunks : 0, tid, prof_idx);
-            ok = grid_barrier(p, ++bar_no * ncta, abort_flag, tid, prof_idx, top_up) && ok;
+            ok = grid_barrier(p, ++bar_no * ncta, abort_flag, &s_released, tid, prof_idx, top_up) && ok;
         }
     }
     if (ok) ok = gemv_phase(p, s_ph, s_rng, 4 * p.n_layers, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token, 0, tid, prof_idx);
