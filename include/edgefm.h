@@ -145,6 +145,39 @@ edgefm_status edgefm_sync_status(edgefm_ctx *ctx, void *stream);
  * out_host may be NULL to query the sizes. */
 edgefm_status edgefm_debug_profile(edgefm_ctx *ctx, uint64_t *out_host, int64_t capacity, int32_t *n_ctas, int32_t *stride);
 
+/*
+ * edgefm_decode_step_static -- one decode step that allocates nothing (the paper has no counterpart; this
+ * entry point exists for callers that cannot allocate device memory).
+ *
+ * Who needs it: code that runs inside another framework's allocation-free region (a fixed memory plan it is
+ * recording or replaying), processes whose device memory is handed out entirely by a pool they do not own,
+ * and latency-critical threads that cannot take the implicit device synchronisation of cudaMalloc / cudaFree.
+ * edgefm_create allocates a KV cache and work buffers; this call does neither.  It is the same persistent step
+ * kernel as edgefm_decode_step, with all its work buffers (residual stream, queries, attention partials, MLP
+ * activations, schedule, counters, device state) carved out of a fixed 2 MiB array that is part of the loaded
+ * library image on every GPU, and with the KV cache owned by the caller:
+ *   shape, weights   as for edgefm_create (read during the call; device buffers borrowed until the step has run);
+ *                    at most 96 layers, and the work buffers of the shape must fit the 2 MiB, else
+ *                    EDGEFM_ERR_BAD_SHAPE with a message that states the limit.
+ *   k_cache, v_cache DEVICE bf16 [n_layers][n_kv_heads][max_context][head_dim] (the layout edgefm_export_kv
+ *                    writes), 16-byte aligned; slots 0 .. cur_len-1 are read, slot cur_len is written.
+ *   cur_len          filled slots before the step (the caller keeps the count; 0 <= cur_len < max_context).
+ *   token_id, position  both explicit (>= 0); nothing is remembered between calls.
+ *   logits_out       DEVICE fp32 [vocab] or NULL;  next_token_out  DEVICE int32 [1] or NULL.
+ * The work is enqueued on `stream` (small stream-ordered copies and one memset of the counters, then the
+ * kernel) and the call returns without synchronising.  It calls no cudaMalloc, cudaFree or other allocating
+ * routine.  The first call on a device also looks up the device address of the scratch array (once per device,
+ * with that device current); make that first call outside any stream capture.
+ * All calls on a device share the one scratch array, which keeps the previous call's contents: the call
+ * clears what must start at zero itself, but two calls that overlap on the GPU (different streams, different
+ * threads, or a context created by edgefm_create is NOT affected -- it has its own buffers) race on it and
+ * give wrong results; order them on one stream or with events.
+ * Errors: INVALID_ARG, BAD_SHAPE, CONTEXT_FULL (cur_len == max_context), CUDA; message via edgefm_last_error(NULL).
+ */
+edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, const edgefm_weights *weights, void *k_cache, void *v_cache,
+                                        int32_t max_context, int32_t cur_len, int32_t token_id, int32_t position, void *stream,
+                                        float *logits_out, int32_t *next_token_out);
+
 /* Message of the last error on this context ("" if none); ctx == NULL: last error of edgefm_create
  * on the calling thread. The string is owned by the library. */
 const char *edgefm_last_error(const edgefm_ctx *ctx);

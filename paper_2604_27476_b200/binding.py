@@ -47,7 +47,7 @@ class _Weights(ctypes.Structure):
 
 EXPORTS = ("edgefm_create", "edgefm_prefill_kv", "edgefm_decode_step", "edgefm_destroy", "edgefm_get_length",
            "edgefm_export_kv", "edgefm_get_launches_per_step", "edgefm_last_error", "edgefm_version",
-           "edgefm_sync_status", "edgefm_debug_profile")
+           "edgefm_sync_status", "edgefm_debug_profile", "edgefm_decode_step_static")
 
 
 def library_path() -> Path:
@@ -58,10 +58,13 @@ def load_library():
     global _lib
     if _lib is not None:
         return _lib
-    if not _LIB_PATH.exists():
-        raise FileNotFoundError(f"{_LIB_PATH} is missing: build it with `python -m paper_2604_27476_b200.build` "
+    import os
+    alt = os.environ.get("EDGEFM_LIBRARY")   # e.g. an instrumented build of the same sources
+    path = Path(alt) if alt else _LIB_PATH
+    if not path.exists():
+        raise FileNotFoundError(f"{path} is missing: build it with `python -m paper_2604_27476_b200.build` "
                                 "(there is no CPU fallback)")
-    L = ctypes.CDLL(str(_LIB_PATH))
+    L = ctypes.CDLL(str(path))
     vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
     L.edgefm_create.restype = ctypes.c_int
     L.edgefm_create.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Weights), i32, ctypes.POINTER(vp)]
@@ -81,6 +84,8 @@ def load_library():
     L.edgefm_sync_status.argtypes = [vp, vp]
     L.edgefm_debug_profile.restype = ctypes.c_int
     L.edgefm_debug_profile.argtypes = [vp, vp, i64, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    L.edgefm_decode_step_static.restype = ctypes.c_int
+    L.edgefm_decode_step_static.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Weights), vp, vp, i32, i32, i32, i32, vp, vp, vp]
     L.edgefm_last_error.restype = ctypes.c_char_p
     L.edgefm_last_error.argtypes = [vp]
     L.edgefm_version.restype = ctypes.c_char_p
@@ -141,6 +146,25 @@ def edgefm_get_launches_per_step(ctx) -> int:
     n = ctypes.c_int32()
     _check(load_library().edgefm_get_launches_per_step(ctx, ctypes.byref(n)), ctx)
     return n.value
+
+
+def _marshal_weights(weights: dict):
+    layers = weights["layers"]
+    arr = (_LayerWeights * max(1, len(layers)))()
+    for i, lw in enumerate(layers):
+        for name, _ in _LayerWeights._fields_:
+            setattr(arr[i], name, lw.get(name))
+    return _Weights(weights["embed"], weights["final_norm"], weights["lm_head"], arr), arr
+
+
+def edgefm_decode_step_static(shape: dict, weights: dict, k_cache_ptr, v_cache_ptr, max_context, cur_len, token_id, position,
+                              stream=None, logits_out=None, next_token_out=None):
+    """One decode step with no allocation anywhere: work buffers come from the library's fixed scratch array, the
+    KV cache ([L][n_kv][max_context][d] bf16, device) and the cache length are the caller's."""
+    sh = _Shape(**shape)
+    w, keep = _marshal_weights(weights)
+    _check(load_library().edgefm_decode_step_static(ctypes.byref(sh), ctypes.byref(w), k_cache_ptr, v_cache_ptr, max_context,
+                                                    cur_len, token_id, position, stream, logits_out, next_token_out))
 
 
 def edgefm_sync_status(ctx, stream=None):

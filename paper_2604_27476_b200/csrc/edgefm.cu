@@ -767,3 +767,214 @@ edgefm_status edgefm_export_kv(edgefm_ctx *ctx, void *k_out, void *v_out, void *
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------------------
+// edgefm_decode_step_static -- one decode step that allocates nothing.
+//
+// Some callers must not allocate device memory at all: a step issued from inside another framework's
+// allocation-free region (for example while that framework is replaying or recording its own work with a
+// fixed memory plan), from a process whose device memory is handed out entirely by a pool it does not own,
+// or from a latency-critical thread where the implicit device synchronisation of cudaMalloc / cudaFree is
+// not acceptable.  For them the work buffers of the persistent step kernel (residual stream, queries,
+// attention partials, MLP activations, schedule, counters, device state: everything edgefm_create would
+// allocate except the KV cache) live in a fixed array that is part of the loaded library image.  The
+// caller owns the KV cache and the cache length and passes them in, so the call keeps no context.
+//
+// The array is EDGEFM_STATIC_SCRATCH_BYTES (2 MiB) on every GPU that loads the library, until exit.
+namespace {
+
+constexpr size_t EDGEFM_STATIC_SCRATCH_BYTES = 2u << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[EDGEFM_STATIC_SCRATCH_BYTES];
+
+// In host code `g_static_scratch` is only a host-side stand-in for the symbol, not a device address.
+// The device address is looked up once per device, with that device current.
+constexpr int kMaxDevices = 64;
+unsigned char *g_scratch_dev_ptr[kMaxDevices] = {};
+
+struct ScratchCarver {
+    unsigned char *base;
+    size_t off = 0;
+    template <typename T>
+    T *take(size_t count) {
+        T *p = reinterpret_cast<T *>(base + off);
+        off = (off + count * sizeof(T) + 255) / 256 * 256;
+        return p;
+    }
+};
+
+}  // namespace
+
+extern "C" edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, const edgefm_weights *weights, void *k_cache,
+                                                   void *v_cache, int32_t max_context, int32_t cur_len, int32_t token_id,
+                                                   int32_t position, void *stream, float *logits_out,
+                                                   int32_t *next_token_out) {
+    if (!shape || !weights || !weights->layers || !k_cache || !v_cache)
+        return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "null argument");
+    const edgefm_shape &sh = *shape;
+    constexpr int kMaxLayers = 96;
+    if (sh.n_layers < 1 || sh.n_layers > kMaxLayers || sh.hidden < 8 || sh.hidden % 8 || sh.ffn < 8 || sh.ffn % 8 ||
+        (sh.head_dim != 64 && sh.head_dim != 128) || sh.n_q_heads < 1 || sh.n_kv_heads < 1 || sh.n_q_heads % sh.n_kv_heads ||
+        sh.n_q_heads / sh.n_kv_heads > 8 || sh.vocab < 1 || !(sh.rms_eps >= 0.f) || !(sh.rope_theta > 0.f))
+        return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "unsupported model shape (same limits as edgefm_create; at most %d layers)", kMaxLayers);
+    if (max_context < 1 || cur_len < 0 || cur_len >= max_context)
+        return fail(nullptr, cur_len >= max_context ? EDGEFM_ERR_CONTEXT_FULL : EDGEFM_ERR_INVALID_ARG, "cur_len %d / max_context %d", cur_len, max_context);
+    if (token_id < 0 || token_id >= sh.vocab || position < 0) return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "token or position out of range");
+    if (!weights->embed || !weights->final_norm || !weights->lm_head) return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "null weight pointer");
+    for (int l = 0; l < sh.n_layers; ++l) {
+        const edgefm_layer_weights &w = weights->layers[l];
+        if (!w.input_norm || !w.wqkv || !w.wo || !w.post_norm || !w.w_gate_up || !w.w_down || (sh.qkv_bias && !w.bqkv))
+            return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "null weight pointer in layer %d", l);
+        if (!aligned16(w.wqkv) || !aligned16(w.wo) || !aligned16(w.w_gate_up) || !aligned16(w.w_down) || !aligned16(w.input_norm) ||
+            !aligned16(w.post_norm))
+            return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "weight pointers must be 16-byte aligned (layer %d)", l);
+    }
+    if (!aligned16(weights->embed) || !aligned16(weights->lm_head) || !aligned16(weights->final_norm) || !aligned16(k_cache) || !aligned16(v_cache))
+        return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "pointers must be 16-byte aligned");
+
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        cudaGetLastError();
+        return fail(nullptr, EDGEFM_ERR_CUDA, "no usable CUDA device (this library has no CPU path)");
+    }
+    const int H = sh.hidden, d = sh.head_dim, nq = sh.n_q_heads, nkv = sh.n_kv_heads, F = sh.ffn, G = nq / nkv;
+    const int R = (nq + 2 * nkv) * d;
+    int num_sms = 0, smem_optin = 0, coop = 0;
+    CUDA_TRY(nullptr, cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
+    CUDA_TRY(nullptr, cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    CUDA_TRY(nullptr, cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
+    if (!coop) return fail(nullptr, EDGEFM_ERR_CUDA, "device lacks cooperative launch");
+
+    // ---- set-up, once per device: the device address of the scratch array (never the host-side symbol) ----
+    if (!g_scratch_dev_ptr[dev]) {
+        unsigned char *ptr = nullptr;
+        CUDA_TRY(nullptr, cudaGetSymbolAddress(reinterpret_cast<void **>(&ptr), g_static_scratch));
+        if (!ptr) return fail(nullptr, EDGEFM_ERR_CUDA, "cudaGetSymbolAddress returned a null scratch address");
+        g_scratch_dev_ptr[dev] = ptr;
+    }
+    MegaKernel kern = d == 64 ? mega_kernel_g<64>(G) : mega_kernel_g<128>(G);
+
+    // ---- the same plan edgefm_create makes, on the stack ----------------------------------------------------
+    const int grid = num_sms;
+    const int max_chunks = grid / nkv > 0 ? grid / nkv : 1;
+    int max_k = H;
+    if (nq * d > max_k) max_k = nq * d;
+    if (F > max_k) max_k = F;
+    const size_t att_bytes = (static_cast<size_t>(G) * d + MK_NW * G * MK_ATT_TILE + 2 * MK_ATT_MW * G +
+                              static_cast<size_t>(MK_ATT_MW) * G * d + 2 * static_cast<size_t>(G) * max_chunks) * 4;
+    size_t xbuf = static_cast<size_t>(max_k) * 4;
+    if (att_bytes > xbuf) xbuf = att_bytes;
+    xbuf = (xbuf + 255) / 256 * 256;
+    cudaFuncAttributes fa{};
+    CUDA_TRY(nullptr, cudaFuncGetAttributes(&fa, kern));
+    const size_t static_smem = fa.sharedSizeBytes + 1024;
+    const int n_phases = 4 * sh.n_layers + 1;
+    const size_t sched = (static_cast<size_t>(n_phases) * (sizeof(MkPhase) + sizeof(int2)) + 127) / 128 * 128;
+    if (xbuf + sched + static_smem + static_cast<size_t>(MK_NW) * 1024 > static_cast<size_t>(smem_optin))
+        return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "model shape does not fit the shared-memory plan");
+    const size_t avail = smem_optin - static_smem - xbuf - sched;
+    int budget = 8192;
+    {
+        const int fit1 = static_cast<int>(avail / MK_NW / 128 * 128);
+        if (budget > fit1) budget = fit1;
+    }
+
+    // carve the scratch array; reject shapes that need more than it holds
+    ScratchCarver sc{g_scratch_dev_ptr[dev]};
+    MkPhase *d_phases = sc.take<MkPhase>(n_phases);
+    float *x = sc.take<float>(H);
+    float *q = sc.take<float>(static_cast<size_t>(nq) * d);
+    float *attn = sc.take<float>(static_cast<size_t>(nq) * d);
+    float *act = sc.take<float>(F);
+    double *inv_freq = sc.take<double>(d / 2);
+    float *part_m = sc.take<float>(static_cast<size_t>(nq) * max_chunks);
+    float *part_l = sc.take<float>(static_cast<size_t>(nq) * max_chunks);
+    float *part_o = sc.take<float>(static_cast<size_t>(nq) * max_chunks * d);
+    float *lm_val = sc.take<float>(grid);
+    int *lm_idx = sc.take<int>(grid);
+    unsigned *counters = sc.take<unsigned>(static_cast<size_t>(nq) + nkv + 2 + 64);   // tickets, then the grid barrier counter
+    StepState *state = sc.take<StepState>(1);
+    StepRequest *req = sc.take<StepRequest>(1);
+    if (sc.off > EDGEFM_STATIC_SCRATCH_BYTES)
+        return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "this shape needs %zu bytes of work buffers; the static scratch holds %zu", sc.off,
+                    EDGEFM_STATIC_SCRATCH_BYTES);
+    unsigned *tickets = counters;
+    unsigned *grid_bar = counters + nq + nkv + 2 + 32;
+
+    MkPhase phases[4 * kMaxLayers + 1];
+    int n_ph = 0, max_tile = 0;
+    bool split_overflow = false;
+    auto add = [&](int kind, const void *W, int K, int units, const void *bias, const void *norm, const float *xsrc, float *out, int layer) {
+        MkPhase ph{};
+        const bool paired = kind == PH_QKV || kind == PH_SWIGLU;
+        choose_tile(K, paired, kind == PH_QKV ? d / 2 : 4, units, grid, budget, &ph.rw, &ph.ksplit, &ph.split);
+        ph.s_shift = 0;
+        while ((1 << ph.s_shift) < ph.ksplit) ++ph.s_shift;
+        ph.W = (const uint16_t *)W; ph.bias = (const uint16_t *)bias; ph.norm_w = (const uint16_t *)norm;
+        ph.x_src = xsrc; ph.out = out; ph.K = K; ph.kind = kind; ph.kcs = K / 8 / ph.ksplit;
+        ph.units_total = units; ph.items_total = (units + ph.rw - 1) / ph.rw; ph.layer = layer;
+        const int tile = ph.rw * (paired ? 2 : 1) * ph.kcs * 16;
+        if (tile > max_tile) max_tile = tile;
+        if (ph.split) {
+            const long long per_cta = (ph.items_total + grid - 1) / grid + 1;
+            if (per_cta * ph.ksplit * (paired ? 2 : 1) > MK_PARTIAL_FLOATS) split_overflow = true;
+        }
+        phases[n_ph++] = ph;
+    };
+    for (int l = 0; l < sh.n_layers; ++l) {
+        const edgefm_layer_weights &w = weights->layers[l];
+        add(PH_QKV, w.wqkv, H, R / 2, sh.qkv_bias ? w.bqkv : nullptr, w.input_norm, l == 0 ? nullptr : x, q, l);
+        add(PH_RESID, w.wo, nq * d, H, nullptr, nullptr, attn, x, l);
+        add(PH_SWIGLU, w.w_gate_up, H, F, nullptr, w.post_norm, x, act, l);
+        add(PH_RESID, w.w_down, F, H, nullptr, nullptr, act, x, l);
+    }
+    add(PH_LMHEAD, weights->lm_head, H, sh.vocab, nullptr, weights->final_norm, x, nullptr, sh.n_layers);
+    if (split_overflow || max_tile > budget) return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "model shape does not fit the tile plan");
+    const int slot_bytes = (max_tile + 127) / 128 * 128;
+    const int ring_bytes = static_cast<int>(avail / MK_NW / 128 * 128);
+    if (slot_bytes > ring_bytes || ring_bytes > (0xffff << 4)) return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "weight rows do not fit the shared-memory ring");
+    const size_t dyn_smem = xbuf + sched + static_cast<size_t>(ring_bytes) * MK_NW;
+    // raise the kernel's dynamic shared-memory limit (a function attribute, not an allocation); repeated on every
+    // call because edgefm_create sets the same attribute for its own contexts
+    CUDA_TRY(nullptr, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(dyn_smem)));
+
+    MkParams m{};
+    m.phases = d_phases; m.nph = n_ph; m.n_layers = sh.n_layers; m.H = H; m.nq = nq; m.nkv = nkv; m.d = d; m.F = F; m.V = sh.vocab;
+    m.half_shift = d == 64 ? 5 : 6;
+    m.eps = sh.rms_eps; m.scale = static_cast<float>(1.0 / std::sqrt(static_cast<double>(d)));
+    m.max_context = max_context; m.k_cache = static_cast<uint16_t *>(k_cache); m.v_cache = static_cast<uint16_t *>(v_cache);
+    m.embed = (const uint16_t *)weights->embed; m.inv_freq = inv_freq; m.x = x; m.q = q; m.attn = attn;
+    m.part_m = part_m; m.part_l = part_l; m.part_o = part_o; m.max_chunks = max_chunks;
+    m.att_chunk_shared = 256; m.att_chunk_split = 64; m.att_split_max_n = 8192;
+    m.tickets = tickets; m.barrier = grid_bar; m.lm_part_val = lm_val; m.lm_part_idx = lm_idx; m.state = state; m.req = req;
+    m.ring_bytes = ring_bytes; m.slot_bytes = slot_bytes; m.xbuf_bytes = static_cast<int>(xbuf); m.sched_bytes = static_cast<int>(sched);
+    m.spin_limit = 1000000000u; m.prof = nullptr; m.prof_stride = 0;
+
+    // ---- stream-ordered set-up of the shared scratch: it still holds the previous call's contents ----------
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    double inv[64];
+    for (int i = 0; i < d / 2; ++i) inv[i] = std::pow(static_cast<double>(sh.rope_theta), -2.0 * i / d);
+    StepState st{};
+    st.cur_len = cur_len; st.next_position = position;
+    StepRequest rq{token_id, position, logits_out, next_token_out};
+    // counters (attention tickets, lm_head ticket, grid barrier) must start at zero
+    CUDA_TRY(nullptr, cudaMemsetAsync(counters, 0, (static_cast<size_t>(nq) + nkv + 2 + 64) * sizeof(unsigned), s));
+    // small pageable copies: the runtime stages the bytes before returning, so stack sources are fine
+    CUDA_TRY(nullptr, cudaMemcpyAsync(d_phases, phases, static_cast<size_t>(n_ph) * sizeof(MkPhase), cudaMemcpyHostToDevice, s));
+    CUDA_TRY(nullptr, cudaMemcpyAsync(inv_freq, inv, static_cast<size_t>(d / 2) * sizeof(double), cudaMemcpyHostToDevice, s));
+    CUDA_TRY(nullptr, cudaMemcpyAsync(state, &st, sizeof st, cudaMemcpyHostToDevice, s));
+    CUDA_TRY(nullptr, cudaMemcpyAsync(req, &rq, sizeof rq, cudaMemcpyHostToDevice, s));
+
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(MK_NT);
+    cfg.dynamicSmemBytes = dyn_smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    CUDA_TRY(nullptr, cudaLaunchKernelEx(&cfg, kern, m));
+    g_create_error.clear();
+    return EDGEFM_OK;
+}
