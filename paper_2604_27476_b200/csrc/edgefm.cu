@@ -167,17 +167,20 @@ AttnPlan make_attn_plan_g(int G, cudaError_t *err) {
 
 using MegaKernel = void (*)(const MkParams);
 
+// long_ctx = false: the variant without the grouped (one CTA per GQA group) attention code, for contexts that
+// never need it.
 template <int D>
-MegaKernel mega_kernel_g(int G) {
+MegaKernel mega_kernel_g(int G, bool long_ctx) {
+    if (!long_ctx) return decode_megakernel<D, 1, false>;   // G is only used by the grouped attention
     switch (G) {
-        case 1: return decode_megakernel<D, 1>;
-        case 2: return decode_megakernel<D, 2>;
-        case 3: return decode_megakernel<D, 3>;
-        case 4: return decode_megakernel<D, 4>;
-        case 5: return decode_megakernel<D, 5>;
-        case 6: return decode_megakernel<D, 6>;
-        case 7: return decode_megakernel<D, 7>;
-        case 8: return decode_megakernel<D, 8>;
+        case 1: return decode_megakernel<D, 1, true>;
+        case 2: return decode_megakernel<D, 2, true>;
+        case 3: return decode_megakernel<D, 3, true>;
+        case 4: return decode_megakernel<D, 4, true>;
+        case 5: return decode_megakernel<D, 5, true>;
+        case 6: return decode_megakernel<D, 6, true>;
+        case 7: return decode_megakernel<D, 7, true>;
+        case 8: return decode_megakernel<D, 8, true>;
     }
     return nullptr;
 }
@@ -498,7 +501,8 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
     }
     std::vector<MkPhase> phases;
     if (c->use_mega) {
-        c->mega = d == 64 ? mega_kernel_g<64>(G) : mega_kernel_g<128>(G);
+        const bool long_ctx = max_context > 8192 || static_cast<long long>(nq) * MK_ATT_SPLIT_MAXC * 2 > MK_PARTIAL_FLOATS;
+        c->mega = d == 64 ? mega_kernel_g<64>(G, long_ctx) : mega_kernel_g<128>(G, long_ctx);
         int smem_optin = 0, coop = 0;
         CREATE_TRY(cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
         CREATE_TRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
@@ -629,7 +633,9 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
         m.nph = static_cast<int>(phases.size());
         m.half_shift = d == 64 ? 5 : 6;
         m.att_chunk_shared = 256; m.att_chunk_split = 64; m.att_split_max_n = 8192;
-        if (const char *ac = getenv("EDGEFM_ATT_SPLIT_MAX")) { const int v = atoi(ac); if (v >= 0) m.att_split_max_n = v; }
+        if (max_context > 8192) {   // only the long-context kernel variant has both attention modes
+            if (const char *ac = getenv("EDGEFM_ATT_SPLIT_MAX")) { const int v = atoi(ac); if (v >= 0) m.att_split_max_n = v; }
+        }
         if (const char *ac = getenv("EDGEFM_ATT_CHUNK")) { const int v = atoi(ac); if (v >= 8) { m.att_chunk_shared = v; m.att_chunk_split = v; } }
         m.lm_part_val = c->lm_part_val; m.lm_part_idx = c->lm_part_idx; m.state = c->state; m.req = c->req;
         m.spin_limit = 1000000000u;  // 1 s
@@ -851,7 +857,8 @@ extern "C" edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, co
         if (!ptr) return fail(nullptr, EDGEFM_ERR_CUDA, "cudaGetSymbolAddress returned a null scratch address");
         g_scratch_dev_ptr[dev] = ptr;
     }
-    MegaKernel kern = d == 64 ? mega_kernel_g<64>(G) : mega_kernel_g<128>(G);
+    const bool long_ctx = max_context > 8192 || static_cast<long long>(nq) * MK_ATT_SPLIT_MAXC * 2 > MK_PARTIAL_FLOATS;
+    MegaKernel kern = d == 64 ? mega_kernel_g<64>(G, long_ctx) : mega_kernel_g<128>(G, long_ctx);
 
     // ---- the same plan edgefm_create makes, on the stack ----------------------------------------------------
     const int grid = num_sms;

@@ -905,7 +905,10 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
 }
 
 // ---- the kernel -----------------------------------------------------------------------------------------------
-template <int D, int G>
+// LONG = false: contexts that always run attention with one query head per CTA group (max_context <=
+// att_split_max_n); the grouped variant is then not compiled in, which keeps the register footprint of the
+// streaming state small.
+template <int D, int G, bool LONG>
 __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) {
     extern __shared__ __align__(128) unsigned char mk_smem[];
     unsigned char *smem = mk_smem;
@@ -990,15 +993,19 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
     prof_stamp(p, tid, prof_idx);
     auto top_up = [&]() { __syncwarp(); if (ok && !*abort_flag) refill(p, s_ph, s_rng, ws, abort_flag, warp, lane); };
     const int n_att = slot_row + 1;
-    const bool att_split = n_att <= p.att_split_max_n && static_cast<long long>(p.nq) * MK_ATT_SPLIT_MAXC * 2 <= MK_PARTIAL_FLOATS;
+    const bool att_split = !LONG || (n_att <= p.att_split_max_n && static_cast<long long>(p.nq) * MK_ATT_SPLIT_MAXC * 2 <= MK_PARTIAL_FLOATS);
     int merge_chunks = 0;   // chunks per head the O-projection prologue has to merge (split mode)
     if (att_split) { int cl; att_chunking(p, n_att, 1, p.att_chunk_split, ncta, merge_chunks, cl); }
     for (int l = 0; l < p.n_layers && ok; ++l) {
         ok = gemv_phase(p, s_ph, s_rng, 4 * l, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token, 0, tid, prof_idx);
         ok = grid_barrier(p, ++bar_no * ncta, abort_flag, &s_released, tid, prof_idx, top_up) && ok;
         if (ok) {
-            if (att_split) attention_phase<D, 1>(p, l, n_att, p.att_chunk_split, true, smem, tid, &s_flag);
-            else attention_phase<D, G>(p, l, n_att, p.att_chunk_shared, false, smem, tid, &s_flag);
+            if constexpr (LONG) {
+                if (att_split) attention_phase<D, 1>(p, l, n_att, p.att_chunk_split, true, smem, tid, &s_flag);
+                else attention_phase<D, G>(p, l, n_att, p.att_chunk_shared, false, smem, tid, &s_flag);
+            } else {
+                attention_phase<D, 1>(p, l, n_att, p.att_chunk_split, true, smem, tid, &s_flag);
+            }
         }
         ok = grid_barrier(p, ++bar_no * ncta, abort_flag, &s_released, tid, prof_idx, top_up) && ok;
         for (int k = 1; k < 4 && ok; ++k) {
