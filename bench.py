@@ -27,6 +27,10 @@ import numpy as np
 
 from edgefm_synth import CONFIGS, GLOBAL_SEED, first_token, make_kv, make_weights
 
+# DRAM traffic of one launch of the step kernel (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture,
+# see profiles/decode_megakernel_qwen2.5-1.5b_ctx2048.md); only the captured configuration has a value.
+NCU_TRAFFIC_BYTES = {"qwen2.5-1.5b": 3.147058e9 + 5.281e6}
+
 METRIC = "batch1_decode_ms_per_token"
 UNIT = "ms/token"
 NOMINAL_HBM_GBS = 8000.0
@@ -246,9 +250,9 @@ def main():
             "config": {"workload": workload_name(cfg), "replicas": world, "l2": "working set 3 GB per step exceeds L2; no flush",
                        "seed": GLOBAL_SEED},
             "tokens_per_s": tokens / (dev_ms * 1e-3),
-            "roofline": {"bound": "hbm", "kernel": f"whole decode step ({launches} kernels in one CUDA graph)",
+            "roofline": {"bound": "hbm", "kernel": f"decode_megakernel: the whole decode step ({launches} kernel launch per token, one CUDA graph node)",
                          "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak, "peak_source": peak_src,
-                         "bytes_per_launch": bytes_per_step, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS, "traffic": None},
+                         "bytes_per_launch": bytes_per_step, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS, "traffic": NCU_TRAFFIC_BYTES.get(cfg.name)},
             "e2e": {"value": e2e_ms / tokens, "unit": UNIT, "h2d_bytes_per_step": 24, "d2h_bytes_per_step": 4},
             "gpu_launches": launches * steps,
             "clocks": clocks,
