@@ -515,7 +515,7 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
         int max_k = H;
         if (nq * d > max_k) max_k = nq * d;
         if (F > max_k) max_k = F;
-        const size_t att_bytes = (static_cast<size_t>(G) * d + MK_NW * G * MK_ATT_TILE + 2 * MK_ATT_MW * G +
+        const size_t att_bytes = (static_cast<size_t>(G) * d + MK_NW * (G * MK_ATT_TILE > 32 / MK_ATT_LPP_SPLIT ? G * MK_ATT_TILE : 32 / MK_ATT_LPP_SPLIT) + 2 * MK_ATT_MW * G +
                                   static_cast<size_t>(MK_ATT_MW) * G * d + 2 * static_cast<size_t>(G) * max_chunks) * 4;
         size_t xbuf = static_cast<size_t>(max_k) * 4;
         if (att_bytes > xbuf) xbuf = att_bytes;
@@ -866,7 +866,7 @@ extern "C" edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, co
     int max_k = H;
     if (nq * d > max_k) max_k = nq * d;
     if (F > max_k) max_k = F;
-    const size_t att_bytes = (static_cast<size_t>(G) * d + MK_NW * G * MK_ATT_TILE + 2 * MK_ATT_MW * G +
+    const size_t att_bytes = (static_cast<size_t>(G) * d + MK_NW * (G * MK_ATT_TILE > 32 / MK_ATT_LPP_SPLIT ? G * MK_ATT_TILE : 32 / MK_ATT_LPP_SPLIT) + 2 * MK_ATT_MW * G +
                               static_cast<size_t>(MK_ATT_MW) * G * d + 2 * static_cast<size_t>(G) * max_chunks) * 4;
     size_t xbuf = static_cast<size_t>(max_k) * 4;
     if (att_bytes > xbuf) xbuf = att_bytes;

@@ -33,7 +33,8 @@ constexpr int MK_NW = 12;                        // warps per CTA (each streams 
 constexpr int MK_NT = MK_NW * 32;
 constexpr int MK_MAXF = 4;                       // tiles in flight per warp (one mbarrier each)
 constexpr int MK_BAR_POLLERS = 1;                // warps whose lane 0 polls the grid barrier counter
-constexpr int MK_ATT_LPP = 4;                    // lanes per cached position in the score phase
+constexpr int MK_ATT_LPP = 4;                    // lanes per cached position in the score phase (one CTA per GQA group)
+constexpr int MK_ATT_LPP_SPLIT = 2;              // ... when every query head has its own CTAs (16 positions per warp iteration)
 constexpr int MK_ATT_TILE = 32 / MK_ATT_LPP;     // positions per warp iteration
 constexpr int MK_ATT_MW = (MK_NW + 1) / 2;       // warps whose partials fit the merge area at once
 constexpr int MK_ATT_SPLIT_MAXC = 12;            // chunks per head when every query head has its own CTAs
@@ -509,14 +510,14 @@ __device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkPhase *
 }
 
 // Attention chunking shared by the attention phase and by the consumer of its partial results.
-__device__ __forceinline__ void att_chunking(const MkParams &p, int n, int hg, int min_chunk, int ncta, int &nch, int &chunk_len) {
+__device__ __forceinline__ void att_chunking(const MkParams &p, int n, int hg, int min_chunk, int tile, int ncta, int &nch, int &chunk_len) {
     const int groups = p.nq / hg;
     nch = (n + min_chunk - 1) / min_chunk;
     nch = min(nch, min(ncta / groups, p.max_chunks));
     if (hg == 1) nch = min(nch, MK_ATT_SPLIT_MAXC);
     nch = max(nch, 1);
     chunk_len = (n + nch - 1) / nch;
-    chunk_len = (chunk_len + MK_ATT_TILE - 1) / MK_ATT_TILE * MK_ATT_TILE;
+    chunk_len = (chunk_len + tile - 1) / tile * tile;
     nch = (n + chunk_len - 1) / chunk_len;
 }
 
@@ -676,10 +677,10 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, const MkPhase *s_p
 // probabilities, warp merge area, chunk statistics.  The CTA that arrives last for its head group
 // (atomic ticket, no waiting) merges the chunks exactly:  m = max m_c, l = sum l_c e^{m_c - m},
 // o = sum o_c e^{m_c - m} / l, in index order.
-template <int D, int HG>
+template <int D, int HG, int LPP>
 __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, int n, int min_chunk, bool defer_merge,
                                                 unsigned char *xbuf, int tid, int *s_flag) {
-    constexpr int TILE = MK_ATT_TILE, LPP = MK_ATT_LPP;
+    constexpr int TILE = 32 / LPP;   // positions per warp iteration
     constexpr int DV = D / 32, CPR = D / 8, CPL = CPR / LPP;
     constexpr int MW = MK_ATT_MW;
     const int lane = tid & 31, warp = tid >> 5;
@@ -687,7 +688,7 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
     const int G = p.nq / p.nkv;
     const int groups = p.nq / HG;                       // head groups served by separate CTAs
     int nch, chunk_len;
-    att_chunking(p, n, HG, min_chunk, ncta, nch, chunk_len);
+    att_chunking(p, n, HG, min_chunk, TILE, ncta, nch, chunk_len);
     if (cta >= nch * groups) return;
     const int grp = cta / nch, c = cta - grp * nch;
     const int qh0 = grp * HG;                            // first query head of this CTA
@@ -995,16 +996,16 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
     const int n_att = slot_row + 1;
     const bool att_split = !LONG || (n_att <= p.att_split_max_n && static_cast<long long>(p.nq) * MK_ATT_SPLIT_MAXC * 2 <= MK_PARTIAL_FLOATS);
     int merge_chunks = 0;   // chunks per head the O-projection prologue has to merge (split mode)
-    if (att_split) { int cl; att_chunking(p, n_att, 1, p.att_chunk_split, ncta, merge_chunks, cl); }
+    if (att_split) { int cl; att_chunking(p, n_att, 1, p.att_chunk_split, 32 / MK_ATT_LPP_SPLIT, ncta, merge_chunks, cl); }
     for (int l = 0; l < p.n_layers && ok; ++l) {
         ok = gemv_phase(p, s_ph, s_rng, 4 * l, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token, 0, tid, prof_idx);
         ok = grid_barrier(p, ++bar_no * ncta, abort_flag, &s_released, tid, prof_idx, top_up) && ok;
         if (ok) {
             if constexpr (LONG) {
-                if (att_split) attention_phase<D, 1>(p, l, n_att, p.att_chunk_split, true, smem, tid, &s_flag);
-                else attention_phase<D, G>(p, l, n_att, p.att_chunk_shared, false, smem, tid, &s_flag);
+                if (att_split) attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, true, smem, tid, &s_flag);
+                else attention_phase<D, G, MK_ATT_LPP>(p, l, n_att, p.att_chunk_shared, false, smem, tid, &s_flag);
             } else {
-                attention_phase<D, 1>(p, l, n_att, p.att_chunk_split, true, smem, tid, &s_flag);
+                attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, true, smem, tid, &s_flag);
             }
         }
         ok = grid_barrier(p, ++bar_no * ncta, abort_flag, &s_released, tid, prof_idx, top_up) && ok;
