@@ -40,7 +40,8 @@ typedef enum {
     EDGEFM_ERR_CONTEXT_FULL = 3,  /* the KV cache has no free slot / prefill longer than max_context */
     EDGEFM_ERR_OUT_OF_MEMORY = 4, /* device or host allocation failed                                */
     EDGEFM_ERR_CUDA = 5,          /* a CUDA runtime call failed; see edgefm_last_error               */
-    EDGEFM_ERR_TIMEOUT = 6        /* reserved: a bounded device-side wait expired                     */
+    EDGEFM_ERR_TIMEOUT = 6        /* a bounded device-side wait expired or a device self-check failed
+                                     (reported by edgefm_sync_status)                                 */
 } edgefm_status;
 
 /* Model shape (the public Qwen2.5 decoder block). */

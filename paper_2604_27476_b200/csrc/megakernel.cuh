@@ -155,9 +155,6 @@ __device__ __forceinline__ void bulk_copy_g2s(void *dst, const void *src, unsign
         ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
         : "memory");
 }
-__device__ __forceinline__ void bulk_prefetch_l2(const void *src, unsigned bytes) {
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
-}
 __device__ __forceinline__ void cta_sync() { __syncthreads(); }
 
 __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned *p) {
