@@ -13,7 +13,18 @@
 #include "attention.cuh"
 #include "common.cuh"
 #include "gemv.cuh"
+#include "megakernel_types.cuh"
+// the persistent kernel, built twice: 12 warps per CTA (short contexts) and 8 warps per CTA (long contexts)
+#define MK_NS mk_short
+#define MK_NW_VALUE MK_NW_SHORT
 #include "megakernel.cuh"
+#undef MK_NS
+#undef MK_NW_VALUE
+#define MK_NS mk_long
+#define MK_NW_VALUE MK_NW_LONG
+#include "megakernel.cuh"
+#undef MK_NS
+#undef MK_NW_VALUE
 
 namespace edgefm {
 
@@ -171,16 +182,16 @@ using MegaKernel = void (*)(const MkParams);
 // never need it.
 template <int D>
 MegaKernel mega_kernel_g(int G, bool long_ctx) {
-    if (!long_ctx) return decode_megakernel<D, 1, false>;   // G is only used by the grouped attention
+    if (!long_ctx) return mk_short::decode_megakernel<D, 1, false>;   // G is only used by the grouped attention
     switch (G) {
-        case 1: return decode_megakernel<D, 1, true>;
-        case 2: return decode_megakernel<D, 2, true>;
-        case 3: return decode_megakernel<D, 3, true>;
-        case 4: return decode_megakernel<D, 4, true>;
-        case 5: return decode_megakernel<D, 5, true>;
-        case 6: return decode_megakernel<D, 6, true>;
-        case 7: return decode_megakernel<D, 7, true>;
-        case 8: return decode_megakernel<D, 8, true>;
+        case 1: return mk_long::decode_megakernel<D, 1, true>;
+        case 2: return mk_long::decode_megakernel<D, 2, true>;
+        case 3: return mk_long::decode_megakernel<D, 3, true>;
+        case 4: return mk_long::decode_megakernel<D, 4, true>;
+        case 5: return mk_long::decode_megakernel<D, 5, true>;
+        case 6: return mk_long::decode_megakernel<D, 6, true>;
+        case 7: return mk_long::decode_megakernel<D, 7, true>;
+        case 8: return mk_long::decode_megakernel<D, 8, true>;
     }
     return nullptr;
 }
@@ -191,23 +202,23 @@ MegaKernel mega_kernel_g(int G, bool long_ctx) {
 //  * short operators, and rows longer than a slot: one row (pair) per item, cut into `ksplit` K slices
 //    (a power of two dividing the row) that go to different warps, so that all warps of a CTA share the
 //    latency of the operator; their partial sums meet in shared memory.
-inline void choose_tile(int K, bool paired, int pair_align, int units, int ncta, int budget_bytes, int *rw, int *ksplit, int *split) {
+inline void choose_tile(int K, bool paired, int pair_align, int units, int ncta, int nw, int budget_bytes, int *rw, int *ksplit, int *split) {
     const int kc = K / 8;
     const int mult = paired ? 2 : 1;
     const long long row_bytes = static_cast<long long>(K) * 2 * mult;
     const double per_cta = static_cast<double>(units) / ncta;
     *rw = 1; *ksplit = 1; *split = 0;
-    if (row_bytes <= budget_bytes && per_cta >= 2.0 * MK_NW) {
+    if (row_bytes <= budget_bytes && per_cta >= 2.0 * nw) {
         int r = paired ? 4 : 8;
-        while (r > 1 && (row_bytes * r > budget_bytes || (paired && pair_align % r != 0) || per_cta / r < 2.0 * MK_NW)) r >>= 1;
+        while (r > 1 && (row_bytes * r > budget_bytes || (paired && pair_align % r != 0) || per_cta / r < 2.0 * nw)) r >>= 1;
         *rw = r;
         return;
     }
     int s = 1;
     auto can_double = [&](int min_kcs) { return kc % (2 * s) == 0 && kc / (2 * s) >= min_kcs && 2 * s <= 16; };
     while (row_bytes / s > budget_bytes && kc % (2 * s) == 0) s *= 2;           // must fit a slot
-    while (per_cta * s < MK_NW && can_double(64)) s *= 2;                       // at least one tile per warp
-    while (per_cta * s < 2.0 * MK_NW && can_double(256)) s *= 2;                // two per warp while slices stay long
+    while (per_cta * s < nw && can_double(64)) s *= 2;                       // at least one tile per warp
+    while (per_cta * s < 2.0 * nw && can_double(256)) s *= 2;                // two per warp while slices stay long
     *ksplit = s;
     *split = s > 1 ? 1 : 0;
 }
@@ -254,6 +265,7 @@ struct edgefm_ctx {
     int prof_stride = 0;
     MkParams mk{};
     size_t mega_smem = 0;
+    int mega_threads = 0;
     int mega_grid = 0;
 
     cudaStream_t build_stream = nullptr;
@@ -328,7 +340,7 @@ cudaError_t enqueue_step(edgefm_ctx *c, cudaStream_t s, int *n_launches) {
         // one cooperative launch: all CTAs are co-resident, which the grid barriers rely on
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(c->mega_grid);
-        cfg.blockDim = dim3(MK_NT);
+        cfg.blockDim = dim3(c->mega_threads);
         cfg.dynamicSmemBytes = c->mega_smem;
         cfg.stream = s;
         cudaLaunchAttribute attr[1];
@@ -503,6 +515,9 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
     if (c->use_mega) {
         const bool long_ctx = max_context > 8192 || static_cast<long long>(nq) * MK_ATT_SPLIT_MAXC * 2 > MK_PARTIAL_FLOATS;
         c->mega = d == 64 ? mega_kernel_g<64>(G, long_ctx) : mega_kernel_g<128>(G, long_ctx);
+        const int NW = long_ctx ? MK_NW_LONG : MK_NW_SHORT;   // warps per CTA of the chosen build
+        const int ATT_MW = (NW + 1) / 2;
+        c->mega_threads = NW * 32;
         int smem_optin = 0, coop = 0;
         CREATE_TRY(cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
         CREATE_TRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
@@ -515,8 +530,8 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
         int max_k = H;
         if (nq * d > max_k) max_k = nq * d;
         if (F > max_k) max_k = F;
-        const size_t att_bytes = (static_cast<size_t>(G) * d + MK_NW * (G * MK_ATT_TILE > 32 / MK_ATT_LPP_SPLIT ? G * MK_ATT_TILE : 32 / MK_ATT_LPP_SPLIT) + 2 * MK_ATT_MW * G +
-                                  static_cast<size_t>(MK_ATT_MW) * G * d + 2 * static_cast<size_t>(G) * max_chunks) * 4;
+        const size_t att_bytes = (static_cast<size_t>(G) * d + NW * (G * MK_ATT_TILE > 32 / MK_ATT_LPP_SPLIT ? G * MK_ATT_TILE : 32 / MK_ATT_LPP_SPLIT) + 2 * ATT_MW * G +
+                                  static_cast<size_t>(ATT_MW) * G * d + 2 * static_cast<size_t>(G) * max_chunks) * 4;
         size_t xbuf = static_cast<size_t>(max_k) * 4;
         if (att_bytes > xbuf) xbuf = att_bytes;
         xbuf = (xbuf + 255) / 256 * 256;
@@ -525,14 +540,14 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
         const size_t static_smem = fa.sharedSizeBytes + 1024;  // the kernel's static shared memory (mbarriers, tables, scratch) + margin
         const size_t n_phases = 4 * static_cast<size_t>(sh.n_layers) + 1;
         const size_t sched = (n_phases * (sizeof(MkPhase) + sizeof(int2)) + 127) / 128 * 128;
-        if (xbuf + sched + static_smem + static_cast<size_t>(MK_NW) * 1024 > static_cast<size_t>(smem_optin))
+        if (xbuf + sched + static_smem + static_cast<size_t>(NW) * 1024 > static_cast<size_t>(smem_optin))
             return bail(EDGEFM_ERR_CUDA, "model shape does not fit the shared-memory plan", cudaErrorInvalidValue);
         const size_t avail = smem_optin - static_smem - xbuf - sched;
         // ring: `depth` slots per warp; prefer two slots of a natural tile size, deeper rings for small tiles
         int budget = 8192;   // upper bound of one tile
         if (const char *tb = getenv("EDGEFM_TILE_BYTES")) { const int v = atoi(tb); if (v >= 1024 && v <= 65536) budget = v; }
         {
-            const int fit1 = static_cast<int>(avail / MK_NW / 128 * 128);   // a tile must fit a warp's ring
+            const int fit1 = static_cast<int>(avail / NW / 128 * 128);   // a tile must fit a warp's ring
             if (budget > fit1) budget = fit1;
         }
         int max_tile = 0;
@@ -541,7 +556,7 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
                        float *out, int layer) {
             MkPhase ph{};
             const bool paired = kind == PH_QKV || kind == PH_SWIGLU;
-            choose_tile(K, paired, kind == PH_QKV ? d / 2 : 4, units, c->mega_grid, budget, &ph.rw, &ph.ksplit, &ph.split);
+            choose_tile(K, paired, kind == PH_QKV ? d / 2 : 4, units, c->mega_grid, NW, budget, &ph.rw, &ph.ksplit, &ph.split);
             ph.s_shift = 0;
             while ((1 << ph.s_shift) < ph.ksplit) ++ph.s_shift;
             ph.W = (const uint16_t *)W; ph.bias = (const uint16_t *)bias; ph.norm_w = (const uint16_t *)norm;
@@ -567,15 +582,15 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
         if (split_overflow || max_tile > budget)
             return bail(EDGEFM_ERR_CUDA, "model shape does not fit the tile plan", cudaErrorInvalidValue);
         const int slot_bytes = (max_tile + 127) / 128 * 128;
-        const int ring_bytes = static_cast<int>(avail / MK_NW / 128 * 128);
+        const int ring_bytes = static_cast<int>(avail / NW / 128 * 128);
         if (slot_bytes > ring_bytes || ring_bytes > (0xffff << 4))
             return bail(EDGEFM_ERR_CUDA, "weight rows do not fit the shared-memory ring", cudaErrorInvalidValue);
         c->mk.ring_bytes = ring_bytes; c->mk.slot_bytes = slot_bytes; c->mk.xbuf_bytes = static_cast<int>(xbuf);
         c->mk.sched_bytes = static_cast<int>(sched);
-        c->mega_smem = xbuf + sched + static_cast<size_t>(ring_bytes) * MK_NW;
+        c->mega_smem = xbuf + sched + static_cast<size_t>(ring_bytes) * NW;
         CREATE_TRY(cudaFuncSetAttribute(c->mega, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(c->mega_smem)));
         int per_sm = 0;
-        CREATE_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, c->mega, MK_NT, c->mega_smem));
+        CREATE_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, c->mega, c->mega_threads, c->mega_smem));
         if (per_sm < 1) return bail(EDGEFM_ERR_CUDA, "persistent kernel does not fit one CTA per SM", cudaErrorInvalidValue);
         c->p_attn.max_chunks = max_chunks;  // sizes the partial buffers below
         c->p_lm.grid = c->mega_grid;
@@ -642,8 +657,8 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
         const char *pe_ = getenv("EDGEFM_PROFILE");
         if (pe_ && pe_[0] == '1') {
             c->prof_stride = 3 + 14 * sh.n_layers;
-            CREATE_TRY(dev_alloc(&c->prof, static_cast<size_t>(c->mega_grid + 1) * c->prof_stride + MK_NW * 16));
-            CREATE_TRY(cudaMemset(c->prof, 0, (static_cast<size_t>(c->mega_grid + 1) * c->prof_stride + MK_NW * 16) * 8));
+            CREATE_TRY(dev_alloc(&c->prof, static_cast<size_t>(c->mega_grid + 1) * c->prof_stride + MK_NW_SHORT * 16));
+            CREATE_TRY(cudaMemset(c->prof, 0, (static_cast<size_t>(c->mega_grid + 1) * c->prof_stride + MK_NW_SHORT * 16) * 8));
             m.prof = c->prof; m.prof_stride = c->prof_stride;
         }
     }
@@ -741,7 +756,7 @@ edgefm_status edgefm_debug_profile(edgefm_ctx *ctx, uint64_t *out_host, int64_t 
     *stride = ctx->prof_stride;
     if (!ctx->prof || !out_host) return EDGEFM_OK;
     int64_t n = static_cast<int64_t>(ctx->mega_grid) * ctx->prof_stride;
-    if (capacity >= n + MK_NW * 16) n += MK_NW * 16;   // optional per-warp trace behind the table
+    if (capacity >= n + MK_NW_SHORT * 16) n += MK_NW_SHORT * 16;   // optional per-warp trace behind the table
     if (capacity < n) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "profile buffer too small");
     DeviceGuard guard(ctx->device);
     CUDA_TRY(ctx, cudaDeviceSynchronize());
@@ -859,6 +874,8 @@ extern "C" edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, co
     }
     const bool long_ctx = max_context > 8192 || static_cast<long long>(nq) * MK_ATT_SPLIT_MAXC * 2 > MK_PARTIAL_FLOATS;
     MegaKernel kern = d == 64 ? mega_kernel_g<64>(G, long_ctx) : mega_kernel_g<128>(G, long_ctx);
+    const int NW = long_ctx ? MK_NW_LONG : MK_NW_SHORT;   // warps per CTA of the chosen build
+    const int ATT_MW = (NW + 1) / 2;
 
     // ---- the same plan edgefm_create makes, on the stack ----------------------------------------------------
     const int grid = num_sms;
@@ -866,8 +883,8 @@ extern "C" edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, co
     int max_k = H;
     if (nq * d > max_k) max_k = nq * d;
     if (F > max_k) max_k = F;
-    const size_t att_bytes = (static_cast<size_t>(G) * d + MK_NW * (G * MK_ATT_TILE > 32 / MK_ATT_LPP_SPLIT ? G * MK_ATT_TILE : 32 / MK_ATT_LPP_SPLIT) + 2 * MK_ATT_MW * G +
-                              static_cast<size_t>(MK_ATT_MW) * G * d + 2 * static_cast<size_t>(G) * max_chunks) * 4;
+    const size_t att_bytes = (static_cast<size_t>(G) * d + NW * (G * MK_ATT_TILE > 32 / MK_ATT_LPP_SPLIT ? G * MK_ATT_TILE : 32 / MK_ATT_LPP_SPLIT) + 2 * ATT_MW * G +
+                              static_cast<size_t>(ATT_MW) * G * d + 2 * static_cast<size_t>(G) * max_chunks) * 4;
     size_t xbuf = static_cast<size_t>(max_k) * 4;
     if (att_bytes > xbuf) xbuf = att_bytes;
     xbuf = (xbuf + 255) / 256 * 256;
@@ -876,12 +893,12 @@ extern "C" edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, co
     const size_t static_smem = fa.sharedSizeBytes + 1024;
     const int n_phases = 4 * sh.n_layers + 1;
     const size_t sched = (static_cast<size_t>(n_phases) * (sizeof(MkPhase) + sizeof(int2)) + 127) / 128 * 128;
-    if (xbuf + sched + static_smem + static_cast<size_t>(MK_NW) * 1024 > static_cast<size_t>(smem_optin))
+    if (xbuf + sched + static_smem + static_cast<size_t>(NW) * 1024 > static_cast<size_t>(smem_optin))
         return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "model shape does not fit the shared-memory plan");
     const size_t avail = smem_optin - static_smem - xbuf - sched;
     int budget = 8192;
     {
-        const int fit1 = static_cast<int>(avail / MK_NW / 128 * 128);
+        const int fit1 = static_cast<int>(avail / NW / 128 * 128);
         if (budget > fit1) budget = fit1;
     }
 
@@ -913,7 +930,7 @@ extern "C" edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, co
     auto add = [&](int kind, const void *W, int K, int units, const void *bias, const void *norm, const float *xsrc, float *out, int layer) {
         MkPhase ph{};
         const bool paired = kind == PH_QKV || kind == PH_SWIGLU;
-        choose_tile(K, paired, kind == PH_QKV ? d / 2 : 4, units, grid, budget, &ph.rw, &ph.ksplit, &ph.split);
+        choose_tile(K, paired, kind == PH_QKV ? d / 2 : 4, units, grid, NW, budget, &ph.rw, &ph.ksplit, &ph.split);
         ph.s_shift = 0;
         while ((1 << ph.s_shift) < ph.ksplit) ++ph.s_shift;
         ph.W = (const uint16_t *)W; ph.bias = (const uint16_t *)bias; ph.norm_w = (const uint16_t *)norm;
@@ -937,9 +954,9 @@ extern "C" edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, co
     add(PH_LMHEAD, weights->lm_head, H, sh.vocab, nullptr, weights->final_norm, x, nullptr, sh.n_layers);
     if (split_overflow || max_tile > budget) return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "model shape does not fit the tile plan");
     const int slot_bytes = (max_tile + 127) / 128 * 128;
-    const int ring_bytes = static_cast<int>(avail / MK_NW / 128 * 128);
+    const int ring_bytes = static_cast<int>(avail / NW / 128 * 128);
     if (slot_bytes > ring_bytes || ring_bytes > (0xffff << 4)) return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "weight rows do not fit the shared-memory ring");
-    const size_t dyn_smem = xbuf + sched + static_cast<size_t>(ring_bytes) * MK_NW;
+    const size_t dyn_smem = xbuf + sched + static_cast<size_t>(ring_bytes) * NW;
     // raise the kernel's dynamic shared-memory limit (a function attribute, not an allocation); repeated on every
     // call because edgefm_create sets the same attribute for its own contexts
     CUDA_TRY(nullptr, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(dyn_smem)));
@@ -973,7 +990,7 @@ extern "C" edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, co
 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(MK_NT);
+    cfg.blockDim = dim3(NW * 32);
     cfg.dynamicSmemBytes = dyn_smem;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];

@@ -24,91 +24,30 @@
 //
 // Every wait is bounded: on expiry the CTA records EDGEFM_ERR_TIMEOUT in the device state, stops
 // issuing copies, waits (bounded) for the copies it has in flight and returns.
-#pragma once
-#include "common.cuh"
+// This file is the body of the kernel.  It is included once per build (MK_NS = namespace, MK_NW_VALUE = warps per
+// CTA); everything that does not depend on the number of warps lives in megakernel_types.cuh.
+#include "megakernel_types.cuh"
 
 namespace edgefm {
+namespace MK_NS {
 
-constexpr int MK_NW = 12;                        // warps per CTA (each streams and consumes its own tiles)
+constexpr int MK_NW = MK_NW_VALUE;               // warps per CTA (each streams and consumes its own tiles)
 constexpr int MK_NT = MK_NW * 32;
-constexpr int MK_MAXF = 4;                       // tiles in flight per warp (one mbarrier each)
-constexpr int MK_BAR_POLLERS = 1;                // warps whose lane 0 polls the grid barrier counter
-constexpr int MK_ATT_LPP = 4;                    // lanes per cached position in the score phase (one CTA per GQA group)
-constexpr int MK_ATT_LPP_SPLIT = 2;              // ... when every query head has its own CTAs (16 positions per warp iteration)
-constexpr int MK_ATT_TILE = 32 / MK_ATT_LPP;     // positions per warp iteration
 constexpr int MK_ATT_MW = (MK_NW + 1) / 2;       // warps whose partials fit the merge area at once
-constexpr int MK_ATT_SPLIT_MAXC = 12;            // chunks per head when every query head has its own CTAs
-constexpr int MK_PARTIAL_FLOATS = 2048;          // shared-memory scratch: split-K partial sums / chunk statistics
-
-enum { PH_QKV = 0, PH_RESID = 1, PH_SWIGLU = 2, PH_LMHEAD = 3 };
-
-// One weight-streaming operator of the step.
-struct alignas(16) MkPhase {
-    const uint16_t *W;       // bf16 [rows][K]
-    const uint16_t *bias;    // PH_QKV: bf16 [rows] or null
-    const uint16_t *norm_w;  // RMSNorm weight of the prologue (bf16 [K]) or null = plain copy of x_src
-    const float *x_src;      // fp32 [K] input vector in global memory; null = embedding row of the token
-    float *out;              // PH_QKV: q fp32; PH_RESID: x (+=); PH_SWIGLU: act; PH_LMHEAD: unused
-    int K;                   // columns (multiple of 8)
-    int kind;
-    int rw;                  // units per work item (rows, or row pairs for PH_QKV / PH_SWIGLU); 1 when split
-    int ksplit;              // K slices per item (tiles per item)
-    int kcs;                 // 16-byte pieces per row slice = K / 8 / ksplit
-    int units_total;         // rows (PH_RESID, PH_LMHEAD), pairs (PH_QKV: rows/2, PH_SWIGLU: F)
-    int items_total;         // ceil(units_total / rw)
-    int layer;
-    int s_shift;             // log2(ksplit); ksplit is a power of two
-    int split;               // 1: the tiles of an item go to different warps, partial sums meet in shared memory
-    int pad_;
-};
-static_assert(sizeof(MkPhase) % 16 == 0, "descriptor is copied in 16-byte pieces");
-
-struct MkParams {
-    const MkPhase *phases;   // [nph]
-    int nph;                 // 4 * n_layers + 1
-    int n_layers, H, nq, nkv, d, F, V;
-    int half_shift;          // log2(d / 2)
-    float eps, scale;
-    int max_context;
-    uint16_t *k_cache, *v_cache;   // [L][nkv][max_context][d]
-    const uint16_t *embed;
-    const double *inv_freq;        // [d/2]
-    float *x, *q, *attn;
-    float *part_m, *part_l, *part_o;
-    int max_chunks;                // row stride of the attention partial buffers (>= any chunk count)
-    int att_chunk_shared;          // smallest chunk (positions) when one CTA serves a whole GQA group
-    int att_chunk_split;           // smallest chunk when every query head has its own CTAs
-    int att_split_max_n;           // contexts up to this length use one-head-per-CTA attention
-    unsigned *tickets;             // [nq] attention, [nq] = lm_head
-    unsigned *barrier;             // grid barrier counter (0 between launches)
-    float *lm_part_val;
-    int *lm_part_idx;
-    StepState *state;
-    const StepRequest *req;
-    int ring_bytes;                // shared-memory ring of one warp
-    int slot_bytes;                // largest tile (checked against ring_bytes on the host)
-    int xbuf_bytes, sched_bytes;
-    unsigned spin_limit;           // upper bound of every device-side wait, nanoseconds
-    unsigned long long *prof;      // optional timestamps [gridDim.x][prof_stride] (diagnostics), or null
-    int prof_stride;
-};
 
 // Optional fine-grained trace of one operator in CTA 0 (compile with -DEDGEFM_TRACE_PHASE=<operator index>):
 // lane 0 of every warp appends %globaltimer stamps behind the regular profile table.
+#ifndef MK_TRACE
 #ifdef EDGEFM_TRACE_PHASE
 #define MK_TRACE(p, ph, warp, lane, slot)                                                                          \
     do {                                                                                                           \
         if ((p).prof && (ph) == EDGEFM_TRACE_PHASE && blockIdx.x == 0 && (lane) == 0 && (slot) < 16)               \
-            (p).prof[static_cast<size_t>(gridDim.x) * (p).prof_stride + (warp) * 16 + (slot)] = global_ns_();        \
+            (p).prof[static_cast<size_t>(gridDim.x) * (p).prof_stride + (warp) * 16 + (slot)] = global_ns();        \
     } while (0)
-__device__ __forceinline__ unsigned long long global_ns_() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
 #else
 #define MK_TRACE(p, ph, warp, lane, slot) do {} while (0)
 #endif
+#endif  // MK_TRACE
 
 // ---- mbarrier / bulk copy primitives -----------------------------------------------------------------
 __device__ __forceinline__ unsigned smem_u32(const void *p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
@@ -1075,4 +1014,5 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
     }
 }
 
+}  // namespace MK_NS
 }  // namespace edgefm
