@@ -195,3 +195,18 @@ def test_statefulness_export_then_prefill():
         ctx2.close()
     finally:
         pair.close()
+
+
+@pytest.mark.parametrize("variant", ["g2_d64", "g7_d128_bias"])
+def test_long_context_build_crosses_the_attention_mode_switch(variant):
+    """max_context > 8192 selects the long-context build of the kernel (8 warps per CTA, both attention modes).
+    Starting at 8188 cached positions, the steps cross the switch from one-head-per-CTA attention (merged in the
+    O-projection prologue) to grouped attention (merged by the last CTA of a group)."""
+    cfg = TINY if variant == "g2_d64" else TINY.with_(n_q_heads=7, n_kv_heads=1, head_dim=128, hidden=320, ffn=512, vocab=3000,
+                                                         qkv_bias=True)
+    pair = Pair(cfg, seed=77, cache_len=8188, max_context=8200)
+    try:
+        run_teacher_forced(pair, 9, 5, 8188)          # attends 8189 .. 8197 positions
+        check_cache_against_oracle(pair, 8188, 9)
+    finally:
+        pair.close()
