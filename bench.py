@@ -247,7 +247,8 @@ def main():
             "metric": METRIC, "value": ms_per_token, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
             "ms_per_step": dev_ms / steps, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16 weights/KV, fp32 accumulate", "data": "synthetic",
-            "config": {"workload": workload_name(cfg), "replicas": world, "l2": "working set 3 GB per step exceeds L2; no flush",
+            "config": {"workload": workload_name(cfg), "replicas": world, "l2": (f"working set {cfg.mean_step_bytes() / 1e9:.2f} GB per step exceeds the 126 MB L2; no flush"
+                              if cfg.mean_step_bytes() > 2.5e8 else "working set fits L2: NOT an HBM measurement"),
                        "seed": GLOBAL_SEED},
             "tokens_per_s": tokens / (dev_ms * 1e-3),
             "roofline": {"bound": "hbm", "kernel": f"decode_megakernel: the whole decode step ({launches} kernel launch per token, one CUDA graph node)",
