@@ -18,10 +18,14 @@ _p = ctypes.c_void_p
 
 def build_oracle(force: bool = False) -> Path:
     src = _HERE / "edgefm_oracle.cpp"
-    if force or not _SO.exists() or _SO.stat().st_mtime < src.stat().st_mtime:
+    import hashlib
+    stamp = _SO.with_suffix(".so.srchash")
+    digest = hashlib.sha256(src.read_bytes()).hexdigest()
+    if force or not _SO.exists() or not stamp.exists() or stamp.read_text().strip() != digest:
         tmp = _SO.with_suffix(f".so.tmp{os.getpid()}")
         subprocess.check_call(["g++", "-std=c++17", "-O2", "-fPIC", "-shared", "-fopenmp", "-o", str(tmp), str(src)])
         os.replace(tmp, _SO)
+        stamp.write_text(digest + "\n")
     return _SO
 
 

@@ -14,14 +14,10 @@
 #include "common.cuh"
 #include "gemv.cuh"
 #include "megakernel_types.cuh"
-// the persistent kernel, built twice: 12 warps per CTA (short contexts) and 8 warps per CTA (long contexts)
+// the persistent kernel is built twice: 12 warps per CTA (short contexts, here) and 8 warps per CTA (long contexts,
+// in the megakernel_long_*.cu translation units)
 #define MK_NS mk_short
 #define MK_NW_VALUE MK_NW_SHORT
-#include "megakernel.cuh"
-#undef MK_NS
-#undef MK_NW_VALUE
-#define MK_NS mk_long
-#define MK_NW_VALUE MK_NW_LONG
 #include "megakernel.cuh"
 #undef MK_NS
 #undef MK_NW_VALUE
@@ -176,26 +172,14 @@ AttnPlan make_attn_plan_g(int G, cudaError_t *err) {
     return AttnPlan();
 }
 
-using MegaKernel = void (*)(const MkParams);
-
 // long_ctx = false: the variant without the grouped (one CTA per GQA group) attention code, for contexts that
 // never need it.
 template <int D>
 MegaKernel mega_kernel_g(int G, bool long_ctx) {
     if (!long_ctx) return mk_short::decode_megakernel<D, 1, false>;   // G is only used by the grouped attention
-    switch (G) {
-        case 1: return mk_long::decode_megakernel<D, 1, true>;
-        case 2: return mk_long::decode_megakernel<D, 2, true>;
-        case 3: return mk_long::decode_megakernel<D, 3, true>;
-        case 4: return mk_long::decode_megakernel<D, 4, true>;
-        case 5: return mk_long::decode_megakernel<D, 5, true>;
-        case 6: return mk_long::decode_megakernel<D, 6, true>;
-        case 7: return mk_long::decode_megakernel<D, 7, true>;
-        case 8: return mk_long::decode_megakernel<D, 8, true>;
-    }
-    return nullptr;
+    if (D == 64) return G <= 4 ? mega_kernel_long_d64_lo(G) : mega_kernel_long_d64_hi(G);
+    return G <= 4 ? mega_kernel_long_d128_lo(G) : mega_kernel_long_d128_hi(G);
 }
-
 // Tile geometry of one weight-streaming operator.
 //  * long operators (many rows per CTA): whole rows, as many per tile (rw rows or row pairs) as fit the
 //    slot budget while every warp keeps about two tiles;

@@ -69,4 +69,11 @@ struct MkParams {
     int prof_stride;
 };
 
+using MegaKernel = void (*)(const MkParams);
+// long-context kernel variants, defined in megakernel_long_d*_*.cu
+MegaKernel mega_kernel_long_d64_lo(int G);
+MegaKernel mega_kernel_long_d64_hi(int G);
+MegaKernel mega_kernel_long_d128_lo(int G);
+MegaKernel mega_kernel_long_d128_hi(int G);
+
 }  // namespace edgefm
