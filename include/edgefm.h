@@ -138,6 +138,24 @@ edgefm_status edgefm_get_launches_per_step(const edgefm_ctx *ctx, int32_t *n_lau
  * expired (EDGEFM_ERR_TIMEOUT; the context is then unusable and must be destroyed) or all is well. */
 edgefm_status edgefm_sync_status(edgefm_ctx *ctx, void *stream);
 
+/*
+ * edgefm_set_vocab_subset -- vocabulary pruning of the output layer (named among the base-layer optimisations in
+ * the caption of Fig. 2; the paper gives no algorithm, so the reading is: greedy decoding restricted to a
+ * caller-chosen set of token ids).
+ *   token_ids  HOST int32 [n], strictly ascending, each in [0, vocab); read before the call returns.
+ *   n          subset size; n == 0 (token_ids may be NULL) restores the full vocabulary.
+ * After the call every decode step of this context computes only the n logits  W_lm[token_ids[r]] . x_f  and
+ *   next token = token_ids[argmax_r logit_r]   (equal maxima: the lowest token id wins, as without pruning);
+ *   logits_out, when given, receives fp32 [n] in subset order (entries past n are left untouched).
+ * The rows are gathered once into a contiguous bf16 [n][hidden] matrix owned by the context (n * hidden * 2 bytes of
+ * device memory, freed by the next call or by edgefm_destroy), so the pruned step streams n rows instead of vocab.
+ * Input token ids stay full-vocabulary ids.  The call synchronises `stream` (steps already enqueued there finish with
+ * the previous subset) and returns after its own copies are done; use the stream the decode steps run on.
+ * Errors: INVALID_ARG (unsorted, duplicate or out-of-range ids, n outside [0, vocab], debug kernel path),
+ * BAD_SHAPE (the subset does not fit the tile plan), OUT_OF_MEMORY, CUDA.  On error the previous subset stays.
+ */
+edgefm_status edgefm_set_vocab_subset(edgefm_ctx *ctx, const int32_t *token_ids, int32_t n, void *stream);
+
 /* Diagnostics.  When the environment variable EDGEFM_PROFILE=1 was set at edgefm_create, every CTA of
  * the persistent step kernel records device timestamps (ns) at fixed points of the last step: start,
  * then per layer {QKV: staged, done, released; attention: done, released; O, gate/up, down: staged,

@@ -114,6 +114,15 @@ def argmax(v: np.ndarray) -> int:
     return int(lib().oracle_argmax(v.ctypes.data, v.size))
 
 
+def restricted_greedy(logits: np.ndarray, token_ids) -> tuple[np.ndarray, int]:
+    """Vocabulary pruning (named in the caption of Fig. 2, no algorithm given; reading: the greedy choice restricted
+    to a subset of token ids, ascending).  -> (the subset's logits in subset order, the token id of the largest;
+    equal maxima: the lowest id)."""
+    ids = np.asarray(token_ids, np.int64)
+    sub = _f32(logits)[ids]
+    return sub, int(ids[argmax(sub)])
+
+
 def f32_to_bf16(f: float) -> int:
     return int(lib().oracle_f32_to_bf16(f))
 

@@ -47,7 +47,7 @@ class _Weights(ctypes.Structure):
 
 EXPORTS = ("edgefm_create", "edgefm_prefill_kv", "edgefm_decode_step", "edgefm_destroy", "edgefm_get_length",
            "edgefm_export_kv", "edgefm_get_launches_per_step", "edgefm_last_error", "edgefm_version",
-           "edgefm_sync_status", "edgefm_debug_profile", "edgefm_decode_step_static")
+           "edgefm_sync_status", "edgefm_debug_profile", "edgefm_decode_step_static", "edgefm_set_vocab_subset")
 
 
 def library_path() -> Path:
@@ -86,6 +86,8 @@ def load_library():
     L.edgefm_debug_profile.argtypes = [vp, vp, i64, ctypes.POINTER(i32), ctypes.POINTER(i32)]
     L.edgefm_decode_step_static.restype = ctypes.c_int
     L.edgefm_decode_step_static.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Weights), vp, vp, i32, i32, i32, i32, vp, vp, vp]
+    L.edgefm_set_vocab_subset.restype = ctypes.c_int
+    L.edgefm_set_vocab_subset.argtypes = [vp, vp, i32, vp]
     L.edgefm_last_error.restype = ctypes.c_char_p
     L.edgefm_last_error.argtypes = [vp]
     L.edgefm_version.restype = ctypes.c_char_p
@@ -167,6 +169,14 @@ def edgefm_decode_step_static(shape: dict, weights: dict, k_cache_ptr, v_cache_p
                                                     cur_len, token_id, position, stream, logits_out, next_token_out))
 
 
+def edgefm_set_vocab_subset(ctx, token_ids, stream=None):
+    """token_ids: strictly ascending int32 ids (any sequence or numpy array) the greedy choice is restricted to;
+    None or empty restores the full vocabulary."""
+    import numpy as np
+    ids = np.ascontiguousarray(np.asarray([] if token_ids is None else token_ids, dtype=np.int32))
+    _check(load_library().edgefm_set_vocab_subset(ctx, ids.ctypes.data if ids.size else None, int(ids.size), stream), ctx)
+
+
 def edgefm_sync_status(ctx, stream=None):
     _check(load_library().edgefm_sync_status(ctx, stream), ctx)
 
@@ -246,6 +256,11 @@ class DecodeContext:
         edgefm_decode_step(self.handle, token_id, position, self._stream(),
                            self.logits.data_ptr() if want_logits else None,
                            self.next_token.data_ptr() if want_token else None)
+
+    def set_vocab_subset(self, token_ids):
+        """Restrict the output layer to these token ids (ascending); None restores the full vocabulary.  With a subset
+        of n ids, logits[:n] holds the subset's logits in subset order."""
+        edgefm_set_vocab_subset(self.handle, token_ids, self._stream())
 
     def export_kv(self):
         import torch

@@ -89,6 +89,18 @@ __global__ void __launch_bounds__(256) prefill_copy_kernel(const uint16_t *k, co
     }
 }
 
+// Vocabulary pruning: row r of the compact lm_head is row ids[r] of the full one.  One warp per row, 16-byte pieces.
+__global__ void __launch_bounds__(256) gather_rows_kernel(const uint16_t *src, const int *ids, uint16_t *dst, int n, int H) {
+    const int warps = (gridDim.x * blockDim.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    const int k16 = H >> 3;
+    for (int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < n; r += warps) {
+        const uint4 *s4 = reinterpret_cast<const uint4 *>(src + static_cast<size_t>(ids[r]) * H);
+        uint4 *d4 = reinterpret_cast<uint4 *>(dst + static_cast<size_t>(r) * H);
+        for (int c = lane; c < k16; c += 32) d4[c] = s4[c];
+    }
+}
+
 // ---- launch helpers ------------------------------------------------------------------------------
 
 template <typename Kern, typename... Args>
@@ -251,6 +263,13 @@ struct edgefm_ctx {
     size_t mega_smem = 0;
     int mega_threads = 0;
     int mega_grid = 0;
+    // vocabulary pruning: the full-vocabulary lm_head descriptor, the tile budget it was planned with, the
+    // gathered rows of the current subset and their token ids
+    MkPhase lm_phase_full{};
+    int tile_budget = 0;
+    int *vocab_ids = nullptr;       // [vocab]
+    uint16_t *sub_lm = nullptr;     // [vocab_subset][hidden] or null
+    int vocab_subset = 0;           // 0 = full vocabulary
 
     cudaStream_t build_stream = nullptr;
     cudaGraph_t graph = nullptr;
@@ -306,7 +325,8 @@ void free_all(edgefm_ctx *c) {
     if (c->graph) cudaGraphDestroy(c->graph);
     if (c->build_stream) cudaStreamDestroy(c->build_stream);
     void *bufs[] = {c->k_cache, c->v_cache, c->x, c->q, c->attn, c->act, c->rope_cs, c->inv_freq, c->part_m, c->part_l,
-                    c->part_o, c->lm_part_val, c->lm_part_idx, c->tickets, c->state, c->req, c->d_phases, c->grid_bar, c->prof};
+                    c->part_o, c->lm_part_val, c->lm_part_idx, c->tickets, c->state, c->req, c->d_phases, c->grid_bar, c->prof,
+                    c->vocab_ids, c->sub_lm};
     for (void *b : bufs) if (b) cudaFree(b);
 }
 
@@ -534,6 +554,7 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
             const int fit1 = static_cast<int>(avail / NW / 128 * 128);   // a tile must fit a warp's ring
             if (budget > fit1) budget = fit1;
         }
+        c->tile_budget = budget;
         int max_tile = 0;
         bool split_overflow = false;
         auto add = [&](int kind, const void *W, int K, int units, const void *bias, const void *norm, const float *xsrc,
@@ -623,7 +644,11 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
             else { ph.x_src = c->act; ph.out = c->x; }
         }
         CREATE_TRY(cudaMemcpy(c->d_phases, phases.data(), phases.size() * sizeof(MkPhase), cudaMemcpyHostToDevice));
+        c->lm_phase_full = phases.back();
+        CREATE_TRY(dev_alloc(&c->vocab_ids, static_cast<size_t>(sh.vocab)));
+        CREATE_TRY(cudaMemset(c->vocab_ids, 0, static_cast<size_t>(sh.vocab) * sizeof(int)));
         MkParams &m = c->mk;
+        m.vocab_ids = c->vocab_ids;
         m.phases = c->d_phases; m.n_layers = sh.n_layers; m.H = H; m.nq = nq; m.nkv = nkv; m.d = d; m.F = F; m.V = sh.vocab;
         m.eps = sh.rms_eps; m.scale = static_cast<float>(1.0 / std::sqrt(static_cast<double>(d)));
         m.max_context = max_context; m.k_cache = c->k_cache; m.v_cache = c->v_cache; m.embed = (const uint16_t *)c->embed;
@@ -725,6 +750,64 @@ edgefm_status edgefm_destroy(edgefm_ctx *ctx) {
 edgefm_status edgefm_get_length(const edgefm_ctx *ctx, int32_t *cur_len_host) {
     if (!ctx || !cur_len_host) return EDGEFM_ERR_INVALID_ARG;
     *cur_len_host = ctx->cur_len;
+    return EDGEFM_OK;
+}
+
+edgefm_status edgefm_set_vocab_subset(edgefm_ctx *ctx, const int32_t *token_ids, int32_t n, void *stream) {
+    if (!ctx) return EDGEFM_ERR_INVALID_ARG;
+    if (!ctx->use_mega) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "vocabulary pruning needs the persistent-kernel path");
+    if (n < 0 || n > ctx->shape.vocab) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "subset size %d outside [0, %d]", n, ctx->shape.vocab);
+    if (n > 0 && !token_ids) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "null token_ids");
+    for (int i = 0; i < n; ++i) {
+        if (token_ids[i] < 0 || token_ids[i] >= ctx->shape.vocab)
+            return fail(ctx, EDGEFM_ERR_INVALID_ARG, "token_ids[%d] = %d out of range", i, token_ids[i]);
+        if (i > 0 && token_ids[i] <= token_ids[i - 1])
+            return fail(ctx, EDGEFM_ERR_INVALID_ARG, "token_ids must be strictly ascending (entry %d)", i);
+    }
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int H = ctx->shape.hidden;
+    MkPhase ph = ctx->lm_phase_full;
+    uint16_t *fresh = nullptr;
+    if (n > 0) {
+        // plan the operator for n rows with the tile budget of the context; it has to fit what the step kernel was
+        // launched with (largest tile, partial-sum scratch)
+        const int NW = ctx->mega_threads / 32;
+        choose_tile(H, false, 4, n, ctx->mega_grid, NW, ctx->tile_budget, &ph.rw, &ph.ksplit, &ph.split);
+        ph.s_shift = 0;
+        while ((1 << ph.s_shift) < ph.ksplit) ++ph.s_shift;
+        ph.kcs = H / 8 / ph.ksplit;
+        ph.units_total = n;
+        ph.items_total = (n + ph.rw - 1) / ph.rw;
+        ph.remap = 1;
+        const long long per_cta = (ph.items_total + ctx->mega_grid - 1) / ctx->mega_grid + 1;
+        if (ph.rw * ph.kcs * 16 > ctx->mk.slot_bytes || (ph.split && per_cta * ph.ksplit > MK_PARTIAL_FLOATS))
+            return fail(ctx, EDGEFM_ERR_BAD_SHAPE, "a subset of %d rows does not fit the tile plan of this context", n);
+        CUDA_TRY(ctx, cudaMalloc(&fresh, static_cast<size_t>(n) * H * sizeof(uint16_t)));
+        ph.W = fresh;
+    }
+    // steps already enqueued on the stream still read the previous subset
+    cudaError_t e = cudaStreamSynchronize(s);
+    if (e == cudaSuccess && n > 0) {
+        e = cudaMemcpyAsync(ctx->vocab_ids, token_ids, static_cast<size_t>(n) * sizeof(int32_t), cudaMemcpyHostToDevice, s);
+        if (e == cudaSuccess) {
+            int blocks = (n + 7) / 8;
+            if (blocks > ctx->num_sms * 8) blocks = ctx->num_sms * 8;
+            gather_rows_kernel<<<blocks, 256, 0, s>>>(static_cast<const uint16_t *>(ctx->lm_head), ctx->vocab_ids, fresh, n, H);
+            e = cudaGetLastError();
+        }
+    }
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(ctx->d_phases + (ctx->mk.nph - 1), &ph, sizeof ph, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);   // token_ids and ph are read before the call returns
+    if (e != cudaSuccess) {
+        if (fresh) cudaFree(fresh);
+        return fail(ctx, EDGEFM_ERR_CUDA, "set_vocab_subset: %s", cudaGetErrorString(e));
+    }
+    if (ctx->sub_lm) cudaFree(ctx->sub_lm);
+    ctx->sub_lm = fresh;
+    ctx->vocab_subset = n;
+    ctx->err.clear();
     return EDGEFM_OK;
 }
 

@@ -1003,6 +1003,7 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
         }
         if (lane == 0) {
             if (bi == 0x7fffffff) bi = 0;
+            if (s_ph[p.nph - 1].remap) bi = p.vocab_ids[bi];   // pruned vocabulary: row index -> token id
             int *nto = p.req->next_token_out;
             if (nto) *nto = bi;
             p.state->next_token = bi;

@@ -35,7 +35,7 @@ struct alignas(16) MkPhase {
     int layer;
     int s_shift;             // log2(ksplit); ksplit is a power of two
     int split;               // 1: the tiles of an item go to different warps, partial sums meet in shared memory
-    int pad_;
+    int remap;               // PH_LMHEAD: 1 = rows are a vocabulary subset; row r stands for token MkParams::vocab_ids[r]
 };
 static_assert(sizeof(MkPhase) % 16 == 0, "descriptor is copied in 16-byte pieces");
 
@@ -59,6 +59,7 @@ struct MkParams {
     unsigned *barrier;             // grid barrier counter (0 between launches)
     float *lm_part_val;
     int *lm_part_idx;
+    const int *vocab_ids;          // [V] token id of every row of a pruned lm_head (used when the last operator says remap)
     StepState *state;
     const StepRequest *req;
     int ring_bytes;                // shared-memory ring of one warp

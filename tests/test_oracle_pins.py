@@ -182,6 +182,29 @@ def test_argmax_planted_and_ties():
     assert O.argmax(np.full(5, -np.inf, np.float32)) == 0
 
 
+def test_restricted_greedy_against_brute_force():
+    """Vocabulary pruning (caption of Fig. 2): the greedy choice over a subset of ids.  Pinned by the full vocabulary
+    reducing to the plain argmax, a planted maximum outside the subset being ignored, ties, and a brute-force loop."""
+    rng = np.random.default_rng(5)
+    V = 5000
+    logits = rng.standard_normal(V).astype(np.float32)
+    sub, nxt = O.restricted_greedy(logits, np.arange(V))
+    assert np.array_equal(sub, logits) and nxt == O.argmax(logits) == int(np.argmax(logits))
+    ids = np.sort(rng.choice(V, 700, replace=False))
+    outside = int(np.setdiff1d(np.arange(V), ids)[17])
+    planted = logits.copy(); planted[outside] = 100.0                   # the global maximum is not in the subset
+    sub, nxt = O.restricted_greedy(planted, ids)
+    best, best_id = -np.inf, -1
+    for t in ids:                                                       # brute force
+        if planted[t] > best:
+            best, best_id = planted[t], int(t)
+    assert nxt == best_id and nxt != outside
+    assert np.array_equal(sub, np.array([planted[t] for t in ids], np.float32))
+    tie = logits.copy(); tie[ids[600]] = 50.0; tie[ids[40]] = 50.0
+    assert O.restricted_greedy(tie, ids)[1] == int(ids[40])             # equal maxima: the lowest id
+    assert O.restricted_greedy(logits, [1234])[1] == 1234               # a single candidate always wins
+
+
 # ---- attention ------------------------------------------------------------------------------
 def test_attention_single_position_returns_v_exactly():
     rng = np.random.default_rng(5)
