@@ -139,6 +139,21 @@ edgefm_status edgefm_get_launches_per_step(const edgefm_ctx *ctx, int32_t *n_lau
 edgefm_status edgefm_sync_status(edgefm_ctx *ctx, void *stream);
 
 /*
+ * edgefm_append_kv -- fixed-prefix cache reuse (Sec. 3.9, Eq. 5: KV = Concat(KV_p, KV_u)).
+ * Copies n_positions of caller-provided KV (same element layout and strides as edgefm_prefill_kv, keys already
+ * rotated) into cache slots [start, start + n_positions) and sets the cache length to start + n_positions.
+ *   start == current length: plain append behind what the cache holds;
+ *   start <  current length: slots from `start` on are dropped first -- the first `start` slots (a prefix computed
+ *                            once at start-up) are kept as they are and serve the next request without being copied again;
+ *   n_positions == 0       : only the truncation (k, v may be NULL).
+ * start > current length is INVALID_ARG (the cache has no holes); start + n_positions > max_context is CONTEXT_FULL;
+ * in both cases nothing is written.  Asynchronous on `stream` like edgefm_prefill_kv; the next step's default
+ * position (position = -1) becomes start + n_positions.
+ */
+edgefm_status edgefm_append_kv(edgefm_ctx *ctx, const void *k, const void *v, int32_t start, int32_t n_positions,
+                               int64_t stride_layer, int64_t stride_head, int64_t stride_pos, void *stream);
+
+/*
  * edgefm_set_vocab_subset -- vocabulary pruning of the output layer (named among the base-layer optimisations in
  * the caption of Fig. 2; the paper gives no algorithm, so the reading is: greedy decoding restricted to a
  * caller-chosen set of token ids).

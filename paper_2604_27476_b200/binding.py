@@ -47,7 +47,7 @@ class _Weights(ctypes.Structure):
 
 EXPORTS = ("edgefm_create", "edgefm_prefill_kv", "edgefm_decode_step", "edgefm_destroy", "edgefm_get_length",
            "edgefm_export_kv", "edgefm_get_launches_per_step", "edgefm_last_error", "edgefm_version",
-           "edgefm_sync_status", "edgefm_debug_profile", "edgefm_decode_step_static", "edgefm_set_vocab_subset")
+           "edgefm_sync_status", "edgefm_debug_profile", "edgefm_decode_step_static", "edgefm_set_vocab_subset", "edgefm_append_kv")
 
 
 def library_path() -> Path:
@@ -86,6 +86,8 @@ def load_library():
     L.edgefm_debug_profile.argtypes = [vp, vp, i64, ctypes.POINTER(i32), ctypes.POINTER(i32)]
     L.edgefm_decode_step_static.restype = ctypes.c_int
     L.edgefm_decode_step_static.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Weights), vp, vp, i32, i32, i32, i32, vp, vp, vp]
+    L.edgefm_append_kv.restype = ctypes.c_int
+    L.edgefm_append_kv.argtypes = [vp, vp, vp, i32, i32, i64, i64, i64, vp]
     L.edgefm_set_vocab_subset.restype = ctypes.c_int
     L.edgefm_set_vocab_subset.argtypes = [vp, vp, i32, vp]
     L.edgefm_last_error.restype = ctypes.c_char_p
@@ -169,6 +171,10 @@ def edgefm_decode_step_static(shape: dict, weights: dict, k_cache_ptr, v_cache_p
                                                     cur_len, token_id, position, stream, logits_out, next_token_out))
 
 
+def edgefm_append_kv(ctx, k_ptr, v_ptr, start, n_positions, stride_layer, stride_head, stride_pos, stream=None):
+    _check(load_library().edgefm_append_kv(ctx, k_ptr, v_ptr, start, n_positions, stride_layer, stride_head, stride_pos, stream), ctx)
+
+
 def edgefm_set_vocab_subset(ctx, token_ids, stream=None):
     """token_ids: strictly ascending int32 ids (any sequence or numpy array) the greedy choice is restricted to;
     None or empty restores the full vocabulary."""
@@ -247,6 +253,14 @@ class DecodeContext:
         n = k.shape[2]
         assert k.stride() == v.stride() and k.stride(3) == 1
         edgefm_prefill_kv(self.handle, k.data_ptr(), v.data_ptr(), n, k.stride(0), k.stride(1), k.stride(2), self._stream())
+
+    def append_kv(self, start, k=None, v=None):
+        """Keep the first `start` slots, then append k, v ([L][n_kv][n][d], device) behind them; k = None only truncates."""
+        if k is None:
+            edgefm_append_kv(self.handle, None, None, start, 0, 0, 0, 0, self._stream())
+            return
+        assert k.stride() == v.stride() and k.stride(3) == 1
+        edgefm_append_kv(self.handle, k.data_ptr(), v.data_ptr(), start, k.shape[2], k.stride(0), k.stride(1), k.stride(2), self._stream())
 
     def reset(self):
         """Empty the cache (cache length 0)."""

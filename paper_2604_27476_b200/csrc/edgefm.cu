@@ -50,13 +50,14 @@ __global__ void __launch_bounds__(256) step_begin_kernel(const StepRequest *req,
     }
 }
 
-// Strided copy of a caller-provided KV prefix into the cache; also sets the device state.
+// Strided copy of n caller-provided KV positions into cache slots [slot0, slot0 + n); also sets the device state
+// (cache length slot0 + n).
 __global__ void __launch_bounds__(256) prefill_copy_kernel(const uint16_t *k, const uint16_t *v, uint16_t *kc, uint16_t *vc,
                                                            int L, int nkv, int n, int d, int max_context, long long s_layer,
-                                                           long long s_head, long long s_pos, int vec_ok, StepState *st) {
+                                                           long long s_head, long long s_pos, int vec_ok, StepState *st, int slot0) {
     if (blockIdx.x == 0 && threadIdx.x == 0) {
-        st->cur_len = n;
-        st->next_position = n;
+        st->cur_len = slot0 + n;
+        st->next_position = slot0 + n;
         st->status = 0;
     }
     const long long total = static_cast<long long>(L) * nkv * n * d;
@@ -70,7 +71,7 @@ __global__ void __launch_bounds__(256) prefill_copy_kernel(const uint16_t *k, co
             const int g = static_cast<int>(r % nkv);
             const int l = static_cast<int>(r / nkv);
             const long long src = l * s_layer + g * s_head + t * s_pos + j * 8;
-            const long long dst = ((static_cast<long long>(l) * nkv + g) * max_context + t) * d + j * 8;
+            const long long dst = ((static_cast<long long>(l) * nkv + g) * max_context + slot0 + t) * d + j * 8;
             *reinterpret_cast<uint4 *>(kc + dst) = *reinterpret_cast<const uint4 *>(k + src);
             *reinterpret_cast<uint4 *>(vc + dst) = *reinterpret_cast<const uint4 *>(v + src);
         }
@@ -82,7 +83,7 @@ __global__ void __launch_bounds__(256) prefill_copy_kernel(const uint16_t *k, co
             const int g = static_cast<int>(r % nkv);
             const int l = static_cast<int>(r / nkv);
             const long long src = l * s_layer + g * s_head + t * s_pos + j;
-            const long long dst = ((static_cast<long long>(l) * nkv + g) * max_context + t) * d + j;
+            const long long dst = ((static_cast<long long>(l) * nkv + g) * max_context + slot0 + t) * d + j;
             kc[dst] = k[src];
             vc[dst] = v[src];
         }
@@ -690,12 +691,13 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
     return EDGEFM_OK;
 }
 
-edgefm_status edgefm_prefill_kv(edgefm_ctx *ctx, const void *k, const void *v, int32_t n_positions, int64_t stride_layer,
-                                int64_t stride_head, int64_t stride_pos, void *stream) {
-    if (!ctx) return EDGEFM_ERR_INVALID_ARG;
+namespace {
+// Common part of edgefm_prefill_kv (slot0 = 0) and edgefm_append_kv.
+edgefm_status copy_kv_in(edgefm_ctx *ctx, const void *k, const void *v, int32_t slot0, int32_t n_positions, int64_t stride_layer,
+                         int64_t stride_head, int64_t stride_pos, void *stream) {
     if (n_positions < 0) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "n_positions < 0");
-    if (n_positions > ctx->max_context)
-        return fail(ctx, EDGEFM_ERR_CONTEXT_FULL, "n_positions %d exceeds max_context %d", n_positions, ctx->max_context);
+    if (static_cast<int64_t>(slot0) + n_positions > ctx->max_context)
+        return fail(ctx, EDGEFM_ERR_CONTEXT_FULL, "%d positions from slot %d exceed max_context %d", n_positions, slot0, ctx->max_context);
     if (n_positions > 0 && (!k || !v)) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "null k or v");
     if (n_positions > 0 && (stride_layer < 0 || stride_head < 0 || stride_pos < ctx->shape.head_dim))
         return fail(ctx, EDGEFM_ERR_INVALID_ARG, "bad strides");
@@ -709,11 +711,26 @@ edgefm_status edgefm_prefill_kv(edgefm_ctx *ctx, const void *k, const void *v, i
     if (blocks > ctx->num_sms * 16) blocks = ctx->num_sms * 16;
     prefill_copy_kernel<<<static_cast<unsigned>(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const uint16_t *>(k), static_cast<const uint16_t *>(v), ctx->k_cache, ctx->v_cache, sh.n_layers,
-        sh.n_kv_heads, n_positions, sh.head_dim, ctx->max_context, stride_layer, stride_head, stride_pos, vec_ok, ctx->state);
+        sh.n_kv_heads, n_positions, sh.head_dim, ctx->max_context, stride_layer, stride_head, stride_pos, vec_ok, ctx->state, slot0);
     CUDA_TRY(ctx, cudaGetLastError());
-    ctx->cur_len = n_positions;
+    ctx->cur_len = slot0 + n_positions;
     ctx->err.clear();
     return EDGEFM_OK;
+}
+}  // namespace
+
+edgefm_status edgefm_prefill_kv(edgefm_ctx *ctx, const void *k, const void *v, int32_t n_positions, int64_t stride_layer,
+                                int64_t stride_head, int64_t stride_pos, void *stream) {
+    if (!ctx) return EDGEFM_ERR_INVALID_ARG;
+    return copy_kv_in(ctx, k, v, 0, n_positions, stride_layer, stride_head, stride_pos, stream);
+}
+
+edgefm_status edgefm_append_kv(edgefm_ctx *ctx, const void *k, const void *v, int32_t start, int32_t n_positions, int64_t stride_layer,
+                               int64_t stride_head, int64_t stride_pos, void *stream) {
+    if (!ctx) return EDGEFM_ERR_INVALID_ARG;
+    if (start < 0 || start > ctx->cur_len)
+        return fail(ctx, EDGEFM_ERR_INVALID_ARG, "start %d outside [0, %d]: the cache may not have holes", start, ctx->cur_len);
+    return copy_kv_in(ctx, k, v, start, n_positions, stride_layer, stride_head, stride_pos, stream);
 }
 
 edgefm_status edgefm_decode_step(edgefm_ctx *ctx, int32_t token_id, int32_t position, void *stream, float *logits_out,
