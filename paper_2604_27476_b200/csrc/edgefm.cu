@@ -1,6 +1,7 @@
 // C ABI of the batch-1 decode step (see include/edgefm.h) and the assembly of the step as a CUDA graph.
 #include "../../include/edgefm.h"
 
+#include <algorithm>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -221,6 +222,121 @@ inline void choose_tile(int K, bool paired, int pair_align, int units, int ncta,
     while (per_cta * s < 2.0 * nw && can_double(256)) s *= 2;                // two per warp while slices stay long
     *ksplit = s;
     *split = s > 1 ? 1 : 0;
+}
+
+
+// Bytes of one tile of an operator.
+inline int phase_tile_bytes(const MkPhase &ph) {
+    const bool paired = ph.kind == PH_QKV || ph.kind == PH_SWIGLU;
+    return ph.rw * (paired ? 2 : 1) * ph.kcs * 16;
+}
+
+// ---- launch plan of the persistent step kernel (shared by edgefm_create and edgefm_decode_step_static) ----------------
+struct StepPlan {
+    MegaKernel kernel = nullptr;
+    bool long_ctx = false;
+    int nw = 0;            // warps per CTA of the chosen kernel build
+    int grid = 0;          // CTAs (one per SM)
+    int max_chunks = 0;    // row stride of the attention partial buffers
+    int n_phases = 0;      // 4 per layer + lm_head
+    int budget = 0;        // upper bound of one weight tile, bytes
+    size_t xbuf = 0, sched = 0, avail = 0;   // shared memory: activation / attention scratch, schedule, what is left for the rings
+    int ring_bytes = 0, slot_bytes = 0;      // filled by plan_phases
+    size_t dyn_smem = 0;
+};
+
+// Kernel variant and shared-memory split for a model shape.  Returns null, or why the shape does not fit.
+inline const char *plan_step(const edgefm_shape &sh, int max_context, int num_sms, int smem_optin, StepPlan *pl, cudaError_t *cuda_err) {
+    const int H = sh.hidden, d = sh.head_dim, nq = sh.n_q_heads, nkv = sh.n_kv_heads, F = sh.ffn, G = nq / nkv;
+    *cuda_err = cudaSuccess;
+    pl->long_ctx = max_context > 8192 || static_cast<long long>(nq) * MK_ATT_SPLIT_MAXC * 2 > MK_PARTIAL_FLOATS;
+    pl->kernel = d == 64 ? mega_kernel_g<64>(G, pl->long_ctx) : mega_kernel_g<128>(G, pl->long_ctx);
+    pl->nw = pl->long_ctx ? MK_NW_LONG : MK_NW_SHORT;
+    pl->grid = num_sms;
+    pl->max_chunks = pl->grid / nkv > 0 ? pl->grid / nkv : 1;
+    pl->n_phases = 4 * sh.n_layers + 1;
+    const int NW = pl->nw, ATT_MW = (NW + 1) / 2;
+    int max_k = H;
+    if (nq * d > max_k) max_k = nq * d;
+    if (F > max_k) max_k = F;
+    // attention scratch: queries, probabilities, warp merge area, chunk statistics
+    const size_t att_bytes = (static_cast<size_t>(G) * d + NW * (G * MK_ATT_TILE > 32 / MK_ATT_LPP_SPLIT ? G * MK_ATT_TILE : 32 / MK_ATT_LPP_SPLIT) +
+                              2 * ATT_MW * G + static_cast<size_t>(ATT_MW) * G * d + 2 * static_cast<size_t>(G) * pl->max_chunks) * 4;
+    size_t xbuf = static_cast<size_t>(max_k) * 4;
+    if (att_bytes > xbuf) xbuf = att_bytes;
+    pl->xbuf = (xbuf + 255) / 256 * 256;
+    cudaFuncAttributes fa{};
+    *cuda_err = cudaFuncGetAttributes(&fa, pl->kernel);
+    if (*cuda_err != cudaSuccess) return "cudaFuncGetAttributes";
+    const size_t static_smem = fa.sharedSizeBytes + 1024;   // the kernel's static shared memory (mbarriers, tables, scratch) + margin
+    pl->sched = (static_cast<size_t>(pl->n_phases) * (sizeof(MkPhase) + sizeof(int2)) + 127) / 128 * 128;
+    if (pl->xbuf + pl->sched + static_smem + static_cast<size_t>(NW) * 1024 > static_cast<size_t>(smem_optin))
+        return "model shape does not fit the shared-memory plan";
+    pl->avail = smem_optin - static_smem - pl->xbuf - pl->sched;
+    pl->budget = 8192;
+    if (const char *tb = getenv("EDGEFM_TILE_BYTES")) { const int v = atoi(tb); if (v >= 1024 && v <= 65536) pl->budget = v; }
+    const int fit1 = static_cast<int>(pl->avail / NW / 128 * 128);   // a tile must fit a warp's ring
+    if (pl->budget > fit1) pl->budget = fit1;
+    return nullptr;
+}
+
+// Descriptor of one weight-streaming operator (tile shape chosen for its aspect ratio).  False: it does not fit the plan.
+inline bool plan_phase(const StepPlan &pl, int head_dim, int kind, const void *W, int K, int units, const void *bias, const void *norm,
+                       const float *x_src, float *out, int layer, MkPhase *ph_out) {
+    MkPhase ph{};
+    const bool paired = kind == PH_QKV || kind == PH_SWIGLU;
+    choose_tile(K, paired, kind == PH_QKV ? head_dim / 2 : 4, units, pl.grid, pl.nw, pl.budget, &ph.rw, &ph.ksplit, &ph.split);
+    ph.s_shift = 0;
+    while ((1 << ph.s_shift) < ph.ksplit) ++ph.s_shift;
+    ph.W = static_cast<const uint16_t *>(W); ph.bias = static_cast<const uint16_t *>(bias); ph.norm_w = static_cast<const uint16_t *>(norm);
+    ph.x_src = x_src; ph.out = out; ph.K = K; ph.kind = kind; ph.kcs = K / 8 / ph.ksplit;
+    ph.units_total = units; ph.items_total = (units + ph.rw - 1) / ph.rw; ph.layer = layer;
+    *ph_out = ph;
+    if (phase_tile_bytes(ph) > pl.budget) return false;
+    if (ph.split) {   // partial sums of one CTA's share must fit the shared-memory scratch
+        const long long per_cta = (ph.items_total + pl.grid - 1) / pl.grid + 1;
+        if (per_cta * ph.ksplit * (paired ? 2 : 1) > MK_PARTIAL_FLOATS) return false;
+    }
+    return true;
+}
+
+// All operators of the step, in execution order, wired to the work buffers; then the ring geometry.
+// Returns null, or why the shape does not fit.
+inline const char *plan_phases(StepPlan *pl, const edgefm_shape &sh, const edgefm_layer_weights *layers, const void *final_norm,
+                               const void *lm_head, float *x, float *q, float *attn, float *act, MkPhase *out) {
+    const int H = sh.hidden, d = sh.head_dim, nq = sh.n_q_heads, nkv = sh.n_kv_heads, F = sh.ffn;
+    const int R = (nq + 2 * nkv) * d;
+    bool fits = true;
+    int n = 0;
+    for (int l = 0; l < sh.n_layers; ++l) {
+        const edgefm_layer_weights &w = layers[l];
+        fits &= plan_phase(*pl, d, PH_QKV, w.wqkv, H, R / 2, sh.qkv_bias ? w.bqkv : nullptr, w.input_norm, l == 0 ? nullptr : x, q, l, &out[n++]);
+        fits &= plan_phase(*pl, d, PH_RESID, w.wo, nq * d, H, nullptr, nullptr, attn, x, l, &out[n++]);
+        fits &= plan_phase(*pl, d, PH_SWIGLU, w.w_gate_up, H, F, nullptr, w.post_norm, x, act, l, &out[n++]);
+        fits &= plan_phase(*pl, d, PH_RESID, w.w_down, F, H, nullptr, nullptr, act, x, l, &out[n++]);
+    }
+    fits &= plan_phase(*pl, d, PH_LMHEAD, lm_head, H, sh.vocab, nullptr, final_norm, x, nullptr, sh.n_layers, &out[n++]);
+    if (!fits) return "model shape does not fit the tile plan";
+    int max_tile = 0;
+    for (int i = 0; i < n; ++i) max_tile = std::max(max_tile, phase_tile_bytes(out[i]));
+    pl->slot_bytes = (max_tile + 127) / 128 * 128;
+    pl->ring_bytes = static_cast<int>(pl->avail / pl->nw / 128 * 128);
+    if (pl->slot_bytes > pl->ring_bytes || pl->ring_bytes > (0xffff << 4)) return "weight rows do not fit the shared-memory ring";
+    pl->dyn_smem = pl->xbuf + pl->sched + static_cast<size_t>(pl->ring_bytes) * pl->nw;
+    return nullptr;
+}
+
+// Shape-derived kernel parameters common to both entry points (buffers, cache and schedule pointers are the caller's).
+inline void fill_shape_params(MkParams *m, const edgefm_shape &sh, int max_context, const StepPlan &pl) {
+    m->nph = pl.n_phases; m->n_layers = sh.n_layers; m->H = sh.hidden; m->nq = sh.n_q_heads; m->nkv = sh.n_kv_heads;
+    m->d = sh.head_dim; m->F = sh.ffn; m->V = sh.vocab;
+    m->half_shift = sh.head_dim == 64 ? 5 : 6;
+    m->eps = sh.rms_eps; m->scale = static_cast<float>(1.0 / std::sqrt(static_cast<double>(sh.head_dim)));
+    m->max_context = max_context; m->max_chunks = pl.max_chunks;
+    m->att_chunk_shared = 256; m->att_chunk_split = 64; m->att_split_max_n = 8192;
+    m->ring_bytes = pl.ring_bytes; m->slot_bytes = pl.slot_bytes; m->xbuf_bytes = static_cast<int>(pl.xbuf);
+    m->sched_bytes = static_cast<int>(pl.sched);
+    m->spin_limit = 1000000000u;   // 1 s
 }
 
 }  // namespace edgefm
@@ -519,90 +635,21 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
         const char *impl = getenv("EDGEFM_IMPL");
         c->use_mega = !(impl && std::strcmp(impl, "kernels") == 0);
     }
-    std::vector<MkPhase> phases;
+    StepPlan pl;
     if (c->use_mega) {
-        const bool long_ctx = max_context > 8192 || static_cast<long long>(nq) * MK_ATT_SPLIT_MAXC * 2 > MK_PARTIAL_FLOATS;
-        c->mega = d == 64 ? mega_kernel_g<64>(G, long_ctx) : mega_kernel_g<128>(G, long_ctx);
-        const int NW = long_ctx ? MK_NW_LONG : MK_NW_SHORT;   // warps per CTA of the chosen build
-        const int ATT_MW = (NW + 1) / 2;
-        c->mega_threads = NW * 32;
         int smem_optin = 0, coop = 0;
         CREATE_TRY(cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
         CREATE_TRY(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev));
         if (!coop) return bail(EDGEFM_ERR_CUDA, "device lacks cooperative launch", cudaErrorNotSupported);
-        c->mega_grid = c->num_sms;
-        // shared-memory plan: activation / attention scratch, the schedule, then the weight ring split
-        // into one private sub-ring of `depth` slots per consumer warp
-        const int max_chunks = c->mega_grid / nkv > 0 ? c->mega_grid / nkv : 1;
-        c->mk.max_chunks = max_chunks;
-        int max_k = H;
-        if (nq * d > max_k) max_k = nq * d;
-        if (F > max_k) max_k = F;
-        const size_t att_bytes = (static_cast<size_t>(G) * d + NW * (G * MK_ATT_TILE > 32 / MK_ATT_LPP_SPLIT ? G * MK_ATT_TILE : 32 / MK_ATT_LPP_SPLIT) + 2 * ATT_MW * G +
-                                  static_cast<size_t>(ATT_MW) * G * d + 2 * static_cast<size_t>(G) * max_chunks) * 4;
-        size_t xbuf = static_cast<size_t>(max_k) * 4;
-        if (att_bytes > xbuf) xbuf = att_bytes;
-        xbuf = (xbuf + 255) / 256 * 256;
-        cudaFuncAttributes fa{};
-        CREATE_TRY(cudaFuncGetAttributes(&fa, c->mega));
-        const size_t static_smem = fa.sharedSizeBytes + 1024;  // the kernel's static shared memory (mbarriers, tables, scratch) + margin
-        const size_t n_phases = 4 * static_cast<size_t>(sh.n_layers) + 1;
-        const size_t sched = (n_phases * (sizeof(MkPhase) + sizeof(int2)) + 127) / 128 * 128;
-        if (xbuf + sched + static_smem + static_cast<size_t>(NW) * 1024 > static_cast<size_t>(smem_optin))
-            return bail(EDGEFM_ERR_CUDA, "model shape does not fit the shared-memory plan", cudaErrorInvalidValue);
-        const size_t avail = smem_optin - static_smem - xbuf - sched;
-        // ring: `depth` slots per warp; prefer two slots of a natural tile size, deeper rings for small tiles
-        int budget = 8192;   // upper bound of one tile
-        if (const char *tb = getenv("EDGEFM_TILE_BYTES")) { const int v = atoi(tb); if (v >= 1024 && v <= 65536) budget = v; }
-        {
-            const int fit1 = static_cast<int>(avail / NW / 128 * 128);   // a tile must fit a warp's ring
-            if (budget > fit1) budget = fit1;
-        }
-        c->tile_budget = budget;
-        int max_tile = 0;
-        bool split_overflow = false;
-        auto add = [&](int kind, const void *W, int K, int units, const void *bias, const void *norm, const float *xsrc,
-                       float *out, int layer) {
-            MkPhase ph{};
-            const bool paired = kind == PH_QKV || kind == PH_SWIGLU;
-            choose_tile(K, paired, kind == PH_QKV ? d / 2 : 4, units, c->mega_grid, NW, budget, &ph.rw, &ph.ksplit, &ph.split);
-            ph.s_shift = 0;
-            while ((1 << ph.s_shift) < ph.ksplit) ++ph.s_shift;
-            ph.W = (const uint16_t *)W; ph.bias = (const uint16_t *)bias; ph.norm_w = (const uint16_t *)norm;
-            ph.x_src = xsrc; ph.out = out; ph.K = K; ph.kind = kind; ph.kcs = K / 8 / ph.ksplit;
-            ph.units_total = units; ph.items_total = (units + ph.rw - 1) / ph.rw; ph.layer = layer;
-            const int tile = ph.rw * (paired ? 2 : 1) * ph.kcs * 16;
-            if (tile > max_tile) max_tile = tile;
-            if (ph.split) {  // partial sums of one CTA's share must fit the shared-memory scratch
-                const long long per_cta = (ph.items_total + c->mega_grid - 1) / c->mega_grid + 1;
-                if (per_cta * ph.ksplit * (paired ? 2 : 1) > MK_PARTIAL_FLOATS) split_overflow = true;
-            }
-            phases.push_back(ph);
-        };
-        // buffers are allocated below; the descriptors' buffer pointers are filled after allocation
-        for (int l = 0; l < sh.n_layers; ++l) {
-            const edgefm_layer_weights &w = c->layers[l];
-            add(PH_QKV, w.wqkv, H, R / 2, sh.qkv_bias ? w.bqkv : nullptr, w.input_norm, nullptr, nullptr, l);
-            add(PH_RESID, w.wo, nq * d, H, nullptr, nullptr, nullptr, nullptr, l);
-            add(PH_SWIGLU, w.w_gate_up, H, F, nullptr, w.post_norm, nullptr, nullptr, l);
-            add(PH_RESID, w.w_down, F, H, nullptr, nullptr, nullptr, nullptr, l);
-        }
-        add(PH_LMHEAD, c->lm_head, H, sh.vocab, nullptr, c->final_norm, nullptr, nullptr, sh.n_layers);
-        if (split_overflow || max_tile > budget)
-            return bail(EDGEFM_ERR_CUDA, "model shape does not fit the tile plan", cudaErrorInvalidValue);
-        const int slot_bytes = (max_tile + 127) / 128 * 128;
-        const int ring_bytes = static_cast<int>(avail / NW / 128 * 128);
-        if (slot_bytes > ring_bytes || ring_bytes > (0xffff << 4))
-            return bail(EDGEFM_ERR_CUDA, "weight rows do not fit the shared-memory ring", cudaErrorInvalidValue);
-        c->mk.ring_bytes = ring_bytes; c->mk.slot_bytes = slot_bytes; c->mk.xbuf_bytes = static_cast<int>(xbuf);
-        c->mk.sched_bytes = static_cast<int>(sched);
-        c->mega_smem = xbuf + sched + static_cast<size_t>(ring_bytes) * NW;
-        CREATE_TRY(cudaFuncSetAttribute(c->mega, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(c->mega_smem)));
-        int per_sm = 0;
-        CREATE_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, c->mega, c->mega_threads, c->mega_smem));
-        if (per_sm < 1) return bail(EDGEFM_ERR_CUDA, "persistent kernel does not fit one CTA per SM", cudaErrorInvalidValue);
-        c->p_attn.max_chunks = max_chunks;  // sizes the partial buffers below
-        c->p_lm.grid = c->mega_grid;
+        cudaError_t ce = cudaSuccess;
+        if (const char *why = plan_step(sh, max_context, c->num_sms, smem_optin, &pl, &ce))
+            return bail(EDGEFM_ERR_CUDA, why, ce != cudaSuccess ? ce : cudaErrorInvalidValue);
+        c->mega = pl.kernel;
+        c->mega_threads = pl.nw * 32;
+        c->mega_grid = pl.grid;
+        c->tile_budget = pl.budget;
+        c->p_attn.max_chunks = pl.max_chunks;  // sizes the partial buffers below
+        c->p_lm.grid = pl.grid;
     }
 
     const size_t kv_elems = static_cast<size_t>(sh.n_layers) * nkv * max_context * d;
@@ -635,38 +682,33 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
     }
 
     if (c->use_mega) {
+        // the operators of the step wired to the work buffers, then the shared-memory rings
+        std::vector<MkPhase> phases(static_cast<size_t>(pl.n_phases));
+        if (const char *why = plan_phases(&pl, sh, c->layers.data(), c->final_norm, c->lm_head, c->x, c->q, c->attn, c->act, phases.data()))
+            return bail(EDGEFM_ERR_CUDA, why, cudaErrorInvalidValue);
+        c->mega_smem = pl.dyn_smem;
+        CREATE_TRY(cudaFuncSetAttribute(c->mega, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(c->mega_smem)));
+        int per_sm = 0;
+        CREATE_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, c->mega, c->mega_threads, c->mega_smem));
+        if (per_sm < 1) return bail(EDGEFM_ERR_CUDA, "persistent kernel does not fit one CTA per SM", cudaErrorInvalidValue);
         CREATE_TRY(dev_alloc(&c->d_phases, phases.size()));
         CREATE_TRY(dev_alloc(&c->grid_bar, 1));
         CREATE_TRY(cudaMemset(c->grid_bar, 0, sizeof(unsigned)));
-        for (size_t i = 0; i < phases.size(); ++i) {
-            MkPhase &ph = phases[i];
-            const int k = static_cast<int>(i % 4);
-            if (i + 1 == phases.size()) { ph.x_src = c->x; ph.out = nullptr; }
-            else if (k == 0) { ph.x_src = ph.layer == 0 ? nullptr : c->x; ph.out = c->q; }
-            else if (k == 1) { ph.x_src = c->attn; ph.out = c->x; }
-            else if (k == 2) { ph.x_src = c->x; ph.out = c->act; }
-            else { ph.x_src = c->act; ph.out = c->x; }
-        }
         CREATE_TRY(cudaMemcpy(c->d_phases, phases.data(), phases.size() * sizeof(MkPhase), cudaMemcpyHostToDevice));
         c->lm_phase_full = phases.back();
         CREATE_TRY(dev_alloc(&c->vocab_ids, static_cast<size_t>(sh.vocab)));
         CREATE_TRY(cudaMemset(c->vocab_ids, 0, static_cast<size_t>(sh.vocab) * sizeof(int)));
         MkParams &m = c->mk;
-        m.vocab_ids = c->vocab_ids;
-        m.phases = c->d_phases; m.n_layers = sh.n_layers; m.H = H; m.nq = nq; m.nkv = nkv; m.d = d; m.F = F; m.V = sh.vocab;
-        m.eps = sh.rms_eps; m.scale = static_cast<float>(1.0 / std::sqrt(static_cast<double>(d)));
-        m.max_context = max_context; m.k_cache = c->k_cache; m.v_cache = c->v_cache; m.embed = (const uint16_t *)c->embed;
+        fill_shape_params(&m, sh, max_context, pl);
+        m.phases = c->d_phases; m.vocab_ids = c->vocab_ids;
+        m.k_cache = c->k_cache; m.v_cache = c->v_cache; m.embed = (const uint16_t *)c->embed;
         m.inv_freq = c->inv_freq; m.x = c->x; m.q = c->q; m.attn = c->attn; m.part_m = c->part_m; m.part_l = c->part_l;
         m.part_o = c->part_o; m.tickets = c->tickets; m.barrier = c->grid_bar;
-        m.nph = static_cast<int>(phases.size());
-        m.half_shift = d == 64 ? 5 : 6;
-        m.att_chunk_shared = 256; m.att_chunk_split = 64; m.att_split_max_n = 8192;
         if (max_context > 8192) {   // only the long-context kernel variant has both attention modes
             if (const char *ac = getenv("EDGEFM_ATT_SPLIT_MAX")) { const int v = atoi(ac); if (v >= 0) m.att_split_max_n = v; }
         }
         if (const char *ac = getenv("EDGEFM_ATT_CHUNK")) { const int v = atoi(ac); if (v >= 8) { m.att_chunk_shared = v; m.att_chunk_split = v; } }
         m.lm_part_val = c->lm_part_val; m.lm_part_idx = c->lm_part_idx; m.state = c->state; m.req = c->req;
-        m.spin_limit = 1000000000u;  // 1 s
         const char *pe_ = getenv("EDGEFM_PROFILE");
         if (pe_ && pe_[0] == '1') {
             c->prof_stride = 3 + 14 * sh.n_layers;
@@ -792,16 +834,12 @@ edgefm_status edgefm_set_vocab_subset(edgefm_ctx *ctx, const int32_t *token_ids,
     if (n > 0) {
         // plan the operator for n rows with the tile budget of the context; it has to fit what the step kernel was
         // launched with (largest tile, partial-sum scratch)
-        const int NW = ctx->mega_threads / 32;
-        choose_tile(H, false, 4, n, ctx->mega_grid, NW, ctx->tile_budget, &ph.rw, &ph.ksplit, &ph.split);
-        ph.s_shift = 0;
-        while ((1 << ph.s_shift) < ph.ksplit) ++ph.s_shift;
-        ph.kcs = H / 8 / ph.ksplit;
-        ph.units_total = n;
-        ph.items_total = (n + ph.rw - 1) / ph.rw;
+        StepPlan pl;
+        pl.grid = ctx->mega_grid; pl.nw = ctx->mega_threads / 32; pl.budget = ctx->tile_budget;
+        const MkPhase &full = ctx->lm_phase_full;
+        const bool fits = plan_phase(pl, ctx->shape.head_dim, PH_LMHEAD, nullptr, H, n, nullptr, full.norm_w, full.x_src, nullptr, full.layer, &ph);
         ph.remap = 1;
-        const long long per_cta = (ph.items_total + ctx->mega_grid - 1) / ctx->mega_grid + 1;
-        if (ph.rw * ph.kcs * 16 > ctx->mk.slot_bytes || (ph.split && per_cta * ph.ksplit > MK_PARTIAL_FLOATS))
+        if (!fits || phase_tile_bytes(ph) > ctx->mk.slot_bytes)
             return fail(ctx, EDGEFM_ERR_BAD_SHAPE, "a subset of %d rows does not fit the tile plan of this context", n);
         CUDA_TRY(ctx, cudaMalloc(&fresh, static_cast<size_t>(n) * H * sizeof(uint16_t)));
         ph.W = fresh;
@@ -944,8 +982,7 @@ extern "C" edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, co
         cudaGetLastError();
         return fail(nullptr, EDGEFM_ERR_CUDA, "no usable CUDA device (this library has no CPU path)");
     }
-    const int H = sh.hidden, d = sh.head_dim, nq = sh.n_q_heads, nkv = sh.n_kv_heads, F = sh.ffn, G = nq / nkv;
-    const int R = (nq + 2 * nkv) * d;
+    const int H = sh.hidden, d = sh.head_dim, nq = sh.n_q_heads, nkv = sh.n_kv_heads, F = sh.ffn;
     int num_sms = 0, smem_optin = 0, coop = 0;
     CUDA_TRY(nullptr, cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
     CUDA_TRY(nullptr, cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
@@ -959,35 +996,15 @@ extern "C" edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, co
         if (!ptr) return fail(nullptr, EDGEFM_ERR_CUDA, "cudaGetSymbolAddress returned a null scratch address");
         g_scratch_dev_ptr[dev] = ptr;
     }
-    const bool long_ctx = max_context > 8192 || static_cast<long long>(nq) * MK_ATT_SPLIT_MAXC * 2 > MK_PARTIAL_FLOATS;
-    MegaKernel kern = d == 64 ? mega_kernel_g<64>(G, long_ctx) : mega_kernel_g<128>(G, long_ctx);
-    const int NW = long_ctx ? MK_NW_LONG : MK_NW_SHORT;   // warps per CTA of the chosen build
-    const int ATT_MW = (NW + 1) / 2;
-
     // ---- the same plan edgefm_create makes, on the stack ----------------------------------------------------
-    const int grid = num_sms;
-    const int max_chunks = grid / nkv > 0 ? grid / nkv : 1;
-    int max_k = H;
-    if (nq * d > max_k) max_k = nq * d;
-    if (F > max_k) max_k = F;
-    const size_t att_bytes = (static_cast<size_t>(G) * d + NW * (G * MK_ATT_TILE > 32 / MK_ATT_LPP_SPLIT ? G * MK_ATT_TILE : 32 / MK_ATT_LPP_SPLIT) + 2 * ATT_MW * G +
-                              static_cast<size_t>(ATT_MW) * G * d + 2 * static_cast<size_t>(G) * max_chunks) * 4;
-    size_t xbuf = static_cast<size_t>(max_k) * 4;
-    if (att_bytes > xbuf) xbuf = att_bytes;
-    xbuf = (xbuf + 255) / 256 * 256;
-    cudaFuncAttributes fa{};
-    CUDA_TRY(nullptr, cudaFuncGetAttributes(&fa, kern));
-    const size_t static_smem = fa.sharedSizeBytes + 1024;
-    const int n_phases = 4 * sh.n_layers + 1;
-    const size_t sched = (static_cast<size_t>(n_phases) * (sizeof(MkPhase) + sizeof(int2)) + 127) / 128 * 128;
-    if (xbuf + sched + static_smem + static_cast<size_t>(NW) * 1024 > static_cast<size_t>(smem_optin))
-        return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "model shape does not fit the shared-memory plan");
-    const size_t avail = smem_optin - static_smem - xbuf - sched;
-    int budget = 8192;
+    StepPlan pl;
     {
-        const int fit1 = static_cast<int>(avail / NW / 128 * 128);
-        if (budget > fit1) budget = fit1;
+        cudaError_t ce = cudaSuccess;
+        if (const char *why = plan_step(sh, max_context, num_sms, smem_optin, &pl, &ce))
+            return fail(nullptr, ce != cudaSuccess ? EDGEFM_ERR_CUDA : EDGEFM_ERR_BAD_SHAPE, "%s", why);
     }
+    MegaKernel kern = pl.kernel;
+    const int NW = pl.nw, grid = pl.grid, max_chunks = pl.max_chunks, n_phases = pl.n_phases;
 
     // carve the scratch array; reject shapes that need more than it holds
     ScratchCarver sc{g_scratch_dev_ptr[dev]};
@@ -1012,53 +1029,22 @@ extern "C" edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, co
     unsigned *grid_bar = counters + nq + nkv + 2 + 32;
 
     MkPhase phases[4 * kMaxLayers + 1];
-    int n_ph = 0, max_tile = 0;
-    bool split_overflow = false;
-    auto add = [&](int kind, const void *W, int K, int units, const void *bias, const void *norm, const float *xsrc, float *out, int layer) {
-        MkPhase ph{};
-        const bool paired = kind == PH_QKV || kind == PH_SWIGLU;
-        choose_tile(K, paired, kind == PH_QKV ? d / 2 : 4, units, grid, NW, budget, &ph.rw, &ph.ksplit, &ph.split);
-        ph.s_shift = 0;
-        while ((1 << ph.s_shift) < ph.ksplit) ++ph.s_shift;
-        ph.W = (const uint16_t *)W; ph.bias = (const uint16_t *)bias; ph.norm_w = (const uint16_t *)norm;
-        ph.x_src = xsrc; ph.out = out; ph.K = K; ph.kind = kind; ph.kcs = K / 8 / ph.ksplit;
-        ph.units_total = units; ph.items_total = (units + ph.rw - 1) / ph.rw; ph.layer = layer;
-        const int tile = ph.rw * (paired ? 2 : 1) * ph.kcs * 16;
-        if (tile > max_tile) max_tile = tile;
-        if (ph.split) {
-            const long long per_cta = (ph.items_total + grid - 1) / grid + 1;
-            if (per_cta * ph.ksplit * (paired ? 2 : 1) > MK_PARTIAL_FLOATS) split_overflow = true;
-        }
-        phases[n_ph++] = ph;
-    };
-    for (int l = 0; l < sh.n_layers; ++l) {
-        const edgefm_layer_weights &w = weights->layers[l];
-        add(PH_QKV, w.wqkv, H, R / 2, sh.qkv_bias ? w.bqkv : nullptr, w.input_norm, l == 0 ? nullptr : x, q, l);
-        add(PH_RESID, w.wo, nq * d, H, nullptr, nullptr, attn, x, l);
-        add(PH_SWIGLU, w.w_gate_up, H, F, nullptr, w.post_norm, x, act, l);
-        add(PH_RESID, w.w_down, F, H, nullptr, nullptr, act, x, l);
-    }
-    add(PH_LMHEAD, weights->lm_head, H, sh.vocab, nullptr, weights->final_norm, x, nullptr, sh.n_layers);
-    if (split_overflow || max_tile > budget) return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "model shape does not fit the tile plan");
-    const int slot_bytes = (max_tile + 127) / 128 * 128;
-    const int ring_bytes = static_cast<int>(avail / NW / 128 * 128);
-    if (slot_bytes > ring_bytes || ring_bytes > (0xffff << 4)) return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "weight rows do not fit the shared-memory ring");
-    const size_t dyn_smem = xbuf + sched + static_cast<size_t>(ring_bytes) * NW;
+    if (const char *why = plan_phases(&pl, sh, weights->layers, weights->final_norm, weights->lm_head, x, q, attn, act, phases))
+        return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "%s", why);
+    const int n_ph = n_phases;
+    const size_t dyn_smem = pl.dyn_smem;
     // raise the kernel's dynamic shared-memory limit (a function attribute, not an allocation); repeated on every
     // call because edgefm_create sets the same attribute for its own contexts
     CUDA_TRY(nullptr, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(dyn_smem)));
 
     MkParams m{};
-    m.phases = d_phases; m.nph = n_ph; m.n_layers = sh.n_layers; m.H = H; m.nq = nq; m.nkv = nkv; m.d = d; m.F = F; m.V = sh.vocab;
-    m.half_shift = d == 64 ? 5 : 6;
-    m.eps = sh.rms_eps; m.scale = static_cast<float>(1.0 / std::sqrt(static_cast<double>(d)));
-    m.max_context = max_context; m.k_cache = static_cast<uint16_t *>(k_cache); m.v_cache = static_cast<uint16_t *>(v_cache);
+    fill_shape_params(&m, sh, max_context, pl);
+    m.phases = d_phases;
+    m.k_cache = static_cast<uint16_t *>(k_cache); m.v_cache = static_cast<uint16_t *>(v_cache);
     m.embed = (const uint16_t *)weights->embed; m.inv_freq = inv_freq; m.x = x; m.q = q; m.attn = attn;
-    m.part_m = part_m; m.part_l = part_l; m.part_o = part_o; m.max_chunks = max_chunks;
-    m.att_chunk_shared = 256; m.att_chunk_split = 64; m.att_split_max_n = 8192;
+    m.part_m = part_m; m.part_l = part_l; m.part_o = part_o;
     m.tickets = tickets; m.barrier = grid_bar; m.lm_part_val = lm_val; m.lm_part_idx = lm_idx; m.state = state; m.req = req;
-    m.ring_bytes = ring_bytes; m.slot_bytes = slot_bytes; m.xbuf_bytes = static_cast<int>(xbuf); m.sched_bytes = static_cast<int>(sched);
-    m.spin_limit = 1000000000u; m.prof = nullptr; m.prof_stride = 0;
+    m.prof = nullptr; m.prof_stride = 0;
 
     // ---- stream-ordered set-up of the shared scratch: it still holds the previous call's contents ----------
     cudaStream_t s = static_cast<cudaStream_t>(stream);
