@@ -313,7 +313,9 @@ inline const char *plan_phases(StepPlan *pl, const edgefm_shape &sh, const edgef
         fits &= plan_phase(*pl, d, PH_QKV, w.wqkv, H, R / 2, sh.qkv_bias ? w.bqkv : nullptr, w.input_norm, l == 0 ? nullptr : x, q, l, &out[n++]);
         fits &= plan_phase(*pl, d, PH_RESID, w.wo, nq * d, H, nullptr, nullptr, attn, x, l, &out[n++]);
         fits &= plan_phase(*pl, d, PH_SWIGLU, w.w_gate_up, H, F, nullptr, w.post_norm, x, act, l, &out[n++]);
+        out[n - 1].flags |= PHF_OUT_SPLIT;   // the MLP activations go to memory in the layout the down projection stages
         fits &= plan_phase(*pl, d, PH_RESID, w.w_down, F, H, nullptr, nullptr, act, x, l, &out[n++]);
+        out[n - 1].flags |= PHF_X_BULK;
     }
     fits &= plan_phase(*pl, d, PH_LMHEAD, lm_head, H, sh.vocab, nullptr, final_norm, x, nullptr, sh.n_layers, &out[n++]);
     if (!fits) return "model shape does not fit the tile plan";
@@ -838,7 +840,7 @@ edgefm_status edgefm_set_vocab_subset(edgefm_ctx *ctx, const int32_t *token_ids,
         pl.grid = ctx->mega_grid; pl.nw = ctx->mega_threads / 32; pl.budget = ctx->tile_budget;
         const MkPhase &full = ctx->lm_phase_full;
         const bool fits = plan_phase(pl, ctx->shape.head_dim, PH_LMHEAD, nullptr, H, n, nullptr, full.norm_w, full.x_src, nullptr, full.layer, &ph);
-        ph.remap = 1;
+        ph.flags = PHF_REMAP;
         if (!fits || phase_tile_bytes(ph) > ctx->mk.slot_bytes)
             return fail(ctx, EDGEFM_ERR_BAD_SHAPE, "a subset of %d rows does not fit the tile plan of this context", n);
         CUDA_TRY(ctx, cudaMalloc(&fresh, static_cast<size_t>(n) * H * sizeof(uint16_t)));

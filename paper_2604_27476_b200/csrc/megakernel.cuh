@@ -94,6 +94,11 @@ __device__ __forceinline__ void bulk_copy_g2s(void *dst, const void *src, unsign
         ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
         : "memory");
 }
+__device__ __forceinline__ void bulk_copy_g2s_plain(void *dst, const void *src, unsigned bytes, unsigned long long *bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
 __device__ __forceinline__ void cta_sync() { __syncthreads(); }
 
 __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned *p) {
@@ -315,7 +320,13 @@ __device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkPhase 
         if (cx.logits_out) cx.logits_out[u] = lo;
         if (arg_better(lo, u, cx.best_v, cx.best_i)) { cx.best_v = lo; cx.best_i = u; }
     } else if (P.kind == PH_SWIGLU) {
-        P.out[u] = lo / (1.f + expf(-lo)) * hi;
+        const float a = lo / (1.f + expf(-lo)) * hi;
+        if (P.flags & PHF_OUT_SPLIT) {   // the layout the next operator's prologue copies straight into shared memory
+            const int i4 = u >> 2;
+            P.out[(i4 & 1) * (P.units_total >> 1) + ((i4 >> 1) << 2) + (u & 3)] = a;
+        } else {
+            P.out[u] = a;
+        }
     } else {  // PH_QKV: bias, rotate-half RoPE of q and k, q to the work buffer, k and v to the cache row of this step
         const int half = p.d >> 1;
         const int head = u >> p.half_shift, i = u & (half - 1);
@@ -463,7 +474,7 @@ __device__ __forceinline__ void att_chunking(const MkParams &p, int n, int hg, i
 // (m, l, unnormalised o); the exact log-sum-exp merge is done here, in chunk order, by every CTA.
 __device__ __forceinline__ bool gemv_phase(const MkParams &p, const MkPhase *s_ph, const int2 *s_rng, int ph, WarpStream &ws, float4 *xsA,
                                            float4 *xsB, volatile int *abort_flag, float *s_part, float *s_partial, ItemCtx &cx, int token,
-                                           int merge_attn, int tid, int &prof_idx) {
+                                           int merge_attn, int tid, int &prof_idx, unsigned long long *x_bar, unsigned &x_parity) {
     const MkPhase &P = s_ph[ph];
     const int lane = tid & 31, warp = tid >> 5;
     const int cta = blockIdx.x;
@@ -510,6 +521,19 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, const MkPhase *s_p
             acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
             if (o4 & 1) xsB[o4 >> 1] = acc; else xsA[o4 >> 1] = acc;
         }
+    } else if (P.flags & PHF_X_BULK) {
+        // the vector is already in the split layout and needs no transform: two bulk copies, every thread waits for them
+        // (the CTA-wide sync of the grid barrier ordered all earlier reads of the buffer before this point)
+        if (tid == 0) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            const unsigned half_bytes = static_cast<unsigned>(P.K) * 2u;
+            mbar_arrive_expect_tx(x_bar, 2u * half_bytes);
+            bulk_copy_g2s_plain(xsA, P.x_src, half_bytes, x_bar);
+            bulk_copy_g2s_plain(xsB, P.x_src + (P.K >> 1), half_bytes, x_bar);
+        }
+        const bool arrived = mbar_wait(x_bar, x_parity, abort_flag, p.spin_limit);
+        x_parity ^= 1u;
+        if (!arrived && tid == 0) p.state->status = 6;
     } else {
         constexpr int PU = 4;  // loads in flight per thread
         for (int base = tid; base < n4; base += MK_NT * PU) {
@@ -855,6 +879,7 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
     int2 *s_rng = reinterpret_cast<int2 *>(s_ph + p.nph);                      // this CTA's item range per operator
     unsigned char *ring = smem + p.xbuf_bytes + p.sched_bytes;
     __shared__ __align__(8) unsigned long long full_bar[MK_NW * MK_MAXF];
+    __shared__ __align__(8) unsigned long long x_bar;   // completion of bulk-copied activation vectors
     __shared__ float s_rope[128];
     __shared__ float s_part[MK_NW];
     __shared__ float s_partial[MK_PARTIAL_FLOATS];
@@ -868,6 +893,7 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
     const int cta = blockIdx.x, ncta = gridDim.x;
     if (tid == 0) {
         for (int i = 0; i < MK_NW * MK_MAXF; ++i) mbar_init(&full_bar[i], 1);
+        mbar_init(&x_bar, 1);
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -926,6 +952,7 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
     cx.logits_out = p.req->logits_out;
 
     unsigned bar_no = 0;
+    unsigned x_parity = 0;
     int prof_idx = 0;
     prof_stamp(p, tid, prof_idx);
     auto top_up = [&]() { __syncwarp(); if (ok && !*abort_flag) refill(p, s_ph, s_rng, ws, abort_flag, warp, lane); };
@@ -934,7 +961,7 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
     int merge_chunks = 0;   // chunks per head the O-projection prologue has to merge (split mode)
     if (att_split) { int cl; att_chunking(p, n_att, 1, p.att_chunk_split, 32 / MK_ATT_LPP_SPLIT, ncta, merge_chunks, cl); }
     for (int l = 0; l < p.n_layers && ok; ++l) {
-        ok = gemv_phase(p, s_ph, s_rng, 4 * l, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token, 0, tid, prof_idx);
+        ok = gemv_phase(p, s_ph, s_rng, 4 * l, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token, 0, tid, prof_idx, &x_bar, x_parity);
         ok = grid_barrier(p, ++bar_no * ncta, abort_flag, &s_released, tid, prof_idx, top_up) && ok;
         if (ok) {
             if constexpr (LONG) {
@@ -947,11 +974,11 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
         ok = grid_barrier(p, ++bar_no * ncta, abort_flag, &s_released, tid, prof_idx, top_up) && ok;
         for (int k = 1; k < 4 && ok; ++k) {
             ok = gemv_phase(p, s_ph, s_rng, 4 * l + k, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token,
-                            k == 1 ? merge_chunks : 0, tid, prof_idx);
+                            k == 1 ? merge_chunks : 0, tid, prof_idx, &x_bar, x_parity);
             ok = grid_barrier(p, ++bar_no * ncta, abort_flag, &s_released, tid, prof_idx, top_up) && ok;
         }
     }
-    if (ok) ok = gemv_phase(p, s_ph, s_rng, 4 * p.n_layers, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token, 0, tid, prof_idx);
+    if (ok) ok = gemv_phase(p, s_ph, s_rng, 4 * p.n_layers, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token, 0, tid, prof_idx, &x_bar, x_parity);
     prof_stamp(p, tid, prof_idx);
     if (!ok || *abort_flag) {
         // aborted: wait (bounded) for the copies this warp still has in flight, then leave
@@ -1003,7 +1030,7 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
         }
         if (lane == 0) {
             if (bi == 0x7fffffff) bi = 0;
-            if (s_ph[p.nph - 1].remap) bi = p.vocab_ids[bi];   // pruned vocabulary: row index -> token id
+            if (s_ph[p.nph - 1].flags & PHF_REMAP) bi = p.vocab_ids[bi];   // pruned vocabulary: row index -> token id
             int *nto = p.req->next_token_out;
             if (nto) *nto = bi;
             p.state->next_token = bi;

@@ -19,6 +19,13 @@ constexpr int MK_NW_LONG = 8;
 enum { PH_QKV = 0, PH_RESID = 1, PH_SWIGLU = 2, PH_LMHEAD = 3 };
 
 // One weight-streaming operator of the step.
+// MkPhase::flags
+enum : int {
+    PHF_REMAP = 1,      // PH_LMHEAD: rows are a vocabulary subset; row r stands for token MkParams::vocab_ids[r]
+    PHF_OUT_SPLIT = 2,  // PH_SWIGLU: the output vector is stored as [even 16-byte pieces | odd 16-byte pieces]
+    PHF_X_BULK = 4,     // the input vector has that layout already and needs no transform: staged by two bulk copies
+};
+
 struct alignas(16) MkPhase {
     const uint16_t *W;       // bf16 [rows][K]
     const uint16_t *bias;    // PH_QKV: bf16 [rows] or null
@@ -35,7 +42,7 @@ struct alignas(16) MkPhase {
     int layer;
     int s_shift;             // log2(ksplit); ksplit is a power of two
     int split;               // 1: the tiles of an item go to different warps, partial sums meet in shared memory
-    int remap;               // PH_LMHEAD: 1 = rows are a vocabulary subset; row r stands for token MkParams::vocab_ids[r]
+    int flags;               // PHF_* bits
 };
 static_assert(sizeof(MkPhase) % 16 == 0, "descriptor is copied in 16-byte pieces");
 
@@ -59,7 +66,7 @@ struct MkParams {
     unsigned *barrier;             // grid barrier counter (0 between launches)
     float *lm_part_val;
     int *lm_part_idx;
-    const int *vocab_ids;          // [V] token id of every row of a pruned lm_head (used when the last operator says remap)
+    const int *vocab_ids;          // [V] token id of every row of a pruned lm_head (used when the last operator has PHF_REMAP)
     StepState *state;
     const StepRequest *req;
     int ring_bytes;                // shared-memory ring of one warp
