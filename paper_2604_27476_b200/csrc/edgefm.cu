@@ -312,6 +312,7 @@ inline const char *plan_phases(StepPlan *pl, const edgefm_shape &sh, const edgef
         const edgefm_layer_weights &w = layers[l];
         fits &= plan_phase(*pl, d, PH_QKV, w.wqkv, H, R / 2, sh.qkv_bias ? w.bqkv : nullptr, w.input_norm, l == 0 ? nullptr : x, q, l, &out[n++]);
         fits &= plan_phase(*pl, d, PH_RESID, w.wo, nq * d, H, nullptr, nullptr, attn, x, l, &out[n++]);
+        out[n - 1].flags |= PHF_X_BULK;      // the attention phase stores its output in the staged layout
         fits &= plan_phase(*pl, d, PH_SWIGLU, w.w_gate_up, H, F, nullptr, w.post_norm, x, act, l, &out[n++]);
         out[n - 1].flags |= PHF_OUT_SPLIT;   // the MLP activations go to memory in the layout the down projection stages
         fits &= plan_phase(*pl, d, PH_RESID, w.w_down, F, H, nullptr, nullptr, act, x, l, &out[n++]);

@@ -49,6 +49,12 @@ constexpr int MK_ATT_MW = (MK_NW + 1) / 2;       // warps whose partials fit the
 #endif
 #endif  // MK_TRACE
 
+// 1: one-head-per-CTA attention leaves the merge of its chunks to the O projection's prologue (every CTA merges);
+// 0: the last CTA of every head merges (atomic ticket) and the O projection stages the finished vector
+#ifndef MK_SPLIT_DEFER
+#define MK_SPLIT_DEFER 1
+#endif
+
 // ---- mbarrier / bulk copy primitives -----------------------------------------------------------------
 __device__ __forceinline__ unsigned smem_u32(const void *p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
 __device__ __forceinline__ void mbar_init(unsigned long long *b, unsigned count) {
@@ -628,6 +634,10 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, const MkPhase *s_p
     return ok;
 }
 
+// The attention output vector (n4 16-byte pieces) is stored as [even pieces | odd pieces], the layout of the shared-memory
+// activation buffers, so that the O projection stages it with two bulk copies.
+__device__ __forceinline__ int split_piece(int i4, int n4) { return (i4 & 1) * (n4 >> 1) + (i4 >> 1); }
+
 // ---- attention -----------------------------------------------------------------------------------------------
 // A CTA serves HG query heads of one GQA group over one chunk of the cached positions: HG = G (the whole
 // group shares every K/V row read: least traffic, for long contexts) or HG = 1 (every query head has
@@ -806,7 +816,7 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
         }
         const int qh = qh0 + h;
         if (nch == 1 && !defer_merge) {  // nothing to merge across CTAs
-            p.attn[qh * D + j] = oo / ll;
+            p.attn[split_piece((qh * D + j) >> 2, (p.nq * D) >> 2) * 4 + (j & 3)] = oo / ll;
         } else {
             p.part_o[(static_cast<size_t>(qh) * p.max_chunks + c) * D + j] = oo;
             if (j == 0) { p.part_m[qh * p.max_chunks + c] = mm; p.part_l[qh * p.max_chunks + c] = ll; }
@@ -860,7 +870,7 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
         }
         const float inv = 1.f / ll;
         acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-        reinterpret_cast<float4 *>(p.attn + (qh0 + oh) * D)[oj4] = acc;
+        reinterpret_cast<float4 *>(p.attn)[split_piece((qh0 + oh) * (D / 4) + oj4, (p.nq * D) >> 2)] = acc;
     }
     if (tid == 0) p.tickets[grp] = 0u;
 }
@@ -959,16 +969,16 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
     const int n_att = slot_row + 1;
     const bool att_split = !LONG || (n_att <= p.att_split_max_n && static_cast<long long>(p.nq) * MK_ATT_SPLIT_MAXC * 2 <= MK_PARTIAL_FLOATS);
     int merge_chunks = 0;   // chunks per head the O-projection prologue has to merge (split mode)
-    if (att_split) { int cl; att_chunking(p, n_att, 1, p.att_chunk_split, 32 / MK_ATT_LPP_SPLIT, ncta, merge_chunks, cl); }
+    if (att_split && MK_SPLIT_DEFER) { int cl; att_chunking(p, n_att, 1, p.att_chunk_split, 32 / MK_ATT_LPP_SPLIT, ncta, merge_chunks, cl); }
     for (int l = 0; l < p.n_layers && ok; ++l) {
         ok = gemv_phase(p, s_ph, s_rng, 4 * l, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token, 0, tid, prof_idx, &x_bar, x_parity);
         ok = grid_barrier(p, ++bar_no * ncta, abort_flag, &s_released, tid, prof_idx, top_up) && ok;
         if (ok) {
             if constexpr (LONG) {
-                if (att_split) attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, true, smem, tid, &s_flag);
+                if (att_split) attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, smem, tid, &s_flag);
                 else attention_phase<D, G, MK_ATT_LPP>(p, l, n_att, p.att_chunk_shared, false, smem, tid, &s_flag);
             } else {
-                attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, true, smem, tid, &s_flag);
+                attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, smem, tid, &s_flag);
             }
         }
         ok = grid_barrier(p, ++bar_no * ncta, abort_flag, &s_released, tid, prof_idx, top_up) && ok;
