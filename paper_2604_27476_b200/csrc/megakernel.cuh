@@ -970,25 +970,28 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
     const bool att_split = !LONG || (n_att <= p.att_split_max_n && static_cast<long long>(p.nq) * MK_ATT_SPLIT_MAXC * 2 <= MK_PARTIAL_FLOATS);
     int merge_chunks = 0;   // chunks per head the O-projection prologue has to merge (split mode)
     if (att_split && MK_SPLIT_DEFER) { int cl; att_chunking(p, n_att, 1, p.att_chunk_split, 32 / MK_ATT_LPP_SPLIT, ncta, merge_chunks, cl); }
-    for (int l = 0; l < p.n_layers && ok; ++l) {
-        ok = gemv_phase(p, s_ph, s_rng, 4 * l, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token, 0, tid, prof_idx, &x_bar, x_parity);
-        ok = grid_barrier(p, ++bar_no * ncta, abort_flag, &s_released, tid, prof_idx, top_up) && ok;
-        if (ok) {
+    // One loop over the operators of the step, with a single inlined copy of the streaming operator and of the grid barrier
+    // (the code of a step is executed once per layer: a small instruction footprint matters).  Operator 4l+1 (the O
+    // projection) is preceded by the attention of layer l.
+    const int n_layer_ops = 4 * p.n_layers;
+    for (int ph = 0; ph < p.nph && ok; ++ph) {
+        const bool layer_op = ph < n_layer_ops;
+        const bool after_attention = layer_op && (ph & 3) == 1;
+        if (after_attention) {
+            const int l = ph >> 2;
             if constexpr (LONG) {
                 if (att_split) attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, smem, tid, &s_flag);
                 else attention_phase<D, G, MK_ATT_LPP>(p, l, n_att, p.att_chunk_shared, false, smem, tid, &s_flag);
             } else {
                 attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, smem, tid, &s_flag);
             }
-        }
-        ok = grid_barrier(p, ++bar_no * ncta, abort_flag, &s_released, tid, prof_idx, top_up) && ok;
-        for (int k = 1; k < 4 && ok; ++k) {
-            ok = gemv_phase(p, s_ph, s_rng, 4 * l + k, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token,
-                            k == 1 ? merge_chunks : 0, tid, prof_idx, &x_bar, x_parity);
             ok = grid_barrier(p, ++bar_no * ncta, abort_flag, &s_released, tid, prof_idx, top_up) && ok;
+            if (!ok) break;
         }
+        ok = gemv_phase(p, s_ph, s_rng, ph, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token, after_attention ? merge_chunks : 0, tid,
+                        prof_idx, &x_bar, x_parity);
+        if (layer_op) ok = grid_barrier(p, ++bar_no * ncta, abort_flag, &s_released, tid, prof_idx, top_up) && ok;
     }
-    if (ok) ok = gemv_phase(p, s_ph, s_rng, 4 * p.n_layers, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token, 0, tid, prof_idx, &x_bar, x_parity);
     prof_stamp(p, tid, prof_idx);
     if (!ok || *abort_flag) {
         // aborted: wait (bounded) for the copies this warp still has in flight, then leave
