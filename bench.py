@@ -29,7 +29,7 @@ from edgefm_synth import CONFIGS, GLOBAL_SEED, first_token, make_kv, make_weight
 
 # DRAM traffic of one launch of the step kernel (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture,
 # see profiles/decode_megakernel_qwen2.5-1.5b_ctx2048.md); only the captured configuration has a value.
-NCU_TRAFFIC_BYTES = {"qwen2.5-1.5b": 3.147349e9 + 5.966e6}
+NCU_TRAFFIC_BYTES = {"qwen2.5-1.5b": 3.146461e9 + 3.875e6}
 
 METRIC = "batch1_decode_ms_per_token"
 UNIT = "ms/token"

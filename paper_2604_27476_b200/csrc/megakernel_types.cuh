@@ -13,8 +13,14 @@ constexpr int MK_ATT_SPLIT_MAXC = 12;            // chunks per head when every q
 constexpr int MK_PARTIAL_FLOATS = 2048;          // shared-memory scratch: split-K partial sums / chunk statistics
 // Warps per CTA of the two builds of the kernel: the short-context build favours instruction streams, the
 // long-context build (grouped attention keeps G heads of accumulators per warp) favours registers.
-constexpr int MK_NW_SHORT = 12;
-constexpr int MK_NW_LONG = 8;
+#ifndef MK_NW_SHORT_VALUE
+#define MK_NW_SHORT_VALUE 12
+#endif
+#ifndef MK_NW_LONG_VALUE
+#define MK_NW_LONG_VALUE 8
+#endif
+constexpr int MK_NW_SHORT = MK_NW_SHORT_VALUE;
+constexpr int MK_NW_LONG = MK_NW_LONG_VALUE;
 
 enum { PH_QKV = 0, PH_RESID = 1, PH_SWIGLU = 2, PH_LMHEAD = 3 };
 
