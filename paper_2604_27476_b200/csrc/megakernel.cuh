@@ -439,24 +439,24 @@ __device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkPhase *
         MK_TRACE(p, ph_index, warp, lane, trace_slot); ++trace_slot;
         if (!consume_tile<NR>(p, s_ph, s_rng, kcs, j & smask, do_refill, ws, xsA, xsB, abort_flag, y, warp, lane)) return false;
         MK_TRACE(p, ph_index, warp, lane, trace_slot); ++trace_slot;
-        if (split) {
+        // every lane holds all sums of the tile; lane r takes those of unit r, so that the units finish side by side in one
+        // pass over one copy of the epilogue code
+        const bool paired = kind == PH_QKV || kind == PH_SWIGLU;
+        constexpr int NU = NR >= 2 ? NR / 2 : 1;
+        float lo = y[0], hi = NR >= 2 ? y[NU] : 0.f;
 #pragma unroll
-            for (int r = 0; r < NR; ++r)
-                if (lane == r) s_partial[j * NR + r] = y[r];
-        } else {
-            const int u0 = (it0 + j) * rw;
-            constexpr int NU = NR >= 2 ? NR / 2 : 1;
-            if (kind == PH_QKV || kind == PH_SWIGLU) {
-                if constexpr (NR >= 2) {
-#pragma unroll
-                    for (int r = 0; r < NU; ++r)
-                        if (lane == r && u0 + r < units_total) apply_epilogue(p, P, cx, u0 + r, y[r] * cx.rscale, y[r + NU] * cx.rscale);
-                }
-            } else {
-#pragma unroll
-                for (int r = 0; r < NR; ++r)
-                    if (lane == r && u0 + r < units_total) apply_epilogue(p, P, cx, u0 + r, y[r] * cx.rscale, 0.f);
+        for (int r = 1; r < NR; ++r) {
+            if (lane == r) {
+                lo = y[r];
+                if (r < NU) hi = y[r + NU];
             }
+        }
+        if (split) {
+            if (lane < NR) s_partial[j * NR + lane] = lo;
+        } else {
+            const int u = (it0 + j) * rw + lane;
+            const int cnt = paired ? NU : NR;
+            if ((NR >= 2 || !paired) && lane < cnt && u < units_total) apply_epilogue(p, P, cx, u, lo * cx.rscale, hi * cx.rscale);
         }
     }
     return true;
