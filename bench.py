@@ -146,8 +146,15 @@ def main():
     ap.add_argument("--cpu-steps", type=int, default=3)
     ap.add_argument("--vocab-subset", type=int, default=0,
                     help="prune the output layer to this many evenly spaced token ids (0 = full vocabulary, the headline workload)")
+    ap.add_argument("--phase-timeline", action="store_true",
+                    help="instead of the benchmark: print the per-operator timeline of one step from the kernel's own device timestamps")
     args = ap.parse_args()
     cfg = CONFIGS[args.config]
+    if args.phase_timeline:
+        from paper_2604_27476_b200 import build as cuda_build, timeline
+        cuda_build.build()
+        print(timeline.format_table(timeline.summarize(timeline.collect(cfg), cfg), cfg))
+        return
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

@@ -47,7 +47,8 @@ class _Weights(ctypes.Structure):
 
 EXPORTS = ("edgefm_create", "edgefm_prefill_kv", "edgefm_decode_step", "edgefm_destroy", "edgefm_get_length",
            "edgefm_export_kv", "edgefm_get_launches_per_step", "edgefm_last_error", "edgefm_version",
-           "edgefm_sync_status", "edgefm_debug_profile", "edgefm_decode_step_static", "edgefm_set_vocab_subset", "edgefm_append_kv")
+           "edgefm_sync_status", "edgefm_debug_profile", "edgefm_debug_set_wait_limit", "edgefm_decode_step_static", "edgefm_set_vocab_subset",
+           "edgefm_append_kv")
 
 
 def library_path() -> Path:
@@ -58,9 +59,7 @@ def load_library():
     global _lib
     if _lib is not None:
         return _lib
-    import os
-    alt = os.environ.get("EDGEFM_LIBRARY")   # e.g. an instrumented build of the same sources
-    path = Path(alt) if alt else _LIB_PATH
+    path = _LIB_PATH
     if not path.exists():
         raise FileNotFoundError(f"{path} is missing: build it with `python -m paper_2604_27476_b200.build` "
                                 "(there is no CPU fallback)")
@@ -84,6 +83,8 @@ def load_library():
     L.edgefm_sync_status.argtypes = [vp, vp]
     L.edgefm_debug_profile.restype = ctypes.c_int
     L.edgefm_debug_profile.argtypes = [vp, vp, i64, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    L.edgefm_debug_set_wait_limit.restype = ctypes.c_int
+    L.edgefm_debug_set_wait_limit.argtypes = [vp, ctypes.c_uint32, i32]
     L.edgefm_decode_step_static.restype = ctypes.c_int
     L.edgefm_decode_step_static.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Weights), vp, vp, i32, i32, i32, i32, vp, vp, vp]
     L.edgefm_append_kv.restype = ctypes.c_int
@@ -185,6 +186,10 @@ def edgefm_set_vocab_subset(ctx, token_ids, stream=None):
 
 def edgefm_sync_status(ctx, stream=None):
     _check(load_library().edgefm_sync_status(ctx, stream), ctx)
+
+
+def edgefm_debug_set_wait_limit(ctx, limit_ns, extra_barrier_arrivals=0):
+    _check(load_library().edgefm_debug_set_wait_limit(ctx, limit_ns, extra_barrier_arrivals), ctx)
 
 
 def edgefm_debug_profile(ctx):

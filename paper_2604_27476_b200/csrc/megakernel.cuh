@@ -4,50 +4,39 @@
 // split over five operators that depend on one another.  Separate kernels drain and refill the memory
 // pipeline at every boundary.  Here the weight stream is decoupled from the dependency chain:
 //
-//   * The step's weight traffic is a static schedule (QKV, O, gate/up, down of every layer, then
-//     lm_head).  Every CTA owns a fixed share of each operator's rows, and every warp of the CTA a fixed
-//     sequence of tiles (a few rows, or one K slice of a long row) across the WHOLE step.
-//   * Each warp keeps a private byte ring in shared memory filled with its next tiles (up to MK_MAXF in
-//     flight, variable size, allocated first-in first-out) by bulk async copies (TMA: cp.async.bulk +
-//     mbarrier complete_tx).  When it has consumed a tile it immediately fetches as many further tiles
-//     as now fit -- regardless of operator boundaries -- so the short operators of a layer are already
-//     on chip when their turn comes, and HBM keeps streaming while the arithmetic waits at a grid
-//     barrier, stages an activation vector or runs attention.
-//     Ring space and mbarriers are armed and drained by the same warp, in program order, so the one-bit
-//     mbarrier phase parity cannot alias and no "empty" barrier is needed (a proxy fence orders the
-//     warp's reads before the next asynchronous write).
-//   * A tile is multiplied with the activation vector staged in shared memory; the fused epilogues
-//     (bias + RoPE + KV append, residual add, SwiGLU, logits + argmax) run in the warp that owns the rows.
+//   * The step's weight traffic is a static schedule made on the host (QKV, O, gate/up, down of every layer,
+//     then lm_head).  Every CTA owns a fixed share of each operator's rows; the share is cut into tiles of up
+//     to 16 rows x 256 columns, and every consumer warp owns a fixed list of tiles (the same for every layer).
+//   * One more warp of the CTA only FEEDS: lane w walks the tile list of consumer warp w over the whole step
+//     and fetches the tiles with 2-D TMA tensor copies (cp.async.bulk.tensor.2d, mbarrier complete_tx) into
+//     warp w's private ring of shared-memory slots.  It never waits: every pass it tests which slots have been
+//     released and refills those.  The weights do not depend on the computation, so the stream runs ahead
+//     across operator boundaries; HBM keeps streaming while the consumers wait at a grid barrier, stage an
+//     activation vector or run attention.  Every slot has a "full" and an "empty" mbarrier, armed by one lane
+//     and drained by one warp strictly in order, so the one-bit phase parity cannot alias.
+//   * A consumer warp waits for its next tile, multiplies it with the 256 activations of the tile's columns
+//     (8 per lane, from the vector staged in shared memory) into 16 row accumulators and releases the slot.
+//     Consecutive tiles of a warp cover the same rows; only at the end of a run of tiles are the 16 sums
+//     reduced across the lanes (a butterfly of 16 + 1 shuffles).  The fused epilogues (bias + RoPE + KV append,
+//     residual add, SwiGLU, logits + argmax) run in the warp when it has seen all columns of its rows, else the
+//     sums meet in shared memory after the operator, in a fixed order.
 //   * Between dependent operators all CTAs meet at a grid barrier (monotonic counter in global memory,
 //     release/acquire, bounded spin).  Attention (split-KV, exact log-sum-exp merge) runs between two
 //     barriers.
 //
 // Every wait is bounded: on expiry the CTA records EDGEFM_ERR_TIMEOUT in the device state, stops
 // issuing copies, waits (bounded) for the copies it has in flight and returns.
-// This file is the body of the kernel.  It is included once per build (MK_NS = namespace, MK_NW_VALUE = warps per
-// CTA); everything that does not depend on the number of warps lives in megakernel_types.cuh.
+// This file is the body of the kernel.  It is included once per build (MK_NS = namespace, MK_NW_VALUE = consumer
+// warps per CTA); everything that does not depend on the number of warps lives in megakernel_types.cuh.
 #include "megakernel_types.cuh"
 
 namespace edgefm {
 namespace MK_NS {
 
-constexpr int MK_NW = MK_NW_VALUE;               // warps per CTA (each streams and consumes its own tiles)
-constexpr int MK_NT = MK_NW * 32;
+constexpr int MK_NW = MK_NW_VALUE;               // consumer warps per CTA
+constexpr int MK_NT = MK_NW * 32;                // consumer threads
+constexpr int MK_THREADS = MK_NT + 32;           // + the feeding warp
 constexpr int MK_ATT_MW = (MK_NW + 1) / 2;       // warps whose partials fit the merge area at once
-
-// Optional fine-grained trace of one operator in CTA 0 (compile with -DEDGEFM_TRACE_PHASE=<operator index>):
-// lane 0 of every warp appends %globaltimer stamps behind the regular profile table.
-#ifndef MK_TRACE
-#ifdef EDGEFM_TRACE_PHASE
-#define MK_TRACE(p, ph, warp, lane, slot)                                                                          \
-    do {                                                                                                           \
-        if ((p).prof && (ph) == EDGEFM_TRACE_PHASE && blockIdx.x == 0 && (lane) == 0 && (slot) < 16)               \
-            (p).prof[static_cast<size_t>(gridDim.x) * (p).prof_stride + (warp) * 16 + (slot)] = global_ns();        \
-    } while (0)
-#else
-#define MK_TRACE(p, ph, warp, lane, slot) do {} while (0)
-#endif
-#endif  // MK_TRACE
 
 // 1: one-head-per-CTA attention leaves the merge of its chunks to the O projection's prologue (every CTA merges);
 // 0: the last CTA of every head merges (atomic ticket) and the O projection stages the finished vector
@@ -60,6 +49,9 @@ __device__ __forceinline__ unsigned smem_u32(const void *p) { return static_cast
 __device__ __forceinline__ void mbar_init(unsigned long long *b, unsigned count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(b)), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(unsigned long long *b) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(b)) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long *b, unsigned bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(bytes) : "memory");
 }
@@ -68,6 +60,18 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long *b, unsigned pa
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(b)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// non-blocking test (the feeding lanes poll many barriers and must never sleep on one)
+__device__ __forceinline__ bool mbar_test_wait(unsigned long long *b, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(smem_u32(b)), "r"(parity)
@@ -93,19 +97,21 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long *b, unsigned parity
     *abort_flag = 1;
     return false;
 }
-__device__ __forceinline__ void bulk_copy_g2s(void *dst, const void *src, unsigned bytes, unsigned long long *bar,
-                                              unsigned long long policy) {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
-        ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
-        : "memory");
-}
 __device__ __forceinline__ void bulk_copy_g2s_plain(void *dst, const void *src, unsigned bytes, unsigned long long *bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
                  : "memory");
 }
-__device__ __forceinline__ void cta_sync() { __syncthreads(); }
+// One box of a weight matrix (tensor map `map`: 256 columns x the map's box height) starting at (column x, row y).
+// x * 2 bytes is a multiple of 16 by construction (x is a multiple of 256); no multicast.
+__device__ __forceinline__ void tma_load_box(void *dst, const void *map, int x, int y, unsigned long long *bar, unsigned long long policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(policy)
+        : "memory");
+}
+// all consumer threads of the CTA (the feeding warp never joins)
+__device__ __forceinline__ void cta_sync() { asm volatile("bar.sync 1, %0;" ::"n"(MK_NT) : "memory"); }
 
 __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned *p) {
     unsigned v;
@@ -131,180 +137,110 @@ __device__ __forceinline__ bool diag_fail(const MkParams &p, volatile int *abort
     return false;
 }
 
-// All threads of all CTAs meet here.  Returns false when the wait expired (step aborted).
-// While the CTA waits, every warp tops up its weight ring (the fetches short operators skipped).
-template <typename Refill>
-__device__ __forceinline__ bool grid_barrier(const MkParams &p, unsigned target, volatile int *abort_flag, volatile int *s_released,
-                                             int tid, int &prof_idx, Refill &&refill_fn) {
+// All consumer threads of all CTAs meet here.  Returns false when the wait expired (step aborted).
+__device__ __forceinline__ bool grid_barrier(const MkParams &p, unsigned target, volatile int *abort_flag, int tid, int &prof_idx) {
     cta_sync();
     prof_stamp(p, tid, prof_idx);   // this CTA's share of the operator is done
     if (tid == 0 && !*abort_flag) {
-        *s_released = 0;
         asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.barrier) : "memory");
-    }
-    refill_fn();
-    // lane 0 of the first MK_BAR_POLLERS warps polls the counter; their polls interleave in time, which shortens the
-    // delay between the last arrival and its detection; whoever sees it first releases the others
-    if ((tid & 31) == 0 && (tid >> 5) < MK_BAR_POLLERS && !*abort_flag) {
         unsigned it = 0;
         unsigned long long t0 = 0;
         while (ld_acquire_gpu(p.barrier) < target) {
-            if (*s_released) break;
             if ((++it & 63u) == 0u) {
                 const unsigned long long now = global_ns();
                 if (t0 == 0) t0 = now;
                 else if (now - t0 > p.spin_limit) { *abort_flag = 1; p.state->status = 6; break; }
             }
         }
-        *s_released = 1;
     }
     cta_sync();
     prof_stamp(p, tid, prof_idx);   // released by the slowest CTA
     return !*abort_flag;
 }
 
-// Work items [it0, it1) of CTA `cta` in a phase with `total` items.
-__device__ __forceinline__ void item_range(int total, int cta, int ncta, int &it0, int &it1) {
-    it0 = static_cast<int>((static_cast<long long>(total) * cta) / ncta);
-    it1 = static_cast<int>((static_cast<long long>(total) * (cta + 1)) / ncta);
-}
-
-// First row of block `blk` (0 = low/plain, 1 = partner rows) of item `it`, and the number of valid units.
-__device__ __forceinline__ int item_rows(const MkPhase &P, const MkParams &p, int it, int blk, int &cnt) {
-    const int u0 = it * P.rw;
-    cnt = min(P.rw, P.units_total - u0);
-    if (P.kind == PH_QKV) {
+// First weight row of unit u of an operator (its partner row, if any, is `partner` rows further).
+__device__ __forceinline__ int unit_row(const MkParams &p, int kind, int u) {
+    if (kind == PH_QKV) {
         const int half = p.d >> 1;
-        const int head = u0 >> p.half_shift, i0 = u0 & (half - 1);
-        return head * p.d + i0 + blk * half;
+        return (u >> p.half_shift) * p.d + (u & (half - 1));
     }
-    if (P.kind == PH_SWIGLU) return u0 + blk * p.F;
-    return u0;
+    return u;
 }
 
-// ---- a warp's position in its tile sequence over the whole step ----------------------------------------
-// Tile j of a CTA's share of an operator is slice (j & (ksplit-1)) of item (j >> s_shift); warp w owns the
-// tiles j = w, w + NW, ...  The CTA's item range of every operator is tabulated once per launch (s_rng).
-// The cursor keeps the constants of its operator in registers so that issuing a tile costs no shared-memory
-// round trips.
-struct TileCursor {
-    int ph;        // operator index (nph = past the end)
-    int j;         // tile index inside this CTA's share of the operator
-    int it0;       // first item of this CTA in operator ph
-    int n_tiles;   // tiles of this CTA in operator ph
-    // cached from s_ph[ph]
-    const uint16_t *W;
-    int K, rw, s_shift, smask, units_total, kind;
-    unsigned seg_bytes;      // bytes of one row slice
-    unsigned alloc_bytes;    // ring bytes of one tile
-    unsigned partner_elems;  // elements between the two blocks of a paired tile (0: single block)
-};
-__device__ __forceinline__ void cursor_enter_phase(TileCursor &c, const MkParams &p, const MkPhase *s_ph, const int2 *s_rng, int warp) {
-    while (c.ph < p.nph) {  // skip operators in which this warp owns no tile
-        const MkPhase &P = s_ph[c.ph];
-        const int2 r = s_rng[c.ph];
-        c.it0 = r.x;
-        c.n_tiles = (r.y - r.x) << P.s_shift;
-        if (warp < c.n_tiles) {
-            c.j = warp;
-            c.W = P.W; c.K = P.K; c.rw = P.rw; c.s_shift = P.s_shift; c.smask = P.ksplit - 1; c.units_total = P.units_total;
-            c.kind = P.kind;
-            c.seg_bytes = static_cast<unsigned>(P.kcs) * 16u;
-            const bool paired = P.kind == PH_QKV || P.kind == PH_SWIGLU;
-            c.alloc_bytes = (paired ? 2u : 1u) * P.rw * c.seg_bytes;
-            c.partner_elems = !paired ? 0u : static_cast<unsigned>(P.kind == PH_QKV ? (p.d >> 1) : p.F) * static_cast<unsigned>(P.K);
-            return;
-        }
-        ++c.ph;
-    }
-}
-__device__ __forceinline__ void cursor_advance(TileCursor &c, const MkParams &p, const MkPhase *s_ph, const int2 *s_rng, int warp) {
-    c.j += MK_NW;
-    if (c.j < c.n_tiles) return;
-    ++c.ph;
-    cursor_enter_phase(c, p, s_ph, s_rng, warp);
-}
-
-// Fetch the tile under cursor `c` into ring space.  Called by a whole warp after __syncwarp(); lane 0 issues.
-__device__ __forceinline__ bool issue_tile(const MkParams &p, const TileCursor &c, unsigned char *dst, unsigned long long *bar,
-                                           unsigned long long policy, volatile int *abort_flag, int lane) {
-    const int it = c.it0 + (c.j >> c.s_shift);
-    const int sl = c.j & c.smask;
-    const int u0 = it * c.rw;
-    const int cnt = min(c.rw, c.units_total - u0);
-    int row_lo = u0;
-    if (c.kind == PH_QKV) {
-        const int half = p.d >> 1;
-        row_lo = (u0 >> p.half_shift) * p.d + (u0 & (half - 1));
-    }
-    const unsigned bytes = static_cast<unsigned>(cnt) * c.seg_bytes;   // one contiguous run per block
-    // bounds: at least one row, inside the matrix (16-byte rule holds by construction: K % 8 == 0, slices of
-    // kcs 16-byte pieces, 16-byte aligned bases and ring offsets, all checked on the host)
-    if (cnt < 1 || (sl + 1) * static_cast<int>(c.seg_bytes >> 1) > c.K) return diag_fail(p, abort_flag, 1, c.ph, it);
-    if (lane == 0) {
-        const uint16_t *src = c.W + static_cast<size_t>(row_lo) * c.K + static_cast<size_t>(sl) * (c.seg_bytes >> 1);
-        if (c.partner_elems) {
-            mbar_arrive_expect_tx(bar, bytes * 2u);
-            bulk_copy_g2s(dst, src, bytes, bar, policy);
-            bulk_copy_g2s(dst + static_cast<size_t>(c.rw) * c.seg_bytes, src + c.partner_elems, bytes, bar, policy);
-        } else {
-            mbar_arrive_expect_tx(bar, bytes);
-            bulk_copy_g2s(dst, src, bytes, bar, policy);
-        }
-    }
-    return true;
-}
-
-// Per-warp streaming state.
-struct WarpStream {
-    TileCursor pf;            // next tile to fetch into shared memory
-    unsigned consumed;        // tiles consumed so far by this warp
-    unsigned issued;          // tiles fetched so far (issued - consumed <= MK_MAXF)
-    unsigned char *ring;      // this warp's byte ring
-    int head, tail;           // ring offsets: [head, tail) (cyclically) holds the tiles in flight
-    bool wrapped;             // tail has wrapped around the ring end and head has not yet
-    unsigned long long fifo;  // ring offset / 16 of tile k in the 16-bit field k % MK_MAXF
-    unsigned long long *bars; // [MK_MAXF]
+// ---- the feeding warp: lane w refills the ring of consumer warp w -------------------------------------------
+// Tiles are fetched in the order the consumer takes them; slot k % S of round k / S.  A slot is refilled once its
+// "empty" barrier has completed the previous round (the consumer arrives there after its last read of the slot).
+__device__ __forceinline__ void feed_rings(const MkParams &p, const MkOp *s_ops, const int *s_tab, unsigned char *ring,
+                                           unsigned long long *full_bar, unsigned long long *empty_bar, volatile int *abort_flag,
+                                           volatile unsigned *s_issued, int lane) {
+    if (lane >= MK_NW) return;
+    const int *tab = s_tab + lane * MK_WARP_TAB;
+    const int n_layer = tab[1] + tab[2] + tab[3] + tab[4], n_lm = tab[6];
+    const uint2 *layer_list = p.tiles + tab[0], *lm_list = p.tiles + tab[5];
+    const long long total = static_cast<long long>(n_layer) * p.n_layers + n_lm;
+    unsigned char *my_ring = ring + static_cast<size_t>(lane) * p.slots * p.slot_bytes;
+    unsigned long long *fb = full_bar + lane * MK_MAX_SLOTS, *eb = empty_bar + lane * MK_MAX_SLOTS;
     unsigned long long policy;
-};
-static_assert(MK_MAXF == 4, "fifo packs four 16-bit offsets into one register");
-__device__ __forceinline__ int fifo_get(const WarpStream &ws, unsigned k) {
-    return static_cast<int>((ws.fifo >> ((k & 3u) * 16u)) & 0xffffull) << 4;
-}
-__device__ __forceinline__ void fifo_set(WarpStream &ws, unsigned k, int off) {
-    const unsigned sh = (k & 3u) * 16u;
-    ws.fifo = (ws.fifo & ~(0xffffull << sh)) | (static_cast<unsigned long long>(off >> 4) << sh);
-}
-
-// Fetch as many of this warp's next tiles as fit its ring (first-in first-out space, at most MK_MAXF in
-// flight).  Whole warp, after __syncwarp() when ring space has just been read.
-__device__ __forceinline__ bool refill(const MkParams &p, const MkPhase *s_ph, const int2 *s_rng, WarpStream &ws,
-                                       volatile int *abort_flag, int warp, int lane) {
-    bool fenced = false;
-    while (ws.issued - ws.consumed < MK_MAXF && ws.pf.ph < p.nph) {
-        const int sz = static_cast<int>(ws.pf.alloc_bytes);
-        if (ws.issued == ws.consumed) { ws.head = 0; ws.tail = 0; ws.wrapped = false; }   // empty: restart at the base
-        int off;
-        if (!ws.wrapped) {                   // in flight: [head, tail); free: [tail, R) and [0, head)
-            if (ws.tail + sz <= p.ring_bytes) off = ws.tail;
-            else if (sz <= ws.head) { off = 0; ws.wrapped = true; }   // wrap (the bytes behind tail stay unused this round)
-            else break;
-        } else {                              // in flight: [head, R) and [0, tail); free: [tail, head)
-            if (ws.tail + sz <= ws.head) off = ws.tail;
-            else break;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    int slot = 0;
+    unsigned round = 0;          // times this lane has gone around its ring
+    int layer = 0, i = 0;        // next tile: i-th of the layer list (layer < n_layers) or of the output-layer list
+    if (n_layer == 0) layer = p.n_layers;
+    long long done = 0;
+    int fenced_op = -1;
+    unsigned idle = 0;
+    unsigned long long t_idle = 0;
+    uint2 d = make_uint2(0u, 0u);
+    if (total > 0) d = __ldg(layer < p.n_layers ? layer_list : lm_list);
+    while (done < total) {
+        if (round > 0 && !mbar_test_wait(&eb[slot], (round - 1) & 1u)) {
+            // nothing to do for this lane right now; give up after the bound (the consumers never released the slot)
+            if ((++idle & 255u) == 0u) {
+                if (*abort_flag) break;
+                const unsigned long long now = global_ns();
+                if (t_idle == 0) t_idle = now;
+                else if (now - t_idle > p.spin_limit) { *abort_flag = 1; break; }
+            }
+            continue;
         }
-        if (!fenced) {
-            // ring space was read through the generic proxy by this warp: order those reads before async writes
-            if (lane == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            fenced = true;
+        idle = 0; t_idle = 0;
+        if (*abort_flag) break;
+        const bool lm = layer >= p.n_layers;
+        const int op = static_cast<int>((d.y >> 20) & 7u);
+        const int opi = lm ? 4 * p.n_layers : 4 * layer + op;
+        const MkOp &P = s_ops[opi];
+        const int m = static_cast<int>(d.y & 31u), kcol = static_cast<int>((d.x >> 20) & 0xffu);
+        const int variant = static_cast<int>((d.x >> 28) & 3u);
+        const int u0 = static_cast<int>(d.x & 0xfffffu);
+        const bool paired = P.kind == PH_QKV || P.kind == PH_SWIGLU;
+        const int row = unit_row(p, P.kind, u0);
+        const unsigned box_bytes = static_cast<unsigned>(m) * (MK_TILE_COLS * 2);
+        // bounds (the host made the schedule; a corrupt entry must not reach the copy engine)
+        if (m < 1 || m > MK_TILE_ROWS || (paired && m > 8) || kcol * MK_TILE_COLS >= P.K || u0 + m > P.units_total ||
+            static_cast<int>(box_bytes) * (paired ? 2 : 1) > p.slot_bytes || (lm ? op != 4 : op > 3)) {
+            diag_fail(p, abort_flag, 1, opi, u0);
+            break;
         }
-        if (!issue_tile(p, ws.pf, ws.ring + off, &ws.bars[ws.issued & (MK_MAXF - 1)], ws.policy, abort_flag, lane)) return false;
-        fifo_set(ws, ws.issued, off);
-        ws.tail = off + sz;
-        ++ws.issued;
-        cursor_advance(ws.pf, p, s_ph, s_rng, warp);
+        const unsigned char *map = p.maps + (static_cast<size_t>(opi) * MK_MAX_VARIANTS + variant) * 128;
+        if (opi != fenced_op && (p.map_fence == 2 || (p.map_fence == 1 && lm))) {
+            // the host may have rewritten this operator's tensor maps since the last launch (another vocabulary subset, or a
+            // static call with other weights): order the copy engine's view of them behind what is in memory now
+            fenced_op = opi;
+            for (int v = 0; v < MK_MAX_VARIANTS; ++v)
+                asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(p.maps + (static_cast<size_t>(opi) * MK_MAX_VARIANTS + v) * 128) : "memory");
+        }
+        unsigned char *dst = my_ring + static_cast<size_t>(slot) * p.slot_bytes;
+        mbar_arrive_expect_tx(&fb[slot], paired ? 2u * box_bytes : box_bytes);
+        tma_load_box(dst, map, kcol * MK_TILE_COLS, row, &fb[slot], policy);
+        if (paired) tma_load_box(dst + p.hi_off, map, kcol * MK_TILE_COLS, row + (P.kind == PH_QKV ? (p.d >> 1) : p.F), &fb[slot], policy);
+        ++done;
+        s_issued[lane] = static_cast<unsigned>(done);
+        if (++slot == p.slots) { slot = 0; ++round; }
+        // next tile
+        ++i;
+        if (!lm && i == n_layer) { i = 0; ++layer; }
+        if (done < total) d = __ldg((layer < p.n_layers ? layer_list : lm_list) + i);
     }
-    return true;
 }
 
 struct ItemCtx {
@@ -317,11 +253,9 @@ struct ItemCtx {
 };
 
 // ---- fused epilogue of one output unit (a row, or a row pair) ------------------------------------------------
-// pre: the value the epilogue adds (old residual / the two biases) was fetched ahead into pre_lo, pre_hi.
-__device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkPhase &P, ItemCtx &cx, int u, float lo, float hi,
-                                               bool pre = false, float pre_lo = 0.f, float pre_hi = 0.f) {
+__device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkOp &P, ItemCtx &cx, int u, float lo, float hi) {
     if (P.kind == PH_RESID) {
-        P.out[u] = (pre ? pre_lo : __ldcg(P.out + u)) + lo;
+        P.out[u] = __ldcg(P.out + u) + lo;
     } else if (P.kind == PH_LMHEAD) {
         if (cx.logits_out) cx.logits_out[u] = lo;
         if (arg_better(lo, u, cx.best_v, cx.best_i)) { cx.best_v = lo; cx.best_i = u; }
@@ -338,8 +272,8 @@ __device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkPhase 
         const int head = u >> p.half_shift, i = u & (half - 1);
         const int row_lo = head * p.d + i, row_hi = row_lo + half;
         if (P.bias) {
-            lo += pre ? pre_lo : bf16_bits_to_f32(P.bias[row_lo]);
-            hi += pre ? pre_hi : bf16_bits_to_f32(P.bias[row_hi]);
+            lo += bf16_bits_to_f32(P.bias[row_lo]);
+            hi += bf16_bits_to_f32(P.bias[row_hi]);
         }
         const size_t layer_off = static_cast<size_t>(P.layer) * p.nkv * p.max_context * p.d;
         if (head < p.nq + p.nkv) {
@@ -361,104 +295,87 @@ __device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkPhase 
     }
 }
 
-// ---- one tile (NR row slices of kcs 16-byte pieces) by one warp: wait, multiply, re-arm the slot ------------
-template <int NR>
-__device__ __forceinline__ bool consume_tile(const MkParams &p, const MkPhase *s_ph, const int2 *s_rng, int kcs, int slice, bool do_refill,
-                                             WarpStream &ws, const float4 *xsA, const float4 *xsB, volatile int *abort_flag,
-                                             float (&out)[NR], int warp, int lane) {
-    float acc[NR], acc2[NR];   // two chains per row halve the dependent-FMA latency
+// Sum the 16 accumulator rows across the 32 lanes: afterwards lanes 2r and 2r+1 hold the sum of row r.
+// Each step pairs lanes `off` apart: a lane keeps one half of its values and hands the other half over,
+// 8 + 4 + 2 + 1 exchanges, then one more exchange between the two lanes that share a row.
+__device__ __forceinline__ float reduce_rows(float (&a)[MK_TILE_ROWS], int lane) {
 #pragma unroll
-    for (int r = 0; r < NR; ++r) { acc[r] = 0.f; acc2[r] = 0.f; }
-    if (ws.consumed == ws.issued) {   // not fetched yet (short operator whose tiles exceed the ring): fetch on demand
-        __syncwarp();
-        if (!refill(p, s_ph, s_rng, ws, abort_flag, warp, lane)) return false;
-        if (ws.consumed == ws.issued) return diag_fail(p, abort_flag, 2, kcs, NR);
-    }
-    const unsigned q = ws.consumed & (MK_MAXF - 1);
-    const unsigned par = (ws.consumed / MK_MAXF) & 1u;
-    if (!mbar_wait(&ws.bars[q], par, abort_flag, p.spin_limit)) return false;
-    const uint4 *t = reinterpret_cast<const uint4 *>(ws.ring + fifo_get(ws, ws.consumed));
-    const float4 *a = xsA + slice * kcs, *b = xsB + slice * kcs;
-    auto fma_chunk = [&](const uint4 &w, const float4 &x0, const float4 &x1, int r) {
-        acc[r] = fmaf(bf16lo(w.x), x0.x, acc[r]);  acc2[r] = fmaf(bf16hi(w.x), x0.y, acc2[r]);
-        acc[r] = fmaf(bf16lo(w.y), x0.z, acc[r]);  acc2[r] = fmaf(bf16hi(w.y), x0.w, acc2[r]);
-        acc[r] = fmaf(bf16lo(w.z), x1.x, acc[r]);  acc2[r] = fmaf(bf16hi(w.z), x1.y, acc2[r]);
-        acc[r] = fmaf(bf16lo(w.w), x1.z, acc[r]);  acc2[r] = fmaf(bf16hi(w.w), x1.w, acc2[r]);
-    };
-    constexpr int UN = NR >= 8 ? 1 : (NR == 4 ? 2 : 3);   // lane-chunks whose loads are issued together
-    int c = lane;
-    for (; c + 32 * (UN - 1) < kcs; c += 32 * UN) {
-        float4 x0[UN], x1[UN];
-        uint4 w[UN][NR];
+    for (int off = 16, n = MK_TILE_ROWS; off >= 2; off >>= 1, n >>= 1) {
+        const bool up = (lane & off) != 0;
 #pragma unroll
-        for (int u = 0; u < UN; ++u) {
-            x0[u] = a[c + 32 * u]; x1[u] = b[c + 32 * u];
-#pragma unroll
-            for (int r = 0; r < NR; ++r) w[u][r] = t[r * kcs + c + 32 * u];
-        }
-#pragma unroll
-        for (int u = 0; u < UN; ++u)
-#pragma unroll
-            for (int r = 0; r < NR; ++r) fma_chunk(w[u][r], x0[u], x1[u], r);
-    }
-    for (; c < kcs; c += 32) {
-        const float4 x0 = a[c], x1 = b[c];
-#pragma unroll
-        for (int r = 0; r < NR; ++r) fma_chunk(t[r * kcs + c], x0, x1, r);
-    }
-    ++ws.consumed;
-    {   // free the tile's bytes: head moves to the next tile in flight (back to the ring start once it passes the wrap)
-        const int nh = ws.consumed < ws.issued ? fifo_get(ws, ws.consumed) : ws.tail;
-        if (nh < ws.head) ws.wrapped = false;
-        ws.head = nh;
-    }
-    __syncwarp();
-    if (do_refill && !refill(p, s_ph, s_rng, ws, abort_flag, warp, lane)) return false;
-#pragma unroll
-    for (int r = 0; r < NR; ++r) out[r] = warp_sum(acc[r] + acc2[r]);
-    return true;
-}
-
-// Tiles of this warp in one operator.  Whole items (ksplit == 1): the warp that owns the rows finishes
-// them (lane r = unit r).  Split items: the partial sum of every tile goes to shared memory.
-template <int NR>
-__device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkPhase *s_ph, const int2 *s_rng, const MkPhase &P, int it0,
-                                              int n_tiles, WarpStream &ws, const float4 *xsA, const float4 *xsB,
-                                              volatile int *abort_flag, ItemCtx &cx, float *s_partial, int warp, int lane,
-                                              int ph_index) {
-    int trace_slot = 1;
-    // operator constants in registers (the asm memory clobbers would otherwise force shared-memory reloads)
-    const int kcs = P.kcs, smask = P.ksplit - 1, rw = P.rw, kind = P.kind, units_total = P.units_total;
-    const bool split = P.split != 0;
-    if (NR * kcs * 16 > p.slot_bytes || P.ksplit * kcs * 32 > p.xbuf_bytes) return diag_fail(p, abort_flag, 2, kcs, NR);
-    // short operators leave the ring alone (it is topped up while the CTA waits at the grid barrier), so that
-    // nothing but the arithmetic sits on their critical path; streaming operators refill after every tile
-    const bool do_refill = n_tiles > 2 * MK_NW;
-    for (int j = warp; j < n_tiles; j += MK_NW) {
-        float y[NR];
-        MK_TRACE(p, ph_index, warp, lane, trace_slot); ++trace_slot;
-        if (!consume_tile<NR>(p, s_ph, s_rng, kcs, j & smask, do_refill, ws, xsA, xsB, abort_flag, y, warp, lane)) return false;
-        MK_TRACE(p, ph_index, warp, lane, trace_slot); ++trace_slot;
-        // every lane holds all sums of the tile; lane r takes those of unit r, so that the units finish side by side in one
-        // pass over one copy of the epilogue code
-        const bool paired = kind == PH_QKV || kind == PH_SWIGLU;
-        constexpr int NU = NR >= 2 ? NR / 2 : 1;
-        float lo = y[0], hi = NR >= 2 ? y[NU] : 0.f;
-#pragma unroll
-        for (int r = 1; r < NR; ++r) {
-            if (lane == r) {
-                lo = y[r];
-                if (r < NU) hi = y[r + NU];
+        for (int i = 0; i < MK_TILE_ROWS / 2; ++i) {
+            if (i < n / 2) {
+                const float send = up ? a[i] : a[i + n / 2];
+                const float keep = up ? a[i + n / 2] : a[i];
+                a[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
             }
         }
-        if (split) {
-            if (lane < NR) s_partial[j * NR + lane] = lo;
-        } else {
-            const int u = (it0 + j) * rw + lane;
-            const int cnt = paired ? NU : NR;
-            if ((NR >= 2 || !paired) && lane < cnt && u < units_total) apply_epilogue(p, P, cx, u, lo * cx.rscale, hi * cx.rscale);
-        }
     }
+    return a[0] + __shfl_xor_sync(0xffffffffu, a[0], 1);
+}
+
+// ---- the consumer side of the weight stream --------------------------------------------------------------------
+struct WarpStream {
+    const uint2 *list;          // next tile of this warp (layer list or output-layer list)
+    unsigned char *ring;        // this warp's slots
+    unsigned long long *full_bar, *empty_bar;   // [slots]
+    int slot;
+    unsigned round;
+    unsigned consumed;          // tiles taken so far
+};
+
+// This warp's `n` tiles of operator P: wait, multiply, release; reduce and finish rows where the schedule says so.
+__device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkOp &P, int n, WarpStream &ws, const float4 *xsA, const float4 *xsB,
+                                              volatile int *abort_flag, ItemCtx &cx, float *s_partial, int lane) {
+    float acc[MK_TILE_ROWS];   // 16 independent chains: enough to cover the FMA latency
+    const bool paired = P.kind == PH_QKV || P.kind == PH_SWIGLU;
+    const int hoff = paired ? p.hi_off : 8 * MK_TILE_COLS * 2;   // accumulator rows 8.. of an unpaired tile simply follow rows 0..7
+    uint2 d = n > 0 ? __ldg(ws.list) : make_uint2(0u, 0u);
+    for (int t = 0; t < n; ++t) {
+        const uint2 dn = t + 1 < n ? __ldg(ws.list + t + 1) : make_uint2(0u, 0u);
+        if (d.x & MKT_FIRST) {
+#pragma unroll
+            for (int r = 0; r < MK_TILE_ROWS; ++r) acc[r] = 0.f;
+        }
+        const int m = static_cast<int>(d.y & 31u), kcol = static_cast<int>((d.x >> 20) & 0xffu);
+        const float4 xa = xsA[kcol * 32 + lane], xb = xsB[kcol * 32 + lane];
+        if (!mbar_wait(&ws.full_bar[ws.slot], ws.round & 1u, abort_flag, p.spin_limit)) return false;
+        const unsigned char *tile = ws.ring + static_cast<size_t>(ws.slot) * p.slot_bytes + lane * 16;
+        auto row = [&](int r) {
+            const uint4 w = *reinterpret_cast<const uint4 *>(tile + (r < 8 ? r * (MK_TILE_COLS * 2) : hoff + (r - 8) * (MK_TILE_COLS * 2)));
+            acc[r] = dot8(w, xa, xb, acc[r]);
+        };
+        if (paired ? m == 8 : m == MK_TILE_ROWS) {
+#pragma unroll
+            for (int r = 0; r < MK_TILE_ROWS; ++r) row(r);
+        } else {
+            // rows the tile does not have hold stale bytes: skip them (their sums are never used, but need not be computed)
+            const unsigned mask = paired ? ((1u << m) - 1u) * 0x101u : (1u << m) - 1u;
+#pragma unroll
+            for (int r = 0; r < MK_TILE_ROWS; ++r)
+                if (mask >> r & 1u) row(r);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ws.empty_bar[ws.slot]);   // the slot may be refilled
+        if (++ws.slot == p.slots) { ws.slot = 0; ++ws.round; }
+        ++ws.consumed;
+        if (d.x & MKT_FLUSH) {
+            const float v = reduce_rows(acc, lane);        // lanes 2r, 2r+1: row r (the accumulators start over with the next FIRST tile)
+            const int j = lane >> 1;
+            if (d.y & MKT_DIRECT) {
+                const float hi = __shfl_down_sync(0xffffffffu, v, 16);   // partner row 8 + j of unit j
+                const int v0 = static_cast<int>((d.y >> 5) & 15u);
+                const int u = static_cast<int>(d.x & 0xfffffu) + j;
+                if (!(lane & 1) && j < m && j >= v0 && (!paired || lane < 16)) apply_epilogue(p, P, cx, u, v * cx.rscale, hi * cx.rscale);
+            } else {
+                const int slot = static_cast<int>((d.y >> 10) & 1023u);
+                if (slot >= MK_PARTIAL_SLOTS) return diag_fail(p, abort_flag, 2, slot, 0);
+                if (!(lane & 1)) s_partial[slot * MK_TILE_ROWS + j] = v;
+            }
+        }
+        d = dn;
+    }
+    ws.list += n;
     return true;
 }
 
@@ -475,16 +392,21 @@ __device__ __forceinline__ void att_chunking(const MkParams &p, int n, int hg, i
 }
 
 // One weight-streaming operator: prologue (stage the activation vector, RMSNorm folded in: x*w is staged
-// and the scalar rsqrt(mean x^2 + eps) is applied to the dot products), then this warp's tiles.
+// and the scalar rsqrt(mean x^2 + eps) is applied to the dot products), then this warp's tiles, then the units
+// whose columns were shared between warps.
 // merge_attn > 0: the input is the attention output, still split into merge_attn chunk partials per head
 // (m, l, unnormalised o); the exact log-sum-exp merge is done here, in chunk order, by every CTA.
-__device__ __forceinline__ bool gemv_phase(const MkParams &p, const MkPhase *s_ph, const int2 *s_rng, int ph, WarpStream &ws, float4 *xsA,
-                                           float4 *xsB, volatile int *abort_flag, float *s_part, float *s_partial, ItemCtx &cx, int token,
-                                           int merge_attn, int tid, int &prof_idx, unsigned long long *x_bar, unsigned &x_parity) {
-    const MkPhase &P = s_ph[ph];
+__device__ __forceinline__ bool gemv_phase(const MkParams &p, const MkOp *s_ops, const int *s_tab, int ph, int op_in_layer, WarpStream &ws,
+                                           float4 *xsA, float4 *xsB, volatile int *abort_flag, float *s_part, float *s_partial, ItemCtx &cx,
+                                           int token, int merge_attn, int tid, int &prof_idx, unsigned long long *x_bar, unsigned &x_parity) {
+    const MkOp &P = s_ops[ph];
     const int lane = tid & 31, warp = tid >> 5;
     const int cta = blockIdx.x;
     const int n4 = P.K >> 2;
+    {   // columns past K of the last 256-column piece multiply zero-filled weights: keep the activations there finite (zero)
+        const int pc0 = P.K >> 3, pc1 = ((P.K + MK_TILE_COLS - 1) / MK_TILE_COLS) * (MK_TILE_COLS / 8);
+        for (int pc = pc0 + tid; pc < pc1; pc += MK_NT) { xsA[pc] = make_float4(0.f, 0.f, 0.f, 0.f); xsB[pc] = make_float4(0.f, 0.f, 0.f, 0.f); }
+    }
     float ss = 0.f;
     if (merge_attn > 0) {
         const int nch = merge_attn;
@@ -530,8 +452,11 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, const MkPhase *s_p
     } else if (P.flags & PHF_X_BULK) {
         // the vector is already in the split layout and needs no transform: two bulk copies, every thread waits for them
         // (the CTA-wide sync of the grid barrier ordered all earlier reads of the buffer before this point)
+        // The vector was written by other CTAs of this launch with ordinary stores and acquired at the grid barrier;
+        // the bulk copy reads it through the asynchronous proxy, so a full proxy fence comes first (it also orders
+        // this CTA's earlier reads of the buffer before the copy's writes).
         if (tid == 0) {
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            asm volatile("fence.proxy.async;" ::: "memory");
             const unsigned half_bytes = static_cast<unsigned>(P.K) * 2u;
             mbar_arrive_expect_tx(x_bar, 2u * half_bytes);
             bulk_copy_g2s_plain(xsA, P.x_src, half_bytes, x_bar);
@@ -586,50 +511,30 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, const MkPhase *s_p
         for (int w = 0; w < MK_NW; ++w) tot += s_part[w];
         cx.rscale = rsqrtf(tot / static_cast<float>(P.K) + p.eps);
     }
-    MK_TRACE(p, ph, warp, lane, 0);
-    const int2 rng = s_rng[ph];
-    const int n_items = rng.y - rng.x;
-    const int n_tiles = n_items << P.s_shift;
-    const bool paired = P.kind == PH_QKV || P.kind == PH_SWIGLU;
-    // split operators: thread u finishes unit u after the tiles; fetch what its epilogue adds (old residual
-    // value, bias) now, so that the load latency overlaps the arithmetic
-    float pre_lo = 0.f, pre_hi = 0.f;
-    if (P.split && tid < n_items) {
-        const int u = rng.x + tid;
-        if (P.kind == PH_RESID) {
-            pre_lo = __ldcg(P.out + u);
-        } else if (P.kind == PH_QKV && P.bias) {
-            const int half = p.d >> 1;
-            const int row_lo = (u >> p.half_shift) * p.d + (u & (half - 1));
-            pre_lo = bf16_bits_to_f32(P.bias[row_lo]);
-            pre_hi = bf16_bits_to_f32(P.bias[row_lo + half]);
-        }
-    }
-    const int nr = paired ? 2 * P.rw : P.rw;
-    bool ok;
-    switch (nr) {
-        case 1: ok = consume_tiles<1>(p, s_ph, s_rng, P, rng.x, n_tiles, ws, xsA, xsB, abort_flag, cx, s_partial, warp, lane, ph); break;
-        case 2: ok = consume_tiles<2>(p, s_ph, s_rng, P, rng.x, n_tiles, ws, xsA, xsB, abort_flag, cx, s_partial, warp, lane, ph); break;
-        case 4: ok = consume_tiles<4>(p, s_ph, s_rng, P, rng.x, n_tiles, ws, xsA, xsB, abort_flag, cx, s_partial, warp, lane, ph); break;
-        default: ok = consume_tiles<8>(p, s_ph, s_rng, P, rng.x, n_tiles, ws, xsA, xsB, abort_flag, cx, s_partial, warp, lane, ph); break;
-    }
-    MK_TRACE(p, ph, warp, lane, 12);
-    if (P.split) {
-        // partial sums of the K slices meet here; thread u finishes unit u of this CTA (rw == 1), slices in order
+    const int *tab = s_tab + warp * MK_WARP_TAB;
+    const int n_tiles = op_in_layer < 4 ? tab[1 + op_in_layer] : tab[6];
+    bool ok = consume_tiles(p, P, n_tiles, ws, xsA, xsB, abort_flag, cx, s_partial, lane);
+    // units whose columns were shared between warps: their partial sums meet here, slots in order
+    const int *ctab = s_tab + MK_NW * MK_WARP_TAB + 2 * op_in_layer;
+    const int n_comb = ctab[1];
+    if (n_comb > 0) {
         cta_sync();
-        MK_TRACE(p, ph, warp, lane, 13);
-        if (!*abort_flag) {
-            for (int u = tid; u < n_items; u += MK_NT) {
+        if (ok && !*abort_flag) {
+            const MkCombine *cb = p.combines + ctab[0];
+            const bool paired = P.kind == PH_QKV || P.kind == PH_SWIGLU;
+            for (int idx = tid; idx < n_comb * MK_TILE_ROWS; idx += MK_NT) {
+                const MkCombine e = __ldg(cb + (idx >> 4));
+                const int j = idx & 15, m = static_cast<int>(e.y & 0xffu), v0 = static_cast<int>(e.y >> 8);
+                if (j >= m || j < v0 || (paired && j >= 8)) continue;
                 float lo = 0.f, hi = 0.f;
-                for (int sl = 0; sl < P.ksplit; ++sl) {
-                    const int j = (u << P.s_shift) + sl;
-                    if (paired) { lo += s_partial[2 * j]; hi += s_partial[2 * j + 1]; } else { lo += s_partial[j]; }
+                for (unsigned s = 0; s < e.w; ++s) {
+                    const float *sp = s_partial + (e.z + s) * MK_TILE_ROWS;
+                    lo += sp[j];
+                    if (paired) hi += sp[8 + j];
                 }
-                const bool pre = u == tid;   // operands fetched ahead (first MK_NT units)
-                apply_epilogue(p, P, cx, rng.x + u, lo * cx.rscale, hi * cx.rscale, pre, pre_lo, pre_hi);
+                apply_epilogue(p, P, cx, static_cast<int>(e.x) + j, lo * cx.rscale, hi * cx.rscale);
             }
         }
-        MK_TRACE(p, ph, warp, lane, 14);
     }
     return ok;
 }
@@ -877,68 +782,73 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
 
 // ---- the kernel -----------------------------------------------------------------------------------------------
 // LONG = false: contexts that always run attention with one query head per CTA group (max_context <=
-// att_split_max_n); the grouped variant is then not compiled in, which keeps the register footprint of the
-// streaming state small.
+// att_split_max_n); the grouped variant is then not compiled in, which keeps the register footprint small.
 template <int D, int G, bool LONG>
-__global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) {
-    extern __shared__ __align__(128) unsigned char mk_smem[];
+__global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParams p) {
+    extern __shared__ __align__(1024) unsigned char mk_smem[];
     unsigned char *smem = mk_smem;
     float4 *xsA = reinterpret_cast<float4 *>(smem);
     float4 *xsB = reinterpret_cast<float4 *>(smem + p.xbuf_bytes / 2);
-    MkPhase *s_ph = reinterpret_cast<MkPhase *>(smem + p.xbuf_bytes);          // the step's schedule
-    int2 *s_rng = reinterpret_cast<int2 *>(s_ph + p.nph);                      // this CTA's item range per operator
-    unsigned char *ring = smem + p.xbuf_bytes + p.sched_bytes;
-    __shared__ __align__(8) unsigned long long full_bar[MK_NW * MK_MAXF];
+    MkOp *s_ops = reinterpret_cast<MkOp *>(smem + p.xbuf_bytes);                       // the step's operators
+    int *s_tab = reinterpret_cast<int *>(smem + p.xbuf_bytes + p.ops_bytes);           // this CTA's schedule table
+    unsigned char *ring = smem + p.xbuf_bytes + p.ops_bytes + p.tab_bytes;             // [MK_NW][slots][slot_bytes]
+    __shared__ __align__(8) unsigned long long full_bar[MK_NW * MK_MAX_SLOTS];
+    __shared__ __align__(8) unsigned long long empty_bar[MK_NW * MK_MAX_SLOTS];
     __shared__ __align__(8) unsigned long long x_bar;   // completion of bulk-copied activation vectors
     __shared__ float s_rope[128];
     __shared__ float s_part[MK_NW];
-    __shared__ float s_partial[MK_PARTIAL_FLOATS];
+    __shared__ __align__(16) float s_partial[MK_PARTIAL_FLOATS];
     __shared__ float s_bv[MK_NW];
     __shared__ int s_bi[MK_NW];
     __shared__ int s_flag;
     __shared__ int s_abort;
-    __shared__ int s_released;
+    __shared__ unsigned s_issued[MK_NW];   // tiles fetched so far per consumer warp (written by the feeding lanes)
+    __shared__ int s_feed_done;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int cta = blockIdx.x, ncta = gridDim.x;
     if (tid == 0) {
-        for (int i = 0; i < MK_NW * MK_MAXF; ++i) mbar_init(&full_bar[i], 1);
+        for (int i = 0; i < MK_NW * MK_MAX_SLOTS; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], 1); }
         mbar_init(&x_bar, 1);
         s_abort = 0;
+        s_feed_done = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (tid < MK_NW) s_issued[tid] = 0u;
     {
-        const int n16 = p.nph * static_cast<int>(sizeof(MkPhase) / 16);
-        const uint4 *src = reinterpret_cast<const uint4 *>(p.phases);
-        uint4 *dst = reinterpret_cast<uint4 *>(s_ph);
-        for (int i = tid; i < n16; i += MK_NT) dst[i] = src[i];
-        for (int i = tid; i < p.nph; i += MK_NT) {
-            int it0, it1;
-            item_range(p.phases[i].items_total, cta, ncta, it0, it1);
-            s_rng[i] = make_int2(it0, it1);
-        }
+        const int n16 = p.nph * static_cast<int>(sizeof(MkOp) / 16);
+        const uint4 *src = reinterpret_cast<const uint4 *>(p.ops);
+        uint4 *dst = reinterpret_cast<uint4 *>(s_ops);
+        for (int i = tid; i < n16; i += MK_THREADS) dst[i] = src[i];
+        const int *tsrc = p.cta_tab + static_cast<size_t>(cta) * p.cta_tab_ints;
+        for (int i = tid; i < p.cta_tab_ints; i += MK_THREADS) s_tab[i] = tsrc[i];
     }
-    __syncthreads();
+    __syncthreads();   // the only CTA-wide sync: from here on the feeding warp and the consumers go separate ways
     volatile int *abort_flag = &s_abort;
+
+    if (warp == MK_NW) {
+        feed_rings(p, s_ops, s_tab, ring, full_bar, empty_bar, abort_flag, s_issued, lane);
+        __syncwarp();
+        if (lane == 0) { __threadfence_block(); s_feed_done = 1; }
+        return;
+    }
 
     // The small per-layer vectors (norm weights, biases) are read on the critical path right after a grid barrier;
     // ask L2 for all of them now (they stay: the weight stream is evict-first).
     for (int i = cta * MK_NT + tid; i < p.nph * 64; i += ncta * MK_NT) {
-        const MkPhase &P = s_ph[i >> 6];
+        const MkOp &P = s_ops[i >> 6];
         const int line = i & 63;   // 128-byte line of the vector
         if (P.norm_w && line * 64 < P.K) asm volatile("prefetch.global.L2 [%0];" ::"l"(P.norm_w + line * 64));
         if (P.bias && P.kind == PH_QKV && line * 64 < 2 * P.units_total) asm volatile("prefetch.global.L2 [%0];" ::"l"(P.bias + line * 64));
     }
 
-    // ---- start this warp's weight stream: fill its ring, then run the L2 prefetch ahead ---------------
     WarpStream ws;
-    ws.consumed = 0; ws.issued = 0; ws.head = 0; ws.tail = 0; ws.wrapped = false; ws.fifo = 0;
-    ws.ring = ring + static_cast<size_t>(warp) * p.ring_bytes;
-    ws.bars = &full_bar[warp * MK_MAXF];
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(ws.policy));
-    ws.pf.ph = 0;
-    cursor_enter_phase(ws.pf, p, s_ph, s_rng, warp);
-    bool ok = refill(p, s_ph, s_rng, ws, abort_flag, warp, lane);
+    ws.ring = ring + static_cast<size_t>(warp) * p.slots * p.slot_bytes;
+    ws.full_bar = &full_bar[warp * MK_MAX_SLOTS];
+    ws.empty_bar = &empty_bar[warp * MK_MAX_SLOTS];
+    ws.slot = 0; ws.round = 0; ws.consumed = 0;
+    ws.list = p.tiles + s_tab[warp * MK_WARP_TAB];
+    bool ok = true;
     const int rt = p.req->token, rp = p.req->position;
     const int token = rt >= 0 ? rt : p.state->next_token;
     const int pos = rp >= 0 ? rp : p.state->next_position;
@@ -955,17 +865,17 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
         s_rope[half + tid] = static_cast<float>(sn);
     }
     if (ok && cta == 0 && tid == 0) { p.state->token = token; p.state->position = pos; }
-    // (s_rope is published by the __syncthreads of the first prologue)
+    // (s_rope is published by the sync of the first prologue)
 
     ItemCtx cx;
     cx.rscale = 1.f; cx.slot_row = slot_row; cx.rope = s_rope; cx.best_v = -INFINITY; cx.best_i = 0x7fffffff;
     cx.logits_out = p.req->logits_out;
 
     unsigned bar_no = 0;
+    const unsigned bar_arrivals = static_cast<unsigned>(ncta + p.barrier_extra);
     unsigned x_parity = 0;
     int prof_idx = 0;
     prof_stamp(p, tid, prof_idx);
-    auto top_up = [&]() { __syncwarp(); if (ok && !*abort_flag) refill(p, s_ph, s_rng, ws, abort_flag, warp, lane); };
     const int n_att = slot_row + 1;
     const bool att_split = !LONG || (n_att <= p.att_split_max_n && static_cast<long long>(p.nq) * MK_ATT_SPLIT_MAXC * 2 <= MK_PARTIAL_FLOATS);
     int merge_chunks = 0;   // chunks per head the O-projection prologue has to merge (split mode)
@@ -977,6 +887,8 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
     for (int ph = 0; ph < p.nph && ok; ++ph) {
         const bool layer_op = ph < n_layer_ops;
         const bool after_attention = layer_op && (ph & 3) == 1;
+        if (layer_op && (ph & 3) == 0) ws.list = p.tiles + s_tab[warp * MK_WARP_TAB];          // every layer walks the same list
+        if (!layer_op) ws.list = p.tiles + s_tab[warp * MK_WARP_TAB + 5];
         if (after_attention) {
             const int l = ph >> 2;
             if constexpr (LONG) {
@@ -985,23 +897,27 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
             } else {
                 attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, smem, tid, &s_flag);
             }
-            ok = grid_barrier(p, ++bar_no * ncta, abort_flag, &s_released, tid, prof_idx, top_up) && ok;
+            ok = grid_barrier(p, ++bar_no * bar_arrivals, abort_flag, tid, prof_idx) && ok;
             if (!ok) break;
         }
-        ok = gemv_phase(p, s_ph, s_rng, ph, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token, after_attention ? merge_chunks : 0, tid,
-                        prof_idx, &x_bar, x_parity);
-        if (layer_op) ok = grid_barrier(p, ++bar_no * ncta, abort_flag, &s_released, tid, prof_idx, top_up) && ok;
+        ok = gemv_phase(p, s_ops, s_tab, ph, layer_op ? (ph & 3) : 4, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token,
+                        after_attention ? merge_chunks : 0, tid, prof_idx, &x_bar, x_parity);
+        if (layer_op) ok = grid_barrier(p, ++bar_no * bar_arrivals, abort_flag, tid, prof_idx) && ok;
     }
     prof_stamp(p, tid, prof_idx);
     if (!ok || *abort_flag) {
-        // aborted: wait (bounded) for the copies this warp still has in flight, then leave
+        // aborted: once the feeding warp has stopped, wait (bounded) for the copies still in flight into this warp's ring
+        *abort_flag = 1;
         if (tid == 0 && p.state->status == 0) p.state->status = 6;
-        for (unsigned k = ws.consumed; k < ws.issued; ++k) {
-            const unsigned q = k & (MK_MAXF - 1);
-            const unsigned par = (k / MK_MAXF) & 1u;
-            const unsigned long long t0 = global_ns();
-            while (!mbar_try_wait(&ws.bars[q], par))
-                if (global_ns() - t0 > p.spin_limit) break;
+        const unsigned long long t0 = global_ns();
+        while (!*reinterpret_cast<volatile int *>(&s_feed_done))
+            if (global_ns() - t0 > p.spin_limit) break;
+        const unsigned issued = *reinterpret_cast<volatile unsigned *>(&s_issued[warp]);
+        for (unsigned k = ws.consumed; k < issued; ++k) {
+            const unsigned long long t1 = global_ns();
+            while (!mbar_try_wait(&ws.full_bar[ws.slot], ws.round & 1u))
+                if (global_ns() - t1 > p.spin_limit) break;
+            if (++ws.slot == p.slots) { ws.slot = 0; ++ws.round; }
         }
         return;
     }
@@ -1043,7 +959,7 @@ __global__ void __launch_bounds__(MK_NT, 1) decode_megakernel(const MkParams p) 
         }
         if (lane == 0) {
             if (bi == 0x7fffffff) bi = 0;
-            if (s_ph[p.nph - 1].flags & PHF_REMAP) bi = p.vocab_ids[bi];   // pruned vocabulary: row index -> token id
+            if (s_ops[p.nph - 1].flags & PHF_REMAP) bi = p.vocab_ids[bi];   // pruned vocabulary: row index -> token id
             int *nto = p.req->next_token_out;
             if (nto) *nto = bi;
             p.state->next_token = bi;

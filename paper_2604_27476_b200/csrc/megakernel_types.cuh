@@ -4,56 +4,77 @@
 
 namespace edgefm {
 
-constexpr int MK_MAXF = 4;                       // tiles in flight per warp (one mbarrier each)
 constexpr int MK_BAR_POLLERS = 1;                // warps whose lane 0 polls the grid barrier counter
 constexpr int MK_ATT_LPP = 2;                    // lanes per cached position in the score phase (one CTA per GQA group)
 constexpr int MK_ATT_LPP_SPLIT = 2;              // ... when every query head has its own CTAs (16 positions per warp iteration)
 constexpr int MK_ATT_TILE = 32 / MK_ATT_LPP;     // positions per warp iteration (grouped mode)
 constexpr int MK_ATT_SPLIT_MAXC = 12;            // chunks per head when every query head has its own CTAs
-constexpr int MK_PARTIAL_FLOATS = 2048;          // shared-memory scratch: split-K partial sums / chunk statistics
-// Warps per CTA of the two builds of the kernel: the short-context build favours instruction streams, the
-// long-context build (grouped attention keeps G heads of accumulators per warp) favours registers.
+constexpr int MK_PARTIAL_SLOTS = 48;             // shared-memory scratch: partial row sums, 16 floats per slot
+constexpr int MK_PARTIAL_FLOATS = MK_PARTIAL_SLOTS * 16;   // (also the chunk statistics of the attention merge)
+constexpr int MK_TILE_COLS = 256;                // columns of a weight tile: one 16-byte piece per lane
+constexpr int MK_TILE_ROWS = 16;                 // accumulator rows of a consumer warp (largest tile: 16 x 256 bf16 = 8 KB)
+constexpr int MK_MAX_VARIANTS = 4;               // tensor maps (box heights) per weight matrix
+constexpr int MK_MAX_SLOTS = 4;                  // ring slots per consumer warp
+constexpr int MK_WARP_TAB = 8;                   // ints per warp in the per-CTA table
+// Consumer warps per CTA of the two builds of the kernel (one more warp feeds them): the short-context build favours
+// instruction streams, the long-context build (grouped attention keeps G heads of accumulators per warp) registers.
 #ifndef MK_NW_SHORT_VALUE
-#define MK_NW_SHORT_VALUE 12
+#define MK_NW_SHORT_VALUE 11
 #endif
 #ifndef MK_NW_LONG_VALUE
-#define MK_NW_LONG_VALUE 8
+#define MK_NW_LONG_VALUE 7
 #endif
 constexpr int MK_NW_SHORT = MK_NW_SHORT_VALUE;
 constexpr int MK_NW_LONG = MK_NW_LONG_VALUE;
+constexpr int MK_NW_MAX = MK_NW_SHORT > MK_NW_LONG ? MK_NW_SHORT : MK_NW_LONG;
 
 enum { PH_QKV = 0, PH_RESID = 1, PH_SWIGLU = 2, PH_LMHEAD = 3 };
 
-// One weight-streaming operator of the step.
-// MkPhase::flags
+// MkOp::flags
 enum : int {
     PHF_REMAP = 1,      // PH_LMHEAD: rows are a vocabulary subset; row r stands for token MkParams::vocab_ids[r]
     PHF_OUT_SPLIT = 2,  // PH_SWIGLU: the output vector is stored as [even 16-byte pieces | odd 16-byte pieces]
     PHF_X_BULK = 4,     // the input vector has that layout already and needs no transform: staged by two bulk copies
 };
 
-struct alignas(16) MkPhase {
-    const uint16_t *W;       // bf16 [rows][K]
+// One weight-streaming operator of the step (its weights are reached through tensor maps, see MkParams::maps).
+struct alignas(16) MkOp {
     const uint16_t *bias;    // PH_QKV: bf16 [rows] or null
     const uint16_t *norm_w;  // RMSNorm weight of the prologue (bf16 [K]) or null = plain copy of x_src
     const float *x_src;      // fp32 [K] input vector in global memory; null = embedding row of the token
     float *out;              // PH_QKV: q fp32; PH_RESID: x (+=); PH_SWIGLU: act; PH_LMHEAD: unused
     int K;                   // columns (multiple of 8)
     int kind;
-    int rw;                  // units per work item (rows, or row pairs for PH_QKV / PH_SWIGLU); 1 when split
-    int ksplit;              // K slices per item (tiles per item)
-    int kcs;                 // 16-byte pieces per row slice = K / 8 / ksplit
     int units_total;         // rows (PH_RESID, PH_LMHEAD), pairs (PH_QKV: rows/2, PH_SWIGLU: F)
-    int items_total;         // ceil(units_total / rw)
     int layer;
-    int s_shift;             // log2(ksplit); ksplit is a power of two
-    int split;               // 1: the tiles of an item go to different warps, partial sums meet in shared memory
     int flags;               // PHF_* bits
+    int pad[3];
 };
-static_assert(sizeof(MkPhase) % 16 == 0, "descriptor is copied in 16-byte pieces");
+static_assert(sizeof(MkOp) % 16 == 0, "descriptor is copied in 16-byte pieces");
+
+// ---- the tile schedule ------------------------------------------------------------------------------------------
+// A tile is a box of m rows x 256 columns of one weight matrix (for PH_QKV / PH_SWIGLU: m "low" rows and their m
+// partner rows, two boxes), fetched by one TMA tensor copy per box into a ring slot of the consumer warp that owns it.
+// The host lays out, for every CTA and every consumer warp, the list of tiles of one layer (operators in order) and of
+// the output layer; the lists are the same for every layer.  8 bytes per tile:
+//   x: unit_base [0,20) | column piece [20,28) | tensor-map variant [28,30) | FIRST 30 | FLUSH 31
+//   y: m [0,5) | first valid unit v0 [5,9) | DIRECT 9 | partial slot [10,20) | operator in layer (4 = output layer) [20,23)
+// FIRST: the warp's accumulators start at zero with this tile.  FLUSH: after this tile the 16 row sums are reduced
+// across the lanes; DIRECT: the warp has seen all columns of these rows and finishes them itself; otherwise the sums
+// go to partial slot `slot` and the units are finished after the operator by summing their slots in order.
+constexpr uint32_t MKT_FIRST = 1u << 30, MKT_FLUSH = 1u << 31, MKT_DIRECT = 1u << 9;
+__host__ __device__ inline uint2 mk_tile_desc(uint32_t unit_base, uint32_t kcol, uint32_t variant, bool first, bool flush, uint32_t m,
+                                              uint32_t v0, bool direct, uint32_t slot, uint32_t op) {
+    uint2 d;
+    d.x = (unit_base & 0xfffffu) | (kcol & 0xffu) << 20 | (variant & 3u) << 28 | (first ? MKT_FIRST : 0u) | (flush ? MKT_FLUSH : 0u);
+    d.y = (m & 31u) | (v0 & 15u) << 5 | (direct ? MKT_DIRECT : 0u) | (slot & 1023u) << 10 | (op & 7u) << 20;
+    return d;
+}
+// Units whose row sums were left in partial slots: unit_base, m | v0 << 8, first slot, number of slots.
+using MkCombine = uint4;
 
 struct MkParams {
-    const MkPhase *phases;   // [nph]
+    const MkOp *ops;         // [nph]
     int nph;                 // 4 * n_layers + 1
     int n_layers, H, nq, nkv, d, F, V;
     int half_shift;          // log2(d / 2)
@@ -75,9 +96,19 @@ struct MkParams {
     const int *vocab_ids;          // [V] token id of every row of a pruned lm_head (used when the last operator has PHF_REMAP)
     StepState *state;
     const StepRequest *req;
-    int ring_bytes;                // shared-memory ring of one warp
-    int slot_bytes;                // largest tile (checked against ring_bytes on the host)
-    int xbuf_bytes, sched_bytes;
+    // weight streaming
+    const unsigned char *maps;     // CUtensorMap [(4 * n_layers + 1) * MK_MAX_VARIANTS], 128 bytes each, index (4 l + op) * 4 + variant
+    const uint2 *tiles;            // all tile lists
+    const int *cta_tab;            // [gridDim.x][cta_tab_ints]: per consumer warp {layer list offset, tiles per operator x4, output-layer
+                                   // list offset, output-layer tiles, 0}, then per operator (5) {combine offset, combine count}
+    const MkCombine *combines;
+    int cta_tab_ints;
+    int slots;                     // ring slots per consumer warp
+    int slot_bytes;                // bytes of one slot (a multiple of 1024)
+    int hi_off;                    // offset of the partner box inside a slot
+    int xbuf_bytes, ops_bytes, tab_bytes;
+    int map_fence;                 // tensor maps the host may have rewritten since the last launch: 0 none, 1 the output layer's, 2 all
+    int barrier_extra;             // test hook: arrivals the grid barrier expects beyond the CTAs present (0 in production)
     unsigned spin_limit;           // upper bound of every device-side wait, nanoseconds
     unsigned long long *prof;      // optional timestamps [gridDim.x][prof_stride] (diagnostics), or null
     int prof_stride;

@@ -1,5 +1,5 @@
-"""Secondary launch modes and diagnostics of the library on a GPU: the multi-kernel debug mode, the in-kernel
-timestamps, the status query, and a second context on the same weights."""
+"""Diagnostics of the library on a GPU: the in-kernel timestamps, the status query, and a second context on the
+same weights."""
 import os
 import subprocess
 import sys
@@ -45,11 +45,6 @@ print("LAUNCHES", pair.ctx.launches_per_step, "WORST", worst, "PROF", None if pr
       None if prof is None else bool((np.diff(prof[:, :3 + 14 * cfg.n_layers].astype(np.int64), axis=1) >= 0).all()))
 pair.close()
 '''
-
-
-def test_multi_kernel_debug_mode_matches_oracle():
-    out = _run_child(CHILD, {"EDGEFM_IMPL": "kernels"})
-    assert "LAUNCHES 12 " in out                    # 1 + 5 per layer + 1 kernels for the 2-layer model
 
 
 def test_persistent_kernel_with_timestamps_matches_oracle_and_timestamps_are_ordered():
