@@ -47,7 +47,7 @@ class _Weights(ctypes.Structure):
 
 EXPORTS = ("edgefm_create", "edgefm_prefill_kv", "edgefm_decode_step", "edgefm_destroy", "edgefm_get_length",
            "edgefm_export_kv", "edgefm_get_launches_per_step", "edgefm_last_error", "edgefm_version",
-           "edgefm_sync_status", "edgefm_debug_profile", "edgefm_debug_set_wait_limit", "edgefm_decode_step_static", "edgefm_set_vocab_subset",
+           "edgefm_sync_status", "edgefm_debug_profile", "edgefm_debug_set_wait_limit", "edgefm_debug_plan", "edgefm_debug_plan_operator", "edgefm_decode_step_static", "edgefm_set_vocab_subset",
            "edgefm_append_kv")
 
 
@@ -85,6 +85,10 @@ def load_library():
     L.edgefm_debug_profile.argtypes = [vp, vp, i64, ctypes.POINTER(i32), ctypes.POINTER(i32)]
     L.edgefm_debug_set_wait_limit.restype = ctypes.c_int
     L.edgefm_debug_set_wait_limit.argtypes = [vp, ctypes.c_uint32, i32]
+    L.edgefm_debug_plan.restype = ctypes.c_int
+    L.edgefm_debug_plan.argtypes = [vp, ctypes.POINTER(i32)]
+    L.edgefm_debug_plan_operator.restype = ctypes.c_int
+    L.edgefm_debug_plan_operator.argtypes = [i32] * 8 + [vp, i64, vp, vp, i64, vp, vp, ctypes.POINTER(i64), ctypes.POINTER(i64)]
     L.edgefm_decode_step_static.restype = ctypes.c_int
     L.edgefm_decode_step_static.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Weights), vp, vp, i32, i32, i32, i32, vp, vp, vp]
     L.edgefm_append_kv.restype = ctypes.c_int
@@ -190,6 +194,53 @@ def edgefm_sync_status(ctx, stream=None):
 
 def edgefm_debug_set_wait_limit(ctx, limit_ns, extra_barrier_arrivals=0):
     _check(load_library().edgefm_debug_set_wait_limit(ctx, limit_ns, extra_barrier_arrivals), ctx)
+
+
+def edgefm_debug_plan(ctx) -> dict:
+    """Launch geometry of the context's step kernel."""
+    out = (ctypes.c_int32 * 8)()
+    _check(load_library().edgefm_debug_plan(ctx, out), ctx)
+    keys = ("ctas", "consumer_warps", "ring_slots_per_warp", "slot_bytes", "dynamic_smem_bytes", "max_tiles_per_cta", "schedule_smem_bytes",
+            "long_context_build")
+    return dict(zip(keys, list(out)))
+
+
+def edgefm_debug_plan_operator(kind, units, K, head_half, op_index, n_ctas, n_warps, slot_rows):
+    """Host-only: the tile schedule the planner makes for one operator.  Returns a dict with
+    tiles [cta][warp] -> list of decoded tile dicts, combines [cta] -> list of dicts, variant_rows."""
+    import numpy as np
+    L = load_library()
+    per_warp = np.zeros(n_ctas * n_warps, np.int32)
+    per_cta = np.zeros(n_ctas, np.int32)
+    variants = np.zeros(4, np.int32)
+    nt, nc = ctypes.c_int64(), ctypes.c_int64()
+    args = (kind, units, K, head_half, op_index, n_ctas, n_warps, slot_rows)
+    _check(L.edgefm_debug_plan_operator(*args, None, 0, per_warp.ctypes.data, None, 0, per_cta.ctypes.data, variants.ctypes.data,
+                                        ctypes.byref(nt), ctypes.byref(nc)))
+    tiles = np.zeros(max(nt.value, 1), np.uint64)
+    comb = np.zeros(max(nc.value, 1) * 4, np.uint32)
+    _check(L.edgefm_debug_plan_operator(*args, tiles.ctypes.data, tiles.size, per_warp.ctypes.data, comb.ctypes.data, nc.value, per_cta.ctypes.data,
+                                        variants.ctypes.data, ctypes.byref(nt), ctypes.byref(nc)))
+    out_tiles, pos = [], 0
+    for c in range(n_ctas):
+        row = []
+        for w in range(n_warps):
+            lst = []
+            for _ in range(per_warp[c * n_warps + w]):
+                d = int(tiles[pos]); pos += 1
+                x, y = d & 0xffffffff, d >> 32
+                lst.append(dict(unit_base=x & 0xfffff, kcol=(x >> 20) & 0xff, variant=(x >> 28) & 3, first=bool(x >> 30 & 1), flush=bool(x >> 31 & 1),
+                                m=y & 31, v0=(y >> 5) & 15, direct=bool(y >> 9 & 1), slot=(y >> 10) & 1023, op=(y >> 20) & 7))
+            row.append(lst)
+        out_tiles.append(row)
+    out_comb, pos = [], 0
+    for c in range(n_ctas):
+        lst = []
+        for _ in range(per_cta[c]):
+            e = comb[4 * pos: 4 * pos + 4]; pos += 1
+            lst.append(dict(unit_base=int(e[0]), m=int(e[1]) & 0xff, v0=int(e[1]) >> 8, first_slot=int(e[2]), n_slots=int(e[3])))
+        out_comb.append(lst)
+    return dict(tiles=out_tiles, combines=out_comb, variant_rows=[int(v) for v in variants if v])
 
 
 def edgefm_debug_profile(ctx):

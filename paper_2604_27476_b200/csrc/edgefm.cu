@@ -15,7 +15,7 @@
 #include "megakernel_types.cuh"
 #include "step_plan.h"
 // the persistent kernel is built twice: 11 consumer warps per CTA (short contexts, here) and 7 (long contexts,
-// in the megakernel_long_*.cu translation units), plus the warp that feeds them
+// in the megakernel_long_*.cu translation units), plus the warp that prefetches into L2
 #define MK_NS mk_short
 #define MK_NW_VALUE MK_NW_SHORT
 #include "megakernel.cuh"
@@ -95,13 +95,14 @@ struct StepPlan {
     int grid = 0;          // CTAs (one per SM)
     int max_chunks = 0;    // row stride of the attention partial buffers
     int n_ops = 0;         // 4 per layer + lm_head
-    size_t xbuf = 0, ops_bytes = 0, tab_bytes = 0;   // shared memory: activation / attention scratch, operators, schedule table
-    int slots = 0, slot_bytes = 0, slot_rows = 0, hi_off = 0;   // ring of one consumer warp
+    size_t xbuf = 0, ops_bytes = 0, tab_bytes = 0, sched_bytes = 0;   // shared memory: activation / attention scratch, operators, schedule table, tile lists
+    int slots = 0, slot_bytes = 0, slot_rows = 0;   // ring of one consumer warp
     size_t dyn_smem = 0;
 };
 
 // Kernel variant and shared-memory split for a model shape.  Returns null, or why the shape does not fit.
-inline const char *plan_step(const edgefm_shape &sh, int max_context, int num_sms, int smem_optin, StepPlan *pl, cudaError_t *cuda_err) {
+// sched_reserve: bytes to set aside for the CTA's tile lists.
+inline const char *plan_step(const edgefm_shape &sh, int max_context, int num_sms, int smem_optin, size_t sched_reserve, StepPlan *pl, cudaError_t *cuda_err) {
     const int H = sh.hidden, d = sh.head_dim, nq = sh.n_q_heads, nkv = sh.n_kv_heads, F = sh.ffn, G = nq / nkv;
     *cuda_err = cudaSuccess;
     pl->long_ctx = max_context > 8192 || static_cast<long long>(nq) * MK_ATT_SPLIT_MAXC * 2 > MK_PARTIAL_FLOATS;
@@ -127,22 +128,23 @@ inline const char *plan_step(const edgefm_shape &sh, int max_context, int num_sm
     const size_t static_smem = fa.sharedSizeBytes + 256;   // the kernel's static shared memory (mbarriers, tables, scratch) + margin
     pl->ops_bytes = static_cast<size_t>(pl->n_ops) * sizeof(MkOp);
     const size_t tab = static_cast<size_t>(cta_tab_ints_for(NW)) * sizeof(int);
-    const size_t head = (pl->xbuf + pl->ops_bytes + tab + 1023) / 1024 * 1024;   // the rings start on a 1 KB boundary
-    pl->tab_bytes = head - pl->xbuf - pl->ops_bytes;
-    if (head + static_smem + static_cast<size_t>(NW) * 2 * 2048 > static_cast<size_t>(smem_optin))
+    pl->tab_bytes = (tab + 15) / 16 * 16;
+    const size_t head = (pl->ops_bytes + pl->tab_bytes + sched_reserve + 1023) / 1024 * 1024;   // the rings start on a 1 KB boundary
+    pl->sched_bytes = head - pl->ops_bytes - pl->tab_bytes;
+    // behind the rings: the activation vector; at least one full tile (8 KB) of valid shared memory follows the last slot
+    const size_t tail = std::max(pl->xbuf, static_cast<size_t>(MK_TILE_ROWS) * MK_TILE_COLS * 2);
+    if (head + tail + static_smem + static_cast<size_t>(NW) * 2 * 2048 > static_cast<size_t>(smem_optin))
         return "model shape does not fit the shared-memory plan";
-    const size_t per_warp = (smem_optin - static_smem - head) / NW;
-    // two slots per warp at least; a slot holds up to 16 rows x 256 columns (8 KB) and is a whole number of KB
+    const size_t per_warp = (smem_optin - static_smem - head - tail) / NW;
+    // two slots per warp at least; a slot holds up to 16 rows x 256 columns (8 KB) and is a whole number of KB (an even number of rows)
     size_t slot = per_warp / 2 / 1024 * 1024;
     if (slot > static_cast<size_t>(MK_TILE_ROWS) * MK_TILE_COLS * 2) slot = static_cast<size_t>(MK_TILE_ROWS) * MK_TILE_COLS * 2;
-    slot = slot / 2048 * 2048;   // an even number of rows: the partner box starts in the middle of the slot
     if (slot < 2048) return "model shape does not fit the shared-memory plan";
     pl->slot_bytes = static_cast<int>(slot);
     pl->slot_rows = pl->slot_bytes / (MK_TILE_COLS * 2);
-    pl->hi_off = pl->slot_bytes / 2;
     pl->slots = static_cast<int>(per_warp / slot);
     if (pl->slots > MK_MAX_SLOTS) pl->slots = MK_MAX_SLOTS;
-    pl->dyn_smem = head + static_cast<size_t>(NW) * pl->slots * slot;
+    pl->dyn_smem = head + static_cast<size_t>(NW) * pl->slots * slot + tail;
     return nullptr;
 }
 
@@ -167,25 +169,26 @@ inline void op_shapes(const edgefm_shape &sh, int lm_rows, OpShape os[5]) {
 }
 
 // The operators of the step in execution order, wired to the work buffers.
-inline void fill_ops(const edgefm_shape &sh, const edgefm_layer_weights *layers, const void *final_norm, float *x, float *attn, float *q,
-                     float *act, MkOp *out) {
+inline void fill_ops(const edgefm_shape &sh, const edgefm_layer_weights *layers, const void *final_norm, const void *lm_head, float *x, float *attn, float *q,
+                     float *act, MkOp *out, const uint16_t **weights_out) {
     OpShape os[5];
     op_shapes(sh, sh.vocab, os);
     int n = 0;
-    auto mk = [&](const OpShape &o, const void *bias, const void *norm, const float *x_src, float *dst, int layer, int flags) {
+    auto mk = [&](const OpShape &o, const void *W, const void *bias, const void *norm, const float *x_src, float *dst, int layer, int flags) {
         MkOp op{};
+        weights_out[n] = static_cast<const uint16_t *>(W);
         op.bias = static_cast<const uint16_t *>(bias); op.norm_w = static_cast<const uint16_t *>(norm); op.x_src = x_src; op.out = dst;
-        op.K = o.K; op.kind = o.kind; op.units_total = o.units; op.layer = layer; op.flags = flags;
+        op.K = o.K; op.kind = o.kind; op.units_total = o.units; op.layer_flags = layer << 8 | flags;
         out[n++] = op;
     };
     for (int l = 0; l < sh.n_layers; ++l) {
         const edgefm_layer_weights &w = layers[l];
-        mk(os[0], sh.qkv_bias ? w.bqkv : nullptr, w.input_norm, l == 0 ? nullptr : x, q, l, 0);
-        mk(os[1], nullptr, nullptr, attn, x, l, PHF_X_BULK);        // the attention phase stores its output in the staged layout
-        mk(os[2], nullptr, w.post_norm, x, act, l, PHF_OUT_SPLIT);  // the MLP activations go to memory in the layout the down projection stages
-        mk(os[3], nullptr, nullptr, act, x, l, PHF_X_BULK);
+        mk(os[0], w.wqkv, sh.qkv_bias ? w.bqkv : nullptr, w.input_norm, l == 0 ? nullptr : x, q, l, 0);
+        mk(os[1], w.wo, nullptr, nullptr, attn, x, l, PHF_X_BULK);        // the attention phase stores its output in the staged layout
+        mk(os[2], w.w_gate_up, nullptr, w.post_norm, x, act, l, PHF_OUT_SPLIT);  // the MLP activations go to memory in the layout the down projection stages
+        mk(os[3], w.w_down, nullptr, nullptr, act, x, l, PHF_X_BULK);
     }
-    mk(os[4], nullptr, final_norm, x, nullptr, sh.n_layers, 0);
+    mk(os[4], lm_head, nullptr, final_norm, x, nullptr, sh.n_layers, 0);
 }
 
 // Tile schedule of the step for the plan's geometry.  Returns null, or why the shape does not fit.
@@ -198,6 +201,21 @@ inline const char *plan_schedule(const StepPlan &pl, const edgefm_shape &sh, int
     return nullptr;
 }
 
+// Shared-memory plan and tile schedule together: the tile lists live in shared memory, so their size (known only once
+// the schedule exists) takes room from the rings, whose slot size shapes the schedule.  A few rounds settle it.
+inline const char *plan_step_and_schedule(const edgefm_shape &sh, int max_context, int num_sms, int smem_optin, StepPlan *pl, StepSchedule *ss,
+                                          cudaError_t *cuda_err) {
+    size_t reserve = 0;
+    for (int attempt = 0; attempt < 6; ++attempt) {
+        if (const char *why = plan_step(sh, max_context, num_sms, smem_optin, reserve, pl, cuda_err)) return why;
+        if (const char *why = plan_schedule(*pl, sh, sh.vocab, ss)) return why;
+        const size_t need = static_cast<size_t>(ss->max_cta_tiles) * sizeof(uint2);
+        if (need <= pl->sched_bytes) return nullptr;
+        reserve = need + (attempt > 0 ? need / 8 : 0);
+    }
+    return "model shape does not fit the shared-memory plan";
+}
+
 // Tensor maps of all weight matrices: [(4 l + op) * MK_MAX_VARIANTS + variant]; the output layer's come last.
 inline const char *encode_maps(const StepSchedule &ss, const edgefm_shape &sh, const edgefm_layer_weights *layers, const void *lm_head, int lm_rows,
                                CUtensorMap *maps) {
@@ -207,7 +225,8 @@ inline const char *encode_maps(const StepSchedule &ss, const edgefm_shape &sh, c
         for (int v = 0; v < MK_MAX_VARIANTS; ++v) {
             CUtensorMap *m = &maps[static_cast<size_t>(opi) * MK_MAX_VARIANTS + v];
             if (v >= ss.ops[o].n_variants) { std::memset(m, 0, sizeof *m); continue; }
-            if (!encode_weight_map(m, W, os[o].rows, os[o].K, ss.ops[o].variant_rows[v])) return false;
+            const int pair_rows = os[o].kind == PH_QKV ? os[o].head_half : (os[o].kind == PH_SWIGLU ? os[o].units : 0);
+            if (!encode_weight_map(m, W, os[o].rows, os[o].K, ss.ops[o].variant_rows[v], pair_rows, os[o].kind == PH_QKV)) return false;
         }
         return true;
     };
@@ -228,10 +247,12 @@ inline void fill_shape_params(MkParams *m, const edgefm_shape &sh, int max_conte
     m->eps = sh.rms_eps; m->scale = static_cast<float>(1.0 / std::sqrt(static_cast<double>(sh.head_dim)));
     m->max_context = max_context; m->max_chunks = pl.max_chunks;
     m->att_chunk_shared = 256; m->att_chunk_split = 64; m->att_split_max_n = 8192;
-    m->slots = pl.slots; m->slot_bytes = pl.slot_bytes; m->hi_off = pl.hi_off;
+    m->slots = pl.slots; m->slot_bytes = pl.slot_bytes;
     m->xbuf_bytes = static_cast<int>(pl.xbuf); m->ops_bytes = static_cast<int>(pl.ops_bytes); m->tab_bytes = static_cast<int>(pl.tab_bytes);
+    m->sched_bytes = static_cast<int>(pl.sched_bytes);
     m->cta_tab_ints = ss.cta_tab_ints;
     m->barrier_extra = 0;
+    m->pf_tiles = 4;   // measured: 3 .. 8 equal, 16 thrashes L2 (1.5B shape)
     m->map_fence = 1;   // edgefm_set_vocab_subset rewrites the output layer's maps between steps
     m->spin_limit = 1000000000u;   // 1 s
 }
@@ -264,6 +285,7 @@ struct edgefm_ctx {
     StepState *state = nullptr;
     StepRequest *req = nullptr;
     MkOp *d_ops = nullptr;
+    const uint16_t **d_op_w = nullptr;   // base of every operator's weight matrix
     unsigned char *d_maps = nullptr;   // CUtensorMap [(4 L + 1) * MK_MAX_VARIANTS]
     uint2 *d_tiles = nullptr;
     int *d_cta_tab = nullptr;
@@ -339,7 +361,7 @@ void free_all(edgefm_ctx *c) {
     if (c->graph) cudaGraphDestroy(c->graph);
     if (c->build_stream) cudaStreamDestroy(c->build_stream);
     void *bufs[] = {c->k_cache, c->v_cache, c->x, c->q, c->attn, c->act, c->inv_freq, c->part_m, c->part_l,
-                    c->part_o, c->lm_part_val, c->lm_part_idx, c->tickets, c->state, c->req, c->d_ops, c->d_maps, c->d_tiles,
+                    c->part_o, c->lm_part_val, c->lm_part_idx, c->tickets, c->state, c->req, c->d_ops, c->d_op_w, c->d_maps, c->d_tiles,
                     c->d_cta_tab, c->d_combines, c->grid_bar, c->prof, c->vocab_ids, c->sub_lm};
     for (void *b : bufs) if (b) cudaFree(b);
 }
@@ -454,10 +476,9 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
     if (!coop) return bail(EDGEFM_ERR_CUDA, "device lacks cooperative launch", cudaErrorNotSupported);
     {
         cudaError_t ce = cudaSuccess;
-        if (const char *why = plan_step(sh, max_context, c->num_sms, smem_optin, &pl, &ce))
+        if (const char *why = plan_step_and_schedule(sh, max_context, c->num_sms, smem_optin, &pl, &c->sched_full, &ce))
             return bail(ce != cudaSuccess ? EDGEFM_ERR_CUDA : EDGEFM_ERR_BAD_SHAPE, why, ce != cudaSuccess ? ce : cudaErrorInvalidValue);
     }
-    if (const char *why = plan_schedule(pl, sh, sh.vocab, &c->sched_full)) return bail(EDGEFM_ERR_BAD_SHAPE, why, cudaErrorInvalidValue);
     const StepSchedule &ss = c->sched_full;
 
     const size_t kv_elems = static_cast<size_t>(sh.n_layers) * nkv * max_context * d;
@@ -491,7 +512,8 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
     // the operators of the step wired to the work buffers, the tile schedule and the tensor maps of the weights
     {
         std::vector<MkOp> ops(static_cast<size_t>(pl.n_ops));
-        fill_ops(sh, c->layers.data(), c->final_norm, c->x, c->attn, c->q, c->act, ops.data());
+        std::vector<const uint16_t *> op_w(static_cast<size_t>(pl.n_ops));
+        fill_ops(sh, c->layers.data(), c->final_norm, c->lm_head, c->x, c->attn, c->q, c->act, ops.data(), op_w.data());
         c->lm_op_full = ops.back();
         std::vector<CUtensorMap> maps(static_cast<size_t>(pl.n_ops) * MK_MAX_VARIANTS);
         if (const char *why = encode_maps(ss, sh, c->layers.data(), c->lm_head, sh.vocab, maps.data()))
@@ -501,6 +523,8 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
         c->combines_cap = static_cast<size_t>(pl.grid) * 5 * (2 * pl.nw + 4);
         if (ss.combines.size() > c->combines_cap) c->combines_cap = ss.combines.size();
         CREATE_TRY(dev_alloc(&c->d_ops, ops.size()));
+        CREATE_TRY(dev_alloc(&c->d_op_w, op_w.size()));
+        CREATE_TRY(cudaMemcpy(c->d_op_w, op_w.data(), op_w.size() * sizeof(op_w[0]), cudaMemcpyHostToDevice));
         CREATE_TRY(cudaMalloc(reinterpret_cast<void **>(&c->d_maps), maps.size() * sizeof(CUtensorMap)));
         CREATE_TRY(dev_alloc(&c->d_tiles, c->tiles_cap));
         CREATE_TRY(dev_alloc(&c->d_cta_tab, ss.cta_tab.size()));
@@ -522,7 +546,7 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
     CREATE_TRY(cudaMemset(c->vocab_ids, 0, static_cast<size_t>(sh.vocab) * sizeof(int)));
     MkParams &m = c->mk;
     fill_shape_params(&m, sh, max_context, pl, ss);
-    m.ops = c->d_ops; m.maps = c->d_maps; m.tiles = c->d_tiles; m.cta_tab = c->d_cta_tab; m.combines = c->d_combines;
+    m.ops = c->d_ops; m.op_weights = c->d_op_w; m.maps = c->d_maps; m.tiles = c->d_tiles; m.cta_tab = c->d_cta_tab; m.combines = c->d_combines;
     m.vocab_ids = c->vocab_ids;
     m.k_cache = c->k_cache; m.v_cache = c->v_cache; m.embed = (const uint16_t *)c->embed;
     m.inv_freq = c->inv_freq; m.x = c->x; m.q = c->q; m.attn = c->attn; m.part_m = c->part_m; m.part_l = c->part_l;
@@ -531,8 +555,9 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
     const char *pe_ = getenv("EDGEFM_PROFILE");
     if (pe_ && pe_[0] == '1') {
         c->prof_stride = 3 + 14 * sh.n_layers;
-        CREATE_TRY(dev_alloc(&c->prof, static_cast<size_t>(pl.grid) * c->prof_stride));
-        CREATE_TRY(cudaMemset(c->prof, 0, static_cast<size_t>(pl.grid) * c->prof_stride * 8));
+        const size_t n_prof = static_cast<size_t>(pl.grid) * c->prof_stride + MK_NW_MAX * 16 * 4 + 8;   // + the optional per-warp trace
+        CREATE_TRY(dev_alloc(&c->prof, n_prof));
+        CREATE_TRY(cudaMemset(c->prof, 0, n_prof * 8));
         m.prof = c->prof; m.prof_stride = c->prof_stride;
     }
 
@@ -655,7 +680,8 @@ edgefm_status edgefm_set_vocab_subset(edgefm_ctx *ctx, const int32_t *token_ids,
         if (const char *why = plan_op(os[4], 4, pl.grid, pl.nw, pl.slot_rows, &sub.ops[4]))
             return fail(ctx, EDGEFM_ERR_BAD_SHAPE, "a subset of %d rows does not fit the tile plan of this context: %s", n, why);
         assemble_schedule(&sub, pl.grid, pl.nw);
-        if (sub.tiles.size() > ctx->tiles_cap || sub.combines.size() > ctx->combines_cap)
+        if (sub.tiles.size() > ctx->tiles_cap || sub.combines.size() > ctx->combines_cap ||
+            static_cast<size_t>(sub.max_cta_tiles) * sizeof(uint2) > static_cast<size_t>(ctx->mk.sched_bytes))
             return fail(ctx, EDGEFM_ERR_BAD_SHAPE, "a subset of %d rows does not fit the tile plan of this context", n);
         ss = &sub;
         CUDA_TRY(ctx, cudaMalloc(&fresh, static_cast<size_t>(n) * H * sizeof(uint16_t)));
@@ -667,7 +693,7 @@ edgefm_status edgefm_set_vocab_subset(edgefm_ctx *ctx, const int32_t *token_ids,
             }
         }
         op.units_total = n;
-        op.flags = PHF_REMAP;
+        op.layer_flags = (op.layer_flags & ~0xff) | PHF_REMAP;
     }
     // steps already enqueued on the stream still read the previous subset
     cudaError_t e = cudaStreamSynchronize(s);
@@ -681,7 +707,9 @@ edgefm_status edgefm_set_vocab_subset(edgefm_ctx *ctx, const int32_t *token_ids,
         }
     }
     const size_t lm_index = static_cast<size_t>(ctx->mk.nph - 1);
+    const uint16_t *lm_w = n > 0 ? fresh : static_cast<const uint16_t *>(ctx->lm_head);
     if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->d_ops + lm_index, &op, sizeof op, cudaMemcpyHostToDevice, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(ctx->d_op_w + lm_index, &lm_w, sizeof lm_w, cudaMemcpyHostToDevice, s);
     if (e == cudaSuccess)
         e = cudaMemcpyAsync(ctx->d_maps + lm_index * MK_MAX_VARIANTS * sizeof(CUtensorMap), lm_maps.data(), MK_MAX_VARIANTS * sizeof(CUtensorMap),
                             cudaMemcpyHostToDevice, s);
@@ -712,11 +740,20 @@ edgefm_status edgefm_debug_profile(edgefm_ctx *ctx, uint64_t *out_host, int64_t 
     *n_ctas = ctx->prof ? ctx->plan.grid : 0;
     *stride = ctx->prof_stride;
     if (!ctx->prof || !out_host) return EDGEFM_OK;
-    const int64_t n = static_cast<int64_t>(ctx->plan.grid) * ctx->prof_stride;
+    int64_t n = static_cast<int64_t>(ctx->plan.grid) * ctx->prof_stride;
     if (capacity < n) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "profile buffer too small");
+    if (capacity >= n + MK_NW_MAX * 16 * 4 + 8) n += MK_NW_MAX * 16 * 4 + 8;   // optional per-warp trace behind the table
     DeviceGuard guard(ctx->device);
     CUDA_TRY(ctx, cudaDeviceSynchronize());
     CUDA_TRY(ctx, cudaMemcpy(out_host, ctx->prof, static_cast<size_t>(n) * 8, cudaMemcpyDeviceToHost));
+    return EDGEFM_OK;
+}
+
+edgefm_status edgefm_debug_plan(const edgefm_ctx *ctx, int32_t *out8) {
+    if (!ctx || !out8) return EDGEFM_ERR_INVALID_ARG;
+    const StepPlan &pl = ctx->plan;
+    out8[0] = pl.grid; out8[1] = pl.nw; out8[2] = pl.slots; out8[3] = pl.slot_bytes; out8[4] = static_cast<int32_t>(pl.dyn_smem);
+    out8[5] = ctx->sched_full.max_cta_tiles; out8[6] = static_cast<int32_t>(pl.sched_bytes); out8[7] = pl.long_ctx ? 1 : 0;
     return EDGEFM_OK;
 }
 
@@ -843,19 +880,19 @@ extern "C" edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, co
     }
     // ---- the same plan edgefm_create makes, in host memory -------------------------------------------------
     StepPlan pl;
+    StepSchedule ss;
     {
         cudaError_t ce = cudaSuccess;
-        if (const char *why = plan_step(sh, max_context, num_sms, smem_optin, &pl, &ce))
+        if (const char *why = plan_step_and_schedule(sh, max_context, num_sms, smem_optin, &pl, &ss, &ce))
             return fail(nullptr, ce != cudaSuccess ? EDGEFM_ERR_CUDA : EDGEFM_ERR_BAD_SHAPE, "%s", why);
     }
-    StepSchedule ss;
-    if (const char *why = plan_schedule(pl, sh, sh.vocab, &ss)) return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "%s", why);
     const int grid = pl.grid, max_chunks = pl.max_chunks, n_ops = pl.n_ops;
 
     // carve the scratch array; reject shapes that need more than it holds
     ScratchCarver sc{g_scratch_dev_ptr[dev]};
     unsigned char *d_maps = sc.take<unsigned char>(static_cast<size_t>(n_ops) * MK_MAX_VARIANTS * sizeof(CUtensorMap));
     MkOp *d_ops = sc.take<MkOp>(n_ops);
+    const uint16_t **d_op_w = sc.take<const uint16_t *>(n_ops);
     uint2 *d_tiles = sc.take<uint2>(ss.tiles.size());
     int *d_cta_tab = sc.take<int>(ss.cta_tab.size());
     MkCombine *d_combines = sc.take<MkCombine>(ss.combines.size() + 1);
@@ -879,7 +916,8 @@ extern "C" edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, co
     unsigned *grid_bar = counters + nq + nkv + 2 + 32;
 
     std::vector<MkOp> ops(static_cast<size_t>(n_ops));
-    fill_ops(sh, weights->layers, weights->final_norm, x, attn, q, act, ops.data());
+    std::vector<const uint16_t *> op_w(static_cast<size_t>(n_ops));
+    fill_ops(sh, weights->layers, weights->final_norm, weights->lm_head, x, attn, q, act, ops.data(), op_w.data());
     std::vector<CUtensorMap> maps(static_cast<size_t>(n_ops) * MK_MAX_VARIANTS);
     if (const char *why = encode_maps(ss, sh, weights->layers, weights->lm_head, sh.vocab, maps.data()))
         return fail(nullptr, EDGEFM_ERR_CUDA, "%s", why);
@@ -887,7 +925,7 @@ extern "C" edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, co
 
     MkParams m{};
     fill_shape_params(&m, sh, max_context, pl, ss);
-    m.ops = d_ops; m.maps = d_maps; m.tiles = d_tiles; m.cta_tab = d_cta_tab; m.combines = d_combines;
+    m.ops = d_ops; m.op_weights = d_op_w; m.maps = d_maps; m.tiles = d_tiles; m.cta_tab = d_cta_tab; m.combines = d_combines;
     m.k_cache = static_cast<uint16_t *>(k_cache); m.v_cache = static_cast<uint16_t *>(v_cache);
     m.embed = (const uint16_t *)weights->embed; m.inv_freq = inv_freq; m.x = x; m.q = q; m.attn = attn;
     m.part_m = part_m; m.part_l = part_l; m.part_o = part_o;
@@ -905,6 +943,7 @@ extern "C" edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, co
     CUDA_TRY(nullptr, cudaMemsetAsync(counters, 0, (static_cast<size_t>(nq) + nkv + 2 + 64) * sizeof(unsigned), s));
     // pageable copies: the runtime stages the bytes before returning, so the sources may be freed after the call
     CUDA_TRY(nullptr, cudaMemcpyAsync(d_ops, ops.data(), ops.size() * sizeof(MkOp), cudaMemcpyHostToDevice, s));
+    CUDA_TRY(nullptr, cudaMemcpyAsync(d_op_w, op_w.data(), op_w.size() * sizeof(op_w[0]), cudaMemcpyHostToDevice, s));
     CUDA_TRY(nullptr, cudaMemcpyAsync(d_maps, maps.data(), maps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice, s));
     CUDA_TRY(nullptr, cudaMemcpyAsync(d_tiles, ss.tiles.data(), ss.tiles.size() * sizeof(uint2), cudaMemcpyHostToDevice, s));
     CUDA_TRY(nullptr, cudaMemcpyAsync(d_cta_tab, ss.cta_tab.data(), ss.cta_tab.size() * sizeof(int), cudaMemcpyHostToDevice, s));
@@ -939,5 +978,37 @@ extern "C" edgefm_status edgefm_sync_status(edgefm_ctx *ctx, void *stream) {
     if (st.status != 0)
         return fail(ctx, EDGEFM_ERR_TIMEOUT, "device status %d (6 = a bounded wait expired, 100+ = self-check code) operands %d %d; "
                     "the context must be destroyed", st.status, st.pad[0], st.pad[1]);
+    return EDGEFM_OK;
+}
+
+// Host-only diagnostics: the tile schedule of one operator, in the form the kernel reads, for checking the planner
+// without a GPU.  tiles_out receives the tiles CTA by CTA, warp by warp (tiles_per_warp [n_ctas * n_warps] counts them);
+// combines_out four words per entry (combines_per_cta [n_ctas]); variant_rows [4] the box heights of the tensor maps.
+extern "C" edgefm_status edgefm_debug_plan_operator(int32_t kind, int32_t units, int32_t K, int32_t head_half, int32_t op_index, int32_t n_ctas,
+                                                    int32_t n_warps, int32_t slot_rows, uint64_t *tiles_out, int64_t tiles_cap,
+                                                    int32_t *tiles_per_warp, uint32_t *combines_out, int64_t combines_cap,
+                                                    int32_t *combines_per_cta, int32_t *variant_rows, int64_t *n_tiles, int64_t *n_combines) {
+    if (!tiles_per_warp || !combines_per_cta || !variant_rows || !n_tiles || !n_combines || n_ctas < 1 || n_warps < 1)
+        return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "bad argument");
+    OpShape os{kind, units, K, op_paired(kind) ? 2 * units : units, head_half};
+    OpSchedule S;
+    if (const char *why = plan_op(os, op_index, n_ctas, n_warps, slot_rows, &S)) return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "%s", why);
+    int64_t nt = 0, nc = 0;
+    for (int c = 0; c < n_ctas; ++c) {
+        for (int w = 0; w < n_warps; ++w) {
+            tiles_per_warp[c * n_warps + w] = static_cast<int32_t>(S.tiles[c][w].size());
+            for (const uint2 &d : S.tiles[c][w]) {
+                if (tiles_out && nt < tiles_cap) tiles_out[nt] = static_cast<uint64_t>(d.x) | static_cast<uint64_t>(d.y) << 32;
+                ++nt;
+            }
+        }
+        combines_per_cta[c] = static_cast<int32_t>(S.combines[c].size());
+        for (const MkCombine &e : S.combines[c]) {
+            if (combines_out && nc < combines_cap) { combines_out[4 * nc] = e.x; combines_out[4 * nc + 1] = e.y; combines_out[4 * nc + 2] = e.z; combines_out[4 * nc + 3] = e.w; }
+            ++nc;
+        }
+    }
+    for (int v = 0; v < MK_MAX_VARIANTS; ++v) variant_rows[v] = v < S.n_variants ? S.variant_rows[v] : 0;
+    *n_tiles = nt; *n_combines = nc;
     return EDGEFM_OK;
 }

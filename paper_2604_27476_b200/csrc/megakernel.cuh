@@ -7,13 +7,14 @@
 //   * The step's weight traffic is a static schedule made on the host (QKV, O, gate/up, down of every layer,
 //     then lm_head).  Every CTA owns a fixed share of each operator's rows; the share is cut into tiles of up
 //     to 16 rows x 256 columns, and every consumer warp owns a fixed list of tiles (the same for every layer).
-//   * One more warp of the CTA only FEEDS: lane w walks the tile list of consumer warp w over the whole step
-//     and fetches the tiles with 2-D TMA tensor copies (cp.async.bulk.tensor.2d, mbarrier complete_tx) into
-//     warp w's private ring of shared-memory slots.  It never waits: every pass it tests which slots have been
-//     released and refills those.  The weights do not depend on the computation, so the stream runs ahead
-//     across operator boundaries; HBM keeps streaming while the consumers wait at a grid barrier, stage an
-//     activation vector or run attention.  Every slot has a "full" and an "empty" mbarrier, armed by one lane
-//     and drained by one warp strictly in order, so the one-bit phase parity cannot alias.
+//   * Every consumer warp keeps a private ring of shared-memory slots filled with its next tiles by 2-D TMA tensor
+//     copies (cp.async.bulk.tensor, mbarrier complete_tx): when it has multiplied a tile, its lane 0 at once fetches
+//     the tile that comes S places later in its sequence into the freed slot -- regardless of operator boundaries,
+//     the weights do not depend on the computation.  So the short operators of a layer are on chip when their turn
+//     comes and HBM keeps streaming while the arithmetic waits at a grid barrier, stages an activation vector or
+//     runs attention.  One more warp of the CTA computes nothing: it runs ahead of the rings and pulls the tiles
+//     that come next into L2 (prefetch.global.L2), because the rings alone hold too little to keep HBM busy through
+//     the stalls and a refill from L2 returns much sooner than one from HBM.
 //   * A consumer warp waits for its next tile, multiplies it with the 256 activations of the tile's columns
 //     (8 per lane, from the vector staged in shared memory) into 16 row accumulators and releases the slot.
 //     Consecutive tiles of a warp cover the same rows; only at the end of a run of tiles are the 16 sums
@@ -28,6 +29,8 @@
 // issuing copies, waits (bounded) for the copies it has in flight and returns.
 // This file is the body of the kernel.  It is included once per build (MK_NS = namespace, MK_NW_VALUE = consumer
 // warps per CTA); everything that does not depend on the number of warps lives in megakernel_types.cuh.
+#include <type_traits>
+
 #include "megakernel_types.cuh"
 
 namespace edgefm {
@@ -35,7 +38,7 @@ namespace MK_NS {
 
 constexpr int MK_NW = MK_NW_VALUE;               // consumer warps per CTA
 constexpr int MK_NT = MK_NW * 32;                // consumer threads
-constexpr int MK_THREADS = MK_NT + 32;           // + the feeding warp
+constexpr int MK_THREADS = MK_NT + 32;           // + the L2 prefetch warp
 constexpr int MK_ATT_MW = (MK_NW + 1) / 2;       // warps whose partials fit the merge area at once
 
 // 1: one-head-per-CTA attention leaves the merge of its chunks to the O projection's prologue (every CTA merges);
@@ -110,6 +113,20 @@ __device__ __forceinline__ void tma_load_box(void *dst, const void *map, int x, 
         ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(policy)
         : "memory");
 }
+// A pair of boxes in one copy: gate rows and their up rows (3-D view [2][F][K] of the gate/up matrix) ...
+__device__ __forceinline__ void tma_load_box3(void *dst, const void *map, int x, int y, int z, unsigned long long *bar, unsigned long long policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar)), "l"(policy)
+        : "memory");
+}
+// ... or rows i.. and i + d/2.. of one head (4-D view [heads][2][d/2][K] of the QKV matrix).
+__device__ __forceinline__ void tma_load_box4(void *dst, const void *map, int x, int y, int z, int w, unsigned long long *bar, unsigned long long policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(smem_u32(bar)), "l"(policy)
+        : "memory");
+}
 // all consumer threads of the CTA (the feeding warp never joins)
 __device__ __forceinline__ void cta_sync() { asm volatile("bar.sync 1, %0;" ::"n"(MK_NT) : "memory"); }
 
@@ -167,79 +184,122 @@ __device__ __forceinline__ int unit_row(const MkParams &p, int kind, int u) {
     return u;
 }
 
-// ---- the feeding warp: lane w refills the ring of consumer warp w -------------------------------------------
-// Tiles are fetched in the order the consumer takes them; slot k % S of round k / S.  A slot is refilled once its
-// "empty" barrier has completed the previous round (the consumer arrives there after its last read of the slot).
-__device__ __forceinline__ void feed_rings(const MkParams &p, const MkOp *s_ops, const int *s_tab, unsigned char *ring,
-                                           unsigned long long *full_bar, unsigned long long *empty_bar, volatile int *abort_flag,
-                                           volatile unsigned *s_issued, int lane) {
-    if (lane >= MK_NW) return;
-    const int *tab = s_tab + lane * MK_WARP_TAB;
-    const int n_layer = tab[1] + tab[2] + tab[3] + tab[4], n_lm = tab[6];
-    const uint2 *layer_list = p.tiles + tab[0], *lm_list = p.tiles + tab[5];
-    const long long total = static_cast<long long>(n_layer) * p.n_layers + n_lm;
-    unsigned char *my_ring = ring + static_cast<size_t>(lane) * p.slots * p.slot_bytes;
-    unsigned long long *fb = full_bar + lane * MK_MAX_SLOTS, *eb = empty_bar + lane * MK_MAX_SLOTS;
-    unsigned long long policy;
+// ---- fetching a warp's tiles ------------------------------------------------------------------------------------
+// Every consumer warp keeps S tiles in flight in its own ring: slot k % S holds tile k of the warp's sequence over the
+// whole step (its layer list once per layer, then its output-layer list).  Right after the warp has multiplied a tile,
+// its lane 0 fetches the tile S places further into the slot that has just become free -- whatever operator that tile
+// belongs to, so the stream runs ahead across operator boundaries.  One lane arms and one warp drains every "full"
+// barrier strictly in order, so the one-bit phase parity cannot alias and no "empty" barrier is needed.
+struct TileCursor {
+    int layer, i;          // next tile: i-th of the layer list (layer < n_layers) or of the output-layer list
+    unsigned count;        // tiles passed so far
+};
+__device__ __forceinline__ void cursor_step(TileCursor &c, int n_layer, int n_layers) {
+    ++c.count;
+    ++c.i;
+    if (c.layer < n_layers && c.i == n_layer) { c.i = 0; ++c.layer; }
+}
+struct WarpStream {
+    const uint2 *layer_list, *lm_list;   // this warp's tile lists (shared memory)
+    int n_layer;                // tiles per layer
+    unsigned total;             // tiles of the whole step
+    TileCursor next;            // next tile to fetch (lane 0's view)
+    const uint2 *list;          // next tile to multiply
+    unsigned char *ring;        // this warp's slots
+    unsigned long long *full_bar;   // [slots]
+    int slot;                   // slot of the next tile to multiply
+    unsigned round;
+    unsigned consumed;          // tiles multiplied so far
+    int fenced_op;
+};
+// Lane 0 only: fetch tile ws.next into ring slot `slot` (whose previous contents this warp has finished reading).
+__device__ __forceinline__ bool fetch_next_tile(const MkParams &p, WarpStream &ws, int slot, volatile int *abort_flag, volatile unsigned *s_issued,
+                                                int warp) {
+    if (ws.next.count >= ws.total) return true;
+    const bool lm = ws.next.layer >= p.n_layers;
+    const uint2 d = lm ? ws.lm_list[ws.next.i] : ws.layer_list[ws.next.i];
+    // the operators of a layer are QKV, O, gate/up, down in this order; 4 = the output layer
+    const int op = static_cast<int>((d.y >> 20) & 7u);
+    const int opi = lm ? 4 * p.n_layers : 4 * ws.next.layer + op;
+    const int m = static_cast<int>(d.y & 31u), x = static_cast<int>((d.x >> 20) & 0xffu) * MK_TILE_COLS;
+    const int u0 = static_cast<int>(d.x & 0xfffffu);
+    const bool paired = op == 0 || op == 2;
+    const unsigned bytes = static_cast<unsigned>(m) * (MK_TILE_COLS * 2) * (paired ? 2u : 1u);
+    // (the host made the schedule; a corrupt entry must still not write past the slot)
+    if (m < 1 || bytes > static_cast<unsigned>(p.slot_bytes) || (lm ? op != 4 : op > 3)) return diag_fail(p, abort_flag, 1, opi, u0);
+    const unsigned char *map = p.maps + (static_cast<size_t>(opi) * MK_MAX_VARIANTS + ((d.x >> 28) & 3u)) * 128;
+    if (opi != ws.fenced_op && (p.map_fence == 2 || (p.map_fence == 1 && lm))) {
+        // the host may have rewritten this operator's tensor maps since the last launch (another vocabulary subset, or a
+        // static call with other weights): order the copy engine's view of them behind what is in memory now
+        ws.fenced_op = opi;
+        for (int v = 0; v < MK_MAX_VARIANTS; ++v)
+            asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(p.maps + (static_cast<size_t>(opi) * MK_MAX_VARIANTS + v) * 128) : "memory");
+    }
+    unsigned char *dst = ws.ring + static_cast<size_t>(slot) * p.slot_bytes;
+    unsigned long long *bar = &ws.full_bar[slot];
+    unsigned long long policy;   // weights are read once per step: first out of L2
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
-    int slot = 0;
-    unsigned round = 0;          // times this lane has gone around its ring
-    int layer = 0, i = 0;        // next tile: i-th of the layer list (layer < n_layers) or of the output-layer list
-    if (n_layer == 0) layer = p.n_layers;
-    long long done = 0;
-    int fenced_op = -1;
+    // the warp read the slot through the generic proxy: order those reads before the asynchronous write
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    mbar_arrive_expect_tx(bar, bytes);
+    if (op == 0) tma_load_box4(dst, map, x, u0 & ((p.d >> 1) - 1), 0, u0 >> p.half_shift, bar, policy);
+    else if (op == 2) tma_load_box3(dst, map, x, u0, 0, bar, policy);
+    else tma_load_box(dst, map, x, u0, bar, policy);
+    cursor_step(ws.next, ws.n_layer, p.n_layers);
+    s_issued[warp] = ws.next.count;     // read by the L2 prefetch warp
+    return true;
+}
+
+// ---- the L2 prefetch warp ------------------------------------------------------------------------------------
+// The ring of a consumer warp holds only a few tiles, so HBM would idle whenever the consumers stall (grid barriers,
+// attention) and every refill would pay the full HBM latency.  One more warp therefore runs ahead of the rings: lanes w
+// and 16 + w walk the tile list of consumer warp w (low rows / partner rows of every tile) and ask L2 for the lines of
+// every tile that is at most `pf_tiles` tiles ahead of what the feeding lane of that warp has fetched (plain
+// prefetch.global.L2, one 128-byte line per instruction).  The lanes only read counters; nobody ever waits for them,
+// and a tile the ring has already fetched is skipped.
+__device__ __forceinline__ void prefetch_tiles(const MkParams &p, const MkOp *s_ops, const int *s_tab, const uint2 *s_tiles,
+                                               volatile int *abort_flag, volatile unsigned *s_issued, int lane) {
+    const int w = lane & 15, half = lane >> 4;
+    if (p.pf_tiles <= 0 || w >= MK_NW) return;
+    const int *tab = s_tab + w * MK_WARP_TAB;
+    const int n_layer = tab[1] + tab[2] + tab[3] + tab[4], n_lm = tab[6];
+    const uint2 *layer_list = s_tiles + tab[0], *lm_list = s_tiles + tab[5];
+    const unsigned total = static_cast<unsigned>(n_layer) * p.n_layers + n_lm;
+    unsigned k = 0;              // next tile of this warp's whole-step sequence to ask for
     unsigned idle = 0;
-    unsigned long long t_idle = 0;
-    uint2 d = make_uint2(0u, 0u);
-    if (total > 0) d = __ldg(layer < p.n_layers ? layer_list : lm_list);
-    while (done < total) {
-        if (round > 0 && !mbar_test_wait(&eb[slot], (round - 1) & 1u)) {
-            // nothing to do for this lane right now; give up after the bound (the consumers never released the slot)
-            if ((++idle & 255u) == 0u) {
-                if (*abort_flag) break;
-                const unsigned long long now = global_ns();
-                if (t_idle == 0) t_idle = now;
-                else if (now - t_idle > p.spin_limit) { *abort_flag = 1; break; }
-            }
+    while (k < total) {
+        const unsigned issued = s_issued[w];
+        if (k < issued) k = issued;                         // the ring got there first
+        if (k >= total) break;
+        if (k >= issued + static_cast<unsigned>(p.pf_tiles)) {   // far enough ahead: wait for the ring to move
+            if (*abort_flag || ++idle > (1u << 22)) return;  // bounded: give up (prefetching is only a hint)
+            __nanosleep(200);
             continue;
         }
-        idle = 0; t_idle = 0;
-        if (*abort_flag) break;
-        const bool lm = layer >= p.n_layers;
+        idle = 0;
+        const unsigned in_layers = static_cast<unsigned>(n_layer) * p.n_layers;
+        const bool lm = k >= in_layers;
+        const int layer = lm ? p.n_layers : static_cast<int>(k / n_layer);
+        const uint2 d = lm ? lm_list[k - in_layers] : layer_list[k - static_cast<unsigned>(layer) * n_layer];
         const int op = static_cast<int>((d.y >> 20) & 7u);
         const int opi = lm ? 4 * p.n_layers : 4 * layer + op;
         const MkOp &P = s_ops[opi];
-        const int m = static_cast<int>(d.y & 31u), kcol = static_cast<int>((d.x >> 20) & 0xffu);
-        const int variant = static_cast<int>((d.x >> 28) & 3u);
-        const int u0 = static_cast<int>(d.x & 0xfffffu);
         const bool paired = P.kind == PH_QKV || P.kind == PH_SWIGLU;
-        const int row = unit_row(p, P.kind, u0);
-        const unsigned box_bytes = static_cast<unsigned>(m) * (MK_TILE_COLS * 2);
-        // bounds (the host made the schedule; a corrupt entry must not reach the copy engine)
-        if (m < 1 || m > MK_TILE_ROWS || (paired && m > 8) || kcol * MK_TILE_COLS >= P.K || u0 + m > P.units_total ||
-            static_cast<int>(box_bytes) * (paired ? 2 : 1) > p.slot_bytes || (lm ? op != 4 : op > 3)) {
-            diag_fail(p, abort_flag, 1, opi, u0);
-            break;
+        const int m = static_cast<int>(d.y & 31u), kcol = static_cast<int>((d.x >> 20) & 0xffu);
+        const int u0 = static_cast<int>(d.x & 0xfffffu);
+        ++k;
+        if (m < 1 || m > MK_TILE_ROWS || u0 + m > P.units_total || kcol * MK_TILE_COLS >= P.K || (lm ? op != 4 : op > 3)) return;
+        // rows of this lane: the low box (or rows 0..7), the partner box (or rows 8..)
+        int row = unit_row(p, P.kind, u0), n_rows = paired ? m : min(m, 8);
+        if (half) {
+            if (paired) row += P.kind == PH_QKV ? (p.d >> 1) : p.F;
+            else { row += 8; n_rows = m - 8; }
         }
-        const unsigned char *map = p.maps + (static_cast<size_t>(opi) * MK_MAX_VARIANTS + variant) * 128;
-        if (opi != fenced_op && (p.map_fence == 2 || (p.map_fence == 1 && lm))) {
-            // the host may have rewritten this operator's tensor maps since the last launch (another vocabulary subset, or a
-            // static call with other weights): order the copy engine's view of them behind what is in memory now
-            fenced_op = opi;
-            for (int v = 0; v < MK_MAX_VARIANTS; ++v)
-                asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(p.maps + (static_cast<size_t>(opi) * MK_MAX_VARIANTS + v) * 128) : "memory");
-        }
-        unsigned char *dst = my_ring + static_cast<size_t>(slot) * p.slot_bytes;
-        mbar_arrive_expect_tx(&fb[slot], paired ? 2u * box_bytes : box_bytes);
-        tma_load_box(dst, map, kcol * MK_TILE_COLS, row, &fb[slot], policy);
-        if (paired) tma_load_box(dst + p.hi_off, map, kcol * MK_TILE_COLS, row + (P.kind == PH_QKV ? (p.d >> 1) : p.F), &fb[slot], policy);
-        ++done;
-        s_issued[lane] = static_cast<unsigned>(done);
-        if (++slot == p.slots) { slot = 0; ++round; }
-        // next tile
-        ++i;
-        if (!lm && i == n_layer) { i = 0; ++layer; }
-        if (done < total) d = __ldg((layer < p.n_layers ? layer_list : lm_list) + i);
+        const int row_bytes = P.K * 2, col0 = kcol * (MK_TILE_COLS * 2);
+        const int n_lines = min(MK_TILE_COLS * 2, row_bytes - col0 + 127) / 128;
+        const unsigned char *base = reinterpret_cast<const unsigned char *>(p.op_weights[opi]) + static_cast<size_t>(row) * row_bytes + col0;
+        for (int r = 0; r < n_rows; ++r)
+            for (int l = 0; l < n_lines; ++l) asm volatile("prefetch.global.L2 [%0];" ::"l"(base + static_cast<size_t>(r) * row_bytes + l * 128));
     }
 }
 
@@ -261,7 +321,7 @@ __device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkOp &P,
         if (arg_better(lo, u, cx.best_v, cx.best_i)) { cx.best_v = lo; cx.best_i = u; }
     } else if (P.kind == PH_SWIGLU) {
         const float a = lo / (1.f + expf(-lo)) * hi;
-        if (P.flags & PHF_OUT_SPLIT) {   // the layout the next operator's prologue copies straight into shared memory
+        if (P.flags() & PHF_OUT_SPLIT) {   // the layout the next operator's prologue copies straight into shared memory
             const int i4 = u >> 2;
             P.out[(i4 & 1) * (P.units_total >> 1) + ((i4 >> 1) << 2) + (u & 3)] = a;
         } else {
@@ -275,7 +335,7 @@ __device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkOp &P,
             lo += bf16_bits_to_f32(P.bias[row_lo]);
             hi += bf16_bits_to_f32(P.bias[row_hi]);
         }
-        const size_t layer_off = static_cast<size_t>(P.layer) * p.nkv * p.max_context * p.d;
+        const size_t layer_off = static_cast<size_t>(P.layer()) * p.nkv * p.max_context * p.d;
         if (head < p.nq + p.nkv) {
             const float c = cx.rope[i], sn = cx.rope[half + i];
             const float rlo = lo * c - hi * sn, rhi = hi * c + lo * sn;
@@ -315,48 +375,59 @@ __device__ __forceinline__ float reduce_rows(float (&a)[MK_TILE_ROWS], int lane)
 }
 
 // ---- the consumer side of the weight stream --------------------------------------------------------------------
-struct WarpStream {
-    const uint2 *list;          // next tile of this warp (layer list or output-layer list)
-    unsigned char *ring;        // this warp's slots
-    unsigned long long *full_bar, *empty_bar;   // [slots]
-    int slot;
-    unsigned round;
-    unsigned consumed;          // tiles taken so far
-};
-
+// Optional fine-grained trace of one operator in CTA 0 (compile with -DEDGEFM_TRACE_OP=<operator index>): lane 0 of every
+// consumer warp appends %globaltimer stamps (before the wait, data there, tile multiplied) behind the profile table.
+#ifdef EDGEFM_TRACE_OP
+#define MK_TRACE(k)                                                                                                           \
+    do {                                                                                                                      \
+        if (p.prof && (&P - p_ops_base) == EDGEFM_TRACE_OP && blockIdx.x == 0 && lane == 0 && t < 16)                          \
+            p.prof[static_cast<size_t>(gridDim.x) * p.prof_stride + ((threadIdx.x >> 5) * 16 + t) * 3 + (k)] = global_ns();     \
+    } while (0)
+#else
+#define MK_TRACE(k) do {} while (0)
+#endif
 // This warp's `n` tiles of operator P: wait, multiply, release; reduce and finish rows where the schedule says so.
-__device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkOp &P, int n, WarpStream &ws, const float4 *xsA, const float4 *xsB,
-                                              volatile int *abort_flag, ItemCtx &cx, float *s_partial, int lane) {
+__device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkOp *p_ops_base, const MkOp &P, int n, WarpStream &ws, const float4 *xsA, const float4 *xsB,
+                                              volatile int *abort_flag, ItemCtx &cx, float *s_partial, volatile unsigned *s_issued, int lane) {
     float acc[MK_TILE_ROWS];   // 16 independent chains: enough to cover the FMA latency
     const bool paired = P.kind == PH_QKV || P.kind == PH_SWIGLU;
-    const int hoff = paired ? p.hi_off : 8 * MK_TILE_COLS * 2;   // accumulator rows 8.. of an unpaired tile simply follow rows 0..7
-    uint2 d = n > 0 ? __ldg(ws.list) : make_uint2(0u, 0u);
+    uint2 d = n > 0 ? *ws.list : make_uint2(0u, 0u);
     for (int t = 0; t < n; ++t) {
-        const uint2 dn = t + 1 < n ? __ldg(ws.list + t + 1) : make_uint2(0u, 0u);
+        const uint2 dn = t + 1 < n ? ws.list[t + 1] : make_uint2(0u, 0u);
         if (d.x & MKT_FIRST) {
 #pragma unroll
             for (int r = 0; r < MK_TILE_ROWS; ++r) acc[r] = 0.f;
         }
         const int m = static_cast<int>(d.y & 31u), kcol = static_cast<int>((d.x >> 20) & 0xffu);
         const float4 xa = xsA[kcol * 32 + lane], xb = xsB[kcol * 32 + lane];
+        MK_TRACE(0);
         if (!mbar_wait(&ws.full_bar[ws.slot], ws.round & 1u, abort_flag, p.spin_limit)) return false;
+        MK_TRACE(1);
         const unsigned char *tile = ws.ring + static_cast<size_t>(ws.slot) * p.slot_bytes + lane * 16;
-        auto row = [&](int r) {
-            const uint4 w = *reinterpret_cast<const uint4 *>(tile + (r < 8 ? r * (MK_TILE_COLS * 2) : hoff + (r - 8) * (MK_TILE_COLS * 2)));
-            acc[r] = dot8(w, xa, xb, acc[r]);
+        // accumulator rows 8.. : the partner rows of a paired tile follow its m low rows; those of an unpaired tile follow rows 0..7
+        const int hoff = (paired ? m : 8) * (MK_TILE_COLS * 2);
+        // rows of the tile as a compile-time mask: the loop is fully unrolled and free of branches, so the loads of all rows are in
+        // flight together (rows a tile does not have read stale bytes of the slot; their sums are never used)
+        auto rows = [&](auto mask_c) {
+            constexpr unsigned MASK = decltype(mask_c)::value;
+#pragma unroll
+            for (int r = 0; r < MK_TILE_ROWS; ++r) {
+                if (MASK >> r & 1u) {
+                    const uint4 w = *reinterpret_cast<const uint4 *>(tile + (r < 8 ? r * (MK_TILE_COLS * 2) : hoff + (r - 8) * (MK_TILE_COLS * 2)));
+                    acc[r] = dot8(w, xa, xb, acc[r]);
+                }
+            }
         };
-        if (paired ? m == 8 : m == MK_TILE_ROWS) {
-#pragma unroll
-            for (int r = 0; r < MK_TILE_ROWS; ++r) row(r);
+        if (paired) {
+            if (m <= 4) rows(std::integral_constant<unsigned, 0x0f0fu>()); else rows(std::integral_constant<unsigned, 0xffffu>());
         } else {
-            // rows the tile does not have hold stale bytes: skip them (their sums are never used, but need not be computed)
-            const unsigned mask = paired ? ((1u << m) - 1u) * 0x101u : (1u << m) - 1u;
-#pragma unroll
-            for (int r = 0; r < MK_TILE_ROWS; ++r)
-                if (mask >> r & 1u) row(r);
+            if (m <= 8) rows(std::integral_constant<unsigned, 0x00ffu>());
+            else if (m <= 12) rows(std::integral_constant<unsigned, 0x0fffu>());
+            else rows(std::integral_constant<unsigned, 0xffffu>());
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(&ws.empty_bar[ws.slot]);   // the slot may be refilled
+        MK_TRACE(2);
+        if (lane == 0 && !fetch_next_tile(p, ws, ws.slot, abort_flag, s_issued, static_cast<int>(threadIdx.x >> 5))) return false;   // refill the slot
         if (++ws.slot == p.slots) { ws.slot = 0; ++ws.round; }
         ++ws.consumed;
         if (d.x & MKT_FLUSH) {
@@ -398,7 +469,8 @@ __device__ __forceinline__ void att_chunking(const MkParams &p, int n, int hg, i
 // (m, l, unnormalised o); the exact log-sum-exp merge is done here, in chunk order, by every CTA.
 __device__ __forceinline__ bool gemv_phase(const MkParams &p, const MkOp *s_ops, const int *s_tab, int ph, int op_in_layer, WarpStream &ws,
                                            float4 *xsA, float4 *xsB, volatile int *abort_flag, float *s_part, float *s_partial, ItemCtx &cx,
-                                           int token, int merge_attn, int tid, int &prof_idx, unsigned long long *x_bar, unsigned &x_parity) {
+                                           int token, int merge_attn, int tid, int &prof_idx, unsigned long long *x_bar, unsigned &x_parity,
+                                           volatile unsigned *s_issued) {
     const MkOp &P = s_ops[ph];
     const int lane = tid & 31, warp = tid >> 5;
     const int cta = blockIdx.x;
@@ -449,7 +521,7 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, const MkOp *s_ops,
             acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
             if (o4 & 1) xsB[o4 >> 1] = acc; else xsA[o4 >> 1] = acc;
         }
-    } else if (P.flags & PHF_X_BULK) {
+    } else if (P.flags() & PHF_X_BULK) {
         // the vector is already in the split layout and needs no transform: two bulk copies, every thread waits for them
         // (the CTA-wide sync of the grid barrier ordered all earlier reads of the buffer before this point)
         // The vector was written by other CTAs of this launch with ordinary stores and acquired at the grid barrier;
@@ -513,7 +585,7 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, const MkOp *s_ops,
     }
     const int *tab = s_tab + warp * MK_WARP_TAB;
     const int n_tiles = op_in_layer < 4 ? tab[1 + op_in_layer] : tab[6];
-    bool ok = consume_tiles(p, P, n_tiles, ws, xsA, xsB, abort_flag, cx, s_partial, lane);
+    bool ok = consume_tiles(p, s_ops, P, n_tiles, ws, xsA, xsB, abort_flag, cx, s_partial, s_issued, lane);
     // units whose columns were shared between warps: their partial sums meet here, slots in order
     const int *ctab = s_tab + MK_NW * MK_WARP_TAB + 2 * op_in_layer;
     const int n_comb = ctab[1];
@@ -734,35 +806,29 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
     cta_sync();
     if (!*s_flag) return;
 
-    // Last CTA of this head group: merge the chunks.  All loads of a batch (chunk statistics and up to
-    // CB partial vectors per thread) are issued before any is used.
+    // Last CTA of this head group: merge the chunks.  All loads of a batch (up to CB partial vectors per thread) are
+    // issued before any is used.
     __threadfence();
     constexpr int CB = 8;
-    const bool has_out = tid < HG * D / 4;       // output (h, j4) of this thread, if any
-    const int oh = has_out ? tid / (D / 4) : 0, oj4 = has_out ? tid - oh * (D / 4) : 0;
-    const float4 *po = reinterpret_cast<const float4 *>(p.part_o + static_cast<size_t>(qh0 + oh) * p.max_chunks * D) + oj4;
-    float4 ob[CB];
-#pragma unroll
-    for (int u = 0; u < CB; ++u)
-        ob[u] = (has_out && u < nch) ? __ldcg(po + static_cast<size_t>(u) * (D / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
     for (int i = tid; i < HG * nch; i += MK_NT) {
         const int h = i / nch, cc = i - h * nch;
         cm[h * p.max_chunks + cc] = __ldcg(p.part_m + (qh0 + h) * p.max_chunks + cc);
         cl[h * p.max_chunks + cc] = __ldcg(p.part_l + (qh0 + h) * p.max_chunks + cc);
     }
     cta_sync();
-    if (has_out) {
+    for (int out = tid; out < HG * D / 4; out += MK_NT) {     // output (h, j4) of this thread
+        const int oh = out / (D / 4), oj4 = out - oh * (D / 4);
+        const float4 *po = reinterpret_cast<const float4 *>(p.part_o + static_cast<size_t>(qh0 + oh) * p.max_chunks * D) + oj4;
         const float *hm = cm + oh * p.max_chunks, *hl = cl + oh * p.max_chunks;
         float mm = -INFINITY;
         for (int cc = 0; cc < nch; ++cc) mm = fmaxf(mm, hm[cc]);
         float ll = 0.f;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
         for (int c0 = 0; c0 < nch; c0 += CB) {
-            if (c0 > 0) {
+            float4 ob[CB];
 #pragma unroll
-                for (int u = 0; u < CB; ++u)
-                    ob[u] = (c0 + u < nch) ? __ldcg(po + static_cast<size_t>(c0 + u) * (D / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
+            for (int u = 0; u < CB; ++u)
+                ob[u] = (c0 + u < nch) ? __ldcg(po + static_cast<size_t>(c0 + u) * (D / 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
             for (int u = 0; u < CB; ++u) {
                 if (c0 + u < nch) {
@@ -787,13 +853,17 @@ template <int D, int G, bool LONG>
 __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParams p) {
     extern __shared__ __align__(1024) unsigned char mk_smem[];
     unsigned char *smem = mk_smem;
-    float4 *xsA = reinterpret_cast<float4 *>(smem);
-    float4 *xsB = reinterpret_cast<float4 *>(smem + p.xbuf_bytes / 2);
-    MkOp *s_ops = reinterpret_cast<MkOp *>(smem + p.xbuf_bytes);                       // the step's operators
-    int *s_tab = reinterpret_cast<int *>(smem + p.xbuf_bytes + p.ops_bytes);           // this CTA's schedule table
-    unsigned char *ring = smem + p.xbuf_bytes + p.ops_bytes + p.tab_bytes;             // [MK_NW][slots][slot_bytes]
+    // dynamic shared memory: operators | schedule table | tile lists | rings | activation vector (also the attention scratch).
+    // The vector comes last on purpose: a tile of fewer than 16 rows is multiplied with a fixed, branch-free row loop
+    // that may read (and ignore) bytes behind the tile, i.e. behind the last slot of the last ring.
+    MkOp *s_ops = reinterpret_cast<MkOp *>(smem);                                      // the step's operators
+    int *s_tab = reinterpret_cast<int *>(smem + p.ops_bytes);                          // this CTA's schedule table
+    uint2 *s_tiles = reinterpret_cast<uint2 *>(smem + p.ops_bytes + p.tab_bytes);      // this CTA's tile lists
+    unsigned char *ring = smem + p.ops_bytes + p.tab_bytes + p.sched_bytes;            // [MK_NW][slots][slot_bytes]
+    unsigned char *xbuf = ring + static_cast<size_t>(MK_NW) * p.slots * p.slot_bytes;
+    float4 *xsA = reinterpret_cast<float4 *>(xbuf);
+    float4 *xsB = reinterpret_cast<float4 *>(xbuf + p.xbuf_bytes / 2);
     __shared__ __align__(8) unsigned long long full_bar[MK_NW * MK_MAX_SLOTS];
-    __shared__ __align__(8) unsigned long long empty_bar[MK_NW * MK_MAX_SLOTS];
     __shared__ __align__(8) unsigned long long x_bar;   // completion of bulk-copied activation vectors
     __shared__ float s_rope[128];
     __shared__ float s_part[MK_NW];
@@ -802,16 +872,14 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
     __shared__ int s_bi[MK_NW];
     __shared__ int s_flag;
     __shared__ int s_abort;
-    __shared__ unsigned s_issued[MK_NW];   // tiles fetched so far per consumer warp (written by the feeding lanes)
-    __shared__ int s_feed_done;
+    __shared__ unsigned s_issued[MK_NW];   // tiles fetched so far per consumer warp (read by the L2 prefetch warp)
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int cta = blockIdx.x, ncta = gridDim.x;
     if (tid == 0) {
-        for (int i = 0; i < MK_NW * MK_MAX_SLOTS; ++i) { mbar_init(&full_bar[i], 1); mbar_init(&empty_bar[i], 1); }
+        for (int i = 0; i < MK_NW * MK_MAX_SLOTS; ++i) mbar_init(&full_bar[i], 1);
         mbar_init(&x_bar, 1);
         s_abort = 0;
-        s_feed_done = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (tid < MK_NW) s_issued[tid] = 0u;
@@ -822,14 +890,14 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
         for (int i = tid; i < n16; i += MK_THREADS) dst[i] = src[i];
         const int *tsrc = p.cta_tab + static_cast<size_t>(cta) * p.cta_tab_ints;
         for (int i = tid; i < p.cta_tab_ints; i += MK_THREADS) s_tab[i] = tsrc[i];
+        const int t0 = tsrc[MK_NW * MK_WARP_TAB + 10], nt = min(tsrc[MK_NW * MK_WARP_TAB + 11], p.sched_bytes / 8);
+        for (int i = tid; i < nt; i += MK_THREADS) s_tiles[i] = p.tiles[t0 + i];
     }
-    __syncthreads();   // the only CTA-wide sync: from here on the feeding warp and the consumers go separate ways
+    __syncthreads();   // the only CTA-wide sync: from here on the prefetch warp and the consumers go separate ways
     volatile int *abort_flag = &s_abort;
 
     if (warp == MK_NW) {
-        feed_rings(p, s_ops, s_tab, ring, full_bar, empty_bar, abort_flag, s_issued, lane);
-        __syncwarp();
-        if (lane == 0) { __threadfence_block(); s_feed_done = 1; }
+        prefetch_tiles(p, s_ops, s_tab, s_tiles, abort_flag, s_issued, lane);
         return;
     }
 
@@ -843,11 +911,19 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
     }
 
     WarpStream ws;
+    {
+        const int *tab = s_tab + warp * MK_WARP_TAB;
+        ws.layer_list = s_tiles + tab[0];
+        ws.lm_list = s_tiles + tab[5];
+        ws.n_layer = tab[1] + tab[2] + tab[3] + tab[4];
+        ws.total = static_cast<unsigned>(ws.n_layer) * p.n_layers + tab[6];
+        ws.next = TileCursor{ws.n_layer == 0 ? p.n_layers : 0, 0, 0u};
+    }
     ws.ring = ring + static_cast<size_t>(warp) * p.slots * p.slot_bytes;
     ws.full_bar = &full_bar[warp * MK_MAX_SLOTS];
-    ws.empty_bar = &empty_bar[warp * MK_MAX_SLOTS];
     ws.slot = 0; ws.round = 0; ws.consumed = 0;
-    ws.list = p.tiles + s_tab[warp * MK_WARP_TAB];
+    ws.list = ws.layer_list;
+    ws.fenced_op = -1;
     bool ok = true;
     const int rt = p.req->token, rp = p.req->position;
     const int token = rt >= 0 ? rt : p.state->next_token;
@@ -866,6 +942,11 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
     }
     if (ok && cta == 0 && tid == 0) { p.state->token = token; p.state->position = pos; }
     // (s_rope is published by the sync of the first prologue)
+
+    // start this warp's weight stream: fill its ring
+    if (ok && lane == 0)
+        for (int sl = 0; sl < p.slots && ok; ++sl) ok = fetch_next_tile(p, ws, sl, abort_flag, s_issued, warp);
+    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
 
     ItemCtx cx;
     cx.rscale = 1.f; cx.slot_row = slot_row; cx.rope = s_rope; cx.best_v = -INFINITY; cx.best_i = 0x7fffffff;
@@ -887,32 +968,29 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
     for (int ph = 0; ph < p.nph && ok; ++ph) {
         const bool layer_op = ph < n_layer_ops;
         const bool after_attention = layer_op && (ph & 3) == 1;
-        if (layer_op && (ph & 3) == 0) ws.list = p.tiles + s_tab[warp * MK_WARP_TAB];          // every layer walks the same list
-        if (!layer_op) ws.list = p.tiles + s_tab[warp * MK_WARP_TAB + 5];
+        if (layer_op && (ph & 3) == 0) ws.list = ws.layer_list;          // every layer walks the same list
+        if (!layer_op) ws.list = ws.lm_list;
         if (after_attention) {
             const int l = ph >> 2;
             if constexpr (LONG) {
-                if (att_split) attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, smem, tid, &s_flag);
-                else attention_phase<D, G, MK_ATT_LPP>(p, l, n_att, p.att_chunk_shared, false, smem, tid, &s_flag);
+                if (att_split) attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, xbuf, tid, &s_flag);
+                else attention_phase<D, G, MK_ATT_LPP>(p, l, n_att, p.att_chunk_shared, false, xbuf, tid, &s_flag);
             } else {
-                attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, smem, tid, &s_flag);
+                attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, xbuf, tid, &s_flag);
             }
             ok = grid_barrier(p, ++bar_no * bar_arrivals, abort_flag, tid, prof_idx) && ok;
             if (!ok) break;
         }
         ok = gemv_phase(p, s_ops, s_tab, ph, layer_op ? (ph & 3) : 4, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token,
-                        after_attention ? merge_chunks : 0, tid, prof_idx, &x_bar, x_parity);
+                        after_attention ? merge_chunks : 0, tid, prof_idx, &x_bar, x_parity, s_issued);
         if (layer_op) ok = grid_barrier(p, ++bar_no * bar_arrivals, abort_flag, tid, prof_idx) && ok;
     }
     prof_stamp(p, tid, prof_idx);
     if (!ok || *abort_flag) {
-        // aborted: once the feeding warp has stopped, wait (bounded) for the copies still in flight into this warp's ring
+        // aborted: wait (bounded) for the copies still in flight into this warp's ring, then leave
         *abort_flag = 1;
         if (tid == 0 && p.state->status == 0) p.state->status = 6;
-        const unsigned long long t0 = global_ns();
-        while (!*reinterpret_cast<volatile int *>(&s_feed_done))
-            if (global_ns() - t0 > p.spin_limit) break;
-        const unsigned issued = *reinterpret_cast<volatile unsigned *>(&s_issued[warp]);
+        const unsigned issued = __shfl_sync(0xffffffffu, ws.next.count, 0);
         for (unsigned k = ws.consumed; k < issued; ++k) {
             const unsigned long long t1 = global_ns();
             while (!mbar_try_wait(&ws.full_bar[ws.slot], ws.round & 1u))
@@ -959,7 +1037,7 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
         }
         if (lane == 0) {
             if (bi == 0x7fffffff) bi = 0;
-            if (s_ops[p.nph - 1].flags & PHF_REMAP) bi = p.vocab_ids[bi];   // pruned vocabulary: row index -> token id
+            if (s_ops[p.nph - 1].flags() & PHF_REMAP) bi = p.vocab_ids[bi];   // pruned vocabulary: row index -> token id
             int *nto = p.req->next_token_out;
             if (nto) *nto = bi;
             p.state->next_token = bi;

@@ -16,7 +16,7 @@ constexpr int MK_TILE_ROWS = 16;                 // accumulator rows of a consum
 constexpr int MK_MAX_VARIANTS = 4;               // tensor maps (box heights) per weight matrix
 constexpr int MK_MAX_SLOTS = 4;                  // ring slots per consumer warp
 constexpr int MK_WARP_TAB = 8;                   // ints per warp in the per-CTA table
-// Consumer warps per CTA of the two builds of the kernel (one more warp feeds them): the short-context build favours
+// Consumer warps per CTA of the two builds of the kernel (one more warp prefetches into L2): the short-context build favours
 // instruction streams, the long-context build (grouped attention keeps G heads of accumulators per warp) registers.
 #ifndef MK_NW_SHORT_VALUE
 #define MK_NW_SHORT_VALUE 11
@@ -46,9 +46,9 @@ struct alignas(16) MkOp {
     int K;                   // columns (multiple of 8)
     int kind;
     int units_total;         // rows (PH_RESID, PH_LMHEAD), pairs (PH_QKV: rows/2, PH_SWIGLU: F)
-    int layer;
-    int flags;               // PHF_* bits
-    int pad[3];
+    int layer_flags;         // layer << 8 | PHF_* bits
+    __host__ __device__ int layer() const { return layer_flags >> 8; }
+    __host__ __device__ int flags() const { return layer_flags & 0xff; }
 };
 static_assert(sizeof(MkOp) % 16 == 0, "descriptor is copied in 16-byte pieces");
 
@@ -97,16 +97,18 @@ struct MkParams {
     StepState *state;
     const StepRequest *req;
     // weight streaming
+    const uint16_t *const *op_weights;   // [nph] base of every operator's matrix (the L2 prefetch uses plain addresses)
     const unsigned char *maps;     // CUtensorMap [(4 * n_layers + 1) * MK_MAX_VARIANTS], 128 bytes each, index (4 l + op) * 4 + variant
-    const uint2 *tiles;            // all tile lists
-    const int *cta_tab;            // [gridDim.x][cta_tab_ints]: per consumer warp {layer list offset, tiles per operator x4, output-layer
-                                   // list offset, output-layer tiles, 0}, then per operator (5) {combine offset, combine count}
+    const uint2 *tiles;            // all tile lists, one contiguous block per CTA (copied to shared memory when the kernel starts)
+    const int *cta_tab;            // [gridDim.x][cta_tab_ints]: per consumer warp {layer list offset in the CTA's block, tiles per
+                                   // operator x4, output-layer list offset, output-layer tiles, 0}, then per operator (5) {combine
+                                   // offset, combine count}, then {first tile of the CTA's block, tiles in the block}
     const MkCombine *combines;
     int cta_tab_ints;
     int slots;                     // ring slots per consumer warp
     int slot_bytes;                // bytes of one slot (a multiple of 1024)
-    int hi_off;                    // offset of the partner box inside a slot
-    int xbuf_bytes, ops_bytes, tab_bytes;
+    int xbuf_bytes, ops_bytes, tab_bytes, sched_bytes;   // shared-memory areas: operators, table, tile lists, [rings], activation vector
+    int pf_tiles;                  // tiles per consumer warp the L2 prefetch runs ahead of the ring
     int map_fence;                 // tensor maps the host may have rewritten since the last launch: 0 none, 1 the output layer's, 2 all
     int barrier_extra;             // test hook: arrivals the grid barrier expects beyond the CTAs present (0 in production)
     unsigned spin_limit;           // upper bound of every device-side wait, nanoseconds

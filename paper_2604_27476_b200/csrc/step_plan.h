@@ -39,7 +39,7 @@ inline bool op_paired(int kind) { return kind == PH_QKV || kind == PH_SWIGLU; }
 // op_index: 0..3 inside a layer, 4 = output layer.  Returns null, or why the operator does not fit.
 inline const char *plan_op(const OpShape &os, int op_index, int ncta, int nw, int slot_rows, OpSchedule *out) {
     const bool paired = op_paired(os.kind);
-    const int B = paired ? std::min(8, slot_rows / 2) : std::min(MK_TILE_ROWS, slot_rows);   // units per block
+    int B = paired ? std::min(8, slot_rows / 2) : std::min(MK_TILE_ROWS, slot_rows);   // units per block
     if (B < 1) return "ring slots too small for a tile";
     const int nkb = (os.K + MK_TILE_COLS - 1) / MK_TILE_COLS;
     if (nkb > 255) return "rows too long for the tile schedule";
@@ -67,6 +67,7 @@ inline const char *plan_op(const OpShape &os, int op_index, int ncta, int nw, in
         }
         if (best < 0) granule = 1;
         if (os.units % granule) return "QKV rows do not split into blocks";
+        B = B / granule * granule;   // blocks of whole granules: at most four different heights (granule, 2 granules, ...)
     }
     struct Block { int u0, m, v0, variant; };
     for (int c = 0; c < ncta; ++c) {
@@ -125,47 +126,51 @@ inline const char *plan_op(const OpShape &os, int op_index, int ncta, int nw, in
 // The step's schedule in the form the kernel reads.
 struct StepSchedule {
     OpSchedule ops[5];
-    std::vector<uint2> tiles;        // per CTA, per warp: the layer list (operators 0..3), then, behind all of them, the output-layer lists
+    std::vector<uint2> tiles;        // per CTA one block: the warps' layer lists (operators 0..3), then their output-layer lists
     std::vector<int> cta_tab;        // [ncta][cta_tab_ints]
     std::vector<MkCombine> combines;
     int cta_tab_ints = 0;
-    size_t lm_tiles_begin = 0;       // first output-layer tile in `tiles`
+    int max_cta_tiles = 0;           // largest block (sizes the shared-memory copy)
 };
 
-inline int cta_tab_ints_for(int nw) { return (nw * MK_WARP_TAB + 10 + 3) / 4 * 4; }
+inline int cta_tab_ints_for(int nw) { return (nw * MK_WARP_TAB + 12 + 3) / 4 * 4; }
 
 inline void assemble_schedule(StepSchedule *ss, int ncta, int nw) {
     ss->cta_tab_ints = cta_tab_ints_for(nw);
     ss->cta_tab.assign(static_cast<size_t>(ncta) * ss->cta_tab_ints, 0);
     ss->tiles.clear();
     ss->combines.clear();
-    for (int c = 0; c < ncta; ++c)
+    ss->max_cta_tiles = 0;
+    for (int c = 0; c < ncta; ++c) {
+        int *ctab = &ss->cta_tab[static_cast<size_t>(c) * ss->cta_tab_ints];
+        const size_t base = ss->tiles.size();
         for (int w = 0; w < nw; ++w) {
-            int *tab = &ss->cta_tab[static_cast<size_t>(c) * ss->cta_tab_ints + w * MK_WARP_TAB];
-            tab[0] = static_cast<int>(ss->tiles.size());
+            int *tab = ctab + w * MK_WARP_TAB;
+            tab[0] = static_cast<int>(ss->tiles.size() - base);
             for (int o = 0; o < 4; ++o) {
                 const auto &l = ss->ops[o].tiles[c][w];
                 tab[1 + o] = static_cast<int>(l.size());
                 ss->tiles.insert(ss->tiles.end(), l.begin(), l.end());
             }
         }
-    ss->lm_tiles_begin = ss->tiles.size();
-    for (int c = 0; c < ncta; ++c)
         for (int w = 0; w < nw; ++w) {
-            int *tab = &ss->cta_tab[static_cast<size_t>(c) * ss->cta_tab_ints + w * MK_WARP_TAB];
+            int *tab = ctab + w * MK_WARP_TAB;
             const auto &l = ss->ops[4].tiles[c][w];
-            tab[5] = static_cast<int>(ss->tiles.size());
+            tab[5] = static_cast<int>(ss->tiles.size() - base);
             tab[6] = static_cast<int>(l.size());
             ss->tiles.insert(ss->tiles.end(), l.begin(), l.end());
         }
-    for (int c = 0; c < ncta; ++c)
         for (int o = 0; o < 5; ++o) {
-            int *ct = &ss->cta_tab[static_cast<size_t>(c) * ss->cta_tab_ints + nw * MK_WARP_TAB + 2 * o];
+            int *ct = ctab + nw * MK_WARP_TAB + 2 * o;
             const auto &l = ss->ops[o].combines[c];
             ct[0] = static_cast<int>(ss->combines.size());
             ct[1] = static_cast<int>(l.size());
             ss->combines.insert(ss->combines.end(), l.begin(), l.end());
         }
+        ctab[nw * MK_WARP_TAB + 10] = static_cast<int>(base);
+        ctab[nw * MK_WARP_TAB + 11] = static_cast<int>(ss->tiles.size() - base);
+        ss->max_cta_tiles = std::max(ss->max_cta_tiles, static_cast<int>(ss->tiles.size() - base));
+    }
 }
 
 // ---- tensor maps ---------------------------------------------------------------------------------------------------
@@ -188,14 +193,30 @@ inline TensorMapEncodeFn tensor_map_encoder() {
 
 // Tensor map of a row-major bf16 [rows][K] matrix on THIS GPU with boxes of box_rows x 256 elements; columns and rows
 // outside the matrix read as zero.  (No multicast is ever used with these maps.)
-inline bool encode_weight_map(CUtensorMap *m, const void *base, int rows, int K, int box_rows) {
+//   pair_rows == 0                : 2-D, coordinates (column, row);
+//   pair_rows  > 0, group == 0    : 3-D view [2][pair_rows][K] (gate rows, up rows): one box = box_rows low rows and their partners;
+//   pair_rows  > 0, group  > 0    : 4-D view [rows / (2 pair_rows)][2][pair_rows][K] (heads of the QKV matrix: rotate-half partners).
+inline bool encode_weight_map(CUtensorMap *m, const void *base, int rows, int K, int box_rows, int pair_rows = 0, bool grouped = false) {
     TensorMapEncodeFn enc = tensor_map_encoder();
     if (!enc) return false;
-    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(rows)};
-    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(K) * 2};
-    const cuuint32_t box[2] = {MK_TILE_COLS, static_cast<cuuint32_t>(box_rows)};
-    const cuuint32_t es[2] = {1, 1};
-    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    const cuuint64_t row_bytes = static_cast<cuuint64_t>(K) * 2;
+    cuuint64_t dims[4] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(rows), 1, 1};
+    cuuint64_t strides[3] = {row_bytes, 0, 0};
+    cuuint32_t box[4] = {MK_TILE_COLS, static_cast<cuuint32_t>(box_rows), 1, 1};
+    const cuuint32_t es[4] = {1, 1, 1, 1};
+    cuuint32_t rank = 2;
+    if (pair_rows > 0) {
+        dims[1] = static_cast<cuuint64_t>(pair_rows); dims[2] = 2;
+        strides[1] = row_bytes * pair_rows;
+        box[2] = 2;
+        rank = 3;
+        if (grouped) {
+            dims[3] = static_cast<cuuint64_t>(rows / (2 * pair_rows));
+            strides[2] = row_bytes * pair_rows * 2;
+            rank = 4;
+        }
+    }
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void *>(base), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 

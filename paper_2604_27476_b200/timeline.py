@@ -33,6 +33,8 @@ def collect(cfg, device="cuda:0", warm_steps=6):
             del os.environ["EDGEFM_PROFILE"]
         else:
             os.environ["EDGEFM_PROFILE"] = old
+    from . import edgefm_debug_plan
+    print("launch plan:", edgefm_debug_plan(ctx.handle))
     kd = torch.from_numpy(k.view(np.int16)).to(device)
     vd = torch.from_numpy(v.view(np.int16)).to(device)
     ctx.prefill_kv(kd, vd)
