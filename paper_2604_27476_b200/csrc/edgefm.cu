@@ -209,7 +209,7 @@ inline const char *plan_step_and_schedule(const edgefm_shape &sh, int max_contex
     for (int attempt = 0; attempt < 6; ++attempt) {
         if (const char *why = plan_step(sh, max_context, num_sms, smem_optin, reserve, pl, cuda_err)) return why;
         if (const char *why = plan_schedule(*pl, sh, sh.vocab, ss)) return why;
-        const size_t need = static_cast<size_t>(ss->max_cta_tiles) * sizeof(uint2);
+        const size_t need = ss->smem_bytes();
         if (need <= pl->sched_bytes) return nullptr;
         reserve = need + (attempt > 0 ? need / 8 : 0);
     }
@@ -681,7 +681,7 @@ edgefm_status edgefm_set_vocab_subset(edgefm_ctx *ctx, const int32_t *token_ids,
             return fail(ctx, EDGEFM_ERR_BAD_SHAPE, "a subset of %d rows does not fit the tile plan of this context: %s", n, why);
         assemble_schedule(&sub, pl.grid, pl.nw);
         if (sub.tiles.size() > ctx->tiles_cap || sub.combines.size() > ctx->combines_cap ||
-            static_cast<size_t>(sub.max_cta_tiles) * sizeof(uint2) > static_cast<size_t>(ctx->mk.sched_bytes))
+            sub.smem_bytes() > static_cast<size_t>(ctx->mk.sched_bytes))
             return fail(ctx, EDGEFM_ERR_BAD_SHAPE, "a subset of %d rows does not fit the tile plan of this context", n);
         ss = &sub;
         CUDA_TRY(ctx, cudaMalloc(&fresh, static_cast<size_t>(n) * H * sizeof(uint16_t)));

@@ -46,6 +46,12 @@ constexpr int MK_ATT_MW = (MK_NW + 1) / 2;       // warps whose partials fit the
 #ifndef MK_SPLIT_DEFER
 #define MK_SPLIT_DEFER 1
 #endif
+#ifndef MK_MERGE_NOUT
+#define MK_MERGE_NOUT 1
+#endif
+#ifndef MK_DEFER_REFILL
+#define MK_DEFER_REFILL 0
+#endif
 
 // ---- mbarrier / bulk copy primitives -----------------------------------------------------------------
 __device__ __forceinline__ unsigned smem_u32(const void *p) { return static_cast<unsigned>(__cvta_generic_to_shared(p)); }
@@ -130,6 +136,26 @@ __device__ __forceinline__ void tma_load_box4(void *dst, const void *map, int x,
 // all consumer threads of the CTA (the feeding warp never joins)
 __device__ __forceinline__ void cta_sync() { asm volatile("bar.sync 1, %0;" ::"n"(MK_NT) : "memory"); }
 
+// Dynamic shared memory: operators | schedule table | tile lists | rings | activation vector (also the attention scratch).
+// The vector comes last on purpose: a tile of fewer than 16 rows is multiplied with a fixed, branch-free row loop that
+// may read (and ignore) bytes behind the tile, i.e. behind the last slot of the last ring.
+// (Addresses are recomputed from the kernel parameters where they are used instead of being carried in registers.)
+extern __shared__ __align__(1024) unsigned char mk_smem[];
+__device__ __forceinline__ MkOp *sm_ops(const MkParams &) { return reinterpret_cast<MkOp *>(mk_smem); }
+__device__ __forceinline__ int *sm_tab(const MkParams &p) { return reinterpret_cast<int *>(mk_smem + p.ops_bytes); }
+__device__ __forceinline__ uint2 *sm_tiles(const MkParams &p) { return reinterpret_cast<uint2 *>(mk_smem + p.ops_bytes + p.tab_bytes); }
+// the CTA's combine entries follow its tiles (16-byte aligned)
+__device__ __forceinline__ MkCombine *sm_combines(const MkParams &p) {
+    const int nt = sm_tab(p)[MK_NW * MK_WARP_TAB + 11];
+    return reinterpret_cast<MkCombine *>(mk_smem + p.ops_bytes + p.tab_bytes + ((nt * 8 + 15) & ~15));
+}
+__device__ __forceinline__ unsigned char *sm_ring(const MkParams &p, int warp) {
+    return mk_smem + p.ops_bytes + p.tab_bytes + p.sched_bytes + warp * (p.slots * p.slot_bytes);
+}
+__device__ __forceinline__ unsigned char *sm_xbuf(const MkParams &p) { return sm_ring(p, MK_NW); }
+__device__ __forceinline__ float4 *sm_xa(const MkParams &p) { return reinterpret_cast<float4 *>(sm_xbuf(p)); }
+__device__ __forceinline__ float4 *sm_xb(const MkParams &p) { return reinterpret_cast<float4 *>(sm_xbuf(p) + p.xbuf_bytes / 2); }
+
 __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned *p) {
     unsigned v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -155,11 +181,15 @@ __device__ __forceinline__ bool diag_fail(const MkParams &p, volatile int *abort
 }
 
 // All consumer threads of all CTAs meet here.  Returns false when the wait expired (step aborted).
-__device__ __forceinline__ bool grid_barrier(const MkParams &p, unsigned target, volatile int *abort_flag, int tid, int &prof_idx) {
+// `while_waiting` runs after this CTA has announced its arrival and before it starts polling (refills that short
+// operators put off: the time is free here).
+template <typename F>
+__device__ __forceinline__ bool grid_barrier(const MkParams &p, unsigned target, volatile int *abort_flag, int tid, int &prof_idx, F &&while_waiting) {
     cta_sync();
     prof_stamp(p, tid, prof_idx);   // this CTA's share of the operator is done
+    if (tid == 0 && !*abort_flag) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.barrier) : "memory");
+    while_waiting();
     if (tid == 0 && !*abort_flag) {
-        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.barrier) : "memory");
         unsigned it = 0;
         unsigned long long t0 = 0;
         while (ld_acquire_gpu(p.barrier) < target) {
@@ -200,24 +230,22 @@ __device__ __forceinline__ void cursor_step(TileCursor &c, int n_layer, int n_la
     if (c.layer < n_layers && c.i == n_layer) { c.i = 0; ++c.layer; }
 }
 struct WarpStream {
-    const uint2 *layer_list, *lm_list;   // this warp's tile lists (shared memory)
-    int n_layer;                // tiles per layer
-    unsigned total;             // tiles of the whole step
+    int list;                   // next tile to multiply: index into the CTA's tile lists
     TileCursor next;            // next tile to fetch (lane 0's view)
-    const uint2 *list;          // next tile to multiply
-    unsigned char *ring;        // this warp's slots
-    unsigned long long *full_bar;   // [slots]
     int slot;                   // slot of the next tile to multiply
     unsigned round;
     unsigned consumed;          // tiles multiplied so far
+    int pending;                // slots read but not refilled yet (short operators leave the refill to the next grid barrier)
     int fenced_op;
 };
 // Lane 0 only: fetch tile ws.next into ring slot `slot` (whose previous contents this warp has finished reading).
 __device__ __forceinline__ bool fetch_next_tile(const MkParams &p, WarpStream &ws, int slot, volatile int *abort_flag, volatile unsigned *s_issued,
-                                                int warp) {
-    if (ws.next.count >= ws.total) return true;
+                                                unsigned long long *full_bar, int warp) {
+    const int *tab = sm_tab(p) + warp * MK_WARP_TAB;
+    const int n_layer = tab[1] + tab[2] + tab[3] + tab[4];
+    if (ws.next.count >= static_cast<unsigned>(n_layer) * p.n_layers + tab[6]) return true;
     const bool lm = ws.next.layer >= p.n_layers;
-    const uint2 d = lm ? ws.lm_list[ws.next.i] : ws.layer_list[ws.next.i];
+    const uint2 d = sm_tiles(p)[(lm ? tab[5] : tab[0]) + ws.next.i];
     // the operators of a layer are QKV, O, gate/up, down in this order; 4 = the output layer
     const int op = static_cast<int>((d.y >> 20) & 7u);
     const int opi = lm ? 4 * p.n_layers : 4 * ws.next.layer + op;
@@ -235,8 +263,8 @@ __device__ __forceinline__ bool fetch_next_tile(const MkParams &p, WarpStream &w
         for (int v = 0; v < MK_MAX_VARIANTS; ++v)
             asm volatile("fence.proxy.tensormap::generic.acquire.gpu [%0], 128;" ::"l"(p.maps + (static_cast<size_t>(opi) * MK_MAX_VARIANTS + v) * 128) : "memory");
     }
-    unsigned char *dst = ws.ring + static_cast<size_t>(slot) * p.slot_bytes;
-    unsigned long long *bar = &ws.full_bar[slot];
+    unsigned char *dst = sm_ring(p, warp) + slot * p.slot_bytes;
+    unsigned long long *bar = &full_bar[warp * MK_MAX_SLOTS + slot];
     unsigned long long policy;   // weights are read once per step: first out of L2
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
     // the warp read the slot through the generic proxy: order those reads before the asynchronous write
@@ -245,9 +273,25 @@ __device__ __forceinline__ bool fetch_next_tile(const MkParams &p, WarpStream &w
     if (op == 0) tma_load_box4(dst, map, x, u0 & ((p.d >> 1) - 1), 0, u0 >> p.half_shift, bar, policy);
     else if (op == 2) tma_load_box3(dst, map, x, u0, 0, bar, policy);
     else tma_load_box(dst, map, x, u0, bar, policy);
-    cursor_step(ws.next, ws.n_layer, p.n_layers);
+    cursor_step(ws.next, n_layer, p.n_layers);
     s_issued[warp] = ws.next.count;     // read by the L2 prefetch warp
     return true;
+}
+
+// Refill the slots a short operator left empty (whole warp; lane 0 issues).
+__device__ __forceinline__ bool refill_pending(const MkParams &p, WarpStream &ws, volatile int *abort_flag, volatile unsigned *s_issued,
+                                               unsigned long long *full_bar, int warp, int lane) {
+    bool ok = true;
+    if (ws.pending > 0 && lane == 0) {
+        int sl = ws.slot - ws.pending;
+        if (sl < 0) sl += p.slots;
+        for (int i = 0; i < ws.pending && ok; ++i) {
+            ok = fetch_next_tile(p, ws, sl, abort_flag, s_issued, full_bar, warp);
+            if (++sl == p.slots) sl = 0;
+        }
+    }
+    ws.pending = 0;
+    return ok;
 }
 
 // ---- the L2 prefetch warp ------------------------------------------------------------------------------------
@@ -257,8 +301,10 @@ __device__ __forceinline__ bool fetch_next_tile(const MkParams &p, WarpStream &w
 // every tile that is at most `pf_tiles` tiles ahead of what the feeding lane of that warp has fetched (plain
 // prefetch.global.L2, one 128-byte line per instruction).  The lanes only read counters; nobody ever waits for them,
 // and a tile the ring has already fetched is skipped.
-__device__ __forceinline__ void prefetch_tiles(const MkParams &p, const MkOp *s_ops, const int *s_tab, const uint2 *s_tiles,
-                                               volatile int *abort_flag, volatile unsigned *s_issued, int lane) {
+__device__ __forceinline__ void prefetch_tiles(const MkParams &p, volatile int *abort_flag, volatile unsigned *s_issued, int lane) {
+    const MkOp *s_ops = sm_ops(p);
+    const int *s_tab = sm_tab(p);
+    const uint2 *s_tiles = sm_tiles(p);
     const int w = lane & 15, half = lane >> 4;
     if (p.pf_tiles <= 0 || w >= MK_NW) return;
     const int *tab = s_tab + w * MK_WARP_TAB;
@@ -306,18 +352,19 @@ __device__ __forceinline__ void prefetch_tiles(const MkParams &p, const MkOp *s_
 struct ItemCtx {
     float rscale;          // deferred RMSNorm factor (1 for plain prologues)
     int slot_row;          // cache slot written by this step
-    const float *rope;     // smem cos[d/2], sin[d/2]
     float best_v;          // PH_LMHEAD running argmax of this lane
     int best_i;
-    float *logits_out;
 };
 
 // ---- fused epilogue of one output unit (a row, or a row pair) ------------------------------------------------
-__device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkOp &P, ItemCtx &cx, int u, float lo, float hi) {
+// pre: the value the epilogue adds (old residual / the two biases) was fetched ahead into pre_lo, pre_hi.
+__device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkOp &P, ItemCtx &cx, const float *s_rope, int u, float lo, float hi,
+                                               bool pre = false, float pre_lo = 0.f, float pre_hi = 0.f) {
     if (P.kind == PH_RESID) {
-        P.out[u] = __ldcg(P.out + u) + lo;
+        P.out[u] = (pre ? pre_lo : __ldcg(P.out + u)) + lo;
     } else if (P.kind == PH_LMHEAD) {
-        if (cx.logits_out) cx.logits_out[u] = lo;
+        float *logits_out = p.req->logits_out;
+        if (logits_out) logits_out[u] = lo;
         if (arg_better(lo, u, cx.best_v, cx.best_i)) { cx.best_v = lo; cx.best_i = u; }
     } else if (P.kind == PH_SWIGLU) {
         const float a = lo / (1.f + expf(-lo)) * hi;
@@ -332,12 +379,12 @@ __device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkOp &P,
         const int head = u >> p.half_shift, i = u & (half - 1);
         const int row_lo = head * p.d + i, row_hi = row_lo + half;
         if (P.bias) {
-            lo += bf16_bits_to_f32(P.bias[row_lo]);
-            hi += bf16_bits_to_f32(P.bias[row_hi]);
+            lo += pre ? pre_lo : bf16_bits_to_f32(P.bias[row_lo]);
+            hi += pre ? pre_hi : bf16_bits_to_f32(P.bias[row_hi]);
         }
         const size_t layer_off = static_cast<size_t>(P.layer()) * p.nkv * p.max_context * p.d;
         if (head < p.nq + p.nkv) {
-            const float c = cx.rope[i], sn = cx.rope[half + i];
+            const float c = s_rope[i], sn = s_rope[half + i];
             const float rlo = lo * c - hi * sn, rhi = hi * c + lo * sn;
             if (head < p.nq) {
                 P.out[row_lo] = rlo;
@@ -387,23 +434,30 @@ __device__ __forceinline__ float reduce_rows(float (&a)[MK_TILE_ROWS], int lane)
 #define MK_TRACE(k) do {} while (0)
 #endif
 // This warp's `n` tiles of operator P: wait, multiply, release; reduce and finish rows where the schedule says so.
-__device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkOp *p_ops_base, const MkOp &P, int n, WarpStream &ws, const float4 *xsA, const float4 *xsB,
-                                              volatile int *abort_flag, ItemCtx &cx, float *s_partial, volatile unsigned *s_issued, int lane) {
+__device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkOp &P, int n, WarpStream &ws, volatile int *abort_flag, ItemCtx &cx,
+                                              float *s_partial, const float *s_rope, volatile unsigned *s_issued, unsigned long long *full_bar, int lane) {
+    const int warp = static_cast<int>(threadIdx.x >> 5);
+    const MkOp *p_ops_base = sm_ops(p);
+    (void)p_ops_base;
     float acc[MK_TILE_ROWS];   // 16 independent chains: enough to cover the FMA latency
     const bool paired = P.kind == PH_QKV || P.kind == PH_SWIGLU;
-    uint2 d = n > 0 ? *ws.list : make_uint2(0u, 0u);
+    // a short operator (all its tiles are already in the ring) leaves the refills to the grid barrier that follows it, so that
+    // nothing but the arithmetic sits on its critical path
+    const bool defer = MK_DEFER_REFILL != 0 && n + ws.pending <= p.slots && P.kind != PH_LMHEAD;
+    const uint2 *list = sm_tiles(p) + ws.list;
+    uint2 d = n > 0 ? list[0] : make_uint2(0u, 0u);
     for (int t = 0; t < n; ++t) {
-        const uint2 dn = t + 1 < n ? ws.list[t + 1] : make_uint2(0u, 0u);
+        const uint2 dn = t + 1 < n ? list[t + 1] : make_uint2(0u, 0u);
         if (d.x & MKT_FIRST) {
 #pragma unroll
             for (int r = 0; r < MK_TILE_ROWS; ++r) acc[r] = 0.f;
         }
         const int m = static_cast<int>(d.y & 31u), kcol = static_cast<int>((d.x >> 20) & 0xffu);
-        const float4 xa = xsA[kcol * 32 + lane], xb = xsB[kcol * 32 + lane];
+        const float4 xa = sm_xa(p)[kcol * 32 + lane], xb = sm_xb(p)[kcol * 32 + lane];
         MK_TRACE(0);
-        if (!mbar_wait(&ws.full_bar[ws.slot], ws.round & 1u, abort_flag, p.spin_limit)) return false;
+        if (!mbar_wait(&full_bar[warp * MK_MAX_SLOTS + ws.slot], ws.round & 1u, abort_flag, p.spin_limit)) return false;
         MK_TRACE(1);
-        const unsigned char *tile = ws.ring + static_cast<size_t>(ws.slot) * p.slot_bytes + lane * 16;
+        const unsigned char *tile = sm_ring(p, warp) + ws.slot * p.slot_bytes + lane * 16;
         // accumulator rows 8.. : the partner rows of a paired tile follow its m low rows; those of an unpaired tile follow rows 0..7
         const int hoff = (paired ? m : 8) * (MK_TILE_COLS * 2);
         // rows of the tile as a compile-time mask: the loop is fully unrolled and free of branches, so the loads of all rows are in
@@ -427,7 +481,8 @@ __device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkOp *p_o
         }
         __syncwarp();
         MK_TRACE(2);
-        if (lane == 0 && !fetch_next_tile(p, ws, ws.slot, abort_flag, s_issued, static_cast<int>(threadIdx.x >> 5))) return false;   // refill the slot
+        if (defer) ++ws.pending;
+        else if (lane == 0 && !fetch_next_tile(p, ws, ws.slot, abort_flag, s_issued, full_bar, warp)) return false;   // refill the slot
         if (++ws.slot == p.slots) { ws.slot = 0; ++ws.round; }
         ++ws.consumed;
         if (d.x & MKT_FLUSH) {
@@ -437,7 +492,7 @@ __device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkOp *p_o
                 const float hi = __shfl_down_sync(0xffffffffu, v, 16);   // partner row 8 + j of unit j
                 const int v0 = static_cast<int>((d.y >> 5) & 15u);
                 const int u = static_cast<int>(d.x & 0xfffffu) + j;
-                if (!(lane & 1) && j < m && j >= v0 && (!paired || lane < 16)) apply_epilogue(p, P, cx, u, v * cx.rscale, hi * cx.rscale);
+                if (!(lane & 1) && j < m && j >= v0 && (!paired || lane < 16)) apply_epilogue(p, P, cx, s_rope, u, v * cx.rscale, hi * cx.rscale);
             } else {
                 const int slot = static_cast<int>((d.y >> 10) & 1023u);
                 if (slot >= MK_PARTIAL_SLOTS) return diag_fail(p, abort_flag, 2, slot, 0);
@@ -467,11 +522,12 @@ __device__ __forceinline__ void att_chunking(const MkParams &p, int n, int hg, i
 // whose columns were shared between warps.
 // merge_attn > 0: the input is the attention output, still split into merge_attn chunk partials per head
 // (m, l, unnormalised o); the exact log-sum-exp merge is done here, in chunk order, by every CTA.
-__device__ __forceinline__ bool gemv_phase(const MkParams &p, const MkOp *s_ops, const int *s_tab, int ph, int op_in_layer, WarpStream &ws,
-                                           float4 *xsA, float4 *xsB, volatile int *abort_flag, float *s_part, float *s_partial, ItemCtx &cx,
-                                           int token, int merge_attn, int tid, int &prof_idx, unsigned long long *x_bar, unsigned &x_parity,
-                                           volatile unsigned *s_issued) {
-    const MkOp &P = s_ops[ph];
+__device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_layer, WarpStream &ws, volatile int *abort_flag, float *s_part,
+                                           float *s_partial, const float *s_rope, ItemCtx &cx, int token, int merge_attn, int tid, int &prof_idx,
+                                           unsigned long long *x_bar, unsigned &x_parity, volatile unsigned *s_issued, unsigned long long *full_bar) {
+    const MkOp &P = sm_ops(p)[ph];
+    float4 *xsA = sm_xa(p), *xsB = sm_xb(p);
+    const int *s_tab = sm_tab(p);
     const int lane = tid & 31, warp = tid >> 5;
     const int cta = blockIdx.x;
     const int n4 = P.K >> 2;
@@ -485,41 +541,51 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, const MkOp *s_ops,
         const int d4 = p.d >> 2;
         float *sm_m = s_partial;                 // [nq][nch] chunk maxima
         float *sm_l = s_partial + p.nq * nch;    // [nq][nch] chunk denominators
-        float4 ob[MK_ATT_SPLIT_MAXC];
-        auto load_partials = [&](int o4) {
+        // every thread merges up to two 16-byte pieces of the vector per round; the partial vectors of both are requested
+        // before anything is waited for, so the whole prologue costs one trip to L2
+        constexpr int NOUT = MK_MERGE_NOUT;
+        float4 ob[NOUT][MK_ATT_SPLIT_MAXC];
+        auto load_partials = [&](int o4, float4 (&dst)[MK_ATT_SPLIT_MAXC]) {
             const int h = o4 / d4, j4 = o4 - h * d4;
             const float4 *po = reinterpret_cast<const float4 *>(p.part_o + static_cast<size_t>(h) * p.max_chunks * p.d) + j4;
 #pragma unroll
             for (int c = 0; c < MK_ATT_SPLIT_MAXC; ++c)
-                if (c < nch) ob[c] = __ldcg(po + static_cast<size_t>(c) * d4);
+                if (c < nch) dst[c] = __ldcg(po + static_cast<size_t>(c) * d4);
         };
-        if (tid < n4) load_partials(tid);        // issued before the statistics are waited for
+#pragma unroll
+        for (int u = 0; u < NOUT; ++u)
+            if (tid + u * MK_NT < n4) load_partials(tid + u * MK_NT, ob[u]);
         for (int i = tid; i < p.nq * nch; i += MK_NT) {
             const int h = i / nch, c = i - h * nch;
             sm_m[i] = __ldcg(p.part_m + h * p.max_chunks + c);
             sm_l[i] = __ldcg(p.part_l + h * p.max_chunks + c);
         }
         cta_sync();
-        for (int o4 = tid; o4 < n4; o4 += MK_NT) {
-            if (o4 != tid) load_partials(o4);
-            const int h = o4 / d4;
-            const float *hm = sm_m + h * nch, *hl = sm_l + h * nch;
-            float mm = -INFINITY;
-            for (int c = 0; c < nch; ++c) mm = fmaxf(mm, hm[c]);
-            float ll = 0.f;
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int base = tid; base < n4; base += NOUT * MK_NT) {
 #pragma unroll
-            for (int c = 0; c < MK_ATT_SPLIT_MAXC; ++c) {
-                if (c < nch) {
-                    const float e = __expf(hm[c] - mm);
-                    ll = fmaf(hl[c], e, ll);
-                    acc.x = fmaf(ob[c].x, e, acc.x); acc.y = fmaf(ob[c].y, e, acc.y);
-                    acc.z = fmaf(ob[c].z, e, acc.z); acc.w = fmaf(ob[c].w, e, acc.w);
+            for (int u = 0; u < NOUT; ++u) {
+                const int o4 = base + u * MK_NT;
+                if (o4 >= n4) break;
+                if (base != tid) load_partials(o4, ob[u]);
+                const int h = o4 / d4;
+                const float *hm = sm_m + h * nch, *hl = sm_l + h * nch;
+                float mm = -INFINITY;
+                for (int c = 0; c < nch; ++c) mm = fmaxf(mm, hm[c]);
+                float ll = 0.f;
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int c = 0; c < MK_ATT_SPLIT_MAXC; ++c) {
+                    if (c < nch) {
+                        const float e = __expf(hm[c] - mm);
+                        ll = fmaf(hl[c], e, ll);
+                        acc.x = fmaf(ob[u][c].x, e, acc.x); acc.y = fmaf(ob[u][c].y, e, acc.y);
+                        acc.z = fmaf(ob[u][c].z, e, acc.z); acc.w = fmaf(ob[u][c].w, e, acc.w);
+                    }
                 }
+                const float inv = 1.f / ll;
+                acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+                if (o4 & 1) xsB[o4 >> 1] = acc; else xsA[o4 >> 1] = acc;
             }
-            const float inv = 1.f / ll;
-            acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-            if (o4 & 1) xsB[o4 >> 1] = acc; else xsA[o4 >> 1] = acc;
         }
     } else if (P.flags() & PHF_X_BULK) {
         // the vector is already in the split layout and needs no transform: two bulk copies, every thread waits for them
@@ -585,17 +651,34 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, const MkOp *s_ops,
     }
     const int *tab = s_tab + warp * MK_WARP_TAB;
     const int n_tiles = op_in_layer < 4 ? tab[1 + op_in_layer] : tab[6];
-    bool ok = consume_tiles(p, s_ops, P, n_tiles, ws, xsA, xsB, abort_flag, cx, s_partial, s_issued, lane);
-    // units whose columns were shared between warps: their partial sums meet here, slots in order
+    // units whose columns are shared between warps are finished after the tiles, one unit per thread; what their epilogue
+    // adds (old residual value, biases) is fetched now so that the load latency overlaps the arithmetic
     const int *ctab = s_tab + MK_NW * MK_WARP_TAB + 2 * op_in_layer;
     const int n_comb = ctab[1];
+    const MkCombine *cb = sm_combines(p) + ctab[0];
+    const bool paired = P.kind == PH_QKV || P.kind == PH_SWIGLU;
+    float pre_lo = 0.f, pre_hi = 0.f;
+    if (tid < n_comb * MK_TILE_ROWS) {
+        const MkCombine e = cb[tid >> 4];
+        const int j = tid & 15, m = static_cast<int>(e.y & 0xffu), v0 = static_cast<int>(e.y >> 8);
+        if (j < m && j >= v0 && !(paired && j >= 8)) {
+            const int u = static_cast<int>(e.x) + j;
+            if (P.kind == PH_RESID) {
+                pre_lo = __ldcg(P.out + u);
+            } else if (P.kind == PH_QKV && P.bias) {
+                const int row_lo = unit_row(p, PH_QKV, u);
+                pre_lo = bf16_bits_to_f32(P.bias[row_lo]);
+                pre_hi = bf16_bits_to_f32(P.bias[row_lo + (p.d >> 1)]);
+            }
+        }
+    }
+    bool ok = consume_tiles(p, P, n_tiles, ws, abort_flag, cx, s_partial, s_rope, s_issued, full_bar, lane);
+    // their partial sums meet here, slots in order
     if (n_comb > 0) {
         cta_sync();
         if (ok && !*abort_flag) {
-            const MkCombine *cb = p.combines + ctab[0];
-            const bool paired = P.kind == PH_QKV || P.kind == PH_SWIGLU;
             for (int idx = tid; idx < n_comb * MK_TILE_ROWS; idx += MK_NT) {
-                const MkCombine e = __ldg(cb + (idx >> 4));
+                const MkCombine e = cb[idx >> 4];
                 const int j = idx & 15, m = static_cast<int>(e.y & 0xffu), v0 = static_cast<int>(e.y >> 8);
                 if (j >= m || j < v0 || (paired && j >= 8)) continue;
                 float lo = 0.f, hi = 0.f;
@@ -604,7 +687,7 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, const MkOp *s_ops,
                     lo += sp[j];
                     if (paired) hi += sp[8 + j];
                 }
-                apply_epilogue(p, P, cx, static_cast<int>(e.x) + j, lo * cx.rscale, hi * cx.rscale);
+                apply_epilogue(p, P, cx, s_rope, static_cast<int>(e.x) + j, lo * cx.rscale, hi * cx.rscale, idx == tid, pre_lo, pre_hi);
             }
         }
     }
@@ -851,18 +934,6 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
 // att_split_max_n); the grouped variant is then not compiled in, which keeps the register footprint small.
 template <int D, int G, bool LONG>
 __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParams p) {
-    extern __shared__ __align__(1024) unsigned char mk_smem[];
-    unsigned char *smem = mk_smem;
-    // dynamic shared memory: operators | schedule table | tile lists | rings | activation vector (also the attention scratch).
-    // The vector comes last on purpose: a tile of fewer than 16 rows is multiplied with a fixed, branch-free row loop
-    // that may read (and ignore) bytes behind the tile, i.e. behind the last slot of the last ring.
-    MkOp *s_ops = reinterpret_cast<MkOp *>(smem);                                      // the step's operators
-    int *s_tab = reinterpret_cast<int *>(smem + p.ops_bytes);                          // this CTA's schedule table
-    uint2 *s_tiles = reinterpret_cast<uint2 *>(smem + p.ops_bytes + p.tab_bytes);      // this CTA's tile lists
-    unsigned char *ring = smem + p.ops_bytes + p.tab_bytes + p.sched_bytes;            // [MK_NW][slots][slot_bytes]
-    unsigned char *xbuf = ring + static_cast<size_t>(MK_NW) * p.slots * p.slot_bytes;
-    float4 *xsA = reinterpret_cast<float4 *>(xbuf);
-    float4 *xsB = reinterpret_cast<float4 *>(xbuf + p.xbuf_bytes / 2);
     __shared__ __align__(8) unsigned long long full_bar[MK_NW * MK_MAX_SLOTS];
     __shared__ __align__(8) unsigned long long x_bar;   // completion of bulk-copied activation vectors
     __shared__ float s_rope[128];
@@ -886,25 +957,29 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
     {
         const int n16 = p.nph * static_cast<int>(sizeof(MkOp) / 16);
         const uint4 *src = reinterpret_cast<const uint4 *>(p.ops);
-        uint4 *dst = reinterpret_cast<uint4 *>(s_ops);
+        uint4 *dst = reinterpret_cast<uint4 *>(sm_ops(p));
         for (int i = tid; i < n16; i += MK_THREADS) dst[i] = src[i];
         const int *tsrc = p.cta_tab + static_cast<size_t>(cta) * p.cta_tab_ints;
-        for (int i = tid; i < p.cta_tab_ints; i += MK_THREADS) s_tab[i] = tsrc[i];
+        for (int i = tid; i < p.cta_tab_ints; i += MK_THREADS) sm_tab(p)[i] = tsrc[i];
         const int t0 = tsrc[MK_NW * MK_WARP_TAB + 10], nt = min(tsrc[MK_NW * MK_WARP_TAB + 11], p.sched_bytes / 8);
-        for (int i = tid; i < nt; i += MK_THREADS) s_tiles[i] = p.tiles[t0 + i];
+        for (int i = tid; i < nt; i += MK_THREADS) sm_tiles(p)[i] = p.tiles[t0 + i];
+        const int c0 = tsrc[MK_NW * MK_WARP_TAB + 12], nc = tsrc[MK_NW * MK_WARP_TAB + 13];
+        MkCombine *cdst = reinterpret_cast<MkCombine *>(mk_smem + p.ops_bytes + p.tab_bytes + ((nt * 8 + 15) & ~15));
+        if ((nt * 8 + 15) / 16 * 16 + nc * 16 <= p.sched_bytes)
+            for (int i = tid; i < nc; i += MK_THREADS) cdst[i] = p.combines[c0 + i];
     }
     __syncthreads();   // the only CTA-wide sync: from here on the prefetch warp and the consumers go separate ways
     volatile int *abort_flag = &s_abort;
 
     if (warp == MK_NW) {
-        prefetch_tiles(p, s_ops, s_tab, s_tiles, abort_flag, s_issued, lane);
+        prefetch_tiles(p, abort_flag, s_issued, lane);
         return;
     }
 
     // The small per-layer vectors (norm weights, biases) are read on the critical path right after a grid barrier;
     // ask L2 for all of them now (they stay: the weight stream is evict-first).
     for (int i = cta * MK_NT + tid; i < p.nph * 64; i += ncta * MK_NT) {
-        const MkOp &P = s_ops[i >> 6];
+        const MkOp &P = sm_ops(p)[i >> 6];
         const int line = i & 63;   // 128-byte line of the vector
         if (P.norm_w && line * 64 < P.K) asm volatile("prefetch.global.L2 [%0];" ::"l"(P.norm_w + line * 64));
         if (P.bias && P.kind == PH_QKV && line * 64 < 2 * P.units_total) asm volatile("prefetch.global.L2 [%0];" ::"l"(P.bias + line * 64));
@@ -912,17 +987,11 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
 
     WarpStream ws;
     {
-        const int *tab = s_tab + warp * MK_WARP_TAB;
-        ws.layer_list = s_tiles + tab[0];
-        ws.lm_list = s_tiles + tab[5];
-        ws.n_layer = tab[1] + tab[2] + tab[3] + tab[4];
-        ws.total = static_cast<unsigned>(ws.n_layer) * p.n_layers + tab[6];
-        ws.next = TileCursor{ws.n_layer == 0 ? p.n_layers : 0, 0, 0u};
+        const int *tab = sm_tab(p) + warp * MK_WARP_TAB;
+        ws.next = TileCursor{tab[1] + tab[2] + tab[3] + tab[4] == 0 ? p.n_layers : 0, 0, 0u};
+        ws.list = tab[0];
     }
-    ws.ring = ring + static_cast<size_t>(warp) * p.slots * p.slot_bytes;
-    ws.full_bar = &full_bar[warp * MK_MAX_SLOTS];
-    ws.slot = 0; ws.round = 0; ws.consumed = 0;
-    ws.list = ws.layer_list;
+    ws.slot = 0; ws.round = 0; ws.consumed = 0; ws.pending = 0;
     ws.fenced_op = -1;
     bool ok = true;
     const int rt = p.req->token, rp = p.req->position;
@@ -945,12 +1014,11 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
 
     // start this warp's weight stream: fill its ring
     if (ok && lane == 0)
-        for (int sl = 0; sl < p.slots && ok; ++sl) ok = fetch_next_tile(p, ws, sl, abort_flag, s_issued, warp);
+        for (int sl = 0; sl < p.slots && ok; ++sl) ok = fetch_next_tile(p, ws, sl, abort_flag, s_issued, full_bar, warp);
     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
 
     ItemCtx cx;
-    cx.rscale = 1.f; cx.slot_row = slot_row; cx.rope = s_rope; cx.best_v = -INFINITY; cx.best_i = 0x7fffffff;
-    cx.logits_out = p.req->logits_out;
+    cx.rscale = 1.f; cx.slot_row = slot_row; cx.best_v = -INFINITY; cx.best_i = 0x7fffffff;
 
     unsigned bar_no = 0;
     const unsigned bar_arrivals = static_cast<unsigned>(ncta + p.barrier_extra);
@@ -965,25 +1033,26 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
     // (the code of a step is executed once per layer: a small instruction footprint matters).  Operator 4l+1 (the O
     // projection) is preceded by the attention of layer l.
     const int n_layer_ops = 4 * p.n_layers;
+    auto refill = [&]() { if (!refill_pending(p, ws, abort_flag, s_issued, full_bar, warp, lane)) *abort_flag = 1; };
     for (int ph = 0; ph < p.nph && ok; ++ph) {
         const bool layer_op = ph < n_layer_ops;
         const bool after_attention = layer_op && (ph & 3) == 1;
-        if (layer_op && (ph & 3) == 0) ws.list = ws.layer_list;          // every layer walks the same list
-        if (!layer_op) ws.list = ws.lm_list;
+        if (layer_op && (ph & 3) == 0) ws.list = sm_tab(p)[warp * MK_WARP_TAB];          // every layer walks the same list
+        if (!layer_op) ws.list = sm_tab(p)[warp * MK_WARP_TAB + 5];
         if (after_attention) {
             const int l = ph >> 2;
             if constexpr (LONG) {
-                if (att_split) attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, xbuf, tid, &s_flag);
-                else attention_phase<D, G, MK_ATT_LPP>(p, l, n_att, p.att_chunk_shared, false, xbuf, tid, &s_flag);
+                if (att_split) attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, sm_xbuf(p), tid, &s_flag);
+                else attention_phase<D, G, MK_ATT_LPP>(p, l, n_att, p.att_chunk_shared, false, sm_xbuf(p), tid, &s_flag);
             } else {
-                attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, xbuf, tid, &s_flag);
+                attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, sm_xbuf(p), tid, &s_flag);
             }
-            ok = grid_barrier(p, ++bar_no * bar_arrivals, abort_flag, tid, prof_idx) && ok;
+            ok = grid_barrier(p, ++bar_no * bar_arrivals, abort_flag, tid, prof_idx, refill) && ok;
             if (!ok) break;
         }
-        ok = gemv_phase(p, s_ops, s_tab, ph, layer_op ? (ph & 3) : 4, ws, xsA, xsB, abort_flag, s_part, s_partial, cx, token,
-                        after_attention ? merge_chunks : 0, tid, prof_idx, &x_bar, x_parity, s_issued);
-        if (layer_op) ok = grid_barrier(p, ++bar_no * bar_arrivals, abort_flag, tid, prof_idx) && ok;
+        ok = gemv_phase(p, ph, layer_op ? (ph & 3) : 4, ws, abort_flag, s_part, s_partial, s_rope, cx, token, after_attention ? merge_chunks : 0, tid,
+                        prof_idx, &x_bar, x_parity, s_issued, full_bar);
+        if (layer_op) ok = grid_barrier(p, ++bar_no * bar_arrivals, abort_flag, tid, prof_idx, refill) && ok;
     }
     prof_stamp(p, tid, prof_idx);
     if (!ok || *abort_flag) {
@@ -993,7 +1062,7 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
         const unsigned issued = __shfl_sync(0xffffffffu, ws.next.count, 0);
         for (unsigned k = ws.consumed; k < issued; ++k) {
             const unsigned long long t1 = global_ns();
-            while (!mbar_try_wait(&ws.full_bar[ws.slot], ws.round & 1u))
+            while (!mbar_try_wait(&full_bar[warp * MK_MAX_SLOTS + ws.slot], ws.round & 1u))
                 if (global_ns() - t1 > p.spin_limit) break;
             if (++ws.slot == p.slots) { ws.slot = 0; ++ws.round; }
         }
@@ -1037,7 +1106,7 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
         }
         if (lane == 0) {
             if (bi == 0x7fffffff) bi = 0;
-            if (s_ops[p.nph - 1].flags() & PHF_REMAP) bi = p.vocab_ids[bi];   // pruned vocabulary: row index -> token id
+            if (sm_ops(p)[p.nph - 1].flags() & PHF_REMAP) bi = p.vocab_ids[bi];   // pruned vocabulary: row index -> token id
             int *nto = p.req->next_token_out;
             if (nto) *nto = bi;
             p.state->next_token = bi;

@@ -8,7 +8,10 @@ constexpr int MK_BAR_POLLERS = 1;                // warps whose lane 0 polls the
 constexpr int MK_ATT_LPP = 2;                    // lanes per cached position in the score phase (one CTA per GQA group)
 constexpr int MK_ATT_LPP_SPLIT = 2;              // ... when every query head has its own CTAs (16 positions per warp iteration)
 constexpr int MK_ATT_TILE = 32 / MK_ATT_LPP;     // positions per warp iteration (grouped mode)
-constexpr int MK_ATT_SPLIT_MAXC = 12;            // chunks per head when every query head has its own CTAs
+#ifndef MK_ATT_SPLIT_MAXC_VALUE
+#define MK_ATT_SPLIT_MAXC_VALUE 12
+#endif
+constexpr int MK_ATT_SPLIT_MAXC = MK_ATT_SPLIT_MAXC_VALUE;   // chunks per head when every query head has its own CTAs
 constexpr int MK_PARTIAL_SLOTS = 48;             // shared-memory scratch: partial row sums, 16 floats per slot
 constexpr int MK_PARTIAL_FLOATS = MK_PARTIAL_SLOTS * 16;   // (also the chunk statistics of the attention merge)
 constexpr int MK_TILE_COLS = 256;                // columns of a weight tile: one 16-byte piece per lane
@@ -102,7 +105,8 @@ struct MkParams {
     const uint2 *tiles;            // all tile lists, one contiguous block per CTA (copied to shared memory when the kernel starts)
     const int *cta_tab;            // [gridDim.x][cta_tab_ints]: per consumer warp {layer list offset in the CTA's block, tiles per
                                    // operator x4, output-layer list offset, output-layer tiles, 0}, then per operator (5) {combine
-                                   // offset, combine count}, then {first tile of the CTA's block, tiles in the block}
+                                   // offset in the CTA's block, combine count}, then {first tile of the CTA's block, tiles in the block, first combine
+                                   // entry of the CTA's block, entries in the block}
     const MkCombine *combines;
     int cta_tab_ints;
     int slots;                     // ring slots per consumer warp

@@ -131,9 +131,12 @@ struct StepSchedule {
     std::vector<MkCombine> combines;
     int cta_tab_ints = 0;
     int max_cta_tiles = 0;           // largest block (sizes the shared-memory copy)
+    int max_cta_combines = 0;
+    // bytes of shared memory the largest CTA block needs: tiles (8 bytes each, padded to 16), then combine entries (16 bytes each)
+    size_t smem_bytes() const { return (static_cast<size_t>(max_cta_tiles) * 8 + 15) / 16 * 16 + static_cast<size_t>(max_cta_combines) * 16; }
 };
 
-inline int cta_tab_ints_for(int nw) { return (nw * MK_WARP_TAB + 12 + 3) / 4 * 4; }
+inline int cta_tab_ints_for(int nw) { return (nw * MK_WARP_TAB + 14 + 3) / 4 * 4; }
 
 inline void assemble_schedule(StepSchedule *ss, int ncta, int nw) {
     ss->cta_tab_ints = cta_tab_ints_for(nw);
@@ -141,6 +144,7 @@ inline void assemble_schedule(StepSchedule *ss, int ncta, int nw) {
     ss->tiles.clear();
     ss->combines.clear();
     ss->max_cta_tiles = 0;
+    ss->max_cta_combines = 0;
     for (int c = 0; c < ncta; ++c) {
         int *ctab = &ss->cta_tab[static_cast<size_t>(c) * ss->cta_tab_ints];
         const size_t base = ss->tiles.size();
@@ -160,15 +164,19 @@ inline void assemble_schedule(StepSchedule *ss, int ncta, int nw) {
             tab[6] = static_cast<int>(l.size());
             ss->tiles.insert(ss->tiles.end(), l.begin(), l.end());
         }
+        const size_t cbase = ss->combines.size();
         for (int o = 0; o < 5; ++o) {
             int *ct = ctab + nw * MK_WARP_TAB + 2 * o;
             const auto &l = ss->ops[o].combines[c];
-            ct[0] = static_cast<int>(ss->combines.size());
+            ct[0] = static_cast<int>(ss->combines.size() - cbase);     // inside the CTA's block
             ct[1] = static_cast<int>(l.size());
             ss->combines.insert(ss->combines.end(), l.begin(), l.end());
         }
         ctab[nw * MK_WARP_TAB + 10] = static_cast<int>(base);
         ctab[nw * MK_WARP_TAB + 11] = static_cast<int>(ss->tiles.size() - base);
+        ctab[nw * MK_WARP_TAB + 12] = static_cast<int>(cbase);
+        ctab[nw * MK_WARP_TAB + 13] = static_cast<int>(ss->combines.size() - cbase);
+        ss->max_cta_combines = std::max(ss->max_cta_combines, static_cast<int>(ss->combines.size() - cbase));
         ss->max_cta_tiles = std::max(ss->max_cta_tiles, static_cast<int>(ss->tiles.size() - base));
     }
 }
