@@ -232,6 +232,7 @@ __device__ __forceinline__ void cursor_step(TileCursor &c, int n_layer, int n_la
 struct WarpStream {
     int list;                   // next tile to multiply: index into the CTA's tile lists
     TileCursor next;            // next tile to fetch (lane 0's view)
+    uint2 nd;                   // its descriptor, read ahead (valid while next.count < total)
     int slot;                   // slot of the next tile to multiply
     unsigned round;
     unsigned consumed;          // tiles multiplied so far
@@ -241,11 +242,17 @@ struct WarpStream {
 // Lane 0 only: fetch tile ws.next into ring slot `slot` (whose previous contents this warp has finished reading).
 __device__ __forceinline__ bool fetch_next_tile(const MkParams &p, WarpStream &ws, int slot, volatile int *abort_flag, volatile unsigned *s_issued,
                                                 unsigned long long *full_bar, int warp) {
+#ifdef EDGEFM_TRACE_OP
+    long long fc[6];
+    fc[0] = clock64();
+#define FSEG(i) fc[i] = clock64()
+#else
+#define FSEG(i) do {} while (0)
+#endif
     const int *tab = sm_tab(p) + warp * MK_WARP_TAB;
-    const int n_layer = tab[1] + tab[2] + tab[3] + tab[4];
-    if (ws.next.count >= static_cast<unsigned>(n_layer) * p.n_layers + tab[6]) return true;
     const bool lm = ws.next.layer >= p.n_layers;
-    const uint2 d = sm_tiles(p)[(lm ? tab[5] : tab[0]) + ws.next.i];
+    if (lm && ws.next.i >= tab[6]) return true;          // the whole step has been fetched
+    const uint2 d = ws.nd;
     // the operators of a layer are QKV, O, gate/up, down in this order; 4 = the output layer
     const int op = static_cast<int>((d.y >> 20) & 7u);
     const int opi = lm ? 4 * p.n_layers : 4 * ws.next.layer + op;
@@ -267,14 +274,27 @@ __device__ __forceinline__ bool fetch_next_tile(const MkParams &p, WarpStream &w
     unsigned long long *bar = &full_bar[warp * MK_MAX_SLOTS + slot];
     unsigned long long policy;   // weights are read once per step: first out of L2
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    FSEG(1);
     // the warp read the slot through the generic proxy: order those reads before the asynchronous write
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    FSEG(2);
     mbar_arrive_expect_tx(bar, bytes);
+    FSEG(3);
     if (op == 0) tma_load_box4(dst, map, x, u0 & ((p.d >> 1) - 1), 0, u0 >> p.half_shift, bar, policy);
     else if (op == 2) tma_load_box3(dst, map, x, u0, 0, bar, policy);
     else tma_load_box(dst, map, x, u0, bar, policy);
-    cursor_step(ws.next, n_layer, p.n_layers);
+    FSEG(4);
+    cursor_step(ws.next, tab[7], p.n_layers);
     s_issued[warp] = ws.next.count;     // read by the L2 prefetch warp
+    ws.nd = sm_tiles(p)[(ws.next.layer >= p.n_layers ? tab[5] : tab[0]) + ws.next.i];   // (one entry behind the lists is readable: the combines follow)
+#ifdef EDGEFM_TRACE_OP
+    FSEG(5);
+    if (p.prof && blockIdx.x == 0 && warp == 3 && opi == EDGEFM_TRACE_OP) {
+        unsigned long long *o = p.prof + static_cast<size_t>(gridDim.x) * p.prof_stride + MK_NW_MAX * 16 * 4;
+        for (int i = 0; i < 5; ++i) o[i] += static_cast<unsigned long long>(fc[i + 1] - fc[i]);
+        o[5] += 1;
+    }
+#endif
     return true;
 }
 
@@ -444,6 +464,12 @@ __device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkOp &P, 
     // a short operator (all its tiles are already in the ring) leaves the refills to the grid barrier that follows it, so that
     // nothing but the arithmetic sits on its critical path
     const bool defer = MK_DEFER_REFILL != 0 && n + ws.pending <= p.slots && P.kind != PH_LMHEAD;
+#ifdef MK_STAGGER
+    if (n > 2) {   // spread the warps' refill requests over time: they share one copy-engine port
+        const long long t0 = clock64();
+        while (clock64() - t0 < static_cast<long long>(warp) * MK_STAGGER) {}
+    }
+#endif
     const uint2 *list = sm_tiles(p) + ws.list;
     uint2 d = n > 0 ? list[0] : make_uint2(0u, 0u);
     for (int t = 0; t < n; ++t) {
@@ -988,7 +1014,8 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
     WarpStream ws;
     {
         const int *tab = sm_tab(p) + warp * MK_WARP_TAB;
-        ws.next = TileCursor{tab[1] + tab[2] + tab[3] + tab[4] == 0 ? p.n_layers : 0, 0, 0u};
+        ws.next = TileCursor{tab[7] == 0 ? p.n_layers : 0, 0, 0u};
+        ws.nd = sm_tiles(p)[(tab[7] == 0 ? tab[5] : tab[0])];
         ws.list = tab[0];
     }
     ws.slot = 0; ws.round = 0; ws.consumed = 0; ws.pending = 0;

@@ -104,7 +104,7 @@ struct MkParams {
     const unsigned char *maps;     // CUtensorMap [(4 * n_layers + 1) * MK_MAX_VARIANTS], 128 bytes each, index (4 l + op) * 4 + variant
     const uint2 *tiles;            // all tile lists, one contiguous block per CTA (copied to shared memory when the kernel starts)
     const int *cta_tab;            // [gridDim.x][cta_tab_ints]: per consumer warp {layer list offset in the CTA's block, tiles per
-                                   // operator x4, output-layer list offset, output-layer tiles, 0}, then per operator (5) {combine
+                                   // operator x4, output-layer list offset, output-layer tiles, tiles per layer}, then per operator (5) {combine
                                    // offset in the CTA's block, combine count}, then {first tile of the CTA's block, tiles in the block, first combine
                                    // entry of the CTA's block, entries in the block}
     const MkCombine *combines;

@@ -154,6 +154,7 @@ inline void assemble_schedule(StepSchedule *ss, int ncta, int nw) {
             for (int o = 0; o < 4; ++o) {
                 const auto &l = ss->ops[o].tiles[c][w];
                 tab[1 + o] = static_cast<int>(l.size());
+                tab[7] += static_cast<int>(l.size());          // tiles per layer
                 ss->tiles.insert(ss->tiles.end(), l.begin(), l.end());
             }
         }
