@@ -27,9 +27,29 @@ import numpy as np
 
 from edgefm_synth import CONFIGS, GLOBAL_SEED, first_token, make_kv, make_weights
 
-# DRAM traffic of one launch of the step kernel (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture,
-# see profiles/decode_megakernel_qwen2.5-1.5b_ctx2048.md); only the captured configuration has a value.
-NCU_TRAFFIC_BYTES = {"qwen2.5-1.5b": 3.146461e9 + 3.875e6}
+# DRAM traffic of one launch of the step kernel: dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture of
+# that kernel, per configuration, with the profile summary (and the source revision it names) the figure comes from.
+# Only captured configurations have a value; a figure is only as current as its summary says.
+NCU_TRAFFIC = {"qwen2.5-1.5b": {"bytes": None, "source": "profiles/decode_megakernel_qwen2.5-1.5b_ctx2048.md"}}
+
+
+def ncu_traffic(name):
+    """(bytes or None, where the figure comes from): parsed from the profile summary, which states read and write bytes."""
+    import re
+    ent = NCU_TRAFFIC.get(name)
+    if not ent:
+        return None, None
+    path = ROOT / ent["source"]
+    try:
+        text = path.read_text()
+        rd = re.search(r"dram__bytes_read\.sum\s*\|\s*([0-9.]+)\s*GB", text)
+        wr = re.search(r"dram__bytes_write\.sum\s*\|\s*([0-9.]+)\s*MB", text)
+        rev = re.search(r"source revision:\s*`?([0-9a-f]{7,40})", text)
+        if rd and wr:
+            return float(rd.group(1)) * 1e9 + float(wr.group(1)) * 1e6, f"{ent['source']}" + (f" (revision {rev.group(1)})" if rev else "")
+    except OSError:
+        pass
+    return None, None
 
 METRIC = "batch1_decode_ms_per_token"
 UNIT = "ms/token"
@@ -124,10 +144,34 @@ def run_reference(args, cfg, rank):
     line = {"impl": "reference", "metric": METRIC, "value": ms, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
             "dtype": "f64 accumulate over bf16 weights", "data": "synthetic",
-            "config": {"workload": workload_name(cfg)},
+            "config": config_block(cfg, workload_name(cfg), 1),
             "cpu_baseline": {"value": ms, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": ms, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
+
+
+def config_block(cfg, workload, world, pruned_bytes=0):
+    """The `config` object of the JSON line (the same keys for both arms)."""
+    return {"workload": workload, "replicas": world,
+            "l2": (f"working set {(cfg.mean_step_bytes() - pruned_bytes) / 1e9:.2f} GB per step exceeds the 126 MB L2; no flush"
+                   if cfg.mean_step_bytes() > 2.5e8 else "working set fits L2: NOT an HBM measurement"),
+            "seed": GLOBAL_SEED}
+
+
+def max_over_ranks(times, world):
+    """Element-wise maximum over the ranks of a 1-D float64 tensor of this rank's timings (the slowest replica decides).
+    N = 1: the tensor itself."""
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    return times
+
+
+def per_token_stats(seq_ms, steps, world):
+    """Median and minimum ms per token over the timed sequences (each entry: max over ranks of one sequence's time);
+    with N replicas N * steps tokens leave the job per sequence."""
+    per = sorted(float(t) / (steps * world) for t in seq_ms)
+    return statistics.median(per), per[0]
 
 
 def workload_name(cfg):
@@ -144,6 +188,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU-oracle timing leg")
     ap.add_argument("--cpu-steps", type=int, default=3)
+    ap.add_argument("--sequences", type=int, default=10,
+                    help="timed repetitions of the --steps-long greedy sequence (each timed on its own; value = median)")
+    ap.add_argument("--warmup-sequences", type=int, default=3, help="untimed sequences before the timed ones (besides --warmup steps)")
     ap.add_argument("--vocab-subset", type=int, default=0,
                     help="prune the output layer to this many evenly spaced token ids (0 = full vocabulary, the headline workload)")
     ap.add_argument("--phase-timeline", action="store_true",
@@ -210,22 +257,29 @@ def main():
             torch.cuda.synchronize()
 
     # ---- device-resident timing (inputs in HBM; weights 3 GB >> L2, so no flush between steps) ---------
+    # --warmup untimed steps, then --warmup-sequences untimed sequences, then --sequences sequences of exactly --steps
+    # steps, each bracketed by its own pair of CUDA events on the launching stream (the cache is reset between sequences,
+    # outside the events).  Reported: median (value) and minimum over the sequences.
     if warmup:
         free_run(warmup)
+    for _ in range(max(args.warmup_sequences, 0)):
+        free_run(steps)
     barrier()
     sampler = ClockSampler(local_rank)
     sampler.start()
-    ctx.prefill_kv(kd, vd)
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    e0.record()
-    edgefm_decode_step(handle, tok0, pos0, stream, None, None)
-    for _ in range(steps - 1):
-        edgefm_decode_step(handle, -1, -1, stream, None, None)
-    e1.record()
-    barrier()
-    dev_ms = e0.elapsed_time(e1)
+    n_seq = max(args.sequences, 1)
+    seq_ms = []
+    for _ in range(n_seq):
+        ctx.prefill_kv(kd, vd)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        edgefm_decode_step(handle, tok0, pos0, stream, None, None)
+        for _ in range(steps - 1):
+            edgefm_decode_step(handle, -1, -1, stream, None, None)
+        e1.record()
+        barrier()
+        seq_ms.append(e0.elapsed_time(e1))
 
     # ---- end to end through the C ABI with host buffers: the token crosses PCIe both ways every step ----
     host_tok = torch.zeros(1, dtype=torch.int32).pin_memory()
@@ -241,18 +295,18 @@ def main():
     e2e_ms = (time.perf_counter() - t0) * 1e3
     clocks = sampler.stop()
 
-    times = torch.tensor([dev_ms, e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    dev_ms, e2e_ms = float(times[0]), float(times[1])
+    times = max_over_ranks(torch.tensor(seq_ms + [e2e_ms], dtype=torch.float64, device=dev), world)
+    seq_ms, e2e_ms = [float(t) for t in times[:-1]], float(times[-1])
     launches = ctx.launches_per_step
 
     if rank == 0:
         tokens = steps * world
-        ms_per_token = dev_ms / tokens
+        ms_per_token, ms_per_token_min = per_token_stats(seq_ms, steps, world)
+        dev_ms = ms_per_token * tokens                                   # median sequence time
         bytes_per_step = float(np.mean([cfg.step_bytes(cfg.cache_len + i) for i in range(steps)])) - pruned_bytes
         gbs = bytes_per_step / (dev_ms / steps * 1e-3) / 1e9          # per GPU
         peak, peak_src = measured_peak()
+        traffic, traffic_src = (None, None) if n_sub else ncu_traffic(cfg.name)
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
             cores = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
@@ -264,15 +318,14 @@ def main():
             "metric": METRIC, "value": ms_per_token, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
             "ms_per_step": dev_ms / steps, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16 weights/KV, fp32 accumulate", "data": "synthetic",
-            "config": {"workload": workload, "replicas": world, "l2": (f"working set {(cfg.mean_step_bytes() - pruned_bytes) / 1e9:.2f} GB per step exceeds the 126 MB L2; no flush"
-                              if cfg.mean_step_bytes() > 2.5e8 else "working set fits L2: NOT an HBM measurement"),
-                       "seed": GLOBAL_SEED},
+            "config": config_block(cfg, workload, world, pruned_bytes),
+            "timed_sequences": n_seq, "ms_per_token_min": ms_per_token_min,
             "tokens_per_s": tokens / (dev_ms * 1e-3),
             "roofline": {"bound": "hbm", "kernel": f"decode_megakernel: the whole decode step ({launches} kernel launch per token, one CUDA graph node)",
                          "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak, "peak_source": peak_src,
-                         "bytes_per_launch": bytes_per_step, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS, "traffic": None if n_sub else NCU_TRAFFIC_BYTES.get(cfg.name)},
+                         "bytes_per_launch": bytes_per_step, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS, "traffic": traffic, "traffic_source": traffic_src},
             "e2e": {"value": e2e_ms / tokens, "unit": UNIT, "h2d_bytes_per_step": 24, "d2h_bytes_per_step": 4},
-            "gpu_launches": launches * steps,
+            "gpu_launches": launches * steps * n_seq,
             "clocks": clocks,
             "cpu_baseline": cpu,
         }

@@ -135,7 +135,8 @@ edgefm_status edgefm_export_kv(edgefm_ctx *ctx, void *k_out, void *v_out, void *
 edgefm_status edgefm_get_launches_per_step(const edgefm_ctx *ctx, int32_t *n_launches_host);
 
 /* Synchronise `stream`, then report whether a bounded device-side wait of the persistent step kernel
- * expired (EDGEFM_ERR_TIMEOUT; the context is then unusable and must be destroyed) or all is well. */
+ * expired or one of its self-checks failed (EDGEFM_ERR_TIMEOUT; the context is then unusable and must be destroyed)
+ * or all is well.  ctx == NULL: the status left by the last edgefm_decode_step_static on the current device. */
 edgefm_status edgefm_sync_status(edgefm_ctx *ctx, void *stream);
 
 /*
@@ -171,41 +172,65 @@ edgefm_status edgefm_append_kv(edgefm_ctx *ctx, const void *k, const void *v, in
  */
 edgefm_status edgefm_set_vocab_subset(edgefm_ctx *ctx, const int32_t *token_ids, int32_t n, void *stream);
 
-/* Diagnostics.  When the environment variable EDGEFM_PROFILE=1 was set at edgefm_create, every CTA of
- * the persistent step kernel records device timestamps (ns) at fixed points of the last step: start,
- * then per layer {QKV: staged, done, released; attention: done, released; O, gate/up, down: staged,
- * done, released}, then lm_head staged, done.  Synchronises the device and copies the
- * [n_ctas][stride] table to out_host (capacity in elements).  n_ctas = 0 when profiling is off;
- * out_host may be NULL to query the sizes. */
+/* Diagnostics.  When the environment variable EDGEFM_PROFILE=1 was set at edgefm_create (the only environment
+ * variable the library reads), every CTA of the persistent step kernel records device timestamps (ns) at fixed points
+ * of the last step: start, then per layer {QKV: staged, done, released; attention: done, released; O, gate/up, down:
+ * staged, done, released}, then lm_head staged, done.  Synchronises the device and copies the [n_ctas][stride] table to
+ * out_host (capacity in elements).  n_ctas = 0 when profiling is off; out_host may be NULL to query the sizes. */
 edgefm_status edgefm_debug_profile(edgefm_ctx *ctx, uint64_t *out_host, int64_t capacity, int32_t *n_ctas, int32_t *stride);
+
+/* Launch geometry of the context's step kernel: out8 = {CTAs, consumer warps per CTA, ring slots per warp, bytes per slot,
+ * dynamic shared memory, tiles of the busiest CTA, shared-memory bytes reserved for the tile lists, 1 = long-context
+ * build of the kernel}.  Host only. */
+edgefm_status edgefm_debug_plan(const edgefm_ctx *ctx, int32_t *out8);
+
+/* Every device-side wait of the step kernel (tile arrival, grid barrier) gives up after a bound (1 s by default), records
+ * EDGEFM_ERR_TIMEOUT in the device state and lets the kernel return; edgefm_sync_status reports it.  This call changes
+ * the bound (limit_ns >= 1000) of the steps enqueued afterwards and, for testing that path without any fault, can make the
+ * grid barrier expect one arrival more than there are CTAs (extra_barrier_arrivals = 1; 0 in production), so that the
+ * first barrier of the next step runs into the bound.  Synchronises the device and re-records the step graph. */
+edgefm_status edgefm_debug_set_wait_limit(edgefm_ctx *ctx, uint32_t limit_ns, int32_t extra_barrier_arrivals);
+
+/* Host-only check of the planner: the tile schedule of one weight-streaming operator (kind: 0 QKV pairs, 1 residual rows,
+ * 2 gate/up pairs, 3 output-layer rows; units rows or pairs; K columns; head_half = head_dim / 2 for kind 0) for n_ctas CTAs
+ * of n_warps consumer warps whose ring slots hold slot_rows rows.  tiles_out receives one 64-bit descriptor per tile, CTA by
+ * CTA and warp by warp (tiles_per_warp [n_ctas * n_warps] counts them); combines_out four 32-bit words per entry
+ * (combines_per_cta [n_ctas]); variant_rows [4] the box heights of the operator's tensor maps; *n_tiles / *n_combines the
+ * totals (call once with NULL outputs to size the buffers).  Needs no GPU.  BAD_SHAPE when the operator does not fit. */
+edgefm_status edgefm_debug_plan_operator(int32_t kind, int32_t units, int32_t K, int32_t head_half, int32_t op_index, int32_t n_ctas,
+                                         int32_t n_warps, int32_t slot_rows, uint64_t *tiles_out, int64_t tiles_cap,
+                                         int32_t *tiles_per_warp, uint32_t *combines_out, int64_t combines_cap,
+                                         int32_t *combines_per_cta, int32_t *variant_rows, int64_t *n_tiles, int64_t *n_combines);
 
 /*
  * edgefm_decode_step_static -- one decode step that allocates nothing (the paper has no counterpart; this
  * entry point exists for callers that cannot allocate device memory).
  *
- * Who needs it: code that runs inside another framework's allocation-free region (a fixed memory plan it is
- * recording or replaying), processes whose device memory is handed out entirely by a pool they do not own,
- * and latency-critical threads that cannot take the implicit device synchronisation of cudaMalloc / cudaFree.
+ * Who needs it: code that runs inside another framework's allocation-free region (a phase in which that framework has
+ * frozen its memory plan), processes whose device memory is handed out entirely by a pool they do not own, and
+ * latency-critical threads that cannot take the implicit device synchronisation of cudaMalloc / cudaFree.
  * edgefm_create allocates a KV cache and work buffers; this call does neither.  It is the same persistent step
  * kernel as edgefm_decode_step, with all its work buffers (residual stream, queries, attention partials, MLP
- * activations, schedule, counters, device state) carved out of a fixed 2 MiB array that is part of the loaded
- * library image on every GPU, and with the KV cache owned by the caller:
+ * activations, operator table, tile schedule, tensor maps, counters, device state) carved out of a fixed 4 MiB array
+ * that is part of the loaded library image on every GPU, and with the KV cache owned by the caller:
  *   shape, weights   as for edgefm_create (read during the call; device buffers borrowed until the step has run);
- *                    at most 96 layers, and the work buffers of the shape must fit the 2 MiB, else
+ *                    at most 96 layers, and the work buffers of the shape must fit the 4 MiB, else
  *                    EDGEFM_ERR_BAD_SHAPE with a message that states the limit.
  *   k_cache, v_cache DEVICE bf16 [n_layers][n_kv_heads][max_context][head_dim] (the layout edgefm_export_kv
  *                    writes), 16-byte aligned; slots 0 .. cur_len-1 are read, slot cur_len is written.
  *   cur_len          filled slots before the step (the caller keeps the count; 0 <= cur_len < max_context).
  *   token_id, position  both explicit (>= 0); nothing is remembered between calls.
  *   logits_out       DEVICE fp32 [vocab] or NULL;  next_token_out  DEVICE int32 [1] or NULL.
- * The work is enqueued on `stream` (small stream-ordered copies and one memset of the counters, then the
+ * The work is enqueued on `stream` (stream-ordered copies of the schedule and one memset of the counters, then the
  * kernel) and the call returns without synchronising.  It calls no cudaMalloc, cudaFree or other allocating
  * routine.  The first call on a device also looks up the device address of the scratch array (once per device,
- * with that device current); make that first call outside any stream capture.
+ * with that device current).  The copies read host memory of the call itself, so `stream` must NOT be in capture
+ * mode: a capturing stream is refused with EDGEFM_ERR_INVALID_ARG before anything is enqueued.
  * All calls on a device share the one scratch array, which keeps the previous call's contents: the call
  * clears what must start at zero itself, but two calls that overlap on the GPU (different streams, different
- * threads, or a context created by edgefm_create is NOT affected -- it has its own buffers) race on it and
- * give wrong results; order them on one stream or with events.
+ * threads; a context created by edgefm_create is NOT affected -- it has its own buffers) race on it and
+ * give wrong results; order them on one stream or with events.  A bounded wait that expired inside such a step is
+ * reported by edgefm_sync_status(NULL, stream).
  * Errors: INVALID_ARG, BAD_SHAPE, CONTEXT_FULL (cur_len == max_context), CUDA; message via edgefm_last_error(NULL).
  */
 edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, const edgefm_weights *weights, void *k_cache, void *v_cache,

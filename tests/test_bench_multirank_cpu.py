@@ -20,15 +20,19 @@ def _free_port():
 
 
 def _worker(rank, world, port, out):
+    """One replica: its own per-sequence timings go through bench.py's reduction (the code the benchmark runs)."""
+    sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+    import bench
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
     dist.init_process_group("gloo", rank=rank, world_size=world)
     dist.barrier()
-    local_ms = torch.tensor([10.0 + 5.0 * rank, 20.0 - 3.0 * rank], dtype=torch.float64)   # (device ms, e2e ms) of this replica
-    dist.all_reduce(local_ms, op=dist.ReduceOp.MAX)
     steps = 7
-    tokens = steps * world
+    # three timed sequences and the end-to-end time of this replica; rank 1 is slower on the device, rank 0 end to end
+    local = torch.tensor([10.0 + 5.0 * rank, 12.0 + 5.0 * rank, 11.0 + 5.0 * rank, 20.0 - 3.0 * rank], dtype=torch.float64)
+    red = bench.max_over_ranks(local, world)
     if rank == 0:
-        out.put((float(local_ms[0]), float(local_ms[1]), local_ms[0].item() / tokens))
+        med, mn = bench.per_token_stats([float(t) for t in red[:-1]], steps, world)
+        out.put(([float(t) for t in red], med, mn))
     dist.barrier()
     dist.destroy_process_group()
 
@@ -41,11 +45,20 @@ def test_max_over_ranks_and_aggregate_value():
     for p in procs:
         p.start()
     for p in procs:
-        p.join(60)
+        p.join(120)
         assert p.exitcode == 0
-    dev_ms, e2e_ms, per_token = q.get(timeout=10)
-    assert dev_ms == 15.0 and e2e_ms == 20.0            # slowest replica decides
-    assert per_token == pytest.approx(15.0 / 14)        # aggregate ms per token over both replicas
+    red, med, mn = q.get(timeout=10)
+    assert red == [15.0, 17.0, 16.0, 20.0]               # slowest replica decides, entry by entry
+    assert med == pytest.approx(16.0 / 14)               # median sequence; 2 replicas x 7 steps = 14 tokens per sequence
+    assert mn == pytest.approx(15.0 / 14)
+
+
+def test_single_rank_reduction_is_the_identity():
+    sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+    import bench
+    t = torch.tensor([3.0, 1.0, 2.0], dtype=torch.float64)
+    assert bench.max_over_ranks(t, 1) is t
+    assert bench.per_token_stats([3.0, 1.0, 2.0], 2, 1) == (1.0, 0.5)
 
 
 def test_reference_arm_line_on_tiny_config():
@@ -57,4 +70,5 @@ def test_reference_arm_line_on_tiny_config():
     line = json.loads(out.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["unit"] == "ms/token" and line["higher_is_better"] is False
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
+    assert set(line["config"]) == {"workload", "replicas", "l2", "seed"}          # the same keys as the CUDA arm's line
     assert line["value"] > 0
