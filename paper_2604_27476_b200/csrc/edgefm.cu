@@ -111,7 +111,7 @@ inline const char *plan_step(const edgefm_shape &sh, int max_context, int num_sm
     pl->grid = num_sms;
     pl->max_chunks = pl->grid / nkv > 0 ? pl->grid / nkv : 1;
     pl->n_ops = 4 * sh.n_layers + 1;
-    const int NW = pl->nw, ATT_MW = (NW + 1) / 2;
+    const int NW = pl->nw, ATT_MW = NW;   // every warp has an entry in the attention merge area
     int max_k = H;
     if (nq * d > max_k) max_k = nq * d;
     if (F > max_k) max_k = F;

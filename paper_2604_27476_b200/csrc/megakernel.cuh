@@ -39,12 +39,14 @@ namespace MK_NS {
 constexpr int MK_NW = MK_NW_VALUE;               // consumer warps per CTA
 constexpr int MK_NT = MK_NW * 32;                // consumer threads
 constexpr int MK_THREADS = MK_NT + 32;           // + the L2 prefetch warp
-constexpr int MK_ATT_MW = (MK_NW + 1) / 2;       // warps whose partials fit the merge area at once
 
 // 1: one-head-per-CTA attention leaves the merge of its chunks to the O projection's prologue (every CTA merges);
 // 0: the last CTA of every head merges (atomic ticket) and the O projection stages the finished vector
 #ifndef MK_SPLIT_DEFER
 #define MK_SPLIT_DEFER 1
+#endif
+#ifndef MK_ATT_HOIST
+#define MK_ATT_HOIST 0
 #endif
 #ifndef MK_MERGE_NOUT
 #define MK_MERGE_NOUT 1
@@ -314,6 +316,18 @@ __device__ __forceinline__ bool refill_pending(const MkParams &p, WarpStream &ws
     return ok;
 }
 
+// Attention chunking shared by the attention phase and by the consumer of its partial results.
+__device__ __forceinline__ void att_chunking(const MkParams &p, int n, int hg, int min_chunk, int tile, int ncta, int &nch, int &chunk_len) {
+    const int groups = p.nq / hg;
+    nch = (n + min_chunk - 1) / min_chunk;
+    nch = min(nch, min(ncta / groups, p.max_chunks));
+    if (hg == 1) nch = min(nch, MK_ATT_SPLIT_MAXC);
+    nch = max(nch, 1);
+    chunk_len = (n + nch - 1) / nch;
+    chunk_len = (chunk_len + tile - 1) / tile * tile;
+    nch = (n + chunk_len - 1) / chunk_len;
+}
+
 // ---- the L2 prefetch warp ------------------------------------------------------------------------------------
 // The ring of a consumer warp holds only a few tiles, so HBM would idle whenever the consumers stall (grid barriers,
 // attention) and every refill would pay the full HBM latency.  One more warp therefore runs ahead of the rings: lanes w
@@ -326,6 +340,36 @@ __device__ __forceinline__ void prefetch_tiles(const MkParams &p, volatile int *
     const int *s_tab = sm_tab(p);
     const uint2 *s_tiles = sm_tiles(p);
     const int w = lane & 15, half = lane >> 4;
+    if (p.pf_tiles > 0 && w >= MK_NW) {
+        // The spare lanes pull the K and V rows this CTA's attention will read into L2, a layer ahead: as soon as warp 0's
+        // ring has started on the tiles of layer l, the chunk of layer l (one-head-per-CTA chunking only).
+        const int n_spare = 2 * (16 - MK_NW), me = (w - MK_NW) * 2 + half;
+        const int n = p.state->cur_len + 1;
+        if (n > p.att_split_max_n || n < 1 || n > p.max_context) return;
+        int nch, chunk_len;
+        att_chunking(p, n, 1, p.att_chunk_split, 32 / MK_ATT_LPP_SPLIT, static_cast<int>(gridDim.x), nch, chunk_len);
+        const int cta = static_cast<int>(blockIdx.x);
+        if (cta >= nch * p.nq) return;
+        const int qh = cta / nch, c = cta - qh * nch, g = qh / (p.nq / p.nkv);
+        const int t0 = c * chunk_len, t1 = min(n, t0 + chunk_len);
+        const int n_lines = ((t1 - t0) * p.d * 2 + 127) / 128;
+        const int n_layer0 = s_tab[7];
+        for (int layer = 0; layer < p.n_layers; ++layer) {
+            unsigned spins = 0;
+            while (s_issued[0] < static_cast<unsigned>(layer) * n_layer0) {
+                if (*abort_flag || ++spins > (1u << 22)) return;
+                __nanosleep(200);
+            }
+            const size_t off = ((static_cast<size_t>(layer) * p.nkv + g) * p.max_context + t0) * p.d * 2;
+            const unsigned char *kb = reinterpret_cast<const unsigned char *>(p.k_cache) + off;
+            const unsigned char *vb = reinterpret_cast<const unsigned char *>(p.v_cache) + off;
+            for (int i = me; i < n_lines; i += n_spare) {
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(kb + static_cast<size_t>(i) * 128));
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(vb + static_cast<size_t>(i) * 128));
+            }
+        }
+        return;
+    }
     if (p.pf_tiles <= 0 || w >= MK_NW) return;
     const int *tab = s_tab + w * MK_WARP_TAB;
     const int n_layer = tab[1] + tab[2] + tab[3] + tab[4], n_lm = tab[6];
@@ -531,18 +575,6 @@ __device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkOp &P, 
     return true;
 }
 
-// Attention chunking shared by the attention phase and by the consumer of its partial results.
-__device__ __forceinline__ void att_chunking(const MkParams &p, int n, int hg, int min_chunk, int tile, int ncta, int &nch, int &chunk_len) {
-    const int groups = p.nq / hg;
-    nch = (n + min_chunk - 1) / min_chunk;
-    nch = min(nch, min(ncta / groups, p.max_chunks));
-    if (hg == 1) nch = min(nch, MK_ATT_SPLIT_MAXC);
-    nch = max(nch, 1);
-    chunk_len = (n + nch - 1) / nch;
-    chunk_len = (chunk_len + tile - 1) / tile * tile;
-    nch = (n + chunk_len - 1) / chunk_len;
-}
-
 // One weight-streaming operator: prologue (stage the activation vector, RMSNorm folded in: x*w is staged
 // and the scalar rsqrt(mean x^2 + eps) is applied to the dot products), then this warp's tiles, then the units
 // whose columns were shared between warps.
@@ -567,51 +599,44 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_
         const int d4 = p.d >> 2;
         float *sm_m = s_partial;                 // [nq][nch] chunk maxima
         float *sm_l = s_partial + p.nq * nch;    // [nq][nch] chunk denominators
-        // every thread merges up to two 16-byte pieces of the vector per round; the partial vectors of both are requested
-        // before anything is waited for, so the whole prologue costs one trip to L2
-        constexpr int NOUT = MK_MERGE_NOUT;
-        float4 ob[NOUT][MK_ATT_SPLIT_MAXC];
-        auto load_partials = [&](int o4, float4 (&dst)[MK_ATT_SPLIT_MAXC]) {
+        // Thread t merges piece t of the vector (16 bytes: 4 dims of one head): all its chunk partials are requested at once,
+        // before the statistics are waited for.  (Spreading the left-over pieces of a vector longer than the CTA over all
+        // threads was measured slower: the extra live registers spill.)
+        float4 ob[MK_ATT_SPLIT_MAXC];
+        auto load_partials = [&](int o4) {
             const int h = o4 / d4, j4 = o4 - h * d4;
             const float4 *po = reinterpret_cast<const float4 *>(p.part_o + static_cast<size_t>(h) * p.max_chunks * p.d) + j4;
 #pragma unroll
             for (int c = 0; c < MK_ATT_SPLIT_MAXC; ++c)
-                if (c < nch) dst[c] = __ldcg(po + static_cast<size_t>(c) * d4);
+                if (c < nch) ob[c] = __ldcg(po + static_cast<size_t>(c) * d4);
         };
-#pragma unroll
-        for (int u = 0; u < NOUT; ++u)
-            if (tid + u * MK_NT < n4) load_partials(tid + u * MK_NT, ob[u]);
+        if (tid < n4) load_partials(tid);
         for (int i = tid; i < p.nq * nch; i += MK_NT) {
             const int h = i / nch, c = i - h * nch;
             sm_m[i] = __ldcg(p.part_m + h * p.max_chunks + c);
             sm_l[i] = __ldcg(p.part_l + h * p.max_chunks + c);
         }
         cta_sync();
-        for (int base = tid; base < n4; base += NOUT * MK_NT) {
+        for (int o4 = tid; o4 < n4; o4 += MK_NT) {
+            if (o4 != tid) load_partials(o4);
+            const int h = o4 / d4;
+            const float *hm = sm_m + h * nch, *hl = sm_l + h * nch;
+            float mm = -INFINITY;
+            for (int c = 0; c < nch; ++c) mm = fmaxf(mm, hm[c]);
+            float ll = 0.f;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-            for (int u = 0; u < NOUT; ++u) {
-                const int o4 = base + u * MK_NT;
-                if (o4 >= n4) break;
-                if (base != tid) load_partials(o4, ob[u]);
-                const int h = o4 / d4;
-                const float *hm = sm_m + h * nch, *hl = sm_l + h * nch;
-                float mm = -INFINITY;
-                for (int c = 0; c < nch; ++c) mm = fmaxf(mm, hm[c]);
-                float ll = 0.f;
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                for (int c = 0; c < MK_ATT_SPLIT_MAXC; ++c) {
-                    if (c < nch) {
-                        const float e = __expf(hm[c] - mm);
-                        ll = fmaf(hl[c], e, ll);
-                        acc.x = fmaf(ob[u][c].x, e, acc.x); acc.y = fmaf(ob[u][c].y, e, acc.y);
-                        acc.z = fmaf(ob[u][c].z, e, acc.z); acc.w = fmaf(ob[u][c].w, e, acc.w);
-                    }
+            for (int c = 0; c < MK_ATT_SPLIT_MAXC; ++c) {
+                if (c < nch) {
+                    const float e = __expf(hm[c] - mm);
+                    ll = fmaf(hl[c], e, ll);
+                    acc.x = fmaf(ob[c].x, e, acc.x); acc.y = fmaf(ob[c].y, e, acc.y);
+                    acc.z = fmaf(ob[c].z, e, acc.z); acc.w = fmaf(ob[c].w, e, acc.w);
                 }
-                const float inv = 1.f / ll;
-                acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-                if (o4 & 1) xsB[o4 >> 1] = acc; else xsA[o4 >> 1] = acc;
             }
+            const float inv = 1.f / ll;
+            acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
+            if (o4 & 1) xsB[o4 >> 1] = acc; else xsA[o4 >> 1] = acc;
         }
     } else if (P.flags() & PHF_X_BULK) {
         // the vector is already in the split layout and needs no transform: two bulk copies, every thread waits for them
@@ -738,7 +763,7 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
                                                 unsigned char *xbuf, int tid, int *s_flag) {
     constexpr int TILE = 32 / LPP;   // positions per warp iteration
     constexpr int DV = D / 32, CPR = D / 8, CPL = CPR / LPP;
-    constexpr int MW = MK_ATT_MW;
+    constexpr int MW = MK_NW;                            // every warp publishes its partial: one sync, then one pass
     const int lane = tid & 31, warp = tid >> 5;
     const int cta = blockIdx.x, ncta = gridDim.x;
     const int G = p.nq / p.nkv;
@@ -759,32 +784,22 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
     float *cm = mg_o + MW * HG * D;                             // [HG][max_chunks] chunk maxima
     float *cl = cm + HG * p.max_chunks;                         // [HG][max_chunks] chunk denominators
 
-    for (int i = tid; i < HG * D; i += MK_NT) qs[i] = __ldcg(p.q + static_cast<size_t>(qh0) * D + i) * p.scale;
-    cta_sync();
-
     const size_t head_off = (static_cast<size_t>(layer) * p.nkv + g) * p.max_context * D;
     const uint16_t *kg = p.k_cache + head_off;
     const uint16_t *vg = p.v_cache + head_off;
     float *pw = ps + warp * (HG * TILE);
     const int pi = lane / LPP, part = lane % LPP;
 
-    float m[HG], l[HG], o[HG][DV];
-#pragma unroll
-    for (int h = 0; h < HG; ++h) {
-        m[h] = -INFINITY; l[h] = 0.f;
-#pragma unroll
-        for (int e = 0; e < DV; ++e) o[h][e] = 0.f;
-    }
-
-    for (int tt = t0 + warp * TILE; tt < t1; tt += MK_NW * TILE) {
+    // K and V rows of one warp iteration: K pieces of this lane's position, raw bf16 pairs of V (converted when used to keep
+    // the register footprint small)
+    uint4 kk[CPL];
+    uint32_t vraw[TILE][DV / 2];
+    auto load_kv = [&](int tt) {
         const bool pvalid = tt + pi < t1;
-        uint4 kk[CPL];
 #pragma unroll
         for (int j = 0; j < CPL; ++j)
             kk[j] = pvalid ? __ldcg(reinterpret_cast<const uint4 *>(kg + static_cast<size_t>(tt + pi) * D) + j * LPP + part)
                            : make_uint4(0, 0, 0, 0);
-        // V rows of the tile, raw bf16 pairs (converted when used to keep the register footprint small)
-        uint32_t vraw[TILE][DV / 2];
 #pragma unroll
         for (int x = 0; x < TILE; ++x) {
             const int t = tt + x;
@@ -796,6 +811,29 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
                 vraw[x][0] = t < t1 ? __ldcg(reinterpret_cast<const unsigned *>(vp)) : 0u;
             }
         }
+    };
+    // the cache rows do not depend on this layer's queries (except the row appended by this step, which the grid barrier
+    // has published): request the first iteration's rows before waiting for the queries
+    int tt = t0 + warp * TILE;
+#if MK_ATT_HOIST
+    if (tt < t1) load_kv(tt);
+#endif
+    for (int i = tid; i < HG * D; i += MK_NT) qs[i] = __ldcg(p.q + static_cast<size_t>(qh0) * D + i) * p.scale;
+    cta_sync();
+
+    float m[HG], l[HG], o[HG][DV];
+#pragma unroll
+    for (int h = 0; h < HG; ++h) {
+        m[h] = -INFINITY; l[h] = 0.f;
+#pragma unroll
+        for (int e = 0; e < DV; ++e) o[h][e] = 0.f;
+    }
+
+    while (tt < t1) {
+        const bool pvalid = tt + pi < t1;
+#if !MK_ATT_HOIST
+        load_kv(tt);
+#endif
         float s[HG];
 #pragma unroll
         for (int h = 0; h < HG; ++h) s[h] = 0.f;
@@ -848,44 +886,22 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
             }
         }
         __syncwarp();
+        tt += MK_NW * TILE;
+#if MK_ATT_HOIST
+        if (tt < t1) load_kv(tt);
+#endif
     }
 
-    // merge the warps of the CTA in two passes through a merge area of MW entries (idle warps carry
-    // m = -inf and weigh 0): upper warps publish, lower warps fold them in, then publish themselves.
+    // merge the warps of the CTA: every warp publishes (m, l, o) (idle warps carry m = -inf and weigh 0), one sync, then
+    // every output element is merged over the warps in index order.
     float lt[HG];
 #pragma unroll
     for (int h = 0; h < HG; ++h) lt[h] = warp_sum(l[h]);
-    if (warp >= MW) {
-        const int u = warp - MW;
 #pragma unroll
-        for (int h = 0; h < HG; ++h) {
-            if (lane == 0) { mg_m[u * HG + h] = m[h]; mg_l[u * HG + h] = lt[h]; }
+    for (int h = 0; h < HG; ++h) {
+        if (lane == 0) { mg_m[warp * HG + h] = m[h]; mg_l[warp * HG + h] = lt[h]; }
 #pragma unroll
-            for (int e = 0; e < DV; ++e) mg_o[(u * HG + h) * D + lane * DV + e] = o[h][e];
-        }
-    }
-    cta_sync();
-    if (warp < MK_NW - MW) {
-#pragma unroll
-        for (int h = 0; h < HG; ++h) {
-            const float m2 = mg_m[warp * HG + h], l2 = mg_l[warp * HG + h];
-            const float mn = fmaxf(m[h], m2);
-            const float e1 = m[h] == mn ? 1.f : __expf(m[h] - mn);
-            const float e2 = m2 == mn ? 1.f : __expf(m2 - mn);
-            lt[h] = lt[h] * e1 + l2 * e2;
-#pragma unroll
-            for (int e = 0; e < DV; ++e) o[h][e] = o[h][e] * e1 + mg_o[(warp * HG + h) * D + lane * DV + e] * e2;
-            m[h] = mn;
-        }
-    }
-    cta_sync();
-    if (warp < MW) {
-#pragma unroll
-        for (int h = 0; h < HG; ++h) {
-            if (lane == 0) { mg_m[warp * HG + h] = m[h]; mg_l[warp * HG + h] = lt[h]; }
-#pragma unroll
-            for (int e = 0; e < DV; ++e) mg_o[(warp * HG + h) * D + lane * DV + e] = o[h][e];
-        }
+        for (int e = 0; e < DV; ++e) mg_o[(warp * HG + h) * D + lane * DV + e] = o[h][e];
     }
     cta_sync();
     for (int i = tid; i < HG * D; i += MK_NT) {
