@@ -103,7 +103,7 @@ struct StepPlan {
 // Kernel variant and shared-memory split for a model shape.  Returns null, or why the shape does not fit.
 // sched_reserve: bytes to set aside for the CTA's tile lists.
 inline const char *plan_step(const edgefm_shape &sh, int max_context, int num_sms, int smem_optin, size_t sched_reserve, StepPlan *pl, cudaError_t *cuda_err) {
-    const int H = sh.hidden, d = sh.head_dim, nq = sh.n_q_heads, nkv = sh.n_kv_heads, F = sh.ffn, G = nq / nkv;
+    const int H = sh.hidden, d = sh.head_dim, nq = sh.n_q_heads, nkv = sh.n_kv_heads, G = nq / nkv;
     *cuda_err = cudaSuccess;
     pl->long_ctx = max_context > 8192 || static_cast<long long>(nq) * MK_ATT_SPLIT_MAXC * 2 > MK_PARTIAL_FLOATS;
     pl->kernel = d == 64 ? mega_kernel_g<64>(G, pl->long_ctx) : mega_kernel_g<128>(G, pl->long_ctx);
@@ -112,27 +112,28 @@ inline const char *plan_step(const edgefm_shape &sh, int max_context, int num_sm
     pl->max_chunks = pl->grid / nkv > 0 ? pl->grid / nkv : 1;
     pl->n_ops = 4 * sh.n_layers + 1;
     const int NW = pl->nw, ATT_MW = NW;   // every warp has an entry in the attention merge area
-    int max_k = H;
-    if (nq * d > max_k) max_k = nq * d;
-    if (F > max_k) max_k = F;
+    int max_k = H;                       // vectors staged in shared memory: the residual stream and the attention output
+    if (nq * d > max_k) max_k = nq * d;   // (the down projection reads the MLP activations from global memory)
     max_k = (max_k + MK_TILE_COLS - 1) / MK_TILE_COLS * MK_TILE_COLS;   // whole 256-column pieces (zero-padded)
     // attention scratch: queries, probabilities, warp merge area, chunk statistics
-    const size_t att_bytes = (static_cast<size_t>(G) * d + NW * (G * MK_ATT_TILE > 32 / MK_ATT_LPP_SPLIT ? G * MK_ATT_TILE : 32 / MK_ATT_LPP_SPLIT) +
-                              2 * ATT_MW * G + static_cast<size_t>(ATT_MW) * G * d + 2 * static_cast<size_t>(G) * pl->max_chunks) * 4;
-    size_t xbuf = static_cast<size_t>(max_k) * 4;
+    // (the short-context build always runs attention with one query head per CTA)
+    const int AG = pl->long_ctx ? G : 1;
+    const size_t att_bytes = (static_cast<size_t>(AG) * d + NW * (AG * MK_ATT_TILE > 32 / MK_ATT_LPP_SPLIT ? AG * MK_ATT_TILE : 32 / MK_ATT_LPP_SPLIT) +
+                              2 * ATT_MW * AG + static_cast<size_t>(ATT_MW) * AG * d + 2 * static_cast<size_t>(AG) * pl->max_chunks) * 4;
+    size_t xbuf = MK_X_SPLITS * (static_cast<size_t>(max_k) * 2 + MK_XS_PAD);   // the staged activation: three bf16 arrays
     if (att_bytes > xbuf) xbuf = att_bytes;
     pl->xbuf = (xbuf + 1023) / 1024 * 1024;
     cudaFuncAttributes fa{};
     *cuda_err = cudaFuncGetAttributes(&fa, pl->kernel);
     if (*cuda_err != cudaSuccess) return "cudaFuncGetAttributes";
-    const size_t static_smem = fa.sharedSizeBytes + 256;   // the kernel's static shared memory (mbarriers, tables, scratch) + margin
+    const size_t static_smem = fa.sharedSizeBytes + 1024;   // the kernel's static shared memory (mbarriers, tables, scratch) + the padding in
+                                                            // front of the 1 KB-aligned dynamic part
     pl->ops_bytes = static_cast<size_t>(pl->n_ops) * sizeof(MkOp);
     const size_t tab = static_cast<size_t>(cta_tab_ints_for(NW)) * sizeof(int);
     pl->tab_bytes = (tab + 15) / 16 * 16;
     const size_t head = (pl->ops_bytes + pl->tab_bytes + sched_reserve + 1023) / 1024 * 1024;   // the rings start on a 1 KB boundary
     pl->sched_bytes = head - pl->ops_bytes - pl->tab_bytes;
-    // behind the rings: the activation vector; at least one full tile (8 KB) of valid shared memory follows the last slot
-    const size_t tail = std::max(pl->xbuf, static_cast<size_t>(MK_TILE_ROWS) * MK_TILE_COLS * 2);
+    const size_t tail = pl->xbuf + static_cast<size_t>(NW) * MK_WBUF_BYTES;   // behind the rings: the activation vector and the warps' small buffers
     if (head + tail + static_smem + static_cast<size_t>(NW) * 2 * 2048 > static_cast<size_t>(smem_optin))
         return "model shape does not fit the shared-memory plan";
     const size_t per_warp = (smem_optin - static_smem - head - tail) / NW;
@@ -178,15 +179,15 @@ inline void fill_ops(const edgefm_shape &sh, const edgefm_layer_weights *layers,
         MkOp op{};
         weights_out[n] = static_cast<const uint16_t *>(W);
         op.bias = static_cast<const uint16_t *>(bias); op.norm_w = static_cast<const uint16_t *>(norm); op.x_src = x_src; op.out = dst;
-        op.K = o.K; op.kind = o.kind; op.units_total = o.units; op.layer_flags = layer << 8 | flags;
+        op.K = o.K; op.kind = o.kind; op.units_total = o.units; op.layer_flags = layer << 8 | flags | (o.K % 64 ? PHF_RAGGED : 0);
         out[n++] = op;
     };
     for (int l = 0; l < sh.n_layers; ++l) {
         const edgefm_layer_weights &w = layers[l];
         mk(os[0], w.wqkv, sh.qkv_bias ? w.bqkv : nullptr, w.input_norm, l == 0 ? nullptr : x, q, l, 0);
-        mk(os[1], w.wo, nullptr, nullptr, attn, x, l, PHF_X_BULK);        // the attention phase stores its output in the staged layout
-        mk(os[2], w.w_gate_up, nullptr, w.post_norm, x, act, l, PHF_OUT_SPLIT);  // the MLP activations go to memory in the layout the down projection stages
-        mk(os[3], w.w_down, nullptr, nullptr, act, x, l, PHF_X_BULK);
+        mk(os[1], w.wo, nullptr, nullptr, attn, x, l, 0);
+        mk(os[2], w.w_gate_up, nullptr, w.post_norm, x, act, l, PHF_OUT_SPLIT);  // the MLP activations go to memory in the form the down projection multiplies
+        mk(os[3], w.w_down, nullptr, nullptr, act, x, l, PHF_X_GLOBAL);
     }
     mk(os[4], lm_head, nullptr, final_norm, x, nullptr, sh.n_layers, 0);
 }
@@ -252,7 +253,7 @@ inline void fill_shape_params(MkParams *m, const edgefm_shape &sh, int max_conte
     m->sched_bytes = static_cast<int>(pl.sched_bytes);
     m->cta_tab_ints = ss.cta_tab_ints;
     m->barrier_extra = 0;
-    m->pf_tiles = 4;   // measured: 3 .. 8 equal, 16 thrashes L2 (1.5B shape)
+    m->pf_tiles = MK_PF_TILES;   // measured: 3 .. 8 equal, 16 thrashes L2 (1.5B shape)
     m->map_fence = 1;   // edgefm_set_vocab_subset rewrites the output layer's maps between steps
     m->spin_limit = 1000000000u;   // 1 s
 }
@@ -487,7 +488,8 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
     CREATE_TRY(dev_alloc(&c->x, H));
     CREATE_TRY(dev_alloc(&c->q, nq * d));
     CREATE_TRY(dev_alloc(&c->attn, nq * d));
-    CREATE_TRY(dev_alloc(&c->act, F));
+    CREATE_TRY(dev_alloc(&c->act, static_cast<size_t>(MK_X_SPLITS) * ((F + MK_TILE_COLS - 1) / MK_TILE_COLS * MK_TILE_COLS) / 2));   // three bf16 arrays of F rounded
+                                                                                         // up to whole column pieces (the pieces of every value)
     CREATE_TRY(dev_alloc(&c->inv_freq, d / 2));
     CREATE_TRY(dev_alloc(&c->part_m, static_cast<size_t>(nq) * pl.max_chunks));
     CREATE_TRY(dev_alloc(&c->part_l, static_cast<size_t>(nq) * pl.max_chunks));
@@ -899,7 +901,7 @@ extern "C" edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, co
     float *x = sc.take<float>(H);
     float *q = sc.take<float>(static_cast<size_t>(nq) * d);
     float *attn = sc.take<float>(static_cast<size_t>(nq) * d);
-    float *act = sc.take<float>(F);
+    float *act = sc.take<float>(static_cast<size_t>(MK_X_SPLITS) * ((F + MK_TILE_COLS - 1) / MK_TILE_COLS * MK_TILE_COLS) / 2);
     double *inv_freq = sc.take<double>(d / 2);
     float *part_m = sc.take<float>(static_cast<size_t>(nq) * max_chunks);
     float *part_l = sc.take<float>(static_cast<size_t>(nq) * max_chunks);

@@ -7,18 +7,19 @@
 //   * The step's weight traffic is a static schedule made on the host (QKV, O, gate/up, down of every layer,
 //     then lm_head).  Every CTA owns a fixed share of each operator's rows; the share is cut into tiles of up
 //     to 16 rows x 256 columns, and every consumer warp owns a fixed list of tiles (the same for every layer).
-//   * Every consumer warp keeps a private ring of shared-memory slots filled with its next tiles by 2-D TMA tensor
-//     copies (cp.async.bulk.tensor, mbarrier complete_tx): when it has multiplied a tile, its lane 0 at once fetches
+//   * Every consumer warp keeps a private ring of shared-memory slots filled with its next tiles by TMA tensor copies
+//     (cp.async.bulk.tensor, 128-byte swizzle, mbarrier complete_tx): when it has multiplied a tile, its lane 0 at once fetches
 //     the tile that comes S places later in its sequence into the freed slot -- regardless of operator boundaries,
 //     the weights do not depend on the computation.  So the short operators of a layer are on chip when their turn
 //     comes and HBM keeps streaming while the arithmetic waits at a grid barrier, stages an activation vector or
 //     runs attention.  One more warp of the CTA computes nothing: it runs ahead of the rings and pulls the tiles
 //     that come next into L2 (prefetch.global.L2), because the rings alone hold too little to keep HBM busy through
 //     the stalls and a refill from L2 returns much sooner than one from HBM.
-//   * A consumer warp waits for its next tile, multiplies it with the 256 activations of the tile's columns
-//     (8 per lane, from the vector staged in shared memory) into 16 row accumulators and releases the slot.
-//     Consecutive tiles of a warp cover the same rows; only at the end of a run of tiles are the 16 sums
-//     reduced across the lanes (a butterfly of 16 + 1 shuffles).  The fused epilogues (bias + RoPE + KV append,
+//   * A consumer warp waits for its next tile, multiplies it with the 256 activations of the tile's columns and releases
+//     the slot.  The multiplication is 16 x (ldmatrix + mma.m16n8k16): the fp32 activations are staged as three bf16
+//     pieces (columns 0..2 of the B operand), the products are exact and accumulate in fp32.  Consecutive tiles of a warp
+//     cover the same rows; only at the end of a run of tiles are the row sums taken out of the accumulator fragments
+//     (three shuffles).  The fused epilogues (bias + RoPE + KV append,
 //     residual add, SwiGLU, logits + argmax) run in the warp when it has seen all columns of its rows, else the
 //     sums meet in shared memory after the operator, in a fixed order.
 //   * Between dependent operators all CTAs meet at a grid barrier (monotonic counter in global memory,
@@ -45,14 +46,8 @@ constexpr int MK_THREADS = MK_NT + 32;           // + the L2 prefetch warp
 #ifndef MK_SPLIT_DEFER
 #define MK_SPLIT_DEFER 1
 #endif
-#ifndef MK_ATT_HOIST
-#define MK_ATT_HOIST 0
-#endif
-#ifndef MK_MERGE_NOUT
-#define MK_MERGE_NOUT 1
-#endif
-#ifndef MK_DEFER_REFILL
-#define MK_DEFER_REFILL 0
+#ifndef MK_ACC_CHAINS
+#define MK_ACC_CHAINS 4   // independent tensor-core accumulation chains per warp
 #endif
 
 // ---- mbarrier / bulk copy primitives -----------------------------------------------------------------
@@ -108,39 +103,38 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long *b, unsigned parity
     *abort_flag = 1;
     return false;
 }
-__device__ __forceinline__ void bulk_copy_g2s_plain(void *dst, const void *src, unsigned bytes, unsigned long long *bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
-                 : "memory");
-}
-// One box of a weight matrix (tensor map `map`: 256 columns x the map's box height) starting at (column x, row y).
-// x * 2 bytes is a multiple of 16 by construction (x is a multiple of 256); no multicast.
+// One box of a weight matrix through tensor map `map`; the coordinates are listed innermost first.  The innermost one is a
+// column (0, or a multiple of 64: x * 2 bytes is a multiple of 16 by construction); no multicast.
 __device__ __forceinline__ void tma_load_box(void *dst, const void *map, int x, int y, unsigned long long *bar, unsigned long long policy) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
         ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(policy)
         : "memory");
 }
-// A pair of boxes in one copy: gate rows and their up rows (3-D view [2][F][K] of the gate/up matrix) ...
+// (more dimensions: the 64-column blocks of a row, the partner rows of gate/up and of rotate-half, the heads)
 __device__ __forceinline__ void tma_load_box3(void *dst, const void *map, int x, int y, int z, unsigned long long *bar, unsigned long long policy) {
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4}], [%5], %6;"
         ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar)), "l"(policy)
         : "memory");
 }
-// ... or rows i.. and i + d/2.. of one head (4-D view [heads][2][d/2][K] of the QKV matrix).
 __device__ __forceinline__ void tma_load_box4(void *dst, const void *map, int x, int y, int z, int w, unsigned long long *bar, unsigned long long policy) {
     asm volatile(
         "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
         ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(smem_u32(bar)), "l"(policy)
         : "memory");
 }
+__device__ __forceinline__ void tma_load_box5(void *dst, const void *map, int x, int y, int z, int w, int v, unsigned long long *bar, unsigned long long policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4, %5, %6}], [%7], %8;"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(v), "r"(smem_u32(bar)), "l"(policy)
+        : "memory");
+}
 // all consumer threads of the CTA (the feeding warp never joins)
 __device__ __forceinline__ void cta_sync() { asm volatile("bar.sync 1, %0;" ::"n"(MK_NT) : "memory"); }
 
-// Dynamic shared memory: operators | schedule table | tile lists | rings | activation vector (also the attention scratch).
-// The vector comes last on purpose: a tile of fewer than 16 rows is multiplied with a fixed, branch-free row loop that
-// may read (and ignore) bytes behind the tile, i.e. behind the last slot of the last ring.
+// Dynamic shared memory: operators | schedule table | tile lists | rings (1 KB-aligned slots) | staged activation vector
+// (also the attention scratch).
 // (Addresses are recomputed from the kernel parameters where they are used instead of being carried in registers.)
 extern __shared__ __align__(1024) unsigned char mk_smem[];
 __device__ __forceinline__ MkOp *sm_ops(const MkParams &) { return reinterpret_cast<MkOp *>(mk_smem); }
@@ -155,8 +149,29 @@ __device__ __forceinline__ unsigned char *sm_ring(const MkParams &p, int warp) {
     return mk_smem + p.ops_bytes + p.tab_bytes + p.sched_bytes + warp * (p.slots * p.slot_bytes);
 }
 __device__ __forceinline__ unsigned char *sm_xbuf(const MkParams &p) { return sm_ring(p, MK_NW); }
-__device__ __forceinline__ float4 *sm_xa(const MkParams &p) { return reinterpret_cast<float4 *>(sm_xbuf(p)); }
-__device__ __forceinline__ float4 *sm_xb(const MkParams &p) { return reinterpret_cast<float4 *>(sm_xbuf(p) + p.xbuf_bytes / 2); }
+// The staged activation vector of an operator with K columns: MK_X_SPLITS bf16 arrays of Kpad = K rounded up to whole
+// 256-column pieces (zero beyond K), xs_stride(K) bytes apart.  Array s holds piece s of every value (value = sum of its
+// pieces to 24 bits), columns in tensor-core fragment order (mk_xs_index).
+__device__ __forceinline__ int xs_stride(int K) { return (K + MK_TILE_COLS - 1) / MK_TILE_COLS * (MK_TILE_COLS * 2) + MK_XS_PAD; }
+// two values -> one bf16x2 word (first value in the low half), round to nearest even
+__device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {
+    unsigned d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+// Split four consecutive values (columns 4 * i4 ..) into their bf16 pieces and store them in fragment order.
+__device__ __forceinline__ void stage_piece(unsigned char *xs, int stride, int i4, float4 t) {
+    const int idx = mk_xs_index(i4 * 4);          // columns c, c+1 are neighbours; c+2, c+3 follow 8 entries later
+    unsigned *dst = reinterpret_cast<unsigned *>(xs) + (idx >> 1);
+#pragma unroll
+    for (int sp = 0; sp < MK_X_SPLITS; ++sp) {
+        const unsigned a = pack_bf16x2(t.x, t.y), b = pack_bf16x2(t.z, t.w);
+        dst[0] = a;
+        dst[4] = b;
+        dst += stride >> 2;
+        t.x -= bf16lo(a); t.y -= bf16hi(a); t.z -= bf16lo(b); t.w -= bf16hi(b);   // exact: the remainder is what the next piece holds
+    }
+}
 
 __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned *p) {
     unsigned v;
@@ -183,14 +198,10 @@ __device__ __forceinline__ bool diag_fail(const MkParams &p, volatile int *abort
 }
 
 // All consumer threads of all CTAs meet here.  Returns false when the wait expired (step aborted).
-// `while_waiting` runs after this CTA has announced its arrival and before it starts polling (refills that short
-// operators put off: the time is free here).
-template <typename F>
-__device__ __forceinline__ bool grid_barrier(const MkParams &p, unsigned target, volatile int *abort_flag, int tid, int &prof_idx, F &&while_waiting) {
+__device__ __forceinline__ bool grid_barrier(const MkParams &p, unsigned target, volatile int *abort_flag, int tid, int &prof_idx) {
     cta_sync();
     prof_stamp(p, tid, prof_idx);   // this CTA's share of the operator is done
     if (tid == 0 && !*abort_flag) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.barrier) : "memory");
-    while_waiting();
     if (tid == 0 && !*abort_flag) {
         unsigned it = 0;
         unsigned long long t0 = 0;
@@ -238,8 +249,10 @@ struct WarpStream {
     int slot;                   // slot of the next tile to multiply
     unsigned round;
     unsigned consumed;          // tiles multiplied so far
-    int pending;                // slots read but not refilled yet (short operators leave the refill to the next grid barrier)
     int fenced_op;
+    unsigned total;             // tiles of this warp over the whole step
+    int n_layer;                // tiles per layer
+    int list_layer, list_lm;    // the warp's two lists in the CTA's tile block
 };
 // Lane 0 only: fetch tile ws.next into ring slot `slot` (whose previous contents this warp has finished reading).
 __device__ __forceinline__ bool fetch_next_tile(const MkParams &p, WarpStream &ws, int slot, volatile int *abort_flag, volatile unsigned *s_issued,
@@ -251,21 +264,20 @@ __device__ __forceinline__ bool fetch_next_tile(const MkParams &p, WarpStream &w
 #else
 #define FSEG(i) do {} while (0)
 #endif
-    const int *tab = sm_tab(p) + warp * MK_WARP_TAB;
+    if (ws.next.count >= ws.total) return true;          // the whole step has been fetched
     const bool lm = ws.next.layer >= p.n_layers;
-    if (lm && ws.next.i >= tab[6]) return true;          // the whole step has been fetched
     const uint2 d = ws.nd;
     // the operators of a layer are QKV, O, gate/up, down in this order; 4 = the output layer
     const int op = static_cast<int>((d.y >> 20) & 7u);
-    const int opi = lm ? 4 * p.n_layers : 4 * ws.next.layer + op;
+    const int opi = 4 * ws.next.layer + (lm ? 0 : op);
     const int m = static_cast<int>(d.y & 31u), x = static_cast<int>((d.x >> 20) & 0xffu) * MK_TILE_COLS;
     const int u0 = static_cast<int>(d.x & 0xfffffu);
     const bool paired = op == 0 || op == 2;
-    const unsigned bytes = static_cast<unsigned>(m) * (MK_TILE_COLS * 2) * (paired ? 2u : 1u);
+    const unsigned bytes = static_cast<unsigned>(m) << (paired ? 10 : 9);   // m rows (and their partners) x 512 bytes
     // (the host made the schedule; a corrupt entry must still not write past the slot)
     if (m < 1 || bytes > static_cast<unsigned>(p.slot_bytes) || (lm ? op != 4 : op > 3)) return diag_fail(p, abort_flag, 1, opi, u0);
     const unsigned char *map = p.maps + (static_cast<size_t>(opi) * MK_MAX_VARIANTS + ((d.x >> 28) & 3u)) * 128;
-    if (opi != ws.fenced_op && (p.map_fence == 2 || (p.map_fence == 1 && lm))) {
+    if (p.map_fence != 0 && opi != ws.fenced_op && (p.map_fence == 2 || lm)) {
         // the host may have rewritten this operator's tensor maps since the last launch (another vocabulary subset, or a
         // static call with other weights): order the copy engine's view of them behind what is in memory now
         ws.fenced_op = opi;
@@ -282,13 +294,24 @@ __device__ __forceinline__ bool fetch_next_tile(const MkParams &p, WarpStream &w
     FSEG(2);
     mbar_arrive_expect_tx(bar, bytes);
     FSEG(3);
-    if (op == 0) tma_load_box4(dst, map, x, u0 & ((p.d >> 1) - 1), 0, u0 >> p.half_shift, bar, policy);
-    else if (op == 2) tma_load_box3(dst, map, x, u0, 0, bar, policy);
-    else tma_load_box(dst, map, x, u0, bar, policy);
+    if (!(d.y & MKT_RAGGED)) {                           // one copy: the tile's four 64-column blocks are a dimension of the map
+        const int cb = x >> 6;
+        if (op == 0) tma_load_box5(dst, map, 0, u0 & ((p.d >> 1) - 1), 0, u0 >> p.half_shift, cb, bar, policy);
+        else if (op == 2) tma_load_box4(dst, map, 0, u0, 0, cb, bar, policy);
+        else tma_load_box3(dst, map, 0, u0, cb, bar, policy);
+    } else {                                               // K has a ragged last block: block by block (blocks past K read as zero)
+        const unsigned blk = bytes >> 2;
+#pragma unroll
+        for (int cb = 0; cb < MK_TILE_COLS / 64; ++cb) {
+            if (op == 0) tma_load_box4(dst + cb * blk, map, x + cb * 64, u0 & ((p.d >> 1) - 1), 0, u0 >> p.half_shift, bar, policy);
+            else if (op == 2) tma_load_box3(dst + cb * blk, map, x + cb * 64, u0, 0, bar, policy);
+            else tma_load_box(dst + cb * blk, map, x + cb * 64, u0, bar, policy);
+        }
+    }
     FSEG(4);
-    cursor_step(ws.next, tab[7], p.n_layers);
+    cursor_step(ws.next, ws.n_layer, p.n_layers);
     s_issued[warp] = ws.next.count;     // read by the L2 prefetch warp
-    ws.nd = sm_tiles(p)[(ws.next.layer >= p.n_layers ? tab[5] : tab[0]) + ws.next.i];   // (one entry behind the lists is readable: the combines follow)
+    ws.nd = sm_tiles(p)[(ws.next.layer >= p.n_layers ? ws.list_lm : ws.list_layer) + ws.next.i];   // (one entry behind the lists is readable: the combines follow)
 #ifdef EDGEFM_TRACE_OP
     FSEG(5);
     if (p.prof && blockIdx.x == 0 && warp == 3 && opi == EDGEFM_TRACE_OP) {
@@ -298,22 +321,6 @@ __device__ __forceinline__ bool fetch_next_tile(const MkParams &p, WarpStream &w
     }
 #endif
     return true;
-}
-
-// Refill the slots a short operator left empty (whole warp; lane 0 issues).
-__device__ __forceinline__ bool refill_pending(const MkParams &p, WarpStream &ws, volatile int *abort_flag, volatile unsigned *s_issued,
-                                               unsigned long long *full_bar, int warp, int lane) {
-    bool ok = true;
-    if (ws.pending > 0 && lane == 0) {
-        int sl = ws.slot - ws.pending;
-        if (sl < 0) sl += p.slots;
-        for (int i = 0; i < ws.pending && ok; ++i) {
-            ok = fetch_next_tile(p, ws, sl, abort_flag, s_issued, full_bar, warp);
-            if (++sl == p.slots) sl = 0;
-        }
-    }
-    ws.pending = 0;
-    return ok;
 }
 
 // Attention chunking shared by the attention phase and by the consumer of its partial results.
@@ -381,7 +388,8 @@ __device__ __forceinline__ void prefetch_tiles(const MkParams &p, volatile int *
         const unsigned issued = s_issued[w];
         if (k < issued) k = issued;                         // the ring got there first
         if (k >= total) break;
-        if (k >= issued + static_cast<unsigned>(p.pf_tiles)) {   // far enough ahead: wait for the ring to move
+        // (the output layer is one long uninterrupted stream: a deeper look-ahead pays there, and only there)
+        if (k >= issued + static_cast<unsigned>(k >= static_cast<unsigned>(n_layer) * p.n_layers ? MK_PF_TILES_LM : p.pf_tiles)) {   // far enough ahead: wait for the ring to move
             if (*abort_flag || ++idle > (1u << 22)) return;  // bounded: give up (prefetching is only a hint)
             __nanosleep(200);
             continue;
@@ -433,8 +441,14 @@ __device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkOp &P,
     } else if (P.kind == PH_SWIGLU) {
         const float a = lo / (1.f + expf(-lo)) * hi;
         if (P.flags() & PHF_OUT_SPLIT) {   // the layout the next operator's prologue copies straight into shared memory
-            const int i4 = u >> 2;
-            P.out[(i4 & 1) * (P.units_total >> 1) + ((i4 >> 1) << 2) + (u & 3)] = a;
+            uint16_t *o = reinterpret_cast<uint16_t *>(P.out) + mk_xs_index(u);
+            float r = a;
+#pragma unroll
+            for (int sp = 0; sp < MK_X_SPLITS; ++sp) {
+                const uint16_t b = f32_to_bf16_bits(r);
+                o[static_cast<size_t>(sp) * ((P.units_total + MK_TILE_COLS - 1) / MK_TILE_COLS * MK_TILE_COLS)] = b;
+                r -= bf16_bits_to_f32(b);
+            }
         } else {
             P.out[u] = a;
         }
@@ -466,25 +480,6 @@ __device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkOp &P,
     }
 }
 
-// Sum the 16 accumulator rows across the 32 lanes: afterwards lanes 2r and 2r+1 hold the sum of row r.
-// Each step pairs lanes `off` apart: a lane keeps one half of its values and hands the other half over,
-// 8 + 4 + 2 + 1 exchanges, then one more exchange between the two lanes that share a row.
-__device__ __forceinline__ float reduce_rows(float (&a)[MK_TILE_ROWS], int lane) {
-#pragma unroll
-    for (int off = 16, n = MK_TILE_ROWS; off >= 2; off >>= 1, n >>= 1) {
-        const bool up = (lane & off) != 0;
-#pragma unroll
-        for (int i = 0; i < MK_TILE_ROWS / 2; ++i) {
-            if (i < n / 2) {
-                const float send = up ? a[i] : a[i + n / 2];
-                const float keep = up ? a[i + n / 2] : a[i];
-                a[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
-            }
-        }
-    }
-    return a[0] + __shfl_xor_sync(0xffffffffu, a[0], 1);
-}
-
 // ---- the consumer side of the weight stream --------------------------------------------------------------------
 // Optional fine-grained trace of one operator in CTA 0 (compile with -DEDGEFM_TRACE_OP=<operator index>): lane 0 of every
 // consumer warp appends %globaltimer stamps (before the wait, data there, tile multiplied) behind the profile table.
@@ -498,71 +493,118 @@ __device__ __forceinline__ float reduce_rows(float (&a)[MK_TILE_ROWS], int lane)
 #define MK_TRACE(k) do {} while (0)
 #endif
 // This warp's `n` tiles of operator P: wait, multiply, release; reduce and finish rows where the schedule says so.
+//
+// The multiplication runs on the tensor cores, not because the operator has the arithmetic intensity of a GEMM (it is a
+// matrix-vector product) but because the scalar form needs 17 instructions per 16 bytes of weights (load, 8 conversions, 8
+// FMAs) and the warp's serial wait - multiply - refill chain, not HBM, bounded the stream.  One mma.m16n8k16 multiplies a
+// 16-row x 16-column block of bf16 weights (A, read with ldmatrix from the swizzled tile) by B = [16 x 8]: columns 0..2 hold
+// the three bf16 pieces of the fp32 activations, columns 3..7 are zero.  Accumulation is fp32; the row sum is the sum of
+// columns 0..2.  Products of two bf16 values are exact in fp32, so the result differs from an fp32 FMA chain only in the
+// order of the additions.
 __device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkOp &P, int n, WarpStream &ws, volatile int *abort_flag, ItemCtx &cx,
                                               float *s_partial, const float *s_rope, volatile unsigned *s_issued, unsigned long long *full_bar, int lane) {
     const int warp = static_cast<int>(threadIdx.x >> 5);
     const MkOp *p_ops_base = sm_ops(p);
     (void)p_ops_base;
-    float acc[MK_TILE_ROWS];   // 16 independent chains: enough to cover the FMA latency
+    // D fragments: rows lane/4 and lane/4 + 8, columns 2 (lane%4), 2 (lane%4) + 1; one accumulator per 64-column block of a tile,
+    // so that four independent chains of tensor-core instructions are in flight
+    float acc[MK_ACC_CHAINS][4];
+#pragma unroll
+    for (int cb = 0; cb < MK_ACC_CHAINS; ++cb) { acc[cb][0] = 0.f; acc[cb][1] = 0.f; acc[cb][2] = 0.f; acc[cb][3] = 0.f; }
     const bool paired = P.kind == PH_QKV || P.kind == PH_SWIGLU;
-    // a short operator (all its tiles are already in the ring) leaves the refills to the grid barrier that follows it, so that
-    // nothing but the arithmetic sits on its critical path
-    const bool defer = MK_DEFER_REFILL != 0 && n + ws.pending <= p.slots && P.kind != PH_LMHEAD;
-#ifdef MK_STAGGER
-    if (n > 2) {   // spread the warps' refill requests over time: they share one copy-engine port
-        const long long t0 = clock64();
-        while (clock64() - t0 < static_cast<long long>(warp) * MK_STAGGER) {}
-    }
-#endif
+    // B fragments: lanes 0..11 hold piece (lane / 4) of the activations, k indices by lane % 4; the other lanes multiply by zero.
+    // They are read from shared memory block by block while the tile is multiplied: from the staged vector, or (PHF_X_GLOBAL:
+    // the vector is in global memory in the same form) from a small buffer of this warp, into which the 1.5 KB of the next
+    // tile are copied asynchronously (no registers held) as soon as the current tile has been multiplied.
+    const bool xg = (P.flags() & PHF_X_GLOBAL) != 0;
+    const int kpad2 = (P.K + MK_TILE_COLS - 1) / MK_TILE_COLS * (MK_TILE_COLS * 2);
+    unsigned char *wbuf = sm_xbuf(p) + p.xbuf_bytes + warp * MK_WBUF_BYTES;
+    const unsigned char *b_base = xg ? wbuf + (lane >> 2) * (MK_TILE_COLS * 2 + MK_XS_PAD) + (lane & 3) * 16
+                                     : sm_xbuf(p) + (lane >> 2) * xs_stride(P.K) + (lane & 3) * 16;
+    auto request_b = [&](int kcol) {
+        const unsigned char *src = reinterpret_cast<const unsigned char *>(P.x_src) + kcol * (MK_TILE_COLS * 2) + lane * 16;
+#pragma unroll
+        for (int sp = 0; sp < MK_X_SPLITS; ++sp)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(wbuf + sp * (MK_TILE_COLS * 2 + MK_XS_PAD) + lane * 16)),
+                         "l"(src + static_cast<size_t>(sp) * kpad2) : "memory");
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    auto load_b = [&](const unsigned char *at) {
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (lane < 4 * MK_X_SPLITS) v = *reinterpret_cast<const uint4 *>(at);
+        return v;
+    };
+    // A fragments: ldmatrix.x4 takes from lane l the address of row l % 8 of matrix l / 8; the four matrices are
+    // (rows 0..7 | rows 8..15) x (k 0..7 | k 8..15) of a 16 x 16 block
+    const int mrow = (lane & 7) + ((lane >> 3) & 1) * 8, khalf = lane >> 4;
     const uint2 *list = sm_tiles(p) + ws.list;
     uint2 d = n > 0 ? list[0] : make_uint2(0u, 0u);
+    if (xg && n > 0) request_b(static_cast<int>((d.x >> 20) & 0xffu));
     for (int t = 0; t < n; ++t) {
         const uint2 dn = t + 1 < n ? list[t + 1] : make_uint2(0u, 0u);
         if (d.x & MKT_FIRST) {
 #pragma unroll
-            for (int r = 0; r < MK_TILE_ROWS; ++r) acc[r] = 0.f;
+            for (int cb = 0; cb < MK_ACC_CHAINS; ++cb) { acc[cb][0] = 0.f; acc[cb][1] = 0.f; acc[cb][2] = 0.f; acc[cb][3] = 0.f; }
         }
-        const int m = static_cast<int>(d.y & 31u), kcol = static_cast<int>((d.x >> 20) & 0xffu);
-        const float4 xa = sm_xa(p)[kcol * 32 + lane], xb = sm_xb(p)[kcol * 32 + lane];
+        const int m = static_cast<int>(d.y & 31u);
+        const unsigned char *bl = b_base + (xg ? 0 : static_cast<int>((d.x >> 20) & 0xffu) * (MK_TILE_COLS * 2));
         MK_TRACE(0);
         if (!mbar_wait(&full_bar[warp * MK_MAX_SLOTS + ws.slot], ws.round & 1u, abort_flag, p.spin_limit)) return false;
         MK_TRACE(1);
-        const unsigned char *tile = sm_ring(p, warp) + ws.slot * p.slot_bytes + lane * 16;
-        // accumulator rows 8.. : the partner rows of a paired tile follow its m low rows; those of an unpaired tile follow rows 0..7
-        const int hoff = (paired ? m : 8) * (MK_TILE_COLS * 2);
-        // rows of the tile as a compile-time mask: the loop is fully unrolled and free of branches, so the loads of all rows are in
-        // flight together (rows a tile does not have read stale bytes of the slot; their sums are never used)
-        auto rows = [&](auto mask_c) {
-            constexpr unsigned MASK = decltype(mask_c)::value;
+        if (xg) {
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            __syncwarp();
+        }
+        uint4 bb0 = load_b(bl), bb1 = load_b(bl + 64);   // two k-steps per 16-byte piece
+        // The tile: [4 column blocks][rows_total][128 bytes]; rows_total = m, or the m low rows followed by their m partners.
+        // M rows 0..7 are rows 0..7 (low rows), M rows 8..15 are rows 8..15 (partners); rows the tile does not have repeat its
+        // last row (their sums are never used).  16-byte chunk j of a row is stored at chunk j ^ (row index in the slot % 8).
+        const int rows_total = paired ? 2 * m : m;
+        const int tr = paired ? (mrow < 8 ? min(mrow, m - 1) : m + min(mrow - 8, m - 1)) : min(mrow, m - 1);
+        const unsigned tile = smem_u32(sm_ring(p, warp) + ws.slot * p.slot_bytes);
 #pragma unroll
-            for (int r = 0; r < MK_TILE_ROWS; ++r) {
-                if (MASK >> r & 1u) {
-                    const uint4 w = *reinterpret_cast<const uint4 *>(tile + (r < 8 ? r * (MK_TILE_COLS * 2) : hoff + (r - 8) * (MK_TILE_COLS * 2)));
-                    acc[r] = dot8(w, xa, xb, acc[r]);
-                }
+        for (int cb = 0; cb < MK_TILE_COLS / 64; ++cb) {
+            const int blk = cb * rows_total + tr;
+            const unsigned row_addr = tile + static_cast<unsigned>(blk) * 128u;
+            const unsigned sw = static_cast<unsigned>(blk & 7);
+            uint4 nb0 = bb0, nb1 = bb1;
+            if (cb + 1 < MK_TILE_COLS / 64) { nb0 = load_b(bl + (cb + 1) * 128); nb1 = load_b(bl + (cb + 1) * 128 + 64); }
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                const int s = cb * 4 + ks;
+                const unsigned addr = row_addr + (((static_cast<unsigned>(ks * 2 + khalf)) ^ sw) << 4);
+                unsigned a0, a1, a2, a3;
+                asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "r"(addr));
+                const uint4 bb = ks < 2 ? bb0 : bb1;
+                const unsigned b0 = (s & 1) ? bb.z : bb.x, b1 = (s & 1) ? bb.w : bb.y;
+                asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                             : "+f"(acc[s % MK_ACC_CHAINS][0]), "+f"(acc[s % MK_ACC_CHAINS][1]), "+f"(acc[s % MK_ACC_CHAINS][2]), "+f"(acc[s % MK_ACC_CHAINS][3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
             }
-        };
-        if (paired) {
-            if (m <= 4) rows(std::integral_constant<unsigned, 0x0f0fu>()); else rows(std::integral_constant<unsigned, 0xffffu>());
-        } else {
-            if (m <= 8) rows(std::integral_constant<unsigned, 0x00ffu>());
-            else if (m <= 12) rows(std::integral_constant<unsigned, 0x0fffu>());
-            else rows(std::integral_constant<unsigned, 0xffffu>());
+            bb0 = nb0; bb1 = nb1;
         }
         __syncwarp();
         MK_TRACE(2);
-        if (defer) ++ws.pending;
-        else if (lane == 0 && !fetch_next_tile(p, ws, ws.slot, abort_flag, s_issued, full_bar, warp)) return false;   // refill the slot
+        if (xg && t + 1 < n) request_b(static_cast<int>((dn.x >> 20) & 0xffu));   // every lane has read the buffer (the sync above)
+        if (lane == 0 && !fetch_next_tile(p, ws, ws.slot, abort_flag, s_issued, full_bar, warp)) return false;   // refill the slot
         if (++ws.slot == p.slots) { ws.slot = 0; ++ws.round; }
         ++ws.consumed;
         if (d.x & MKT_FLUSH) {
-            const float v = reduce_rows(acc, lane);        // lanes 2r, 2r+1: row r (the accumulators start over with the next FIRST tile)
+            // row sums: columns 0, 1 are in the lane with lane % 4 == 0, column 2 in its neighbour; then lanes 2r, 2r+1 take row r
+            // (the accumulators start over with the next FIRST tile)
+            float d0 = acc[0][0], d1 = acc[0][1], d2 = acc[0][2], d3 = acc[0][3];
+#pragma unroll
+            for (int c = 1; c < MK_ACC_CHAINS; ++c) { d0 += acc[c][0]; d1 += acc[c][1]; d2 += acc[c][2]; d3 += acc[c][3]; }
+            const float lo = d0 + d1 + __shfl_down_sync(0xffffffffu, d0, 1);
+            const float hi = d2 + d3 + __shfl_down_sync(0xffffffffu, d2, 1);
+            const int src = ((lane >> 1) & 7) * 4;
+            const float vlo = __shfl_sync(0xffffffffu, lo, src), vhi = __shfl_sync(0xffffffffu, hi, src);
+            const float v = lane < 16 ? vlo : vhi;
             const int j = lane >> 1;
             if (d.y & MKT_DIRECT) {
-                const float hi = __shfl_down_sync(0xffffffffu, v, 16);   // partner row 8 + j of unit j
+                const float hi2 = __shfl_down_sync(0xffffffffu, v, 16);   // partner row 8 + j of unit j
                 const int v0 = static_cast<int>((d.y >> 5) & 15u);
                 const int u = static_cast<int>(d.x & 0xfffffu) + j;
-                if (!(lane & 1) && j < m && j >= v0 && (!paired || lane < 16)) apply_epilogue(p, P, cx, s_rope, u, v * cx.rscale, hi * cx.rscale);
+                if (!(lane & 1) && j < m && j >= v0 && (!paired || lane < 16)) apply_epilogue(p, P, cx, s_rope, u, v * cx.rscale, hi2 * cx.rscale);
             } else {
                 const int slot = static_cast<int>((d.y >> 10) & 1023u);
                 if (slot >= MK_PARTIAL_SLOTS) return diag_fail(p, abort_flag, 2, slot, 0);
@@ -582,17 +624,14 @@ __device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkOp &P, 
 // (m, l, unnormalised o); the exact log-sum-exp merge is done here, in chunk order, by every CTA.
 __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_layer, WarpStream &ws, volatile int *abort_flag, float *s_part,
                                            float *s_partial, const float *s_rope, ItemCtx &cx, int token, int merge_attn, int tid, int &prof_idx,
-                                           unsigned long long *x_bar, unsigned &x_parity, volatile unsigned *s_issued, unsigned long long *full_bar) {
+                                           volatile unsigned *s_issued, unsigned long long *full_bar) {
     const MkOp &P = sm_ops(p)[ph];
-    float4 *xsA = sm_xa(p), *xsB = sm_xb(p);
+    unsigned char *xs = sm_xbuf(p);
+    const int xstride = xs_stride(P.K);
     const int *s_tab = sm_tab(p);
     const int lane = tid & 31, warp = tid >> 5;
     const int cta = blockIdx.x;
     const int n4 = P.K >> 2;
-    {   // columns past K of the last 256-column piece multiply zero-filled weights: keep the activations there finite (zero)
-        const int pc0 = P.K >> 3, pc1 = ((P.K + MK_TILE_COLS - 1) / MK_TILE_COLS) * (MK_TILE_COLS / 8);
-        for (int pc = pc0 + tid; pc < pc1; pc += MK_NT) { xsA[pc] = make_float4(0.f, 0.f, 0.f, 0.f); xsB[pc] = make_float4(0.f, 0.f, 0.f, 0.f); }
-    }
     float ss = 0.f;
     if (merge_attn > 0) {
         const int nch = merge_attn;
@@ -636,24 +675,10 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_
             }
             const float inv = 1.f / ll;
             acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-            if (o4 & 1) xsB[o4 >> 1] = acc; else xsA[o4 >> 1] = acc;
+            stage_piece(xs, xstride, o4, acc);
         }
-    } else if (P.flags() & PHF_X_BULK) {
-        // the vector is already in the split layout and needs no transform: two bulk copies, every thread waits for them
-        // (the CTA-wide sync of the grid barrier ordered all earlier reads of the buffer before this point)
-        // The vector was written by other CTAs of this launch with ordinary stores and acquired at the grid barrier;
-        // the bulk copy reads it through the asynchronous proxy, so a full proxy fence comes first (it also orders
-        // this CTA's earlier reads of the buffer before the copy's writes).
-        if (tid == 0) {
-            asm volatile("fence.proxy.async;" ::: "memory");
-            const unsigned half_bytes = static_cast<unsigned>(P.K) * 2u;
-            mbar_arrive_expect_tx(x_bar, 2u * half_bytes);
-            bulk_copy_g2s_plain(xsA, P.x_src, half_bytes, x_bar);
-            bulk_copy_g2s_plain(xsB, P.x_src + (P.K >> 1), half_bytes, x_bar);
-        }
-        const bool arrived = mbar_wait(x_bar, x_parity, abort_flag, p.spin_limit);
-        x_parity ^= 1u;
-        if (!arrived && tid == 0) p.state->status = 6;
+    } else if (P.flags() & PHF_X_GLOBAL) {
+        // nothing to stage: the consumer warps read the vector from global memory as they go
     } else {
         constexpr int PU = 4;  // loads in flight per thread
         for (int base = tid; base < n4; base += MK_NT * PU) {
@@ -682,10 +707,16 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_
                         ss = fmaf(t.x, t.x, ss); ss = fmaf(t.y, t.y, ss); ss = fmaf(t.z, t.z, ss); ss = fmaf(t.w, t.w, ss);
                         t.x *= bf16lo(w[u].x); t.y *= bf16hi(w[u].x); t.z *= bf16lo(w[u].y); t.w *= bf16hi(w[u].y);
                     }
-                    if (i4 & 1) xsB[i4 >> 1] = t; else xsA[i4 >> 1] = t;
+                    stage_piece(xs, xstride, i4, t);
                 }
             }
         }
+    }
+    if (!(P.flags() & PHF_X_GLOBAL)) {   // columns past K of the last 256-column piece multiply zero-filled weights: the activations there are zero
+        const int c1 = (P.K + MK_TILE_COLS - 1) / MK_TILE_COLS * MK_TILE_COLS;
+        for (int c = P.K + 2 * tid; c < c1; c += 2 * MK_NT)
+#pragma unroll
+            for (int sp = 0; sp < MK_X_SPLITS; ++sp) *reinterpret_cast<unsigned *>(xs + sp * xstride + mk_xs_index(c) * 2) = 0u;
     }
     if (P.norm_w) {
         ss = warp_sum(ss);
@@ -744,10 +775,6 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_
     }
     return ok;
 }
-
-// The attention output vector (n4 16-byte pieces) is stored as [even pieces | odd pieces], the layout of the shared-memory
-// activation buffers, so that the O projection stages it with two bulk copies.
-__device__ __forceinline__ int split_piece(int i4, int n4) { return (i4 & 1) * (n4 >> 1) + (i4 >> 1); }
 
 // ---- attention -----------------------------------------------------------------------------------------------
 // A CTA serves HG query heads of one GQA group over one chunk of the cached positions: HG = G (the whole
@@ -812,12 +839,7 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
             }
         }
     };
-    // the cache rows do not depend on this layer's queries (except the row appended by this step, which the grid barrier
-    // has published): request the first iteration's rows before waiting for the queries
     int tt = t0 + warp * TILE;
-#if MK_ATT_HOIST
-    if (tt < t1) load_kv(tt);
-#endif
     for (int i = tid; i < HG * D; i += MK_NT) qs[i] = __ldcg(p.q + static_cast<size_t>(qh0) * D + i) * p.scale;
     cta_sync();
 
@@ -831,9 +853,7 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
 
     while (tt < t1) {
         const bool pvalid = tt + pi < t1;
-#if !MK_ATT_HOIST
         load_kv(tt);
-#endif
         float s[HG];
 #pragma unroll
         for (int h = 0; h < HG; ++h) s[h] = 0.f;
@@ -887,9 +907,6 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
         }
         __syncwarp();
         tt += MK_NW * TILE;
-#if MK_ATT_HOIST
-        if (tt < t1) load_kv(tt);
-#endif
     }
 
     // merge the warps of the CTA: every warp publishes (m, l, o) (idle warps carry m = -inf and weigh 0), one sync, then
@@ -918,7 +935,7 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
         }
         const int qh = qh0 + h;
         if (nch == 1 && !defer_merge) {  // nothing to merge across CTAs
-            p.attn[split_piece((qh * D + j) >> 2, (p.nq * D) >> 2) * 4 + (j & 3)] = oo / ll;
+            p.attn[qh * D + j] = oo / ll;
         } else {
             p.part_o[(static_cast<size_t>(qh) * p.max_chunks + c) * D + j] = oo;
             if (j == 0) { p.part_m[qh * p.max_chunks + c] = mm; p.part_l[qh * p.max_chunks + c] = ll; }
@@ -966,7 +983,7 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
         }
         const float inv = 1.f / ll;
         acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-        reinterpret_cast<float4 *>(p.attn)[split_piece((qh0 + oh) * (D / 4) + oj4, (p.nq * D) >> 2)] = acc;
+        reinterpret_cast<float4 *>(p.attn)[(qh0 + oh) * (D / 4) + oj4] = acc;
     }
     if (tid == 0) p.tickets[grp] = 0u;
 }
@@ -977,7 +994,6 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
 template <int D, int G, bool LONG>
 __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParams p) {
     __shared__ __align__(8) unsigned long long full_bar[MK_NW * MK_MAX_SLOTS];
-    __shared__ __align__(8) unsigned long long x_bar;   // completion of bulk-copied activation vectors
     __shared__ float s_rope[128];
     __shared__ float s_part[MK_NW];
     __shared__ __align__(16) float s_partial[MK_PARTIAL_FLOATS];
@@ -991,7 +1007,6 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
     const int cta = blockIdx.x, ncta = gridDim.x;
     if (tid == 0) {
         for (int i = 0; i < MK_NW * MK_MAX_SLOTS; ++i) mbar_init(&full_bar[i], 1);
-        mbar_init(&x_bar, 1);
         s_abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -1033,8 +1048,10 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
         ws.next = TileCursor{tab[7] == 0 ? p.n_layers : 0, 0, 0u};
         ws.nd = sm_tiles(p)[(tab[7] == 0 ? tab[5] : tab[0])];
         ws.list = tab[0];
+        ws.n_layer = tab[7]; ws.list_layer = tab[0]; ws.list_lm = tab[5];
+        ws.total = static_cast<unsigned>(tab[7]) * p.n_layers + tab[6];
     }
-    ws.slot = 0; ws.round = 0; ws.consumed = 0; ws.pending = 0;
+    ws.slot = 0; ws.round = 0; ws.consumed = 0;
     ws.fenced_op = -1;
     bool ok = true;
     const int rt = p.req->token, rp = p.req->position;
@@ -1042,8 +1059,8 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
     const int pos = rp >= 0 ? rp : p.state->next_position;
     const int slot_row = p.state->cur_len;
     const int half = p.d >> 1;
-    if (token < 0 || token >= p.V || slot_row < 0 || slot_row >= p.max_context || pos < 0) {
-        if (tid == 0) diag_fail(p, abort_flag, 3, token, slot_row);   // corrupt request/state: compute nothing
+    if (token < 0 || token >= p.V || slot_row < 0 || slot_row >= p.max_context || pos < 0 || (smem_u32(sm_ring(p, 0)) & 1023u)) {
+        if (tid == 0) diag_fail(p, abort_flag, 3, token, slot_row);   // corrupt request/state (or ring slots off their 1 KB boundary): compute nothing
         ok = false;
     }
     if (ok && tid < half) {  // rotary table of this step's position; fp64 angle, rounded once
@@ -1053,6 +1070,15 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
         s_rope[half + tid] = static_cast<float>(sn);
     }
     if (ok && cta == 0 && tid == 0) { p.state->token = token; p.state->position = pos; }
+    if (ok && cta == 1 % ncta && p.nph > 2) {
+        // the MLP activation arrays in global memory are read in whole 256-column pieces: columns F.. of the last piece are zero
+        // (the gate/up epilogues, grid barriers later, write columns < F only)
+        const int fpad = (p.F + MK_TILE_COLS - 1) / MK_TILE_COLS * MK_TILE_COLS;
+        uint16_t *a = reinterpret_cast<uint16_t *>(sm_ops(p)[2].out);
+        for (int c = p.F + tid; c < fpad; c += MK_NT)
+#pragma unroll
+            for (int sp = 0; sp < MK_X_SPLITS; ++sp) a[static_cast<size_t>(sp) * fpad + mk_xs_index(c)] = 0;
+    }
     // (s_rope is published by the sync of the first prologue)
 
     // start this warp's weight stream: fill its ring
@@ -1065,7 +1091,6 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
 
     unsigned bar_no = 0;
     const unsigned bar_arrivals = static_cast<unsigned>(ncta + p.barrier_extra);
-    unsigned x_parity = 0;
     int prof_idx = 0;
     prof_stamp(p, tid, prof_idx);
     const int n_att = slot_row + 1;
@@ -1076,7 +1101,6 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
     // (the code of a step is executed once per layer: a small instruction footprint matters).  Operator 4l+1 (the O
     // projection) is preceded by the attention of layer l.
     const int n_layer_ops = 4 * p.n_layers;
-    auto refill = [&]() { if (!refill_pending(p, ws, abort_flag, s_issued, full_bar, warp, lane)) *abort_flag = 1; };
     for (int ph = 0; ph < p.nph && ok; ++ph) {
         const bool layer_op = ph < n_layer_ops;
         const bool after_attention = layer_op && (ph & 3) == 1;
@@ -1090,12 +1114,12 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
             } else {
                 attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, sm_xbuf(p), tid, &s_flag);
             }
-            ok = grid_barrier(p, ++bar_no * bar_arrivals, abort_flag, tid, prof_idx, refill) && ok;
+            ok = grid_barrier(p, ++bar_no * bar_arrivals, abort_flag, tid, prof_idx) && ok;
             if (!ok) break;
         }
         ok = gemv_phase(p, ph, layer_op ? (ph & 3) : 4, ws, abort_flag, s_part, s_partial, s_rope, cx, token, after_attention ? merge_chunks : 0, tid,
-                        prof_idx, &x_bar, x_parity, s_issued, full_bar);
-        if (layer_op) ok = grid_barrier(p, ++bar_no * bar_arrivals, abort_flag, tid, prof_idx, refill) && ok;
+                        prof_idx, s_issued, full_bar);
+        if (layer_op) ok = grid_barrier(p, ++bar_no * bar_arrivals, abort_flag, tid, prof_idx) && ok;
     }
     prof_stamp(p, tid, prof_idx);
     if (!ok || *abort_flag) {

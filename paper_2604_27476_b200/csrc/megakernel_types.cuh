@@ -14,13 +14,22 @@ constexpr int MK_ATT_TILE = 32 / MK_ATT_LPP;     // positions per warp iteration
 constexpr int MK_ATT_SPLIT_MAXC = MK_ATT_SPLIT_MAXC_VALUE;   // chunks per head when every query head has its own CTAs
 constexpr int MK_PARTIAL_SLOTS = 48;             // shared-memory scratch: partial row sums, 16 floats per slot
 constexpr int MK_PARTIAL_FLOATS = MK_PARTIAL_SLOTS * 16;   // (also the chunk statistics of the attention merge)
-constexpr int MK_TILE_COLS = 256;                // columns of a weight tile: one 16-byte piece per lane
-constexpr int MK_TILE_ROWS = 16;                 // accumulator rows of a consumer warp (largest tile: 16 x 256 bf16 = 8 KB)
+constexpr int MK_TILE_COLS = 256;                // columns of a weight tile: four blocks of 64 columns (128-byte rows, the swizzle span)
+constexpr int MK_TILE_ROWS = 16;                 // rows of a tile: the M of one m16n8k16 tensor-core instruction (largest tile: 8 KB)
+constexpr int MK_X_SPLITS = 3;                   // an fp32 activation is staged as the sum of three bf16 pieces (24 mantissa bits)
+constexpr int MK_XS_PAD = 64;                    // bytes between the three staged arrays beyond the row length (bank spread)
+constexpr int MK_WBUF_BYTES = MK_X_SPLITS * (MK_TILE_COLS * 2 + MK_XS_PAD);   // a consumer warp's buffer for one tile's worth of a vector read from global memory
 constexpr int MK_MAX_VARIANTS = 4;               // tensor maps (box heights) per weight matrix
 constexpr int MK_MAX_SLOTS = 4;                  // ring slots per consumer warp
 constexpr int MK_WARP_TAB = 8;                   // ints per warp in the per-CTA table
 // Consumer warps per CTA of the two builds of the kernel (one more warp prefetches into L2): the short-context build favours
 // instruction streams, the long-context build (grouped attention keeps G heads of accumulators per warp) registers.
+#ifndef MK_PF_TILES
+#define MK_PF_TILES 4   // tiles per consumer warp the helper warp asks L2 for ahead of the ring
+#endif
+#ifndef MK_PF_TILES_LM
+#define MK_PF_TILES_LM 8   // the same within the output layer
+#endif
 #ifndef MK_NW_SHORT_VALUE
 #define MK_NW_SHORT_VALUE 11
 #endif
@@ -36,9 +45,20 @@ enum { PH_QKV = 0, PH_RESID = 1, PH_SWIGLU = 2, PH_LMHEAD = 3 };
 // MkOp::flags
 enum : int {
     PHF_REMAP = 1,      // PH_LMHEAD: rows are a vocabulary subset; row r stands for token MkParams::vocab_ids[r]
-    PHF_OUT_SPLIT = 2,  // PH_SWIGLU: the output vector is stored as [even 16-byte pieces | odd 16-byte pieces]
-    PHF_X_BULK = 4,     // the input vector has that layout already and needs no transform: staged by two bulk copies
+    PHF_OUT_SPLIT = 2,  // PH_SWIGLU: the output vector is stored the way the next operator reads it: three bf16 arrays
+                        // [3][F rounded up to 256] (the pieces of every value) in tensor-core fragment order (mk_xs_index)
+    PHF_X_GLOBAL = 4,   // the input vector has that form already: the consumer warps read their B fragments straight from
+                        // global memory (L2), a tile ahead; nothing is staged in shared memory
+    PHF_RAGGED = 8,     // K is not a multiple of 64: the tile's four 64-column blocks are fetched by one copy each
 };
+
+// Position of column c in a staged activation array.  The columns of every group of 32 are reordered so that the two 32-bit
+// B-fragment registers of two consecutive k-steps of mma.m16n8k16 are one 16-byte piece per lane quad index q:
+// [q][k-step parity][k half][2 values].
+__host__ __device__ inline int mk_xs_index(int c) {
+    const int kk = c & 15;
+    return (c & ~31) + ((kk & 7) >> 1) * 8 + ((c >> 4) & 1) * 4 + (kk >> 3) * 2 + (kk & 1);
+}
 
 // One weight-streaming operator of the step (its weights are reached through tensor maps, see MkParams::maps).
 struct alignas(16) MkOp {
@@ -57,20 +77,22 @@ static_assert(sizeof(MkOp) % 16 == 0, "descriptor is copied in 16-byte pieces");
 
 // ---- the tile schedule ------------------------------------------------------------------------------------------
 // A tile is a box of m rows x 256 columns of one weight matrix (for PH_QKV / PH_SWIGLU: m "low" rows and their m
-// partner rows, two boxes), fetched by one TMA tensor copy per box into a ring slot of the consumer warp that owns it.
+// partner rows), fetched by one TMA tensor copy into a ring slot of the consumer warp that owns it, where it lies as
+// [4 column blocks][partner][m][128 bytes] with the 128-byte swizzle (conflict-free ldmatrix reads).
 // The host lays out, for every CTA and every consumer warp, the list of tiles of one layer (operators in order) and of
 // the output layer; the lists are the same for every layer.  8 bytes per tile:
 //   x: unit_base [0,20) | column piece [20,28) | tensor-map variant [28,30) | FIRST 30 | FLUSH 31
-//   y: m [0,5) | first valid unit v0 [5,9) | DIRECT 9 | partial slot [10,20) | operator in layer (4 = output layer) [20,23)
+//   y: m [0,5) | first valid unit v0 [5,9) | DIRECT 9 | partial slot [10,20) | operator in layer (4 = output layer) [20,23) |
+//      RAGGED 23 (K is not a multiple of 64: the tile is fetched as four copies, see PHF_RAGGED)
 // FIRST: the warp's accumulators start at zero with this tile.  FLUSH: after this tile the 16 row sums are reduced
 // across the lanes; DIRECT: the warp has seen all columns of these rows and finishes them itself; otherwise the sums
 // go to partial slot `slot` and the units are finished after the operator by summing their slots in order.
-constexpr uint32_t MKT_FIRST = 1u << 30, MKT_FLUSH = 1u << 31, MKT_DIRECT = 1u << 9;
+constexpr uint32_t MKT_FIRST = 1u << 30, MKT_FLUSH = 1u << 31, MKT_DIRECT = 1u << 9, MKT_RAGGED = 1u << 23;
 __host__ __device__ inline uint2 mk_tile_desc(uint32_t unit_base, uint32_t kcol, uint32_t variant, bool first, bool flush, uint32_t m,
-                                              uint32_t v0, bool direct, uint32_t slot, uint32_t op) {
+                                              uint32_t v0, bool direct, uint32_t slot, uint32_t op, bool ragged = false) {
     uint2 d;
     d.x = (unit_base & 0xfffffu) | (kcol & 0xffu) << 20 | (variant & 3u) << 28 | (first ? MKT_FIRST : 0u) | (flush ? MKT_FLUSH : 0u);
-    d.y = (m & 31u) | (v0 & 15u) << 5 | (direct ? MKT_DIRECT : 0u) | (slot & 1023u) << 10 | (op & 7u) << 20;
+    d.y = (m & 31u) | (v0 & 15u) << 5 | (direct ? MKT_DIRECT : 0u) | (slot & 1023u) << 10 | (op & 7u) << 20 | (ragged ? MKT_RAGGED : 0u);
     return d;
 }
 // Units whose row sums were left in partial slots: unit_base, m | v0 << 8, first slot, number of slots.

@@ -109,7 +109,7 @@ inline const char *plan_op(const OpShape &os, int op_index, int ncta, int nw, in
                 }
                 for (int k = k0; k < k1; ++k)
                     S.tiles[c][w].push_back(mk_tile_desc(blocks[b].u0, k, blocks[b].variant, k == k0, k == k1 - 1, blocks[b].m, blocks[b].v0,
-                                                         direct, slot, op_index));
+                                                         direct, slot, op_index, os.K % 64 != 0));
                 t += k1 - k0;
             }
         }
@@ -200,19 +200,28 @@ inline TensorMapEncodeFn tensor_map_encoder() {
     return fn;
 }
 
-// Tensor map of a row-major bf16 [rows][K] matrix on THIS GPU with boxes of box_rows x 256 elements; columns and rows
-// outside the matrix read as zero.  (No multicast is ever used with these maps.)
-//   pair_rows == 0                : 2-D, coordinates (column, row);
-//   pair_rows  > 0, group == 0    : 3-D view [2][pair_rows][K] (gate rows, up rows): one box = box_rows low rows and their partners;
-//   pair_rows  > 0, group  > 0    : 4-D view [rows / (2 pair_rows)][2][pair_rows][K] (heads of the QKV matrix: rotate-half partners).
+// Tensor map of a row-major bf16 [rows][K] matrix on THIS GPU.  A box is box_rows rows x 256 columns, delivered to shared
+// memory as four blocks of 64 columns ([block][rows][128 bytes], 128-byte swizzle); columns and rows outside the matrix read as
+// zero.  The 64-column blocks of a row are the LAST dimension of the map (stride 128 bytes), so the column coordinate is
+// always 0 and the block coordinate is 4 * (column piece).  (No multicast is ever used with these maps.)
+//   pair_rows == 0                : (0, row, block);
+//   pair_rows  > 0, !grouped      : view [2][pair_rows][K] (gate rows, up rows): (0, row, 0, block), a box = box_rows low rows
+//                                   and their partners;
+//   pair_rows  > 0, grouped       : view [rows / (2 pair_rows)][2][pair_rows][K] (heads of the QKV matrix, rotate-half partners):
+//                                   (0, row in half, 0, head, block).
+// K not a multiple of 64: the block dimension is left out (its last block would reach into the next row); the map's first
+// dimension is then the K columns, a box is ONE 64-column block, and the caller copies the four blocks of a tile one by one.
 inline bool encode_weight_map(CUtensorMap *m, const void *base, int rows, int K, int box_rows, int pair_rows = 0, bool grouped = false) {
     TensorMapEncodeFn enc = tensor_map_encoder();
     if (!enc) return false;
     const cuuint64_t row_bytes = static_cast<cuuint64_t>(K) * 2;
-    cuuint64_t dims[4] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(rows), 1, 1};
-    cuuint64_t strides[3] = {row_bytes, 0, 0};
-    cuuint32_t box[4] = {MK_TILE_COLS, static_cast<cuuint32_t>(box_rows), 1, 1};
-    const cuuint32_t es[4] = {1, 1, 1, 1};
+    const bool ragged = K % 64 != 0;
+    // dimensions, innermost first: 64 columns (or all K columns when K has a ragged last block), rows [, partner, head],
+    // and last the 64-column blocks of a row (128 bytes apart), so that a box lands block by block
+    cuuint64_t dims[5] = {static_cast<cuuint64_t>(ragged ? K : 64), static_cast<cuuint64_t>(rows), 1, 1, 1};
+    cuuint64_t strides[4] = {row_bytes, 0, 0, 0};
+    cuuint32_t box[5] = {64, static_cast<cuuint32_t>(box_rows), 1, 1, 1};
+    const cuuint32_t es[5] = {1, 1, 1, 1, 1};
     cuuint32_t rank = 2;
     if (pair_rows > 0) {
         dims[1] = static_cast<cuuint64_t>(pair_rows); dims[2] = 2;
@@ -225,8 +234,14 @@ inline bool encode_weight_map(CUtensorMap *m, const void *base, int rows, int K,
             rank = 4;
         }
     }
+    if (!ragged) {
+        dims[rank] = static_cast<cuuint64_t>(K / 64);
+        strides[rank - 1] = 128;
+        box[rank] = MK_TILE_COLS / 64;
+        ++rank;
+    }
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void *>(base), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
-               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace edgefm
