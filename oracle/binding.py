@@ -62,6 +62,14 @@ def lib():
         L.oracle_model_cur_len.argtypes = [_p]
         L.oracle_model_export_kv.restype = None
         L.oracle_model_export_kv.argtypes = [_p, _p, _p]
+        L.oracle_model_use_int8_kv.restype = ctypes.c_int
+        L.oracle_model_use_int8_kv.argtypes = [_p]
+        L.oracle_quantize_row.restype = None
+        L.oracle_quantize_row.argtypes = [_p, _i64, _p, _p]
+        L.oracle_attention_q8.restype = None
+        L.oracle_attention_q8.argtypes = [_p, _p, _p, _p, _p, _i64, _i64, _i64, _i64, _p]
+        L.oracle_model_export_kv_q8.restype = None
+        L.oracle_model_export_kv_q8.argtypes = [_p, _p, _p, _p, _p]
         L.oracle_model_step.restype = _i64
         L.oracle_model_step.argtypes = [_p, _i64, _i64, _p]
         _lib = L
@@ -144,12 +152,35 @@ def attention(q: np.ndarray, K: np.ndarray, V: np.ndarray) -> np.ndarray:
     return out
 
 
+def quantize_row(x: np.ndarray) -> tuple[np.ndarray, float]:
+    """Compression of one cache row (Sec. 3.9, C): fp32 [d] -> (int8 codes [d], fp32 scale)."""
+    x = _f32(x)
+    codes = np.empty(x.size, np.int8)
+    scale = np.zeros(1, np.float32)
+    lib().oracle_quantize_row(x.ctypes.data, x.size, codes.ctypes.data, scale.ctypes.data)
+    return codes, float(scale[0])
+
+
+def attention_q8(q: np.ndarray, K8: np.ndarray, Ks: np.ndarray, V8: np.ndarray, Vs: np.ndarray) -> np.ndarray:
+    """q fp32 [n_q][d]; K8, V8 int8 [n_kv][n][d]; Ks, Vs fp32 [n_kv][n] -> fp32 [n_q][d]."""
+    q = _f32(q)
+    K8 = np.ascontiguousarray(K8, np.int8); V8 = np.ascontiguousarray(V8, np.int8)
+    Ks = _f32(Ks); Vs = _f32(Vs)
+    n_q, d = q.shape
+    n_kv, n, d2 = K8.shape
+    assert d2 == d and V8.shape == K8.shape and Ks.shape == (n_kv, n) and Vs.shape == (n_kv, n)
+    out = np.empty_like(q)
+    lib().oracle_attention_q8(q.ctypes.data, K8.ctypes.data, Ks.ctypes.data, V8.ctypes.data, Vs.ctypes.data, n_q, n_kv, d, n, out.ctypes.data)
+    return out
+
+
 class OracleModel:
     """Whole decoder with its own KV cache.  `weights` is the dict edgefm_synth.make_weights returns
     (or any dict of the same layout); the arrays are borrowed and kept alive here."""
 
-    def __init__(self, cfg, weights: dict, max_context: int):
+    def __init__(self, cfg, weights: dict, max_context: int, kv_format: str = "bf16"):
         self.cfg = cfg
+        self.kv_format = kv_format
         self._keep = weights
         ptrs = []
         for lw in weights["layers"]:
@@ -164,6 +195,11 @@ class OracleModel:
         if not self._h:
             raise MemoryError("oracle_model_create failed")
         self.max_context = max_context
+        if kv_format == "int8":
+            if lib().oracle_model_use_int8_kv(self._h):
+                raise RuntimeError("oracle_model_use_int8_kv failed")
+        elif kv_format != "bf16":
+            raise ValueError(kv_format)
 
     def load_kv(self, k: np.ndarray, v: np.ndarray) -> None:
         k = np.ascontiguousarray(k, np.uint16)
@@ -183,6 +219,15 @@ class OracleModel:
         v = np.empty(shape, np.uint16)
         lib().oracle_model_export_kv(self._h, k.ctypes.data, v.ctypes.data)
         return k, v
+
+    def export_kv_q8(self):
+        """-> (K codes int8, V codes int8 [L][n_kv][max_context][d], K scales fp32, V scales fp32 [L][n_kv][max_context])."""
+        c = self.cfg
+        shape = (c.n_layers, c.n_kv_heads, self.max_context, c.head_dim)
+        k8 = np.empty(shape, np.int8); v8 = np.empty(shape, np.int8)
+        ks = np.empty(shape[:3], np.float32); vs = np.empty(shape[:3], np.float32)
+        lib().oracle_model_export_kv_q8(self._h, k8.ctypes.data, v8.ctypes.data, ks.ctypes.data, vs.ctypes.data)
+        return k8, v8, ks, vs
 
     def step(self, token: int, pos: int):
         """-> (logits fp32[V], next_token)."""

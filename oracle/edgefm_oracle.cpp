@@ -19,6 +19,13 @@
 //     written included, as rounded to bf16), no mask.
 //   * new k (after RoPE) and v are rounded to bf16 (round to nearest even) when appended.
 //   * greedy sampling (Sec. 4.2: temperature 0, top_k = 1): lowest index among the maxima.
+//   * compressed cache (Sec. 3.9, KV~ = C(KV) with on-demand reconstruction; the paper fixes no C): every cached
+//     row (one position of one kv head, d values) of K and of V is stored as d signed 8-bit codes and one fp32 scale,
+//     scale = amax / 127, code_j = clamp(rint(x_j * (127 / amax)), -127, 127), both evaluated in fp32 (a
+//     floating-point value decides an integer here, so the decision is taken in the precision the CUDA path uses);
+//     an all-zero row has scale 0.  Attention reads code * scale (fp32 product) wherever the uncompressed path reads
+//     the bf16 value, the row appended by the step itself included; the appended row is compressed from the fp32 k
+//     (after RoPE) and v, not from a bf16 rounding of them.
 //
 // Parity pins: every function below is pinned by tests/test_oracle_pins.py (closed forms,
 // brute force, invariants) and the whole step by an independent numpy fp64 uncached forward
@@ -130,6 +137,53 @@ void attention(const float *q, const uint16_t *K, const uint16_t *V, int64_t n_q
     }
 }
 
+// C of Sec. 3.9 for one cache row: d values -> d codes and a scale.  fp32 arithmetic on purpose (see the header).
+void quantize_row(const float *x, int64_t d, int8_t *codes, float *scale) {
+    float amax = 0.f;
+    for (int64_t j = 0; j < d; ++j) amax = std::fabs(x[j]) > amax ? std::fabs(x[j]) : amax;
+    if (!(amax > 0.f)) {
+        for (int64_t j = 0; j < d; ++j) codes[j] = 0;
+        *scale = 0.f;
+        return;
+    }
+    const float inv = 127.0f / amax;
+    for (int64_t j = 0; j < d; ++j) {
+        float c = std::nearbyintf(x[j] * inv);   // round to nearest, ties to even (default rounding mode)
+        c = c > 127.f ? 127.f : (c < -127.f ? -127.f : c);
+        codes[j] = static_cast<int8_t>(c);
+    }
+    *scale = amax / 127.0f;
+}
+
+// Attention over a compressed cache: as attention(), every K / V value reconstructed as code * scale (fp32).
+// K8, V8: element (g, t, j) at g * stride_head + t * stride_pos + j;  scales: (g, t) at g * stride_head_s + t.
+void attention_q8(const float *q, const int8_t *K8, const float *Ks, const int8_t *V8, const float *Vs, int64_t n_q, int64_t n_kv,
+                  int64_t d, int64_t n, int64_t stride_head, int64_t stride_pos, int64_t stride_head_s, float *out) {
+    const int64_t group = n_q / n_kv;
+    const double scale = 1.0 / std::sqrt(static_cast<double>(d));
+#pragma omp parallel for schedule(static)
+    for (int64_t h = 0; h < n_q; ++h) {
+        const int64_t g = h / group;
+        const float *qh = q + h * d;
+        std::vector<float> s(n);
+        for (int64_t t = 0; t < n; ++t) {
+            const int8_t *kt = K8 + g * stride_head + t * stride_pos;
+            const float ks = Ks[g * stride_head_s + t];
+            double acc = 0.0;
+            for (int64_t j = 0; j < d; ++j) acc += static_cast<double>(qh[j]) * static_cast<double>(static_cast<float>(kt[j]) * ks);
+            s[t] = static_cast<float>(acc * scale);
+        }
+        softmax(s.data(), n);
+        for (int64_t j = 0; j < d; ++j) {
+            double acc = 0.0;
+            for (int64_t t = 0; t < n; ++t)
+                acc += static_cast<double>(s[t]) *
+                       static_cast<double>(static_cast<float>(V8[g * stride_head + t * stride_pos + j]) * Vs[g * stride_head_s + t]);
+            out[h * d + j] = static_cast<float>(acc);
+        }
+    }
+}
+
 struct LayerW {
     const uint16_t *input_norm, *wqkv, *bqkv, *wo, *post_norm, *w_gate_up, *w_down;
 };
@@ -140,8 +194,12 @@ struct Model {
     std::vector<LayerW> layers;
     const uint16_t *embed, *final_norm, *lm_head;
     std::vector<uint16_t> K, Vc;  // [L][nkv][Tmax][d]
+    bool q8 = false;              // compressed cache: codes [L][nkv][Tmax][d] and scales [L][nkv][Tmax] instead of K, Vc
+    std::vector<int8_t> K8, V8;
+    std::vector<float> Ks, Vs;
     int64_t cur_len = 0;
     int64_t kv_index(int64_t l, int64_t g, int64_t t) const { return ((l * nkv + g) * Tmax + t) * d; }
+    int64_t sc_index(int64_t l, int64_t g, int64_t t) const { return (l * nkv + g) * Tmax + t; }
 };
 
 }  // namespace
@@ -187,6 +245,33 @@ void *oracle_model_create(int64_t n_layers, int64_t hidden, int64_t n_q, int64_t
 
 void oracle_model_destroy(void *h) { delete static_cast<Model *>(h); }
 
+// Switch an empty model to the compressed cache of Sec. 3.9 (before any load or step).
+int oracle_model_use_int8_kv(void *h) {
+    Model *m = static_cast<Model *>(h);
+    if (m->cur_len != 0) return 1;
+    m->q8 = true;
+    m->K8.assign(m->K.size(), 0);
+    m->V8.assign(m->K.size(), 0);
+    m->Ks.assign(static_cast<size_t>(m->L * m->nkv * m->Tmax), 0.f);
+    m->Vs.assign(m->Ks.size(), 0.f);
+    return 0;
+}
+
+void oracle_quantize_row(const float *x, int64_t d, int8_t *codes, float *scale) { quantize_row(x, d, codes, scale); }
+void oracle_attention_q8(const float *q, const int8_t *K8, const float *Ks, const int8_t *V8, const float *Vs, int64_t n_q, int64_t n_kv,
+                         int64_t d, int64_t n, float *out) {
+    attention_q8(q, K8, Ks, V8, Vs, n_q, n_kv, d, n, n * d, d, n, out);
+}
+
+// Codes and scales of the compressed cache in its internal layout: [L][n_kv][max_context][d] and [L][n_kv][max_context].
+void oracle_model_export_kv_q8(void *h, int8_t *k8, int8_t *v8, float *ks, float *vs) {
+    Model *m = static_cast<Model *>(h);
+    std::memcpy(k8, m->K8.data(), m->K8.size());
+    std::memcpy(v8, m->V8.data(), m->V8.size());
+    std::memcpy(ks, m->Ks.data(), m->Ks.size() * 4);
+    std::memcpy(vs, m->Vs.data(), m->Vs.size() * 4);
+}
+
 // Load n positions of K/V (bf16, [L][n_kv][n][d] contiguous, keys already rotated) into slots 0..n-1.
 int oracle_model_load_kv(void *h, const uint16_t *k, const uint16_t *v, int64_t n) {
     Model *m = static_cast<Model *>(h);
@@ -194,6 +279,16 @@ int oracle_model_load_kv(void *h, const uint16_t *k, const uint16_t *v, int64_t 
     for (int64_t l = 0; l < m->L; ++l)
         for (int64_t g = 0; g < m->nkv; ++g) {
             const int64_t src = ((l * m->nkv + g) * n) * m->d;
+            if (m->q8) {   // the given rows are compressed one by one
+                std::vector<float> row(m->d);
+                for (int64_t t = 0; t < n; ++t) {
+                    for (int64_t j = 0; j < m->d; ++j) row[j] = bf16_to_f32(k[src + t * m->d + j]);
+                    quantize_row(row.data(), m->d, &m->K8[m->kv_index(l, g, t)], &m->Ks[m->sc_index(l, g, t)]);
+                    for (int64_t j = 0; j < m->d; ++j) row[j] = bf16_to_f32(v[src + t * m->d + j]);
+                    quantize_row(row.data(), m->d, &m->V8[m->kv_index(l, g, t)], &m->Vs[m->sc_index(l, g, t)]);
+                }
+                continue;
+            }
             std::memcpy(&m->K[m->kv_index(l, g, 0)], k + src, static_cast<size_t>(n * m->d) * 2);
             std::memcpy(&m->Vc[m->kv_index(l, g, 0)], v + src, static_cast<size_t>(n * m->d) * 2);
         }
@@ -227,13 +322,22 @@ int64_t oracle_model_step(void *h, int64_t token, int64_t pos, float *logits_out
         float *q = qkv.data(), *k = q + nq * d, *v = k + nkv * d;
         for (int64_t hh = 0; hh < nq; ++hh) rope(q + hh * d, d, pos, m->theta);
         for (int64_t g = 0; g < nkv; ++g) rope(k + g * d, d, pos, m->theta);
-        for (int64_t g = 0; g < nkv; ++g)
-            for (int64_t j = 0; j < d; ++j) {
-                m->K[m->kv_index(l, g, slot) + j] = f32_to_bf16(k[g * d + j]);
-                m->Vc[m->kv_index(l, g, slot) + j] = f32_to_bf16(v[g * d + j]);
+        if (m->q8) {
+            for (int64_t g = 0; g < nkv; ++g) {
+                quantize_row(k + g * d, d, &m->K8[m->kv_index(l, g, slot)], &m->Ks[m->sc_index(l, g, slot)]);
+                quantize_row(v + g * d, d, &m->V8[m->kv_index(l, g, slot)], &m->Vs[m->sc_index(l, g, slot)]);
             }
-        attention(q, &m->K[m->kv_index(l, 0, 0)], &m->Vc[m->kv_index(l, 0, 0)], nq, nkv, d, slot + 1, m->Tmax * d, d,
-                  attn.data());
+            attention_q8(q, &m->K8[m->kv_index(l, 0, 0)], &m->Ks[m->sc_index(l, 0, 0)], &m->V8[m->kv_index(l, 0, 0)],
+                         &m->Vs[m->sc_index(l, 0, 0)], nq, nkv, d, slot + 1, m->Tmax * d, d, m->Tmax, attn.data());
+        } else {
+            for (int64_t g = 0; g < nkv; ++g)
+                for (int64_t j = 0; j < d; ++j) {
+                    m->K[m->kv_index(l, g, slot) + j] = f32_to_bf16(k[g * d + j]);
+                    m->Vc[m->kv_index(l, g, slot) + j] = f32_to_bf16(v[g * d + j]);
+                }
+            attention(q, &m->K[m->kv_index(l, 0, 0)], &m->Vc[m->kv_index(l, 0, 0)], nq, nkv, d, slot + 1, m->Tmax * d, d,
+                      attn.data());
+        }
         gemv(w.wo, attn.data(), nullptr, H, nq * d, proj.data());
         for (int64_t i = 0; i < H; ++i) x[i] = static_cast<float>(static_cast<double>(x[i]) + static_cast<double>(proj[i]));
         rmsnorm(x.data(), w.post_norm, H, m->eps, xn.data());

@@ -41,8 +41,20 @@ def _rope_all(u, positions, theta):
     return _f32(np.concatenate([a * c - b * s, b * c + a * s], axis=-1))
 
 
-def full_forward(cfg, weights: dict, tokens, positions) -> np.ndarray:
-    """Logits fp64 [T][V] of a causal forward over all tokens at once, starting from an empty cache."""
+def _int8_rows(x64: np.ndarray) -> np.ndarray:
+    """Compression of Sec. 3.9 as the oracle reads it, written with numpy fp32 array operations: per row (last axis)
+    scale = amax / 127, code = clip(rint(x * (127 / amax))), value seen by attention = code * scale."""
+    x = x64.astype(np.float32)
+    amax = np.abs(x).max(axis=-1, keepdims=True)
+    safe = np.where(amax > 0, amax, np.float32(1))
+    codes = np.clip(np.rint(x * (np.float32(127) / safe)), -127, 127).astype(np.float32)
+    scale = np.where(amax > 0, amax / np.float32(127), np.float32(0)).astype(np.float32)
+    return (codes * scale).astype(np.float64)
+
+
+def full_forward(cfg, weights: dict, tokens, positions, kv_int8: bool = False) -> np.ndarray:
+    """Logits fp64 [T][V] of a causal forward over all tokens at once, starting from an empty cache.
+    kv_int8: k (after RoPE) and v pass through the 8-bit row compression instead of the bf16 rounding."""
     T = len(tokens)
     nq, nkv, d, F = cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.ffn
     G = nq // nkv
@@ -57,7 +69,7 @@ def full_forward(cfg, weights: dict, tokens, positions) -> np.ndarray:
         q = _rope_all(qkv[:, : nq * d].reshape(T, nq, d), positions, cfg.rope_theta)
         k = _rope_all(qkv[:, nq * d: (nq + nkv) * d].reshape(T, nkv, d), positions, cfg.rope_theta)
         v = qkv[:, (nq + nkv) * d:].reshape(T, nkv, d)
-        k, v = _round_bf16(k), _round_bf16(v)
+        k, v = (_int8_rows(k), _int8_rows(v)) if kv_int8 else (_round_bf16(k), _round_bf16(v))
         kq = np.repeat(k, G, axis=1)                                           # kv head h//G for q head h
         vq = np.repeat(v, G, axis=1)
         s = _f32(np.einsum("thd,shd->hts", q, kq) / np.sqrt(d))

@@ -296,6 +296,83 @@ def test_cached_decoding_equals_full_causal_recompute(variant):
     assert m.cur_len == T
 
 
+# ---- compressed cache (Sec. 3.9: KV~ = C(KV), reconstruction on demand) ---------------------------------------
+def test_int8_row_compression_worked_example_and_properties():
+    # by hand: amax = 2, 127 / 2 = 63.5;  1 -> 63.5 -> 64 (tie to even), -2 -> -127, 0.5 -> 31.75 -> 32, 0 -> 0;  scale = 2 / 127
+    codes, scale = O.quantize_row(np.array([1.0, -2.0, 0.5, 0.0], np.float32))
+    assert codes.tolist() == [64, -127, 32, 0]
+    assert scale == np.float32(2.0) / np.float32(127.0)
+    codes, scale = O.quantize_row(np.zeros(8, np.float32))
+    assert codes.tolist() == [0] * 8 and scale == 0.0
+    rng = np.random.default_rng(5)
+    for d in (4, 64, 128):
+        x = rng.standard_normal(d).astype(np.float32) * np.float32(rng.uniform(1e-3, 50))
+        codes, scale = O.quantize_row(x)
+        assert np.abs(codes).max() == 127 and np.abs(codes[np.argmax(np.abs(x))]) == 127      # the largest value takes the end of the range
+        assert np.abs(codes.astype(np.float64) * scale - x).max() <= scale * 0.5 * (1 + 1e-6)   # nearest code
+        c2, s2 = O.quantize_row(-x)
+        assert (c2 == -codes).all() and s2 == scale                                              # odd symmetry
+        c3, s3 = O.quantize_row(x * np.float32(4))                                               # a power of two moves the scale only
+        assert (c3 == codes).all() and s3 == scale * np.float32(4)
+
+
+def test_attention_over_compressed_cache_reduces_to_plain_attention_on_exact_rows():
+    # rows of integers with amax 127, times a power of two, compress without loss (codes = integers, scale = the power of
+    # two) and are exact in bf16 as well: both attention routines must then see the same numbers
+    rng = np.random.default_rng(6)
+    n_q, n_kv, d, n = 4, 2, 32, 9
+    Ki = rng.integers(-127, 128, (n_kv, n, d)); Vi = rng.integers(-127, 128, (n_kv, n, d))
+    Ki[..., 0] = 127; Vi[..., 1] = -127                                    # every row reaches the end of the range
+    sk = 2.0 ** rng.integers(-6, 0, (n_kv, n)); sv = 2.0 ** rng.integers(-4, 2, (n_kv, n))
+    K = (Ki * sk[..., None]).astype(np.float32); V = (Vi * sv[..., None]).astype(np.float32)
+    q = rng.standard_normal((n_q, d)).astype(np.float32)
+    K8 = np.empty_like(Ki, dtype=np.int8); V8 = np.empty_like(Vi, dtype=np.int8)
+    Ks = np.empty((n_kv, n), np.float32); Vs = np.empty((n_kv, n), np.float32)
+    for g in range(n_kv):
+        for t in range(n):
+            K8[g, t], Ks[g, t] = O.quantize_row(K[g, t])
+            V8[g, t], Vs[g, t] = O.quantize_row(V[g, t])
+    assert (K8 == Ki).all() and (V8 == Vi).all() and (Ks == sk).all() and (Vs == sv).all()
+    to_bits = lambda a: (a.view(np.uint32) >> 16).astype(np.uint16)
+    assert ((to_bits(K).astype(np.uint32) << 16).view(np.float32) == K).all()           # exact in bf16
+    plain = O.attention(q, to_bits(K), to_bits(V))
+    comp = O.attention_q8(q, K8, Ks, V8, Vs)
+    assert np.array_equal(plain, comp)
+
+
+@pytest.mark.parametrize("variant", ["plain", "bias_gqa"])
+def test_cached_decoding_with_compressed_cache_equals_full_causal_recompute(variant):
+    cfg = TINY if variant == "plain" else TINY.with_(qkv_bias=True, n_layers=3)
+    w = make_weights(cfg, seed=13)
+    rng = np.random.default_rng(14)
+    T = 12
+    toks = rng.integers(0, cfg.vocab, T).tolist()
+    pos = (np.arange(T) + 7).tolist()
+    m = OracleModel(cfg, w, T, kv_format="int8")
+    got = np.stack([m.step(t, p)[0] for t, p in zip(toks, pos)])
+    ref = tiny_ref.full_forward(cfg, w, toks, pos, kv_int8=True)
+    assert np.abs(got - ref).max() < 1e-5
+    # and the compression is visible: the same run over the bf16 cache differs by far more than that
+    plain = tiny_ref.full_forward(cfg, w, toks, pos)
+    assert np.abs(plain - ref).max() > 1e-4
+    k8, v8, ks, vs = m.export_kv_q8()
+    assert np.abs(k8[:, :, :T]).max(axis=-1).min() == 127 and (ks[:, :, :T] > 0).all()
+
+
+def test_compressed_cache_load_compresses_the_given_rows(tiny_weights):
+    from edgefm_synth import make_kv
+    cfg, w = TINY, tiny_weights
+    k, v = make_kv(cfg, n_positions=5)
+    m = OracleModel(cfg, w, 8, kv_format="int8")
+    m.load_kv(k, v)
+    k8, v8, ks, vs = m.export_kv_q8()
+    for (l, g, t) in [(0, 0, 0), (1, 1, 4), (0, 1, 2)]:
+        row = (k[l, g, t].astype(np.uint32) << 16).view(np.float32)
+        codes, scale = O.quantize_row(row)
+        assert (k8[l, g, t] == codes).all() and ks[l, g, t] == scale
+    assert (k8[:, :, 5:] == 0).all() and (vs[:, :, 5:] == 0).all() and m.cur_len == 5
+
+
 def test_position_is_independent_of_slot(tiny_weights):
     # Same cache content, same token, different RoPE position => different logits; the slot written
     # is cur_len in both cases (vision-token prefixes make position != slot).
