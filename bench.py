@@ -116,10 +116,10 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def time_oracle(cfg, weights, k, v, steps: int, warmup: int):
+def time_oracle(cfg, weights, k, v, steps: int, warmup: int, kv_format: str = "bf16"):
     """The CPU oracle as it stands, on the host cores: `steps` decode steps from the configured cache."""
     from oracle import OracleModel
-    m = OracleModel(cfg, weights, cfg.cache_len + steps + warmup)
+    m = OracleModel(cfg, weights, cfg.cache_len + steps + warmup, kv_format=kv_format)
     m.load_kv(k, v)
     tok, pos = first_token(cfg), cfg.first_position
     for _ in range(warmup):
@@ -139,12 +139,12 @@ def run_reference(args, cfg, rank):
     os.environ["OMP_NUM_THREADS"] = str(cores)
     weights = make_weights(cfg)
     k, v = make_kv(cfg)
-    ms = time_oracle(cfg, weights, k, v, args.steps, args.warmup)
+    ms = time_oracle(cfg, weights, k, v, args.steps, args.warmup, args.kv_format)
     sample = f"{args.steps} full oracle decode steps of {cfg.name} from a {cfg.cache_len}-position cache (fp64 accumulation)"
     line = {"impl": "reference", "metric": METRIC, "value": ms, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
             "dtype": "f64 accumulate over bf16 weights", "data": "synthetic",
-            "config": config_block(cfg, workload_name(cfg), 1),
+            "config": config_block(cfg, workload_name(cfg, args.kv_format), 1),
             "cpu_baseline": {"value": ms, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": ms, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
@@ -174,8 +174,15 @@ def per_token_stats(seq_ms, steps, world):
     return statistics.median(per), per[0]
 
 
-def workload_name(cfg):
-    return (f"{cfg.name}-shaped decoder, batch 1, {cfg.cache_len}-position bf16 KV cache, greedy decode steps "
+def kv_saved_bytes(cfg, cur_len: int) -> int:
+    """Bytes the compressed cache (head_dim codes + one fp32 scale per row instead of 2 head_dim bytes) saves per step at
+    cache length cur_len: cur_len + 1 rows of K and of V read and one written, per layer and kv head."""
+    return 2 * cfg.n_layers * cfg.n_kv_heads * (cfg.head_dim - 4) * (cur_len + 2)
+
+
+def workload_name(cfg, kv_format="bf16"):
+    cache = "bf16" if kv_format == "bf16" else "compressed (8-bit codes + fp32 scale per row)"
+    return (f"{cfg.name}-shaped decoder, batch 1, {cfg.cache_len}-position {cache} KV cache, greedy decode steps "
             f"(L={cfg.n_layers} H={cfg.hidden} heads={cfg.n_q_heads}/{cfg.n_kv_heads} d={cfg.head_dim} F={cfg.ffn} V={cfg.vocab})")
 
 
@@ -193,6 +200,8 @@ def main():
     ap.add_argument("--warmup-sequences", type=int, default=3, help="untimed sequences before the timed ones (besides --warmup steps)")
     ap.add_argument("--vocab-subset", type=int, default=0,
                     help="prune the output layer to this many evenly spaced token ids (0 = full vocabulary, the headline workload)")
+    ap.add_argument("--kv-format", default="bf16", choices=["bf16", "int8"],
+                    help="cache format: int8 = the compressed cache (edgefm_create_with_options); not the headline configuration")
     ap.add_argument("--phase-timeline", action="store_true",
                     help="instead of the benchmark: print the per-operator timeline of one step from the kernel's own device timestamps")
     args = ap.parse_args()
@@ -229,7 +238,7 @@ def main():
     k, v = make_kv(cfg)
     ptrs, keep = upload_weights(weights, dev)
     span = max(steps, warmup, 1)
-    ctx = DecodeContext(cfg, ptrs, cfg.cache_len + span, dev)
+    ctx = DecodeContext(cfg, ptrs, cfg.cache_len + span, dev, kv_format=None if args.kv_format == "bf16" else args.kv_format)
     kd = torch.from_numpy(k.view(np.int16)).to(dev)
     vd = torch.from_numpy(v.view(np.int16)).to(dev)
     stream = torch.cuda.current_stream().cuda_stream
@@ -241,7 +250,7 @@ def main():
         ctx.set_vocab_subset(ids)
         n_sub = int(ids.size)
     pruned_bytes = (cfg.vocab - n_sub) * cfg.hidden * 2 if n_sub else 0      # lm_head rows the pruned step does not read
-    workload = workload_name(cfg) + (f", output layer pruned to {n_sub} of {cfg.vocab} token ids" if n_sub else "")
+    workload = workload_name(cfg, args.kv_format) + (f", output layer pruned to {n_sub} of {cfg.vocab} token ids" if n_sub else "")
 
     def free_run(n):
         """n chained greedy steps, token and position carried on the device (one graph launch per token)."""
@@ -303,21 +312,23 @@ def main():
         tokens = steps * world
         ms_per_token, ms_per_token_min = per_token_stats(seq_ms, steps, world)
         dev_ms = ms_per_token * tokens                                   # median sequence time
-        bytes_per_step = float(np.mean([cfg.step_bytes(cfg.cache_len + i) for i in range(steps)])) - pruned_bytes
+        bytes_per_step = float(np.mean([cfg.step_bytes(cfg.cache_len + i) - (kv_saved_bytes(cfg, cfg.cache_len + i) if args.kv_format == "int8" else 0)
+                                        for i in range(steps)])) - pruned_bytes
         gbs = bytes_per_step / (dev_ms / steps * 1e-3) / 1e9          # per GPU
         peak, peak_src = measured_peak()
-        traffic, traffic_src = (None, None) if n_sub else ncu_traffic(cfg.name)
+        traffic, traffic_src = (None, None) if (n_sub or args.kv_format != "bf16") else ncu_traffic(cfg.name)
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
             cores = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
-            cpu_ms = time_oracle(cfg, weights, k, v, args.cpu_steps, 1)
+            cpu_ms = time_oracle(cfg, weights, k, v, args.cpu_steps, 1, args.kv_format)
             cpu = {"value": cpu_ms, "unit": UNIT, "cores": cores, "kind": "oracle",
                    "sample": f"{args.cpu_steps} full oracle decode steps at context {cfg.cache_len} (after 1 warm-up step)"
                              + ("; the oracle computes the whole output layer and restricts afterwards" if n_sub else "")}
         line = {
             "metric": METRIC, "value": ms_per_token, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
             "ms_per_step": dev_ms / steps, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16 weights/KV, fp32 accumulate", "data": "synthetic",
+            "dtype": "bf16 weights/KV, fp32 accumulate" if args.kv_format == "bf16" else "bf16 weights, 8-bit KV codes with fp32 row scales, fp32 accumulate",
+            "data": "synthetic",
             "config": config_block(cfg, workload, world, pruned_bytes),
             "timed_sequences": n_seq, "ms_per_token_min": ms_per_token_min,
             "tokens_per_s": tokens / (dev_ms * 1e-3),

@@ -89,6 +89,28 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
                             edgefm_ctx **out);
 
 /*
+ * edgefm_create_with_options -- edgefm_create with a choice of cache format (Sec. 3.9, "KV Cache Compression":
+ * KV~ = C(KV) with on-demand reconstruction; the paper leaves C open).
+ *   options->kv_format = EDGEFM_KV_BF16 : the plain cache of edgefm_create (options == NULL means the same);
+ *                        EDGEFM_KV_INT8 : every cached row (one position of one kv head, head_dim values) of K and of V is
+ *     kept as head_dim signed 8-bit codes and one fp32 scale: scale = amax / 127, code_j = clamp(rint(x_j * (127 / amax)),
+ *     -127, 127), both in fp32 (round to nearest even; an all-zero row has scale 0).  Attention multiplies with
+ *     code * scale wherever the plain cache is read, the row appended by the step itself included; that row is
+ *     compressed from the fp32 k (after RoPE) and v.  Rows given to edgefm_prefill_kv / edgefm_append_kv (bf16) are
+ *     compressed as they are copied in.  The cache takes head_dim + 4 bytes per row instead of 2 head_dim.
+ *     edgefm_export_kv is refused on such a context (use edgefm_export_kv_int8), and so is edgefm_decode_step_static.
+ *   options->reserved must be zero.
+ * Errors: as edgefm_create; INVALID_ARG for an unknown format or non-zero reserved fields.
+ */
+enum { EDGEFM_KV_BF16 = 0, EDGEFM_KV_INT8 = 1 };
+typedef struct {
+    int32_t kv_format;
+    int32_t reserved[7];
+} edgefm_options;
+edgefm_status edgefm_create_with_options(const edgefm_shape *shape, const edgefm_weights *weights, int32_t max_context,
+                                         const edgefm_options *options, edgefm_ctx **out);
+
+/*
  * edgefm_prefill_kv -- load an already computed KV cache (Eq. 3: KV <- Prefill(x_1:T); here the
  * result of the prefill is given, vision-token positions included; Sec. 3.9 Eq. 5 prefix reuse).
  * k, v: DEVICE bf16; element (layer l, kv head g, position t, j) is read at
@@ -130,6 +152,12 @@ edgefm_status edgefm_get_length(const edgefm_ctx *ctx, int32_t *cur_len_host);
 /* Copy the whole cache, internal layout bf16 [n_layers][n_kv_heads][max_context][head_dim], to the
  * DEVICE buffers k_out / v_out (asynchronous on `stream`). */
 edgefm_status edgefm_export_kv(edgefm_ctx *ctx, void *k_out, void *v_out, void *stream);
+
+/* The same for a context with the EDGEFM_KV_INT8 cache: codes int8 [n_layers][n_kv_heads][max_context][head_dim] and
+ * scales fp32 [n_layers][n_kv_heads][max_context] of K and of V, to DEVICE buffers (asynchronous on `stream`).
+ * Errors: INVALID_ARG (null pointers, or the context has the plain cache), CUDA. */
+edgefm_status edgefm_export_kv_int8(edgefm_ctx *ctx, void *k_codes_out, void *v_codes_out, float *k_scales_out,
+                                    float *v_scales_out, void *stream);
 
 /* Number of kernel launches one decode step performs (nodes of the step graph). */
 edgefm_status edgefm_get_launches_per_step(const edgefm_ctx *ctx, int32_t *n_launches_host);

@@ -36,6 +36,10 @@ class _Shape(ctypes.Structure):
                 ("qkv_bias", ctypes.c_int32)]
 
 
+class _Options(ctypes.Structure):
+    _fields_ = [("kv_format", ctypes.c_int32), ("reserved", ctypes.c_int32 * 7)]
+
+
 class _LayerWeights(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in ("input_norm", "wqkv", "bqkv", "wo", "post_norm", "w_gate_up", "w_down")]
 
@@ -48,7 +52,7 @@ class _Weights(ctypes.Structure):
 EXPORTS = ("edgefm_create", "edgefm_prefill_kv", "edgefm_decode_step", "edgefm_destroy", "edgefm_get_length",
            "edgefm_export_kv", "edgefm_get_launches_per_step", "edgefm_last_error", "edgefm_version",
            "edgefm_sync_status", "edgefm_debug_profile", "edgefm_debug_set_wait_limit", "edgefm_debug_plan", "edgefm_debug_plan_operator", "edgefm_decode_step_static", "edgefm_set_vocab_subset",
-           "edgefm_append_kv")
+           "edgefm_append_kv", "edgefm_create_with_options", "edgefm_export_kv_int8")
 
 
 def library_path() -> Path:
@@ -67,6 +71,10 @@ def load_library():
     vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
     L.edgefm_create.restype = ctypes.c_int
     L.edgefm_create.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Weights), i32, ctypes.POINTER(vp)]
+    L.edgefm_create_with_options.restype = ctypes.c_int
+    L.edgefm_create_with_options.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Weights), i32, ctypes.POINTER(_Options), ctypes.POINTER(vp)]
+    L.edgefm_export_kv_int8.restype = ctypes.c_int
+    L.edgefm_export_kv_int8.argtypes = [vp, vp, vp, vp, vp, vp]
     L.edgefm_prefill_kv.restype = ctypes.c_int
     L.edgefm_prefill_kv.argtypes = [vp, vp, vp, i32, i64, i64, i64, vp]
     L.edgefm_decode_step.restype = ctypes.c_int
@@ -117,9 +125,13 @@ def edgefm_last_error(ctx=None) -> str:
     return load_library().edgefm_last_error(ctx).decode()
 
 
-def edgefm_create(shape: dict, weights: dict, max_context: int):
+KV_FORMATS = {"bf16": 0, "int8": 1}
+
+
+def edgefm_create(shape: dict, weights: dict, max_context: int, kv_format: str | int | None = None, reserved=None):
     """shape: dict with the fields of edgefm_shape; weights: {"embed", "final_norm", "lm_head": device
-    pointers (int), "layers": [ {field: device pointer or None} ]}.  Returns the opaque context handle."""
+    pointers (int), "layers": [ {field: device pointer or None} ]}.  Returns the opaque context handle.
+    kv_format: None = edgefm_create; "bf16" / "int8" (or the raw integer) = edgefm_create_with_options."""
     L = load_library()
     sh = _Shape(**shape)
     layers = weights["layers"]
@@ -129,7 +141,11 @@ def edgefm_create(shape: dict, weights: dict, max_context: int):
             setattr(arr[i], name, lw.get(name))
     w = _Weights(weights["embed"], weights["final_norm"], weights["lm_head"], arr)
     out = ctypes.c_void_p()
-    _check(L.edgefm_create(ctypes.byref(sh), ctypes.byref(w), max_context, ctypes.byref(out)))
+    if kv_format is None:
+        _check(L.edgefm_create(ctypes.byref(sh), ctypes.byref(w), max_context, ctypes.byref(out)))
+    else:
+        opt = _Options(KV_FORMATS.get(kv_format, kv_format) if isinstance(kv_format, str) else int(kv_format), (ctypes.c_int32 * 7)(*(reserved or [0] * 7)))
+        _check(L.edgefm_create_with_options(ctypes.byref(sh), ctypes.byref(w), max_context, ctypes.byref(opt), ctypes.byref(out)))
     return out
 
 
@@ -260,6 +276,10 @@ def edgefm_export_kv(ctx, k_out_ptr, v_out_ptr, stream=None):
     _check(load_library().edgefm_export_kv(ctx, k_out_ptr, v_out_ptr, stream), ctx)
 
 
+def edgefm_export_kv_int8(ctx, k_codes_ptr, v_codes_ptr, k_scales_ptr, v_scales_ptr, stream=None):
+    _check(load_library().edgefm_export_kv_int8(ctx, k_codes_ptr, v_codes_ptr, k_scales_ptr, v_scales_ptr, stream), ctx)
+
+
 # ---- convenience for tests and the benchmark: torch owns the device memory ------------------------
 def upload_weights(host_weights: dict, device="cuda:0"):
     """Copy a dict of numpy uint16 (bf16 bits) arrays (layout of edgefm_weights) to the device.
@@ -286,17 +306,18 @@ def upload_weights(host_weights: dict, device="cuda:0"):
 class DecodeContext:
     """RAII wrapper of one edgefm context with torch-allocated I/O buffers."""
 
-    def __init__(self, cfg, device_weight_ptrs: dict, max_context: int, device="cuda:0"):
+    def __init__(self, cfg, device_weight_ptrs: dict, max_context: int, device="cuda:0", kv_format: str | None = None):
         import torch
 
         self.cfg = cfg
+        self.kv_format = kv_format or "bf16"
         self.device = torch.device(device)
         self.max_context = max_context
         shape = dict(n_layers=cfg.n_layers, hidden=cfg.hidden, n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads,
                      head_dim=cfg.head_dim, ffn=cfg.ffn, vocab=cfg.vocab, rms_eps=cfg.rms_eps,
                      rope_theta=cfg.rope_theta, qkv_bias=int(cfg.qkv_bias))
         with torch.cuda.device(self.device):
-            self.handle = edgefm_create(shape, device_weight_ptrs, max_context)
+            self.handle = edgefm_create(shape, device_weight_ptrs, max_context, kv_format)
         self.logits = torch.empty(cfg.vocab, dtype=torch.float32, device=self.device)
         self.next_token = torch.zeros(1, dtype=torch.int32, device=self.device)
 
@@ -340,6 +361,18 @@ class DecodeContext:
         v = torch.empty(shape, dtype=torch.int16, device=self.device)
         edgefm_export_kv(self.handle, k.data_ptr(), v.data_ptr(), self._stream())
         return k, v
+
+    def export_kv_int8(self):
+        """Compressed cache: (K codes, V codes int8 [L][n_kv][max_context][d], K scales, V scales fp32 [L][n_kv][max_context])."""
+        import torch
+        c = self.cfg
+        shape = (c.n_layers, c.n_kv_heads, self.max_context, c.head_dim)
+        k8 = torch.empty(shape, dtype=torch.int8, device=self.device)
+        v8 = torch.empty(shape, dtype=torch.int8, device=self.device)
+        ks = torch.empty(shape[:3], dtype=torch.float32, device=self.device)
+        vs = torch.empty(shape[:3], dtype=torch.float32, device=self.device)
+        edgefm_export_kv_int8(self.handle, k8.data_ptr(), v8.data_ptr(), ks.data_ptr(), vs.data_ptr(), self._stream())
+        return k8, v8, ks, vs
 
     @property
     def cur_len(self) -> int:

@@ -66,6 +66,45 @@ __global__ void __launch_bounds__(256) prefill_copy_kernel(const uint16_t *k, co
     }
 }
 
+// The same for the compressed cache (Sec. 3.9): one warp per given row; the row's largest magnitude fixes its scale,
+// scale = amax / 127, code = clamp(rint(x * (127 / amax))) in fp32.
+__global__ void __launch_bounds__(256) prefill_quantize_kernel(const uint16_t *k, const uint16_t *v, signed char *kc, signed char *vc,
+                                                               float *ks, float *vs, int L, int nkv, int n, int d, int max_context,
+                                                               long long s_layer, long long s_head, long long s_pos, StepState *st,
+                                                               int slot0) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        st->cur_len = slot0 + n;
+        st->next_position = slot0 + n;
+        st->status = 0;
+    }
+    const int warps = (gridDim.x * blockDim.x) >> 5, lane = threadIdx.x & 31;
+    const long long rows = static_cast<long long>(L) * nkv * n * 2;          // K rows, then V rows
+    for (long long r = (blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x) >> 5; r < rows; r += warps) {
+        const bool is_v = r >= rows / 2;
+        long long rr = is_v ? r - rows / 2 : r;
+        const int t = static_cast<int>(rr % n); rr /= n;
+        const int g = static_cast<int>(rr % nkv);
+        const int l = static_cast<int>(rr / nkv);
+        const uint16_t *src = (is_v ? v : k) + l * s_layer + g * s_head + t * s_pos;
+        const long long row = (static_cast<long long>(l) * nkv + g) * max_context + slot0 + t;
+        float x[4];                                                          // d <= 128: at most 4 values per lane
+        float amax = 0.f;
+        for (int e = 0; e < 4; ++e) {
+            const int j = lane + 32 * e;
+            x[e] = j < d ? bf16_bits_to_f32(src[j]) : 0.f;
+            amax = fmaxf(amax, fabsf(x[e]));
+        }
+        amax = warp_max(amax);
+        const float inv = amax > 0.f ? __fdiv_rn(127.0f, amax) : 0.f;
+        signed char *dst = (is_v ? vc : kc) + row * d;
+        for (int e = 0; e < 4; ++e) {
+            const int j = lane + 32 * e;
+            if (j < d) dst[j] = static_cast<signed char>(static_cast<int>(fminf(fmaxf(rintf(__fmul_rn(x[e], inv)), -127.f), 127.f)));
+        }
+        if (lane == 0) (is_v ? vs : ks)[row] = amax > 0.f ? __fdiv_rn(amax, 127.0f) : 0.f;
+    }
+}
+
 // Vocabulary pruning: row r of the compact lm_head is row ids[r] of the full one.  One warp per row, 16-byte pieces.
 __global__ void __launch_bounds__(256) gather_rows_kernel(const uint16_t *src, const int *ids, uint16_t *dst, int n, int H) {
     const int warps = (gridDim.x * blockDim.x) >> 5;
@@ -102,10 +141,12 @@ struct StepPlan {
 
 // Kernel variant and shared-memory split for a model shape.  Returns null, or why the shape does not fit.
 // sched_reserve: bytes to set aside for the CTA's tile lists.
-inline const char *plan_step(const edgefm_shape &sh, int max_context, int num_sms, int smem_optin, size_t sched_reserve, StepPlan *pl, cudaError_t *cuda_err) {
+inline const char *plan_step(const edgefm_shape &sh, int max_context, int num_sms, int smem_optin, size_t sched_reserve, StepPlan *pl, cudaError_t *cuda_err,
+                             bool kv8 = false) {
     const int H = sh.hidden, d = sh.head_dim, nq = sh.n_q_heads, nkv = sh.n_kv_heads, G = nq / nkv;
     *cuda_err = cudaSuccess;
-    pl->long_ctx = max_context > 8192 || static_cast<long long>(nq) * MK_ATT_SPLIT_MAXC * 2 > MK_PARTIAL_FLOATS;
+    // (the compressed cache is attended by the grouped attention of the long-context build only)
+    pl->long_ctx = kv8 || max_context > 8192 || static_cast<long long>(nq) * MK_ATT_SPLIT_MAXC * 2 > MK_PARTIAL_FLOATS;
     pl->kernel = d == 64 ? mega_kernel_g<64>(G, pl->long_ctx) : mega_kernel_g<128>(G, pl->long_ctx);
     pl->nw = pl->long_ctx ? MK_NW_LONG : MK_NW_SHORT;
     pl->grid = num_sms;
@@ -205,10 +246,10 @@ inline const char *plan_schedule(const StepPlan &pl, const edgefm_shape &sh, int
 // Shared-memory plan and tile schedule together: the tile lists live in shared memory, so their size (known only once
 // the schedule exists) takes room from the rings, whose slot size shapes the schedule.  A few rounds settle it.
 inline const char *plan_step_and_schedule(const edgefm_shape &sh, int max_context, int num_sms, int smem_optin, StepPlan *pl, StepSchedule *ss,
-                                          cudaError_t *cuda_err) {
+                                          cudaError_t *cuda_err, bool kv8 = false) {
     size_t reserve = 0;
     for (int attempt = 0; attempt < 6; ++attempt) {
-        if (const char *why = plan_step(sh, max_context, num_sms, smem_optin, reserve, pl, cuda_err)) return why;
+        if (const char *why = plan_step(sh, max_context, num_sms, smem_optin, reserve, pl, cuda_err, kv8)) return why;
         if (const char *why = plan_schedule(*pl, sh, sh.vocab, ss)) return why;
         const size_t need = ss->smem_bytes();
         if (need <= pl->sched_bytes) return nullptr;
@@ -273,7 +314,10 @@ struct edgefm_ctx {
     const void *embed = nullptr, *final_norm = nullptr, *lm_head = nullptr;
 
     // owned device memory
-    uint16_t *k_cache = nullptr, *v_cache = nullptr;  // [L][nkv][max_context][d]
+    uint16_t *k_cache = nullptr, *v_cache = nullptr;  // [L][nkv][max_context][d] (bf16, or one signed byte per element)
+    int kv_format = EDGEFM_KV_BF16;
+    float *k_scale = nullptr, *v_scale = nullptr;     // compressed cache: [L][nkv][max_context]
+    float *kv_stage = nullptr;                        // compressed cache: fp32 k, v rows of the step's token [2][nkv][d]
     float *x = nullptr;          // residual stream [H]
     float *q = nullptr;          // rotated queries [nq*d]
     float *attn = nullptr;       // attention output [nq*d]
@@ -363,7 +407,7 @@ void free_all(edgefm_ctx *c) {
     if (c->build_stream) cudaStreamDestroy(c->build_stream);
     void *bufs[] = {c->k_cache, c->v_cache, c->x, c->q, c->attn, c->act, c->inv_freq, c->part_m, c->part_l,
                     c->part_o, c->lm_part_val, c->lm_part_idx, c->tickets, c->state, c->req, c->d_ops, c->d_op_w, c->d_maps, c->d_tiles,
-                    c->d_cta_tab, c->d_combines, c->grid_bar, c->prof, c->vocab_ids, c->sub_lm};
+                    c->d_cta_tab, c->d_combines, c->grid_bar, c->prof, c->vocab_ids, c->sub_lm, c->k_scale, c->v_scale, c->kv_stage};
     for (void *b : bufs) if (b) cudaFree(b);
 }
 
@@ -408,7 +452,19 @@ const char *edgefm_last_error(const edgefm_ctx *ctx) { return ctx ? ctx->err.c_s
 
 edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *weights, int32_t max_context,
                             edgefm_ctx **out) {
+    return edgefm_create_with_options(shape, weights, max_context, nullptr, out);
+}
+
+edgefm_status edgefm_create_with_options(const edgefm_shape *shape, const edgefm_weights *weights, int32_t max_context,
+                                         const edgefm_options *options, edgefm_ctx **out) {
     if (out) *out = nullptr;
+    if (options) {
+        if (options->kv_format != EDGEFM_KV_BF16 && options->kv_format != EDGEFM_KV_INT8)
+            return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "unknown kv_format %d", options->kv_format);
+        for (int r : options->reserved)
+            if (r != 0) return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "reserved option fields must be zero");
+    }
+    const bool kv8 = options && options->kv_format == EDGEFM_KV_INT8;
     if (!shape || !weights || !out) return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "null argument");
     if (max_context < 1) return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "max_context must be >= 1");
     const edgefm_shape &sh = *shape;
@@ -449,6 +505,7 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
     edgefm_ctx *c = new (std::nothrow) edgefm_ctx();
     if (!c) return fail(nullptr, EDGEFM_ERR_OUT_OF_MEMORY, "host allocation failed");
     c->shape = sh;
+    c->kv_format = kv8 ? EDGEFM_KV_INT8 : EDGEFM_KV_BF16;
     c->max_context = max_context;
     c->device = dev;
     c->num_sms = prop.multiProcessorCount;
@@ -477,14 +534,24 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
     if (!coop) return bail(EDGEFM_ERR_CUDA, "device lacks cooperative launch", cudaErrorNotSupported);
     {
         cudaError_t ce = cudaSuccess;
-        if (const char *why = plan_step_and_schedule(sh, max_context, c->num_sms, smem_optin, &pl, &c->sched_full, &ce))
+        if (const char *why = plan_step_and_schedule(sh, max_context, c->num_sms, smem_optin, &pl, &c->sched_full, &ce, kv8))
             return bail(ce != cudaSuccess ? EDGEFM_ERR_CUDA : EDGEFM_ERR_BAD_SHAPE, why, ce != cudaSuccess ? ce : cudaErrorInvalidValue);
     }
     const StepSchedule &ss = c->sched_full;
 
     const size_t kv_elems = static_cast<size_t>(sh.n_layers) * nkv * max_context * d;
-    CREATE_TRY(dev_alloc(&c->k_cache, kv_elems));
-    CREATE_TRY(dev_alloc(&c->v_cache, kv_elems));
+    const size_t kv_bytes = kv8 ? kv_elems : kv_elems * 2;
+    CREATE_TRY(dev_alloc(&c->k_cache, (kv_bytes + 1) / 2));
+    CREATE_TRY(dev_alloc(&c->v_cache, (kv_bytes + 1) / 2));
+    if (kv8) {
+        const size_t kv_rows = static_cast<size_t>(sh.n_layers) * nkv * max_context;
+        CREATE_TRY(dev_alloc(&c->k_scale, kv_rows));
+        CREATE_TRY(dev_alloc(&c->v_scale, kv_rows));
+        CREATE_TRY(dev_alloc(&c->kv_stage, static_cast<size_t>(2) * nkv * d));
+        CREATE_TRY(cudaMemset(c->k_scale, 0, kv_rows * sizeof(float)));
+        CREATE_TRY(cudaMemset(c->v_scale, 0, kv_rows * sizeof(float)));
+        CREATE_TRY(cudaMemset(c->kv_stage, 0, static_cast<size_t>(2) * nkv * d * sizeof(float)));
+    }
     CREATE_TRY(dev_alloc(&c->x, H));
     CREATE_TRY(dev_alloc(&c->q, nq * d));
     CREATE_TRY(dev_alloc(&c->attn, nq * d));
@@ -499,8 +566,8 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
     CREATE_TRY(dev_alloc(&c->tickets, nq + nkv + 2));
     CREATE_TRY(dev_alloc(&c->state, 1));
     CREATE_TRY(dev_alloc(&c->req, 1));
-    CREATE_TRY(cudaMemset(c->k_cache, 0, kv_elems * 2));
-    CREATE_TRY(cudaMemset(c->v_cache, 0, kv_elems * 2));
+    CREATE_TRY(cudaMemset(c->k_cache, 0, kv_bytes));
+    CREATE_TRY(cudaMemset(c->v_cache, 0, kv_bytes));
     CREATE_TRY(cudaMemset(c->tickets, 0, (nq + nkv + 2) * sizeof(unsigned)));
     CREATE_TRY(cudaMemset(c->state, 0, sizeof(StepState)));
     {
@@ -551,6 +618,7 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
     m.ops = c->d_ops; m.op_weights = c->d_op_w; m.maps = c->d_maps; m.tiles = c->d_tiles; m.cta_tab = c->d_cta_tab; m.combines = c->d_combines;
     m.vocab_ids = c->vocab_ids;
     m.k_cache = c->k_cache; m.v_cache = c->v_cache; m.embed = (const uint16_t *)c->embed;
+    m.kv8 = kv8 ? 1 : 0; m.k_scale = c->k_scale; m.v_scale = c->v_scale; m.kv_stage = c->kv_stage;
     m.inv_freq = c->inv_freq; m.x = c->x; m.q = c->q; m.attn = c->attn; m.part_m = c->part_m; m.part_l = c->part_l;
     m.part_o = c->part_o; m.tickets = c->tickets; m.barrier = c->grid_bar;
     m.lm_part_val = c->lm_part_val; m.lm_part_idx = c->lm_part_idx; m.state = c->state; m.req = c->req;
@@ -584,6 +652,19 @@ edgefm_status copy_kv_in(edgefm_ctx *ctx, const void *k, const void *v, int32_t 
         return fail(ctx, EDGEFM_ERR_INVALID_ARG, "bad strides");
     DeviceGuard guard(ctx->device);
     const edgefm_shape &sh = ctx->shape;
+    if (ctx->kv_format == EDGEFM_KV_INT8) {
+        long long blocks = (static_cast<long long>(sh.n_layers) * sh.n_kv_heads * n_positions * 2 + 7) / 8;   // 8 warps (rows) per block
+        if (blocks < 1) blocks = 1;
+        if (blocks > ctx->num_sms * 16) blocks = ctx->num_sms * 16;
+        prefill_quantize_kernel<<<static_cast<unsigned>(blocks), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+            static_cast<const uint16_t *>(k), static_cast<const uint16_t *>(v), reinterpret_cast<signed char *>(ctx->k_cache),
+            reinterpret_cast<signed char *>(ctx->v_cache), ctx->k_scale, ctx->v_scale, sh.n_layers, sh.n_kv_heads, n_positions, sh.head_dim,
+            ctx->max_context, stride_layer, stride_head, stride_pos, ctx->state, slot0);
+        CUDA_TRY(ctx, cudaGetLastError());
+        ctx->cur_len = slot0 + n_positions;
+        ctx->err.clear();
+        return EDGEFM_OK;
+    }
     const int vec_ok = n_positions > 0 && aligned16(k) && aligned16(v) && stride_layer % 8 == 0 && stride_head % 8 == 0 &&
                        stride_pos % 8 == 0;
     const long long total = static_cast<long long>(sh.n_layers) * sh.n_kv_heads * n_positions * sh.head_dim;
@@ -775,11 +856,28 @@ edgefm_status edgefm_debug_set_wait_limit(edgefm_ctx *ctx, uint32_t limit_ns, in
 edgefm_status edgefm_export_kv(edgefm_ctx *ctx, void *k_out, void *v_out, void *stream) {
     if (!ctx) return EDGEFM_ERR_INVALID_ARG;
     if (!k_out || !v_out) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "null output");
+    if (ctx->kv_format != EDGEFM_KV_BF16) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "this context has a compressed cache: use edgefm_export_kv_int8");
     DeviceGuard guard(ctx->device);
     const edgefm_shape &sh = ctx->shape;
     const size_t bytes = static_cast<size_t>(sh.n_layers) * sh.n_kv_heads * ctx->max_context * sh.head_dim * 2;
     CUDA_TRY(ctx, cudaMemcpyAsync(k_out, ctx->k_cache, bytes, cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(stream)));
     CUDA_TRY(ctx, cudaMemcpyAsync(v_out, ctx->v_cache, bytes, cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(stream)));
+    return EDGEFM_OK;
+}
+
+edgefm_status edgefm_export_kv_int8(edgefm_ctx *ctx, void *k_codes_out, void *v_codes_out, float *k_scales_out, float *v_scales_out,
+                                    void *stream) {
+    if (!ctx) return EDGEFM_ERR_INVALID_ARG;
+    if (!k_codes_out || !v_codes_out || !k_scales_out || !v_scales_out) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "null output");
+    if (ctx->kv_format != EDGEFM_KV_INT8) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "this context has the plain bf16 cache: use edgefm_export_kv");
+    DeviceGuard guard(ctx->device);
+    const edgefm_shape &sh = ctx->shape;
+    const size_t rows = static_cast<size_t>(sh.n_layers) * sh.n_kv_heads * ctx->max_context;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CUDA_TRY(ctx, cudaMemcpyAsync(k_codes_out, ctx->k_cache, rows * sh.head_dim, cudaMemcpyDeviceToDevice, s));
+    CUDA_TRY(ctx, cudaMemcpyAsync(v_codes_out, ctx->v_cache, rows * sh.head_dim, cudaMemcpyDeviceToDevice, s));
+    CUDA_TRY(ctx, cudaMemcpyAsync(k_scales_out, ctx->k_scale, rows * sizeof(float), cudaMemcpyDeviceToDevice, s));
+    CUDA_TRY(ctx, cudaMemcpyAsync(v_scales_out, ctx->v_scale, rows * sizeof(float), cudaMemcpyDeviceToDevice, s));
     return EDGEFM_OK;
 }
 

@@ -352,7 +352,7 @@ __device__ __forceinline__ void prefetch_tiles(const MkParams &p, volatile int *
         // ring has started on the tiles of layer l, the chunk of layer l (one-head-per-CTA chunking only).
         const int n_spare = 2 * (16 - MK_NW), me = (w - MK_NW) * 2 + half;
         const int n = p.state->cur_len + 1;
-        if (n > p.att_split_max_n || n < 1 || n > p.max_context) return;
+        if (p.kv8 || n > p.att_split_max_n || n < 1 || n > p.max_context) return;
         int nch, chunk_len;
         att_chunking(p, n, 1, p.att_chunk_split, 32 / MK_ATT_LPP_SPLIT, static_cast<int>(gridDim.x), nch, chunk_len);
         const int cta = static_cast<int>(blockIdx.x);
@@ -467,11 +467,19 @@ __device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkOp &P,
             if (head < p.nq) {
                 P.out[row_lo] = rlo;
                 P.out[row_hi] = rhi;
+            } else if (p.kv8) {   // compressed cache: the row is left in fp32 for the attention phase, which compresses it whole
+                float *dst = p.kv_stage + static_cast<size_t>(head - p.nq) * p.d;
+                dst[i] = rlo;
+                dst[i + half] = rhi;
             } else {
                 uint16_t *dst = p.k_cache + layer_off + (static_cast<size_t>(head - p.nq) * p.max_context + cx.slot_row) * p.d;
                 dst[i] = f32_to_bf16_bits(rlo);
                 dst[i + half] = f32_to_bf16_bits(rhi);
             }
+        } else if (p.kv8) {
+            float *dst = p.kv_stage + static_cast<size_t>(p.nkv + head - p.nq - p.nkv) * p.d;
+            dst[i] = lo;
+            dst[i + half] = hi;
         } else {
             uint16_t *dst = p.v_cache + layer_off + (static_cast<size_t>(head - p.nq - p.nkv) * p.max_context + cx.slot_row) * p.d;
             dst[i] = f32_to_bf16_bits(lo);
@@ -785,11 +793,26 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_
 // probabilities, warp merge area, chunk statistics.  The CTA that arrives last for its head group
 // (atomic ticket, no waiting) merges the chunks exactly:  m = max m_c, l = sum l_c e^{m_c - m},
 // o = sum o_c e^{m_c - m} / l, in index order.
-template <int D, int HG, int LPP>
+//
+// Q8: the compressed cache (Sec. 3.9 of the paper, KV~ = C(KV) with reconstruction on demand; the paper fixes no C): every
+// cached row is d signed 8-bit codes and one fp32 scale (scale = amax / 127).  The codes are turned into fp32 exactly, two
+// instructions each (the byte + 128 dropped into the mantissa of 2^23, minus 2^23 + 128); the K scale multiplies the finished
+// score, the V scale the probability.  The row this step appends was left in fp32 by the QKV epilogue; the CTA whose chunk
+// ends with it compresses it into the cache (two warps, one row each) before anybody reads it.
+__device__ __forceinline__ void codes4_to_f32(uint32_t w, float (&f)[4]) {
+    const uint32_t u = w ^ 0x80808080u;     // two's complement -> offset binary
+    f[0] = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7440)) - 8388736.f;
+    f[1] = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7441)) - 8388736.f;
+    f[2] = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7442)) - 8388736.f;
+    f[3] = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7443)) - 8388736.f;
+}
+template <int D, int HG, int LPP, bool Q8 = false>
 __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, int n, int min_chunk, bool defer_merge,
                                                 unsigned char *xbuf, int tid, int *s_flag) {
     constexpr int TILE = 32 / LPP;   // positions per warp iteration
     constexpr int DV = D / 32, CPR = D / 8, CPL = CPR / LPP;
+    constexpr int CPL8 = D / 16 / LPP;                  // 16-byte pieces (16 codes) of a compressed K row per lane
+    static_assert(!Q8 || (D / 16) % LPP == 0, "compressed rows are split into whole 16-byte pieces");
     constexpr int MW = MK_NW;                            // every warp publishes its partial: one sync, then one pass
     const int lane = tid & 31, warp = tid >> 5;
     const int cta = blockIdx.x, ncta = gridDim.x;
@@ -814,28 +837,74 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
     const size_t head_off = (static_cast<size_t>(layer) * p.nkv + g) * p.max_context * D;
     const uint16_t *kg = p.k_cache + head_off;
     const uint16_t *vg = p.v_cache + head_off;
+    // compressed cache: the same arrays hold one byte per element; the scales are [L][nkv][max_context]
+    const unsigned char *kg8 = reinterpret_cast<const unsigned char *>(p.k_cache) + head_off;
+    const unsigned char *vg8 = reinterpret_cast<const unsigned char *>(p.v_cache) + head_off;
+    const float *ksg = p.k_scale + (static_cast<size_t>(layer) * p.nkv + g) * p.max_context;
+    const float *vsg = p.v_scale + (static_cast<size_t>(layer) * p.nkv + g) * p.max_context;
     float *pw = ps + warp * (HG * TILE);
     const int pi = lane / LPP, part = lane % LPP;
 
-    // K and V rows of one warp iteration: K pieces of this lane's position, raw bf16 pairs of V (converted when used to keep
-    // the register footprint small)
-    uint4 kk[CPL];
-    uint32_t vraw[TILE][DV / 2];
+    if constexpr (Q8) {
+        if (t1 == n && warp < 2) {
+            // the row appended by this step: warp 0 compresses k (after RoPE), warp 1 v; every lane DV values
+            const float *src = p.kv_stage + (static_cast<size_t>(warp) * p.nkv + g) * D + lane * DV;
+            float xv[DV];
+            float amax = 0.f;
+#pragma unroll
+            for (int e = 0; e < DV; ++e) { xv[e] = __ldcg(src + e); amax = fmaxf(amax, fabsf(xv[e])); }
+            amax = warp_max(amax);
+            const float inv = amax > 0.f ? __fdiv_rn(127.0f, amax) : 0.f;
+            uint32_t packed = 0u;
+#pragma unroll
+            for (int e = 0; e < DV; ++e) {
+                const float c = fminf(fmaxf(rintf(__fmul_rn(xv[e], inv)), -127.f), 127.f);
+                packed |= (static_cast<uint32_t>(static_cast<int>(c)) & 0xffu) << (8 * e);
+            }
+            unsigned char *dst = const_cast<unsigned char *>(warp == 0 ? kg8 : vg8) + static_cast<size_t>(n - 1) * D + lane * DV;
+            if constexpr (DV == 4) *reinterpret_cast<uint32_t *>(dst) = packed;
+            else *reinterpret_cast<uint16_t *>(dst) = static_cast<uint16_t>(packed);
+            if (lane == 0) const_cast<float *>(warp == 0 ? ksg : vsg)[n - 1] = amax > 0.f ? __fdiv_rn(amax, 127.0f) : 0.f;
+        }
+        // (published to the rest of the CTA by the sync that follows the staging of the queries)
+    }
+
+    // K and V rows of one warp iteration: K pieces of this lane's position, raw bf16 pairs (or 8-bit codes) of V (converted when
+    // used to keep the register footprint small)
+    uint4 kk[Q8 ? CPL8 : CPL];
+    uint32_t vraw[TILE][Q8 ? 1 : DV / 2];
+    float ksc = 0.f, vsc = 0.f;   // scales of this lane's position (compressed cache)
     auto load_kv = [&](int tt) {
         const bool pvalid = tt + pi < t1;
+        if constexpr (Q8) {
 #pragma unroll
-        for (int j = 0; j < CPL; ++j)
-            kk[j] = pvalid ? __ldcg(reinterpret_cast<const uint4 *>(kg + static_cast<size_t>(tt + pi) * D) + j * LPP + part)
-                           : make_uint4(0, 0, 0, 0);
+            for (int j = 0; j < CPL8; ++j)
+                kk[j] = pvalid ? __ldcg(reinterpret_cast<const uint4 *>(kg8 + static_cast<size_t>(tt + pi) * D) + j * LPP + part)
+                               : make_uint4(0u, 0u, 0u, 0u);
+            ksc = pvalid ? __ldcg(ksg + tt + pi) : 0.f;
+            vsc = pvalid ? __ldcg(vsg + tt + pi) : 0.f;
 #pragma unroll
-        for (int x = 0; x < TILE; ++x) {
-            const int t = tt + x;
-            const uint16_t *vp = vg + static_cast<size_t>(t) * D + lane * DV;
-            if constexpr (DV == 4) {
-                const uint2 w = t < t1 ? __ldcg(reinterpret_cast<const uint2 *>(vp)) : make_uint2(0u, 0u);
-                vraw[x][0] = w.x; vraw[x][1] = w.y;
-            } else {
-                vraw[x][0] = t < t1 ? __ldcg(reinterpret_cast<const unsigned *>(vp)) : 0u;
+            for (int x = 0; x < TILE; ++x) {
+                const int t = tt + x;
+                const unsigned char *vp = vg8 + static_cast<size_t>(t) * D + lane * DV;
+                if constexpr (DV == 4) vraw[x][0] = t < t1 ? __ldcg(reinterpret_cast<const unsigned *>(vp)) : 0u;
+                else vraw[x][0] = t < t1 ? static_cast<unsigned>(__ldcg(reinterpret_cast<const unsigned short *>(vp))) : 0u;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < CPL; ++j)
+                kk[j] = pvalid ? __ldcg(reinterpret_cast<const uint4 *>(kg + static_cast<size_t>(tt + pi) * D) + j * LPP + part)
+                               : make_uint4(0, 0, 0, 0);
+#pragma unroll
+            for (int x = 0; x < TILE; ++x) {
+                const int t = tt + x;
+                const uint16_t *vp = vg + static_cast<size_t>(t) * D + lane * DV;
+                if constexpr (DV == 4) {
+                    const uint2 w = t < t1 ? __ldcg(reinterpret_cast<const uint2 *>(vp)) : make_uint2(0u, 0u);
+                    vraw[x][0] = w.x; vraw[x][1] = w.y;
+                } else {
+                    vraw[x][0] = t < t1 ? __ldcg(reinterpret_cast<const unsigned *>(vp)) : 0u;
+                }
             }
         }
     };
@@ -857,20 +926,40 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
         float s[HG];
 #pragma unroll
         for (int h = 0; h < HG; ++h) s[h] = 0.f;
+        if constexpr (Q8) {
 #pragma unroll
-        for (int j = 0; j < CPL; ++j) {
-            const int cc = j * LPP + part;
+            for (int j = 0; j < CPL8; ++j) {
+                const int cc = j * LPP + part;
+                const uint32_t words[4] = {kk[j].x, kk[j].y, kk[j].z, kk[j].w};
 #pragma unroll
-            for (int h = 0; h < HG; ++h) {
-                const float4 q0 = *reinterpret_cast<const float4 *>(qs + h * D + cc * 8);
-                const float4 q1 = *reinterpret_cast<const float4 *>(qs + h * D + cc * 8 + 4);
-                s[h] = dot8(kk[j], q0, q1, s[h]);
+                for (int wi = 0; wi < 4; ++wi) {
+                    float f[4];
+                    codes4_to_f32(words[wi], f);
+#pragma unroll
+                    for (int h = 0; h < HG; ++h) {
+                        const float4 q4 = *reinterpret_cast<const float4 *>(qs + h * D + cc * 16 + wi * 4);
+                        s[h] = fmaf(f[0], q4.x, s[h]); s[h] = fmaf(f[1], q4.y, s[h]);
+                        s[h] = fmaf(f[2], q4.z, s[h]); s[h] = fmaf(f[3], q4.w, s[h]);
+                    }
+                }
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < CPL; ++j) {
+                const int cc = j * LPP + part;
+#pragma unroll
+                for (int h = 0; h < HG; ++h) {
+                    const float4 q0 = *reinterpret_cast<const float4 *>(qs + h * D + cc * 8);
+                    const float4 q1 = *reinterpret_cast<const float4 *>(qs + h * D + cc * 8 + 4);
+                    s[h] = dot8(kk[j], q0, q1, s[h]);
+                }
             }
         }
 #pragma unroll
         for (int h = 0; h < HG; ++h) {
 #pragma unroll
             for (int x = 1; x < LPP; x <<= 1) s[h] += __shfl_xor_sync(0xffffffffu, s[h], x);
+            if constexpr (Q8) s[h] *= ksc;
             if (!pvalid) s[h] = -INFINITY;
             const float mn = fmaxf(m[h], warp_max(s[h]));
             const float corr = __expf(m[h] - mn);
@@ -879,7 +968,7 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
 #pragma unroll
             for (int e = 0; e < DV; ++e) o[h][e] *= corr;
             m[h] = mn;
-            if (part == 0) pw[h * TILE + pi] = pr;
+            if (part == 0) pw[h * TILE + pi] = Q8 ? pr * vsc : pr;
         }
         __syncwarp();
 #pragma unroll
@@ -887,10 +976,17 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
             float v[4][DV];
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
+                if constexpr (Q8) {
+                    float f[4];
+                    codes4_to_f32(vraw[tb + x][0], f);
 #pragma unroll
-                for (int e = 0; e < DV; e += 2) {
-                    v[x][e] = bf16lo(vraw[tb + x][e / 2]);
-                    v[x][e + 1] = bf16hi(vraw[tb + x][e / 2]);
+                    for (int e = 0; e < DV; ++e) v[x][e] = f[e];
+                } else {
+#pragma unroll
+                    for (int e = 0; e < DV; e += 2) {
+                        v[x][e] = bf16lo(vraw[tb + x][e / 2]);
+                        v[x][e + 1] = bf16hi(vraw[tb + x][e / 2]);
+                    }
                 }
             }
 #pragma unroll
@@ -1094,7 +1190,8 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
     int prof_idx = 0;
     prof_stamp(p, tid, prof_idx);
     const int n_att = slot_row + 1;
-    const bool att_split = !LONG || (n_att <= p.att_split_max_n && static_cast<long long>(p.nq) * MK_ATT_SPLIT_MAXC * 2 <= MK_PARTIAL_FLOATS);
+    // (a compressed cache is always attended with one CTA per kv head and chunk: one CTA then owns the row the step appends)
+    const bool att_split = !LONG || (!p.kv8 && n_att <= p.att_split_max_n && static_cast<long long>(p.nq) * MK_ATT_SPLIT_MAXC * 2 <= MK_PARTIAL_FLOATS);
     int merge_chunks = 0;   // chunks per head the O-projection prologue has to merge (split mode)
     if (att_split && MK_SPLIT_DEFER) { int cl; att_chunking(p, n_att, 1, p.att_chunk_split, 32 / MK_ATT_LPP_SPLIT, ncta, merge_chunks, cl); }
     // One loop over the operators of the step, with a single inlined copy of the streaming operator and of the grid barrier
@@ -1110,6 +1207,7 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
             const int l = ph >> 2;
             if constexpr (LONG) {
                 if (att_split) attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, sm_xbuf(p), tid, &s_flag);
+                else if (p.kv8) attention_phase<D, G, MK_ATT_LPP, true>(p, l, n_att, p.att_chunk_shared, false, sm_xbuf(p), tid, &s_flag);
                 else attention_phase<D, G, MK_ATT_LPP>(p, l, n_att, p.att_chunk_shared, false, sm_xbuf(p), tid, &s_flag);
             } else {
                 attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, sm_xbuf(p), tid, &s_flag);

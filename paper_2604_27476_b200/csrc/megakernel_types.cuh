@@ -105,7 +105,10 @@ struct MkParams {
     int half_shift;          // log2(d / 2)
     float eps, scale;
     int max_context;
-    uint16_t *k_cache, *v_cache;   // [L][nkv][max_context][d]
+    uint16_t *k_cache, *v_cache;   // [L][nkv][max_context][d] bf16; compressed cache (kv8): the same shape in signed bytes
+    int kv8;                       // 1: compressed cache (8-bit codes + one fp32 scale per cached row)
+    float *k_scale, *v_scale;      // kv8: [L][nkv][max_context]
+    float *kv_stage;               // kv8: the fp32 k (after RoPE) and v rows of the step's token, [2][nkv][d], reused by every layer
     const uint16_t *embed;
     const double *inv_freq;        // [d/2]
     float *x, *q, *attn;

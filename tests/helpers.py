@@ -55,7 +55,7 @@ def assert_appended_rows_close(gpu_bits: np.ndarray, ref_bits: np.ndarray):
 class Pair:
     """The oracle model and the CUDA context fed from the same host weights and KV prefix."""
 
-    def __init__(self, cfg, seed=GLOBAL_SEED, cache_len=None, max_context=None, weights=None):
+    def __init__(self, cfg, seed=GLOBAL_SEED, cache_len=None, max_context=None, weights=None, kv_format=None):
         import torch
         from oracle import OracleModel
         from paper_2604_27476_b200 import DecodeContext, upload_weights
@@ -65,11 +65,11 @@ class Pair:
         self.max_context = max_context or (self.T0 + cfg.steps)
         self.weights = weights if weights is not None else make_weights(cfg, seed)
         self.k, self.v = make_kv(cfg, seed, self.T0)
-        self.oracle = OracleModel(cfg, self.weights, self.max_context)
+        self.oracle = OracleModel(cfg, self.weights, self.max_context, kv_format=kv_format or "bf16")
         if self.T0:
             self.oracle.load_kv(self.k, self.v)
         self.ptrs, self.keep = upload_weights(self.weights)
-        self.ctx = DecodeContext(cfg, self.ptrs, self.max_context)
+        self.ctx = DecodeContext(cfg, self.ptrs, self.max_context, kv_format=kv_format)
         self.kd = torch.from_numpy(self.k.view(np.int16)).cuda()
         self.vd = torch.from_numpy(self.v.view(np.int16)).cuda()
         if self.T0:
