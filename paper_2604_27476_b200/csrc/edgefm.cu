@@ -563,12 +563,12 @@ edgefm_status edgefm_create_with_options(const edgefm_shape *shape, const edgefm
     CREATE_TRY(dev_alloc(&c->part_o, static_cast<size_t>(nq) * pl.max_chunks * d));
     CREATE_TRY(dev_alloc(&c->lm_part_val, pl.grid));
     CREATE_TRY(dev_alloc(&c->lm_part_idx, pl.grid));
-    CREATE_TRY(dev_alloc(&c->tickets, nq + nkv + 2));
+    CREATE_TRY(dev_alloc(&c->tickets, nq + nkv + 2 + nq + 2 * nkv));   // tickets, then the per-head counters of the QKV projection
     CREATE_TRY(dev_alloc(&c->state, 1));
     CREATE_TRY(dev_alloc(&c->req, 1));
     CREATE_TRY(cudaMemset(c->k_cache, 0, kv_bytes));
     CREATE_TRY(cudaMemset(c->v_cache, 0, kv_bytes));
-    CREATE_TRY(cudaMemset(c->tickets, 0, (nq + nkv + 2) * sizeof(unsigned)));
+    CREATE_TRY(cudaMemset(c->tickets, 0, (nq + nkv + 2 + nq + 2 * nkv) * sizeof(unsigned)));
     CREATE_TRY(cudaMemset(c->state, 0, sizeof(StepState)));
     {
         StepRequest r{-1, -1, nullptr, nullptr};
@@ -621,6 +621,7 @@ edgefm_status edgefm_create_with_options(const edgefm_shape *shape, const edgefm
     m.kv8 = kv8 ? 1 : 0; m.k_scale = c->k_scale; m.v_scale = c->v_scale; m.kv_stage = c->kv_stage;
     m.inv_freq = c->inv_freq; m.x = c->x; m.q = c->q; m.attn = c->attn; m.part_m = c->part_m; m.part_l = c->part_l;
     m.part_o = c->part_o; m.tickets = c->tickets; m.barrier = c->grid_bar;
+    m.head_ready = c->tickets + nq + nkv + 2; m.head_flags = pl.long_ctx ? 0 : MK_HEAD_FLAGS;
     m.lm_part_val = c->lm_part_val; m.lm_part_idx = c->lm_part_idx; m.state = c->state; m.req = c->req;
     const char *pe_ = getenv("EDGEFM_PROFILE");
     if (pe_ && pe_[0] == '1') {
@@ -1006,7 +1007,7 @@ extern "C" edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, co
     float *part_o = sc.take<float>(static_cast<size_t>(nq) * max_chunks * d);
     float *lm_val = sc.take<float>(grid);
     int *lm_idx = sc.take<int>(grid);
-    unsigned *counters = sc.take<unsigned>(static_cast<size_t>(nq) + nkv + 2 + 64);   // tickets, then the grid barrier counter
+    unsigned *counters = sc.take<unsigned>(static_cast<size_t>(nq) + nkv + 2 + 64 + nq + 2 * nkv);   // tickets, the grid barrier counter, the per-head counters
     StepState *state = sc.take<StepState>(1);
     StepRequest *req = sc.take<StepRequest>(1);
     if (sc.off > EDGEFM_STATIC_SCRATCH_BYTES)
@@ -1029,6 +1030,7 @@ extern "C" edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, co
     m.k_cache = static_cast<uint16_t *>(k_cache); m.v_cache = static_cast<uint16_t *>(v_cache);
     m.embed = (const uint16_t *)weights->embed; m.inv_freq = inv_freq; m.x = x; m.q = q; m.attn = attn;
     m.part_m = part_m; m.part_l = part_l; m.part_o = part_o;
+    m.head_ready = counters + nq + nkv + 2 + 64; m.head_flags = pl.long_ctx ? 0 : MK_HEAD_FLAGS;
     m.tickets = tickets; m.barrier = grid_bar; m.lm_part_val = lm_val; m.lm_part_idx = lm_idx; m.state = state; m.req = req;
     m.prof = nullptr; m.prof_stride = 0;
     m.map_fence = 2;   // every call rewrites all tensor maps in the shared scratch
@@ -1040,7 +1042,7 @@ extern "C" edgefm_status edgefm_decode_step_static(const edgefm_shape *shape, co
     st.cur_len = cur_len; st.next_position = position;
     StepRequest rq{token_id, position, logits_out, next_token_out};
     // counters (attention tickets, lm_head ticket, grid barrier) must start at zero
-    CUDA_TRY(nullptr, cudaMemsetAsync(counters, 0, (static_cast<size_t>(nq) + nkv + 2 + 64) * sizeof(unsigned), s));
+    CUDA_TRY(nullptr, cudaMemsetAsync(counters, 0, (static_cast<size_t>(nq) + nkv + 2 + 64 + nq + 2 * nkv) * sizeof(unsigned), s));
     // pageable copies: the runtime stages the bytes before returning, so the sources may be freed after the call
     CUDA_TRY(nullptr, cudaMemcpyAsync(d_ops, ops.data(), ops.size() * sizeof(MkOp), cudaMemcpyHostToDevice, s));
     CUDA_TRY(nullptr, cudaMemcpyAsync(d_op_w, op_w.data(), op_w.size() * sizeof(op_w[0]), cudaMemcpyHostToDevice, s));

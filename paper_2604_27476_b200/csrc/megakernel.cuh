@@ -455,6 +455,10 @@ __device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkOp &P,
     } else {  // PH_QKV: bias, rotate-half RoPE of q and k, q to the work buffer, k and v to the cache row of this step
         const int half = p.d >> 1;
         const int head = u >> p.half_shift, i = u & (half - 1);
+        struct Publish {   // when the unit's stores are done: one more finished unit of this head (release: the stores come first)
+            unsigned *counter;
+            __device__ ~Publish() { if (counter) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(counter) : "memory"); }
+        } publish{p.head_flags ? p.head_ready + head : nullptr};
         const int row_lo = head * p.d + i, row_hi = row_lo + half;
         if (P.bias) {
             lo += pre ? pre_lo : bf16_bits_to_f32(P.bias[row_lo]);
@@ -807,9 +811,13 @@ __device__ __forceinline__ void codes4_to_f32(uint32_t w, float (&f)[4]) {
     f[2] = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7442)) - 8388736.f;
     f[3] = __uint_as_float(__byte_perm(u, 0x4B000000u, 0x7443)) - 8388736.f;
 }
+// wait_heads: there was no grid barrier behind the QKV projection; the CTA waits (bounded) until the heads it reads are
+// complete: its query head and, if its chunk ends with the row this step appends, the K and V head of its group.  Every
+// finished unit (row pair) of a head adds one to the head's counter (apply_epilogue), d/2 per layer.
 template <int D, int HG, int LPP, bool Q8 = false>
 __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, int n, int min_chunk, bool defer_merge,
-                                                unsigned char *xbuf, int tid, int *s_flag) {
+                                                unsigned char *xbuf, int tid, int *s_flag, bool wait_heads = false,
+                                                volatile int *abort_flag = nullptr, int *prof_idx = nullptr) {
     constexpr int TILE = 32 / LPP;   // positions per warp iteration
     constexpr int DV = D / 32, CPR = D / 8, CPL = CPR / LPP;
     constexpr int CPL8 = D / 16 / LPP;                  // 16-byte pieces (16 codes) of a compressed K row per lane
@@ -821,11 +829,28 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
     const int groups = p.nq / HG;                       // head groups served by separate CTAs
     int nch, chunk_len;
     att_chunking(p, n, HG, min_chunk, TILE, ncta, nch, chunk_len);
-    if (cta >= nch * groups) return;
+    if (cta >= nch * groups) {
+        if (wait_heads) prof_stamp(p, tid, *prof_idx);
+        return;
+    }
     const int grp = cta / nch, c = cta - grp * nch;
     const int qh0 = grp * HG;                            // first query head of this CTA
     const int g = qh0 / G;                               // its kv head
     const int t0 = c * chunk_len, t1 = min(n, t0 + chunk_len);
+    if (wait_heads) {
+        if (tid == 0 && !*abort_flag) {
+            const unsigned target = static_cast<unsigned>(layer + 1) * (D / 2);
+            const unsigned long long w0 = global_ns();
+            for (unsigned it = 0;; ++it) {
+                bool ready = ld_acquire_gpu(p.head_ready + qh0) >= target;
+                if (ready && t1 == n) ready = ld_acquire_gpu(p.head_ready + p.nq + g) >= target && ld_acquire_gpu(p.head_ready + p.nq + p.nkv + g) >= target;
+                if (ready) break;
+                if ((it & 63u) == 63u && global_ns() - w0 > p.spin_limit) { *abort_flag = 1; p.state->status = 6; break; }
+            }
+        }
+        cta_sync();
+        prof_stamp(p, tid, *prof_idx);   // the heads this CTA reads are complete
+    }
 
     float *qs = reinterpret_cast<float *>(xbuf);               // [HG][D]
     float *ps = qs + HG * D;                                    // [NW][HG][TILE]
@@ -1211,14 +1236,23 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
                 else if (p.kv8) attention_phase<D, G, MK_ATT_LPP, true>(p, l, n_att, p.att_chunk_shared, false, sm_xbuf(p), tid, &s_flag);
                 else attention_phase<D, G, MK_ATT_LPP>(p, l, n_att, p.att_chunk_shared, false, sm_xbuf(p), tid, &s_flag);
             } else {
-                attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, sm_xbuf(p), tid, &s_flag);
+                attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, sm_xbuf(p), tid, &s_flag,
+                                                        p.head_flags != 0, abort_flag, &prof_idx);
             }
             ok = grid_barrier(p, ++bar_no * bar_arrivals, abort_flag, tid, prof_idx) && ok;
             if (!ok) break;
         }
         ok = gemv_phase(p, ph, layer_op ? (ph & 3) : 4, ws, abort_flag, s_part, s_partial, s_rope, cx, token, after_attention ? merge_chunks : 0, tid,
                         prof_idx, s_issued, full_bar);
-        if (layer_op) ok = grid_barrier(p, ++bar_no * bar_arrivals, abort_flag, tid, prof_idx) && ok;
+        if (!LONG && p.head_flags && layer_op && (ph & 3) == 0) {
+            // no grid barrier behind the QKV projection: the attention phase waits for the heads it reads (the CTA-wide sync
+            // keeps the attention scratch, which shares the staged vector's memory, from being written under slower warps)
+            cta_sync();
+            prof_stamp(p, tid, prof_idx);
+            ok = ok && !*abort_flag;
+        } else if (layer_op) {
+            ok = grid_barrier(p, ++bar_no * bar_arrivals, abort_flag, tid, prof_idx) && ok;
+        }
     }
     prof_stamp(p, tid, prof_idx);
     if (!ok || *abort_flag) {
@@ -1280,6 +1314,8 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
             p.state->cur_len = slot_row + 1;
             p.tickets[p.nq] = 0u;
             *p.barrier = 0u;  // every CTA has passed the last grid barrier
+            if (p.head_flags)
+                for (int h = 0; h < p.nq + 2 * p.nkv; ++h) p.head_ready[h] = 0u;
         }
     }
 }

@@ -24,6 +24,9 @@ constexpr int MK_MAX_SLOTS = 4;                  // ring slots per consumer warp
 constexpr int MK_WARP_TAB = 8;                   // ints per warp in the per-CTA table
 // Consumer warps per CTA of the two builds of the kernel (one more warp prefetches into L2): the short-context build favours
 // instruction streams, the long-context build (grouped attention keeps G heads of accumulators per warp) registers.
+#ifndef MK_HEAD_FLAGS
+#define MK_HEAD_FLAGS 1   // short build: per-head completion counters instead of the grid barrier between QKV and attention
+#endif
 #ifndef MK_PF_TILES
 #define MK_PF_TILES 4   // tiles per consumer warp the helper warp asks L2 for ahead of the ring
 #endif
@@ -119,6 +122,8 @@ struct MkParams {
     int att_split_max_n;           // contexts up to this length use one-head-per-CTA attention
     unsigned *tickets;             // [nq] attention, [nq] = lm_head
     unsigned *barrier;             // grid barrier counter (0 between launches)
+    unsigned *head_ready;          // [nq + 2 nkv] finished units per head of the QKV projection, all layers of the step (0 between launches)
+    int head_flags;                // 1: no grid barrier between the QKV projection and attention; attention waits on head_ready (short build)
     float *lm_part_val;
     int *lm_part_idx;
     const int *vocab_ids;          // [V] token id of every row of a pruned lm_head (used when the last operator has PHF_REMAP)
