@@ -120,7 +120,11 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const uint16_t *src, c
 // long_ctx = false: the variant without the grouped (one CTA per GQA group) attention code, for contexts that
 // never need it.
 template <int D>
-MegaKernel mega_kernel_g(int G, bool long_ctx) {
+MegaKernel mega_kernel_g(int G, bool long_ctx, bool kv8 = false) {
+    if (kv8) {
+        if (D == 64) return G <= 4 ? mega_kernel_q8_d64_lo(G) : mega_kernel_q8_d64_hi(G);
+        return G <= 4 ? mega_kernel_q8_d128_lo(G) : mega_kernel_q8_d128_hi(G);
+    }
     if (!long_ctx) return mk_short::decode_megakernel<D, 1, false>;   // G is only used by the grouped attention
     if (D == 64) return G <= 4 ? mega_kernel_long_d64_lo(G) : mega_kernel_long_d64_hi(G);
     return G <= 4 ? mega_kernel_long_d128_lo(G) : mega_kernel_long_d128_hi(G);
@@ -147,7 +151,7 @@ inline const char *plan_step(const edgefm_shape &sh, int max_context, int num_sm
     *cuda_err = cudaSuccess;
     // (the compressed cache is attended by the grouped attention of the long-context build only)
     pl->long_ctx = kv8 || max_context > 8192 || static_cast<long long>(nq) * MK_ATT_SPLIT_MAXC * 2 > MK_PARTIAL_FLOATS;
-    pl->kernel = d == 64 ? mega_kernel_g<64>(G, pl->long_ctx) : mega_kernel_g<128>(G, pl->long_ctx);
+    pl->kernel = d == 64 ? mega_kernel_g<64>(G, pl->long_ctx, kv8) : mega_kernel_g<128>(G, pl->long_ctx, kv8);
     pl->nw = pl->long_ctx ? MK_NW_LONG : MK_NW_SHORT;
     pl->grid = num_sms;
     pl->max_chunks = pl->grid / nkv > 0 ? pl->grid / nkv : 1;

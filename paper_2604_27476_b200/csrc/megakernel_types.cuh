@@ -156,5 +156,10 @@ MegaKernel mega_kernel_long_d64_lo(int G);
 MegaKernel mega_kernel_long_d64_hi(int G);
 MegaKernel mega_kernel_long_d128_lo(int G);
 MegaKernel mega_kernel_long_d128_hi(int G);
+// ... and their variants for the compressed cache, defined in megakernel_q8_d*_*.cu
+MegaKernel mega_kernel_q8_d64_lo(int G);
+MegaKernel mega_kernel_q8_d64_hi(int G);
+MegaKernel mega_kernel_q8_d128_lo(int G);
+MegaKernel mega_kernel_q8_d128_hi(int G);
 
 }  // namespace edgefm

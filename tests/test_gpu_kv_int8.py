@@ -111,3 +111,31 @@ def test_unknown_cache_format_is_rejected():
         assert ei.value.status == Status.ERR_INVALID_ARG
     finally:
         pair.close()
+
+
+def test_prefix_plus_suffix_with_compressed_cache_equals_whole_prefill():
+    """edgefm_append_kv on a compressed cache compresses only the rows it appends: prefix + suffix gives the same codes,
+    scales and logits as one prefill of the whole (strided views of the device arrays as sources)."""
+    import torch
+    cfg = CONFIGS["tiny"]
+    pair = Pair(cfg, max_context=cfg.cache_len + 4, kv_format="int8")
+    try:
+        whole = [t.cpu().numpy() for t in pair.ctx.export_kv_int8()]
+        tok, pos = first_token(cfg), cfg.first_position
+        pair.ctx.step(tok, pos)
+        torch.cuda.synchronize()
+        logits_whole = pair.ctx.logits.cpu().numpy().copy()
+        pair.ctx.prefill_kv(pair.kd[:, :, :96], pair.vd[:, :, :96])
+        pair.ctx.append_kv(96, pair.kd[:, :, 96:], pair.vd[:, :, 96:])
+        assert pair.ctx.cur_len == cfg.cache_len
+        again = [t.cpu().numpy() for t in pair.ctx.export_kv_int8()]
+        n = cfg.cache_len
+        for a, b in zip(whole, again):
+            assert np.array_equal(a[:, :, :n], b[:, :, :n])
+        pair.ctx.step(tok, pos)
+        torch.cuda.synchronize()
+        assert np.array_equal(pair.ctx.logits.cpu().numpy(), logits_whole)
+        ref, _ = pair.oracle.step(tok, pos)
+        assert_logits_close(logits_whole, ref, "compressed prefix + suffix")
+    finally:
+        pair.close()
