@@ -16,14 +16,19 @@ struct StepState {
     int next_position;  // position the next step uses when the caller passes -1
     int status;         // 0 = ok (reserved for bounded-wait failures)
     int pad[2];
+    int n_accepted;     // tokens of the last block the cache was advanced by (1 for a plain step)
+    int reserved[3];
 };
 
 // What the host asks of the next step; uploaded only when it differs from the previous request.
 struct StepRequest {
     int token;          // >= 0 explicit, -1 = StepState::next_token
     int position;       // >= 0 explicit, -1 = StepState::next_position
-    float *logits_out;  // device fp32[V] or null
+    float *logits_out;  // device fp32[V] (a block of m tokens: [m][V]) or null
     int *next_token_out;  // device int32[1] or null
+    int m;              // tokens in this call: 1 = a plain decode step; > 1 = a block to verify (Sec. 3.11): `token` followed by
+    int draft[3];       // ... the proposed continuation draft[0 .. m-2]
+    int *n_accepted_out;  // device int32[1] or null: how many of the m tokens entered the cache (1 + accepted proposals)
 };
 
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }

@@ -38,6 +38,15 @@ namespace edgefm {
 namespace MK_NS {
 
 constexpr int MK_NW = MK_NW_VALUE;               // consumer warps per CTA
+#ifndef MK_M_VALUE
+#define MK_M_VALUE 1
+#endif
+// Tokens one call may carry.  1: the plain decode step.  M > 1 (a build of its own): a block of up to M tokens is pushed
+// through the step together -- the token to decode and proposed continuations (Sec. 3.11 of the paper: the base model
+// verifies a proposed block); the weights are streamed once, every token has its own activation vectors, and the tensor-core
+// product carries the tokens side by side in the columns of its B operand (three columns per token).
+constexpr int MK_M = MK_M_VALUE;
+static_assert(MK_M >= 1 && MK_M * MK_X_SPLITS <= 8, "the tokens of a block share the eight columns of one B operand");
 constexpr int MK_NT = MK_NW * 32;                // consumer threads
 constexpr int MK_THREADS = MK_NT + 32;           // + the L2 prefetch warp
 
@@ -421,27 +430,32 @@ __device__ __forceinline__ void prefetch_tiles(const MkParams &p, volatile int *
     }
 }
 
-struct ItemCtx {
-    float rscale;          // deferred RMSNorm factor (1 for plain prologues)
-    int slot_row;          // cache slot written by this step
-    float best_v;          // PH_LMHEAD running argmax of this lane
-    int best_i;
+struct ItemCtx {             // per token of the call
+    float rscale[MK_M];    // deferred RMSNorm factor (1 for plain prologues)
+    int slot_row;          // cache slot written by the first token (token t writes slot_row + t)
+    int m_run;             // tokens in this call (<= MK_M)
+    float best_v[MK_M];    // PH_LMHEAD running argmax of this lane
+    int best_i[MK_M];
 };
 
 // ---- fused epilogue of one output unit (a row, or a row pair) ------------------------------------------------
 // pre: the value the epilogue adds (old residual / the two biases) was fetched ahead into pre_lo, pre_hi.
+// tok: the token of the call this value belongs to (0 in the plain step).
 __device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkOp &P, ItemCtx &cx, const float *s_rope, int u, float lo, float hi,
-                                               bool pre = false, float pre_lo = 0.f, float pre_hi = 0.f) {
+                                               bool pre = false, float pre_lo = 0.f, float pre_hi = 0.f, int tok = 0) {
+    float *const out = MK_M > 1 ? P.out + static_cast<size_t>(tok) * P.out_tok_stride : P.out;
     if (P.kind == PH_RESID) {
-        P.out[u] = (pre ? pre_lo : __ldcg(P.out + u)) + lo;
+        out[u] = (pre ? pre_lo : __ldcg(out + u)) + lo;
     } else if (P.kind == PH_LMHEAD) {
         float *logits_out = p.req->logits_out;
-        if (logits_out) logits_out[u] = lo;
-        if (arg_better(lo, u, cx.best_v, cx.best_i)) { cx.best_v = lo; cx.best_i = u; }
+        if (logits_out) logits_out[(MK_M > 1 ? static_cast<size_t>(tok) * P.units_total : 0) + u] = lo;
+#pragma unroll
+        for (int t = 0; t < MK_M; ++t)
+            if (t == tok && arg_better(lo, u, cx.best_v[t], cx.best_i[t])) { cx.best_v[t] = lo; cx.best_i[t] = u; }
     } else if (P.kind == PH_SWIGLU) {
         const float a = lo / (1.f + expf(-lo)) * hi;
         if (P.flags() & PHF_OUT_SPLIT) {   // the layout the next operator's prologue copies straight into shared memory
-            uint16_t *o = reinterpret_cast<uint16_t *>(P.out) + mk_xs_index(u);
+            uint16_t *o = reinterpret_cast<uint16_t *>(P.out) + (MK_M > 1 ? static_cast<size_t>(tok) * P.out_tok_stride : 0) + mk_xs_index(u);
             float r = a;
 #pragma unroll
             for (int sp = 0; sp < MK_X_SPLITS; ++sp) {
@@ -450,7 +464,7 @@ __device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkOp &P,
                 r -= bf16_bits_to_f32(b);
             }
         } else {
-            P.out[u] = a;
+            out[u] = a;
         }
     } else {  // PH_QKV: bias, rotate-half RoPE of q and k, q to the work buffer, k and v to the cache row of this step
         const int half = p.d >> 1;
@@ -466,17 +480,17 @@ __device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkOp &P,
         }
         const size_t layer_off = static_cast<size_t>(P.layer()) * p.nkv * p.max_context * p.d;
         if (head < p.nq + p.nkv) {
-            const float c = s_rope[i], sn = s_rope[half + i];
+            const float c = s_rope[tok * 128 + i], sn = s_rope[tok * 128 + half + i];   // the table of this token's position
             const float rlo = lo * c - hi * sn, rhi = hi * c + lo * sn;
             if (head < p.nq) {
-                P.out[row_lo] = rlo;
-                P.out[row_hi] = rhi;
+                out[row_lo] = rlo;
+                out[row_hi] = rhi;
             } else if (p.kv8) {   // compressed cache: the row is left in fp32 for the attention phase, which compresses it whole
                 float *dst = p.kv_stage + static_cast<size_t>(head - p.nq) * p.d;
                 dst[i] = rlo;
                 dst[i + half] = rhi;
             } else {
-                uint16_t *dst = p.k_cache + layer_off + (static_cast<size_t>(head - p.nq) * p.max_context + cx.slot_row) * p.d;
+                uint16_t *dst = p.k_cache + layer_off + (static_cast<size_t>(head - p.nq) * p.max_context + cx.slot_row + tok) * p.d;
                 dst[i] = f32_to_bf16_bits(rlo);
                 dst[i + half] = f32_to_bf16_bits(rhi);
             }
@@ -485,7 +499,7 @@ __device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkOp &P,
             dst[i] = lo;
             dst[i + half] = hi;
         } else {
-            uint16_t *dst = p.v_cache + layer_off + (static_cast<size_t>(head - p.nq - p.nkv) * p.max_context + cx.slot_row) * p.d;
+            uint16_t *dst = p.v_cache + layer_off + (static_cast<size_t>(head - p.nq - p.nkv) * p.max_context + cx.slot_row + tok) * p.d;
             dst[i] = f32_to_bf16_bits(lo);
             dst[i + half] = f32_to_bf16_bits(hi);
         }
@@ -530,20 +544,20 @@ __device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkOp &P, 
     // tile are copied asynchronously (no registers held) as soon as the current tile has been multiplied.
     const bool xg = (P.flags() & PHF_X_GLOBAL) != 0;
     const int kpad2 = (P.K + MK_TILE_COLS - 1) / MK_TILE_COLS * (MK_TILE_COLS * 2);
-    unsigned char *wbuf = sm_xbuf(p) + p.xbuf_bytes + warp * MK_WBUF_BYTES;
+    unsigned char *wbuf = sm_xbuf(p) + p.xbuf_bytes + warp * (MK_WBUF_BYTES * MK_M);   // [token][piece][512 + pad bytes]
     const unsigned char *b_base = xg ? wbuf + (lane >> 2) * (MK_TILE_COLS * 2 + MK_XS_PAD) + (lane & 3) * 16
                                      : sm_xbuf(p) + (lane >> 2) * xs_stride(P.K) + (lane & 3) * 16;
     auto request_b = [&](int kcol) {
         const unsigned char *src = reinterpret_cast<const unsigned char *>(P.x_src) + kcol * (MK_TILE_COLS * 2) + lane * 16;
 #pragma unroll
-        for (int sp = 0; sp < MK_X_SPLITS; ++sp)
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(wbuf + sp * (MK_TILE_COLS * 2 + MK_XS_PAD) + lane * 16)),
-                         "l"(src + static_cast<size_t>(sp) * kpad2) : "memory");
+        for (int c = 0; c < MK_X_SPLITS * MK_M; ++c)   // array c: piece c % 3 of token c / 3
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(wbuf + c * (MK_TILE_COLS * 2 + MK_XS_PAD) + lane * 16)),
+                         "l"(src + static_cast<size_t>(c / MK_X_SPLITS) * P.x_tok_stride * 2 + static_cast<size_t>(c % MK_X_SPLITS) * kpad2) : "memory");
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
     auto load_b = [&](const unsigned char *at) {
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (lane < 4 * MK_X_SPLITS) v = *reinterpret_cast<const uint4 *>(at);
+        if (lane < 4 * MK_X_SPLITS * MK_M) v = *reinterpret_cast<const uint4 *>(at);
         return v;
     };
     // A fragments: ldmatrix.x4 takes from lane l the address of row l % 8 of matrix l / 8; the four matrices are
@@ -606,21 +620,38 @@ __device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkOp &P, 
             float d0 = acc[0][0], d1 = acc[0][1], d2 = acc[0][2], d3 = acc[0][3];
 #pragma unroll
             for (int c = 1; c < MK_ACC_CHAINS; ++c) { d0 += acc[c][0]; d1 += acc[c][1]; d2 += acc[c][2]; d3 += acc[c][3]; }
-            const float lo = d0 + d1 + __shfl_down_sync(0xffffffffu, d0, 1);
-            const float hi = d2 + d3 + __shfl_down_sync(0xffffffffu, d2, 1);
-            const int src = ((lane >> 1) & 7) * 4;
-            const float vlo = __shfl_sync(0xffffffffu, lo, src), vhi = __shfl_sync(0xffffffffu, hi, src);
-            const float v = lane < 16 ? vlo : vhi;
-            const int j = lane >> 1;
-            if (d.y & MKT_DIRECT) {
-                const float hi2 = __shfl_down_sync(0xffffffffu, v, 16);   // partner row 8 + j of unit j
-                const int v0 = static_cast<int>((d.y >> 5) & 15u);
-                const int u = static_cast<int>(d.x & 0xfffffu) + j;
-                if (!(lane & 1) && j < m && j >= v0 && (!paired || lane < 16)) apply_epilogue(p, P, cx, s_rope, u, v * cx.rscale, hi2 * cx.rscale);
-            } else {
-                const int slot = static_cast<int>((d.y >> 10) & 1023u);
-                if (slot >= MK_PARTIAL_SLOTS) return diag_fail(p, abort_flag, 2, slot, 0);
-                if (!(lane & 1)) s_partial[slot * MK_TILE_ROWS + j] = v;
+#pragma unroll
+            for (int tk = 0; tk < MK_M; ++tk) {
+                float lo, hi;
+                if constexpr (MK_M == 1) {
+                    lo = d0 + d1 + __shfl_down_sync(0xffffffffu, d0, 1);
+                    hi = d2 + d3 + __shfl_down_sync(0xffffffffu, d2, 1);
+                } else {
+                    // token tk: columns 3 tk .. 3 tk + 2; column c is register c % 2 of the lane with lane % 4 == c / 2
+                    lo = 0.f; hi = 0.f;
+#pragma unroll
+                    for (int sp = 0; sp < MK_X_SPLITS; ++sp) {
+                        const int c = MK_X_SPLITS * tk + sp;
+                        lo += __shfl_sync(0xffffffffu, (c & 1) ? d1 : d0, (lane & ~3) + (c >> 1));
+                        hi += __shfl_sync(0xffffffffu, (c & 1) ? d3 : d2, (lane & ~3) + (c >> 1));
+                    }
+                }
+                const int src = ((lane >> 1) & 7) * 4;
+                const float vlo = __shfl_sync(0xffffffffu, lo, src), vhi = __shfl_sync(0xffffffffu, hi, src);
+                const float v = lane < 16 ? vlo : vhi;
+                const int j = lane >> 1;
+                if (tk >= cx.m_run) continue;     // (uniform over the warp)
+                if (d.y & MKT_DIRECT) {
+                    const float hi2 = __shfl_down_sync(0xffffffffu, v, 16);   // partner row 8 + j of unit j
+                    const int v0 = static_cast<int>((d.y >> 5) & 15u);
+                    const int u = static_cast<int>(d.x & 0xfffffu) + j;
+                    if (!(lane & 1) && j < m && j >= v0 && (!paired || lane < 16))
+                        apply_epilogue(p, P, cx, s_rope, u, v * cx.rscale[tk], hi2 * cx.rscale[tk], false, 0.f, 0.f, tk);
+                } else {
+                    const int slot = static_cast<int>((d.y >> 10) & 1023u);
+                    if (slot >= MK_PARTIAL_SLOTS) return diag_fail(p, abort_flag, 2, slot, 0);
+                    if (!(lane & 1)) s_partial[(slot * MK_M + tk) * MK_TILE_ROWS + j] = v;
+                }
             }
         }
         d = dn;
@@ -635,18 +666,25 @@ __device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkOp &P, 
 // merge_attn > 0: the input is the attention output, still split into merge_attn chunk partials per head
 // (m, l, unnormalised o); the exact log-sum-exp merge is done here, in chunk order, by every CTA.
 __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_layer, WarpStream &ws, volatile int *abort_flag, float *s_part,
-                                           float *s_partial, const float *s_rope, ItemCtx &cx, int token, int merge_attn, int tid, int &prof_idx,
-                                           volatile unsigned *s_issued, unsigned long long *full_bar) {
+                                           float *s_partial, const float *s_rope, ItemCtx &cx, const int (&tokens)[MK_M], int merge_attn, int n_att, int tid,
+                                           int &prof_idx, volatile unsigned *s_issued, unsigned long long *full_bar) {
     const MkOp &P = sm_ops(p)[ph];
-    unsigned char *xs = sm_xbuf(p);
+    unsigned char *const xs0 = sm_xbuf(p);
     const int xstride = xs_stride(P.K);
     const int *s_tab = sm_tab(p);
     const int lane = tid & 31, warp = tid >> 5;
     const int cta = blockIdx.x;
     const int n4 = P.K >> 2;
+    // the tokens of the call one after the other: token tk stages its vector into arrays 3 tk .. 3 tk + 2
+    for (int tk = 0; tk < cx.m_run; ++tk) {
+    unsigned char *const xs = xs0 + tk * (MK_X_SPLITS * xstride);
+    const int token = tokens[tk < MK_M ? tk : 0];
     float ss = 0.f;
     if (merge_attn > 0) {
-        const int nch = merge_attn;
+        int nch = merge_attn;
+        if (MK_M > 1) { int cl; att_chunking(p, n_att + tk, 1, p.att_chunk_split, 32 / MK_ATT_LPP_SPLIT, static_cast<int>(gridDim.x), nch, cl); }
+        const float *part_o = p.part_o + static_cast<size_t>(tk) * p.nq * p.max_chunks * p.d;
+        const float *part_m = p.part_m + static_cast<size_t>(tk) * p.nq * p.max_chunks, *part_l = p.part_l + static_cast<size_t>(tk) * p.nq * p.max_chunks;
         const int d4 = p.d >> 2;
         float *sm_m = s_partial;                 // [nq][nch] chunk maxima
         float *sm_l = s_partial + p.nq * nch;    // [nq][nch] chunk denominators
@@ -657,7 +695,7 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_
         float4 ob[MK_ATT_SPLIT_MAXC];
         auto load_partials = [&](int o4) {
             const int h = o4 / d4, j4 = o4 - h * d4;
-            const float4 *po = reinterpret_cast<const float4 *>(p.part_o + static_cast<size_t>(h) * p.max_chunks * p.d) + j4;
+            const float4 *po = reinterpret_cast<const float4 *>(part_o + static_cast<size_t>(h) * p.max_chunks * p.d) + j4;
 #pragma unroll
             for (int c = 0; c < MK_ATT_SPLIT_MAXC; ++c)
                 if (c < nch) ob[c] = __ldcg(po + static_cast<size_t>(c) * d4);
@@ -665,8 +703,8 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_
         if (tid < n4) load_partials(tid);
         for (int i = tid; i < p.nq * nch; i += MK_NT) {
             const int h = i / nch, c = i - h * nch;
-            sm_m[i] = __ldcg(p.part_m + h * p.max_chunks + c);
-            sm_l[i] = __ldcg(p.part_l + h * p.max_chunks + c);
+            sm_m[i] = __ldcg(part_m + h * p.max_chunks + c);
+            sm_l[i] = __ldcg(part_l + h * p.max_chunks + c);
         }
         cta_sync();
         for (int o4 = tid; o4 < n4; o4 += MK_NT) {
@@ -690,6 +728,7 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_
             acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
             stage_piece(xs, xstride, o4, acc);
         }
+        if (MK_M > 1) cta_sync();   // the statistics area is reused by the next token
     } else if (P.flags() & PHF_X_GLOBAL) {
         // nothing to stage: the consumer warps read the vector from global memory as they go
     } else {
@@ -702,7 +741,7 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_
                 const int i4 = base + u * MK_NT;
                 if (i4 < n4) {
                     if (P.x_src) {
-                        v[u] = __ldcg(reinterpret_cast<const float4 *>(P.x_src) + i4);
+                        v[u] = __ldcg(reinterpret_cast<const float4 *>(P.x_src + (MK_M > 1 ? static_cast<size_t>(tk) * P.x_tok_stride : 0)) + i4);
                     } else {  // first operator of the step: the embedding row is the residual stream
                         const uint2 e = *reinterpret_cast<const uint2 *>(p.embed + static_cast<size_t>(token) * p.H + i4 * 4);
                         v[u] = make_float4(bf16lo(e.x), bf16hi(e.x), bf16lo(e.y), bf16hi(e.y));
@@ -715,7 +754,7 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_
                 const int i4 = base + u * MK_NT;
                 if (i4 < n4) {
                     float4 t = v[u];
-                    if (!P.x_src && cta == 0) reinterpret_cast<float4 *>(p.x)[i4] = t;
+                    if (!P.x_src && cta == 0) reinterpret_cast<float4 *>(p.x + (MK_M > 1 ? static_cast<size_t>(tk) * p.H : 0))[i4] = t;
                     if (P.norm_w) {
                         ss = fmaf(t.x, t.x, ss); ss = fmaf(t.y, t.y, ss); ss = fmaf(t.z, t.z, ss); ss = fmaf(t.w, t.w, ss);
                         t.x *= bf16lo(w[u].x); t.y *= bf16hi(w[u].x); t.z *= bf16lo(w[u].y); t.w *= bf16hi(w[u].y);
@@ -733,16 +772,20 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_
     }
     if (P.norm_w) {
         ss = warp_sum(ss);
-        if (lane == 0) s_part[warp] = ss;
+        if (lane == 0) s_part[tk * MK_NW + warp] = ss;
     }
+    }   // tokens
     cta_sync();
     prof_stamp(p, tid, prof_idx);   // activation vector staged
-    cx.rscale = 1.f;
-    if (P.norm_w) {
-        float tot = 0.f;
 #pragma unroll
-        for (int w = 0; w < MK_NW; ++w) tot += s_part[w];
-        cx.rscale = rsqrtf(tot / static_cast<float>(P.K) + p.eps);
+    for (int tk = 0; tk < MK_M; ++tk) {
+        cx.rscale[tk] = 1.f;
+        if (P.norm_w && tk < cx.m_run) {
+            float tot = 0.f;
+#pragma unroll
+            for (int w = 0; w < MK_NW; ++w) tot += s_part[tk * MK_NW + w];
+            cx.rscale[tk] = rsqrtf(tot / static_cast<float>(P.K) + p.eps);
+        }
     }
     const int *tab = s_tab + warp * MK_WARP_TAB;
     const int n_tiles = op_in_layer < 4 ? tab[1 + op_in_layer] : tab[6];
@@ -776,13 +819,19 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_
                 const MkCombine e = cb[idx >> 4];
                 const int j = idx & 15, m = static_cast<int>(e.y & 0xffu), v0 = static_cast<int>(e.y >> 8);
                 if (j >= m || j < v0 || (paired && j >= 8)) continue;
-                float lo = 0.f, hi = 0.f;
-                for (unsigned s = 0; s < e.w; ++s) {
-                    const float *sp = s_partial + (e.z + s) * MK_TILE_ROWS;
-                    lo += sp[j];
-                    if (paired) hi += sp[8 + j];
+#pragma unroll
+                for (int tk = 0; tk < MK_M; ++tk) {
+                    if (tk >= cx.m_run) break;
+                    float lo = 0.f, hi = 0.f;
+                    for (unsigned s = 0; s < e.w; ++s) {
+                        const float *sp = s_partial + ((e.z + s) * MK_M + tk) * MK_TILE_ROWS;
+                        lo += sp[j];
+                        if (paired) hi += sp[8 + j];
+                    }
+                    // (what the epilogue adds was fetched ahead for the first token only)
+                    apply_epilogue(p, P, cx, s_rope, static_cast<int>(e.x) + j, lo * cx.rscale[tk], hi * cx.rscale[tk], idx == tid && (tk == 0 || P.kind == PH_QKV), pre_lo,
+                                   pre_hi, tk);
                 }
-                apply_epilogue(p, P, cx, s_rope, static_cast<int>(e.x) + j, lo * cx.rscale, hi * cx.rscale, idx == tid, pre_lo, pre_hi);
             }
         }
     }
@@ -817,7 +866,9 @@ __device__ __forceinline__ void codes4_to_f32(uint32_t w, float (&f)[4]) {
 template <int D, int HG, int LPP, bool Q8 = false>
 __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, int n, int min_chunk, bool defer_merge,
                                                 unsigned char *xbuf, int tid, int *s_flag, bool wait_heads = false,
-                                                volatile int *abort_flag = nullptr, int *prof_idx = nullptr) {
+                                                volatile int *abort_flag = nullptr, int *prof_idx = nullptr, int tok = 0, int m_run = 1) {
+    static_assert(!(Q8 && MK_M > 1), "blocks of several tokens are built for the plain cache only");
+    // token `tok` of a call of m_run tokens: its own queries and partial results; n counts the rows of the tokens before it
     constexpr int TILE = 32 / LPP;   // positions per warp iteration
     constexpr int DV = D / 32, CPR = D / 8, CPL = CPR / LPP;
     constexpr int CPL8 = D / 16 / LPP;                  // 16-byte pieces (16 codes) of a compressed K row per lane
@@ -830,26 +881,30 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
     int nch, chunk_len;
     att_chunking(p, n, HG, min_chunk, TILE, ncta, nch, chunk_len);
     if (cta >= nch * groups) {
-        if (wait_heads) prof_stamp(p, tid, *prof_idx);
+        if (wait_heads && tok == 0) prof_stamp(p, tid, *prof_idx);
         return;
     }
+    const float *const q_tok = p.q + static_cast<size_t>(tok) * p.nq * D;
+    float *const attn_tok = p.attn + static_cast<size_t>(tok) * p.nq * D;
+    float *const part_o = p.part_o + static_cast<size_t>(tok) * p.nq * p.max_chunks * D;
+    float *const part_m = p.part_m + static_cast<size_t>(tok) * p.nq * p.max_chunks, *const part_l = p.part_l + static_cast<size_t>(tok) * p.nq * p.max_chunks;
     const int grp = cta / nch, c = cta - grp * nch;
     const int qh0 = grp * HG;                            // first query head of this CTA
     const int g = qh0 / G;                               // its kv head
     const int t0 = c * chunk_len, t1 = min(n, t0 + chunk_len);
     if (wait_heads) {
         if (tid == 0 && !*abort_flag) {
-            const unsigned target = static_cast<unsigned>(layer + 1) * (D / 2);
+            const unsigned target = static_cast<unsigned>(layer + 1) * (D / 2) * static_cast<unsigned>(m_run);
             const unsigned long long w0 = global_ns();
             for (unsigned it = 0;; ++it) {
                 bool ready = ld_acquire_gpu(p.head_ready + qh0) >= target;
-                if (ready && t1 == n) ready = ld_acquire_gpu(p.head_ready + p.nq + g) >= target && ld_acquire_gpu(p.head_ready + p.nq + p.nkv + g) >= target;
+                if (ready && t1 > n - 1 - tok) ready = ld_acquire_gpu(p.head_ready + p.nq + g) >= target && ld_acquire_gpu(p.head_ready + p.nq + p.nkv + g) >= target;
                 if (ready) break;
                 if ((it & 63u) == 63u && global_ns() - w0 > p.spin_limit) { *abort_flag = 1; p.state->status = 6; break; }
             }
         }
         cta_sync();
-        prof_stamp(p, tid, *prof_idx);   // the heads this CTA reads are complete
+        if (tok == 0) prof_stamp(p, tid, *prof_idx);   // the heads this CTA reads are complete
     }
 
     float *qs = reinterpret_cast<float *>(xbuf);               // [HG][D]
@@ -935,7 +990,7 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
         }
     };
     int tt = t0 + warp * TILE;
-    for (int i = tid; i < HG * D; i += MK_NT) qs[i] = __ldcg(p.q + static_cast<size_t>(qh0) * D + i) * p.scale;
+    for (int i = tid; i < HG * D; i += MK_NT) qs[i] = __ldcg(q_tok + static_cast<size_t>(qh0) * D + i) * p.scale;
     cta_sync();
 
     float m[HG], l[HG], o[HG][DV];
@@ -1057,10 +1112,10 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
         }
         const int qh = qh0 + h;
         if (nch == 1 && !defer_merge) {  // nothing to merge across CTAs
-            p.attn[qh * D + j] = oo / ll;
+            attn_tok[qh * D + j] = oo / ll;
         } else {
-            p.part_o[(static_cast<size_t>(qh) * p.max_chunks + c) * D + j] = oo;
-            if (j == 0) { p.part_m[qh * p.max_chunks + c] = mm; p.part_l[qh * p.max_chunks + c] = ll; }
+            part_o[(static_cast<size_t>(qh) * p.max_chunks + c) * D + j] = oo;
+            if (j == 0) { part_m[qh * p.max_chunks + c] = mm; part_l[qh * p.max_chunks + c] = ll; }
         }
     }
     if (nch == 1 || defer_merge) return;   // deferred: the next operator's prologue merges the chunks
@@ -1076,13 +1131,13 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
     constexpr int CB = 8;
     for (int i = tid; i < HG * nch; i += MK_NT) {
         const int h = i / nch, cc = i - h * nch;
-        cm[h * p.max_chunks + cc] = __ldcg(p.part_m + (qh0 + h) * p.max_chunks + cc);
-        cl[h * p.max_chunks + cc] = __ldcg(p.part_l + (qh0 + h) * p.max_chunks + cc);
+        cm[h * p.max_chunks + cc] = __ldcg(part_m + (qh0 + h) * p.max_chunks + cc);
+        cl[h * p.max_chunks + cc] = __ldcg(part_l + (qh0 + h) * p.max_chunks + cc);
     }
     cta_sync();
     for (int out = tid; out < HG * D / 4; out += MK_NT) {     // output (h, j4) of this thread
         const int oh = out / (D / 4), oj4 = out - oh * (D / 4);
-        const float4 *po = reinterpret_cast<const float4 *>(p.part_o + static_cast<size_t>(qh0 + oh) * p.max_chunks * D) + oj4;
+        const float4 *po = reinterpret_cast<const float4 *>(part_o + static_cast<size_t>(qh0 + oh) * p.max_chunks * D) + oj4;
         const float *hm = cm + oh * p.max_chunks, *hl = cl + oh * p.max_chunks;
         float mm = -INFINITY;
         for (int cc = 0; cc < nch; ++cc) mm = fmaxf(mm, hm[cc]);
@@ -1105,7 +1160,7 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
         }
         const float inv = 1.f / ll;
         acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-        reinterpret_cast<float4 *>(p.attn)[(qh0 + oh) * (D / 4) + oj4] = acc;
+        reinterpret_cast<float4 *>(attn_tok)[(qh0 + oh) * (D / 4) + oj4] = acc;
     }
     if (tid == 0) p.tickets[grp] = 0u;
 }
@@ -1118,11 +1173,11 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
 template <int D, int G, bool LONG, bool Q8 = false>
 __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParams p) {
     __shared__ __align__(8) unsigned long long full_bar[MK_NW * MK_MAX_SLOTS];
-    __shared__ float s_rope[128];
-    __shared__ float s_part[MK_NW];
-    __shared__ __align__(16) float s_partial[MK_PARTIAL_FLOATS];
-    __shared__ float s_bv[MK_NW];
-    __shared__ int s_bi[MK_NW];
+    __shared__ float s_rope[MK_M * 128];     // per token of the call: cos | sin of its position
+    __shared__ float s_part[MK_M * MK_NW];
+    __shared__ __align__(16) float s_partial[MK_M * MK_PARTIAL_FLOATS];
+    __shared__ float s_bv[MK_M * MK_NW];
+    __shared__ int s_bi[MK_M * MK_NW];
     __shared__ int s_flag;
     __shared__ int s_abort;
     __shared__ unsigned s_issued[MK_NW];   // tiles fetched so far per consumer warp (read by the L2 prefetch warp)
@@ -1183,15 +1238,27 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
     const int pos = rp >= 0 ? rp : p.state->next_position;
     const int slot_row = p.state->cur_len;
     const int half = p.d >> 1;
-    if (token < 0 || token >= p.V || slot_row < 0 || slot_row >= p.max_context || pos < 0 || (smem_u32(sm_ring(p, 0)) & 1023u)) {
+    // a block: the token above followed by the proposed continuation, at consecutive positions and cache slots
+    const int m_run = MK_M > 1 ? min(max(p.req->m, 1), MK_M) : 1;
+    int tokens[MK_M];
+    tokens[0] = token;
+#pragma unroll
+    for (int t = 1; t < MK_M; ++t) tokens[t] = t < m_run ? p.req->draft[t - 1] : 0;
+    bool tokens_ok = true;
+#pragma unroll
+    for (int t = 0; t < MK_M; ++t) tokens_ok = tokens_ok && tokens[t] >= 0 && tokens[t] < p.V;
+    if (!tokens_ok || slot_row < 0 || slot_row + m_run > p.max_context || pos < 0 || (smem_u32(sm_ring(p, 0)) & 1023u)) {
         if (tid == 0) diag_fail(p, abort_flag, 3, token, slot_row);   // corrupt request/state (or ring slots off their 1 KB boundary): compute nothing
         ok = false;
     }
-    if (ok && tid < half) {  // rotary table of this step's position; fp64 angle, rounded once
-        double sn, cs;
-        sincos(static_cast<double>(pos) * p.inv_freq[tid], &sn, &cs);
-        s_rope[tid] = static_cast<float>(cs);
-        s_rope[half + tid] = static_cast<float>(sn);
+    if (ok) {  // rotary tables of the tokens' positions; fp64 angle, rounded once
+        for (int i = tid; i < m_run * half; i += MK_NT) {
+            const int t = i / half, f = i - t * half;
+            double sn, cs;
+            sincos(static_cast<double>(pos + t) * p.inv_freq[f], &sn, &cs);
+            s_rope[t * 128 + f] = static_cast<float>(cs);
+            s_rope[t * 128 + half + f] = static_cast<float>(sn);
+        }
     }
     if (ok && cta == 0 && tid == 0) { p.state->token = token; p.state->position = pos; }
     if (ok && cta == 1 % ncta && p.nph > 2) {
@@ -1201,7 +1268,7 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
         uint16_t *a = reinterpret_cast<uint16_t *>(sm_ops(p)[2].out);
         for (int c = p.F + tid; c < fpad; c += MK_NT)
 #pragma unroll
-            for (int sp = 0; sp < MK_X_SPLITS; ++sp) a[static_cast<size_t>(sp) * fpad + mk_xs_index(c)] = 0;
+            for (int sp = 0; sp < MK_X_SPLITS * MK_M; ++sp) a[static_cast<size_t>(sp) * fpad + mk_xs_index(c)] = 0;   // (the tokens' arrays follow one another)
     }
     // (s_rope is published by the sync of the first prologue)
 
@@ -1211,7 +1278,9 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
 
     ItemCtx cx;
-    cx.rscale = 1.f; cx.slot_row = slot_row; cx.best_v = -INFINITY; cx.best_i = 0x7fffffff;
+    cx.slot_row = slot_row; cx.m_run = m_run;
+#pragma unroll
+    for (int t = 0; t < MK_M; ++t) { cx.rscale[t] = 1.f; cx.best_v[t] = -INFINITY; cx.best_i[t] = 0x7fffffff; }
 
     unsigned bar_no = 0;
     const unsigned bar_arrivals = static_cast<unsigned>(ncta + p.barrier_extra);
@@ -1237,13 +1306,17 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
                 if (att_split) attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, sm_xbuf(p), tid, &s_flag);
                 else attention_phase<D, G, MK_ATT_LPP, Q8>(p, l, n_att, p.att_chunk_shared, false, sm_xbuf(p), tid, &s_flag);
             } else {
-                attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, sm_xbuf(p), tid, &s_flag,
-                                                        p.head_flags != 0, abort_flag, &prof_idx);
+                // (a block: the tokens one after the other; token t also attends to the rows of the tokens before it)
+                for (int t = 0; t < m_run; ++t) {
+                    if (MK_M > 1 && t > 0) cta_sync();   // the scratch of the previous token's pass is free
+                    attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att + t, p.att_chunk_split, MK_SPLIT_DEFER != 0, sm_xbuf(p), tid, &s_flag,
+                                                            p.head_flags != 0, abort_flag, &prof_idx, t, m_run);
+                }
             }
             ok = grid_barrier(p, ++bar_no * bar_arrivals, abort_flag, tid, prof_idx) && ok;
             if (!ok) break;
         }
-        ok = gemv_phase(p, ph, layer_op ? (ph & 3) : 4, ws, abort_flag, s_part, s_partial, s_rope, cx, token, after_attention ? merge_chunks : 0, tid,
+        ok = gemv_phase(p, ph, layer_op ? (ph & 3) : 4, ws, abort_flag, s_part, s_partial, s_rope, cx, tokens, after_attention ? merge_chunks : 0, n_att, tid,
                         prof_idx, s_issued, full_bar);
         if (!LONG && p.head_flags && layer_op && (ph & 3) == 0) {
             // no grid barrier behind the QKV projection: the attention phase waits for the heads it reads (the CTA-wide sync
@@ -1271,21 +1344,30 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
     }
 
     // ---- greedy sampling: warp -> CTA -> last CTA reduces all partials, then the state advances -------------
-    float bv = cx.best_v;
-    int bi = cx.best_i;
+    // (a block: one greedy token per token of the call; partials of token t at [t][cta])
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-        if (arg_better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+    for (int t = 0; t < MK_M; ++t) {
+        float bv = cx.best_v[t];
+        int bi = cx.best_i[t];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (arg_better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+        }
+        if (lane == 0) { s_bv[t * MK_NW + warp] = bv; s_bi[t * MK_NW + warp] = bi; }
     }
-    if (lane == 0) { s_bv[warp] = bv; s_bi[warp] = bi; }
     cta_sync();
     if (tid == 0) {
-        for (int w = 1; w < MK_NW; ++w)
-            if (arg_better(s_bv[w], s_bi[w], bv, bi)) { bv = s_bv[w]; bi = s_bi[w]; }
-        p.lm_part_val[cta] = bv;
-        p.lm_part_idx[cta] = bi;
+#pragma unroll
+        for (int t = 0; t < MK_M; ++t) {
+            float bv = s_bv[t * MK_NW];
+            int bi = s_bi[t * MK_NW];
+            for (int w = 1; w < MK_NW; ++w)
+                if (arg_better(s_bv[t * MK_NW + w], s_bi[t * MK_NW + w], bv, bi)) { bv = s_bv[t * MK_NW + w]; bi = s_bi[t * MK_NW + w]; }
+            p.lm_part_val[t * ncta + cta] = bv;
+            p.lm_part_idx[t * ncta + cta] = bi;
+        }
         __threadfence();
         s_flag = (atomicAdd(p.tickets + p.nq, 1u) == static_cast<unsigned>(ncta - 1)) ? 1 : 0;
     }
@@ -1293,26 +1375,45 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
     if (!s_flag) return;
     __threadfence();
     if (warp == 0) {
-        bv = -INFINITY; bi = 0x7fffffff;
-        for (int i = lane; i < ncta; i += 32) {
-            const float v = __ldcg(p.lm_part_val + i);
-            const int ix = __ldcg(p.lm_part_idx + i);
-            if (arg_better(v, ix, bv, bi)) { bv = v; bi = ix; }
-        }
+        int greedy[MK_M];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-            if (arg_better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
-        }
-        if (lane == 0) {
+        for (int t = 0; t < MK_M; ++t) {
+            float bv = -INFINITY;
+            int bi = 0x7fffffff;
+            for (int i = lane; i < ncta; i += 32) {
+                const float v = __ldcg(p.lm_part_val + t * ncta + i);
+                const int ix = __ldcg(p.lm_part_idx + t * ncta + i);
+                if (arg_better(v, ix, bv, bi)) { bv = v; bi = ix; }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                if (arg_better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+            }
             if (bi == 0x7fffffff) bi = 0;
             if (sm_ops(p)[p.nph - 1].flags() & PHF_REMAP) bi = p.vocab_ids[bi];   // pruned vocabulary: row index -> token id
+            greedy[t] = bi;
+        }
+        if (lane == 0) {
+            // Verification (Sec. 3.11): proposal t + 1 is accepted if it is the base model's greedy choice after token t;
+            // it stops at the first rejection.  The cache advances by the accepted tokens; the rows of the rejected ones
+            // stay behind the cache length and are overwritten by the next call.
+            int n_acc = 1;
+#pragma unroll
+            for (int t = 1; t < MK_M; ++t)
+                if (t < m_run && n_acc == t && tokens[t] == greedy[t - 1]) n_acc = t + 1;
+            int bi = greedy[0];
+#pragma unroll
+            for (int t = 1; t < MK_M; ++t)
+                if (n_acc == t + 1) bi = greedy[t];
             int *nto = p.req->next_token_out;
             if (nto) *nto = bi;
+            if (MK_M > 1 && p.req->n_accepted_out) *p.req->n_accepted_out = n_acc;
             p.state->next_token = bi;
-            p.state->next_position = pos + 1;
-            p.state->cur_len = slot_row + 1;
+            p.state->next_position = pos + n_acc;
+            p.state->cur_len = slot_row + n_acc;
+            p.state->n_accepted = n_acc;
             p.tickets[p.nq] = 0u;
             *p.barrier = 0u;  // every CTA has passed the last grid barrier
             if (p.head_flags)

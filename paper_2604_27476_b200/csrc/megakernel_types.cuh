@@ -73,6 +73,9 @@ struct alignas(16) MkOp {
     int kind;
     int units_total;         // rows (PH_RESID, PH_LMHEAD), pairs (PH_QKV: rows/2, PH_SWIGLU: F)
     int layer_flags;         // layer << 8 | PHF_* bits
+    int x_tok_stride;        // a block of several tokens: elements (of x_src's type; PHF_X_GLOBAL: bf16) between the tokens' input vectors
+    int out_tok_stride;      // ... and between their output vectors (floats; PHF_OUT_SPLIT: bf16)
+    int pad_[2];
     __host__ __device__ int layer() const { return layer_flags >> 8; }
     __host__ __device__ int flags() const { return layer_flags & 0xff; }
 };
@@ -117,6 +120,9 @@ struct MkParams {
     float *x, *q, *attn;
     float *part_m, *part_l, *part_o;
     int max_chunks;                // row stride of the attention partial buffers (>= any chunk count)
+    int block_tokens;              // tokens a call may carry (1, or the M of the block build); buffers below hold that many vectors:
+                                   // x [M][H], q / attn [M][nq d], part_m / part_l [M][nq][max_chunks], part_o [M][nq][max_chunks][d],
+                                   // lm_part_val / lm_part_idx [M][gridDim.x]
     int att_chunk_shared;          // smallest chunk (positions) when one CTA serves a whole GQA group
     int att_chunk_split;           // smallest chunk when every query head has its own CTAs
     int att_split_max_n;           // contexts up to this length use one-head-per-CTA attention
