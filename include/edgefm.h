@@ -99,13 +99,20 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
  *     compressed from the fp32 k (after RoPE) and v.  Rows given to edgefm_prefill_kv / edgefm_append_kv (bf16) are
  *     compressed as they are copied in.  The cache takes head_dim + 4 bytes per row instead of 2 head_dim.
  *     edgefm_export_kv is refused on such a context (use edgefm_export_kv_int8), and so is edgefm_decode_step_static.
+ *   options->block_tokens = 0 or 1 : plain decode steps only;
+ *                           2      : the context can also verify a block of two tokens per call (edgefm_verify_block).
+ *     It then runs a build of the step kernel that carries two tokens side by side (work buffers for two tokens,
+ *     somewhat smaller weight tiles); edgefm_decode_step works as before on such a context.  Needs the plain bf16
+ *     cache and max_context <= 8192.
  *   options->reserved must be zero.
- * Errors: as edgefm_create; INVALID_ARG for an unknown format or non-zero reserved fields.
+ * Errors: as edgefm_create; INVALID_ARG for an unknown format, an unsupported block size or non-zero reserved fields;
+ * BAD_SHAPE when block_tokens = 2 is combined with the compressed cache or a context beyond 8192 positions.
  */
 enum { EDGEFM_KV_BF16 = 0, EDGEFM_KV_INT8 = 1 };
 typedef struct {
     int32_t kv_format;
-    int32_t reserved[7];
+    int32_t block_tokens;
+    int32_t reserved[6];
 } edgefm_options;
 edgefm_status edgefm_create_with_options(const edgefm_shape *shape, const edgefm_weights *weights, int32_t max_context,
                                          const edgefm_options *options, edgefm_ctx **out);
@@ -140,6 +147,31 @@ edgefm_status edgefm_prefill_kv(edgefm_ctx *ctx, const void *k, const void *v, i
  */
 edgefm_status edgefm_decode_step(edgefm_ctx *ctx, int32_t token_id, int32_t position, void *stream,
                                  float *logits_out, int32_t *next_token_out);
+
+/*
+ * edgefm_verify_block -- verification of a proposed block (Sec. 3.11 of the paper, "Verification" and "Commit"; the draft
+ * model that proposes the block is not part of this library).  tokens[0] is the token to decode (or -1: the token the
+ * previous call left on the device), tokens[1 .. m-1] the proposed continuation.  All m tokens pass through the model in
+ * ONE step at rotary positions position, position + 1, ... (position = -1: continue from the previous call) and cache slots
+ * cur_len, cur_len + 1, ...: the weights are streamed once, token t attends to the cache and to tokens 0 .. t of the block.
+ * With g_t the greedy token after token t, proposal t + 1 is accepted if tokens[t + 1] == g_t, and acceptance stops at the
+ * first mismatch.  n_accepted = 1 + accepted proposals (>= 1: tokens[0] itself always enters the cache); the cache length
+ * grows by n_accepted (the rows of rejected tokens stay behind it and are overwritten later); the next token is
+ * g_{n_accepted - 1}.  The result is what n_accepted plain decode steps would have produced.
+ *   tokens          : HOST int32 [m], read during the call.  m = 1 .. block_tokens of the context (m = 1 is a decode step).
+ *   logits_out      : DEVICE fp32 [m][vocab] (row t: the logits after token t; rows >= n_accepted belong to rejected
+ *                     tokens) or NULL.
+ *   n_accepted_out, next_token_out : DEVICE int32 [1] or NULL.
+ * The host-side cache length (edgefm_get_length) cannot know n_accepted: after this call it is the upper bound
+ * cur_len + m until edgefm_sync_length has been called.
+ * Errors: INVALID_ARG (context created without block_tokens, m out of range, token out of range, tokens[0] == -1 before
+ * any step), CONTEXT_FULL (fewer than m free slots; nothing is launched), CUDA.
+ */
+edgefm_status edgefm_verify_block(edgefm_ctx *ctx, const int32_t *tokens, int32_t m, int32_t position, void *stream,
+                                  float *logits_out, int32_t *n_accepted_out, int32_t *next_token_out);
+
+/* Wait for `stream`, then read the cache length from the device (exact again after edgefm_verify_block calls). */
+edgefm_status edgefm_sync_length(edgefm_ctx *ctx, void *stream, int32_t *cur_len_host);
 
 /* edgefm_destroy -- synchronise the device, then free everything the context owns (Sec. 3.7 step 4). NULL is a no-op. */
 edgefm_status edgefm_destroy(edgefm_ctx *ctx);

@@ -62,6 +62,8 @@ def lib():
         L.oracle_model_cur_len.argtypes = [_p]
         L.oracle_model_export_kv.restype = None
         L.oracle_model_export_kv.argtypes = [_p, _p, _p]
+        L.oracle_model_truncate.restype = ctypes.c_int
+        L.oracle_model_truncate.argtypes = [_p, _i64]
         L.oracle_model_use_int8_kv.restype = ctypes.c_int
         L.oracle_model_use_int8_kv.argtypes = [_p]
         L.oracle_quantize_row.restype = None
@@ -219,6 +221,26 @@ class OracleModel:
         v = np.empty(shape, np.uint16)
         lib().oracle_model_export_kv(self._h, k.ctypes.data, v.ctypes.data)
         return k, v
+
+    def truncate(self, n: int) -> None:
+        if lib().oracle_model_truncate(self._h, n):
+            raise ValueError("truncate beyond the cache length")
+
+    def verify_block(self, tokens, pos: int):
+        """Block verification as Sec. 3.11 states it, token by token: step every token of the block in turn (token t at
+        position pos + t); proposal t + 1 is accepted if it equals the greedy token after token t, verification stops at the
+        first rejection; the cache keeps the rows of the accepted tokens only.
+        -> (logits fp32 [m][V] of all m tokens, n_accepted, next_token)."""
+        start = self.cur_len
+        logits, greedy = [], []
+        for t, tok in enumerate(tokens):
+            lg, nx = self.step(int(tok), pos + t)
+            logits.append(lg); greedy.append(nx)
+        n_acc = 1
+        while n_acc < len(tokens) and int(tokens[n_acc]) == greedy[n_acc - 1]:
+            n_acc += 1
+        self.truncate(start + n_acc)
+        return np.stack(logits), n_acc, greedy[n_acc - 1]
 
     def export_kv_q8(self):
         """-> (K codes int8, V codes int8 [L][n_kv][max_context][d], K scales fp32, V scales fp32 [L][n_kv][max_context])."""

@@ -298,6 +298,15 @@ int oracle_model_load_kv(void *h, const uint16_t *k, const uint16_t *v, int64_t 
 
 int64_t oracle_model_cur_len(void *h) { return static_cast<Model *>(h)->cur_len; }
 
+// Drop the cache rows from slot n on (n <= cache length): the "Commit" of block verification (Sec. 3.11) keeps only the
+// rows of the accepted tokens.
+int oracle_model_truncate(void *h, int64_t n) {
+    Model *m = static_cast<Model *>(h);
+    if (n < 0 || n > m->cur_len) return 1;
+    m->cur_len = n;
+    return 0;
+}
+
 // Copy the whole cache out in its internal layout [L][n_kv][max_context][d].
 void oracle_model_export_kv(void *h, uint16_t *k_out, uint16_t *v_out) {
     Model *m = static_cast<Model *>(h);

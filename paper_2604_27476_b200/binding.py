@@ -37,7 +37,7 @@ class _Shape(ctypes.Structure):
 
 
 class _Options(ctypes.Structure):
-    _fields_ = [("kv_format", ctypes.c_int32), ("reserved", ctypes.c_int32 * 7)]
+    _fields_ = [("kv_format", ctypes.c_int32), ("block_tokens", ctypes.c_int32), ("reserved", ctypes.c_int32 * 6)]
 
 
 class _LayerWeights(ctypes.Structure):
@@ -52,7 +52,7 @@ class _Weights(ctypes.Structure):
 EXPORTS = ("edgefm_create", "edgefm_prefill_kv", "edgefm_decode_step", "edgefm_destroy", "edgefm_get_length",
            "edgefm_export_kv", "edgefm_get_launches_per_step", "edgefm_last_error", "edgefm_version",
            "edgefm_sync_status", "edgefm_debug_profile", "edgefm_debug_set_wait_limit", "edgefm_debug_plan", "edgefm_debug_plan_operator", "edgefm_decode_step_static", "edgefm_set_vocab_subset",
-           "edgefm_append_kv", "edgefm_create_with_options", "edgefm_export_kv_int8")
+           "edgefm_append_kv", "edgefm_create_with_options", "edgefm_export_kv_int8", "edgefm_verify_block", "edgefm_sync_length")
 
 
 def library_path() -> Path:
@@ -73,6 +73,10 @@ def load_library():
     L.edgefm_create.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Weights), i32, ctypes.POINTER(vp)]
     L.edgefm_create_with_options.restype = ctypes.c_int
     L.edgefm_create_with_options.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Weights), i32, ctypes.POINTER(_Options), ctypes.POINTER(vp)]
+    L.edgefm_verify_block.restype = ctypes.c_int
+    L.edgefm_verify_block.argtypes = [vp, ctypes.POINTER(i32), i32, i32, vp, vp, vp, vp]
+    L.edgefm_sync_length.restype = ctypes.c_int
+    L.edgefm_sync_length.argtypes = [vp, vp, ctypes.POINTER(i32)]
     L.edgefm_export_kv_int8.restype = ctypes.c_int
     L.edgefm_export_kv_int8.argtypes = [vp, vp, vp, vp, vp, vp]
     L.edgefm_prefill_kv.restype = ctypes.c_int
@@ -128,7 +132,7 @@ def edgefm_last_error(ctx=None) -> str:
 KV_FORMATS = {"bf16": 0, "int8": 1}
 
 
-def edgefm_create(shape: dict, weights: dict, max_context: int, kv_format: str | int | None = None, reserved=None):
+def edgefm_create(shape: dict, weights: dict, max_context: int, kv_format: str | int | None = None, reserved=None, block_tokens: int = 0):
     """shape: dict with the fields of edgefm_shape; weights: {"embed", "final_norm", "lm_head": device
     pointers (int), "layers": [ {field: device pointer or None} ]}.  Returns the opaque context handle.
     kv_format: None = edgefm_create; "bf16" / "int8" (or the raw integer) = edgefm_create_with_options."""
@@ -141,10 +145,11 @@ def edgefm_create(shape: dict, weights: dict, max_context: int, kv_format: str |
             setattr(arr[i], name, lw.get(name))
     w = _Weights(weights["embed"], weights["final_norm"], weights["lm_head"], arr)
     out = ctypes.c_void_p()
-    if kv_format is None:
+    if kv_format is None and not block_tokens and not reserved:
         _check(L.edgefm_create(ctypes.byref(sh), ctypes.byref(w), max_context, ctypes.byref(out)))
     else:
-        opt = _Options(KV_FORMATS.get(kv_format, kv_format) if isinstance(kv_format, str) else int(kv_format), (ctypes.c_int32 * 7)(*(reserved or [0] * 7)))
+        fmt = 0 if kv_format is None else (KV_FORMATS.get(kv_format, kv_format) if isinstance(kv_format, str) else int(kv_format))
+        opt = _Options(fmt, int(block_tokens), (ctypes.c_int32 * 6)(*(list(reserved or [])[:6] + [0] * 6)[:6]))
         _check(L.edgefm_create_with_options(ctypes.byref(sh), ctypes.byref(w), max_context, ctypes.byref(opt), ctypes.byref(out)))
     return out
 
@@ -276,6 +281,17 @@ def edgefm_export_kv(ctx, k_out_ptr, v_out_ptr, stream=None):
     _check(load_library().edgefm_export_kv(ctx, k_out_ptr, v_out_ptr, stream), ctx)
 
 
+def edgefm_verify_block(ctx, tokens, position, stream=None, logits_out=None, n_accepted_out=None, next_token_out=None):
+    arr = (ctypes.c_int32 * max(1, len(tokens)))(*[int(t) for t in tokens])
+    _check(load_library().edgefm_verify_block(ctx, arr, len(tokens), position, stream, logits_out, n_accepted_out, next_token_out), ctx)
+
+
+def edgefm_sync_length(ctx, stream=None) -> int:
+    n = ctypes.c_int32()
+    _check(load_library().edgefm_sync_length(ctx, stream, ctypes.byref(n)), ctx)
+    return n.value
+
+
 def edgefm_export_kv_int8(ctx, k_codes_ptr, v_codes_ptr, k_scales_ptr, v_scales_ptr, stream=None):
     _check(load_library().edgefm_export_kv_int8(ctx, k_codes_ptr, v_codes_ptr, k_scales_ptr, v_scales_ptr, stream), ctx)
 
@@ -306,7 +322,7 @@ def upload_weights(host_weights: dict, device="cuda:0"):
 class DecodeContext:
     """RAII wrapper of one edgefm context with torch-allocated I/O buffers."""
 
-    def __init__(self, cfg, device_weight_ptrs: dict, max_context: int, device="cuda:0", kv_format: str | None = None):
+    def __init__(self, cfg, device_weight_ptrs: dict, max_context: int, device="cuda:0", kv_format: str | None = None, block_tokens: int = 0):
         import torch
 
         self.cfg = cfg
@@ -317,9 +333,12 @@ class DecodeContext:
                      head_dim=cfg.head_dim, ffn=cfg.ffn, vocab=cfg.vocab, rms_eps=cfg.rms_eps,
                      rope_theta=cfg.rope_theta, qkv_bias=int(cfg.qkv_bias))
         with torch.cuda.device(self.device):
-            self.handle = edgefm_create(shape, device_weight_ptrs, max_context, kv_format)
-        self.logits = torch.empty(cfg.vocab, dtype=torch.float32, device=self.device)
+            self.handle = edgefm_create(shape, device_weight_ptrs, max_context, kv_format, block_tokens=block_tokens)
+        self.block_tokens = max(1, block_tokens)
+        self.block_logits = torch.empty((self.block_tokens, cfg.vocab), dtype=torch.float32, device=self.device)
+        self.logits = self.block_logits[0]
         self.next_token = torch.zeros(1, dtype=torch.int32, device=self.device)
+        self.n_accepted = torch.zeros(1, dtype=torch.int32, device=self.device)
 
     def _stream(self):
         import torch
@@ -347,6 +366,14 @@ class DecodeContext:
         edgefm_decode_step(self.handle, token_id, position, self._stream(),
                            self.logits.data_ptr() if want_logits else None,
                            self.next_token.data_ptr() if want_token else None)
+
+    def verify_block(self, tokens, position=-1, want_logits=True):
+        """One call for a block of tokens (tokens[0] may be -1); results in block_logits[:m], n_accepted, next_token."""
+        edgefm_verify_block(self.handle, tokens, position, self._stream(), self.block_logits.data_ptr() if want_logits else None,
+                            self.n_accepted.data_ptr(), self.next_token.data_ptr())
+
+    def sync_length(self) -> int:
+        return edgefm_sync_length(self.handle, self._stream())
 
     def set_vocab_subset(self, token_ids):
         """Restrict the output layer to these token ids (ascending); None restores the full vocabulary.  With a subset

@@ -119,8 +119,11 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const uint16_t *src, c
 
 // long_ctx = false: the variant without the grouped (one CTA per GQA group) attention code, for contexts that
 // never need it.
+MegaKernel mega_kernel_block2(int head_dim);   // megakernel_block2.cu
+
 template <int D>
-MegaKernel mega_kernel_g(int G, bool long_ctx, bool kv8 = false) {
+MegaKernel mega_kernel_g(int G, bool long_ctx, bool kv8 = false, int block_tokens = 1) {
+    if (block_tokens == 2) return mega_kernel_block2(D);
     if (kv8) {
         if (D == 64) return G <= 4 ? mega_kernel_q8_d64_lo(G) : mega_kernel_q8_d64_hi(G);
         return G <= 4 ? mega_kernel_q8_d128_lo(G) : mega_kernel_q8_d128_hi(G);
@@ -141,17 +144,20 @@ struct StepPlan {
     size_t xbuf = 0, ops_bytes = 0, tab_bytes = 0, sched_bytes = 0;   // shared memory: activation / attention scratch, operators, schedule table, tile lists
     int slots = 0, slot_bytes = 0, slot_rows = 0;   // ring of one consumer warp
     size_t dyn_smem = 0;
+    int block_tokens = 1;  // tokens a call may carry (the M of the chosen kernel build)
 };
 
 // Kernel variant and shared-memory split for a model shape.  Returns null, or why the shape does not fit.
 // sched_reserve: bytes to set aside for the CTA's tile lists.
 inline const char *plan_step(const edgefm_shape &sh, int max_context, int num_sms, int smem_optin, size_t sched_reserve, StepPlan *pl, cudaError_t *cuda_err,
-                             bool kv8 = false) {
+                             bool kv8 = false, int block_tokens = 1) {
     const int H = sh.hidden, d = sh.head_dim, nq = sh.n_q_heads, nkv = sh.n_kv_heads, G = nq / nkv;
     *cuda_err = cudaSuccess;
     // (the compressed cache is attended by the grouped attention of the long-context build only)
     pl->long_ctx = kv8 || max_context > 8192 || static_cast<long long>(nq) * MK_ATT_SPLIT_MAXC * 2 > MK_PARTIAL_FLOATS;
-    pl->kernel = d == 64 ? mega_kernel_g<64>(G, pl->long_ctx, kv8) : mega_kernel_g<128>(G, pl->long_ctx, kv8);
+    if (block_tokens > 1 && pl->long_ctx) return "blocks of several tokens need the plain cache and max_context <= 8192";
+    pl->block_tokens = block_tokens;
+    pl->kernel = d == 64 ? mega_kernel_g<64>(G, pl->long_ctx, kv8, block_tokens) : mega_kernel_g<128>(G, pl->long_ctx, kv8, block_tokens);
     pl->nw = pl->long_ctx ? MK_NW_LONG : MK_NW_SHORT;
     pl->grid = num_sms;
     pl->max_chunks = pl->grid / nkv > 0 ? pl->grid / nkv : 1;
@@ -165,7 +171,7 @@ inline const char *plan_step(const edgefm_shape &sh, int max_context, int num_sm
     const int AG = pl->long_ctx ? G : 1;
     const size_t att_bytes = (static_cast<size_t>(AG) * d + NW * (AG * MK_ATT_TILE > 32 / MK_ATT_LPP_SPLIT ? AG * MK_ATT_TILE : 32 / MK_ATT_LPP_SPLIT) +
                               2 * ATT_MW * AG + static_cast<size_t>(ATT_MW) * AG * d + 2 * static_cast<size_t>(AG) * pl->max_chunks) * 4;
-    size_t xbuf = MK_X_SPLITS * (static_cast<size_t>(max_k) * 2 + MK_XS_PAD);   // the staged activation: three bf16 arrays
+    size_t xbuf = block_tokens * MK_X_SPLITS * (static_cast<size_t>(max_k) * 2 + MK_XS_PAD);   // the staged activations: three bf16 arrays per token
     if (att_bytes > xbuf) xbuf = att_bytes;
     pl->xbuf = (xbuf + 1023) / 1024 * 1024;
     cudaFuncAttributes fa{};
@@ -178,7 +184,7 @@ inline const char *plan_step(const edgefm_shape &sh, int max_context, int num_sm
     pl->tab_bytes = (tab + 15) / 16 * 16;
     const size_t head = (pl->ops_bytes + pl->tab_bytes + sched_reserve + 1023) / 1024 * 1024;   // the rings start on a 1 KB boundary
     pl->sched_bytes = head - pl->ops_bytes - pl->tab_bytes;
-    const size_t tail = pl->xbuf + static_cast<size_t>(NW) * MK_WBUF_BYTES;   // behind the rings: the activation vector and the warps' small buffers
+    const size_t tail = pl->xbuf + static_cast<size_t>(NW) * MK_WBUF_BYTES * block_tokens;   // behind the rings: the activation vector and the warps' small buffers
     if (head + tail + static_smem + static_cast<size_t>(NW) * 2 * 2048 > static_cast<size_t>(smem_optin))
         return "model shape does not fit the shared-memory plan";
     const size_t per_warp = (smem_optin - static_smem - head - tail) / NW;
@@ -217,11 +223,15 @@ inline void op_shapes(const edgefm_shape &sh, int lm_rows, OpShape os[5]) {
 // The operators of the step in execution order, wired to the work buffers.
 inline void fill_ops(const edgefm_shape &sh, const edgefm_layer_weights *layers, const void *final_norm, const void *lm_head, float *x, float *attn, float *q,
                      float *act, MkOp *out, const uint16_t **weights_out) {
+    // distance between the vectors of consecutive tokens of a block (see MkParams::block_tokens)
+    const int sx = sh.hidden, sq = sh.n_q_heads * sh.head_dim, sa = MK_X_SPLITS * ((sh.ffn + MK_TILE_COLS - 1) / MK_TILE_COLS * MK_TILE_COLS);
     OpShape os[5];
     op_shapes(sh, sh.vocab, os);
     int n = 0;
-    auto mk = [&](const OpShape &o, const void *W, const void *bias, const void *norm, const float *x_src, float *dst, int layer, int flags) {
+    auto mk = [&](const OpShape &o, const void *W, const void *bias, const void *norm, const float *x_src, float *dst, int layer, int flags, int xs_ = 0,
+                  int os_ = 0) {
         MkOp op{};
+        op.x_tok_stride = xs_; op.out_tok_stride = os_;
         weights_out[n] = static_cast<const uint16_t *>(W);
         op.bias = static_cast<const uint16_t *>(bias); op.norm_w = static_cast<const uint16_t *>(norm); op.x_src = x_src; op.out = dst;
         op.K = o.K; op.kind = o.kind; op.units_total = o.units; op.layer_flags = layer << 8 | flags | (o.K % 64 ? PHF_RAGGED : 0);
@@ -229,12 +239,12 @@ inline void fill_ops(const edgefm_shape &sh, const edgefm_layer_weights *layers,
     };
     for (int l = 0; l < sh.n_layers; ++l) {
         const edgefm_layer_weights &w = layers[l];
-        mk(os[0], w.wqkv, sh.qkv_bias ? w.bqkv : nullptr, w.input_norm, l == 0 ? nullptr : x, q, l, 0);
-        mk(os[1], w.wo, nullptr, nullptr, attn, x, l, 0);
-        mk(os[2], w.w_gate_up, nullptr, w.post_norm, x, act, l, PHF_OUT_SPLIT);  // the MLP activations go to memory in the form the down projection multiplies
-        mk(os[3], w.w_down, nullptr, nullptr, act, x, l, PHF_X_GLOBAL);
+        mk(os[0], w.wqkv, sh.qkv_bias ? w.bqkv : nullptr, w.input_norm, l == 0 ? nullptr : x, q, l, 0, sx, sq);
+        mk(os[1], w.wo, nullptr, nullptr, attn, x, l, 0, sq, sx);
+        mk(os[2], w.w_gate_up, nullptr, w.post_norm, x, act, l, PHF_OUT_SPLIT, sx, sa);  // the MLP activations go to memory in the form the down projection multiplies
+        mk(os[3], w.w_down, nullptr, nullptr, act, x, l, PHF_X_GLOBAL, sa, sx);
     }
-    mk(os[4], lm_head, nullptr, final_norm, x, nullptr, sh.n_layers, 0);
+    mk(os[4], lm_head, nullptr, final_norm, x, nullptr, sh.n_layers, 0, sx, 0);
 }
 
 // Tile schedule of the step for the plan's geometry.  Returns null, or why the shape does not fit.
@@ -250,10 +260,10 @@ inline const char *plan_schedule(const StepPlan &pl, const edgefm_shape &sh, int
 // Shared-memory plan and tile schedule together: the tile lists live in shared memory, so their size (known only once
 // the schedule exists) takes room from the rings, whose slot size shapes the schedule.  A few rounds settle it.
 inline const char *plan_step_and_schedule(const edgefm_shape &sh, int max_context, int num_sms, int smem_optin, StepPlan *pl, StepSchedule *ss,
-                                          cudaError_t *cuda_err, bool kv8 = false) {
+                                          cudaError_t *cuda_err, bool kv8 = false, int block_tokens = 1) {
     size_t reserve = 0;
     for (int attempt = 0; attempt < 6; ++attempt) {
-        if (const char *why = plan_step(sh, max_context, num_sms, smem_optin, reserve, pl, cuda_err, kv8)) return why;
+        if (const char *why = plan_step(sh, max_context, num_sms, smem_optin, reserve, pl, cuda_err, kv8, block_tokens)) return why;
         if (const char *why = plan_schedule(*pl, sh, sh.vocab, ss)) return why;
         const size_t need = ss->smem_bytes();
         if (need <= pl->sched_bytes) return nullptr;
@@ -291,7 +301,7 @@ inline void fill_shape_params(MkParams *m, const edgefm_shape &sh, int max_conte
     m->d = sh.head_dim; m->F = sh.ffn; m->V = sh.vocab;
     m->half_shift = sh.head_dim == 64 ? 5 : 6;
     m->eps = sh.rms_eps; m->scale = static_cast<float>(1.0 / std::sqrt(static_cast<double>(sh.head_dim)));
-    m->max_context = max_context; m->max_chunks = pl.max_chunks;
+    m->max_context = max_context; m->max_chunks = pl.max_chunks; m->block_tokens = pl.block_tokens;
     m->att_chunk_shared = 256; m->att_chunk_split = 64; m->att_split_max_n = 8192;
     m->slots = pl.slots; m->slot_bytes = pl.slot_bytes;
     m->xbuf_bytes = static_cast<int>(pl.xbuf); m->ops_bytes = static_cast<int>(pl.ops_bytes); m->tab_bytes = static_cast<int>(pl.tab_bytes);
@@ -320,6 +330,7 @@ struct edgefm_ctx {
     // owned device memory
     uint16_t *k_cache = nullptr, *v_cache = nullptr;  // [L][nkv][max_context][d] (bf16, or one signed byte per element)
     int kv_format = EDGEFM_KV_BF16;
+    int block_tokens = 1;        // tokens a call may carry (edgefm_verify_block)
     float *k_scale = nullptr, *v_scale = nullptr;     // compressed cache: [L][nkv][max_context]
     float *kv_stage = nullptr;                        // compressed cache: fp32 k, v rows of the step's token [2][nkv][d]
     float *x = nullptr;          // residual stream [H]
@@ -469,6 +480,10 @@ edgefm_status edgefm_create_with_options(const edgefm_shape *shape, const edgefm
             if (r != 0) return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "reserved option fields must be zero");
     }
     const bool kv8 = options && options->kv_format == EDGEFM_KV_INT8;
+    if (options && (options->block_tokens < 0 || options->block_tokens > 2))
+        return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "block_tokens %d is not supported (0, 1 or 2)", options->block_tokens);
+    const int M = options && options->block_tokens == 2 ? 2 : 1;
+    if (M > 1 && kv8) return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "blocks of several tokens need the plain bf16 cache");
     if (!shape || !weights || !out) return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "null argument");
     if (max_context < 1) return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "max_context must be >= 1");
     const edgefm_shape &sh = *shape;
@@ -510,6 +525,7 @@ edgefm_status edgefm_create_with_options(const edgefm_shape *shape, const edgefm
     if (!c) return fail(nullptr, EDGEFM_ERR_OUT_OF_MEMORY, "host allocation failed");
     c->shape = sh;
     c->kv_format = kv8 ? EDGEFM_KV_INT8 : EDGEFM_KV_BF16;
+    c->block_tokens = M;
     c->max_context = max_context;
     c->device = dev;
     c->num_sms = prop.multiProcessorCount;
@@ -538,7 +554,7 @@ edgefm_status edgefm_create_with_options(const edgefm_shape *shape, const edgefm
     if (!coop) return bail(EDGEFM_ERR_CUDA, "device lacks cooperative launch", cudaErrorNotSupported);
     {
         cudaError_t ce = cudaSuccess;
-        if (const char *why = plan_step_and_schedule(sh, max_context, c->num_sms, smem_optin, &pl, &c->sched_full, &ce, kv8))
+        if (const char *why = plan_step_and_schedule(sh, max_context, c->num_sms, smem_optin, &pl, &c->sched_full, &ce, kv8, M))
             return bail(ce != cudaSuccess ? EDGEFM_ERR_CUDA : EDGEFM_ERR_BAD_SHAPE, why, ce != cudaSuccess ? ce : cudaErrorInvalidValue);
     }
     const StepSchedule &ss = c->sched_full;
@@ -556,17 +572,18 @@ edgefm_status edgefm_create_with_options(const edgefm_shape *shape, const edgefm
         CREATE_TRY(cudaMemset(c->v_scale, 0, kv_rows * sizeof(float)));
         CREATE_TRY(cudaMemset(c->kv_stage, 0, static_cast<size_t>(2) * nkv * d * sizeof(float)));
     }
-    CREATE_TRY(dev_alloc(&c->x, H));
-    CREATE_TRY(dev_alloc(&c->q, nq * d));
-    CREATE_TRY(dev_alloc(&c->attn, nq * d));
-    CREATE_TRY(dev_alloc(&c->act, static_cast<size_t>(MK_X_SPLITS) * ((F + MK_TILE_COLS - 1) / MK_TILE_COLS * MK_TILE_COLS) / 2));   // three bf16 arrays of F rounded
+    // (work buffers hold one vector per token of a block)
+    CREATE_TRY(dev_alloc(&c->x, static_cast<size_t>(M) * H));
+    CREATE_TRY(dev_alloc(&c->q, static_cast<size_t>(M) * nq * d));
+    CREATE_TRY(dev_alloc(&c->attn, static_cast<size_t>(M) * nq * d));
+    CREATE_TRY(dev_alloc(&c->act, static_cast<size_t>(M) * MK_X_SPLITS * ((F + MK_TILE_COLS - 1) / MK_TILE_COLS * MK_TILE_COLS) / 2));   // three bf16 arrays of F rounded
                                                                                          // up to whole column pieces (the pieces of every value)
     CREATE_TRY(dev_alloc(&c->inv_freq, d / 2));
-    CREATE_TRY(dev_alloc(&c->part_m, static_cast<size_t>(nq) * pl.max_chunks));
-    CREATE_TRY(dev_alloc(&c->part_l, static_cast<size_t>(nq) * pl.max_chunks));
-    CREATE_TRY(dev_alloc(&c->part_o, static_cast<size_t>(nq) * pl.max_chunks * d));
-    CREATE_TRY(dev_alloc(&c->lm_part_val, pl.grid));
-    CREATE_TRY(dev_alloc(&c->lm_part_idx, pl.grid));
+    CREATE_TRY(dev_alloc(&c->part_m, static_cast<size_t>(M) * nq * pl.max_chunks));
+    CREATE_TRY(dev_alloc(&c->part_l, static_cast<size_t>(M) * nq * pl.max_chunks));
+    CREATE_TRY(dev_alloc(&c->part_o, static_cast<size_t>(M) * nq * pl.max_chunks * d));
+    CREATE_TRY(dev_alloc(&c->lm_part_val, static_cast<size_t>(M) * pl.grid));
+    CREATE_TRY(dev_alloc(&c->lm_part_idx, static_cast<size_t>(M) * pl.grid));
     CREATE_TRY(dev_alloc(&c->tickets, nq + nkv + 2 + nq + 2 * nkv));   // tickets, then the per-head counters of the QKV projection
     CREATE_TRY(dev_alloc(&c->state, 1));
     CREATE_TRY(dev_alloc(&c->req, 1));
@@ -722,6 +739,48 @@ edgefm_status edgefm_decode_step(edgefm_ctx *ctx, int32_t token_id, int32_t posi
     ctx->cur_len += 1;
     ctx->have_token = true;
     ctx->err.clear();
+    return EDGEFM_OK;
+}
+
+edgefm_status edgefm_verify_block(edgefm_ctx *ctx, const int32_t *tokens, int32_t m, int32_t position, void *stream, float *logits_out,
+                                  int32_t *n_accepted_out, int32_t *next_token_out) {
+    if (!ctx) return EDGEFM_ERR_INVALID_ARG;
+    if (!tokens) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "null tokens");
+    if (m < 1 || m > ctx->block_tokens)
+        return fail(ctx, EDGEFM_ERR_INVALID_ARG, "m = %d: this context verifies blocks of 1 .. %d tokens (edgefm_options::block_tokens)", m, ctx->block_tokens);
+    if (tokens[0] < -1 || tokens[0] >= ctx->shape.vocab) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "tokens[0] = %d out of range", tokens[0]);
+    for (int t = 1; t < m; ++t)
+        if (tokens[t] < 0 || tokens[t] >= ctx->shape.vocab) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "tokens[%d] = %d out of range", t, tokens[t]);
+    if (position < -1) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "position %d out of range", position);
+    if (tokens[0] == -1 && !ctx->have_token) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "tokens[0] = -1 needs a previous step on this context");
+    if (ctx->cur_len + m > ctx->max_context)
+        return fail(ctx, EDGEFM_ERR_CONTEXT_FULL, "%d tokens do not fit behind %d of %d cache slots", m, ctx->cur_len, ctx->max_context);
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    StepRequest r{tokens[0], position, logits_out, next_token_out};
+    r.m = m;
+    for (int t = 1; t < m && t <= 3; ++t) r.draft[t - 1] = tokens[t];
+    r.n_accepted_out = n_accepted_out;
+    if (!ctx->req_valid || std::memcmp(&r, &ctx->last_req, sizeof r) != 0) {
+        CUDA_TRY(ctx, cudaMemcpyAsync(ctx->req, &r, sizeof r, cudaMemcpyHostToDevice, s));
+        ctx->last_req = r;
+        ctx->req_valid = true;
+    }
+    CUDA_TRY(ctx, cudaGraphLaunch(ctx->exec, s));
+    ctx->cur_len += m;     // an upper bound until edgefm_sync_length: the device decides how many tokens are accepted
+    ctx->have_token = true;
+    ctx->err.clear();
+    return EDGEFM_OK;
+}
+
+edgefm_status edgefm_sync_length(edgefm_ctx *ctx, void *stream, int32_t *cur_len_host) {
+    if (!ctx || !cur_len_host) return EDGEFM_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->device);
+    CUDA_TRY(ctx, cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    StepState st{};
+    CUDA_TRY(ctx, cudaMemcpy(&st, ctx->state, sizeof st, cudaMemcpyDeviceToHost));
+    ctx->cur_len = st.cur_len;
+    *cur_len_host = st.cur_len;
     return EDGEFM_OK;
 }
 

@@ -55,7 +55,7 @@ def assert_appended_rows_close(gpu_bits: np.ndarray, ref_bits: np.ndarray):
 class Pair:
     """The oracle model and the CUDA context fed from the same host weights and KV prefix."""
 
-    def __init__(self, cfg, seed=GLOBAL_SEED, cache_len=None, max_context=None, weights=None, kv_format=None):
+    def __init__(self, cfg, seed=GLOBAL_SEED, cache_len=None, max_context=None, weights=None, kv_format=None, block_tokens=0):
         import torch
         from oracle import OracleModel
         from paper_2604_27476_b200 import DecodeContext, upload_weights
@@ -69,7 +69,7 @@ class Pair:
         if self.T0:
             self.oracle.load_kv(self.k, self.v)
         self.ptrs, self.keep = upload_weights(self.weights)
-        self.ctx = DecodeContext(cfg, self.ptrs, self.max_context, kv_format=kv_format)
+        self.ctx = DecodeContext(cfg, self.ptrs, self.max_context, kv_format=kv_format, block_tokens=block_tokens)
         self.kd = torch.from_numpy(self.k.view(np.int16)).cuda()
         self.vd = torch.from_numpy(self.v.view(np.int16)).cuda()
         if self.T0:

@@ -1,0 +1,120 @@
+"""Block verification (Sec. 3.11 of the paper): two tokens pass through the step kernel in one call, the weights streamed
+once.  The oracle verifies the block as the paper states it, token by token with plain decode steps; the draft model is not
+part of either side, proposals are made here (the oracle's own greedy token = a proposal that must be accepted, anything
+else = one that must be rejected)."""
+import numpy as np
+import pytest
+
+from edgefm_synth import CONFIGS, first_token
+from helpers import Pair, assert_logits_close, top2_margin, TOKEN_MARGIN
+
+pytestmark = pytest.mark.gpu
+
+SHAPES = {
+    "tiny_d64": (CONFIGS["tiny"], 100),
+    "d128_bias": (CONFIGS["tiny"].with_(hidden=512, n_q_heads=8, n_kv_heads=2, head_dim=128, ffn=1536, vocab=3000, n_layers=3, qkv_bias=True), 70),
+    "ragged_g7": (CONFIGS["tiny"].with_(n_q_heads=7, n_kv_heads=1, hidden=136, ffn=72, vocab=333, n_layers=3, qkv_bias=True), 0),
+}
+
+
+def _peek_greedy(pair, tok, pos):
+    """The oracle's greedy token after `tok`, without changing its cache."""
+    n = pair.oracle.cur_len
+    _, nxt = pair.oracle.step(tok, pos)
+    pair.oracle.truncate(n)
+    return nxt
+
+
+@pytest.mark.parametrize("name", sorted(SHAPES))
+def test_blocks_of_two_match_the_oracle_verification(name):
+    import torch
+    cfg, T0 = SHAPES[name]
+    rounds = 8
+    pair = Pair(cfg, cache_len=T0, max_context=T0 + 2 * rounds + 2, block_tokens=2)
+    try:
+        tok, pos = first_token(cfg), T0 + 5
+        for r in range(rounds):
+            good = _peek_greedy(pair, tok, pos)
+            proposal = good if r % 3 != 1 else (good + 1 + r) % cfg.vocab          # every third round: a wrong proposal
+            ref_logits, ref_acc, ref_next = pair.oracle.verify_block([tok, proposal], pos)
+            pair.ctx.verify_block([tok if r % 2 == 0 else -1, proposal], pos if r % 2 == 0 else -1)   # odd rounds: chained on the device
+            torch.cuda.synchronize()
+            got = pair.ctx.block_logits.cpu().numpy()
+            assert_logits_close(got[0], ref_logits[0], f"{name} round {r} token 0")
+            assert_logits_close(got[1], ref_logits[1], f"{name} round {r} token 1")
+            assert int(pair.ctx.n_accepted.item()) == ref_acc == (2 if proposal == good else 1)
+            margins_ok = all(top2_margin(ref_logits[t]) > TOKEN_MARGIN for t in range(ref_acc))
+            if margins_ok:
+                assert int(pair.ctx.next_token.item()) == ref_next
+            assert pair.ctx.sync_length() == pair.oracle.cur_len
+            tok, pos = ref_next, pos + ref_acc
+            if not margins_ok:      # a near-tie: the two sides may legitimately continue with different tokens
+                break
+        # the cache: rows up to the common length agree with the oracle's (appended rows within one bf16 step)
+        from helpers import assert_appended_rows_close
+        n = pair.oracle.cur_len
+        kg, vg = [t.cpu().numpy().view(np.uint16) for t in pair.ctx.export_kv()]
+        ko, vo = pair.oracle.export_kv()
+        assert np.array_equal(kg[:, :, :T0], ko[:, :, :T0]) and np.array_equal(vg[:, :, :T0], vo[:, :, :T0])
+        if n > T0:
+            assert_appended_rows_close(kg[:, :, T0:n], ko[:, :, T0:n])
+            assert_appended_rows_close(vg[:, :, T0:n], vo[:, :, T0:n])
+    finally:
+        pair.close()
+
+
+def test_plain_steps_and_single_token_blocks_on_a_block_context():
+    """edgefm_decode_step and m = 1 blocks on a context built for blocks give the plain step's results."""
+    import torch
+    cfg = CONFIGS["tiny"]
+    pair = Pair(cfg, cache_len=64, max_context=80, block_tokens=2)
+    try:
+        tok, pos = first_token(cfg), 64
+        for s in range(4):
+            ref, nxt = pair.oracle.step(tok, pos)
+            if s % 2 == 0:
+                pair.ctx.step(tok, pos)
+            else:
+                pair.ctx.verify_block([tok], pos)
+            torch.cuda.synchronize()
+            assert_logits_close(pair.ctx.logits.cpu().numpy(), ref, f"step {s}")
+            if s % 2 == 1:
+                assert int(pair.ctx.n_accepted.item()) == 1
+            tok, pos = nxt, pos + 1
+        assert pair.ctx.sync_length() == pair.oracle.cur_len == 68
+    finally:
+        pair.close()
+
+
+def test_block_calls_are_validated():
+    from paper_2604_27476_b200 import EdgefmError, Status, edgefm_create
+    cfg = CONFIGS["tiny"]
+    plain = Pair(cfg, cache_len=0, max_context=4)
+    block = Pair(cfg, cache_len=3, max_context=4, block_tokens=2)
+    try:
+        with pytest.raises(EdgefmError) as ei:
+            plain.ctx.verify_block([1, 2], 0)                      # context not built for blocks
+        assert ei.value.status == Status.ERR_INVALID_ARG
+        with pytest.raises(EdgefmError) as ei:
+            block.ctx.verify_block([1, 2, 3], 3)                   # more tokens than the build carries
+        assert ei.value.status == Status.ERR_INVALID_ARG
+        with pytest.raises(EdgefmError) as ei:
+            block.ctx.verify_block([1, cfg.vocab], 3)
+        assert ei.value.status == Status.ERR_INVALID_ARG
+        with pytest.raises(EdgefmError) as ei:
+            block.ctx.verify_block([1, 2], 3)                      # one free slot, two tokens
+        assert ei.value.status == Status.ERR_CONTEXT_FULL
+        assert block.ctx.cur_len == 3
+        shape = dict(n_layers=cfg.n_layers, hidden=cfg.hidden, n_q_heads=cfg.n_q_heads, n_kv_heads=cfg.n_kv_heads, head_dim=cfg.head_dim,
+                     ffn=cfg.ffn, vocab=cfg.vocab, rms_eps=cfg.rms_eps, rope_theta=cfg.rope_theta, qkv_bias=0)
+        with pytest.raises(EdgefmError) as ei:
+            edgefm_create(shape, plain.ptrs, 16, kv_format="int8", block_tokens=2)
+        assert ei.value.status == Status.ERR_BAD_SHAPE
+        with pytest.raises(EdgefmError) as ei:
+            edgefm_create(shape, plain.ptrs, 9000, block_tokens=2)
+        assert ei.value.status == Status.ERR_BAD_SHAPE
+        with pytest.raises(EdgefmError) as ei:
+            edgefm_create(shape, plain.ptrs, 16, block_tokens=3)
+        assert ei.value.status == Status.ERR_INVALID_ARG
+    finally:
+        plain.close(); block.close()
