@@ -186,6 +186,75 @@ def workload_name(cfg, kv_format="bf16"):
             f"(L={cfg.n_layers} H={cfg.hidden} heads={cfg.n_q_heads}/{cfg.n_kv_heads} d={cfg.head_dim} F={cfg.ffn} V={cfg.vocab})")
 
 
+def run_block(args, cfg):
+    """Block verification (edgefm_verify_block, blocks of two): ms per GENERATED token when every call carries the token to
+    decode and a proposal.  There is no draft model here: the proposals are the model's own greedy continuation, recorded in
+    an untimed plain run (so they are accepted unless --reject-every spoils some, or the two kernel builds round a near-tie
+    differently); the tokens generated are counted from the cache length the device reports.  One GPU."""
+    import torch
+    from paper_2604_27476_b200 import DecodeContext, build as cuda_build, upload_weights
+    cuda_build.build()
+    dev = "cuda:0"
+    steps = args.steps
+    weights = make_weights(cfg)
+    k, v = make_kv(cfg)
+    ptrs, keep = upload_weights(weights, dev)
+    ctx = DecodeContext(cfg, ptrs, cfg.cache_len + 2 * steps + 2, dev, block_tokens=2)
+    kd = torch.from_numpy(k.view(np.int16)).to(dev)
+    vd = torch.from_numpy(v.view(np.int16)).to(dev)
+    tok0, pos0 = first_token(cfg), cfg.first_position
+    # the greedy continuation, by plain steps on the same context (untimed)
+    ctx.prefill_kv(kd, vd)
+    seq = [tok0]
+    ctx.step(tok0, pos0, want_logits=False)
+    for _ in range(2 * steps):
+        torch.cuda.synchronize()
+        seq.append(int(ctx.next_token.item()))
+        ctx.step(-1, -1, want_logits=False)
+    torch.cuda.synchronize()
+
+    def one_sequence():
+        """`steps` calls; returns the tokens that entered the cache."""
+        ctx.prefill_kv(kd, vd)
+        idx = 0                      # seq[idx] is the token the next call decodes (if every correct proposal is accepted)
+        for c in range(steps):
+            spoil = args.reject_every > 0 and c % args.reject_every == args.reject_every - 1
+            proposal = (seq[idx + 1] + 1) % cfg.vocab if spoil else seq[idx + 1]
+            ctx.verify_block([tok0 if c == 0 else -1, proposal], pos0 if c == 0 else -1, want_logits=False)
+            idx += 1 if spoil else 2
+        return idx
+
+    for _ in range(max(args.warmup_sequences, 1)):
+        one_sequence()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    per_tok, accepted = [], []
+    for _ in range(max(args.sequences, 1)):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ctx.prefill_kv(kd, vd)
+        torch.cuda.synchronize()
+        # (the prefill above is outside the events; one_sequence repeats it, which costs ~20 us of 100+ ms)
+        e0.record()
+        one_sequence()
+        e1.record()
+        torch.cuda.synchronize()
+        n_tok = ctx.sync_length() - cfg.cache_len
+        per_tok.append(e0.elapsed_time(e1) / n_tok)
+        accepted.append(n_tok / steps)
+    clocks = sampler.stop()
+    per_tok.sort()
+    ms = statistics.median(per_tok)
+    line = {"metric": METRIC, "value": ms, "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": 0, "ms_per_step": ms * statistics.median(accepted),
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 weights/KV, fp32 accumulate", "data": "synthetic",
+            "config": config_block(cfg, workload_name(cfg) + ", verified in blocks of 2 tokens (proposals: the model's own greedy continuation"
+                                   + (f", every {args.reject_every}th spoiled" if args.reject_every else "") + ")", 1),
+            "timed_sequences": len(per_tok), "ms_per_token_min": per_tok[0], "tokens_per_call": statistics.median(accepted),
+            "tokens_per_s": 1e3 / ms, "gpu_launches": steps * len(per_tok), "clocks": clocks}
+    print(json.dumps(line), flush=True)
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -202,6 +271,9 @@ def main():
                     help="prune the output layer to this many evenly spaced token ids (0 = full vocabulary, the headline workload)")
     ap.add_argument("--kv-format", default="bf16", choices=["bf16", "int8"],
                     help="cache format: int8 = the compressed cache (edgefm_create_with_options); not the headline configuration")
+    ap.add_argument("--block-tokens", type=int, default=1, choices=[1, 2],
+                    help="2: generate through edgefm_verify_block, two tokens per call (not the headline configuration)")
+    ap.add_argument("--reject-every", type=int, default=0, help="with --block-tokens 2: spoil every n-th proposal (0 = none)")
     ap.add_argument("--phase-timeline", action="store_true",
                     help="instead of the benchmark: print the per-operator timeline of one step from the kernel's own device timestamps")
     args = ap.parse_args()
@@ -217,6 +289,10 @@ def main():
 
     if args.impl == "reference":
         run_reference(args, cfg, rank)
+        return
+    if args.block_tokens > 1:
+        if rank == 0:
+            run_block(args, cfg)
         return
 
     import torch
