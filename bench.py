@@ -411,7 +411,7 @@ def main():
             "roofline": {"bound": "hbm", "kernel": f"decode_megakernel: the whole decode step ({launches} kernel launch per token, one CUDA graph node)",
                          "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak, "peak_source": peak_src,
                          "bytes_per_launch": bytes_per_step, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS, "traffic": traffic, "traffic_source": traffic_src},
-            "e2e": {"value": e2e_ms / tokens, "unit": UNIT, "h2d_bytes_per_step": 24, "d2h_bytes_per_step": 4},
+            "e2e": {"value": e2e_ms / tokens, "unit": UNIT, "h2d_bytes_per_step": 48, "d2h_bytes_per_step": 4},
             "gpu_launches": launches * steps * n_seq,
             "clocks": clocks,
             "cpu_baseline": cpu,

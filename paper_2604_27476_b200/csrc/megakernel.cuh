@@ -333,8 +333,9 @@ __device__ __forceinline__ bool fetch_next_tile(const MkParams &p, WarpStream &w
 }
 
 // Attention chunking shared by the attention phase and by the consumer of its partial results.
-__device__ __forceinline__ void att_chunking(const MkParams &p, int n, int hg, int min_chunk, int tile, int ncta, int &nch, int &chunk_len) {
-    const int groups = p.nq / hg;
+// mult: tokens of a block that are attended in the same pass (each with its own CTAs); n is then the longest token's length.
+__device__ __forceinline__ void att_chunking(const MkParams &p, int n, int hg, int min_chunk, int tile, int ncta, int &nch, int &chunk_len, int mult = 1) {
+    const int groups = p.nq / hg * mult;
     nch = (n + min_chunk - 1) / min_chunk;
     nch = min(nch, min(ncta / groups, p.max_chunks));
     if (hg == 1) nch = min(nch, MK_ATT_SPLIT_MAXC);
@@ -360,13 +361,14 @@ __device__ __forceinline__ void prefetch_tiles(const MkParams &p, volatile int *
         // The spare lanes pull the K and V rows this CTA's attention will read into L2, a layer ahead: as soon as warp 0's
         // ring has started on the tiles of layer l, the chunk of layer l (one-head-per-CTA chunking only).
         const int n_spare = 2 * (16 - MK_NW), me = (w - MK_NW) * 2 + half;
-        const int n = p.state->cur_len + 1;
+        const int m_run = MK_M > 1 ? min(max(p.req->m, 1), MK_M) : 1;
+        const int n = p.state->cur_len + m_run;
         if (p.kv8 || n > p.att_split_max_n || n < 1 || n > p.max_context) return;
         int nch, chunk_len;
-        att_chunking(p, n, 1, p.att_chunk_split, 32 / MK_ATT_LPP_SPLIT, static_cast<int>(gridDim.x), nch, chunk_len);
+        att_chunking(p, n, 1, p.att_chunk_split, 32 / MK_ATT_LPP_SPLIT, static_cast<int>(gridDim.x), nch, chunk_len, m_run);
         const int cta = static_cast<int>(blockIdx.x);
-        if (cta >= nch * p.nq) return;
-        const int qh = cta / nch, c = cta - qh * nch, g = qh / (p.nq / p.nkv);
+        if (cta >= nch * p.nq * m_run) return;
+        const int qh = (cta / nch) % p.nq, c = cta % nch, g = qh / (p.nq / p.nkv);
         const int t0 = c * chunk_len, t1 = min(n, t0 + chunk_len);
         const int n_lines = ((t1 - t0) * p.d * 2 + 127) / 128;
         const int n_layer0 = s_tab[7];
@@ -675,42 +677,44 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_
     const int lane = tid & 31, warp = tid >> 5;
     const int cta = blockIdx.x;
     const int n4 = P.K >> 2;
-    // the tokens of the call one after the other: token tk stages its vector into arrays 3 tk .. 3 tk + 2
-    for (int tk = 0; tk < cx.m_run; ++tk) {
-    unsigned char *const xs = xs0 + tk * (MK_X_SPLITS * xstride);
-    const int token = tokens[tk < MK_M ? tk : 0];
-    float ss = 0.f;
+    // Token tk of the call stages its vector into arrays 3 tk .. 3 tk + 2.  The pieces of all tokens form one list of items
+    // (token-major) that the threads share, so that the loads of all tokens are in flight together.
+    const int m_run = cx.m_run;
+    const int n_items = m_run * n4;
+    float ss[MK_M];
+#pragma unroll
+    for (int t = 0; t < MK_M; ++t) ss[t] = 0.f;
     if (merge_attn > 0) {
-        int nch = merge_attn;
-        if (MK_M > 1) { int cl; att_chunking(p, n_att + tk, 1, p.att_chunk_split, 32 / MK_ATT_LPP_SPLIT, static_cast<int>(gridDim.x), nch, cl); }
-        const float *part_o = p.part_o + static_cast<size_t>(tk) * p.nq * p.max_chunks * p.d;
-        const float *part_m = p.part_m + static_cast<size_t>(tk) * p.nq * p.max_chunks, *part_l = p.part_l + static_cast<size_t>(tk) * p.nq * p.max_chunks;
+        const int nch = merge_attn;   // chunks per head of the attention pass, the same for every token of the call
         const int d4 = p.d >> 2;
-        float *sm_m = s_partial;                 // [nq][nch] chunk maxima
-        float *sm_l = s_partial + p.nq * nch;    // [nq][nch] chunk denominators
-        // Thread t merges piece t of the vector (16 bytes: 4 dims of one head): all its chunk partials are requested at once,
-        // before the statistics are waited for.  (Spreading the left-over pieces of a vector longer than the CTA over all
-        // threads, parked in shared memory and summed after one more sync, was measured slower twice: 4.6 instead of 3.7 us
-        // for this prologue at the 1.5B shape even without spills.)
+        const int n_stat = p.nq * nch;
+        float *sm_m = s_partial;                     // [token][nq][nch] chunk maxima
+        float *sm_l = s_partial + m_run * n_stat;    // [token][nq][nch] chunk denominators
+        // A thread merges piece o4 of a token's vector (16 bytes: 4 dims of one head): all its chunk partials are requested at
+        // once, before the statistics are waited for.  (Spreading the left-over pieces of a vector longer than the CTA over
+        // all threads, parked in shared memory and summed after one more sync, was measured slower twice: 4.6 instead of
+        // 3.7 us for this prologue at the 1.5B shape even without spills.)
         float4 ob[MK_ATT_SPLIT_MAXC];
-        auto load_partials = [&](int o4) {
+        auto load_partials = [&](int item) {
+            const int tk = MK_M > 1 ? item / n4 : 0, o4 = item - tk * n4;
             const int h = o4 / d4, j4 = o4 - h * d4;
-            const float4 *po = reinterpret_cast<const float4 *>(part_o + static_cast<size_t>(h) * p.max_chunks * p.d) + j4;
+            const float4 *po = reinterpret_cast<const float4 *>(p.part_o + (static_cast<size_t>(tk) * p.nq + h) * p.max_chunks * p.d) + j4;
 #pragma unroll
             for (int c = 0; c < MK_ATT_SPLIT_MAXC; ++c)
                 if (c < nch) ob[c] = __ldcg(po + static_cast<size_t>(c) * d4);
         };
-        if (tid < n4) load_partials(tid);
-        for (int i = tid; i < p.nq * nch; i += MK_NT) {
-            const int h = i / nch, c = i - h * nch;
-            sm_m[i] = __ldcg(part_m + h * p.max_chunks + c);
-            sm_l[i] = __ldcg(part_l + h * p.max_chunks + c);
+        if (tid < n_items) load_partials(tid);
+        for (int i = tid; i < m_run * n_stat; i += MK_NT) {
+            const int hh = i / nch, c = i - hh * nch;      // hh = token * nq + head
+            sm_m[i] = __ldcg(p.part_m + hh * p.max_chunks + c);
+            sm_l[i] = __ldcg(p.part_l + hh * p.max_chunks + c);
         }
         cta_sync();
-        for (int o4 = tid; o4 < n4; o4 += MK_NT) {
-            if (o4 != tid) load_partials(o4);
+        for (int item = tid; item < n_items; item += MK_NT) {
+            if (item != tid) load_partials(item);
+            const int tk = MK_M > 1 ? item / n4 : 0, o4 = item - tk * n4;
             const int h = o4 / d4;
-            const float *hm = sm_m + h * nch, *hl = sm_l + h * nch;
+            const float *hm = sm_m + (tk * p.nq + h) * nch, *hl = sm_l + (tk * p.nq + h) * nch;
             float mm = -INFINITY;
             for (int c = 0; c < nch; ++c) mm = fmaxf(mm, hm[c]);
             float ll = 0.f;
@@ -726,23 +730,26 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_
             }
             const float inv = 1.f / ll;
             acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-            stage_piece(xs, xstride, o4, acc);
+            stage_piece(xs0 + tk * (MK_X_SPLITS * xstride), xstride, o4, acc);
         }
-        if (MK_M > 1) cta_sync();   // the statistics area is reused by the next token
     } else if (P.flags() & PHF_X_GLOBAL) {
         // nothing to stage: the consumer warps read the vector from global memory as they go
     } else {
         constexpr int PU = 4;  // loads in flight per thread
-        for (int base = tid; base < n4; base += MK_NT * PU) {
+        for (int base = tid; base < n_items; base += MK_NT * PU) {
             float4 v[PU];
             uint2 w[PU];
 #pragma unroll
             for (int u = 0; u < PU; ++u) {
-                const int i4 = base + u * MK_NT;
-                if (i4 < n4) {
+                const int item = base + u * MK_NT;
+                if (item < n_items) {
+                    const int tk = MK_M > 1 ? item / n4 : 0, i4 = item - tk * n4;
                     if (P.x_src) {
                         v[u] = __ldcg(reinterpret_cast<const float4 *>(P.x_src + (MK_M > 1 ? static_cast<size_t>(tk) * P.x_tok_stride : 0)) + i4);
                     } else {  // first operator of the step: the embedding row is the residual stream
+                        int token = tokens[0];
+#pragma unroll
+                        for (int t = 1; t < MK_M; ++t) token = tk == t ? tokens[t] : token;
                         const uint2 e = *reinterpret_cast<const uint2 *>(p.embed + static_cast<size_t>(token) * p.H + i4 * 4);
                         v[u] = make_float4(bf16lo(e.x), bf16hi(e.x), bf16lo(e.y), bf16hi(e.y));
                     }
@@ -751,15 +758,19 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_
             }
 #pragma unroll
             for (int u = 0; u < PU; ++u) {
-                const int i4 = base + u * MK_NT;
-                if (i4 < n4) {
+                const int item = base + u * MK_NT;
+                if (item < n_items) {
+                    const int tk = MK_M > 1 ? item / n4 : 0, i4 = item - tk * n4;
                     float4 t = v[u];
                     if (!P.x_src && cta == 0) reinterpret_cast<float4 *>(p.x + (MK_M > 1 ? static_cast<size_t>(tk) * p.H : 0))[i4] = t;
                     if (P.norm_w) {
-                        ss = fmaf(t.x, t.x, ss); ss = fmaf(t.y, t.y, ss); ss = fmaf(t.z, t.z, ss); ss = fmaf(t.w, t.w, ss);
+                        float sq = 0.f;
+                        sq = fmaf(t.x, t.x, sq); sq = fmaf(t.y, t.y, sq); sq = fmaf(t.z, t.z, sq); sq = fmaf(t.w, t.w, sq);
+#pragma unroll
+                        for (int tt = 0; tt < MK_M; ++tt) ss[tt] += tk == tt ? sq : 0.f;
                         t.x *= bf16lo(w[u].x); t.y *= bf16hi(w[u].x); t.z *= bf16lo(w[u].y); t.w *= bf16hi(w[u].y);
                     }
-                    stage_piece(xs, xstride, i4, t);
+                    stage_piece(xs0 + tk * (MK_X_SPLITS * xstride), xstride, i4, t);
                 }
             }
         }
@@ -768,13 +779,15 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_
         const int c1 = (P.K + MK_TILE_COLS - 1) / MK_TILE_COLS * MK_TILE_COLS;
         for (int c = P.K + 2 * tid; c < c1; c += 2 * MK_NT)
 #pragma unroll
-            for (int sp = 0; sp < MK_X_SPLITS; ++sp) *reinterpret_cast<unsigned *>(xs + sp * xstride + mk_xs_index(c) * 2) = 0u;
+            for (int sp = 0; sp < MK_X_SPLITS * MK_M; ++sp) *reinterpret_cast<unsigned *>(xs0 + sp * xstride + mk_xs_index(c) * 2) = 0u;
     }
     if (P.norm_w) {
-        ss = warp_sum(ss);
-        if (lane == 0) s_part[tk * MK_NW + warp] = ss;
+#pragma unroll
+        for (int t = 0; t < MK_M; ++t) {
+            const float tot = warp_sum(ss[t]);
+            if (lane == 0) s_part[t * MK_NW + warp] = tot;
+        }
     }
-    }   // tokens
     cta_sync();
     prof_stamp(p, tid, prof_idx);   // activation vector staged
 #pragma unroll
@@ -879,16 +892,23 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
     const int G = p.nq / p.nkv;
     const int groups = p.nq / HG;                       // head groups served by separate CTAs
     int nch, chunk_len;
-    att_chunking(p, n, HG, min_chunk, TILE, ncta, nch, chunk_len);
-    if (cta >= nch * groups) {
-        if (wait_heads && tok == 0) prof_stamp(p, tid, *prof_idx);
+    // a block (m_run > 1, tok < 0): all its tokens in this one pass, every (token, head) with CTAs of its own; n is the
+    // longest token's length and token t attends to n - (m_run - 1 - t) rows
+    const bool all_tokens = MK_M > 1 && tok < 0;
+    att_chunking(p, n, HG, min_chunk, TILE, ncta, nch, chunk_len, all_tokens ? m_run : 1);
+    if (all_tokens) {
+        tok = min(cta / (nch * groups), m_run - 1);
+        n -= m_run - 1 - tok;
+    }
+    if (cta >= nch * groups * (all_tokens ? m_run : 1)) {
+        if (wait_heads && (all_tokens || tok == 0)) prof_stamp(p, tid, *prof_idx);
         return;
     }
     const float *const q_tok = p.q + static_cast<size_t>(tok) * p.nq * D;
     float *const attn_tok = p.attn + static_cast<size_t>(tok) * p.nq * D;
     float *const part_o = p.part_o + static_cast<size_t>(tok) * p.nq * p.max_chunks * D;
     float *const part_m = p.part_m + static_cast<size_t>(tok) * p.nq * p.max_chunks, *const part_l = p.part_l + static_cast<size_t>(tok) * p.nq * p.max_chunks;
-    const int grp = cta / nch, c = cta - grp * nch;
+    const int grp = (cta / nch) % groups, c = cta % nch;
     const int qh0 = grp * HG;                            // first query head of this CTA
     const int g = qh0 / G;                               // its kv head
     const int t0 = c * chunk_len, t1 = min(n, t0 + chunk_len);
@@ -904,7 +924,7 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
             }
         }
         cta_sync();
-        if (tok == 0) prof_stamp(p, tid, *prof_idx);   // the heads this CTA reads are complete
+        if (all_tokens || tok == 0) prof_stamp(p, tid, *prof_idx);   // the heads this CTA reads are complete
     }
 
     float *qs = reinterpret_cast<float *>(xbuf);               // [HG][D]
@@ -1290,7 +1310,7 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
     // (a compressed cache is always attended with one CTA per kv head and chunk: one CTA then owns the row the step appends)
     const bool att_split = !LONG || (!Q8 && n_att <= p.att_split_max_n && static_cast<long long>(p.nq) * MK_ATT_SPLIT_MAXC * 2 <= MK_PARTIAL_FLOATS);
     int merge_chunks = 0;   // chunks per head the O-projection prologue has to merge (split mode)
-    if (att_split && MK_SPLIT_DEFER) { int cl; att_chunking(p, n_att, 1, p.att_chunk_split, 32 / MK_ATT_LPP_SPLIT, ncta, merge_chunks, cl); }
+    if (att_split && MK_SPLIT_DEFER) { int cl; att_chunking(p, n_att + m_run - 1, 1, p.att_chunk_split, 32 / MK_ATT_LPP_SPLIT, ncta, merge_chunks, cl, m_run); }
     // One loop over the operators of the step, with a single inlined copy of the streaming operator and of the grid barrier
     // (the code of a step is executed once per layer: a small instruction footprint matters).  Operator 4l+1 (the O
     // projection) is preceded by the attention of layer l.
@@ -1306,12 +1326,9 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
                 if (att_split) attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, sm_xbuf(p), tid, &s_flag);
                 else attention_phase<D, G, MK_ATT_LPP, Q8>(p, l, n_att, p.att_chunk_shared, false, sm_xbuf(p), tid, &s_flag);
             } else {
-                // (a block: the tokens one after the other; token t also attends to the rows of the tokens before it)
-                for (int t = 0; t < m_run; ++t) {
-                    if (MK_M > 1 && t > 0) cta_sync();   // the scratch of the previous token's pass is free
-                    attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att + t, p.att_chunk_split, MK_SPLIT_DEFER != 0, sm_xbuf(p), tid, &s_flag,
-                                                            p.head_flags != 0, abort_flag, &prof_idx, t, m_run);
-                }
+                // (a block: all its tokens in one pass; token t also attends to the rows of the tokens before it)
+                attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att + m_run - 1, p.att_chunk_split, MK_SPLIT_DEFER != 0, sm_xbuf(p), tid, &s_flag,
+                                                        p.head_flags != 0, abort_flag, &prof_idx, MK_M > 1 ? -1 : 0, m_run);
             }
             ok = grid_barrier(p, ++bar_no * bar_arrivals, abort_flag, tid, prof_idx) && ok;
             if (!ok) break;
