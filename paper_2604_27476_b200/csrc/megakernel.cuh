@@ -368,7 +368,7 @@ __device__ __forceinline__ void prefetch_tiles(const MkParams &p, volatile int *
         att_chunking(p, n, 1, p.att_chunk_split, 32 / MK_ATT_LPP_SPLIT, static_cast<int>(gridDim.x), nch, chunk_len, m_run);
         const int cta = static_cast<int>(blockIdx.x);
         if (cta >= nch * p.nq * m_run) return;
-        const int qh = (cta / nch) % p.nq, c = cta % nch, g = qh / (p.nq / p.nkv);
+        const int qh = MK_M > 1 ? (cta / nch) % p.nq : cta / nch, c = cta - (cta / nch) * nch, g = qh / (p.nq / p.nkv);
         const int t0 = c * chunk_len, t1 = min(n, t0 + chunk_len);
         const int n_lines = ((t1 - t0) * p.d * 2 + 127) / 128;
         const int n_layer0 = s_tab[7];
@@ -908,7 +908,7 @@ __device__ __forceinline__ void attention_phase(const MkParams &p, int layer, in
     float *const attn_tok = p.attn + static_cast<size_t>(tok) * p.nq * D;
     float *const part_o = p.part_o + static_cast<size_t>(tok) * p.nq * p.max_chunks * D;
     float *const part_m = p.part_m + static_cast<size_t>(tok) * p.nq * p.max_chunks, *const part_l = p.part_l + static_cast<size_t>(tok) * p.nq * p.max_chunks;
-    const int grp = (cta / nch) % groups, c = cta % nch;
+    const int grp = MK_M > 1 ? (cta / nch) % groups : cta / nch, c = cta - (cta / nch) * nch;
     const int qh0 = grp * HG;                            // first query head of this CTA
     const int g = qh0 / G;                               // its kv head
     const int t0 = c * chunk_len, t1 = min(n, t0 + chunk_len);
@@ -1310,7 +1310,11 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
     // (a compressed cache is always attended with one CTA per kv head and chunk: one CTA then owns the row the step appends)
     const bool att_split = !LONG || (!Q8 && n_att <= p.att_split_max_n && static_cast<long long>(p.nq) * MK_ATT_SPLIT_MAXC * 2 <= MK_PARTIAL_FLOATS);
     int merge_chunks = 0;   // chunks per head the O-projection prologue has to merge (split mode)
-    if (att_split && MK_SPLIT_DEFER) { int cl; att_chunking(p, n_att + m_run - 1, 1, p.att_chunk_split, 32 / MK_ATT_LPP_SPLIT, ncta, merge_chunks, cl, m_run); }
+    if (att_split && MK_SPLIT_DEFER) {
+        int cl;
+        if constexpr (MK_M > 1) att_chunking(p, n_att + m_run - 1, 1, p.att_chunk_split, 32 / MK_ATT_LPP_SPLIT, ncta, merge_chunks, cl, m_run);
+        else att_chunking(p, n_att, 1, p.att_chunk_split, 32 / MK_ATT_LPP_SPLIT, ncta, merge_chunks, cl);
+    }
     // One loop over the operators of the step, with a single inlined copy of the streaming operator and of the grid barrier
     // (the code of a step is executed once per layer: a small instruction footprint matters).  Operator 4l+1 (the O
     // projection) is preceded by the attention of layer l.
@@ -1327,8 +1331,13 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
                 else attention_phase<D, G, MK_ATT_LPP, Q8>(p, l, n_att, p.att_chunk_shared, false, sm_xbuf(p), tid, &s_flag);
             } else {
                 // (a block: all its tokens in one pass; token t also attends to the rows of the tokens before it)
-                attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att + m_run - 1, p.att_chunk_split, MK_SPLIT_DEFER != 0, sm_xbuf(p), tid, &s_flag,
-                                                        p.head_flags != 0, abort_flag, &prof_idx, MK_M > 1 ? -1 : 0, m_run);
+                if constexpr (MK_M > 1) {
+                    attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att + m_run - 1, p.att_chunk_split, MK_SPLIT_DEFER != 0, sm_xbuf(p), tid, &s_flag,
+                                                            p.head_flags != 0, abort_flag, &prof_idx, -1, m_run);
+                } else {
+                    attention_phase<D, 1, MK_ATT_LPP_SPLIT>(p, l, n_att, p.att_chunk_split, MK_SPLIT_DEFER != 0, sm_xbuf(p), tid, &s_flag,
+                                                            p.head_flags != 0, abort_flag, &prof_idx);
+                }
             }
             ok = grid_barrier(p, ++bar_no * bar_arrivals, abort_flag, tid, prof_idx) && ok;
             if (!ok) break;
