@@ -281,7 +281,7 @@ def main():
     if args.phase_timeline:
         from paper_2604_27476_b200 import build as cuda_build, timeline
         cuda_build.build()
-        print(timeline.format_table(timeline.summarize(timeline.collect(cfg), cfg), cfg))
+        print(timeline.format_table(timeline.summarize(timeline.collect(cfg, block_tokens=args.block_tokens if args.block_tokens > 1 else 0), cfg), cfg))
         return
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

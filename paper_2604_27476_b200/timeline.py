@@ -14,9 +14,10 @@ STAMPS = ["qkv_staged", "qkv_done", "qkv_released", "att_done", "att_released", 
           "gu_staged", "gu_done", "gu_released", "dn_staged", "dn_done", "dn_released"]
 
 
-def collect(cfg, device="cuda:0", warm_steps=6):
+def collect(cfg, device="cuda:0", warm_steps=6, block_tokens=0):
     """Run warm_steps chained steps of cfg from its configured cache and return the stamp table of the last one,
-    int64 [n_ctas][3 + 14 * n_layers] in nanoseconds."""
+    int64 [n_ctas][3 + 14 * n_layers] in nanoseconds.  block_tokens = 2: calls of edgefm_verify_block with two tokens
+    (the proposal is arbitrary: an accepted and a rejected token cost the same)."""
     import torch
     from edgefm_synth import first_token, make_kv, make_weights
     from . import DecodeContext, edgefm_debug_profile, edgefm_sync_status, upload_weights
@@ -27,7 +28,7 @@ def collect(cfg, device="cuda:0", warm_steps=6):
         w = make_weights(cfg)
         k, v = make_kv(cfg)
         ptrs, keep = upload_weights(w, device)
-        ctx = DecodeContext(cfg, ptrs, cfg.cache_len + warm_steps + 2, device)
+        ctx = DecodeContext(cfg, ptrs, cfg.cache_len + 2 * warm_steps + 2, device, block_tokens=block_tokens)
     finally:
         if old is None:
             del os.environ["EDGEFM_PROFILE"]
@@ -38,9 +39,14 @@ def collect(cfg, device="cuda:0", warm_steps=6):
     kd = torch.from_numpy(k.view(np.int16)).to(device)
     vd = torch.from_numpy(v.view(np.int16)).to(device)
     ctx.prefill_kv(kd, vd)
-    ctx.step(first_token(cfg), cfg.first_position, want_logits=False, want_token=False)
-    for _ in range(warm_steps - 1):
-        ctx.step(-1, -1, want_logits=False, want_token=False)
+    if block_tokens > 1:
+        ctx.verify_block([first_token(cfg), 5 % cfg.vocab], cfg.first_position, want_logits=False)
+        for _ in range(warm_steps - 1):
+            ctx.verify_block([-1, 7 % cfg.vocab], -1, want_logits=False)
+    else:
+        ctx.step(first_token(cfg), cfg.first_position, want_logits=False, want_token=False)
+        for _ in range(warm_steps - 1):
+            ctx.step(-1, -1, want_logits=False, want_token=False)
     edgefm_sync_status(ctx.handle, torch.cuda.current_stream(torch.device(device)).cuda_stream)
     t = edgefm_debug_profile(ctx.handle).astype(np.int64)
     ctx.close()

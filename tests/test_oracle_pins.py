@@ -373,6 +373,28 @@ def test_compressed_cache_load_compresses_the_given_rows(tiny_weights):
     assert (k8[:, :, 5:] == 0).all() and (vs[:, :, 5:] == 0).all() and m.cur_len == 5
 
 
+def test_block_verification_is_what_plain_steps_would_have_produced(tiny_weights):
+    """Sec. 3.11: verify token by token, stop at the first rejection, commit the accepted prefix.  Whatever the proposals,
+    the cache and the next token after a block equal those of n_accepted plain greedy steps."""
+    cfg, w = TINY, tiny_weights
+    plain = OracleModel(cfg, w, 16)
+    seq, tok = [], 17
+    for p in range(6):                       # the greedy continuation 17 -> seq[0] -> seq[1] ...
+        _, tok = plain.step(tok if p else 17, p)
+        seq.append(tok)
+    m = OracleModel(cfg, w, 16)
+    logits, n_acc, nxt = m.verify_block([17, seq[0], seq[1]], 0)            # all proposals right
+    assert (n_acc, nxt, m.cur_len, logits.shape) == (3, seq[2], 3, (3, cfg.vocab))
+    logits, n_acc, nxt = m.verify_block([seq[2], (seq[3] + 1) % cfg.vocab, seq[4]], 3)   # first proposal wrong: the right one behind it is not looked at
+    assert (n_acc, nxt, m.cur_len) == (1, seq[3], 4)
+    logits, n_acc, nxt = m.verify_block([seq[3], seq[4], (seq[5] + 1) % cfg.vocab], 4)   # second proposal wrong
+    assert (n_acc, nxt, m.cur_len) == (2, seq[5], 6)
+    ka, va = m.export_kv(); kb, vb = plain.export_kv()
+    assert np.array_equal(ka[:, :, :6], kb[:, :, :6]) and np.array_equal(va[:, :, :6], vb[:, :, :6])
+    with pytest.raises(ValueError):
+        m.truncate(7)
+
+
 def test_position_is_independent_of_slot(tiny_weights):
     # Same cache content, same token, different RoPE position => different logits; the slot written
     # is cur_len in both cases (vision-token prefixes make position != slot).
