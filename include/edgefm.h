@@ -170,6 +170,19 @@ edgefm_status edgefm_decode_step(edgefm_ctx *ctx, int32_t token_id, int32_t posi
 edgefm_status edgefm_verify_block(edgefm_ctx *ctx, const int32_t *tokens, int32_t m, int32_t position, void *stream,
                                   float *logits_out, int32_t *n_accepted_out, int32_t *next_token_out);
 
+/*
+ * edgefm_prefill_tokens -- compute the cache rows of n given tokens from the weights (Eq. 3 of the paper, KV <- Prefill(x);
+ * Sec. 3.9: KV_u of a request's own suffix behind a prefix).  The tokens pass through the decode-step kernel, as many per
+ * call as the context's build carries (1, or 2 with block_tokens = 2), at rotary positions position, position + 1, ... and
+ * cache slots cur_len, cur_len + 1, ...; every token enters the cache.  Afterwards the device holds the greedy token that
+ * follows tokens[n-1], so decoding continues with edgefm_decode_step(ctx, -1, -1, ...).
+ * This is prefill at the weight traffic of n (or n / 2) decode steps: it is exact and needs no other kernel, but it is not
+ * the GEMM-shaped prefill the paper's engine runs for long prompts (not part of this library); meant for short suffixes.
+ *   tokens : HOST int32 [n], read during the call.
+ * Errors: INVALID_ARG, CONTEXT_FULL (fewer than n free slots; nothing is launched), CUDA.
+ */
+edgefm_status edgefm_prefill_tokens(edgefm_ctx *ctx, const int32_t *tokens, int32_t n, int32_t position, void *stream);
+
 /* Wait for `stream`, then read the cache length from the device (exact again after edgefm_verify_block calls). */
 edgefm_status edgefm_sync_length(edgefm_ctx *ctx, void *stream, int32_t *cur_len_host);
 

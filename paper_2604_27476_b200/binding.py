@@ -52,7 +52,7 @@ class _Weights(ctypes.Structure):
 EXPORTS = ("edgefm_create", "edgefm_prefill_kv", "edgefm_decode_step", "edgefm_destroy", "edgefm_get_length",
            "edgefm_export_kv", "edgefm_get_launches_per_step", "edgefm_last_error", "edgefm_version",
            "edgefm_sync_status", "edgefm_debug_profile", "edgefm_debug_set_wait_limit", "edgefm_debug_plan", "edgefm_debug_plan_operator", "edgefm_decode_step_static", "edgefm_set_vocab_subset",
-           "edgefm_append_kv", "edgefm_create_with_options", "edgefm_export_kv_int8", "edgefm_verify_block", "edgefm_sync_length")
+           "edgefm_append_kv", "edgefm_create_with_options", "edgefm_export_kv_int8", "edgefm_verify_block", "edgefm_sync_length", "edgefm_prefill_tokens")
 
 
 def library_path() -> Path:
@@ -75,6 +75,8 @@ def load_library():
     L.edgefm_create_with_options.argtypes = [ctypes.POINTER(_Shape), ctypes.POINTER(_Weights), i32, ctypes.POINTER(_Options), ctypes.POINTER(vp)]
     L.edgefm_verify_block.restype = ctypes.c_int
     L.edgefm_verify_block.argtypes = [vp, ctypes.POINTER(i32), i32, i32, vp, vp, vp, vp]
+    L.edgefm_prefill_tokens.restype = ctypes.c_int
+    L.edgefm_prefill_tokens.argtypes = [vp, ctypes.POINTER(i32), i32, i32, vp]
     L.edgefm_sync_length.restype = ctypes.c_int
     L.edgefm_sync_length.argtypes = [vp, vp, ctypes.POINTER(i32)]
     L.edgefm_export_kv_int8.restype = ctypes.c_int
@@ -286,6 +288,11 @@ def edgefm_verify_block(ctx, tokens, position, stream=None, logits_out=None, n_a
     _check(load_library().edgefm_verify_block(ctx, arr, len(tokens), position, stream, logits_out, n_accepted_out, next_token_out), ctx)
 
 
+def edgefm_prefill_tokens(ctx, tokens, position, stream=None):
+    arr = (ctypes.c_int32 * max(1, len(tokens)))(*[int(t) for t in tokens])
+    _check(load_library().edgefm_prefill_tokens(ctx, arr, len(tokens), position, stream), ctx)
+
+
 def edgefm_sync_length(ctx, stream=None) -> int:
     n = ctypes.c_int32()
     _check(load_library().edgefm_sync_length(ctx, stream, ctypes.byref(n)), ctx)
@@ -371,6 +378,10 @@ class DecodeContext:
         """One call for a block of tokens (tokens[0] may be -1); results in block_logits[:m], n_accepted, next_token."""
         edgefm_verify_block(self.handle, tokens, position, self._stream(), self.block_logits.data_ptr() if want_logits else None,
                             self.n_accepted.data_ptr(), self.next_token.data_ptr())
+
+    def prefill_tokens(self, tokens, position):
+        """Append the cache rows of the given tokens (computed from the weights); the greedy next token stays on the device."""
+        edgefm_prefill_tokens(self.handle, tokens, position, self._stream())
 
     def sync_length(self) -> int:
         return edgefm_sync_length(self.handle, self._stream())

@@ -759,7 +759,7 @@ edgefm_status edgefm_verify_block(edgefm_ctx *ctx, const int32_t *tokens, int32_
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     StepRequest r{tokens[0], position, logits_out, next_token_out};
     r.m = m;
-    for (int t = 1; t < m && t <= 3; ++t) r.draft[t - 1] = tokens[t];
+    for (int t = 1; t < m && t <= 2; ++t) r.draft[t - 1] = tokens[t];
     r.n_accepted_out = n_accepted_out;
     if (!ctx->req_valid || std::memcmp(&r, &ctx->last_req, sizeof r) != 0) {
         CUDA_TRY(ctx, cudaMemcpyAsync(ctx->req, &r, sizeof r, cudaMemcpyHostToDevice, s));
@@ -769,6 +769,34 @@ edgefm_status edgefm_verify_block(edgefm_ctx *ctx, const int32_t *tokens, int32_
     CUDA_TRY(ctx, cudaGraphLaunch(ctx->exec, s));
     ctx->cur_len += m;     // an upper bound until edgefm_sync_length: the device decides how many tokens are accepted
     ctx->have_token = true;
+    ctx->err.clear();
+    return EDGEFM_OK;
+}
+
+edgefm_status edgefm_prefill_tokens(edgefm_ctx *ctx, const int32_t *tokens, int32_t n, int32_t position, void *stream) {
+    if (!ctx) return EDGEFM_ERR_INVALID_ARG;
+    if (n < 0 || (n > 0 && !tokens)) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "bad token list");
+    if (position < 0) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "position %d out of range", position);
+    for (int i = 0; i < n; ++i)
+        if (tokens[i] < 0 || tokens[i] >= ctx->shape.vocab) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "tokens[%d] = %d out of range", i, tokens[i]);
+    if (ctx->cur_len + n > ctx->max_context)
+        return fail(ctx, EDGEFM_ERR_CONTEXT_FULL, "%d tokens do not fit behind %d of %d cache slots", n, ctx->cur_len, ctx->max_context);
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int M = ctx->block_tokens;
+    for (int i = 0; i < n; i += M) {   // the step kernel, as many given tokens per call as the context's build carries
+        const int m = n - i < M ? n - i : M;
+        StepRequest r{tokens[i], position + i, nullptr, nullptr};
+        r.m = m;
+        for (int t = 1; t < m; ++t) r.draft[t - 1] = tokens[i + t];
+        r.flags = 1;
+        CUDA_TRY(ctx, cudaMemcpyAsync(ctx->req, &r, sizeof r, cudaMemcpyHostToDevice, s));
+        ctx->last_req = r;
+        ctx->req_valid = true;
+        CUDA_TRY(ctx, cudaGraphLaunch(ctx->exec, s));
+        ctx->cur_len += m;
+        ctx->have_token = true;
+    }
     ctx->err.clear();
     return EDGEFM_OK;
 }

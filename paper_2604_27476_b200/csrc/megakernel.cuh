@@ -1426,9 +1426,10 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
             // it stops at the first rejection.  The cache advances by the accepted tokens; the rows of the rejected ones
             // stay behind the cache length and are overwritten by the next call.
             int n_acc = 1;
+            const bool given = MK_M > 1 && (p.req->flags & 1);   // prompt tokens: nothing to verify
 #pragma unroll
             for (int t = 1; t < MK_M; ++t)
-                if (t < m_run && n_acc == t && tokens[t] == greedy[t - 1]) n_acc = t + 1;
+                if (t < m_run && n_acc == t && (given || tokens[t] == greedy[t - 1])) n_acc = t + 1;
             int bi = greedy[0];
 #pragma unroll
             for (int t = 1; t < MK_M; ++t)
