@@ -20,6 +20,8 @@ def _shapes():
         "d128_bias_gqa4": (base.with_(hidden=512, n_q_heads=8, n_kv_heads=2, head_dim=128, ffn=1536, vocab=3000, n_layers=3, qkv_bias=True), 300, 320),
         "long_ragged_chunks": (base.with_(hidden=384, n_q_heads=6, n_kv_heads=1, head_dim=128, ffn=1024, vocab=2000), 9001, 9010),
         "empty_cache": (base, 0, 6),
+        # the size and cache length bench.py --config qwen2.5-7b-32k --kv-format int8 times (two steps)
+        "qwen2.5-7b-32k_full_size": (CONFIGS["qwen2.5-7b-32k"], CONFIGS["qwen2.5-7b-32k"].cache_len, CONFIGS["qwen2.5-7b-32k"].cache_len + 2),
     }
 
 
@@ -45,7 +47,7 @@ def test_steps_with_compressed_cache_match_oracle(name):
                 assert int(pair.ctx.next_token.item()) == nxt
             tok, pos = nxt, pos + 1
         assert pair.ctx.cur_len == T0 + steps == pair.oracle.cur_len
-        # the appended rows: exactly rows T0 .. T0 + steps - 1 changed; codes within one step of the oracle's, scales equal to 1e-6
+        # the appended rows: exactly rows T0 .. T0 + steps - 1 changed; codes within one step of the oracle's, scales to 5e-5
         k8b, v8b, ksb, vsb = [t.cpu().numpy() for t in pair.ctx.export_kv_int8()]
         ok8, ov8, oks, ovs = pair.oracle.export_kv_q8()
         for got_c, got_s, ref_c, ref_s, before_c, before_s in ((k8b, ksb, ok8, oks, k8, ks), (v8b, vsb, ov8, ovs, v8, vs)):
@@ -55,7 +57,9 @@ def test_steps_with_compressed_cache_match_oracle(name):
             diff = np.abs(got_c[:, :, new].astype(np.int32) - ref_c[:, :, new].astype(np.int32))
             assert diff.max() <= 1 and (diff != 0).mean() < 0.02, (diff.max(), (diff != 0).mean())
             assert np.abs(got_c[:, :, new]).max(axis=-1).min() == 127                                           # every row uses the whole range
-            np.testing.assert_allclose(got_s[:, :, new], ref_s[:, :, new], rtol=2e-6)
+            # the scale is amax / 127 of a row whose fp32 values differ between the sides by the summation error of the path
+            # (fp32 against fp64 sums, growing with K and the number of layers: < 1e-5 at the 7B size); 5e-5 is 1/150 of a code step
+            np.testing.assert_allclose(got_s[:, :, new], ref_s[:, :, new], rtol=5e-5)
     finally:
         pair.close()
 
