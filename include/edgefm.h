@@ -160,7 +160,8 @@ edgefm_status edgefm_decode_step(edgefm_ctx *ctx, int32_t token_id, int32_t posi
  * g_{n_accepted - 1}.  The result is what n_accepted plain decode steps would have produced.
  *   tokens          : HOST int32 [m], read during the call.  m = 1 .. block_tokens of the context (m = 1 is a decode step).
  *   logits_out      : DEVICE fp32 [m][vocab] (row t: the logits after token t; rows >= n_accepted belong to rejected
- *                     tokens) or NULL.
+ *                     tokens) or NULL.  With a vocabulary subset of n ids (edgefm_set_vocab_subset) the rows are n long,
+ *                     [m][n], and the greedy tokens -- hence the acceptance -- are taken over the subset.
  *   n_accepted_out, next_token_out : DEVICE int32 [1] or NULL.
  * The host-side cache length (edgefm_get_length) cannot know n_accepted: after this call it is the upper bound
  * cur_len + m until edgefm_sync_length has been called.

@@ -120,3 +120,37 @@ def test_block_calls_are_validated():
         assert ei.value.status == Status.ERR_INVALID_ARG
     finally:
         plain.close(); block.close()
+
+
+def test_block_verification_over_a_pruned_vocabulary():
+    """With edgefm_set_vocab_subset the greedy tokens of a block, and with them the acceptance, are taken over the subset."""
+    import torch
+    from oracle import binding as O
+    cfg = CONFIGS["tiny"]
+    pair = Pair(cfg, cache_len=30, max_context=40, block_tokens=2)
+    try:
+        ids = np.unique(np.linspace(3, cfg.vocab - 1, 300).astype(np.int32))
+        pair.ctx.set_vocab_subset(ids)
+        tok, pos = int(ids[5]), 30
+        for r in range(3):
+            n0 = pair.oracle.cur_len
+            l0, _ = pair.oracle.step(tok, pos)
+            sub0, g0 = O.restricted_greedy(l0, ids)
+            proposal = g0 if r != 1 else int(ids[(int(np.searchsorted(ids, g0)) + 1) % ids.size])
+            l1, _ = pair.oracle.step(proposal, pos + 1)
+            sub1, g1 = O.restricted_greedy(l1, ids)
+            n_acc = 2 if proposal == g0 else 1
+            pair.oracle.truncate(n0 + n_acc)
+            pair.ctx.verify_block([tok, proposal], pos)
+            torch.cuda.synchronize()
+            got = pair.ctx.block_logits.cpu().numpy().reshape(-1)[:2 * ids.size].reshape(2, ids.size)   # rows of the subset's length
+            assert_logits_close(got[0], sub0, f"round {r} token 0")
+            assert_logits_close(got[1], sub1, f"round {r} token 1")
+            assert int(pair.ctx.n_accepted.item()) == n_acc
+            nxt = g1 if n_acc == 2 else g0
+            if top2_margin(sub0) > TOKEN_MARGIN and (n_acc == 1 or top2_margin(sub1) > TOKEN_MARGIN):
+                assert int(pair.ctx.next_token.item()) == nxt
+            assert pair.ctx.sync_length() == pair.oracle.cur_len
+            tok, pos = nxt, pos + n_acc
+    finally:
+        pair.close()
