@@ -9,7 +9,7 @@ namespace edgefm {
 // Device-resident dynamic parameters of the step graph (Sec. 3.10 of the paper: dynamic
 // parameters live in GPU buffers so that one fixed graph serves every decode iteration).
 struct StepState {
-    int token;          // input token of the step in flight (resolved by step_begin_kernel)
+    int token;          // input token of the step in flight
     int position;       // its rotary position
     int cur_len;        // filled cache slots before the step == slot the step writes
     int next_token;     // greedy result of the last finished step
@@ -31,28 +31,6 @@ struct StepRequest {
     int flags;          // bit 0: the tokens are given, not proposed (prompt tokens): all m enter the cache
     int *n_accepted_out;  // device int32[1] or null: how many of the m tokens entered the cache (1 + accepted proposals)
 };
-
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
-// 128-bit streaming load of read-only data that is used once: bypass L1, prefetch the L2 sector pair.
-__device__ __forceinline__ uint4 ldg_stream16(const void *p) {
-    uint4 v;
-    asm("ld.global.nc.L1::no_allocate.L2::256B.v4.u32 {%0,%1,%2,%3}, [%4];"
-        : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-        : "l"(p));
-    return v;
-}
-__device__ __forceinline__ uint2 ldg_stream8(const void *p) {
-    uint2 v;
-    asm("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "l"(p));
-    return v;
-}
-__device__ __forceinline__ uint32_t ldg_stream4(const void *p) {
-    uint32_t v;
-    asm("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
-    return v;
-}
 
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }

@@ -64,9 +64,6 @@ __device__ __forceinline__ unsigned smem_u32(const void *p) { return static_cast
 __device__ __forceinline__ void mbar_init(unsigned long long *b, unsigned count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(b)), "r"(count) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(unsigned long long *b) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(b)) : "memory");
-}
 __device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long *b, unsigned bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(bytes) : "memory");
 }
@@ -75,18 +72,6 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long *b, unsigned pa
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(b)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// non-blocking test (the feeding lanes poll many barriers and must never sleep on one)
-__device__ __forceinline__ bool mbar_test_wait(unsigned long long *b, unsigned parity) {
-    unsigned ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(smem_u32(b)), "r"(parity)
@@ -668,7 +653,7 @@ __device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkOp &P, 
 // merge_attn > 0: the input is the attention output, still split into merge_attn chunk partials per head
 // (m, l, unnormalised o); the exact log-sum-exp merge is done here, in chunk order, by every CTA.
 __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_layer, WarpStream &ws, volatile int *abort_flag, float *s_part,
-                                           float *s_partial, const float *s_rope, ItemCtx &cx, const int (&tokens)[MK_M], int merge_attn, int n_att, int tid,
+                                           float *s_partial, const float *s_rope, ItemCtx &cx, const int (&tokens)[MK_M], int merge_attn, int tid,
                                            int &prof_idx, volatile unsigned *s_issued, unsigned long long *full_bar) {
     const MkOp &P = sm_ops(p)[ph];
     unsigned char *const xs0 = sm_xbuf(p);
@@ -1342,7 +1327,7 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
             ok = grid_barrier(p, ++bar_no * bar_arrivals, abort_flag, tid, prof_idx) && ok;
             if (!ok) break;
         }
-        ok = gemv_phase(p, ph, layer_op ? (ph & 3) : 4, ws, abort_flag, s_part, s_partial, s_rope, cx, tokens, after_attention ? merge_chunks : 0, n_att, tid,
+        ok = gemv_phase(p, ph, layer_op ? (ph & 3) : 4, ws, abort_flag, s_part, s_partial, s_rope, cx, tokens, after_attention ? merge_chunks : 0, tid,
                         prof_idx, s_issued, full_bar);
         if (!LONG && p.head_flags && layer_op && (ph & 3) == 0) {
             // no grid barrier behind the QKV projection: the attention phase waits for the heads it reads (the CTA-wide sync

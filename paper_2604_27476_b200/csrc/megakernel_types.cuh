@@ -4,7 +4,6 @@
 
 namespace edgefm {
 
-constexpr int MK_BAR_POLLERS = 1;                // warps whose lane 0 polls the grid barrier counter
 constexpr int MK_ATT_LPP = 2;                    // lanes per cached position in the score phase (one CTA per GQA group)
 constexpr int MK_ATT_LPP_SPLIT = 2;              // ... when every query head has its own CTAs (16 positions per warp iteration)
 constexpr int MK_ATT_TILE = 32 / MK_ATT_LPP;     // positions per warp iteration (grouped mode)
