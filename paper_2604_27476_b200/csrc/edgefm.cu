@@ -177,14 +177,14 @@ inline const char *plan_step(const edgefm_shape &sh, int max_context, int num_sm
     cudaFuncAttributes fa{};
     *cuda_err = cudaFuncGetAttributes(&fa, pl->kernel);
     if (*cuda_err != cudaSuccess) return "cudaFuncGetAttributes";
-    const size_t static_smem = fa.sharedSizeBytes + 1024;   // the kernel's static shared memory (mbarriers, tables, scratch) + the padding in
+    const size_t static_smem = fa.sharedSizeBytes + (1024 - fa.sharedSizeBytes % 1024) % 1024;   // the kernel's static shared memory (mbarriers, tables, scratch) + the padding in
                                                             // front of the 1 KB-aligned dynamic part
     pl->ops_bytes = static_cast<size_t>(pl->n_ops) * sizeof(MkOp);
     const size_t tab = static_cast<size_t>(cta_tab_ints_for(NW)) * sizeof(int);
     pl->tab_bytes = (tab + 15) / 16 * 16;
     const size_t head = (pl->ops_bytes + pl->tab_bytes + sched_reserve + 1023) / 1024 * 1024;   // the rings start on a 1 KB boundary
     pl->sched_bytes = head - pl->ops_bytes - pl->tab_bytes;
-    const size_t tail = pl->xbuf + static_cast<size_t>(NW) * MK_WBUF_BYTES * block_tokens;   // behind the rings: the activation vector and the warps' small buffers
+    const size_t tail = pl->xbuf + static_cast<size_t>(NW) * mk_wbuf_bytes(block_tokens);   // behind the rings: the activation vector and the warps' small buffers
     if (head + tail + static_smem + static_cast<size_t>(NW) * 2 * 2048 > static_cast<size_t>(smem_optin))
         return "model shape does not fit the shared-memory plan";
     const size_t per_warp = (smem_optin - static_smem - head - tail) / NW;

@@ -531,14 +531,14 @@ __device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkOp &P, 
     // tile are copied asynchronously (no registers held) as soon as the current tile has been multiplied.
     const bool xg = (P.flags() & PHF_X_GLOBAL) != 0;
     const int kpad2 = (P.K + MK_TILE_COLS - 1) / MK_TILE_COLS * (MK_TILE_COLS * 2);
-    unsigned char *wbuf = sm_xbuf(p) + p.xbuf_bytes + warp * (MK_WBUF_BYTES * MK_M);   // [token][piece][512 + pad bytes]
-    const unsigned char *b_base = xg ? wbuf + (lane >> 2) * (MK_TILE_COLS * 2 + MK_XS_PAD) + (lane & 3) * 16
+    unsigned char *wbuf = sm_xbuf(p) + p.xbuf_bytes + warp * mk_wbuf_bytes(MK_M);   // [token][piece][512 (+ pad) bytes]
+    const unsigned char *b_base = xg ? wbuf + (lane >> 2) * mk_wbuf_array_bytes(MK_M) + (lane & 3) * 16
                                      : sm_xbuf(p) + (lane >> 2) * xs_stride(P.K) + (lane & 3) * 16;
     auto request_b = [&](int kcol) {
         const unsigned char *src = reinterpret_cast<const unsigned char *>(P.x_src) + kcol * (MK_TILE_COLS * 2) + lane * 16;
 #pragma unroll
         for (int c = 0; c < MK_X_SPLITS * MK_M; ++c)   // array c: piece c % 3 of token c / 3
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(wbuf + c * (MK_TILE_COLS * 2 + MK_XS_PAD) + lane * 16)),
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(wbuf + c * mk_wbuf_array_bytes(MK_M) + lane * 16)),
                          "l"(src + static_cast<size_t>(c / MK_X_SPLITS) * P.x_tok_stride * 2 + static_cast<size_t>(c % MK_X_SPLITS) * kpad2) : "memory");
         asm volatile("cp.async.commit_group;" ::: "memory");
     };

@@ -17,7 +17,11 @@ constexpr int MK_TILE_COLS = 256;                // columns of a weight tile: fo
 constexpr int MK_TILE_ROWS = 16;                 // rows of a tile: the M of one m16n8k16 tensor-core instruction (largest tile: 8 KB)
 constexpr int MK_X_SPLITS = 3;                   // an fp32 activation is staged as the sum of three bf16 pieces (24 mantissa bits)
 constexpr int MK_XS_PAD = 64;                    // bytes between the three staged arrays beyond the row length (bank spread)
-constexpr int MK_WBUF_BYTES = MK_X_SPLITS * (MK_TILE_COLS * 2 + MK_XS_PAD);   // a consumer warp's buffer for one tile's worth of a vector read from global memory
+// A consumer warp's buffer for one tile's worth of a vector read from global memory: 3 arrays of 512 bytes per token of the
+// call.  The single-token build spreads them over the banks (pad); a block build has no room for that (its shared memory
+// decides the size of the ring slots) and packs them.
+__host__ __device__ constexpr int mk_wbuf_array_bytes(int block_tokens) { return MK_TILE_COLS * 2 + (block_tokens > 1 ? 0 : MK_XS_PAD); }
+__host__ __device__ constexpr int mk_wbuf_bytes(int block_tokens) { return block_tokens * MK_X_SPLITS * mk_wbuf_array_bytes(block_tokens); }
 constexpr int MK_MAX_VARIANTS = 4;               // tensor maps (box heights) per weight matrix
 constexpr int MK_MAX_SLOTS = 4;                  // ring slots per consumer warp
 constexpr int MK_WARP_TAB = 8;                   // ints per warp in the per-CTA table
