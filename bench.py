@@ -199,7 +199,8 @@ def run_block(args, cfg):
     weights = make_weights(cfg)
     k, v = make_kv(cfg)
     ptrs, keep = upload_weights(weights, dev)
-    ctx = DecodeContext(cfg, ptrs, cfg.cache_len + 2 * steps + 2, dev, block_tokens=2)
+    B = args.block_tokens
+    ctx = DecodeContext(cfg, ptrs, cfg.cache_len + B * steps + B, dev, block_tokens=B)
     kd = torch.from_numpy(k.view(np.int16)).to(dev)
     vd = torch.from_numpy(v.view(np.int16)).to(dev)
     tok0, pos0 = first_token(cfg), cfg.first_position
@@ -207,7 +208,7 @@ def run_block(args, cfg):
     ctx.prefill_kv(kd, vd)
     seq = [tok0]
     ctx.step(tok0, pos0, want_logits=False)
-    for _ in range(2 * steps):
+    for _ in range(B * steps + B):
         torch.cuda.synchronize()
         seq.append(int(ctx.next_token.item()))
         ctx.step(-1, -1, want_logits=False)
@@ -218,10 +219,12 @@ def run_block(args, cfg):
         ctx.prefill_kv(kd, vd)
         idx = 0                      # seq[idx] is the token the next call decodes (if every correct proposal is accepted)
         for c in range(steps):
-            spoil = args.reject_every > 0 and c % args.reject_every == args.reject_every - 1
-            proposal = (seq[idx + 1] + 1) % cfg.vocab if spoil else seq[idx + 1]
-            ctx.verify_block([tok0 if c == 0 else -1, proposal], pos0 if c == 0 else -1, want_logits=False)
-            idx += 1 if spoil else 2
+            spoil = args.reject_every > 0 and c % args.reject_every == args.reject_every - 1   # the LAST proposal of this call is wrong
+            props = [seq[idx + t] for t in range(1, B)]
+            if spoil:
+                props[-1] = (props[-1] + 1) % cfg.vocab
+            ctx.verify_block([tok0 if c == 0 else -1] + props, pos0 if c == 0 else -1, want_logits=False)
+            idx += B - 1 if spoil else B
         return idx
 
     for _ in range(max(args.warmup_sequences, 1)):
@@ -246,9 +249,9 @@ def run_block(args, cfg):
     per_tok.sort()
     ms = statistics.median(per_tok)
     line = {"metric": METRIC, "value": ms, "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": 0, "ms_per_step": ms * statistics.median(accepted),
-            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 weights/KV, fp32 accumulate", "data": "synthetic",
-            "config": config_block(cfg, workload_name(cfg) + ", verified in blocks of 2 tokens (proposals: the model's own greedy continuation"
-                                   + (f", every {args.reject_every}th spoiled" if args.reject_every else "") + ")", 1),
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 weights/KV, fp32 accumulate" + (", activations as two bf16 pieces (16 mantissa bits)" if B > 2 else ""), "data": "synthetic",
+            "config": config_block(cfg, workload_name(cfg) + f", verified in blocks of {B} tokens (proposals: the model's own greedy continuation"
+                                   + (f", the last one of every {args.reject_every}th call spoiled" if args.reject_every else "") + ")", 1),
             "timed_sequences": len(per_tok), "ms_per_token_min": per_tok[0], "tokens_per_call": statistics.median(accepted),
             "tokens_per_s": 1e3 / ms, "gpu_launches": steps * len(per_tok), "clocks": clocks}
     print(json.dumps(line), flush=True)
@@ -271,8 +274,8 @@ def main():
                     help="prune the output layer to this many evenly spaced token ids (0 = full vocabulary, the headline workload)")
     ap.add_argument("--kv-format", default="bf16", choices=["bf16", "int8"],
                     help="cache format: int8 = the compressed cache (edgefm_create_with_options); not the headline configuration")
-    ap.add_argument("--block-tokens", type=int, default=1, choices=[1, 2],
-                    help="2: generate through edgefm_verify_block, two tokens per call (not the headline configuration)")
+    ap.add_argument("--block-tokens", type=int, default=1, choices=[1, 2, 4],
+                    help="2 / 4: generate through edgefm_verify_block, that many tokens per call (not the headline configuration)")
     ap.add_argument("--reject-every", type=int, default=0, help="with --block-tokens 2: spoil every n-th proposal (0 = none)")
     ap.add_argument("--phase-timeline", action="store_true",
                     help="instead of the benchmark: print the per-operator timeline of one step from the kernel's own device timestamps")

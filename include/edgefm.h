@@ -100,13 +100,15 @@ edgefm_status edgefm_create(const edgefm_shape *shape, const edgefm_weights *wei
  *     compressed as they are copied in.  The cache takes head_dim + 4 bytes per row instead of 2 head_dim.
  *     edgefm_export_kv is refused on such a context (use edgefm_export_kv_int8), and so is edgefm_decode_step_static.
  *   options->block_tokens = 0 or 1 : plain decode steps only;
- *                           2      : the context can also verify a block of two tokens per call (edgefm_verify_block).
- *     It then runs a build of the step kernel that carries two tokens side by side (work buffers for two tokens,
- *     somewhat smaller weight tiles); edgefm_decode_step works as before on such a context.  Needs the plain bf16
- *     cache and max_context <= 8192.
+ *                           2 or 4 : the context can also verify a block of up to that many tokens per call
+ *     (edgefm_verify_block).  It then runs a build of the step kernel that carries the tokens side by side (work buffers
+ *     per token, somewhat smaller weight tiles); edgefm_decode_step works as before on such a context.  The 2-token
+ *     build multiplies with the same 24-bit activations as the plain step; the 4-token build stages every activation as
+ *     two bf16 pieces (16 mantissa bits) so that four tokens fit one tensor-core operand.  Needs the plain bf16 cache and
+ *     max_context <= 8192.
  *   options->reserved must be zero.
  * Errors: as edgefm_create; INVALID_ARG for an unknown format, an unsupported block size or non-zero reserved fields;
- * BAD_SHAPE when block_tokens = 2 is combined with the compressed cache or a context beyond 8192 positions.
+ * BAD_SHAPE when block_tokens > 1 is combined with the compressed cache or a context beyond 8192 positions.
  */
 enum { EDGEFM_KV_BF16 = 0, EDGEFM_KV_INT8 = 1 };
 typedef struct {

@@ -27,8 +27,9 @@ struct StepRequest {
     float *logits_out;  // device fp32[V] (a block of m tokens: [m][V]) or null
     int *next_token_out;  // device int32[1] or null
     int m;              // tokens in this call: 1 = a plain decode step; > 1 = a block to verify (Sec. 3.11): `token` followed by
-    int draft[2];       // ... the proposed continuation draft[0 .. m-2]
+    int draft[3];       // ... the proposed continuation draft[0 .. m-2]
     int flags;          // bit 0: the tokens are given, not proposed (prompt tokens): all m enter the cache
+    int pad_;
     int *n_accepted_out;  // device int32[1] or null: how many of the m tokens entered the cache (1 + accepted proposals)
 };
 

@@ -120,10 +120,12 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const uint16_t *src, c
 // long_ctx = false: the variant without the grouped (one CTA per GQA group) attention code, for contexts that
 // never need it.
 MegaKernel mega_kernel_block2(int head_dim);   // megakernel_block2.cu
+MegaKernel mega_kernel_block4(int head_dim);   // megakernel_block4.cu
 
 template <int D>
 MegaKernel mega_kernel_g(int G, bool long_ctx, bool kv8 = false, int block_tokens = 1) {
     if (block_tokens == 2) return mega_kernel_block2(D);
+    if (block_tokens == 4) return mega_kernel_block4(D);
     if (kv8) {
         if (D == 64) return G <= 4 ? mega_kernel_q8_d64_lo(G) : mega_kernel_q8_d64_hi(G);
         return G <= 4 ? mega_kernel_q8_d128_lo(G) : mega_kernel_q8_d128_hi(G);
@@ -171,7 +173,7 @@ inline const char *plan_step(const edgefm_shape &sh, int max_context, int num_sm
     const int AG = pl->long_ctx ? G : 1;
     const size_t att_bytes = (static_cast<size_t>(AG) * d + NW * (AG * MK_ATT_TILE > 32 / MK_ATT_LPP_SPLIT ? AG * MK_ATT_TILE : 32 / MK_ATT_LPP_SPLIT) +
                               2 * ATT_MW * AG + static_cast<size_t>(ATT_MW) * AG * d + 2 * static_cast<size_t>(AG) * pl->max_chunks) * 4;
-    size_t xbuf = block_tokens * MK_X_SPLITS * (static_cast<size_t>(max_k) * 2 + MK_XS_PAD);   // the staged activations: three bf16 arrays per token
+    size_t xbuf = block_tokens * mk_splits(block_tokens) * (static_cast<size_t>(max_k) * 2 + MK_XS_PAD);   // the staged activations: three bf16 arrays per token
     if (att_bytes > xbuf) xbuf = att_bytes;
     pl->xbuf = (xbuf + 1023) / 1024 * 1024;
     cudaFuncAttributes fa{};
@@ -222,9 +224,9 @@ inline void op_shapes(const edgefm_shape &sh, int lm_rows, OpShape os[5]) {
 
 // The operators of the step in execution order, wired to the work buffers.
 inline void fill_ops(const edgefm_shape &sh, const edgefm_layer_weights *layers, const void *final_norm, const void *lm_head, float *x, float *attn, float *q,
-                     float *act, MkOp *out, const uint16_t **weights_out) {
+                     float *act, MkOp *out, const uint16_t **weights_out, int block_tokens = 1) {
     // distance between the vectors of consecutive tokens of a block (see MkParams::block_tokens)
-    const int sx = sh.hidden, sq = sh.n_q_heads * sh.head_dim, sa = MK_X_SPLITS * ((sh.ffn + MK_TILE_COLS - 1) / MK_TILE_COLS * MK_TILE_COLS);
+    const int sx = sh.hidden, sq = sh.n_q_heads * sh.head_dim, sa = mk_splits(block_tokens) * ((sh.ffn + MK_TILE_COLS - 1) / MK_TILE_COLS * MK_TILE_COLS);
     OpShape os[5];
     op_shapes(sh, sh.vocab, os);
     int n = 0;
@@ -480,9 +482,9 @@ edgefm_status edgefm_create_with_options(const edgefm_shape *shape, const edgefm
             if (r != 0) return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "reserved option fields must be zero");
     }
     const bool kv8 = options && options->kv_format == EDGEFM_KV_INT8;
-    if (options && (options->block_tokens < 0 || options->block_tokens > 2))
-        return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "block_tokens %d is not supported (0, 1 or 2)", options->block_tokens);
-    const int M = options && options->block_tokens == 2 ? 2 : 1;
+    if (options && options->block_tokens != 0 && options->block_tokens != 1 && options->block_tokens != 2 && options->block_tokens != 4)
+        return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "block_tokens %d is not supported (0, 1, 2 or 4)", options->block_tokens);
+    const int M = options && options->block_tokens > 1 ? options->block_tokens : 1;
     if (M > 1 && kv8) return fail(nullptr, EDGEFM_ERR_BAD_SHAPE, "blocks of several tokens need the plain bf16 cache");
     if (!shape || !weights || !out) return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "null argument");
     if (max_context < 1) return fail(nullptr, EDGEFM_ERR_INVALID_ARG, "max_context must be >= 1");
@@ -576,7 +578,7 @@ edgefm_status edgefm_create_with_options(const edgefm_shape *shape, const edgefm
     CREATE_TRY(dev_alloc(&c->x, static_cast<size_t>(M) * H));
     CREATE_TRY(dev_alloc(&c->q, static_cast<size_t>(M) * nq * d));
     CREATE_TRY(dev_alloc(&c->attn, static_cast<size_t>(M) * nq * d));
-    CREATE_TRY(dev_alloc(&c->act, static_cast<size_t>(M) * MK_X_SPLITS * ((F + MK_TILE_COLS - 1) / MK_TILE_COLS * MK_TILE_COLS) / 2));   // three bf16 arrays of F rounded
+    CREATE_TRY(dev_alloc(&c->act, static_cast<size_t>(M) * mk_splits(M) * ((F + MK_TILE_COLS - 1) / MK_TILE_COLS * MK_TILE_COLS) / 2));   // three bf16 arrays of F rounded
                                                                                          // up to whole column pieces (the pieces of every value)
     CREATE_TRY(dev_alloc(&c->inv_freq, d / 2));
     CREATE_TRY(dev_alloc(&c->part_m, static_cast<size_t>(M) * nq * pl.max_chunks));
@@ -603,7 +605,7 @@ edgefm_status edgefm_create_with_options(const edgefm_shape *shape, const edgefm
     {
         std::vector<MkOp> ops(static_cast<size_t>(pl.n_ops));
         std::vector<const uint16_t *> op_w(static_cast<size_t>(pl.n_ops));
-        fill_ops(sh, c->layers.data(), c->final_norm, c->lm_head, c->x, c->attn, c->q, c->act, ops.data(), op_w.data());
+        fill_ops(sh, c->layers.data(), c->final_norm, c->lm_head, c->x, c->attn, c->q, c->act, ops.data(), op_w.data(), M);
         c->lm_op_full = ops.back();
         std::vector<CUtensorMap> maps(static_cast<size_t>(pl.n_ops) * MK_MAX_VARIANTS);
         if (const char *why = encode_maps(ss, sh, c->layers.data(), c->lm_head, sh.vocab, maps.data()))
@@ -759,7 +761,7 @@ edgefm_status edgefm_verify_block(edgefm_ctx *ctx, const int32_t *tokens, int32_
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     StepRequest r{tokens[0], position, logits_out, next_token_out};
     r.m = m;
-    for (int t = 1; t < m && t <= 2; ++t) r.draft[t - 1] = tokens[t];
+    for (int t = 1; t < m && t <= 3; ++t) r.draft[t - 1] = tokens[t];
     r.n_accepted_out = n_accepted_out;
     if (!ctx->req_valid || std::memcmp(&r, &ctx->last_req, sizeof r) != 0) {
         CUDA_TRY(ctx, cudaMemcpyAsync(ctx->req, &r, sizeof r, cudaMemcpyHostToDevice, s));

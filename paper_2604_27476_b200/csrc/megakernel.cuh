@@ -46,7 +46,8 @@ constexpr int MK_NW = MK_NW_VALUE;               // consumer warps per CTA
 // verifies a proposed block); the weights are streamed once, every token has its own activation vectors, and the tensor-core
 // product carries the tokens side by side in the columns of its B operand (three columns per token).
 constexpr int MK_M = MK_M_VALUE;
-static_assert(MK_M >= 1 && MK_M * MK_X_SPLITS <= 8, "the tokens of a block share the eight columns of one B operand");
+constexpr int MK_S = mk_splits(MK_M);             // bf16 pieces per activation value in this build
+static_assert(MK_M >= 1 && MK_M * MK_S <= 8, "the tokens of a block share the eight columns of one B operand");
 constexpr int MK_NT = MK_NW * 32;                // consumer threads
 constexpr int MK_THREADS = MK_NT + 32;           // + the L2 prefetch warp
 
@@ -143,7 +144,7 @@ __device__ __forceinline__ unsigned char *sm_ring(const MkParams &p, int warp) {
     return mk_smem + p.ops_bytes + p.tab_bytes + p.sched_bytes + warp * (p.slots * p.slot_bytes);
 }
 __device__ __forceinline__ unsigned char *sm_xbuf(const MkParams &p) { return sm_ring(p, MK_NW); }
-// The staged activation vector of an operator with K columns: MK_X_SPLITS bf16 arrays of Kpad = K rounded up to whole
+// The staged activation vector of an operator with K columns: MK_S (2 or 3) bf16 arrays of Kpad = K rounded up to whole
 // 256-column pieces (zero beyond K), xs_stride(K) bytes apart.  Array s holds piece s of every value (value = sum of its
 // pieces to 24 bits), columns in tensor-core fragment order (mk_xs_index).
 __device__ __forceinline__ int xs_stride(int K) { return (K + MK_TILE_COLS - 1) / MK_TILE_COLS * (MK_TILE_COLS * 2) + MK_XS_PAD; }
@@ -158,7 +159,7 @@ __device__ __forceinline__ void stage_piece(unsigned char *xs, int stride, int i
     const int idx = mk_xs_index(i4 * 4);          // columns c, c+1 are neighbours; c+2, c+3 follow 8 entries later
     unsigned *dst = reinterpret_cast<unsigned *>(xs) + (idx >> 1);
 #pragma unroll
-    for (int sp = 0; sp < MK_X_SPLITS; ++sp) {
+    for (int sp = 0; sp < MK_S; ++sp) {
         const unsigned a = pack_bf16x2(t.x, t.y), b = pack_bf16x2(t.z, t.w);
         dst[0] = a;
         dst[4] = b;
@@ -445,7 +446,7 @@ __device__ __forceinline__ void apply_epilogue(const MkParams &p, const MkOp &P,
             uint16_t *o = reinterpret_cast<uint16_t *>(P.out) + (MK_M > 1 ? static_cast<size_t>(tok) * P.out_tok_stride : 0) + mk_xs_index(u);
             float r = a;
 #pragma unroll
-            for (int sp = 0; sp < MK_X_SPLITS; ++sp) {
+            for (int sp = 0; sp < MK_S; ++sp) {
                 const uint16_t b = f32_to_bf16_bits(r);
                 o[static_cast<size_t>(sp) * ((P.units_total + MK_TILE_COLS - 1) / MK_TILE_COLS * MK_TILE_COLS)] = b;
                 r -= bf16_bits_to_f32(b);
@@ -537,14 +538,14 @@ __device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkOp &P, 
     auto request_b = [&](int kcol) {
         const unsigned char *src = reinterpret_cast<const unsigned char *>(P.x_src) + kcol * (MK_TILE_COLS * 2) + lane * 16;
 #pragma unroll
-        for (int c = 0; c < MK_X_SPLITS * MK_M; ++c)   // array c: piece c % 3 of token c / 3
+        for (int c = 0; c < MK_S * MK_M; ++c)   // array c: piece c % MK_S of token c / MK_S
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(wbuf + c * mk_wbuf_array_bytes(MK_M) + lane * 16)),
-                         "l"(src + static_cast<size_t>(c / MK_X_SPLITS) * P.x_tok_stride * 2 + static_cast<size_t>(c % MK_X_SPLITS) * kpad2) : "memory");
+                         "l"(src + static_cast<size_t>(c / MK_S) * P.x_tok_stride * 2 + static_cast<size_t>(c % MK_S) * kpad2) : "memory");
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
     auto load_b = [&](const unsigned char *at) {
         uint4 v = make_uint4(0u, 0u, 0u, 0u);
-        if (lane < 4 * MK_X_SPLITS * MK_M) v = *reinterpret_cast<const uint4 *>(at);
+        if (lane < 4 * MK_S * MK_M) v = *reinterpret_cast<const uint4 *>(at);
         return v;
     };
     // A fragments: ldmatrix.x4 takes from lane l the address of row l % 8 of matrix l / 8; the four matrices are
@@ -617,8 +618,8 @@ __device__ __forceinline__ bool consume_tiles(const MkParams &p, const MkOp &P, 
                     // token tk: columns 3 tk .. 3 tk + 2; column c is register c % 2 of the lane with lane % 4 == c / 2
                     lo = 0.f; hi = 0.f;
 #pragma unroll
-                    for (int sp = 0; sp < MK_X_SPLITS; ++sp) {
-                        const int c = MK_X_SPLITS * tk + sp;
+                    for (int sp = 0; sp < MK_S; ++sp) {
+                        const int c = MK_S * tk + sp;
                         lo += __shfl_sync(0xffffffffu, (c & 1) ? d1 : d0, (lane & ~3) + (c >> 1));
                         hi += __shfl_sync(0xffffffffu, (c & 1) ? d3 : d2, (lane & ~3) + (c >> 1));
                     }
@@ -715,7 +716,7 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_
             }
             const float inv = 1.f / ll;
             acc.x *= inv; acc.y *= inv; acc.z *= inv; acc.w *= inv;
-            stage_piece(xs0 + tk * (MK_X_SPLITS * xstride), xstride, o4, acc);
+            stage_piece(xs0 + tk * (MK_S * xstride), xstride, o4, acc);
         }
     } else if (P.flags() & PHF_X_GLOBAL) {
         // nothing to stage: the consumer warps read the vector from global memory as they go
@@ -755,7 +756,7 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_
                         for (int tt = 0; tt < MK_M; ++tt) ss[tt] += tk == tt ? sq : 0.f;
                         t.x *= bf16lo(w[u].x); t.y *= bf16hi(w[u].x); t.z *= bf16lo(w[u].y); t.w *= bf16hi(w[u].y);
                     }
-                    stage_piece(xs0 + tk * (MK_X_SPLITS * xstride), xstride, i4, t);
+                    stage_piece(xs0 + tk * (MK_S * xstride), xstride, i4, t);
                 }
             }
         }
@@ -764,7 +765,7 @@ __device__ __forceinline__ bool gemv_phase(const MkParams &p, int ph, int op_in_
         const int c1 = (P.K + MK_TILE_COLS - 1) / MK_TILE_COLS * MK_TILE_COLS;
         for (int c = P.K + 2 * tid; c < c1; c += 2 * MK_NT)
 #pragma unroll
-            for (int sp = 0; sp < MK_X_SPLITS * MK_M; ++sp) *reinterpret_cast<unsigned *>(xs0 + sp * xstride + mk_xs_index(c) * 2) = 0u;
+            for (int sp = 0; sp < MK_S * MK_M; ++sp) *reinterpret_cast<unsigned *>(xs0 + sp * xstride + mk_xs_index(c) * 2) = 0u;
     }
     if (P.norm_w) {
 #pragma unroll
@@ -1273,7 +1274,7 @@ __global__ void __launch_bounds__(MK_THREADS, 1) decode_megakernel(const MkParam
         uint16_t *a = reinterpret_cast<uint16_t *>(sm_ops(p)[2].out);
         for (int c = p.F + tid; c < fpad; c += MK_NT)
 #pragma unroll
-            for (int sp = 0; sp < MK_X_SPLITS * MK_M; ++sp) a[static_cast<size_t>(sp) * fpad + mk_xs_index(c)] = 0;   // (the tokens' arrays follow one another)
+            for (int sp = 0; sp < MK_S * MK_M; ++sp) a[static_cast<size_t>(sp) * fpad + mk_xs_index(c)] = 0;   // (the tokens' arrays follow one another)
     }
     // (s_rope is published by the sync of the first prologue)
 

@@ -15,13 +15,18 @@ constexpr int MK_PARTIAL_SLOTS = 48;             // shared-memory scratch: parti
 constexpr int MK_PARTIAL_FLOATS = MK_PARTIAL_SLOTS * 16;   // (also the chunk statistics of the attention merge)
 constexpr int MK_TILE_COLS = 256;                // columns of a weight tile: four blocks of 64 columns (128-byte rows, the swizzle span)
 constexpr int MK_TILE_ROWS = 16;                 // rows of a tile: the M of one m16n8k16 tensor-core instruction (largest tile: 8 KB)
-constexpr int MK_X_SPLITS = 3;                   // an fp32 activation is staged as the sum of three bf16 pieces (24 mantissa bits)
+constexpr int MK_X_SPLITS = 3;                   // (the most; see mk_splits)
+// bf16 pieces an fp32 activation is staged as.  Three (24 mantissa bits) while the tokens of a call fit the eight B columns
+// that way (1 or 2 tokens); the build for blocks of up to four tokens keeps two pieces per token (16 mantissa bits, twice the
+// precision of the bf16 weights it multiplies).
+__host__ __device__ constexpr int mk_splits(int block_tokens) { return block_tokens > 2 ? 2 : 3; }
+                   // an fp32 activation is staged as the sum of three bf16 pieces (24 mantissa bits)
 constexpr int MK_XS_PAD = 64;                    // bytes between the three staged arrays beyond the row length (bank spread)
 // A consumer warp's buffer for one tile's worth of a vector read from global memory: 3 arrays of 512 bytes per token of the
 // call.  The single-token build spreads them over the banks (pad); a block build has no room for that (its shared memory
 // decides the size of the ring slots) and packs them.
 __host__ __device__ constexpr int mk_wbuf_array_bytes(int block_tokens) { return MK_TILE_COLS * 2 + (block_tokens > 1 ? 0 : MK_XS_PAD); }
-__host__ __device__ constexpr int mk_wbuf_bytes(int block_tokens) { return block_tokens * MK_X_SPLITS * mk_wbuf_array_bytes(block_tokens); }
+__host__ __device__ constexpr int mk_wbuf_bytes(int block_tokens) { return block_tokens * mk_splits(block_tokens) * mk_wbuf_array_bytes(block_tokens); }
 constexpr int MK_MAX_VARIANTS = 4;               // tensor maps (box heights) per weight matrix
 constexpr int MK_MAX_SLOTS = 4;                  // ring slots per consumer warp
 constexpr int MK_WARP_TAB = 8;                   // ints per warp in the per-CTA table

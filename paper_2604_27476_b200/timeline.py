@@ -28,7 +28,7 @@ def collect(cfg, device="cuda:0", warm_steps=6, block_tokens=0):
         w = make_weights(cfg)
         k, v = make_kv(cfg)
         ptrs, keep = upload_weights(w, device)
-        ctx = DecodeContext(cfg, ptrs, cfg.cache_len + 2 * warm_steps + 2, device, block_tokens=block_tokens)
+        ctx = DecodeContext(cfg, ptrs, cfg.cache_len + max(block_tokens, 1) * warm_steps + 4, device, block_tokens=block_tokens)
     finally:
         if old is None:
             del os.environ["EDGEFM_PROFILE"]
@@ -40,9 +40,9 @@ def collect(cfg, device="cuda:0", warm_steps=6, block_tokens=0):
     vd = torch.from_numpy(v.view(np.int16)).to(device)
     ctx.prefill_kv(kd, vd)
     if block_tokens > 1:
-        ctx.verify_block([first_token(cfg), 5 % cfg.vocab], cfg.first_position, want_logits=False)
+        ctx.verify_block([first_token(cfg)] + [5 % cfg.vocab] * (block_tokens - 1), cfg.first_position, want_logits=False)
         for _ in range(warm_steps - 1):
-            ctx.verify_block([-1, 7 % cfg.vocab], -1, want_logits=False)
+            ctx.verify_block([-1] + [7 % cfg.vocab] * (block_tokens - 1), -1, want_logits=False)
     else:
         ctx.step(first_token(cfg), cfg.first_position, want_logits=False, want_token=False)
         for _ in range(warm_steps - 1):

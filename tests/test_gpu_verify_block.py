@@ -116,7 +116,7 @@ def test_block_calls_are_validated():
             edgefm_create(shape, plain.ptrs, 9000, block_tokens=2)
         assert ei.value.status == Status.ERR_BAD_SHAPE
         with pytest.raises(EdgefmError) as ei:
-            edgefm_create(shape, plain.ptrs, 16, block_tokens=3)
+            edgefm_create(shape, plain.ptrs, 16, block_tokens=3)                 # 0, 1, 2 or 4
         assert ei.value.status == Status.ERR_INVALID_ARG
     finally:
         plain.close(); block.close()
@@ -152,5 +152,57 @@ def test_block_verification_over_a_pruned_vocabulary():
                 assert int(pair.ctx.next_token.item()) == nxt
             assert pair.ctx.sync_length() == pair.oracle.cur_len
             tok, pos = nxt, pos + n_acc
+    finally:
+        pair.close()
+
+
+def _peek_chain(pair, tok, pos, k):
+    """The oracle's next k greedy tokens after `tok`, without changing its cache."""
+    n = pair.oracle.cur_len
+    out = []
+    for i in range(k):
+        _, tok = pair.oracle.step(tok, pos + i)
+        out.append(tok)
+    pair.oracle.truncate(n)
+    return out
+
+
+@pytest.mark.parametrize("name", ["tiny_d64", "d128_bias", "qwen2.5-1.5b_full_size"])
+def test_blocks_of_four_match_the_oracle_verification(name):
+    """The four-token build (two bf16 pieces per activation): the first wrong proposal ends the block wherever it stands."""
+    import torch
+    cfg, T0 = SHAPES[name]
+    rounds = 8 if cfg.n_layers < 8 else 4
+    pair = Pair(cfg, cache_len=T0, max_context=T0 + 4 * rounds + 4, block_tokens=4)
+    try:
+        tok, pos = first_token(cfg), T0 + 2
+        for r in range(rounds):
+            props = _peek_chain(pair, tok, pos, 3)
+            wrong_at = r % 4                                   # 0: none wrong; 1..3: proposal wrong_at is wrong
+            if wrong_at:
+                props[wrong_at - 1] = (props[wrong_at - 1] + 7) % cfg.vocab
+            block = [tok] + props
+            m = 4 if r != 5 else 3                             # once a shorter block
+            block = block[:m]
+            ref_logits, ref_acc, ref_next = pair.oracle.verify_block(block, pos)
+            assert ref_acc == (min(wrong_at, m) if wrong_at else m)
+            pair.ctx.verify_block([tok if r % 2 == 0 else -1] + block[1:], pos if r % 2 == 0 else -1)
+            torch.cuda.synchronize()
+            got = pair.ctx.block_logits.cpu().numpy()
+            for t in range(m):
+                assert_logits_close(got[t], ref_logits[t], f"{name} round {r} token {t}")
+            assert int(pair.ctx.n_accepted.item()) == ref_acc
+            assert pair.ctx.sync_length() == pair.oracle.cur_len
+            if not all(top2_margin(ref_logits[t]) > TOKEN_MARGIN for t in range(ref_acc)):
+                break
+            assert int(pair.ctx.next_token.item()) == ref_next
+            tok, pos = ref_next, pos + ref_acc
+        from helpers import assert_appended_rows_close
+        n = pair.oracle.cur_len
+        kg, vg = [t.cpu().numpy().view(np.uint16) for t in pair.ctx.export_kv()]
+        ko, vo = pair.oracle.export_kv()
+        if n > T0:
+            assert_appended_rows_close(kg[:, :, T0:n], ko[:, :, T0:n])
+            assert_appended_rows_close(vg[:, :, T0:n], vo[:, :, T0:n])
     finally:
         pair.close()
