@@ -200,7 +200,7 @@ def run_block(args, cfg):
     k, v = make_kv(cfg)
     ptrs, keep = upload_weights(weights, dev)
     B = args.block_tokens
-    ctx = DecodeContext(cfg, ptrs, cfg.cache_len + B * steps + B, dev, block_tokens=B)
+    ctx = DecodeContext(cfg, ptrs, cfg.cache_len + B * steps + B + 2, dev, block_tokens=B)
     kd = torch.from_numpy(k.view(np.int16)).to(dev)
     vd = torch.from_numpy(v.view(np.int16)).to(dev)
     tok0, pos0 = first_token(cfg), cfg.first_position
