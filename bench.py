@@ -258,6 +258,71 @@ def run_block(args, cfg):
     ctx.close()
 
 
+def run_prefill(args, cfg):
+    """The prefill phase (edgefm_prefill) for a prompt of --prefill tokens into an empty cache: ms per prompt (median over
+    --sequences calls, each between its own CUDA events), prompt tokens/s and the contraction rate.  Not the headline
+    workload.  Flops counted: 2 * tokens * (weights of the four projections of every layer that runs) + causal attention
+    (4 * d * n_q * sum over queries of the keys seen); the last prompt token is a decode step inside the same call."""
+    import torch
+    from paper_2604_27476_b200 import DecodeContext, build as cuda_build, upload_weights
+    cuda_build.build()
+    dev = "cuda:0"
+    T = args.prefill
+    weights = make_weights(cfg)
+    ptrs, keep = upload_weights(weights, dev)
+    ctx = DecodeContext(cfg, ptrs, T + 2, dev)
+    toks = np.random.default_rng(1).integers(0, cfg.vocab, T).tolist()
+    for _ in range(max(args.warmup_sequences, 3)):
+        ctx.reset()
+        ctx.prefill(toks, 0, want_logits=False)
+    torch.cuda.synchronize()
+    ctx.sync_status()
+    sampler = ClockSampler(0)
+    sampler.start()
+    times = []
+    for _ in range(max(args.sequences, 1)):
+        ctx.reset()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        ctx.prefill(toks, 0, want_logits=False)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    clocks = sampler.stop()
+    ctx.sync_status()
+    times.sort()
+    ms = statistics.median(times)
+    H, F, d, nq, nkv, L = cfg.hidden, cfg.ffn, cfg.head_dim, cfg.n_q_heads, cfg.n_kv_heads, cfg.n_layers
+    n = T - 1
+    qkv = (nq + 2 * nkv) * d * H
+    rest = nq * d * H + 3 * H * F
+    flops = 2.0 * n * (L * qkv + (L - 1) * rest) + (L - 1) * 4.0 * d * nq * (n * (n + 1) / 2)
+    peaks = {}
+    try:
+        peaks = json.loads((ROOT / "MEASURED_PEAKS.json").read_text())
+    except Exception:
+        pass
+    peak = float(peaks.get("bf16_tflops_sustained") or 1400.0)   # a prompt is a long step: the sustained figure
+    tf = flops / (ms * 1e-3) / 1e12
+    line = {"metric": "prefill_ms_per_prompt", "value": ms, "unit": "ms", "n_gpus": 1, "steps": len(times), "warmup": max(args.warmup_sequences, 3),
+            "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16 weights/KV, activations as two bf16 pieces, fp32 accumulate (tcgen05)", "data": "synthetic",
+            "config": {"workload": f"{cfg.name}: prefill of {T} prompt tokens into an empty cache (edgefm_prefill; {n} tokens as dense contractions + one decode step)",
+                       "l2": "weights (> 2.6 GB) and activations exceed L2; nothing flushed"},
+            "ms_min": times[0], "prompt_tokens_per_s": T / (ms * 1e-3),
+            "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak, "traffic": None,
+                         "note": "achieved counts the method's flops; the tensor cores execute twice that (two bf16 pieces per activation); peak = measured sustained cuBLAS bf16 rate" + ("" if peaks.get("bf16_tflops_sustained") else " (fallback)")},
+            "gpu_launches": len(times) * ctx_prefill_launches(cfg), "clocks": clocks}
+    print(json.dumps(line), flush=True)
+    ctx.close()
+
+
+def ctx_prefill_launches(cfg):
+    """Kernels one edgefm_prefill call enqueues: rope table + embedding/norm, 7 per layer but the last (QKV only), one step."""
+    return 2 + 7 * (cfg.n_layers - 1) + 1 + 1
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -277,6 +342,8 @@ def main():
     ap.add_argument("--block-tokens", type=int, default=1, choices=[1, 2, 4],
                     help="2 / 4: generate through edgefm_verify_block, that many tokens per call (not the headline configuration)")
     ap.add_argument("--reject-every", type=int, default=0, help="with --block-tokens 2: spoil every n-th proposal (0 = none)")
+    ap.add_argument("--prefill", type=int, default=0,
+                    help="instead of the decode benchmark: time edgefm_prefill for a prompt of this many tokens (not the headline workload)")
     ap.add_argument("--phase-timeline", action="store_true",
                     help="instead of the benchmark: print the per-operator timeline of one step from the kernel's own device timestamps")
     args = ap.parse_args()
@@ -296,6 +363,10 @@ def main():
     if args.block_tokens > 1:
         if rank == 0:
             run_block(args, cfg)
+        return
+    if args.prefill > 0:
+        if rank == 0:
+            run_prefill(args, cfg)
         return
 
     import torch

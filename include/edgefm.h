@@ -176,15 +176,35 @@ edgefm_status edgefm_verify_block(edgefm_ctx *ctx, const int32_t *tokens, int32_
 /*
  * edgefm_prefill_tokens -- compute the cache rows of n given tokens from the weights (Eq. 3 of the paper, KV <- Prefill(x);
  * Sec. 3.9: KV_u of a request's own suffix behind a prefix).  The tokens pass through the decode-step kernel, as many per
- * call as the context's build carries (1, or 2 with block_tokens = 2), at rotary positions position, position + 1, ... and
+ * call as the context's build carries (1, or block_tokens), at rotary positions position, position + 1, ... and
  * cache slots cur_len, cur_len + 1, ...; every token enters the cache.  Afterwards the device holds the greedy token that
  * follows tokens[n-1], so decoding continues with edgefm_decode_step(ctx, -1, -1, ...).
- * This is prefill at the weight traffic of n (or n / 2) decode steps: it is exact and needs no other kernel, but it is not
- * the GEMM-shaped prefill the paper's engine runs for long prompts (not part of this library); meant for short suffixes.
+ * This is prefill at the weight traffic of n / block_tokens decode steps, in the step's own arithmetic (24- or 16-bit
+ * activations); meant for short suffixes and for the compressed cache.  Long prompts: edgefm_prefill.
  *   tokens : HOST int32 [n], read during the call.
  * Errors: INVALID_ARG, CONTEXT_FULL (fewer than n free slots; nothing is launched), CUDA.
  */
 edgefm_status edgefm_prefill_tokens(edgefm_ctx *ctx, const int32_t *tokens, int32_t n, int32_t position, void *stream);
+
+/*
+ * edgefm_prefill -- the prefill phase (Eq. 3 of the paper, KV <- Prefill(x_1:T; theta_p); with a prefix already in the cache,
+ * Eq. 5: KV = Concat(KV_p, KV_u)) as dense contractions.  The first n - 1 tokens pass through the layers TOGETHER (at most
+ * 2048 per pass): every projection is one [tokens x K] x [K x N] product on the tensor cores (tcgen05, fp32 accumulation in
+ * tensor memory; every activation enters as two bf16 pieces, hi + lo = 16 mantissa bits, the weights are bf16 exactly; fp32
+ * residual stream), attention is causal over the cache rows 0 .. cur_len + t; the K and V rows go to cache slots cur_len ..
+ * Token n - 1 then takes an ordinary decode step, so that logits_out / next_token_out and the device state are what
+ * edgefm_decode_step leaves behind; decoding continues with edgefm_decode_step(ctx, -1, -1, ...).
+ * The cache rows agree with those of n decode steps up to the last bf16 step of a value.
+ *   tokens     : HOST int32 [n], n >= 1, read during the call.
+ *   position   : rotary position of tokens[0] (>= 0); token i has position + i.
+ *   logits_out : DEVICE fp32 [vocab] (or the subset's length) or NULL;  next_token_out : DEVICE int32 [1] or NULL.
+ * The work buffers (about (8 H + 8 n_q d + 4 F) bytes per token of a pass) are allocated at the first call and kept.
+ * After edgefm_verify_block call edgefm_sync_length first: the rows are placed behind the host's cache length.
+ * Errors: INVALID_ARG (also: a compressed cache), CONTEXT_FULL (fewer than n free slots; nothing is launched),
+ * OUT_OF_MEMORY, CUDA.  A bounded wait of a contraction that runs out is reported by edgefm_sync_status (TIMEOUT).
+ */
+edgefm_status edgefm_prefill(edgefm_ctx *ctx, const int32_t *tokens, int32_t n, int32_t position, void *stream,
+                             float *logits_out, int32_t *next_token_out);
 
 /* Wait for `stream`, then read the cache length from the device (exact again after edgefm_verify_block calls). */
 edgefm_status edgefm_sync_length(edgefm_ctx *ctx, void *stream, int32_t *cur_len_host);

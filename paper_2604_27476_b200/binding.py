@@ -52,7 +52,7 @@ class _Weights(ctypes.Structure):
 EXPORTS = ("edgefm_create", "edgefm_prefill_kv", "edgefm_decode_step", "edgefm_destroy", "edgefm_get_length",
            "edgefm_export_kv", "edgefm_get_launches_per_step", "edgefm_last_error", "edgefm_version",
            "edgefm_sync_status", "edgefm_debug_profile", "edgefm_debug_set_wait_limit", "edgefm_debug_plan", "edgefm_debug_plan_operator", "edgefm_decode_step_static", "edgefm_set_vocab_subset",
-           "edgefm_append_kv", "edgefm_create_with_options", "edgefm_export_kv_int8", "edgefm_verify_block", "edgefm_sync_length", "edgefm_prefill_tokens")
+           "edgefm_append_kv", "edgefm_create_with_options", "edgefm_export_kv_int8", "edgefm_verify_block", "edgefm_sync_length", "edgefm_prefill_tokens", "edgefm_prefill")
 
 
 def library_path() -> Path:
@@ -77,6 +77,8 @@ def load_library():
     L.edgefm_verify_block.argtypes = [vp, ctypes.POINTER(i32), i32, i32, vp, vp, vp, vp]
     L.edgefm_prefill_tokens.restype = ctypes.c_int
     L.edgefm_prefill_tokens.argtypes = [vp, ctypes.POINTER(i32), i32, i32, vp]
+    L.edgefm_prefill.restype = ctypes.c_int
+    L.edgefm_prefill.argtypes = [vp, ctypes.POINTER(i32), i32, i32, vp, vp, vp]
     L.edgefm_sync_length.restype = ctypes.c_int
     L.edgefm_sync_length.argtypes = [vp, vp, ctypes.POINTER(i32)]
     L.edgefm_export_kv_int8.restype = ctypes.c_int
@@ -293,6 +295,11 @@ def edgefm_prefill_tokens(ctx, tokens, position, stream=None):
     _check(load_library().edgefm_prefill_tokens(ctx, arr, len(tokens), position, stream), ctx)
 
 
+def edgefm_prefill(ctx, tokens, position, stream=None, logits_out=None, next_token_out=None):
+    arr = (ctypes.c_int32 * max(1, len(tokens)))(*[int(t) for t in tokens])
+    _check(load_library().edgefm_prefill(ctx, arr, len(tokens), position, stream, logits_out, next_token_out), ctx)
+
+
 def edgefm_sync_length(ctx, stream=None) -> int:
     n = ctypes.c_int32()
     _check(load_library().edgefm_sync_length(ctx, stream, ctypes.byref(n)), ctx)
@@ -382,6 +389,15 @@ class DecodeContext:
     def prefill_tokens(self, tokens, position):
         """Append the cache rows of the given tokens (computed from the weights); the greedy next token stays on the device."""
         edgefm_prefill_tokens(self.handle, tokens, position, self._stream())
+
+    def prefill(self, tokens, position=0, want_logits=True):
+        """The prefill phase for a prompt: dense contractions for all but the last token, a decode step for the last."""
+        edgefm_prefill(self.handle, tokens, position, self._stream(), self.logits.data_ptr() if want_logits else None,
+                       self.next_token.data_ptr())
+
+    def sync_status(self):
+        """Synchronise the stream and raise EdgefmError(ERR_TIMEOUT) if a bounded device-side wait ran out."""
+        edgefm_sync_status(self.handle, self._stream())
 
     def sync_length(self) -> int:
         return edgefm_sync_length(self.handle, self._stream())

@@ -25,7 +25,7 @@ def source_hash() -> str:
     """Hash of everything the library is built from (content, not time stamps: a copied tree keeps its build)."""
     import hashlib
     h = hashlib.sha256()
-    deps = sorted(list(CSRC.glob("*.cu")) + list(CSRC.glob("*.cuh"))) + [PKG.parent / "include" / "edgefm.h"]
+    deps = sorted(list(CSRC.glob("*.cu")) + list(CSRC.glob("*.cuh")) + list(CSRC.glob("*.h"))) + [PKG.parent / "include" / "edgefm.h"]
     for p in deps:
         h.update(p.name.encode())
         h.update(p.read_bytes())

@@ -14,6 +14,7 @@
 #include "common.cuh"
 #include "megakernel_types.cuh"
 #include "step_plan.h"
+#include "prefill.h"
 // the persistent kernel is built twice: 11 consumer warps per CTA (short contexts, here) and 7 (long contexts,
 // in the megakernel_long_*.cu translation units), plus the warp that prefetches into L2
 #define MK_NS mk_short
@@ -373,6 +374,8 @@ struct edgefm_ctx {
     cudaGraph_t graph = nullptr;
     cudaGraphExec_t exec = nullptr;
     int launches_per_step = 0;
+    PrefillBuffers pf;           // work buffers of edgefm_prefill, allocated at its first call
+    int prefill_launches = 0;    // kernels the last edgefm_prefill enqueued
 
     // host mirrors
     int cur_len = 0;
@@ -426,6 +429,7 @@ void free_all(edgefm_ctx *c) {
                     c->part_o, c->lm_part_val, c->lm_part_idx, c->tickets, c->state, c->req, c->d_ops, c->d_op_w, c->d_maps, c->d_tiles,
                     c->d_cta_tab, c->d_combines, c->grid_bar, c->prof, c->vocab_ids, c->sub_lm, c->k_scale, c->v_scale, c->kv_stage};
     for (void *b : bufs) if (b) cudaFree(b);
+    if (c->pf.chunk) prefill_free(&c->pf);
 }
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -803,6 +807,46 @@ edgefm_status edgefm_prefill_tokens(edgefm_ctx *ctx, const int32_t *tokens, int3
     return EDGEFM_OK;
 }
 
+edgefm_status edgefm_prefill(edgefm_ctx *ctx, const int32_t *tokens, int32_t n, int32_t position, void *stream, float *logits_out,
+                             int32_t *next_token_out) {
+    if (!ctx) return EDGEFM_ERR_INVALID_ARG;
+    if (n < 1 || !tokens) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "bad token list");
+    if (position < 0) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "position %d out of range", position);
+    for (int i = 0; i < n; ++i)
+        if (tokens[i] < 0 || tokens[i] >= ctx->shape.vocab) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "tokens[%d] = %d out of range", i, tokens[i]);
+    if (ctx->kv_format != EDGEFM_KV_BF16)
+        return fail(ctx, EDGEFM_ERR_INVALID_ARG, "edgefm_prefill writes bf16 cache rows: use edgefm_prefill_tokens on a compressed cache");
+    if (ctx->cur_len + n > ctx->max_context)
+        return fail(ctx, EDGEFM_ERR_CONTEXT_FULL, "%d tokens do not fit behind %d of %d cache slots", n, ctx->cur_len, ctx->max_context);
+    DeviceGuard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int n_dense = n - 1;   // the last token takes the decode step, which also yields the logits
+    if (n_dense > 0 && ctx->pf.chunk == 0) {
+        const int chunk = std::min(PF_CHUNK_MAX, ctx->max_context);
+        if (prefill_alloc(&ctx->pf, ctx->shape, chunk) != cudaSuccess) {
+            cudaGetLastError();
+            prefill_free(&ctx->pf);
+            return fail(ctx, EDGEFM_ERR_OUT_OF_MEMORY, "work buffers of edgefm_prefill (%zu bytes)", prefill_buffer_bytes(ctx->shape, chunk));
+        }
+    }
+    PrefillModel pm{ctx->shape, ctx->layers.data(), ctx->embed, ctx->k_cache, ctx->v_cache, ctx->max_context, ctx->state};
+    ctx->prefill_launches = 0;
+    for (int i = 0; i < n_dense;) {
+        const int c = std::min(ctx->pf.chunk, n_dense - i);
+        int launches = 0;
+        if (const char *e = prefill_run(pm, &ctx->pf, tokens + i, c, ctx->cur_len, position + i, s, &launches)) {
+            cudaGetLastError();
+            return fail(ctx, EDGEFM_ERR_CUDA, "%s", e);
+        }
+        ctx->prefill_launches += launches;
+        ctx->cur_len += c;
+        i += c;
+    }
+    const edgefm_status st = edgefm_decode_step(ctx, tokens[n - 1], position + n - 1, stream, logits_out, next_token_out);
+    if (st == EDGEFM_OK) ctx->prefill_launches += ctx->launches_per_step;
+    return st;
+}
+
 edgefm_status edgefm_sync_length(edgefm_ctx *ctx, void *stream, int32_t *cur_len_host) {
     if (!ctx || !cur_len_host) return EDGEFM_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->device);
@@ -1170,6 +1214,11 @@ extern "C" edgefm_status edgefm_sync_status(edgefm_ctx *ctx, void *stream) {
     CUDA_TRY(ctx, cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
     StepState st;
     CUDA_TRY(ctx, cudaMemcpy(&st, where, sizeof st, cudaMemcpyDeviceToHost));
+    if (ctx && ctx->pf.chunk) {
+        int pe = 0;
+        CUDA_TRY(ctx, cudaMemcpy(&pe, ctx->pf.error, sizeof pe, cudaMemcpyDeviceToHost));
+        if (pe != 0) return fail(ctx, EDGEFM_ERR_TIMEOUT, "a bounded wait of a prefill contraction expired; the context must be destroyed");
+    }
     if (st.status != 0)
         return fail(ctx, EDGEFM_ERR_TIMEOUT, "device status %d (6 = a bounded wait expired, 100+ = self-check code) operands %d %d; "
                     "the context must be destroyed", st.status, st.pad[0], st.pad[1]);

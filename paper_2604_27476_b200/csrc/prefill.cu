@@ -1,0 +1,650 @@
+// Prompt processing for sm_100a: KV <- Prefill(x_1:T) (Eq. 3 of the paper).
+//
+// The T given tokens go through the layers together, so every projection is a dense [T x K] x [K x N] contraction:
+//   * prefill_gemm_kernel: one 128 x 128 (gate/up: 128 x 256) output tile per CTA.  A producer thread stages bf16 operand
+//     tiles in shared memory by TMA (128-byte swizzle), one thread issues tcgen05.mma with the fp32 accumulator in tensor
+//     memory, four warps read the accumulator back (tcgen05.ld) and apply the operator's epilogue:
+//       QKV      : + bias, rotate-half RoPE of q and k, q to the work buffer, k and v rows to the cache;
+//       O / down : added to the fp32 residual stream;
+//       gate/up  : SwiGLU, silu(gate) * up, to the bf16 activation buffer.
+//   * prefill_attention_kernel: causal attention of the T queries over the cache rows (prefix + the T new rows), online
+//     softmax, mma.sync tiles (under 6 % of the flops of a 2048-token prompt; not worth a second tcgen05 kernel).
+//   * rmsnorm / embedding kernels: one row per warp.
+// Every activation enters the tensor cores as TWO bf16 pieces (hi + lo, 16 mantissa bits; twice the multiplies, one load of
+// the weight tile), because single bf16 activations put the logits of a 28-layer model outside the step's tolerance
+// (measured: 3.6e-2 max-abs).  The residual stream stays fp32.
+// Every wait on an mbarrier is bounded; a wait that runs out raises PrefillBuffers::error and the CTA drains and returns.
+#include "prefill.h"
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "step_plan.h"
+
+namespace edgefm {
+namespace {
+
+// ---- PTX wrappers ----------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after `limit` polls or as soon as another thread of the CTA has given up.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, uint32_t limit) {
+    for (uint32_t i = 0; i < limit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 63u) == 63u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int x, int y, uint64_t *bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+                     smem_u32(dst)),
+                 "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+                 : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// D[tmem] (+)= A[smem] * B[smem]^T: 128 x N x 16, bf16 operands (both K-major), fp32 accumulator.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// The mbarrier receives one arrival when every tcgen05.mma issued so far by this thread has finished.
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// 32 lanes x 32 columns of fp32: thread i of the warp receives row (lane base + i), columns c .. c + 31.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float *v) {
+    uint32_t *r = reinterpret_cast<uint32_t *>(v);
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, "
+        "%18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major bf16 tile written by TMA with the 128-byte swizzle: rows of 64 elements
+// (128 bytes), groups of 8 rows 1024 bytes apart.  Fields: start address >> 4 (bits 0-13), leading byte offset >> 4 (16-29;
+// 1, unused with this swizzle), stride byte offset >> 4 (32-45) = 64, descriptor version 1 (46-47), layout 2 = 128-byte
+// swizzle (61-63).  A step of 16 elements along K inside the 128-byte row adds 32 bytes to the start address.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr) {
+    return static_cast<uint64_t>((smem_addr >> 4) & 0x3fffu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: fp32 accumulator (bits 4-5 = 1), A and B bf16 (7-9 = 1, 10-12 = 1), both K-major (15, 16 = 0),
+// N >> 3 (17-22), M >> 4 (24-28).
+__host__ __device__ constexpr uint32_t umma_idesc_bf16(int m, int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
+}
+
+__device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
+    return static_cast<uint32_t>(f32_to_bf16_bits(lo)) | (static_cast<uint32_t>(f32_to_bf16_bits(hi)) << 16);
+}
+
+// An fp32 activation as two bf16 pieces, hi = bf16(x), lo = bf16(x - hi): 16 mantissa bits enter the tensor cores (the
+// weights are bf16 exactly), so a contraction's operand rounding stays below 2^-17 relative.
+__device__ __forceinline__ void split2(float x, uint16_t &hi, uint16_t &lo) {
+    hi = f32_to_bf16_bits(x);
+    lo = f32_to_bf16_bits(x - bf16_bits_to_f32(hi));
+}
+__device__ __forceinline__ void split2x2(float a, float b, uint32_t &hi, uint32_t &lo) {
+    uint16_t ah, al, bh, bl;
+    split2(a, ah, al);
+    split2(b, bh, bl);
+    hi = static_cast<uint32_t>(ah) | (static_cast<uint32_t>(bh) << 16);
+    lo = static_cast<uint32_t>(al) | (static_cast<uint32_t>(bl) << 16);
+}
+
+// ---- small kernels -----------------------------------------------------------------------------------------------------
+// (cos, sin) of angle (position + t) * theta^(-2 j / d), evaluated in double and rounded once.
+__global__ void __launch_bounds__(256) prefill_rope_kernel(float2 *rope, int n, int half, int position, double theta) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n * half) return;
+    const int t = i / half, j = i % half;
+    const double inv = pow(theta, -static_cast<double>(j) / static_cast<double>(half));
+    double sn, cs;
+    sincos(static_cast<double>(position + t) * inv, &sn, &cs);
+    rope[i] = make_float2(static_cast<float>(cs), static_cast<float>(sn));
+}
+
+// One warp per row: y = x * rsqrt(mean(x^2) + eps) * w, stored as two bf16 planes (hi, lo; `plane` elements apart).  With `embed` the row is first fetched from the embedding
+// table (bf16 -> fp32) and written to the residual stream.  Thread 0 of the grid also records the new cache length.
+__global__ void __launch_bounds__(256) prefill_norm_kernel(float *resid, uint16_t *xn, size_t plane, const uint16_t *w, const uint16_t *embed,
+                                                           const int *tokens, int n, int H, float eps, StepState *st, int new_len,
+                                                           int new_pos) {
+    if (st && blockIdx.x == 0 && threadIdx.x == 0) {
+        st->cur_len = new_len;
+        st->next_position = new_pos;
+        st->status = 0;
+    }
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= n) return;
+    float *x = resid + static_cast<size_t>(row) * H;
+    if (embed) {
+        const uint16_t *e = embed + static_cast<size_t>(tokens[row]) * H;
+        for (int j = lane; j < H; j += 32) x[j] = bf16_bits_to_f32(e[j]);
+    }
+    float ss = 0.f;
+    for (int j = lane; j < H; j += 32) ss = fmaf(x[j], x[j], ss);
+    ss = warp_sum(ss);
+    const float r = rsqrtf(ss / static_cast<float>(H) + eps);
+    uint16_t *y = xn + static_cast<size_t>(row) * H;
+    for (int j = lane; j < H; j += 32) split2(x[j] * r * bf16_bits_to_f32(w[j]), y[j], y[plane + j]);
+}
+
+// ---- the contraction -------------------------------------------------------------------------------------------------------
+enum { EPI_QKV = 0, EPI_RESID = 1, EPI_SWIGLU = 2 };
+
+struct GemmArgs {
+    int M, N, K;              // rows (tokens), output features (gate/up: F, each of gate and up), reduction length
+    int *error;
+    // QKV
+    const uint16_t *bias;     // [N] or null
+    const float2 *rope;       // [M][d/2]
+    uint16_t *q_out;          // [2][..][nq d]: hi and lo planes
+    size_t q_plane;           // elements between the planes
+    uint16_t *k_rows, *v_rows;  // the layer's cache at the first new slot: + head * head_stride + row * d
+    int nq, nkv, d;
+    long long head_stride;
+    // O / down
+    float *resid;             // [M][N]
+    // gate/up
+    uint16_t *act;            // [2][..][N]: hi and lo planes
+    size_t act_plane;
+};
+
+constexpr int PF_BM = 128, PF_BK = 64;
+constexpr uint32_t PF_WAIT_LIMIT = 1u << 24;   // polls; far beyond any legitimate wait of a tile
+
+template <int EPI> struct GemmCfg {
+    static constexpr int BN = EPI == EPI_SWIGLU ? 256 : 128;
+    static constexpr int STAGES = EPI == EPI_SWIGLU ? 3 : 2;
+    static constexpr int A_BYTES = PF_BM * PF_BK * 2, B_BYTES = BN * PF_BK * 2;
+    static constexpr int STAGE_BYTES = 2 * A_BYTES + B_BYTES;          // A hi, A lo, B
+    static constexpr int SMEM = STAGES * STAGE_BYTES + 1024;   // + room to align the first stage to 1024 bytes
+};
+
+template <int EPI>
+__global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi,
+                                                           const __grid_constant__ CUtensorMap map_a_lo,
+                                                           const __grid_constant__ CUtensorMap map_b, const GemmArgs g) {
+    using C = GemmCfg<EPI>;
+    extern __shared__ uint8_t pf_dyn[];
+    __shared__ uint64_t full_bar[C::STAGES], empty_bar[C::STAGES], accum_bar;
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    uint8_t *tiles = pf_dyn + ((1024u - (smem_u32(pf_dyn) & 1023u)) & 1023u);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.y * PF_BM, n0 = blockIdx.x * 128;
+    const int KB = (g.K + PF_BK - 1) / PF_BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < C::STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        mbar_init(&accum_bar, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {   // the accumulator: BN columns of tensor memory, 128 lanes
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(C::BN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_slot;
+
+    if (warp == 0 && lane == 0) {            // producer: operand tiles by TMA
+        for (int kb = 0; kb < KB; ++kb) {
+            const int s = kb % C::STAGES;
+            if (kb >= C::STAGES && !mbar_wait(&empty_bar[s], ((kb / C::STAGES) - 1) & 1, &abort_flag, PF_WAIT_LIMIT)) break;
+            uint8_t *a = tiles + s * C::STAGE_BYTES, *b = a + 2 * C::A_BYTES;
+            mbar_expect_tx(&full_bar[s], C::STAGE_BYTES);
+            tma_load_2d(a, &map_a_hi, kb * PF_BK, m0, &full_bar[s]);
+            tma_load_2d(a + C::A_BYTES, &map_a_lo, kb * PF_BK, m0, &full_bar[s]);
+            tma_load_2d(b, &map_b, kb * PF_BK, n0, &full_bar[s]);
+            if (EPI == EPI_SWIGLU) tma_load_2d(b + 128 * PF_BK * 2, &map_b, kb * PF_BK, g.N + n0, &full_bar[s]);
+        }
+    } else if (warp == 1 && lane == 0) {     // issuer: per stage 4 tcgen05.mma (K = 16 each) for the hi pieces, 4 for the lo pieces
+        constexpr uint32_t idesc = umma_idesc_bf16(PF_BM, C::BN);
+        bool ok = true;
+        for (int kb = 0; kb < KB && ok; ++kb) {
+            const int s = kb % C::STAGES;
+            ok = mbar_wait(&full_bar[s], (kb / C::STAGES) & 1, &abort_flag, PF_WAIT_LIMIT);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t a = smem_u32(tiles + s * C::STAGE_BYTES), b = a + 2 * C::A_BYTES;
+            const uint64_t da = umma_desc_sw128(a), dl = umma_desc_sw128(a + C::A_BYTES), db = umma_desc_sw128(b);
+#pragma unroll
+            for (int k = 0; k < PF_BK / 16; ++k) umma_bf16(tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+#pragma unroll
+            for (int k = 0; k < PF_BK / 16; ++k) umma_bf16(tmem, dl + 2 * k, db + 2 * k, idesc, 1);
+            umma_commit(&empty_bar[s]);      // the stage is free again when these have read it
+        }
+        if (ok) umma_commit(&accum_bar);
+    } else if (warp >= 2) {                  // epilogue: warp w may read lanes 32 (w % 4) .. + 31 of tensor memory
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(&accum_bar, 0, &abort_flag, PF_WAIT_LIMIT));   // warp-uniform: tcgen05.ld is .aligned
+        tc_fence_after();
+        const int quarter = warp & 3;
+        const int row = m0 + quarter * 32 + lane;
+        const bool live = ok && row < g.M;
+        const uint32_t trow = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
+        if (ok) {
+            if (EPI == EPI_RESID) {
+                for (int c = 0; c < 4; ++c) {
+                    const int n = n0 + c * 32;
+                    if (n >= g.N) break;
+                    float v[32];
+                    tmem_ld32(trow + c * 32, v);
+                    tmem_ld_wait();
+                    if (live) {
+                        float4 *p = reinterpret_cast<float4 *>(g.resid + static_cast<size_t>(row) * g.N + n);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if (n + 4 * i + 3 < g.N) {
+                                float4 o = p[i];
+                                o.x += v[4 * i]; o.y += v[4 * i + 1]; o.z += v[4 * i + 2]; o.w += v[4 * i + 3];
+                                p[i] = o;
+                            }
+                    }
+                }
+            } else if (EPI == EPI_SWIGLU) {
+                for (int c = 0; c < 4; ++c) {
+                    const int n = n0 + c * 32;
+                    if (n >= g.N) break;
+                    float gt[32], up[32];
+                    tmem_ld32(trow + c * 32, gt);
+                    tmem_ld32(trow + 128 + c * 32, up);
+                    tmem_ld_wait();
+                    if (live) {
+                        uint4 *p = reinterpret_cast<uint4 *>(g.act + static_cast<size_t>(row) * g.N + n);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            if (n + 8 * i + 7 < g.N) {
+                                float o[8];
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) o[j] = gt[8 * i + j] / (1.f + __expf(-gt[8 * i + j])) * up[8 * i + j];
+                                uint4 hi, lo;
+                                split2x2(o[0], o[1], hi.x, lo.x); split2x2(o[2], o[3], hi.y, lo.y);
+                                split2x2(o[4], o[5], hi.z, lo.z); split2x2(o[6], o[7], hi.w, lo.w);
+                                p[i] = hi;
+                                *reinterpret_cast<uint4 *>(reinterpret_cast<uint16_t *>(p + i) + g.act_plane) = lo;
+                            }
+                    }
+                }
+            } else {   // EPI_QKV
+                const int half = g.d >> 1;
+                for (int off = 0; off < 128; off += g.d) {
+                    const int col0 = n0 + off;
+                    if (col0 >= g.N) break;
+                    const int head = col0 / g.d;
+                    if (head < g.nq + g.nkv) {   // q or k: rotate-half pairs (j, j + d/2)
+                        const bool is_q = head < g.nq;
+                        uint16_t *dst = is_q ? g.q_out + static_cast<size_t>(row) * g.nq * g.d + static_cast<size_t>(head) * g.d
+                                                    : g.k_rows + (head - g.nq) * g.head_stride + static_cast<size_t>(row) * g.d;
+                        for (int j0 = 0; j0 < half; j0 += 32) {
+                            float lo[32], hi[32];
+                            tmem_ld32(trow + off + j0, lo);
+                            tmem_ld32(trow + off + half + j0, hi);
+                            tmem_ld_wait();
+                            if (live) {
+                                const float2 *cs = g.rope + static_cast<size_t>(row) * half + j0;
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    float a[8], b[8];
+#pragma unroll
+                                    for (int j = 0; j < 8; ++j) {
+                                        const int e = 8 * i + j;
+                                        float x = lo[e], y = hi[e];
+                                        if (g.bias) {
+                                            x += bf16_bits_to_f32(g.bias[col0 + j0 + e]);
+                                            y += bf16_bits_to_f32(g.bias[col0 + half + j0 + e]);
+                                        }
+                                        const float2 t = cs[e];
+                                        a[j] = x * t.x - y * t.y;
+                                        b[j] = y * t.x + x * t.y;
+                                    }
+                                    uint4 ah, al, bh, bl;
+                                    split2x2(a[0], a[1], ah.x, al.x); split2x2(a[2], a[3], ah.y, al.y);
+                                    split2x2(a[4], a[5], ah.z, al.z); split2x2(a[6], a[7], ah.w, al.w);
+                                    split2x2(b[0], b[1], bh.x, bl.x); split2x2(b[2], b[3], bh.y, bl.y);
+                                    split2x2(b[4], b[5], bh.z, bl.z); split2x2(b[6], b[7], bh.w, bl.w);
+                                    *reinterpret_cast<uint4 *>(dst + j0 + 8 * i) = ah;          // k rows: the hi piece IS the bf16 row
+                                    *reinterpret_cast<uint4 *>(dst + half + j0 + 8 * i) = bh;
+                                    if (is_q) {                                                // queries keep both pieces
+                                        *reinterpret_cast<uint4 *>(dst + g.q_plane + j0 + 8 * i) = al;
+                                        *reinterpret_cast<uint4 *>(dst + g.q_plane + half + j0 + 8 * i) = bl;
+                                    }
+                                }
+                            }
+                        }
+                    } else {                     // v: bias only
+                        uint16_t *dst = g.v_rows + (head - g.nq - g.nkv) * g.head_stride + static_cast<size_t>(row) * g.d;
+                        for (int j0 = 0; j0 < g.d; j0 += 32) {
+                            float v[32];
+                            tmem_ld32(trow + off + j0, v);
+                            tmem_ld_wait();
+                            if (live) {
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    float o[8];
+#pragma unroll
+                                    for (int j = 0; j < 8; ++j)
+                                        o[j] = v[8 * i + j] + (g.bias ? bf16_bits_to_f32(g.bias[col0 + j0 + 8 * i + j]) : 0.f);
+                                    *reinterpret_cast<uint4 *>(dst + j0 + 8 * i) =
+                                        make_uint4(pack2_bf16(o[0], o[1]), pack2_bf16(o[2], o[3]), pack2_bf16(o[4], o[5]), pack2_bf16(o[6], o[7]));
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(C::BN) : "memory");
+    }
+    if (threadIdx.x == 0 && abort_flag) atomicExch(g.error, 1);
+}
+
+// ---- causal attention of the new queries over the cache ------------------------------------------------------------------
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_16816(float *c, const uint32_t *a, uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+
+// A [64][D] bf16 tile in shared memory; the 16-byte pieces of a row are permuted by the row's low three bits so that the
+// eight rows an ldmatrix touches fall into different banks.
+template <int D> __device__ __forceinline__ uint32_t tile_addr(uint32_t base, int row, int piece) {
+    return base + row * (D * 2) + ((piece ^ (row & 7)) << 4);
+}
+template <int D>
+__device__ __forceinline__ void load_rows(uint32_t base, const uint16_t *src, long long row_stride, int first, int last_valid, int tid) {
+    constexpr int PIECES = D / 8;
+    for (int i = tid; i < 64 * PIECES; i += 128) {
+        const int r = i / PIECES, c = i % PIECES;
+        const int row = min(first + r, last_valid);
+        cp_async16(tile_addr<D>(base, r, c), src + row * row_stride + c * 8);
+    }
+}
+
+// grid (ceil(T / 64), nq); 4 warps, 16 queries each.  Query t of the chunk sits in cache slot slot0 + t and sees the keys
+// 0 .. slot0 + t.  q: rotated queries [2][..][nq D] (hi and lo bf16 planes, `plane` elements apart); kc / vc: this layer's
+// cache, [nkv][max_context][D]; out: [2][..][nq D], again two planes.  Queries and probabilities enter the tensor cores as
+// two bf16 pieces each (the cache rows are bf16 exactly), sums are fp32.
+template <int D>
+__global__ void __launch_bounds__(128) prefill_attention_kernel(const uint16_t *q, const uint16_t *kc, const uint16_t *vc, uint16_t *out,
+                                                                size_t plane, int T, int slot0, int nq, int group, long long head_stride,
+                                                                float scale_log2) {
+    extern __shared__ __align__(128) uint8_t at_dyn[];
+    constexpr int TILE = 64 * D * 2;
+    const uint32_t sq = smem_u32(at_dyn), sk = sq + 2 * TILE, sv = sk + 2 * TILE;   // q hi, q lo, 2 x k, 2 x v
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gq = lane >> 2, tq = lane & 3;
+    const int t0 = (gridDim.x - 1 - blockIdx.x) * 64;     // long rows first
+    const int h = blockIdx.y, hk = h / group;
+    const uint16_t *kh = kc + hk * head_stride, *vh = vc + hk * head_stride;
+    const int last_key = slot0 + min(t0 + 63, T - 1);
+    const int nkb = last_key / 64 + 1;
+
+    load_rows<D>(sq, q + static_cast<size_t>(h) * D, static_cast<long long>(nq) * D, t0, T - 1, tid);
+    load_rows<D>(sq + TILE, q + plane + static_cast<size_t>(h) * D, static_cast<long long>(nq) * D, t0, T - 1, tid);
+    load_rows<D>(sk, kh, D, 0, last_key, tid);
+    load_rows<D>(sv, vh, D, 0, last_key, tid);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+
+    float o[D / 8][4];
+#pragma unroll
+    for (int i = 0; i < D / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    float mrow[2] = {-INFINITY, -INFINITY}, lrow[2] = {0.f, 0.f};
+    const int qi0 = slot0 + t0 + warp * 16 + gq;          // cache slot of this thread's first row; the second is + 8
+
+    for (int kb = 0; kb < nkb; ++kb) {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncthreads();
+        const uint32_t kbuf = sk + (kb & 1) * TILE, vbuf = sv + (kb & 1) * TILE;
+        if (kb + 1 < nkb) {
+            load_rows<D>(sk + ((kb + 1) & 1) * TILE, kh, D, (kb + 1) * 64, last_key, tid);
+            load_rows<D>(sv + ((kb + 1) & 1) * TILE, vh, D, (kb + 1) * 64, last_key, tid);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        }
+        float s[8][4];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+            uint32_t qh[4], ql[4];
+            ldsm_x4(tile_addr<D>(sq, warp * 16 + (lane & 15), ks * 2 + (lane >> 4)), qh[0], qh[1], qh[2], qh[3]);
+            ldsm_x4(tile_addr<D>(sq + TILE, warp * 16 + (lane & 15), ks * 2 + (lane >> 4)), ql[0], ql[1], ql[2], ql[3]);
+#pragma unroll
+            for (int np = 0; np < 4; ++np) {
+                uint32_t b0, b1, b2, b3;
+                ldsm_x4(tile_addr<D>(kbuf, np * 16 + (lane & 7) + ((lane >> 4) << 3), ks * 2 + ((lane >> 3) & 1)), b0, b1, b2, b3);
+                mma_16816(s[2 * np], qh, b0, b1);
+                mma_16816(s[2 * np + 1], qh, b2, b3);
+                mma_16816(s[2 * np], ql, b0, b1);
+                mma_16816(s[2 * np + 1], ql, b2, b3);
+            }
+        }
+        // causal mask, running maximum, probabilities
+        float mx[2] = {mrow[0], mrow[1]};
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int key = kb * 64 + nt * 8 + 2 * tq + (e & 1);
+                const int r = e >> 1;
+                if (key > qi0 + 8 * r) s[nt][e] = -INFINITY;
+                mx[r] = fmaxf(mx[r], s[nt][e]);
+            }
+        float alpha[2], sum[2] = {0.f, 0.f};
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
+            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
+            alpha[r] = exp2f((mrow[r] - mx[r]) * scale_log2);   // first block: exp2(-inf) = 0
+            mrow[r] = mx[r];
+        }
+        uint32_t pf[4][4], pl[4][4];
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) {
+            float p[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                p[e] = exp2f((s[nt][e] - mx[e >> 1]) * scale_log2);
+                sum[e >> 1] += p[e];
+            }
+            split2x2(p[0], p[1], pf[nt >> 1][(nt & 1) * 2], pl[nt >> 1][(nt & 1) * 2]);
+            split2x2(p[2], p[3], pf[nt >> 1][(nt & 1) * 2 + 1], pl[nt >> 1][(nt & 1) * 2 + 1]);
+        }
+#pragma unroll
+        for (int r = 0; r < 2; ++r) lrow[r] = lrow[r] * alpha[r] + sum[r];
+#pragma unroll
+        for (int i = 0; i < D / 8; ++i) { o[i][0] *= alpha[0]; o[i][1] *= alpha[0]; o[i][2] *= alpha[1]; o[i][3] *= alpha[1]; }
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+#pragma unroll
+            for (int dp = 0; dp < D / 16; ++dp) {
+                uint32_t b0, b1, b2, b3;
+                ldsm_x4_t(tile_addr<D>(vbuf, ks * 16 + (lane & 7) + (((lane >> 3) & 1) << 3), dp * 2 + (lane >> 4)), b0, b1, b2, b3);
+                mma_16816(o[2 * dp], pf[ks], b0, b1);
+                mma_16816(o[2 * dp + 1], pf[ks], b2, b3);
+                mma_16816(o[2 * dp], pl[ks], b0, b1);
+                mma_16816(o[2 * dp + 1], pl[ks], b2, b3);
+            }
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        lrow[r] += __shfl_xor_sync(0xffffffffu, lrow[r], 1);
+        lrow[r] += __shfl_xor_sync(0xffffffffu, lrow[r], 2);
+        const int t = t0 + warp * 16 + gq + 8 * r;
+        if (t < T) {
+            const float inv = 1.f / lrow[r];
+            uint32_t *dst = reinterpret_cast<uint32_t *>(out + static_cast<size_t>(t) * nq * D + static_cast<size_t>(h) * D);
+#pragma unroll
+            for (int i = 0; i < D / 8; ++i) {
+                uint32_t hi, lo;
+                split2x2(o[i][2 * r] * inv, o[i][2 * r + 1] * inv, hi, lo);
+                dst[i * 4 + tq] = hi;
+                dst[plane / 2 + i * 4 + tq] = lo;
+            }
+        }
+    }
+}
+
+// ---- host side ---------------------------------------------------------------------------------------------------------------
+// Map of a row-major bf16 [rows][K] matrix; a box is 128 rows x 64 columns (one 128-byte swizzled row each); rows and
+// columns outside the matrix read as zero.  (No multicast is used with these maps.)
+bool encode_operand_map(CUtensorMap *m, const void *base, long long rows, int K) {
+    TensorMapEncodeFn enc = tensor_map_encoder();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(K) * 2};
+    const cuuint32_t box[2] = {PF_BK, 128};
+    const cuuint32_t es[2] = {1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int EPI>
+const char *launch_gemm(const uint16_t *a, size_t a_plane, const void *w, long long w_rows, const GemmArgs &g, cudaStream_t s) {
+    CUtensorMap ma, ml, mb;
+    if (!encode_operand_map(&ma, a, g.M, g.K) || !encode_operand_map(&ml, a + a_plane, g.M, g.K) || !encode_operand_map(&mb, w, w_rows, g.K))
+        return "cuTensorMapEncodeTiled failed";
+    if (cudaFuncSetAttribute(prefill_gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, GemmCfg<EPI>::SMEM) != cudaSuccess)
+        return "cudaFuncSetAttribute failed";
+    const dim3 grid((g.N + 127) / 128, (g.M + PF_BM - 1) / PF_BM);
+    prefill_gemm_kernel<EPI><<<grid, 192, GemmCfg<EPI>::SMEM, s>>>(ma, ml, mb, g);
+    return cudaGetLastError() == cudaSuccess ? nullptr : "prefill GEMM launch failed";
+}
+
+template <int D>
+const char *launch_attention(const uint16_t *q, const uint16_t *kc, const uint16_t *vc, uint16_t *out, size_t plane, int T, int slot0, int nq, int group,
+                             long long head_stride, cudaStream_t s) {
+    constexpr int smem = 6 * 64 * D * 2;
+    if (cudaFuncSetAttribute(prefill_attention_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+        return "cudaFuncSetAttribute failed";
+    const float scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(D)));
+    prefill_attention_kernel<D><<<dim3((T + 63) / 64, nq), 128, smem, s>>>(q, kc, vc, out, plane, T, slot0, nq, group, head_stride, scale_log2);
+    return cudaGetLastError() == cudaSuccess ? nullptr : "prefill attention launch failed";
+}
+
+}  // namespace
+
+size_t prefill_buffer_bytes(const edgefm_shape &sh, int chunk) {
+    const size_t c = static_cast<size_t>(chunk), qd = static_cast<size_t>(sh.n_q_heads) * sh.head_dim;
+    return c * sh.hidden * 4 + c * sh.hidden * 4 + 2 * c * qd * 4 + c * sh.ffn * 4 + c * (sh.head_dim / 2) * 8 + c * 4 + 256;
+}
+
+cudaError_t prefill_alloc(PrefillBuffers *b, const edgefm_shape &sh, int chunk) {
+    const size_t c = static_cast<size_t>(chunk), qd = static_cast<size_t>(sh.n_q_heads) * sh.head_dim;
+    cudaError_t e;
+    if ((e = cudaMalloc(&b->resid, c * sh.hidden * 4)) != cudaSuccess) return e;
+    if ((e = cudaMalloc(&b->xn, c * sh.hidden * 4)) != cudaSuccess) return e;
+    if ((e = cudaMalloc(&b->q, c * qd * 4)) != cudaSuccess) return e;
+    if ((e = cudaMalloc(&b->attn, c * qd * 4)) != cudaSuccess) return e;
+    if ((e = cudaMalloc(&b->act, c * sh.ffn * 4)) != cudaSuccess) return e;
+    if ((e = cudaMalloc(&b->rope, c * (sh.head_dim / 2) * sizeof(float2))) != cudaSuccess) return e;
+    if ((e = cudaMalloc(&b->tokens, c * 4)) != cudaSuccess) return e;
+    if ((e = cudaMalloc(&b->error, 4)) != cudaSuccess) return e;
+    if ((e = cudaMemset(b->error, 0, 4)) != cudaSuccess) return e;
+    b->chunk = chunk;
+    return cudaSuccess;
+}
+
+void prefill_free(PrefillBuffers *b) {
+    cudaFree(b->resid); cudaFree(b->xn); cudaFree(b->q); cudaFree(b->attn); cudaFree(b->act); cudaFree(b->rope);
+    cudaFree(b->tokens); cudaFree(b->error);
+    *b = PrefillBuffers{};
+}
+
+const char *prefill_run(const PrefillModel &m, PrefillBuffers *b, const int32_t *tokens, int n, int slot0, int position, cudaStream_t s,
+                        int *launches) {
+    const edgefm_shape &sh = m.shape;
+    const int H = sh.hidden, F = sh.ffn, d = sh.head_dim, nq = sh.n_q_heads, nkv = sh.n_kv_heads, qd = nq * d;
+    const int n_qkv = (nq + 2 * nkv) * d;
+    const long long head_stride = static_cast<long long>(m.max_context) * d;
+    const size_t cap = static_cast<size_t>(b->chunk), x_plane = cap * H, q_plane = cap * qd, f_plane = cap * F;   // hi / lo planes
+    int count = 0;
+    if (cudaMemcpyAsync(b->tokens, tokens, static_cast<size_t>(n) * 4, cudaMemcpyHostToDevice, s) != cudaSuccess) return "token upload failed";
+    prefill_rope_kernel<<<(n * (d / 2) + 255) / 256, 256, 0, s>>>(b->rope, n, d / 2, position, static_cast<double>(sh.rope_theta));
+    const int norm_grid = (n + 7) / 8;
+    prefill_norm_kernel<<<norm_grid, 256, 0, s>>>(b->resid, b->xn, x_plane, static_cast<const uint16_t *>(m.layers[0].input_norm),
+                                                  static_cast<const uint16_t *>(m.embed), b->tokens, n, H, sh.rms_eps, m.state,
+                                                  slot0 + n, position + n);
+    count += 2;
+    for (int l = 0; l < sh.n_layers; ++l) {
+        const edgefm_layer_weights &w = m.layers[l];
+        uint16_t *kc = m.k_cache + static_cast<size_t>(l) * nkv * head_stride, *vc = m.v_cache + static_cast<size_t>(l) * nkv * head_stride;
+        GemmArgs g{};
+        g.M = n; g.error = b->error;
+        g.N = n_qkv; g.K = H;
+        g.bias = sh.qkv_bias ? static_cast<const uint16_t *>(w.bqkv) : nullptr;
+        g.rope = b->rope; g.q_out = b->q; g.q_plane = q_plane;
+        g.k_rows = kc + static_cast<size_t>(slot0) * d; g.v_rows = vc + static_cast<size_t>(slot0) * d;
+        g.nq = nq; g.nkv = nkv; g.d = d; g.head_stride = head_stride;
+        if (const char *e = launch_gemm<EPI_QKV>(b->xn, x_plane, w.wqkv, n_qkv, g, s)) return e;
+        ++count;
+        if (l == sh.n_layers - 1) break;   // the rest of the last layer feeds nothing that is kept
+        const char *e = d == 64 ? launch_attention<64>(b->q, kc, vc, b->attn, q_plane, n, slot0, nq, nq / nkv, head_stride, s)
+                                : launch_attention<128>(b->q, kc, vc, b->attn, q_plane, n, slot0, nq, nq / nkv, head_stride, s);
+        if (e) return e;
+        g.N = H; g.K = qd; g.resid = b->resid;
+        if ((e = launch_gemm<EPI_RESID>(b->attn, q_plane, w.wo, H, g, s))) return e;
+        prefill_norm_kernel<<<norm_grid, 256, 0, s>>>(b->resid, b->xn, x_plane, static_cast<const uint16_t *>(w.post_norm), nullptr, nullptr, n, H,
+                                                      sh.rms_eps, nullptr, 0, 0);
+        g.N = F; g.K = H; g.act = b->act; g.act_plane = f_plane;
+        if ((e = launch_gemm<EPI_SWIGLU>(b->xn, x_plane, w.w_gate_up, 2LL * F, g, s))) return e;
+        g.N = H; g.K = F;
+        if ((e = launch_gemm<EPI_RESID>(b->act, f_plane, w.w_down, H, g, s))) return e;
+        prefill_norm_kernel<<<norm_grid, 256, 0, s>>>(b->resid, b->xn, x_plane, static_cast<const uint16_t *>(m.layers[l + 1].input_norm), nullptr,
+                                                      nullptr, n, H, sh.rms_eps, nullptr, 0, 0);
+        count += 6;
+    }
+    if (cudaGetLastError() != cudaSuccess) return "prefill kernel launch failed";
+    if (launches) *launches = count;
+    return nullptr;
+}
+
+}  // namespace edgefm

@@ -1,0 +1,50 @@
+// Prompt processing (Eq. 3 of the paper: KV <- Prefill(x_1:T)) as dense contractions on the 5th-generation tensor cores.
+// Host-side interface between the C ABI (edgefm.cu) and the kernels of prefill.cu.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "common.cuh"
+#include "../../include/edgefm.h"
+
+namespace edgefm {
+
+constexpr int PF_CHUNK_MAX = 2048;   // tokens per pass over the layers (longer prompts take several passes)
+
+// Work buffers of one pass, owned by the context, allocated at the first prefill call.
+struct PrefillBuffers {
+    int chunk = 0;               // rows the buffers hold
+    float *resid = nullptr;      // residual stream fp32 [chunk][H]
+    // activations as two bf16 planes each (hi = bf16(x), lo = bf16(x - hi)):
+    uint16_t *xn = nullptr;      // normalised activations [2][chunk][H]
+    uint16_t *q = nullptr;       // rotated queries [2][chunk][nq d]
+    uint16_t *attn = nullptr;    // attention output [2][chunk][nq d]
+    uint16_t *act = nullptr;     // SwiGLU output [2][chunk][F]
+    float2 *rope = nullptr;      // (cos, sin) of the chunk's positions, [chunk][d/2]
+    int *tokens = nullptr;       // device copy of the chunk's token ids
+    int *error = nullptr;        // device word: non-zero when a bounded wait of a GEMM ran out
+};
+
+struct PrefillModel {
+    edgefm_shape shape;
+    const edgefm_layer_weights *layers;   // host array
+    const void *embed;
+    uint16_t *k_cache, *v_cache;          // bf16 [L][nkv][max_context][d]
+    int max_context;
+    StepState *state;
+};
+
+// Bytes the work buffers of a pass over `chunk` tokens take.
+size_t prefill_buffer_bytes(const edgefm_shape &sh, int chunk);
+// Allocate / free.  Returns a CUDA error.
+cudaError_t prefill_alloc(PrefillBuffers *b, const edgefm_shape &sh, int chunk);
+void prefill_free(PrefillBuffers *b);
+
+// Enqueue the layers for `n` tokens (host ids) whose cache rows go to slots [slot0, slot0 + n) at rotary positions
+// position .. position + n - 1.  Every layer's K and V rows are written; the last layer's attention and MLP are skipped
+// (their result would only feed an output layer nobody reads).  Sets the device state to cache length slot0 + n.
+// Returns nullptr or a message.
+const char *prefill_run(const PrefillModel &m, PrefillBuffers *b, const int32_t *tokens, int n, int slot0, int position,
+                        cudaStream_t stream, int *launches);
+
+}  // namespace edgefm
