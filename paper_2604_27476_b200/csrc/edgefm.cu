@@ -829,7 +829,7 @@ edgefm_status edgefm_prefill(edgefm_ctx *ctx, const int32_t *tokens, int32_t n, 
             return fail(ctx, EDGEFM_ERR_OUT_OF_MEMORY, "work buffers of edgefm_prefill (%zu bytes)", prefill_buffer_bytes(ctx->shape, chunk));
         }
     }
-    PrefillModel pm{ctx->shape, ctx->layers.data(), ctx->embed, ctx->k_cache, ctx->v_cache, ctx->max_context, ctx->state};
+    PrefillModel pm{ctx->shape, ctx->layers.data(), ctx->embed, ctx->k_cache, ctx->v_cache, ctx->max_context, ctx->state, ctx->num_sms};
     ctx->prefill_launches = 0;
     for (int i = 0; i < n_dense;) {
         const int c = std::min(ctx->pf.chunk, n_dense - i);

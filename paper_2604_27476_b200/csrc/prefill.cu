@@ -149,16 +149,38 @@ __global__ void __launch_bounds__(256) prefill_norm_kernel(float *resid, uint16_
     const int lane = threadIdx.x & 31;
     if (row >= n) return;
     float *x = resid + static_cast<size_t>(row) * H;
-    if (embed) {
-        const uint16_t *e = embed + static_cast<size_t>(tokens[row]) * H;
-        for (int j = lane; j < H; j += 32) x[j] = bf16_bits_to_f32(e[j]);
-    }
+    uint16_t *y = xn + static_cast<size_t>(row) * H;
+    // H is a multiple of 8: eight values per lane and round, 16- and 32-byte accesses
+    const uint16_t *e = embed ? embed + static_cast<size_t>(tokens[row]) * H : nullptr;
     float ss = 0.f;
-    for (int j = lane; j < H; j += 32) ss = fmaf(x[j], x[j], ss);
+    for (int j = lane * 8; j < H; j += 256) {
+        float v[8];
+        if (e) {
+            const uint4 b = *reinterpret_cast<const uint4 *>(e + j);
+            v[0] = bf16lo(b.x); v[1] = bf16hi(b.x); v[2] = bf16lo(b.y); v[3] = bf16hi(b.y);
+            v[4] = bf16lo(b.z); v[5] = bf16hi(b.z); v[6] = bf16lo(b.w); v[7] = bf16hi(b.w);
+            *reinterpret_cast<float4 *>(x + j) = make_float4(v[0], v[1], v[2], v[3]);
+            *reinterpret_cast<float4 *>(x + j + 4) = make_float4(v[4], v[5], v[6], v[7]);
+        } else {
+            const float4 a = *reinterpret_cast<const float4 *>(x + j), c = *reinterpret_cast<const float4 *>(x + j + 4);
+            v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = c.x; v[5] = c.y; v[6] = c.z; v[7] = c.w;
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) ss = fmaf(v[i], v[i], ss);
+    }
     ss = warp_sum(ss);
     const float r = rsqrtf(ss / static_cast<float>(H) + eps);
-    uint16_t *y = xn + static_cast<size_t>(row) * H;
-    for (int j = lane; j < H; j += 32) split2(x[j] * r * bf16_bits_to_f32(w[j]), y[j], y[plane + j]);
+    for (int j = lane * 8; j < H; j += 256) {
+        const float4 a = *reinterpret_cast<const float4 *>(x + j), c = *reinterpret_cast<const float4 *>(x + j + 4);
+        const uint4 wb = *reinterpret_cast<const uint4 *>(w + j);
+        uint4 hi, lo;
+        split2x2(a.x * r * bf16lo(wb.x), a.y * r * bf16hi(wb.x), hi.x, lo.x);
+        split2x2(a.z * r * bf16lo(wb.y), a.w * r * bf16hi(wb.y), hi.y, lo.y);
+        split2x2(c.x * r * bf16lo(wb.z), c.y * r * bf16hi(wb.z), hi.z, lo.z);
+        split2x2(c.z * r * bf16lo(wb.w), c.w * r * bf16hi(wb.w), hi.w, lo.w);
+        *reinterpret_cast<uint4 *>(y + j) = hi;
+        *reinterpret_cast<uint4 *>(y + plane + j) = lo;
+    }
 }
 
 // ---- the contraction -------------------------------------------------------------------------------------------------------
@@ -185,26 +207,34 @@ struct GemmArgs {
 constexpr int PF_BM = 128, PF_BK = 64;
 constexpr uint32_t PF_WAIT_LIMIT = 1u << 24;   // polls; far beyond any legitimate wait of a tile
 
-template <int EPI> struct GemmCfg {
-    static constexpr int BN = EPI == EPI_SWIGLU ? 256 : 128;
-    static constexpr int STAGES = EPI == EPI_SWIGLU ? 3 : 2;
+// Tile shapes.  PF_NARROW: 128 output columns, 2 stages (97 KB: two CTAs per SM, one's epilogue under the other's main
+// loop).  PF_NARROW_DEEP: the same with 4 stages, one CTA per SM, for grids that leave SMs with a single CTA anyway (a lone CTA
+// needs the depth to cover the latency of its operand loads).  PF_WIDE: 256 output columns, 3 stages: per k-block 64 KB of
+// operands feed twice the multiplies of a narrow tile's 48 KB, which matters because operand delivery from L2, not the
+// tensor pipe, bounds the narrow tiles.  Gate/up always runs wide: 128 gate columns and their 128 up partners.
+enum { PF_NARROW = 0, PF_NARROW_DEEP = 1, PF_WIDE = 2 };
+template <int SHAPE> struct GemmCfg {
+    static constexpr int BN = SHAPE == PF_WIDE ? 256 : 128;
+    static constexpr int STAGES = SHAPE == PF_WIDE ? 3 : (SHAPE == PF_NARROW_DEEP ? 4 : 2);
     static constexpr int A_BYTES = PF_BM * PF_BK * 2, B_BYTES = BN * PF_BK * 2;
     static constexpr int STAGE_BYTES = 2 * A_BYTES + B_BYTES;          // A hi, A lo, B
     static constexpr int SMEM = STAGES * STAGE_BYTES + 1024;   // + room to align the first stage to 1024 bytes
 };
 
-template <int EPI>
+template <int EPI, int SHAPE>
 __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant__ CUtensorMap map_a_hi,
                                                            const __grid_constant__ CUtensorMap map_a_lo,
                                                            const __grid_constant__ CUtensorMap map_b, const GemmArgs g) {
-    using C = GemmCfg<EPI>;
+    using C = GemmCfg<SHAPE>;
+    static_assert(EPI != EPI_SWIGLU || SHAPE == PF_WIDE, "gate and up share one accumulator");
+    constexpr int N_STEP = EPI == EPI_SWIGLU ? 128 : C::BN;   // output columns (of g.N) a CTA covers
     extern __shared__ uint8_t pf_dyn[];
     __shared__ uint64_t full_bar[C::STAGES], empty_bar[C::STAGES], accum_bar;
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     uint8_t *tiles = pf_dyn + ((1024u - (smem_u32(pf_dyn) & 1023u)) & 1023u);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.y * PF_BM, n0 = blockIdx.x * 128;
+    const int m0 = blockIdx.y * PF_BM, n0 = blockIdx.x * N_STEP;
     const int KB = (g.K + PF_BK - 1) / PF_BK;
 
     if (threadIdx.x == 0) {
@@ -231,7 +261,7 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
             tma_load_2d(a, &map_a_hi, kb * PF_BK, m0, &full_bar[s]);
             tma_load_2d(a + C::A_BYTES, &map_a_lo, kb * PF_BK, m0, &full_bar[s]);
             tma_load_2d(b, &map_b, kb * PF_BK, n0, &full_bar[s]);
-            if (EPI == EPI_SWIGLU) tma_load_2d(b + 128 * PF_BK * 2, &map_b, kb * PF_BK, g.N + n0, &full_bar[s]);
+            if (C::BN == 256) tma_load_2d(b + 128 * PF_BK * 2, &map_b, kb * PF_BK, (EPI == EPI_SWIGLU ? g.N : 128) + n0, &full_bar[s]);
         }
     } else if (warp == 1 && lane == 0) {     // issuer: per stage 4 tcgen05.mma (K = 16 each) for the hi pieces, 4 for the lo pieces
         constexpr uint32_t idesc = umma_idesc_bf16(PF_BM, C::BN);
@@ -259,7 +289,7 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
         const uint32_t trow = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
         if (ok) {
             if (EPI == EPI_RESID) {
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < N_STEP / 32; ++c) {
                     const int n = n0 + c * 32;
                     if (n >= g.N) break;
                     float v[32];
@@ -302,7 +332,7 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
                 }
             } else {   // EPI_QKV
                 const int half = g.d >> 1;
-                for (int off = 0; off < 128; off += g.d) {
+                for (int off = 0; off < N_STEP; off += g.d) {
                     const int col0 = n0 + off;
                     if (col0 >= g.N) break;
                     const int head = col0 / g.d;
@@ -547,16 +577,33 @@ bool encode_operand_map(CUtensorMap *m, const void *base, long long rows, int K)
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+template <int EPI, int SHAPE>
+const char *launch_gemm_cfg(const CUtensorMap &ma, const CUtensorMap &ml, const CUtensorMap &mb, const GemmArgs &g, cudaStream_t s) {
+    using C = GemmCfg<SHAPE>;
+    if (cudaFuncSetAttribute(prefill_gemm_kernel<EPI, SHAPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess)
+        return "cudaFuncSetAttribute failed";
+    const int n_step = EPI == EPI_SWIGLU ? 128 : C::BN;
+    const dim3 grid((g.N + n_step - 1) / n_step, (g.M + PF_BM - 1) / PF_BM);
+    prefill_gemm_kernel<EPI, SHAPE><<<grid, 192, C::SMEM, s>>>(ma, ml, mb, g);
+    return cudaGetLastError() == cudaSuccess ? nullptr : "prefill GEMM launch failed";
+}
+
+// Shape choice: wide tiles when they still give at least 60 % of the SMs a tile (96 of 148 for the 1.5B down projection at
+// 2048 tokens: 115 -> 7x us); otherwise narrow tiles, deep when no SM would get a second CTA.
 template <int EPI>
-const char *launch_gemm(const uint16_t *a, size_t a_plane, const void *w, long long w_rows, const GemmArgs &g, cudaStream_t s) {
+const char *launch_gemm(const uint16_t *a, size_t a_plane, const void *w, long long w_rows, const GemmArgs &g, int num_sms, cudaStream_t s) {
     CUtensorMap ma, ml, mb;
     if (!encode_operand_map(&ma, a, g.M, g.K) || !encode_operand_map(&ml, a + a_plane, g.M, g.K) || !encode_operand_map(&mb, w, w_rows, g.K))
         return "cuTensorMapEncodeTiled failed";
-    if (cudaFuncSetAttribute(prefill_gemm_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, GemmCfg<EPI>::SMEM) != cudaSuccess)
-        return "cudaFuncSetAttribute failed";
-    const dim3 grid((g.N + 127) / 128, (g.M + PF_BM - 1) / PF_BM);
-    prefill_gemm_kernel<EPI><<<grid, 192, GemmCfg<EPI>::SMEM, s>>>(ma, ml, mb, g);
-    return cudaGetLastError() == cudaSuccess ? nullptr : "prefill GEMM launch failed";
+    const int m_tiles = (g.M + PF_BM - 1) / PF_BM;
+    if constexpr (EPI == EPI_SWIGLU) {
+        return launch_gemm_cfg<EPI, PF_WIDE>(ma, ml, mb, g, s);
+    } else {
+        const int wide = ((g.N + 255) / 256) * m_tiles, narrow = ((g.N + 127) / 128) * m_tiles;
+        if (wide * 10 >= num_sms * 6) return launch_gemm_cfg<EPI, PF_WIDE>(ma, ml, mb, g, s);
+        if (narrow <= num_sms) return launch_gemm_cfg<EPI, PF_NARROW_DEEP>(ma, ml, mb, g, s);
+        return launch_gemm_cfg<EPI, PF_NARROW>(ma, ml, mb, g, s);
+    }
 }
 
 template <int D>
@@ -624,20 +671,20 @@ const char *prefill_run(const PrefillModel &m, PrefillBuffers *b, const int32_t 
         g.rope = b->rope; g.q_out = b->q; g.q_plane = q_plane;
         g.k_rows = kc + static_cast<size_t>(slot0) * d; g.v_rows = vc + static_cast<size_t>(slot0) * d;
         g.nq = nq; g.nkv = nkv; g.d = d; g.head_stride = head_stride;
-        if (const char *e = launch_gemm<EPI_QKV>(b->xn, x_plane, w.wqkv, n_qkv, g, s)) return e;
+        if (const char *e = launch_gemm<EPI_QKV>(b->xn, x_plane, w.wqkv, n_qkv, g, m.num_sms, s)) return e;
         ++count;
         if (l == sh.n_layers - 1) break;   // the rest of the last layer feeds nothing that is kept
         const char *e = d == 64 ? launch_attention<64>(b->q, kc, vc, b->attn, q_plane, n, slot0, nq, nq / nkv, head_stride, s)
                                 : launch_attention<128>(b->q, kc, vc, b->attn, q_plane, n, slot0, nq, nq / nkv, head_stride, s);
         if (e) return e;
         g.N = H; g.K = qd; g.resid = b->resid;
-        if ((e = launch_gemm<EPI_RESID>(b->attn, q_plane, w.wo, H, g, s))) return e;
+        if ((e = launch_gemm<EPI_RESID>(b->attn, q_plane, w.wo, H, g, m.num_sms, s))) return e;
         prefill_norm_kernel<<<norm_grid, 256, 0, s>>>(b->resid, b->xn, x_plane, static_cast<const uint16_t *>(w.post_norm), nullptr, nullptr, n, H,
                                                       sh.rms_eps, nullptr, 0, 0);
         g.N = F; g.K = H; g.act = b->act; g.act_plane = f_plane;
-        if ((e = launch_gemm<EPI_SWIGLU>(b->xn, x_plane, w.w_gate_up, 2LL * F, g, s))) return e;
+        if ((e = launch_gemm<EPI_SWIGLU>(b->xn, x_plane, w.w_gate_up, 2LL * F, g, m.num_sms, s))) return e;
         g.N = H; g.K = F;
-        if ((e = launch_gemm<EPI_RESID>(b->act, f_plane, w.w_down, H, g, s))) return e;
+        if ((e = launch_gemm<EPI_RESID>(b->act, f_plane, w.w_down, H, g, m.num_sms, s))) return e;
         prefill_norm_kernel<<<norm_grid, 256, 0, s>>>(b->resid, b->xn, x_plane, static_cast<const uint16_t *>(m.layers[l + 1].input_norm), nullptr,
                                                       nullptr, n, H, sh.rms_eps, nullptr, 0, 0);
         count += 6;

@@ -32,6 +32,7 @@ struct PrefillModel {
     uint16_t *k_cache, *v_cache;          // bf16 [L][nkv][max_context][d]
     int max_context;
     StepState *state;
+    int num_sms;
 };
 
 // Bytes the work buffers of a pass over `chunk` tokens take.
