@@ -33,6 +33,9 @@ __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -207,15 +210,15 @@ struct GemmArgs {
 constexpr int PF_BM = 128, PF_BK = 64;
 constexpr uint32_t PF_WAIT_LIMIT = 1u << 24;   // polls; far beyond any legitimate wait of a tile
 
-// Tile shapes.  PF_NARROW: 128 output columns, 2 stages (97 KB: two CTAs per SM, one's epilogue under the other's main
-// loop).  PF_NARROW_DEEP: the same with 4 stages, one CTA per SM, for grids that leave SMs with a single CTA anyway (a lone CTA
-// needs the depth to cover the latency of its operand loads).  PF_WIDE: 256 output columns, 3 stages: per k-block 64 KB of
-// operands feed twice the multiplies of a narrow tile's 48 KB, which matters because operand delivery from L2, not the
-// tensor pipe, bounds the narrow tiles.  Gate/up always runs wide: 128 gate columns and their 128 up partners.
-enum { PF_NARROW = 0, PF_NARROW_DEEP = 1, PF_WIDE = 2 };
+// Tile shapes.  PF_NARROW: 128 output columns, 4 stages of 48 KB.  PF_WIDE: 256 output columns, 3 stages of 64 KB: per k-block
+// 64 KB of operands feed twice the multiplies of a narrow tile's 48 KB, which matters because operand delivery from L2, not
+// the tensor pipe, bounds the narrow tiles.  Gate/up always runs wide: 128 gate columns and their 128 up partners.
+// The kernel is persistent (one CTA per SM, tiles dealt round-robin, neighbours sharing a weight tile) with TWO accumulators
+// in tensor memory, so that the epilogue of a tile runs under the main loop of the next.
+enum { PF_NARROW = 0, PF_WIDE = 2 };
 template <int SHAPE> struct GemmCfg {
     static constexpr int BN = SHAPE == PF_WIDE ? 256 : 128;
-    static constexpr int STAGES = SHAPE == PF_WIDE ? 3 : (SHAPE == PF_NARROW_DEEP ? 4 : 2);
+    static constexpr int STAGES = SHAPE == PF_WIDE ? 3 : 4;
     static constexpr int A_BYTES = PF_BM * PF_BK * 2, B_BYTES = BN * PF_BK * 2;
     static constexpr int STAGE_BYTES = 2 * A_BYTES + B_BYTES;          // A hi, A lo, B
     static constexpr int SMEM = STAGES * STAGE_BYTES + 1024;   // + room to align the first stage to 1024 bytes
@@ -229,22 +232,23 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
     static_assert(EPI != EPI_SWIGLU || SHAPE == PF_WIDE, "gate and up share one accumulator");
     constexpr int N_STEP = EPI == EPI_SWIGLU ? 128 : C::BN;   // output columns (of g.N) a CTA covers
     extern __shared__ uint8_t pf_dyn[];
-    __shared__ uint64_t full_bar[C::STAGES], empty_bar[C::STAGES], accum_bar;
+    __shared__ uint64_t full_bar[C::STAGES], empty_bar[C::STAGES], acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     uint8_t *tiles = pf_dyn + ((1024u - (smem_u32(pf_dyn) & 1023u)) & 1023u);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.y * PF_BM, n0 = blockIdx.x * N_STEP;
+    const int m_tiles = (g.M + PF_BM - 1) / PF_BM, n_tiles = (g.N + N_STEP - 1) / N_STEP;
+    const int my_tiles = (m_tiles * n_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
     const int KB = (g.K + PF_BK - 1) / PF_BK;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        mbar_init(&accum_bar, 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 4); }
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {   // the accumulator: BN columns of tensor memory, 128 lanes
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(C::BN) : "memory");
+    if (warp == 1) {   // two accumulators: 2 BN columns of tensor memory, 128 lanes
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(2 * C::BN) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -253,41 +257,55 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
     const uint32_t tmem = tmem_slot;
 
     if (warp == 0 && lane == 0) {            // producer: operand tiles by TMA
-        for (int kb = 0; kb < KB; ++kb) {
-            const int s = kb % C::STAGES;
-            if (kb >= C::STAGES && !mbar_wait(&empty_bar[s], ((kb / C::STAGES) - 1) & 1, &abort_flag, PF_WAIT_LIMIT)) break;
+        bool ok = true;
+        for (int i = 0, it = 0; i < my_tiles && ok; ++i) {
+          const int tile = blockIdx.x + i * gridDim.x, m0 = (tile % m_tiles) * PF_BM, n0 = (tile / m_tiles) * N_STEP;
+          for (int kb = 0; kb < KB; ++kb, ++it) {
+            const int s = it % C::STAGES;
+            if (it >= C::STAGES && !mbar_wait(&empty_bar[s], ((it / C::STAGES) - 1) & 1, &abort_flag, PF_WAIT_LIMIT)) { ok = false; break; }
             uint8_t *a = tiles + s * C::STAGE_BYTES, *b = a + 2 * C::A_BYTES;
             mbar_expect_tx(&full_bar[s], C::STAGE_BYTES);
             tma_load_2d(a, &map_a_hi, kb * PF_BK, m0, &full_bar[s]);
             tma_load_2d(a + C::A_BYTES, &map_a_lo, kb * PF_BK, m0, &full_bar[s]);
             tma_load_2d(b, &map_b, kb * PF_BK, n0, &full_bar[s]);
             if (C::BN == 256) tma_load_2d(b + 128 * PF_BK * 2, &map_b, kb * PF_BK, (EPI == EPI_SWIGLU ? g.N : 128) + n0, &full_bar[s]);
+          }
         }
     } else if (warp == 1 && lane == 0) {     // issuer: per stage 4 tcgen05.mma (K = 16 each) for the hi pieces, 4 for the lo pieces
         constexpr uint32_t idesc = umma_idesc_bf16(PF_BM, C::BN);
         bool ok = true;
-        for (int kb = 0; kb < KB && ok; ++kb) {
-            const int s = kb % C::STAGES;
-            ok = mbar_wait(&full_bar[s], (kb / C::STAGES) & 1, &abort_flag, PF_WAIT_LIMIT);
+        for (int i = 0, it = 0; i < my_tiles && ok; ++i) {
+          const int buf = i & 1;
+          const uint32_t acc = tmem + buf * C::BN;
+          if (i >= 2) ok = mbar_wait(&acc_empty[buf], ((i >> 1) - 1) & 1, &abort_flag, PF_WAIT_LIMIT);   // its epilogue has read it
+          if (!ok) break;
+          tc_fence_after();
+          for (int kb = 0; kb < KB; ++kb, ++it) {
+            const int s = it % C::STAGES;
+            ok = mbar_wait(&full_bar[s], (it / C::STAGES) & 1, &abort_flag, PF_WAIT_LIMIT);
             if (!ok) break;
             tc_fence_after();
             const uint32_t a = smem_u32(tiles + s * C::STAGE_BYTES), b = a + 2 * C::A_BYTES;
             const uint64_t da = umma_desc_sw128(a), dl = umma_desc_sw128(a + C::A_BYTES), db = umma_desc_sw128(b);
 #pragma unroll
-            for (int k = 0; k < PF_BK / 16; ++k) umma_bf16(tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+            for (int k = 0; k < PF_BK / 16; ++k) umma_bf16(acc, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
 #pragma unroll
-            for (int k = 0; k < PF_BK / 16; ++k) umma_bf16(tmem, dl + 2 * k, db + 2 * k, idesc, 1);
+            for (int k = 0; k < PF_BK / 16; ++k) umma_bf16(acc, dl + 2 * k, db + 2 * k, idesc, 1);
             umma_commit(&empty_bar[s]);      // the stage is free again when these have read it
+          }
+          if (ok) umma_commit(&acc_full[buf]);
         }
-        if (ok) umma_commit(&accum_bar);
     } else if (warp >= 2) {                  // epilogue: warp w may read lanes 32 (w % 4) .. + 31 of tensor memory
-        const bool ok = __all_sync(0xffffffffu, mbar_wait(&accum_bar, 0, &abort_flag, PF_WAIT_LIMIT));   // warp-uniform: tcgen05.ld is .aligned
+      const int quarter = warp & 3;
+      for (int i = 0; i < my_tiles; ++i) {
+        const int tile = blockIdx.x + i * gridDim.x, m0 = (tile % m_tiles) * PF_BM, n0 = (tile / m_tiles) * N_STEP, buf = i & 1;
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[buf], (i >> 1) & 1, &abort_flag, PF_WAIT_LIMIT));   // warp-uniform: tcgen05.ld is .aligned
+        if (!ok) break;
         tc_fence_after();
-        const int quarter = warp & 3;
         const int row = m0 + quarter * 32 + lane;
-        const bool live = ok && row < g.M;
-        const uint32_t trow = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
-        if (ok) {
+        const bool live = row < g.M;
+        const uint32_t trow = tmem + buf * C::BN + (static_cast<uint32_t>(quarter * 32) << 16);
+        {
             if (EPI == EPI_RESID) {
                 for (int c = 0; c < N_STEP / 32; ++c) {
                     const int n = n0 + c * 32;
@@ -398,12 +416,16 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
                 }
             }
         }
+        tc_fence_before();           // the accumulator may be overwritten: this warp has read its quarter
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&acc_empty[buf]);
+      }
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(C::BN) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(2 * C::BN) : "memory");
     }
     if (threadIdx.x == 0 && abort_flag) atomicExch(g.error, 1);
 }
@@ -578,18 +600,18 @@ bool encode_operand_map(CUtensorMap *m, const void *base, long long rows, int K)
 }
 
 template <int EPI, int SHAPE>
-const char *launch_gemm_cfg(const CUtensorMap &ma, const CUtensorMap &ml, const CUtensorMap &mb, const GemmArgs &g, cudaStream_t s) {
+const char *launch_gemm_cfg(const CUtensorMap &ma, const CUtensorMap &ml, const CUtensorMap &mb, const GemmArgs &g, int num_sms, cudaStream_t s) {
     using C = GemmCfg<SHAPE>;
     if (cudaFuncSetAttribute(prefill_gemm_kernel<EPI, SHAPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess)
         return "cudaFuncSetAttribute failed";
     const int n_step = EPI == EPI_SWIGLU ? 128 : C::BN;
-    const dim3 grid((g.N + n_step - 1) / n_step, (g.M + PF_BM - 1) / PF_BM);
-    prefill_gemm_kernel<EPI, SHAPE><<<grid, 192, C::SMEM, s>>>(ma, ml, mb, g);
+    const int tiles = ((g.N + n_step - 1) / n_step) * ((g.M + PF_BM - 1) / PF_BM);
+    prefill_gemm_kernel<EPI, SHAPE><<<tiles < num_sms ? tiles : num_sms, 192, C::SMEM, s>>>(ma, ml, mb, g);
     return cudaGetLastError() == cudaSuccess ? nullptr : "prefill GEMM launch failed";
 }
 
-// Shape choice: wide tiles when they still give at least 60 % of the SMs a tile (96 of 148 for the 1.5B down projection at
-// 2048 tokens: 115 -> 7x us); otherwise narrow tiles, deep when no SM would get a second CTA.
+// Shape choice: the rounds the SMs need (tiles / SMs, rounded up) times the relative cost of a tile (a wide tile does twice
+// the work of a narrow one for 1.33 x the operand traffic: 1.6), whichever is smaller.
 template <int EPI>
 const char *launch_gemm(const uint16_t *a, size_t a_plane, const void *w, long long w_rows, const GemmArgs &g, int num_sms, cudaStream_t s) {
     CUtensorMap ma, ml, mb;
@@ -597,12 +619,12 @@ const char *launch_gemm(const uint16_t *a, size_t a_plane, const void *w, long l
         return "cuTensorMapEncodeTiled failed";
     const int m_tiles = (g.M + PF_BM - 1) / PF_BM;
     if constexpr (EPI == EPI_SWIGLU) {
-        return launch_gemm_cfg<EPI, PF_WIDE>(ma, ml, mb, g, s);
+        return launch_gemm_cfg<EPI, PF_WIDE>(ma, ml, mb, g, num_sms, s);
     } else {
         const int wide = ((g.N + 255) / 256) * m_tiles, narrow = ((g.N + 127) / 128) * m_tiles;
-        if (wide * 10 >= num_sms * 6) return launch_gemm_cfg<EPI, PF_WIDE>(ma, ml, mb, g, s);
-        if (narrow <= num_sms) return launch_gemm_cfg<EPI, PF_NARROW_DEEP>(ma, ml, mb, g, s);
-        return launch_gemm_cfg<EPI, PF_NARROW>(ma, ml, mb, g, s);
+        const int rounds_wide = (wide + num_sms - 1) / num_sms, rounds_narrow = (narrow + num_sms - 1) / num_sms;
+        if (rounds_wide * 16 <= rounds_narrow * 10) return launch_gemm_cfg<EPI, PF_WIDE>(ma, ml, mb, g, num_sms, s);
+        return launch_gemm_cfg<EPI, PF_NARROW>(ma, ml, mb, g, num_sms, s);
     }
 }
 
