@@ -287,6 +287,13 @@ edgefm_status edgefm_debug_plan(const edgefm_ctx *ctx, int32_t *out8);
  * first barrier of the next step runs into the bound.  Synchronises the device and re-records the step graph. */
 edgefm_status edgefm_debug_set_wait_limit(edgefm_ctx *ctx, uint32_t limit_ns, int32_t extra_barrier_arrivals);
 
+/* The same for the contractions of edgefm_prefill: every wait on a shared-memory barrier gives up after `polls` polls
+ * (2^24 by default; >= 1024), raises an error word that edgefm_sync_status reports as EDGEFM_ERR_TIMEOUT, waits (bounded) for
+ * its own copies and multiplies in flight, frees its tensor memory and returns.  extra_arrivals = 1 (0 in production) makes
+ * the stage barriers expect an arrival nobody makes, so that the first wait of every contraction enqueued afterwards runs
+ * into the bound without any fault.  Host only. */
+edgefm_status edgefm_debug_set_prefill_wait(edgefm_ctx *ctx, uint32_t polls, int32_t extra_arrivals);
+
 /* Host-only check of the planner: the tile schedule of one weight-streaming operator (kind: 0 QKV pairs, 1 residual rows,
  * 2 gate/up pairs, 3 output-layer rows; units rows or pairs; K columns; head_half = head_dim / 2 for kind 0) for n_ctas CTAs
  * of n_warps consumer warps whose ring slots hold slot_rows rows.  tiles_out receives one 64-bit descriptor per tile, CTA by

@@ -51,7 +51,7 @@ class _Weights(ctypes.Structure):
 
 EXPORTS = ("edgefm_create", "edgefm_prefill_kv", "edgefm_decode_step", "edgefm_destroy", "edgefm_get_length",
            "edgefm_export_kv", "edgefm_get_launches_per_step", "edgefm_last_error", "edgefm_version",
-           "edgefm_sync_status", "edgefm_debug_profile", "edgefm_debug_set_wait_limit", "edgefm_debug_plan", "edgefm_debug_plan_operator", "edgefm_decode_step_static", "edgefm_set_vocab_subset",
+           "edgefm_sync_status", "edgefm_debug_profile", "edgefm_debug_set_wait_limit", "edgefm_debug_set_prefill_wait", "edgefm_debug_plan", "edgefm_debug_plan_operator", "edgefm_decode_step_static", "edgefm_set_vocab_subset",
            "edgefm_append_kv", "edgefm_create_with_options", "edgefm_export_kv_int8", "edgefm_verify_block", "edgefm_sync_length", "edgefm_prefill_tokens", "edgefm_prefill")
 
 
@@ -101,6 +101,8 @@ def load_library():
     L.edgefm_debug_profile.argtypes = [vp, vp, i64, ctypes.POINTER(i32), ctypes.POINTER(i32)]
     L.edgefm_debug_set_wait_limit.restype = ctypes.c_int
     L.edgefm_debug_set_wait_limit.argtypes = [vp, ctypes.c_uint32, i32]
+    L.edgefm_debug_set_prefill_wait.restype = ctypes.c_int
+    L.edgefm_debug_set_prefill_wait.argtypes = [vp, ctypes.c_uint32, i32]
     L.edgefm_debug_plan.restype = ctypes.c_int
     L.edgefm_debug_plan.argtypes = [vp, ctypes.POINTER(i32)]
     L.edgefm_debug_plan_operator.restype = ctypes.c_int
@@ -215,6 +217,10 @@ def edgefm_set_vocab_subset(ctx, token_ids, stream=None):
 
 def edgefm_sync_status(ctx, stream=None):
     _check(load_library().edgefm_sync_status(ctx, stream), ctx)
+
+
+def edgefm_debug_set_prefill_wait(ctx, polls, extra_arrivals=0):
+    _check(load_library().edgefm_debug_set_prefill_wait(ctx, polls, extra_arrivals), ctx)
 
 
 def edgefm_debug_set_wait_limit(ctx, limit_ns, extra_barrier_arrivals=0):

@@ -376,6 +376,7 @@ struct edgefm_ctx {
     int launches_per_step = 0;
     PrefillBuffers pf;           // work buffers of edgefm_prefill, allocated at its first call
     int prefill_launches = 0;    // kernels the last edgefm_prefill enqueued
+    uint32_t pf_wait_limit = 1u << 24, pf_extra_arrivals = 0;   // edgefm_debug_set_prefill_wait
 
     // host mirrors
     int cur_len = 0;
@@ -829,6 +830,8 @@ edgefm_status edgefm_prefill(edgefm_ctx *ctx, const int32_t *tokens, int32_t n, 
             return fail(ctx, EDGEFM_ERR_OUT_OF_MEMORY, "work buffers of edgefm_prefill (%zu bytes)", prefill_buffer_bytes(ctx->shape, chunk));
         }
     }
+    ctx->pf.wait_limit = ctx->pf_wait_limit;
+    ctx->pf.extra_arrivals = ctx->pf_extra_arrivals;
     PrefillModel pm{ctx->shape, ctx->layers.data(), ctx->embed, ctx->k_cache, ctx->v_cache, ctx->max_context, ctx->state, ctx->num_sms};
     ctx->prefill_launches = 0;
     for (int i = 0; i < n_dense;) {
@@ -987,6 +990,16 @@ edgefm_status edgefm_debug_set_wait_limit(edgefm_ctx *ctx, uint32_t limit_ns, in
     ctx->mk.spin_limit = limit_ns;
     ctx->mk.barrier_extra = extra_barrier_arrivals;
     CUDA_TRY(ctx, record_graph(ctx));
+    ctx->err.clear();
+    return EDGEFM_OK;
+}
+
+edgefm_status edgefm_debug_set_prefill_wait(edgefm_ctx *ctx, uint32_t polls, int32_t extra_arrivals) {
+    if (!ctx) return EDGEFM_ERR_INVALID_ARG;
+    if (polls < 1024u || extra_arrivals < 0 || extra_arrivals > 1)
+        return fail(ctx, EDGEFM_ERR_INVALID_ARG, "polls must be >= 1024 and extra_arrivals 0 or 1");
+    ctx->pf_wait_limit = polls;
+    ctx->pf_extra_arrivals = static_cast<uint32_t>(extra_arrivals);
     ctx->err.clear();
     return EDGEFM_OK;
 }

@@ -192,6 +192,8 @@ enum { EPI_QKV = 0, EPI_RESID = 1, EPI_SWIGLU = 2 };
 struct GemmArgs {
     int M, N, K;              // rows (tokens), output features (gate/up: F, each of gate and up), reduction length
     int *error;
+    uint32_t wait_limit;      // polls a wait on an mbarrier may take
+    uint32_t extra_arrivals;  // 0; 1 (tests): the stage barriers expect an arrival nobody makes, so the first wait runs out
     // QKV
     const uint16_t *bias;     // [N] or null
     const float2 *rope;       // [M][d/2]
@@ -208,7 +210,6 @@ struct GemmArgs {
 };
 
 constexpr int PF_BM = 128, PF_BK = 64;
-constexpr uint32_t PF_WAIT_LIMIT = 1u << 24;   // polls; far beyond any legitimate wait of a tile
 
 // Tile shapes.  PF_NARROW: 128 output columns, 4 stages of 48 KB.  PF_WIDE: 256 output columns, 3 stages of 64 KB: per k-block
 // 64 KB of operands feed twice the multiplies of a narrow tile's 48 KB, which matters because operand delivery from L2, not
@@ -232,7 +233,7 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
     static_assert(EPI != EPI_SWIGLU || SHAPE == PF_WIDE, "gate and up share one accumulator");
     constexpr int N_STEP = EPI == EPI_SWIGLU ? 128 : C::BN;   // output columns (of g.N) a CTA covers
     extern __shared__ uint8_t pf_dyn[];
-    __shared__ uint64_t full_bar[C::STAGES], empty_bar[C::STAGES], acc_full[2], acc_empty[2];
+    __shared__ uint64_t full_bar[C::STAGES], empty_bar[C::STAGES], acc_full[2], acc_empty[2], drain_bar;
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     uint8_t *tiles = pf_dyn + ((1024u - (smem_u32(pf_dyn) & 1023u)) & 1023u);
@@ -242,8 +243,9 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
     const int KB = (g.K + PF_BK - 1) / PF_BK;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < C::STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int s = 0; s < C::STAGES; ++s) { mbar_init(&full_bar[s], 1 + g.extra_arrivals); mbar_init(&empty_bar[s], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 4); }
+        mbar_init(&drain_bar, 1);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -258,18 +260,25 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
 
     if (warp == 0 && lane == 0) {            // producer: operand tiles by TMA
         bool ok = true;
+        int issued = 0;
         for (int i = 0, it = 0; i < my_tiles && ok; ++i) {
           const int tile = blockIdx.x + i * gridDim.x, m0 = (tile % m_tiles) * PF_BM, n0 = (tile / m_tiles) * N_STEP;
           for (int kb = 0; kb < KB; ++kb, ++it) {
             const int s = it % C::STAGES;
-            if (it >= C::STAGES && !mbar_wait(&empty_bar[s], ((it / C::STAGES) - 1) & 1, &abort_flag, PF_WAIT_LIMIT)) { ok = false; break; }
+            if (it >= C::STAGES && !mbar_wait(&empty_bar[s], ((it / C::STAGES) - 1) & 1, &abort_flag, g.wait_limit)) { ok = false; break; }
             uint8_t *a = tiles + s * C::STAGE_BYTES, *b = a + 2 * C::A_BYTES;
             mbar_expect_tx(&full_bar[s], C::STAGE_BYTES);
             tma_load_2d(a, &map_a_hi, kb * PF_BK, m0, &full_bar[s]);
             tma_load_2d(a + C::A_BYTES, &map_a_lo, kb * PF_BK, m0, &full_bar[s]);
             tma_load_2d(b, &map_b, kb * PF_BK, n0, &full_bar[s]);
             if (C::BN == 256) tma_load_2d(b + 128 * PF_BK * 2, &map_b, kb * PF_BK, (EPI == EPI_SWIGLU ? g.N : 128) + n0, &full_bar[s]);
+            issued = it + 1;
           }
+        }
+        if (abort_flag) {   // giving up: the copies still in flight must land before the CTA's shared memory is released
+            int dummy = 0;
+            for (int j = issued > C::STAGES ? issued - C::STAGES : 0; j < issued; ++j)
+                mbar_wait(&full_bar[j % C::STAGES], (j / C::STAGES) & 1, &dummy, g.wait_limit);
         }
     } else if (warp == 1 && lane == 0) {     // issuer: per stage 4 tcgen05.mma (K = 16 each) for the hi pieces, 4 for the lo pieces
         constexpr uint32_t idesc = umma_idesc_bf16(PF_BM, C::BN);
@@ -277,12 +286,12 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
         for (int i = 0, it = 0; i < my_tiles && ok; ++i) {
           const int buf = i & 1;
           const uint32_t acc = tmem + buf * C::BN;
-          if (i >= 2) ok = mbar_wait(&acc_empty[buf], ((i >> 1) - 1) & 1, &abort_flag, PF_WAIT_LIMIT);   // its epilogue has read it
+          if (i >= 2) ok = mbar_wait(&acc_empty[buf], ((i >> 1) - 1) & 1, &abort_flag, g.wait_limit);   // its epilogue has read it
           if (!ok) break;
           tc_fence_after();
           for (int kb = 0; kb < KB; ++kb, ++it) {
             const int s = it % C::STAGES;
-            ok = mbar_wait(&full_bar[s], (it / C::STAGES) & 1, &abort_flag, PF_WAIT_LIMIT);
+            ok = mbar_wait(&full_bar[s], (it / C::STAGES) & 1, &abort_flag, g.wait_limit);
             if (!ok) break;
             tc_fence_after();
             const uint32_t a = smem_u32(tiles + s * C::STAGE_BYTES), b = a + 2 * C::A_BYTES;
@@ -295,11 +304,16 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
           }
           if (ok) umma_commit(&acc_full[buf]);
         }
+        if (!ok) {          // giving up: the multiplies already issued must finish before the tensor memory is freed
+            int dummy = 0;
+            umma_commit(&drain_bar);
+            mbar_wait(&drain_bar, 0, &dummy, g.wait_limit);
+        }
     } else if (warp >= 2) {                  // epilogue: warp w may read lanes 32 (w % 4) .. + 31 of tensor memory
       const int quarter = warp & 3;
       for (int i = 0; i < my_tiles; ++i) {
         const int tile = blockIdx.x + i * gridDim.x, m0 = (tile % m_tiles) * PF_BM, n0 = (tile / m_tiles) * N_STEP, buf = i & 1;
-        const bool ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[buf], (i >> 1) & 1, &abort_flag, PF_WAIT_LIMIT));   // warp-uniform: tcgen05.ld is .aligned
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[buf], (i >> 1) & 1, &abort_flag, g.wait_limit));   // warp-uniform: tcgen05.ld is .aligned
         if (!ok) break;
         tc_fence_after();
         const int row = m0 + quarter * 32 + lane;
@@ -687,7 +701,7 @@ const char *prefill_run(const PrefillModel &m, PrefillBuffers *b, const int32_t 
         const edgefm_layer_weights &w = m.layers[l];
         uint16_t *kc = m.k_cache + static_cast<size_t>(l) * nkv * head_stride, *vc = m.v_cache + static_cast<size_t>(l) * nkv * head_stride;
         GemmArgs g{};
-        g.M = n; g.error = b->error;
+        g.M = n; g.error = b->error; g.wait_limit = b->wait_limit; g.extra_arrivals = b->extra_arrivals;
         g.N = n_qkv; g.K = H;
         g.bias = sh.qkv_bias ? static_cast<const uint16_t *>(w.bqkv) : nullptr;
         g.rope = b->rope; g.q_out = b->q; g.q_plane = q_plane;

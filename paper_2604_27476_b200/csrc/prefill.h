@@ -23,6 +23,8 @@ struct PrefillBuffers {
     float2 *rope = nullptr;      // (cos, sin) of the chunk's positions, [chunk][d/2]
     int *tokens = nullptr;       // device copy of the chunk's token ids
     int *error = nullptr;        // device word: non-zero when a bounded wait of a GEMM ran out
+    uint32_t wait_limit = 1u << 24;   // polls per wait (far beyond any legitimate wait of a tile)
+    uint32_t extra_arrivals = 0;      // tests only: 1 makes the first wait of every contraction run out
 };
 
 struct PrefillModel {

@@ -43,3 +43,38 @@ def test_grid_barrier_wait_expires_and_is_reported():
         other.close()
     finally:
         pair.close()                                               # destroying the timed-out context succeeds
+
+
+def test_prefill_contraction_wait_expires_and_is_reported():
+    """The same for the contractions of edgefm_prefill: their stage barriers are told to expect an arrival nobody makes and
+    the bound is shortened to 2^16 polls; every contraction gives up at its first wait, drains and returns."""
+    import numpy as np
+    import torch
+    from paper_2604_27476_b200 import DecodeContext, EdgefmError, Status, edgefm_debug_set_prefill_wait, edgefm_sync_status
+    cfg = CONFIGS["tiny"]
+    pair = Pair(cfg, cache_len=4, max_context=64)
+    try:
+        stream = torch.cuda.current_stream().cuda_stream
+        toks = np.random.default_rng(3).integers(0, cfg.vocab, 40).tolist()
+        for i, t in enumerate(toks):
+            ref, _ = pair.oracle.step(t, 4 + i)
+        with pytest.raises(EdgefmError):                           # limits are validated
+            edgefm_debug_set_prefill_wait(pair.ctx.handle, 10, 0)
+        edgefm_debug_set_prefill_wait(pair.ctx.handle, 1 << 16, 1)
+        t0 = time.perf_counter()
+        pair.ctx.prefill(toks, 4)
+        with pytest.raises(EdgefmError) as ei:
+            edgefm_sync_status(pair.ctx.handle, stream)
+        dt = time.perf_counter() - t0
+        assert ei.value.status == Status.ERR_TIMEOUT
+        assert dt < 5.0                                            # five contractions, each gave up within milliseconds
+        # the CUDA context is intact: a fresh edgefm context on the same weights prefills the same prompt correctly
+        other = DecodeContext(cfg, pair.ptrs, 64)
+        other.prefill_kv(pair.kd, pair.vd)
+        other.prefill(toks, 4)
+        torch.cuda.synchronize()
+        other.sync_status()
+        assert_logits_close(other.logits.cpu().numpy(), ref, "fresh context after the expired waits")
+        other.close()
+    finally:
+        pair.close()
