@@ -7,8 +7,8 @@
 //       QKV      : + bias, rotate-half RoPE of q and k, q to the work buffer, k and v rows to the cache;
 //       O / down : added to the fp32 residual stream;
 //       gate/up  : SwiGLU, silu(gate) * up, to the bf16 activation buffer.
-//   * prefill_attention_kernel: causal attention of the T queries over the cache rows (prefix + the T new rows), online
-//     softmax, mma.sync tiles (under 6 % of the flops of a 2048-token prompt; not worth a second tcgen05 kernel).
+//   * prefill_attention_tc_kernel: causal attention of the T queries over the cache rows (prefix + the T new rows), also on
+//     tcgen05: S = Q K^T and O = P V in tensor memory, online softmax by warps that own the rows (see the kernel).
 //   * rmsnorm / embedding kernels: one row per warp.
 // Every activation enters the tensor cores as TWO bf16 pieces (hi + lo, 16 mantissa bits; twice the multiplies, one load of
 // the weight tile), because single bf16 activations put the logits of a 28-layer model outside the step's tolerance
@@ -93,6 +93,24 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float *v) {
         : "r"(taddr)
         : "memory");
 }
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float *v) {
+    uint32_t *r = reinterpret_cast<uint32_t *>(v);
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+template <int N> __device__ __forceinline__ void tmem_ld(uint32_t taddr, float *v) {
+    static_assert(N == 16 || N % 32 == 0, "16 columns or a multiple of 32");
+    if constexpr (N == 16) {
+        tmem_ld16(taddr, v);
+    } else {
+#pragma unroll
+        for (int c = 0; c < N / 32; ++c) tmem_ld32(taddr + c * 32, v + c * 32);
+    }
+}
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor of a K-major bf16 tile written by TMA with the 128-byte swizzle: rows of 64 elements
@@ -108,6 +126,11 @@ __host__ __device__ constexpr uint32_t umma_idesc_bf16(int m, int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
 }
 
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
     return static_cast<uint32_t>(f32_to_bf16_bits(lo)) | (static_cast<uint32_t>(f32_to_bf16_bits(hi)) << 16);
 }
@@ -124,6 +147,15 @@ __device__ __forceinline__ void split2x2(float a, float b, uint32_t &hi, uint32_
     split2(b, bh, bl);
     hi = static_cast<uint32_t>(ah) | (static_cast<uint32_t>(bh) << 16);
     lo = static_cast<uint32_t>(al) | (static_cast<uint32_t>(bl) << 16);
+}
+
+// The same split by truncation (hi = the upper 16 bits of x, lo = the upper 16 bits of x - hi; x - hi is exact): no conversion
+// instruction, which shares the special-function pipe with exp2 in the attention loop.  Error below 2^-16 relative.
+__device__ __forceinline__ void split2x2_trunc(float a, float b, uint32_t &hi, uint32_t &lo) {
+    const uint32_t ab = __float_as_uint(a), bb = __float_as_uint(b);
+    hi = __byte_perm(ab, bb, 0x7632);
+    const float ra = a - __uint_as_float(ab & 0xffff0000u), rb = b - __uint_as_float(bb & 0xffff0000u);
+    lo = __byte_perm(__float_as_uint(ra), __float_as_uint(rb), 0x7632);
 }
 
 // ---- small kernels -----------------------------------------------------------------------------------------------------
@@ -444,170 +476,283 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
     if (threadIdx.x == 0 && abort_flag) atomicExch(g.error, 1);
 }
 
-// ---- causal attention of the new queries over the cache ------------------------------------------------------------------
-__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
-__device__ __forceinline__ void mma_16816(float *c, const uint32_t *a, uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+// ---- causal attention on tcgen05 ---------------------------------------------------------------------------------------------
+// One CTA = 128 queries of one head (a query = a lane of tensor memory = a thread of the softmax warps); keys in blocks of 64.
+// Per block j:  S_j = Q K_j^T (tcgen05.mma, M 128, N 64, K = D; queries as two bf16 pieces) into one of two S buffers in
+// tensor memory;  the softmax warps read their row (tcgen05.ld), mask, update the running maximum and sum, and write the
+// probabilities as two bf16 pieces into shared memory in the swizzled K-major layout of an A operand;  O_j = P_j V_j (M 128,
+// N = D, K = 64 keys; V straight from its cache rows as an MN-major B operand) into a third region of tensor memory;  the
+// softmax warps add O_j to their fp32 row in registers, o = o * alpha_j + O_j, one block late so that the multiply hides under
+// the next block's softmax.  S_{j+1} is issued before P_j is waited for, so the tensor pipe works under the softmax too.
+//   tensor memory: S0 [0, 64), S1 [64, 128), O0 [128, 128 + D), O1 [128 + D, 128 + 2 D)
+//   shared memory: Q 2 x D/64 x 16 KB | 2 stages x (K D/64 x 8 KB, V D/64 x 8 KB) | 2 x P (2 x 16 KB)
+constexpr int AT_BM = 128, AT_BN = 64, AT_PARTS = 2;
+constexpr int AT_THREADS = 64 + 128 * AT_PARTS;
+
+// B operand in MN-major form for P V: the V tile is D/64 blocks of [64 keys][64 d] (128-byte rows, 128-byte swizzle).  N (= d)
+// runs along a row, K (= keys) across rows: groups of 8 keys are 1024 bytes apart (stride byte offset), the 64-column blocks
+// `lbo` bytes apart (leading byte offset).
+__device__ __forceinline__ uint64_t umma_desc_sw128_mn(uint32_t smem_addr, uint32_t lbo) {
+    return static_cast<uint64_t>((smem_addr >> 4) & 0x3fffu) | (static_cast<uint64_t>((lbo >> 4) & 0x3fffu) << 16) | (64ull << 32) |
+           (1ull << 46) | (2ull << 61);
 }
 
-// A [64][D] bf16 tile in shared memory; the 16-byte pieces of a row are permuted by the row's low three bits so that the
-// eight rows an ldmatrix touches fall into different banks.
-template <int D> __device__ __forceinline__ uint32_t tile_addr(uint32_t base, int row, int piece) {
-    return base + row * (D * 2) + ((piece ^ (row & 7)) << 4);
-}
-template <int D>
-__device__ __forceinline__ void load_rows(uint32_t base, const uint16_t *src, long long row_stride, int first, int last_valid, int tid) {
-    constexpr int PIECES = D / 8;
-    for (int i = tid; i < 64 * PIECES; i += 128) {
-        const int r = i / PIECES, c = i % PIECES;
-        const int row = min(first + r, last_valid);
-        cp_async16(tile_addr<D>(base, r, c), src + row * row_stride + c * 8);
-    }
-}
+template <int D> struct AttnCfg {
+    static constexpr int KBLK = D / 64;                        // 64-column blocks of a row of q, k, v
+    static constexpr int Q_BYTES = 2 * KBLK * AT_BM * 128;     // two pieces
+    static constexpr int K_BYTES = KBLK * AT_BN * 128, V_BYTES = K_BYTES;
+    static constexpr int P_BYTES = 2 * AT_BM * 128;            // two pieces of [128][64 keys]
+    static constexpr int SMEM = Q_BYTES + 2 * (K_BYTES + V_BYTES) + 2 * P_BYTES + 1024;   // K/V and P double-buffered
+    static constexpr int TMEM_COLS = 2 * AT_BN + 2 * D <= 256 ? 256 : 512;   // S0, S1, O0, O1
+};
 
-// grid (ceil(T / 64), nq); 4 warps, 16 queries each.  Query t of the chunk sits in cache slot slot0 + t and sees the keys
-// 0 .. slot0 + t.  q: rotated queries [2][..][nq D] (hi and lo bf16 planes, `plane` elements apart); kc / vc: this layer's
-// cache, [nkv][max_context][D]; out: [2][..][nq D], again two planes.  Queries and probabilities enter the tensor cores as
-// two bf16 pieces each (the cache rows are bf16 exactly), sums are fp32.
 template <int D>
-__global__ void __launch_bounds__(128) prefill_attention_kernel(const uint16_t *q, const uint16_t *kc, const uint16_t *vc, uint16_t *out,
-                                                                size_t plane, int T, int slot0, int nq, int group, long long head_stride,
-                                                                float scale_log2) {
-    extern __shared__ __align__(128) uint8_t at_dyn[];
-    constexpr int TILE = 64 * D * 2;
-    const uint32_t sq = smem_u32(at_dyn), sk = sq + 2 * TILE, sv = sk + 2 * TILE;   // q hi, q lo, 2 x k, 2 x v
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, gq = lane >> 2, tq = lane & 3;
-    const int t0 = (gridDim.x - 1 - blockIdx.x) * 64;     // long rows first
+__global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q_hi,
+                                                                   const __grid_constant__ CUtensorMap map_q_lo,
+                                                                   const __grid_constant__ CUtensorMap map_k,
+                                                                   const __grid_constant__ CUtensorMap map_v, uint16_t *out, size_t plane,
+                                                                   int T, int slot0, int nq, int group, int max_context,
+                                                                   float scale_log2, uint32_t wait_limit, int *error) {
+    using C = AttnCfg<D>;
+    extern __shared__ uint8_t at_tc_dyn[];
+    __shared__ uint64_t q_full, kv_full[2], kv_empty[2], s_full[2], s_empty[2], p_full[2], p_empty[2], o_full[2], o_empty[2], drain_bar, pair_bar[4];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    __shared__ float xchg[2][AT_PARTS][AT_BM];      // row maxima / sums passed between the two threads of a row
+    uint8_t *base = at_tc_dyn + ((1024u - (smem_u32(at_tc_dyn) & 1023u)) & 1023u);
+    uint8_t *sq = base, *skv = sq + C::Q_BYTES, *sp = skv + 2 * (C::K_BYTES + C::V_BYTES);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int t0 = (gridDim.x - 1 - blockIdx.x) * AT_BM;      // long rows first
     const int h = blockIdx.y, hk = h / group;
-    const uint16_t *kh = kc + hk * head_stride, *vh = vc + hk * head_stride;
-    const int last_key = slot0 + min(t0 + 63, T - 1);
-    const int nkb = last_key / 64 + 1;
+    const int last_key = slot0 + min(t0 + AT_BM - 1, T - 1);
+    const int nb = last_key / AT_BN + 1;
 
-    load_rows<D>(sq, q + static_cast<size_t>(h) * D, static_cast<long long>(nq) * D, t0, T - 1, tid);
-    load_rows<D>(sq + TILE, q + plane + static_cast<size_t>(h) * D, static_cast<long long>(nq) * D, t0, T - 1, tid);
-    load_rows<D>(sk, kh, D, 0, last_key, tid);
-    load_rows<D>(sv, vh, D, 0, last_key, tid);
-    asm volatile("cp.async.commit_group;" ::: "memory");
+    if (threadIdx.x == 0) {
+        mbar_init(&q_full, 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(&kv_full[i], 1); mbar_init(&kv_empty[i], 1); mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 4 * AT_PARTS); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&p_full[i], 4 * AT_PARTS); mbar_init(&p_empty[i], 1); mbar_init(&o_full[i], 1); mbar_init(&o_empty[i], 4 * AT_PARTS); }
+        mbar_init(&drain_bar, 1);
+        for (int i = 0; i < 4; ++i) mbar_init(&pair_bar[i], AT_PARTS);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(C::TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_slot;
 
-    float o[D / 8][4];
-#pragma unroll
-    for (int i = 0; i < D / 8; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
-    float mrow[2] = {-INFINITY, -INFINITY}, lrow[2] = {0.f, 0.f};
-    const int qi0 = slot0 + t0 + warp * 16 + gq;          // cache slot of this thread's first row; the second is + 8
-
-    for (int kb = 0; kb < nkb; ++kb) {
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
-        __syncthreads();
-        const uint32_t kbuf = sk + (kb & 1) * TILE, vbuf = sv + (kb & 1) * TILE;
-        if (kb + 1 < nkb) {
-            load_rows<D>(sk + ((kb + 1) & 1) * TILE, kh, D, (kb + 1) * 64, last_key, tid);
-            load_rows<D>(sv + ((kb + 1) & 1) * TILE, vh, D, (kb + 1) * 64, last_key, tid);
-            asm volatile("cp.async.commit_group;" ::: "memory");
+    if (warp == 0 && lane == 0) {            // producer: the query tile once, then the K and V rows of every key block
+        mbar_expect_tx(&q_full, C::Q_BYTES);
+        for (int kb = 0; kb < C::KBLK; ++kb) {
+            tma_load_2d(sq + kb * AT_BM * 128, &map_q_hi, h * D + kb * 64, t0, &q_full);
+            tma_load_2d(sq + (C::KBLK + kb) * AT_BM * 128, &map_q_lo, h * D + kb * 64, t0, &q_full);
         }
-        float s[8][4];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) s[i][0] = s[i][1] = s[i][2] = s[i][3] = 0.f;
-#pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
-            uint32_t qh[4], ql[4];
-            ldsm_x4(tile_addr<D>(sq, warp * 16 + (lane & 15), ks * 2 + (lane >> 4)), qh[0], qh[1], qh[2], qh[3]);
-            ldsm_x4(tile_addr<D>(sq + TILE, warp * 16 + (lane & 15), ks * 2 + (lane >> 4)), ql[0], ql[1], ql[2], ql[3]);
-#pragma unroll
-            for (int np = 0; np < 4; ++np) {
-                uint32_t b0, b1, b2, b3;
-                ldsm_x4(tile_addr<D>(kbuf, np * 16 + (lane & 7) + ((lane >> 4) << 3), ks * 2 + ((lane >> 3) & 1)), b0, b1, b2, b3);
-                mma_16816(s[2 * np], qh, b0, b1);
-                mma_16816(s[2 * np + 1], qh, b2, b3);
-                mma_16816(s[2 * np], ql, b0, b1);
-                mma_16816(s[2 * np + 1], ql, b2, b3);
+        int issued = 0;
+        for (int j = 0; j < nb; ++j) {
+            const int st = j & 1;
+            if (j >= 2 && !mbar_wait(&kv_empty[st], ((j >> 1) - 1) & 1, &abort_flag, wait_limit)) break;
+            uint8_t *k = skv + st * (C::K_BYTES + C::V_BYTES), *v = k + C::K_BYTES;
+            mbar_expect_tx(&kv_full[st], C::K_BYTES + C::V_BYTES);
+            for (int kb = 0; kb < C::KBLK; ++kb) {
+                tma_load_2d(k + kb * AT_BN * 128, &map_k, kb * 64, hk * max_context + j * AT_BN, &kv_full[st]);
+                tma_load_2d(v + kb * AT_BN * 128, &map_v, kb * 64, hk * max_context + j * AT_BN, &kv_full[st]);
             }
+            issued = j + 1;
         }
-        // causal mask, running maximum, probabilities
-        float mx[2] = {mrow[0], mrow[1]};
+        if (abort_flag) {   // giving up: the copies in flight must land before the shared memory is released
+            int dummy = 0;
+            mbar_wait(&q_full, 0, &dummy, wait_limit);
+            for (int j = issued > 2 ? issued - 2 : 0; j < issued; ++j) mbar_wait(&kv_full[j & 1], (j >> 1) & 1, &dummy, wait_limit);
+        }
+    } else if (warp == 1 && lane == 0) {     // issuer
+        constexpr uint32_t idesc_s = umma_idesc_bf16(AT_BM, AT_BN);
+        constexpr uint32_t idesc_o = umma_idesc_bf16(AT_BM, D) | (1u << 16);   // B (= V) is MN-major
+        auto issue_s = [&](int j) {          // S_j = Q K_j^T, hi pieces then lo pieces
+            const uint32_t k = smem_u32(skv + (j & 1) * (C::K_BYTES + C::V_BYTES)), acc = tmem + (j & 1) * AT_BN;
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt)
+            for (int piece = 0; piece < 2; ++piece)
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int key = kb * 64 + nt * 8 + 2 * tq + (e & 1);
-                const int r = e >> 1;
-                if (key > qi0 + 8 * r) s[nt][e] = -INFINITY;
-                mx[r] = fmaxf(mx[r], s[nt][e]);
+                for (int kb = 0; kb < C::KBLK; ++kb) {
+                    const uint64_t da = umma_desc_sw128(smem_u32(sq) + (piece * C::KBLK + kb) * AT_BM * 128);
+                    const uint64_t db = umma_desc_sw128(k + kb * AT_BN * 128);
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) umma_bf16(acc, da + 2 * kk, db + 2 * kk, idesc_s, (piece | kb | kk) != 0);
+                }
+            umma_commit(&s_full[j & 1]);
+        };
+        bool ok = mbar_wait(&q_full, 0, &abort_flag, wait_limit) && mbar_wait(&kv_full[0], 0, &abort_flag, wait_limit);
+        if (ok) { tc_fence_after(); issue_s(0); }
+        for (int j = 0; j < nb && ok; ++j) {
+            if (j + 1 < nb) {                // the next block's scores, under this block's softmax
+                const int st = (j + 1) & 1;
+                ok = mbar_wait(&kv_full[st], ((j + 1) >> 1) & 1, &abort_flag, wait_limit);
+                if (ok && j + 1 >= 2) ok = mbar_wait(&s_empty[st], (((j + 1) >> 1) - 1) & 1, &abort_flag, wait_limit);
+                if (!ok) break;
+                tc_fence_after();
+                issue_s(j + 1);
             }
-        float alpha[2], sum[2] = {0.f, 0.f};
+            ok = mbar_wait(&p_full[j & 1], (j >> 1) & 1, &abort_flag, wait_limit);
+            if (ok && j >= 2) ok = mbar_wait(&o_empty[j & 1], ((j >> 1) - 1) & 1, &abort_flag, wait_limit);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t v = smem_u32(skv + (j & 1) * (C::K_BYTES + C::V_BYTES) + C::K_BYTES);
 #pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 1));
-            mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xffffffffu, mx[r], 2));
-            alpha[r] = exp2f((mrow[r] - mx[r]) * scale_log2);   // first block: exp2(-inf) = 0
-            mrow[r] = mx[r];
-        }
-        uint32_t pf[4][4], pl[4][4];
+            for (int piece = 0; piece < 2; ++piece) {
+                const uint64_t da = umma_desc_sw128(smem_u32(sp) + (j & 1) * C::P_BYTES + piece * AT_BM * 128);
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-            float p[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                p[e] = exp2f((s[nt][e] - mx[e >> 1]) * scale_log2);
-                sum[e >> 1] += p[e];
+                for (int kk = 0; kk < 4; ++kk)   // 16 keys = 2 groups of 8 rows = 2048 bytes of the V tile
+                    umma_bf16(tmem + 2 * AT_BN + (j & 1) * D, da + 2 * kk, umma_desc_sw128_mn(v + kk * 2048, AT_BN * 128), idesc_o, (piece | kk) != 0);
             }
-            split2x2(p[0], p[1], pf[nt >> 1][(nt & 1) * 2], pl[nt >> 1][(nt & 1) * 2]);
-            split2x2(p[2], p[3], pf[nt >> 1][(nt & 1) * 2 + 1], pl[nt >> 1][(nt & 1) * 2 + 1]);
+            umma_commit(&o_full[j & 1]);
+            umma_commit(&p_empty[j & 1]);
+            umma_commit(&kv_empty[j & 1]);
         }
+        if (!ok) {
+            int dummy = 0;
+            umma_commit(&drain_bar);
+            mbar_wait(&drain_bar, 0, &dummy, wait_limit);
+        }
+    }
+    else if (warp >= 2) {                    // softmax: AT_PARTS threads per query row (= lane of tensor memory), 16 keys of a block each
+        const int quarter = warp & 3, part = (warp - 2) >> 2, row = quarter * 32 + lane;
+        const uint32_t trow = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
+        const int qi = slot0 + t0 + row;     // cache slot of this query: it sees the keys 0 .. qi
+        constexpr int KP = AT_BN / AT_PARTS; // keys of a block per thread
+        constexpr int DP = D / AT_PARTS;     // this thread's columns of the output row
+        float o[DP];
 #pragma unroll
-        for (int r = 0; r < 2; ++r) lrow[r] = lrow[r] * alpha[r] + sum[r];
+        for (int i = 0; i < DP; ++i) o[i] = 0.f;
+        float m_run = -INFINITY, l_run = 0.f, alpha_prev = 1.f;
+        bool ok = true;
+        // one lane waits / arrives for its warp (an mbarrier operation per thread would cost more than the arithmetic)
+        auto warp_wait = [&](uint64_t *bar, int parity) {
+            int r = 1;
+            if (lane == 0) r = mbar_wait(bar, parity, &abort_flag, wait_limit) ? 1 : 0;
+            return __shfl_sync(0xffffffffu, r, 0) != 0;
+        };
+        auto warp_arrive = [&](uint64_t *bar) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar);
+        };
+        auto row_sync = [&](int round) {     // the AT_PARTS warps of a quarter meet (bounded like every other wait)
+            warp_arrive(&pair_bar[quarter]);
+            return warp_wait(&pair_bar[quarter], round & 1);
+        };
+        auto add_block = [&](int j) {        // o = o * alpha_j + O_j
+            ok = warp_wait(&o_full[j & 1], (j >> 1) & 1);
+            if (!ok) return;
+            tc_fence_after();
+            float v[DP];
+            tmem_ld<DP>(trow + 2 * AT_BN + (j & 1) * D + part * DP, v);
+            tmem_ld_wait();
+            tc_fence_before();
+            warp_arrive(&o_empty[j & 1]);
 #pragma unroll
-        for (int i = 0; i < D / 8; ++i) { o[i][0] *= alpha[0]; o[i][1] *= alpha[0]; o[i][2] *= alpha[1]; o[i][3] *= alpha[1]; }
+            for (int i = 0; i < DP; ++i) o[i] = fmaf(o[i], alpha_prev, v[i]);
+        };
+        for (int j = 0; j < nb; ++j) {
+            ok = warp_wait(&s_full[j & 1], (j >> 1) & 1);
+            if (!ok) break;
+            tc_fence_after();
+            const int key0 = j * AT_BN + part * KP;
+            const bool diagonal = j * AT_BN + AT_BN - 1 > slot0 + t0;   // some query of the tile does not see the whole block
+            float v[KP];
+            tmem_ld<KP>(trow + (j & 1) * AT_BN + part * KP, v);
+            tmem_ld_wait();
+            tc_fence_before();
+            warp_arrive(&s_empty[j & 1]);    // this part of S_j is in registers
+            if (diagonal) {
 #pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {
+                for (int i = 0; i < KP; ++i)
+                    if (key0 + i > qi) v[i] = -INFINITY;
+            }
+            float mx = fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3]));
 #pragma unroll
-            for (int dp = 0; dp < D / 16; ++dp) {
-                uint32_t b0, b1, b2, b3;
-                ldsm_x4_t(tile_addr<D>(vbuf, ks * 16 + (lane & 7) + (((lane >> 3) & 1) << 3), dp * 2 + (lane >> 4)), b0, b1, b2, b3);
-                mma_16816(o[2 * dp], pf[ks], b0, b1);
-                mma_16816(o[2 * dp + 1], pf[ks], b2, b3);
-                mma_16816(o[2 * dp], pl[ks], b0, b1);
-                mma_16816(o[2 * dp + 1], pl[ks], b2, b3);
+            for (int i = 4; i < KP; i += 4) mx = fmaxf(mx, fmaxf(fmaxf(v[i], v[i + 1]), fmaxf(v[i + 2], v[i + 3])));
+            xchg[j & 1][part][row] = mx;     // the row maximum needs the other threads' keys
+            ok = row_sync(j);
+            if (!ok) break;
+            mx = m_run;
+#pragma unroll
+            for (int q = 0; q < AT_PARTS; ++q) mx = fmaxf(mx, xchg[j & 1][q][row]);
+            const float alpha = fast_exp2((m_run - mx) * scale_log2);   // first block: exp2(-inf) = 0
+            m_run = mx;
+            const float neg = -mx * scale_log2;
+            float sum0 = 0.f, sum1 = 0.f;
+            uint4 hi[KP / 8], lo[KP / 8];
+#pragma unroll
+            for (int i8 = 0; i8 < KP / 8; ++i8) {   // probabilities as two bf16 pieces
+                uint32_t *hw = &hi[i8].x, *lw = &lo[i8].x;
+#pragma unroll
+                for (int i2 = 0; i2 < 4; ++i2) {
+                    const int i = i8 * 8 + i2 * 2;
+                    const float p0 = fast_exp2(fmaf(v[i], scale_log2, neg)), p1 = fast_exp2(fmaf(v[i + 1], scale_log2, neg));
+                    sum0 += p0;
+                    sum1 += p1;
+                    split2x2_trunc(p0, p1, hw[i2], lw[i2]);
+                }
+            }
+            l_run = l_run * alpha + (sum0 + sum1);
+            if (j >= 2) {                    // the P buffer's previous block has been multiplied
+                ok = warp_wait(&p_empty[j & 1], ((j >> 1) - 1) & 1);
+                if (!ok) break;
+            }
+            uint8_t *prow_hi = sp + (j & 1) * C::P_BYTES + row * 128, *prow_lo = prow_hi + AT_BM * 128;
+#pragma unroll
+            for (int i8 = 0; i8 < KP / 8; ++i8) {   // into the A-operand layout: 16-byte piece index xor row bits (128-byte swizzle)
+                const int piece16 = ((part * (KP / 8) + i8) ^ (row & 7)) << 4;
+                *reinterpret_cast<uint4 *>(prow_hi + piece16) = hi[i8];
+                *reinterpret_cast<uint4 *>(prow_lo + piece16) = lo[i8];
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P: generic-proxy writes before the tensor core's reads
+            warp_arrive(&p_full[j & 1]);
+            if (j >= 1) { add_block(j - 1); if (!ok) break; }
+            alpha_prev = alpha;
+        }
+        if (ok) add_block(nb - 1);
+        if (ok) {
+            xchg[nb & 1][part][row] = l_run; // the parts of the row sum
+            ok = row_sync(nb);
+            l_run = 0.f;
+#pragma unroll
+            for (int q = 0; q < AT_PARTS; ++q) l_run += xchg[nb & 1][q][row];
+        }
+        const int t = t0 + row;
+        if (ok && t < T) {
+            const float inv = 1.f / l_run;
+            uint16_t *dst = out + static_cast<size_t>(t) * nq * D + static_cast<size_t>(h) * D + part * DP;
+#pragma unroll
+            for (int i = 0; i < DP; i += 8) {
+                uint4 hi, lo;
+                split2x2(o[i] * inv, o[i + 1] * inv, hi.x, lo.x); split2x2(o[i + 2] * inv, o[i + 3] * inv, hi.y, lo.y);
+                split2x2(o[i + 4] * inv, o[i + 5] * inv, hi.z, lo.z); split2x2(o[i + 6] * inv, o[i + 7] * inv, hi.w, lo.w);
+                *reinterpret_cast<uint4 *>(dst + i) = hi;
+                *reinterpret_cast<uint4 *>(dst + plane + i) = lo;
             }
         }
     }
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-        lrow[r] += __shfl_xor_sync(0xffffffffu, lrow[r], 1);
-        lrow[r] += __shfl_xor_sync(0xffffffffu, lrow[r], 2);
-        const int t = t0 + warp * 16 + gq + 8 * r;
-        if (t < T) {
-            const float inv = 1.f / lrow[r];
-            uint32_t *dst = reinterpret_cast<uint32_t *>(out + static_cast<size_t>(t) * nq * D + static_cast<size_t>(h) * D);
-#pragma unroll
-            for (int i = 0; i < D / 8; ++i) {
-                uint32_t hi, lo;
-                split2x2(o[i][2 * r] * inv, o[i][2 * r + 1] * inv, hi, lo);
-                dst[i * 4 + tq] = hi;
-                dst[plane / 2 + i * 4 + tq] = lo;
-            }
-        }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(AttnCfg<D>::TMEM_COLS) : "memory");
     }
+    if (threadIdx.x == 0 && abort_flag) atomicExch(error, 1);
 }
 
 // ---- host side ---------------------------------------------------------------------------------------------------------------
-// Map of a row-major bf16 [rows][K] matrix; a box is 128 rows x 64 columns (one 128-byte swizzled row each); rows and
+// Map of a row-major bf16 [rows][K] matrix; a box is box_rows rows x 64 columns (one 128-byte swizzled row each); rows and
 // columns outside the matrix read as zero.  (No multicast is used with these maps.)
-bool encode_operand_map(CUtensorMap *m, const void *base, long long rows, int K) {
+bool encode_operand_map(CUtensorMap *m, const void *base, long long rows, int K, int box_rows = 128) {
     TensorMapEncodeFn enc = tensor_map_encoder();
     if (!enc) return false;
     const cuuint64_t dims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(rows)};
     const cuuint64_t strides[1] = {static_cast<cuuint64_t>(K) * 2};
-    const cuuint32_t box[2] = {PF_BK, 128};
+    const cuuint32_t box[2] = {PF_BK, static_cast<cuuint32_t>(box_rows)};
     const cuuint32_t es[2] = {1, 1};
     return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -643,13 +788,18 @@ const char *launch_gemm(const uint16_t *a, size_t a_plane, const void *w, long l
 }
 
 template <int D>
-const char *launch_attention(const uint16_t *q, const uint16_t *kc, const uint16_t *vc, uint16_t *out, size_t plane, int T, int slot0, int nq, int group,
-                             long long head_stride, cudaStream_t s) {
-    constexpr int smem = 6 * 64 * D * 2;
-    if (cudaFuncSetAttribute(prefill_attention_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+const char *launch_attention_tc(const uint16_t *q, const uint16_t *kc, const uint16_t *vc, uint16_t *out, size_t plane, int T, int slot0,
+                                int nq, int nkv, int max_context, uint32_t wait_limit, int *error, cudaStream_t s) {
+    CUtensorMap mqh, mql, mk, mv;
+    const long long kv_rows = static_cast<long long>(nkv) * max_context;
+    if (!encode_operand_map(&mqh, q, T, nq * D) || !encode_operand_map(&mql, q + plane, T, nq * D) ||
+        !encode_operand_map(&mk, kc, kv_rows, D, AT_BN) || !encode_operand_map(&mv, vc, kv_rows, D, AT_BN))
+        return "cuTensorMapEncodeTiled failed";
+    if (cudaFuncSetAttribute(prefill_attention_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<D>::SMEM) != cudaSuccess)
         return "cudaFuncSetAttribute failed";
     const float scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(D)));
-    prefill_attention_kernel<D><<<dim3((T + 63) / 64, nq), 128, smem, s>>>(q, kc, vc, out, plane, T, slot0, nq, group, head_stride, scale_log2);
+    prefill_attention_tc_kernel<D><<<dim3((T + AT_BM - 1) / AT_BM, nq), AT_THREADS, AttnCfg<D>::SMEM, s>>>(
+        mqh, mql, mk, mv, out, plane, T, slot0, nq, nq / nkv, max_context, scale_log2, wait_limit, error);
     return cudaGetLastError() == cudaSuccess ? nullptr : "prefill attention launch failed";
 }
 
@@ -710,8 +860,8 @@ const char *prefill_run(const PrefillModel &m, PrefillBuffers *b, const int32_t 
         if (const char *e = launch_gemm<EPI_QKV>(b->xn, x_plane, w.wqkv, n_qkv, g, m.num_sms, s)) return e;
         ++count;
         if (l == sh.n_layers - 1) break;   // the rest of the last layer feeds nothing that is kept
-        const char *e = d == 64 ? launch_attention<64>(b->q, kc, vc, b->attn, q_plane, n, slot0, nq, nq / nkv, head_stride, s)
-                                : launch_attention<128>(b->q, kc, vc, b->attn, q_plane, n, slot0, nq, nq / nkv, head_stride, s);
+        const char *e = d == 64 ? launch_attention_tc<64>(b->q, kc, vc, b->attn, q_plane, n, slot0, nq, nkv, m.max_context, b->wait_limit, b->error, s)
+                                : launch_attention_tc<128>(b->q, kc, vc, b->attn, q_plane, n, slot0, nq, nkv, m.max_context, b->wait_limit, b->error, s);
         if (e) return e;
         g.N = H; g.K = qd; g.resid = b->resid;
         if ((e = launch_gemm<EPI_RESID>(b->attn, q_plane, w.wo, H, g, m.num_sms, s))) return e;
