@@ -88,6 +88,16 @@ def test_prompt_on_the_1_5b_shape():
     run_case(CONFIGS["qwen2.5-1.5b"], 32, 200, 5, follow=False)
 
 
+def test_prompt_on_the_0_5b_shape():
+    """head_dim 64, 14 query heads on 2 kv heads, tied output layer; two query tiles and a ragged third."""
+    run_case(CONFIGS["qwen2.5-0.5b"], 10, 300, 6, follow=False)
+
+
+def test_prompt_on_the_7b_shape():
+    """28 query heads on 4 kv heads (groups of 7), H = 3584, F = 18944 (148 column tiles)."""
+    run_case(CONFIGS["qwen2.5-7b-32k"], 16, 70, 8, follow=False)
+
+
 def test_prefill_argument_checks():
     from paper_2604_27476_b200 import EdgefmError, Status
     cfg = CONFIGS["tiny"]
