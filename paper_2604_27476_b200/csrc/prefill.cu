@@ -174,7 +174,7 @@ __global__ void __launch_bounds__(256) prefill_rope_kernel(float2 *rope, int n, 
 // table (bf16 -> fp32) and written to the residual stream.  Thread 0 of the grid also records the new cache length.
 __global__ void __launch_bounds__(256) prefill_norm_kernel(float *resid, uint16_t *xn, size_t plane, const uint16_t *w, const uint16_t *embed,
                                                            const int *tokens, int n, int H, float eps, StepState *st, int new_len,
-                                                           int new_pos) {
+                                                           int new_pos, const float *part, int splits, size_t part_plane) {
     if (st && blockIdx.x == 0 && threadIdx.x == 0) {
         st->cur_len = new_len;
         st->next_position = new_pos;
@@ -199,6 +199,15 @@ __global__ void __launch_bounds__(256) prefill_norm_kernel(float *resid, uint16_
         } else {
             const float4 a = *reinterpret_cast<const float4 *>(x + j), c = *reinterpret_cast<const float4 *>(x + j + 4);
             v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = c.x; v[5] = c.y; v[6] = c.z; v[7] = c.w;
+            if (splits > 1) {   // the K-split partial sums of the contraction before: added in plane order, written back
+                for (int sp = 0; sp < splits; ++sp) {
+                    const float *q = part + sp * part_plane + static_cast<size_t>(row) * H + j;
+                    const float4 pa = *reinterpret_cast<const float4 *>(q), pc = *reinterpret_cast<const float4 *>(q + 4);
+                    v[0] += pa.x; v[1] += pa.y; v[2] += pa.z; v[3] += pa.w; v[4] += pc.x; v[5] += pc.y; v[6] += pc.z; v[7] += pc.w;
+                }
+                *reinterpret_cast<float4 *>(x + j) = make_float4(v[0], v[1], v[2], v[3]);
+                *reinterpret_cast<float4 *>(x + j + 4) = make_float4(v[4], v[5], v[6], v[7]);
+            }
         }
 #pragma unroll
         for (int i = 0; i < 8; ++i) ss = fmaf(v[i], v[i], ss);
@@ -236,12 +245,16 @@ struct GemmArgs {
     long long head_stride;
     // O / down
     float *resid;             // [M][N]
+    int splits;               // K split into this many units per output tile (1 = none).  With a split the units write their
+    float *part;              // partial sums to part[split][..][N] (planes `part_plane` elements apart) instead of adding to resid;
+    size_t part_plane;        // the norm kernel that follows adds the planes to the residual stream in a fixed order.
     // gate/up
     uint16_t *act;            // [2][..][N]: hi and lo planes
     size_t act_plane;
 };
 
 constexpr int PF_BM = 128, PF_BK = 64;
+constexpr int PF_SPLIT_MAX = 4;               // K splits of a contraction that adds to the residual stream
 
 // Tile shapes.  PF_NARROW: 128 output columns, 4 stages of 48 KB.  PF_WIDE: 256 output columns, 3 stages of 64 KB: per k-block
 // 64 KB of operands feed twice the multiplies of a narrow tile's 48 KB, which matters because operand delivery from L2, not
@@ -271,8 +284,18 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
     uint8_t *tiles = pf_dyn + ((1024u - (smem_u32(pf_dyn) & 1023u)) & 1023u);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m_tiles = (g.M + PF_BM - 1) / PF_BM, n_tiles = (g.N + N_STEP - 1) / N_STEP;
-    const int my_tiles = (m_tiles * n_tiles - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
     const int KB = (g.K + PF_BK - 1) / PF_BK;
+    const int splits = EPI == EPI_RESID ? g.splits : 1;
+    const int my_tiles = (m_tiles * n_tiles * splits - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
+    // unit u of the grid-wide list: row tile u % m_tiles (neighbouring CTAs share a weight tile), then the K split, then the column tile
+    auto unit_of = [&](int i, int &m0, int &n0, int &kb0, int &kb1) {
+        const int u = blockIdx.x + i * gridDim.x, rest = u / m_tiles, sp = rest % splits;
+        m0 = (u % m_tiles) * PF_BM;
+        n0 = (rest / splits) * N_STEP;
+        kb0 = sp * KB / splits;
+        kb1 = (sp + 1) * KB / splits;
+        return sp;
+    };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::STAGES; ++s) { mbar_init(&full_bar[s], 1 + g.extra_arrivals); mbar_init(&empty_bar[s], 1); }
@@ -294,8 +317,9 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
         bool ok = true;
         int issued = 0;
         for (int i = 0, it = 0; i < my_tiles && ok; ++i) {
-          const int tile = blockIdx.x + i * gridDim.x, m0 = (tile % m_tiles) * PF_BM, n0 = (tile / m_tiles) * N_STEP;
-          for (int kb = 0; kb < KB; ++kb, ++it) {
+          int m0, n0, kb0, kb1;
+          unit_of(i, m0, n0, kb0, kb1);
+          for (int kb = kb0; kb < kb1; ++kb, ++it) {
             const int s = it % C::STAGES;
             if (it >= C::STAGES && !mbar_wait(&empty_bar[s], ((it / C::STAGES) - 1) & 1, &abort_flag, g.wait_limit)) { ok = false; break; }
             uint8_t *a = tiles + s * C::STAGE_BYTES, *b = a + 2 * C::A_BYTES;
@@ -321,7 +345,9 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
           if (i >= 2) ok = mbar_wait(&acc_empty[buf], ((i >> 1) - 1) & 1, &abort_flag, g.wait_limit);   // its epilogue has read it
           if (!ok) break;
           tc_fence_after();
-          for (int kb = 0; kb < KB; ++kb, ++it) {
+          int m0, n0, kb0, kb1;
+          unit_of(i, m0, n0, kb0, kb1);
+          for (int kb = kb0; kb < kb1; ++kb, ++it) {
             const int s = it % C::STAGES;
             ok = mbar_wait(&full_bar[s], (it / C::STAGES) & 1, &abort_flag, g.wait_limit);
             if (!ok) break;
@@ -329,7 +355,7 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
             const uint32_t a = smem_u32(tiles + s * C::STAGE_BYTES), b = a + 2 * C::A_BYTES;
             const uint64_t da = umma_desc_sw128(a), dl = umma_desc_sw128(a + C::A_BYTES), db = umma_desc_sw128(b);
 #pragma unroll
-            for (int k = 0; k < PF_BK / 16; ++k) umma_bf16(acc, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0);
+            for (int k = 0; k < PF_BK / 16; ++k) umma_bf16(acc, da + 2 * k, db + 2 * k, idesc, ((kb - kb0) | k) != 0);
 #pragma unroll
             for (int k = 0; k < PF_BK / 16; ++k) umma_bf16(acc, dl + 2 * k, db + 2 * k, idesc, 1);
             umma_commit(&empty_bar[s]);      // the stage is free again when these have read it
@@ -344,7 +370,8 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
     } else if (warp >= 2) {                  // epilogue: warp w may read lanes 32 (w % 4) .. + 31 of tensor memory
       const int quarter = warp & 3;
       for (int i = 0; i < my_tiles; ++i) {
-        const int tile = blockIdx.x + i * gridDim.x, m0 = (tile % m_tiles) * PF_BM, n0 = (tile / m_tiles) * N_STEP, buf = i & 1;
+        int m0, n0, kb0, kb1;
+        const int sp = unit_of(i, m0, n0, kb0, kb1), buf = i & 1;
         const bool ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[buf], (i >> 1) & 1, &abort_flag, g.wait_limit));   // warp-uniform: tcgen05.ld is .aligned
         if (!ok) break;
         tc_fence_after();
@@ -359,7 +386,12 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
                     float v[32];
                     tmem_ld32(trow + c * 32, v);
                     tmem_ld_wait();
-                    if (live) {
+                    if (live && splits > 1) {   // a partial sum: stored, added to the stream by the norm kernel
+                        float4 *p = reinterpret_cast<float4 *>(g.part + sp * g.part_plane + static_cast<size_t>(row) * g.N + n);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            if (n + 4 * i + 3 < g.N) p[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                    } else if (live) {
                         float4 *p = reinterpret_cast<float4 *>(g.resid + static_cast<size_t>(row) * g.N + n);
 #pragma unroll
                         for (int i = 0; i < 8; ++i)
@@ -764,26 +796,40 @@ const char *launch_gemm_cfg(const CUtensorMap &ma, const CUtensorMap &ml, const 
     if (cudaFuncSetAttribute(prefill_gemm_kernel<EPI, SHAPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM) != cudaSuccess)
         return "cudaFuncSetAttribute failed";
     const int n_step = EPI == EPI_SWIGLU ? 128 : C::BN;
-    const int tiles = ((g.N + n_step - 1) / n_step) * ((g.M + PF_BM - 1) / PF_BM);
-    prefill_gemm_kernel<EPI, SHAPE><<<tiles < num_sms ? tiles : num_sms, 192, C::SMEM, s>>>(ma, ml, mb, g);
+    const int units = ((g.N + n_step - 1) / n_step) * ((g.M + PF_BM - 1) / PF_BM) * (EPI == EPI_RESID ? g.splits : 1);
+    prefill_gemm_kernel<EPI, SHAPE><<<units < num_sms ? units : num_sms, 192, C::SMEM, s>>>(ma, ml, mb, g);
     return cudaGetLastError() == cudaSuccess ? nullptr : "prefill GEMM launch failed";
 }
 
-// Shape choice: the rounds the SMs need (tiles / SMs, rounded up) times the relative cost of a tile (a wide tile does twice
-// the work of a narrow one for 1.33 x the operand traffic: 1.6), whichever is smaller.
+// Shape and K split.  Cost model: the rounds the SMs need (units / SMs, rounded up) times the cost of a unit; a wide tile does
+// twice the work of a narrow one for 1.33 x the operand traffic (1.6), a K split divides a unit's cost and adds a little for
+// the partial sums (5 %).  Only the contractions that add to the residual stream split (their partial sums are added by the
+// norm kernel that follows, in a fixed order); a split keeps at least 12 k-blocks per unit and is considered only when the
+// unsplit tiles do not fill the SMs once (with more tiles the partial-sum traffic costs more than the better balance gains:
+// 7B shape, 2048 tokens, 48.0 -> 50.7 ms).
 template <int EPI>
-const char *launch_gemm(const uint16_t *a, size_t a_plane, const void *w, long long w_rows, const GemmArgs &g, int num_sms, cudaStream_t s) {
+const char *launch_gemm(const uint16_t *a, size_t a_plane, const void *w, long long w_rows, GemmArgs &g, int num_sms, cudaStream_t s) {
     CUtensorMap ma, ml, mb;
     if (!encode_operand_map(&ma, a, g.M, g.K) || !encode_operand_map(&ml, a + a_plane, g.M, g.K) || !encode_operand_map(&mb, w, w_rows, g.K))
         return "cuTensorMapEncodeTiled failed";
-    const int m_tiles = (g.M + PF_BM - 1) / PF_BM;
+    const int m_tiles = (g.M + PF_BM - 1) / PF_BM, kb = (g.K + PF_BK - 1) / PF_BK;
+    g.splits = 1;
     if constexpr (EPI == EPI_SWIGLU) {
         return launch_gemm_cfg<EPI, PF_WIDE>(ma, ml, mb, g, num_sms, s);
     } else {
-        const int wide = ((g.N + 255) / 256) * m_tiles, narrow = ((g.N + 127) / 128) * m_tiles;
-        const int rounds_wide = (wide + num_sms - 1) / num_sms, rounds_narrow = (narrow + num_sms - 1) / num_sms;
-        if (rounds_wide * 16 <= rounds_narrow * 10) return launch_gemm_cfg<EPI, PF_WIDE>(ma, ml, mb, g, num_sms, s);
-        return launch_gemm_cfg<EPI, PF_NARROW>(ma, ml, mb, g, num_sms, s);
+        const int tiles[2] = {((g.N + 127) / 128) * m_tiles, ((g.N + 255) / 256) * m_tiles};
+        const double cost[2] = {1.0, 1.6};
+        int best_shape = 0, best_split = 1;
+        double best = 1e30;
+        for (int shape = 0; shape < 2; ++shape)
+            for (int sp = 1; sp <= (EPI == EPI_RESID ? PF_SPLIT_MAX : 1); ++sp) {
+                if (sp > 1 && (kb / sp < 12 || tiles[shape] > num_sms)) break;   // split only grids that leave SMs idle in their one round
+                const int units = tiles[shape] * sp;
+                const double t = ((units + num_sms - 1) / num_sms) * cost[shape] / sp * (sp > 1 ? 1.05 : 1.0);
+                if (t < best - 1e-9) { best = t; best_shape = shape; best_split = sp; }
+            }
+        g.splits = best_split;
+        return best_shape ? launch_gemm_cfg<EPI, PF_WIDE>(ma, ml, mb, g, num_sms, s) : launch_gemm_cfg<EPI, PF_NARROW>(ma, ml, mb, g, num_sms, s);
     }
 }
 
@@ -807,7 +853,7 @@ const char *launch_attention_tc(const uint16_t *q, const uint16_t *kc, const uin
 
 size_t prefill_buffer_bytes(const edgefm_shape &sh, int chunk) {
     const size_t c = static_cast<size_t>(chunk), qd = static_cast<size_t>(sh.n_q_heads) * sh.head_dim;
-    return c * sh.hidden * 4 + c * sh.hidden * 4 + 2 * c * qd * 4 + c * sh.ffn * 4 + c * (sh.head_dim / 2) * 8 + c * 4 + 256;
+    return c * sh.hidden * 4 * (1 + PF_SPLIT_MAX) + c * sh.hidden * 4 + 2 * c * qd * 4 + c * sh.ffn * 4 + c * (sh.head_dim / 2) * 8 + c * 4 + 256;
 }
 
 cudaError_t prefill_alloc(PrefillBuffers *b, const edgefm_shape &sh, int chunk) {
@@ -815,6 +861,7 @@ cudaError_t prefill_alloc(PrefillBuffers *b, const edgefm_shape &sh, int chunk) 
     cudaError_t e;
     if ((e = cudaMalloc(&b->resid, c * sh.hidden * 4)) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->xn, c * sh.hidden * 4)) != cudaSuccess) return e;
+    if ((e = cudaMalloc(&b->part, c * sh.hidden * 4 * PF_SPLIT_MAX)) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->q, c * qd * 4)) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->attn, c * qd * 4)) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->act, c * sh.ffn * 4)) != cudaSuccess) return e;
@@ -827,7 +874,7 @@ cudaError_t prefill_alloc(PrefillBuffers *b, const edgefm_shape &sh, int chunk) 
 }
 
 void prefill_free(PrefillBuffers *b) {
-    cudaFree(b->resid); cudaFree(b->xn); cudaFree(b->q); cudaFree(b->attn); cudaFree(b->act); cudaFree(b->rope);
+    cudaFree(b->resid); cudaFree(b->xn); cudaFree(b->part); cudaFree(b->q); cudaFree(b->attn); cudaFree(b->act); cudaFree(b->rope);
     cudaFree(b->tokens); cudaFree(b->error);
     *b = PrefillBuffers{};
 }
@@ -845,7 +892,7 @@ const char *prefill_run(const PrefillModel &m, PrefillBuffers *b, const int32_t 
     const int norm_grid = (n + 7) / 8;
     prefill_norm_kernel<<<norm_grid, 256, 0, s>>>(b->resid, b->xn, x_plane, static_cast<const uint16_t *>(m.layers[0].input_norm),
                                                   static_cast<const uint16_t *>(m.embed), b->tokens, n, H, sh.rms_eps, m.state,
-                                                  slot0 + n, position + n);
+                                                  slot0 + n, position + n, nullptr, 0, 0);
     count += 2;
     for (int l = 0; l < sh.n_layers; ++l) {
         const edgefm_layer_weights &w = m.layers[l];
@@ -863,16 +910,16 @@ const char *prefill_run(const PrefillModel &m, PrefillBuffers *b, const int32_t 
         const char *e = d == 64 ? launch_attention_tc<64>(b->q, kc, vc, b->attn, q_plane, n, slot0, nq, nkv, m.max_context, b->wait_limit, b->error, s)
                                 : launch_attention_tc<128>(b->q, kc, vc, b->attn, q_plane, n, slot0, nq, nkv, m.max_context, b->wait_limit, b->error, s);
         if (e) return e;
-        g.N = H; g.K = qd; g.resid = b->resid;
+        g.N = H; g.K = qd; g.resid = b->resid; g.part = b->part; g.part_plane = x_plane;
         if ((e = launch_gemm<EPI_RESID>(b->attn, q_plane, w.wo, H, g, m.num_sms, s))) return e;
         prefill_norm_kernel<<<norm_grid, 256, 0, s>>>(b->resid, b->xn, x_plane, static_cast<const uint16_t *>(w.post_norm), nullptr, nullptr, n, H,
-                                                      sh.rms_eps, nullptr, 0, 0);
+                                                      sh.rms_eps, nullptr, 0, 0, b->part, g.splits, x_plane);
         g.N = F; g.K = H; g.act = b->act; g.act_plane = f_plane;
         if ((e = launch_gemm<EPI_SWIGLU>(b->xn, x_plane, w.w_gate_up, 2LL * F, g, m.num_sms, s))) return e;
         g.N = H; g.K = F;
         if ((e = launch_gemm<EPI_RESID>(b->act, f_plane, w.w_down, H, g, m.num_sms, s))) return e;
         prefill_norm_kernel<<<norm_grid, 256, 0, s>>>(b->resid, b->xn, x_plane, static_cast<const uint16_t *>(m.layers[l + 1].input_norm), nullptr,
-                                                      nullptr, n, H, sh.rms_eps, nullptr, 0, 0);
+                                                      nullptr, n, H, sh.rms_eps, nullptr, 0, 0, b->part, g.splits, x_plane);
         count += 6;
     }
     if (cudaGetLastError() != cudaSuccess) return "prefill kernel launch failed";
