@@ -294,6 +294,11 @@ edgefm_status edgefm_debug_set_wait_limit(edgefm_ctx *ctx, uint32_t limit_ns, in
  * into the bound without any fault.  Host only. */
 edgefm_status edgefm_debug_set_prefill_wait(edgefm_ctx *ctx, uint32_t polls, int32_t extra_arrivals);
 
+/* How edgefm_prefill tiles a contraction of [M tokens x K] x [K x N] on num_sms SMs: out2 = {1 = 256-column output tiles
+ * (0 = 128), K units per output tile}.  epilogue: 0 = QKV, 1 = added to the residual stream (O and down projection; only
+ * these split K), 2 = gate/up (always wide, never split).  Host only: for checking the planner without a GPU. */
+edgefm_status edgefm_debug_prefill_plan(int32_t epilogue, int32_t M, int32_t N, int32_t K, int32_t num_sms, int32_t *out2);
+
 /* Host-only check of the planner: the tile schedule of one weight-streaming operator (kind: 0 QKV pairs, 1 residual rows,
  * 2 gate/up pairs, 3 output-layer rows; units rows or pairs; K columns; head_half = head_dim / 2 for kind 0) for n_ctas CTAs
  * of n_warps consumer warps whose ring slots hold slot_rows rows.  tiles_out receives one 64-bit descriptor per tile, CTA by

@@ -51,7 +51,7 @@ class _Weights(ctypes.Structure):
 
 EXPORTS = ("edgefm_create", "edgefm_prefill_kv", "edgefm_decode_step", "edgefm_destroy", "edgefm_get_length",
            "edgefm_export_kv", "edgefm_get_launches_per_step", "edgefm_last_error", "edgefm_version",
-           "edgefm_sync_status", "edgefm_debug_profile", "edgefm_debug_set_wait_limit", "edgefm_debug_set_prefill_wait", "edgefm_debug_plan", "edgefm_debug_plan_operator", "edgefm_decode_step_static", "edgefm_set_vocab_subset",
+           "edgefm_sync_status", "edgefm_debug_profile", "edgefm_debug_set_wait_limit", "edgefm_debug_set_prefill_wait", "edgefm_debug_prefill_plan", "edgefm_debug_plan", "edgefm_debug_plan_operator", "edgefm_decode_step_static", "edgefm_set_vocab_subset",
            "edgefm_append_kv", "edgefm_create_with_options", "edgefm_export_kv_int8", "edgefm_verify_block", "edgefm_sync_length", "edgefm_prefill_tokens", "edgefm_prefill")
 
 
@@ -217,6 +217,16 @@ def edgefm_set_vocab_subset(ctx, token_ids, stream=None):
 
 def edgefm_sync_status(ctx, stream=None):
     _check(load_library().edgefm_sync_status(ctx, stream), ctx)
+
+
+def edgefm_debug_prefill_plan(epilogue, M, N, K, num_sms=148):
+    """(wide, splits) the prefill planner gives a contraction (host only)."""
+    L = load_library()
+    L.edgefm_debug_prefill_plan.restype = ctypes.c_int
+    L.edgefm_debug_prefill_plan.argtypes = [ctypes.c_int32] * 5 + [ctypes.POINTER(ctypes.c_int32)]
+    out = (ctypes.c_int32 * 2)()
+    _check(L.edgefm_debug_prefill_plan(epilogue, M, N, K, num_sms, out), None)
+    return int(out[0]), int(out[1])
 
 
 def edgefm_debug_set_prefill_wait(ctx, polls, extra_arrivals=0):

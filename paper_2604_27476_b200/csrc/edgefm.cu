@@ -1004,6 +1004,15 @@ edgefm_status edgefm_debug_set_prefill_wait(edgefm_ctx *ctx, uint32_t polls, int
     return EDGEFM_OK;
 }
 
+edgefm_status edgefm_debug_prefill_plan(int32_t epilogue, int32_t M, int32_t N, int32_t K, int32_t num_sms, int32_t *out2) {
+    if (!out2 || epilogue < 0 || epilogue > 2 || M < 1 || N < 1 || K < 1 || num_sms < 1) return EDGEFM_ERR_INVALID_ARG;
+    int wide = 0, splits = 0;
+    prefill_plan_contraction(epilogue, M, N, K, num_sms, &wide, &splits);
+    out2[0] = wide;
+    out2[1] = splits;
+    return EDGEFM_OK;
+}
+
 edgefm_status edgefm_export_kv(edgefm_ctx *ctx, void *k_out, void *v_out, void *stream) {
     if (!ctx) return EDGEFM_ERR_INVALID_ARG;
     if (!k_out || !v_out) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "null output");

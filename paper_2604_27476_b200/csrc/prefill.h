@@ -38,6 +38,10 @@ struct PrefillModel {
     int num_sms;
 };
 
+// Tile shape and K split a contraction of [M x K] x [K x N] gets on num_sms SMs (host logic, no device needed).
+// epilogue: 0 = QKV, 1 = added to the residual stream (O, down), 2 = gate/up.  *wide: 256-column tiles; *splits: K units per tile.
+void prefill_plan_contraction(int epilogue, int M, int N, int K, int num_sms, int *wide, int *splits);
+
 // Bytes the work buffers of a pass over `chunk` tokens take.
 size_t prefill_buffer_bytes(const edgefm_shape &sh, int chunk);
 // Allocate / free.  Returns a CUDA error.
