@@ -48,12 +48,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait: gives up after `limit` polls or as soon as another thread of the CTA has given up.
-template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, uint32_t limit) {
     for (uint32_t i = 0; i < limit; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 63u) == 63u && *abort_flag) return false;
-        if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);   // a polling lane takes issue slots from the warps that share its scheduler
     }
     *abort_flag = 1;
     return false;
@@ -522,9 +520,6 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
 //   shared memory: Q 2 x D/64 x 16 KB | 2 stages x (K D/64 x 8 KB, V D/64 x 8 KB) | 2 x P (2 x 16 KB)
 constexpr int AT_BM = 128, AT_BN = 64, AT_PARTS = 2;
 constexpr int AT_THREADS = 64 + 128 * AT_PARTS;
-#ifndef AT_POLL_NS
-#define AT_POLL_NS 40
-#endif
 
 // B operand in MN-major form for P V: the V tile is D/64 blocks of [64 keys][64 d] (128-byte rows, 128-byte swizzle).  N (= d)
 // runs along a row, K (= keys) across rows: groups of 8 keys are 1024 bytes apart (stride byte offset), the 64-column blocks
@@ -591,7 +586,7 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
         int issued = 0;
         for (int j = 0; j < nb; ++j) {
             const int st = j & 1;
-            if (j >= 2 && !mbar_wait<AT_POLL_NS>(&kv_empty[st], ((j >> 1) - 1) & 1, &abort_flag, wait_limit)) break;
+            if (j >= 2 && !mbar_wait(&kv_empty[st], ((j >> 1) - 1) & 1, &abort_flag, wait_limit)) break;
             uint8_t *k = skv + st * (C::K_BYTES + C::V_BYTES), *v = k + C::K_BYTES;
             mbar_expect_tx(&kv_full[st], C::K_BYTES + C::V_BYTES);
             for (int kb = 0; kb < C::KBLK; ++kb) {
@@ -602,8 +597,8 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
         }
         if (abort_flag) {   // giving up: the copies in flight must land before the shared memory is released
             int dummy = 0;
-            mbar_wait<AT_POLL_NS>(&q_full, 0, &dummy, wait_limit);
-            for (int j = issued > 2 ? issued - 2 : 0; j < issued; ++j) mbar_wait<AT_POLL_NS>(&kv_full[j & 1], (j >> 1) & 1, &dummy, wait_limit);
+            mbar_wait(&q_full, 0, &dummy, wait_limit);
+            for (int j = issued > 2 ? issued - 2 : 0; j < issued; ++j) mbar_wait(&kv_full[j & 1], (j >> 1) & 1, &dummy, wait_limit);
         }
     } else if (warp == 1 && lane == 0) {     // issuer
         constexpr uint32_t idesc_s = umma_idesc_bf16(AT_BM, AT_BN);
@@ -621,19 +616,19 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
                 }
             umma_commit(&s_full[j & 1]);
         };
-        bool ok = mbar_wait<AT_POLL_NS>(&q_full, 0, &abort_flag, wait_limit) && mbar_wait<AT_POLL_NS>(&kv_full[0], 0, &abort_flag, wait_limit);
+        bool ok = mbar_wait(&q_full, 0, &abort_flag, wait_limit) && mbar_wait(&kv_full[0], 0, &abort_flag, wait_limit);
         if (ok) { tc_fence_after(); issue_s(0); }
         for (int j = 0; j < nb && ok; ++j) {
             if (j + 1 < nb) {                // the next block's scores, under this block's softmax
                 const int st = (j + 1) & 1;
-                ok = mbar_wait<AT_POLL_NS>(&kv_full[st], ((j + 1) >> 1) & 1, &abort_flag, wait_limit);
-                if (ok && j + 1 >= 2) ok = mbar_wait<AT_POLL_NS>(&s_empty[st], (((j + 1) >> 1) - 1) & 1, &abort_flag, wait_limit);
+                ok = mbar_wait(&kv_full[st], ((j + 1) >> 1) & 1, &abort_flag, wait_limit);
+                if (ok && j + 1 >= 2) ok = mbar_wait(&s_empty[st], (((j + 1) >> 1) - 1) & 1, &abort_flag, wait_limit);
                 if (!ok) break;
                 tc_fence_after();
                 issue_s(j + 1);
             }
-            ok = mbar_wait<AT_POLL_NS>(&p_full[j & 1], (j >> 1) & 1, &abort_flag, wait_limit);
-            if (ok && j >= 2) ok = mbar_wait<AT_POLL_NS>(&o_empty[j & 1], ((j >> 1) - 1) & 1, &abort_flag, wait_limit);
+            ok = mbar_wait(&p_full[j & 1], (j >> 1) & 1, &abort_flag, wait_limit);
+            if (ok && j >= 2) ok = mbar_wait(&o_empty[j & 1], ((j >> 1) - 1) & 1, &abort_flag, wait_limit);
             if (!ok) break;
             tc_fence_after();
             const uint32_t v = smem_u32(skv + (j & 1) * (C::K_BYTES + C::V_BYTES) + C::K_BYTES);
@@ -651,10 +646,10 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
         if (!ok) {
             int dummy = 0;
             umma_commit(&drain_bar);
-            mbar_wait<AT_POLL_NS>(&drain_bar, 0, &dummy, wait_limit);
+            mbar_wait(&drain_bar, 0, &dummy, wait_limit);
         }
     }
-    else if (warp >= 2) {                    // softmax: AT_PARTS threads per query row (= lane of tensor memory), 16 keys of a block each
+    else if (warp >= 2) {                    // softmax: AT_PARTS threads per query row (= lane of tensor memory), AT_BN / AT_PARTS keys of a block each
         const int quarter = warp & 3, part = (warp - 2) >> 2, row = quarter * 32 + lane;
         const uint32_t trow = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
         const int qi = slot0 + t0 + row;     // cache slot of this query: it sees the keys 0 .. qi
