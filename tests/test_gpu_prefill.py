@@ -121,3 +121,48 @@ def test_prefill_argument_checks():
         assert ei.value.status == Status.ERR_INVALID_ARG
     finally:
         pair.close()
+
+
+def test_prefill_then_block_verification_and_pruned_vocabulary():
+    """edgefm_prefill on a context built for block verification, followed by a verified block; then on a context whose output
+    layer is pruned (the logits of the prompt's last token are the subset's)."""
+    import torch
+    cfg = CONFIGS["tiny"].with_(qkv_bias=True)
+    T0, n = 6, 90
+    pair = Pair(cfg, cache_len=T0, max_context=T0 + n + 8, block_tokens=4)
+    try:
+        toks = np.random.default_rng(21).integers(0, cfg.vocab, n).tolist()
+        for i, t in enumerate(toks):
+            ref_logits, ref_next = pair.oracle.step(t, T0 + i)
+        pair.ctx.prefill(toks, T0)
+        torch.cuda.synchronize()
+        pair.ctx.sync_status()
+        assert_logits_close(pair.ctx.logits.cpu().numpy(), ref_logits, "last prompt token on a block context")
+        if top2_margin(ref_logits) > TOKEN_MARGIN:
+            # a block behind the prompt: the token the device holds (-1) and three arbitrary proposals
+            block = [ref_next, 5, 7, 9]
+            ref_rows, ref_acc, ref_nx = pair.oracle.verify_block(block, T0 + n)
+            pair.ctx.verify_block([-1] + block[1:], -1)
+            torch.cuda.synchronize()
+            assert int(pair.ctx.n_accepted.item()) == ref_acc
+            assert pair.ctx.sync_length() == T0 + n + ref_acc == pair.oracle.cur_len
+            got = pair.ctx.block_logits.cpu().numpy()
+            for t in range(ref_acc):
+                assert_logits_close(got[t], ref_rows[t], f"block row {t} behind the prompt")
+            if top2_margin(ref_rows[ref_acc - 1]) > TOKEN_MARGIN:
+                assert int(pair.ctx.next_token.item()) == ref_nx
+    finally:
+        pair.close()
+    pair = Pair(cfg, cache_len=T0, max_context=T0 + n + 2)
+    try:
+        ids = list(range(3, cfg.vocab, 5))
+        pair.ctx.set_vocab_subset(ids)
+        for i, t in enumerate(toks):
+            ref_logits, _ = pair.oracle.step(t, T0 + i)
+        pair.ctx.prefill(toks, T0)
+        torch.cuda.synchronize()
+        got = pair.ctx.logits.cpu().numpy()[:len(ids)]
+        assert_logits_close(got, ref_logits[ids], "last prompt token, pruned output layer")
+        assert int(pair.ctx.next_token.item()) == ids[int(np.argmax(ref_logits[ids]))] or top2_margin(ref_logits[ids]) <= TOKEN_MARGIN
+    finally:
+        pair.close()
