@@ -170,9 +170,9 @@ __global__ void __launch_bounds__(256) prefill_rope_kernel(float2 *rope, int n, 
     rope[i] = make_float2(static_cast<float>(cs), static_cast<float>(sn));
 }
 
-// One warp per row: y = x * rsqrt(mean(x^2) + eps) * w, stored as two bf16 planes (hi, lo; `plane` elements apart).  With `embed` the row is first fetched from the embedding
+// One CTA of 128 threads per row: y = x * rsqrt(mean(x^2) + eps) * w, stored as two bf16 planes (hi, lo; `plane` elements apart).  With `embed` the row is first fetched from the embedding
 // table (bf16 -> fp32) and written to the residual stream.  Thread 0 of the grid also records the new cache length.
-__global__ void __launch_bounds__(256) prefill_norm_kernel(float *resid, uint16_t *xn, size_t plane, const uint16_t *w, const uint16_t *embed,
+__global__ void __launch_bounds__(128) prefill_norm_kernel(float *resid, uint16_t *xn, size_t plane, const uint16_t *w, const uint16_t *embed,
                                                            const int *tokens, int n, int H, float eps, StepState *st, int new_len,
                                                            int new_pos, const float *part, int splits, size_t part_plane) {
     if (st && blockIdx.x == 0 && threadIdx.x == 0) {
@@ -180,15 +180,14 @@ __global__ void __launch_bounds__(256) prefill_norm_kernel(float *resid, uint16_
         st->next_position = new_pos;
         st->status = 0;
     }
-    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (row >= n) return;
+    __shared__ float red[4];
+    const int row = blockIdx.x, tid = threadIdx.x;
     float *x = resid + static_cast<size_t>(row) * H;
     uint16_t *y = xn + static_cast<size_t>(row) * H;
     // H is a multiple of 8: eight values per lane and round, 16- and 32-byte accesses
     const uint16_t *e = embed ? embed + static_cast<size_t>(tokens[row]) * H : nullptr;
     float ss = 0.f;
-    for (int j = lane * 8; j < H; j += 256) {
+    for (int j = tid * 8; j < H; j += 1024) {
         float v[8];
         if (e) {
             const uint4 b = *reinterpret_cast<const uint4 *>(e + j);
@@ -213,8 +212,11 @@ __global__ void __launch_bounds__(256) prefill_norm_kernel(float *resid, uint16_
         for (int i = 0; i < 8; ++i) ss = fmaf(v[i], v[i], ss);
     }
     ss = warp_sum(ss);
+    if ((tid & 31) == 0) red[tid >> 5] = ss;
+    __syncthreads();
+    ss = (red[0] + red[1]) + (red[2] + red[3]);
     const float r = rsqrtf(ss / static_cast<float>(H) + eps);
-    for (int j = lane * 8; j < H; j += 256) {
+    for (int j = tid * 8; j < H; j += 1024) {
         const float4 a = *reinterpret_cast<const float4 *>(x + j), c = *reinterpret_cast<const float4 *>(x + j + 4);
         const uint4 wb = *reinterpret_cast<const uint4 *>(w + j);
         uint4 hi, lo;
@@ -897,8 +899,8 @@ const char *prefill_run(const PrefillModel &m, PrefillBuffers *b, const int32_t 
     int count = 0;
     if (cudaMemcpyAsync(b->tokens, tokens, static_cast<size_t>(n) * 4, cudaMemcpyHostToDevice, s) != cudaSuccess) return "token upload failed";
     prefill_rope_kernel<<<(n * (d / 2) + 255) / 256, 256, 0, s>>>(b->rope, n, d / 2, position, static_cast<double>(sh.rope_theta));
-    const int norm_grid = (n + 7) / 8;
-    prefill_norm_kernel<<<norm_grid, 256, 0, s>>>(b->resid, b->xn, x_plane, static_cast<const uint16_t *>(m.layers[0].input_norm),
+    const int norm_grid = n;
+    prefill_norm_kernel<<<norm_grid, 128, 0, s>>>(b->resid, b->xn, x_plane, static_cast<const uint16_t *>(m.layers[0].input_norm),
                                                   static_cast<const uint16_t *>(m.embed), b->tokens, n, H, sh.rms_eps, m.state,
                                                   slot0 + n, position + n, nullptr, 0, 0);
     count += 2;
@@ -920,13 +922,13 @@ const char *prefill_run(const PrefillModel &m, PrefillBuffers *b, const int32_t 
         if (e) return e;
         g.N = H; g.K = qd; g.resid = b->resid; g.part = b->part; g.part_plane = x_plane;
         if ((e = launch_gemm<EPI_RESID>(b->attn, q_plane, w.wo, H, g, m.num_sms, s))) return e;
-        prefill_norm_kernel<<<norm_grid, 256, 0, s>>>(b->resid, b->xn, x_plane, static_cast<const uint16_t *>(w.post_norm), nullptr, nullptr, n, H,
+        prefill_norm_kernel<<<norm_grid, 128, 0, s>>>(b->resid, b->xn, x_plane, static_cast<const uint16_t *>(w.post_norm), nullptr, nullptr, n, H,
                                                       sh.rms_eps, nullptr, 0, 0, b->part, g.splits, x_plane);
         g.N = F; g.K = H; g.act = b->act; g.act_plane = f_plane;
         if ((e = launch_gemm<EPI_SWIGLU>(b->xn, x_plane, w.w_gate_up, 2LL * F, g, m.num_sms, s))) return e;
         g.N = H; g.K = F;
         if ((e = launch_gemm<EPI_RESID>(b->act, f_plane, w.w_down, H, g, m.num_sms, s))) return e;
-        prefill_norm_kernel<<<norm_grid, 256, 0, s>>>(b->resid, b->xn, x_plane, static_cast<const uint16_t *>(m.layers[l + 1].input_norm), nullptr,
+        prefill_norm_kernel<<<norm_grid, 128, 0, s>>>(b->resid, b->xn, x_plane, static_cast<const uint16_t *>(m.layers[l + 1].input_norm), nullptr,
                                                       nullptr, n, H, sh.rms_eps, nullptr, 0, 0, b->part, g.splits, x_plane);
         count += 6;
     }
