@@ -521,7 +521,7 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
 //   tensor memory: S0 [0, 64), S1 [64, 128), O0 [128, 128 + D), O1 [128 + D, 128 + 2 D)
 //   shared memory: Q 2 x D/64 x 16 KB | 2 stages x (K D/64 x 8 KB, V D/64 x 8 KB) | 2 x P (2 x 16 KB)
 constexpr int AT_BM = 128, AT_BN = 64, AT_PARTS = 2;
-constexpr int AT_THREADS = 64 + 128 * AT_PARTS;
+constexpr int AT_THREADS = 96 + 128 * AT_PARTS;   // producer, two issuers, softmax warps
 
 // B operand in MN-major form for P V: the V tile is D/64 blocks of [64 keys][64 d] (128-byte rows, 128-byte swizzle).  N (= d)
 // runs along a row, K (= keys) across rows: groups of 8 keys are 1024 bytes apart (stride byte offset), the 64-column blocks
@@ -549,23 +549,24 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
                                                                    float scale_log2, uint32_t wait_limit, int *error) {
     using C = AttnCfg<D>;
     extern __shared__ uint8_t at_tc_dyn[];
-    __shared__ uint64_t q_full, kv_full[2], kv_empty[2], s_full[2], s_empty[2], p_full[2], p_empty[2], o_full[2], o_empty[2], drain_bar, pair_bar[4];
+    __shared__ uint64_t q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], s_empty[2], p_full[2], p_empty[2], o_full[2], o_empty[2], drain_bar[2], pair_bar[4];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ float xchg[2][AT_PARTS][AT_BM];      // row maxima / sums passed between the two threads of a row
     uint8_t *base = at_tc_dyn + ((1024u - (smem_u32(at_tc_dyn) & 1023u)) & 1023u);
     uint8_t *sq = base, *skv = sq + C::Q_BYTES, *sp = skv + 2 * (C::K_BYTES + C::V_BYTES);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int t0 = (gridDim.x - 1 - blockIdx.x) * AT_BM;      // long rows first
-    const int h = blockIdx.y, hk = h / group;
+    // grid (heads, query tiles): CTAs start in linear order, so every head's longest tile (the last queries) starts first
+    const int t0 = (gridDim.y - 1 - blockIdx.y) * AT_BM;
+    const int h = blockIdx.x, hk = h / group;
     const int last_key = slot0 + min(t0 + AT_BM - 1, T - 1);
     const int nb = last_key / AT_BN + 1;
 
     if (threadIdx.x == 0) {
         mbar_init(&q_full, 1);
-        for (int i = 0; i < 2; ++i) { mbar_init(&kv_full[i], 1); mbar_init(&kv_empty[i], 1); mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 4 * AT_PARTS); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1); mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 4 * AT_PARTS); }
         for (int i = 0; i < 2; ++i) { mbar_init(&p_full[i], 4 * AT_PARTS); mbar_init(&p_empty[i], 1); mbar_init(&o_full[i], 1); mbar_init(&o_empty[i], 4 * AT_PARTS); }
-        mbar_init(&drain_bar, 1);
+        mbar_init(&drain_bar[0], 1); mbar_init(&drain_bar[1], 1);
         for (int i = 0; i < 4; ++i) mbar_init(&pair_bar[i], AT_PARTS);
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -585,28 +586,39 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
             tma_load_2d(sq + kb * AT_BM * 128, &map_q_hi, h * D + kb * 64, t0, &q_full);
             tma_load_2d(sq + (C::KBLK + kb) * AT_BM * 128, &map_q_lo, h * D + kb * 64, t0, &q_full);
         }
+        // K and V of a block have barriers of their own: the K half of a stage is free again as soon as S_j is done, a block
+        // earlier than the V half, and the next scores need only K
         int issued = 0;
         for (int j = 0; j < nb; ++j) {
             const int st = j & 1;
-            if (j >= 2 && !mbar_wait(&kv_empty[st], ((j >> 1) - 1) & 1, &abort_flag, wait_limit)) break;
             uint8_t *k = skv + st * (C::K_BYTES + C::V_BYTES), *v = k + C::K_BYTES;
-            mbar_expect_tx(&kv_full[st], C::K_BYTES + C::V_BYTES);
-            for (int kb = 0; kb < C::KBLK; ++kb) {
-                tma_load_2d(k + kb * AT_BN * 128, &map_k, kb * 64, hk * max_context + j * AT_BN, &kv_full[st]);
-                tma_load_2d(v + kb * AT_BN * 128, &map_v, kb * 64, hk * max_context + j * AT_BN, &kv_full[st]);
-            }
+            if (j >= 2 && !mbar_wait(&k_empty[st], ((j >> 1) - 1) & 1, &abort_flag, wait_limit)) break;
+            mbar_expect_tx(&k_full[st], C::K_BYTES);
+            for (int kb = 0; kb < C::KBLK; ++kb) tma_load_2d(k + kb * AT_BN * 128, &map_k, kb * 64, hk * max_context + j * AT_BN, &k_full[st]);
+            if (j >= 2 && !mbar_wait(&v_empty[st], ((j >> 1) - 1) & 1, &abort_flag, wait_limit)) { issued = -(j + 1); break; }
+            mbar_expect_tx(&v_full[st], C::V_BYTES);
+            for (int kb = 0; kb < C::KBLK; ++kb) tma_load_2d(v + kb * AT_BN * 128, &map_v, kb * 64, hk * max_context + j * AT_BN, &v_full[st]);
             issued = j + 1;
         }
         if (abort_flag) {   // giving up: the copies in flight must land before the shared memory is released
             int dummy = 0;
             mbar_wait(&q_full, 0, &dummy, wait_limit);
-            for (int j = issued > 2 ? issued - 2 : 0; j < issued; ++j) mbar_wait(&kv_full[j & 1], (j >> 1) & 1, &dummy, wait_limit);
+            const int nk = issued < 0 ? -issued : issued, nv = issued < 0 ? -issued - 1 : issued;
+            for (int j = nk > 2 ? nk - 2 : 0; j < nk; ++j) mbar_wait(&k_full[j & 1], (j >> 1) & 1, &dummy, wait_limit);
+            for (int j = nv > 2 ? nv - 2 : 0; j < nv; ++j) mbar_wait(&v_full[j & 1], (j >> 1) & 1, &dummy, wait_limit);
         }
-    } else if (warp == 1 && lane == 0) {     // issuer
+    } else if (warp == 1 && lane == 0) {     // issuer of the scores: S_j = Q K_j^T, hi pieces then lo pieces
+        // (two issuing threads, scores here and P V in warp 2: a tcgen05.mma takes about 40 ns to issue, and one thread issuing
+        // both, with its six waits per block, was what bounded the kernel: 2.3 us per block)
         constexpr uint32_t idesc_s = umma_idesc_bf16(AT_BM, AT_BN);
-        constexpr uint32_t idesc_o = umma_idesc_bf16(AT_BM, D) | (1u << 16);   // B (= V) is MN-major
-        auto issue_s = [&](int j) {          // S_j = Q K_j^T, hi pieces then lo pieces
-            const uint32_t k = smem_u32(skv + (j & 1) * (C::K_BYTES + C::V_BYTES)), acc = tmem + (j & 1) * AT_BN;
+        bool ok = mbar_wait(&q_full, 0, &abort_flag, wait_limit);
+        for (int j = 0; j < nb && ok; ++j) {
+            const int st = j & 1;
+            ok = mbar_wait(&k_full[st], (j >> 1) & 1, &abort_flag, wait_limit);
+            if (ok && j >= 2) ok = mbar_wait(&s_empty[st], ((j >> 1) - 1) & 1, &abort_flag, wait_limit);   // the softmax has read S_{j-2}
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t k = smem_u32(skv + st * (C::K_BYTES + C::V_BYTES)), acc = tmem + st * AT_BN;
 #pragma unroll
             for (int piece = 0; piece < 2; ++piece)
 #pragma unroll
@@ -616,43 +628,44 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) umma_bf16(acc, da + 2 * kk, db + 2 * kk, idesc_s, (piece | kb | kk) != 0);
                 }
-            umma_commit(&s_full[j & 1]);
-        };
-        bool ok = mbar_wait(&q_full, 0, &abort_flag, wait_limit) && mbar_wait(&kv_full[0], 0, &abort_flag, wait_limit);
-        if (ok) { tc_fence_after(); issue_s(0); }
-        for (int j = 0; j < nb && ok; ++j) {
-            if (j + 1 < nb) {                // the next block's scores, under this block's softmax
-                const int st = (j + 1) & 1;
-                ok = mbar_wait(&kv_full[st], ((j + 1) >> 1) & 1, &abort_flag, wait_limit);
-                if (ok && j + 1 >= 2) ok = mbar_wait(&s_empty[st], (((j + 1) >> 1) - 1) & 1, &abort_flag, wait_limit);
-                if (!ok) break;
-                tc_fence_after();
-                issue_s(j + 1);
-            }
-            ok = mbar_wait(&p_full[j & 1], (j >> 1) & 1, &abort_flag, wait_limit);
-            if (ok && j >= 2) ok = mbar_wait(&o_empty[j & 1], ((j >> 1) - 1) & 1, &abort_flag, wait_limit);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t v = smem_u32(skv + (j & 1) * (C::K_BYTES + C::V_BYTES) + C::K_BYTES);
-#pragma unroll
-            for (int piece = 0; piece < 2; ++piece) {
-                const uint64_t da = umma_desc_sw128(smem_u32(sp) + (j & 1) * C::P_BYTES + piece * AT_BM * 128);
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk)   // 16 keys = 2 groups of 8 rows = 2048 bytes of the V tile
-                    umma_bf16(tmem + 2 * AT_BN + (j & 1) * D, da + 2 * kk, umma_desc_sw128_mn(v + kk * 2048, AT_BN * 128), idesc_o, (piece | kk) != 0);
-            }
-            umma_commit(&o_full[j & 1]);
-            umma_commit(&p_empty[j & 1]);
-            umma_commit(&kv_empty[j & 1]);
+            umma_commit(&s_full[st]);
+            umma_commit(&k_empty[st]);       // the K rows are free when these have read them
         }
         if (!ok) {
             int dummy = 0;
-            umma_commit(&drain_bar);
-            mbar_wait(&drain_bar, 0, &dummy, wait_limit);
+            umma_commit(&drain_bar[0]);
+            mbar_wait(&drain_bar[0], 0, &dummy, wait_limit);
+        }
+    } else if (warp == 2 && lane == 0) {     // issuer of O_j = P_j V_j
+        constexpr uint32_t idesc_o = umma_idesc_bf16(AT_BM, D) | (1u << 16);   // B (= V) is MN-major
+        bool ok = true;
+        for (int j = 0; j < nb && ok; ++j) {
+            const int st = j & 1;
+            ok = mbar_wait(&v_full[st], (j >> 1) & 1, &abort_flag, wait_limit);
+            if (ok && j >= 2) ok = mbar_wait(&o_empty[st], ((j >> 1) - 1) & 1, &abort_flag, wait_limit);   // O_{j-2} has been added
+            if (ok) ok = mbar_wait(&p_full[st], (j >> 1) & 1, &abort_flag, wait_limit);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t v = smem_u32(skv + st * (C::K_BYTES + C::V_BYTES) + C::K_BYTES);
+#pragma unroll
+            for (int piece = 0; piece < 2; ++piece) {
+                const uint64_t da = umma_desc_sw128(smem_u32(sp) + st * C::P_BYTES + piece * AT_BM * 128);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)   // 16 keys = 2 groups of 8 rows = 2048 bytes of the V tile
+                    umma_bf16(tmem + 2 * AT_BN + st * D, da + 2 * kk, umma_desc_sw128_mn(v + kk * 2048, AT_BN * 128), idesc_o, (piece | kk) != 0);
+            }
+            umma_commit(&o_full[st]);
+            umma_commit(&p_empty[st]);
+            umma_commit(&v_empty[st]);
+        }
+        if (!ok) {
+            int dummy = 0;
+            umma_commit(&drain_bar[1]);
+            mbar_wait(&drain_bar[1], 0, &dummy, wait_limit);
         }
     }
-    else if (warp >= 2) {                    // softmax: AT_PARTS threads per query row (= lane of tensor memory), AT_BN / AT_PARTS keys of a block each
-        const int quarter = warp & 3, part = (warp - 2) >> 2, row = quarter * 32 + lane;
+    else if (warp >= 3) {                    // softmax: AT_PARTS threads per query row (= lane of tensor memory), AT_BN / AT_PARTS keys of a block each
+        const int quarter = warp & 3, part = (warp - 3) >> 2, row = quarter * 32 + lane;
         const uint32_t trow = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
         const int qi = slot0 + t0 + row;     // cache slot of this query: it sees the keys 0 .. qi
         constexpr int KP = AT_BN / AT_PARTS; // keys of a block per thread
@@ -834,7 +847,7 @@ const char *launch_attention_tc(const uint16_t *q, const uint16_t *kc, const uin
     if (cudaFuncSetAttribute(prefill_attention_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<D>::SMEM) != cudaSuccess)
         return "cudaFuncSetAttribute failed";
     const float scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(D)));
-    prefill_attention_tc_kernel<D><<<dim3((T + AT_BM - 1) / AT_BM, nq), AT_THREADS, AttnCfg<D>::SMEM, s>>>(
+    prefill_attention_tc_kernel<D><<<dim3(nq, (T + AT_BM - 1) / AT_BM), AT_THREADS, AttnCfg<D>::SMEM, s>>>(
         mqh, mql, mk, mv, out, plane, T, slot0, nq, nq / nkv, max_context, scale_log2, wait_limit, error);
     return cudaGetLastError() == cudaSuccess ? nullptr : "prefill attention launch failed";
 }
