@@ -511,16 +511,20 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
 }
 
 // ---- causal attention on tcgen05 ---------------------------------------------------------------------------------------------
-// One CTA = 128 queries of one head (a query = a lane of tensor memory = a thread of the softmax warps); keys in blocks of 64.
-// Per block j:  S_j = Q K_j^T (tcgen05.mma, M 128, N 64, K = D; queries as two bf16 pieces) into one of two S buffers in
-// tensor memory;  the softmax warps read their row (tcgen05.ld), mask, update the running maximum and sum, and write the
-// probabilities as two bf16 pieces into shared memory in the swizzled K-major layout of an A operand;  O_j = P_j V_j (M 128,
-// N = D, K = 64 keys; V straight from its cache rows as an MN-major B operand) into a third region of tensor memory;  the
-// softmax warps add O_j to their fp32 row in registers, o = o * alpha_j + O_j, one block late so that the multiply hides under
-// the next block's softmax.  S_{j+1} is issued before P_j is waited for, so the tensor pipe works under the softmax too.
-//   tensor memory: S0 [0, 64), S1 [64, 128), O0 [128, 128 + D), O1 [128 + D, 128 + 2 D)
-//   shared memory: Q 2 x D/64 x 16 KB | 2 stages x (K D/64 x 8 KB, V D/64 x 8 KB) | 2 x P (2 x 16 KB)
-constexpr int AT_BM = 128, AT_BN = 64, AT_PARTS = 2;
+// One CTA = 128 queries of one head (a query = a lane of tensor memory, two softmax threads per query); keys in blocks of 128.
+// Per block j:  S_j = Q K_j^T (tcgen05.mma, M 128, N 128, K = D; queries as two bf16 pieces) into one of two S buffers in
+// tensor memory;  the softmax warps read their part of the row twice (tcgen05.ld; once for the maximum, once for the
+// exponentials), mask on diagonal blocks, update the running maximum and sum, and write the probabilities as two bf16 pieces
+// into shared memory in the swizzled K-major layout of an A operand;  O_j = P_j V_j (M 128, N = D, K = 128 keys; V straight
+// from its cache rows as an MN-major B operand) into one of two O buffers;  the softmax warps add O_j to their fp32 row in
+// registers, o = o * alpha_j + O_j, one block late so that the multiply hides under the next block's softmax.  The scores
+// and P V are issued by two threads (warps 1 and 2), the K and V tiles have barriers of their own.
+//   tensor memory: S0 [0, 128), S1 [128, 256), O0 [256, 256 + D), O1 [256 + D, 256 + 2 D)      (512 columns allocated)
+//   shared memory: Q 2 x D/64 x 16 KB | K D/64 x 16 KB | V D/64 x 16 KB | P 2 x 2 x 16 KB
+constexpr int AT_BM = 128, AT_BN = 128, AT_PARTS = 2;
+constexpr int AT_KVS = 1;      // stages of the K / V tiles (one: the next K tile loads under this block's softmax, the next V
+                               // tile under the next block's)
+constexpr int AT_PB = 1;       // buffers of the probabilities
 constexpr int AT_THREADS = 96 + 128 * AT_PARTS;   // producer, two issuers, softmax warps
 
 // B operand in MN-major form for P V: the V tile is D/64 blocks of [64 keys][64 d] (128-byte rows, 128-byte swizzle).  N (= d)
@@ -535,8 +539,9 @@ template <int D> struct AttnCfg {
     static constexpr int KBLK = D / 64;                        // 64-column blocks of a row of q, k, v
     static constexpr int Q_BYTES = 2 * KBLK * AT_BM * 128;     // two pieces
     static constexpr int K_BYTES = KBLK * AT_BN * 128, V_BYTES = K_BYTES;
-    static constexpr int P_BYTES = 2 * AT_BM * 128;            // two pieces of [128][64 keys]
-    static constexpr int SMEM = Q_BYTES + 2 * (K_BYTES + V_BYTES) + 2 * P_BYTES + 1024;   // K/V and P double-buffered
+    static constexpr int P_PIECE = (AT_BN / 64) * AT_BM * 128; // one piece: AT_BN / 64 blocks of [128 rows][64 keys]
+    static constexpr int P_BYTES = 2 * P_PIECE;
+    static constexpr int SMEM = Q_BYTES + AT_KVS * (K_BYTES + V_BYTES) + AT_PB * P_BYTES + 1024;
     static constexpr int TMEM_COLS = 2 * AT_BN + 2 * D <= 256 ? 256 : 512;   // S0, S1, O0, O1
 };
 
@@ -549,12 +554,12 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
                                                                    float scale_log2, uint32_t wait_limit, int *error) {
     using C = AttnCfg<D>;
     extern __shared__ uint8_t at_tc_dyn[];
-    __shared__ uint64_t q_full, k_full[2], k_empty[2], v_full[2], v_empty[2], s_full[2], s_empty[2], p_full[2], p_empty[2], o_full[2], o_empty[2], drain_bar[2], pair_bar[4];
+    __shared__ uint64_t q_full, k_full[AT_KVS], k_empty[AT_KVS], v_full[AT_KVS], v_empty[AT_KVS], s_full[2], s_empty[2], p_full[AT_PB], p_empty[AT_PB], o_full[2], o_empty[2], drain_bar[2], pair_bar[4];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ float xchg[2][AT_PARTS][AT_BM];      // row maxima / sums passed between the two threads of a row
     uint8_t *base = at_tc_dyn + ((1024u - (smem_u32(at_tc_dyn) & 1023u)) & 1023u);
-    uint8_t *sq = base, *skv = sq + C::Q_BYTES, *sp = skv + 2 * (C::K_BYTES + C::V_BYTES);
+    uint8_t *sq = base, *skv = sq + C::Q_BYTES, *sp = skv + AT_KVS * (C::K_BYTES + C::V_BYTES);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // grid (heads, query tiles): CTAs start in linear order, so every head's longest tile (the last queries) starts first
     const int t0 = (gridDim.y - 1 - blockIdx.y) * AT_BM;
@@ -564,8 +569,9 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
 
     if (threadIdx.x == 0) {
         mbar_init(&q_full, 1);
-        for (int i = 0; i < 2; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1); mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 4 * AT_PARTS); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&p_full[i], 4 * AT_PARTS); mbar_init(&p_empty[i], 1); mbar_init(&o_full[i], 1); mbar_init(&o_empty[i], 4 * AT_PARTS); }
+        for (int i = 0; i < AT_KVS; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1); }
+        for (int i = 0; i < AT_PB; ++i) { mbar_init(&p_full[i], 4 * AT_PARTS); mbar_init(&p_empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 4 * AT_PARTS); mbar_init(&o_full[i], 1); mbar_init(&o_empty[i], 4 * AT_PARTS); }
         mbar_init(&drain_bar[0], 1); mbar_init(&drain_bar[1], 1);
         for (int i = 0; i < 4; ++i) mbar_init(&pair_bar[i], AT_PARTS);
         abort_flag = 0;
@@ -590,12 +596,12 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
         // earlier than the V half, and the next scores need only K
         int issued = 0;
         for (int j = 0; j < nb; ++j) {
-            const int st = j & 1;
+            const int st = j % AT_KVS;
             uint8_t *k = skv + st * (C::K_BYTES + C::V_BYTES), *v = k + C::K_BYTES;
-            if (j >= 2 && !mbar_wait(&k_empty[st], ((j >> 1) - 1) & 1, &abort_flag, wait_limit)) break;
+            if (j >= AT_KVS && !mbar_wait(&k_empty[st], ((j / AT_KVS) - 1) & 1, &abort_flag, wait_limit)) break;
             mbar_expect_tx(&k_full[st], C::K_BYTES);
             for (int kb = 0; kb < C::KBLK; ++kb) tma_load_2d(k + kb * AT_BN * 128, &map_k, kb * 64, hk * max_context + j * AT_BN, &k_full[st]);
-            if (j >= 2 && !mbar_wait(&v_empty[st], ((j >> 1) - 1) & 1, &abort_flag, wait_limit)) { issued = -(j + 1); break; }
+            if (j >= AT_KVS && !mbar_wait(&v_empty[st], ((j / AT_KVS) - 1) & 1, &abort_flag, wait_limit)) { issued = -(j + 1); break; }
             mbar_expect_tx(&v_full[st], C::V_BYTES);
             for (int kb = 0; kb < C::KBLK; ++kb) tma_load_2d(v + kb * AT_BN * 128, &map_v, kb * 64, hk * max_context + j * AT_BN, &v_full[st]);
             issued = j + 1;
@@ -604,8 +610,8 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
             int dummy = 0;
             mbar_wait(&q_full, 0, &dummy, wait_limit);
             const int nk = issued < 0 ? -issued : issued, nv = issued < 0 ? -issued - 1 : issued;
-            for (int j = nk > 2 ? nk - 2 : 0; j < nk; ++j) mbar_wait(&k_full[j & 1], (j >> 1) & 1, &dummy, wait_limit);
-            for (int j = nv > 2 ? nv - 2 : 0; j < nv; ++j) mbar_wait(&v_full[j & 1], (j >> 1) & 1, &dummy, wait_limit);
+            for (int j = nk > AT_KVS ? nk - AT_KVS : 0; j < nk; ++j) mbar_wait(&k_full[j % AT_KVS], (j / AT_KVS) & 1, &dummy, wait_limit);
+            for (int j = nv > AT_KVS ? nv - AT_KVS : 0; j < nv; ++j) mbar_wait(&v_full[j % AT_KVS], (j / AT_KVS) & 1, &dummy, wait_limit);
         }
     } else if (warp == 1 && lane == 0) {     // issuer of the scores: S_j = Q K_j^T, hi pieces then lo pieces
         // (two issuing threads, scores here and P V in warp 2: a tcgen05.mma takes about 40 ns to issue, and one thread issuing
@@ -613,12 +619,12 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
         constexpr uint32_t idesc_s = umma_idesc_bf16(AT_BM, AT_BN);
         bool ok = mbar_wait(&q_full, 0, &abort_flag, wait_limit);
         for (int j = 0; j < nb && ok; ++j) {
-            const int st = j & 1;
-            ok = mbar_wait(&k_full[st], (j >> 1) & 1, &abort_flag, wait_limit);
-            if (ok && j >= 2) ok = mbar_wait(&s_empty[st], ((j >> 1) - 1) & 1, &abort_flag, wait_limit);   // the softmax has read S_{j-2}
+            const int st = j % AT_KVS, sb = j & 1;
+            ok = mbar_wait(&k_full[st], (j / AT_KVS) & 1, &abort_flag, wait_limit);
+            if (ok && j >= 2) ok = mbar_wait(&s_empty[sb], ((j >> 1) - 1) & 1, &abort_flag, wait_limit);   // the softmax has read S_{j-2}
             if (!ok) break;
             tc_fence_after();
-            const uint32_t k = smem_u32(skv + st * (C::K_BYTES + C::V_BYTES)), acc = tmem + st * AT_BN;
+            const uint32_t k = smem_u32(skv + st * (C::K_BYTES + C::V_BYTES)), acc = tmem + sb * AT_BN;
 #pragma unroll
             for (int piece = 0; piece < 2; ++piece)
 #pragma unroll
@@ -628,7 +634,7 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) umma_bf16(acc, da + 2 * kk, db + 2 * kk, idesc_s, (piece | kb | kk) != 0);
                 }
-            umma_commit(&s_full[st]);
+            umma_commit(&s_full[sb]);
             umma_commit(&k_empty[st]);       // the K rows are free when these have read them
         }
         if (!ok) {
@@ -640,22 +646,23 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
         constexpr uint32_t idesc_o = umma_idesc_bf16(AT_BM, D) | (1u << 16);   // B (= V) is MN-major
         bool ok = true;
         for (int j = 0; j < nb && ok; ++j) {
-            const int st = j & 1;
-            ok = mbar_wait(&v_full[st], (j >> 1) & 1, &abort_flag, wait_limit);
-            if (ok && j >= 2) ok = mbar_wait(&o_empty[st], ((j >> 1) - 1) & 1, &abort_flag, wait_limit);   // O_{j-2} has been added
-            if (ok) ok = mbar_wait(&p_full[st], (j >> 1) & 1, &abort_flag, wait_limit);
+            const int st = j % AT_KVS, pb = j % AT_PB, ob = j & 1;
+            ok = mbar_wait(&v_full[st], (j / AT_KVS) & 1, &abort_flag, wait_limit);
+            if (ok && j >= 2) ok = mbar_wait(&o_empty[ob], ((j >> 1) - 1) & 1, &abort_flag, wait_limit);   // O_{j-2} has been added
+            if (ok) ok = mbar_wait(&p_full[pb], (j / AT_PB) & 1, &abort_flag, wait_limit);
             if (!ok) break;
             tc_fence_after();
             const uint32_t v = smem_u32(skv + st * (C::K_BYTES + C::V_BYTES) + C::K_BYTES);
 #pragma unroll
             for (int piece = 0; piece < 2; ++piece) {
-                const uint64_t da = umma_desc_sw128(smem_u32(sp) + st * C::P_BYTES + piece * AT_BM * 128);
+                const uint32_t pa = smem_u32(sp) + pb * C::P_BYTES + piece * C::P_PIECE;
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk)   // 16 keys = 2 groups of 8 rows = 2048 bytes of the V tile
-                    umma_bf16(tmem + 2 * AT_BN + st * D, da + 2 * kk, umma_desc_sw128_mn(v + kk * 2048, AT_BN * 128), idesc_o, (piece | kk) != 0);
+                for (int kk = 0; kk < AT_BN / 16; ++kk)   // 16 keys: 32 bytes along a P row (64-key blocks 16 KB apart), 2048 bytes of the V tile
+                    umma_bf16(tmem + 2 * AT_BN + ob * D, umma_desc_sw128(pa + (kk >> 2) * AT_BM * 128) + 2 * (kk & 3),
+                              umma_desc_sw128_mn(v + kk * 2048, AT_BN * 128), idesc_o, (piece | kk) != 0);
             }
-            umma_commit(&o_full[st]);
-            umma_commit(&p_empty[st]);
+            umma_commit(&o_full[ob]);
+            umma_commit(&p_empty[pb]);
             umma_commit(&v_empty[st]);
         }
         if (!ok) {
@@ -707,19 +714,21 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
             tc_fence_after();
             const int key0 = j * AT_BN + part * KP;
             const bool diagonal = j * AT_BN + AT_BN - 1 > slot0 + t0;   // some query of the tile does not see the whole block
-            float v[KP];
-            tmem_ld<KP>(trow + (j & 1) * AT_BN + part * KP, v);
-            tmem_ld_wait();
-            tc_fence_before();
-            warp_arrive(&s_empty[j & 1]);    // this part of S_j is in registers
-            if (diagonal) {
+            const uint32_t srow = trow + (j & 1) * AT_BN + part * KP;
+            float mx = -INFINITY;
 #pragma unroll
-                for (int i = 0; i < KP; ++i)
-                    if (key0 + i > qi) v[i] = -INFINITY;
+            for (int c = 0; c < KP / 32; ++c) {   // pass 1: the maximum over this thread's keys the query sees
+                float v[32];
+                tmem_ld32(srow + c * 32, v);
+                tmem_ld_wait();
+                if (diagonal) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (key0 + c * 32 + i > qi) v[i] = -INFINITY;
+                }
+#pragma unroll
+                for (int i = 0; i < 32; i += 4) mx = fmaxf(mx, fmaxf(fmaxf(v[i], v[i + 1]), fmaxf(v[i + 2], v[i + 3])));
             }
-            float mx = fmaxf(fmaxf(v[0], v[1]), fmaxf(v[2], v[3]));
-#pragma unroll
-            for (int i = 4; i < KP; i += 4) mx = fmaxf(mx, fmaxf(fmaxf(v[i], v[i + 1]), fmaxf(v[i + 2], v[i + 3])));
             xchg[j & 1][part][row] = mx;     // the row maximum needs the other threads' keys
             ok = row_sync(j);
             if (!ok) break;
@@ -729,34 +738,45 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
             const float alpha = fast_exp2((m_run - mx) * scale_log2);   // first block: exp2(-inf) = 0
             m_run = mx;
             const float neg = -mx * scale_log2;
+            if (j >= AT_PB) {                // the P buffer's previous block has been multiplied
+                ok = warp_wait(&p_empty[j % AT_PB], ((j / AT_PB) - 1) & 1);
+                if (!ok) break;
+            }
             float sum0 = 0.f, sum1 = 0.f;
-            uint4 hi[KP / 8], lo[KP / 8];
 #pragma unroll
-            for (int i8 = 0; i8 < KP / 8; ++i8) {   // probabilities as two bf16 pieces
-                uint32_t *hw = &hi[i8].x, *lw = &lo[i8].x;
+            for (int c = 0; c < KP / 32; ++c) {   // pass 2: probabilities as two bf16 pieces, into the A-operand layout
+                float v[32];
+                tmem_ld32(srow + c * 32, v);
+                tmem_ld_wait();
+                if (diagonal) {
 #pragma unroll
-                for (int i2 = 0; i2 < 4; ++i2) {
-                    const int i = i8 * 8 + i2 * 2;
-                    const float p0 = fast_exp2(fmaf(v[i], scale_log2, neg)), p1 = fast_exp2(fmaf(v[i + 1], scale_log2, neg));
-                    sum0 += p0;
-                    sum1 += p1;
-                    split2x2_trunc(p0, p1, hw[i2], lw[i2]);
+                    for (int i = 0; i < 32; ++i)
+                        if (key0 + c * 32 + i > qi) v[i] = -INFINITY;
+                }
+                const int kq = part * KP + c * 32;            // first key of this chunk within the block
+                uint8_t *prow_hi = sp + (j % AT_PB) * C::P_BYTES + (kq >> 6) * AT_BM * 128 + row * 128, *prow_lo = prow_hi + C::P_PIECE;
+#pragma unroll
+                for (int i8 = 0; i8 < 4; ++i8) {
+                    uint4 hi, lo;
+                    uint32_t *hw = &hi.x, *lw = &lo.x;
+#pragma unroll
+                    for (int i2 = 0; i2 < 4; ++i2) {
+                        const int i = i8 * 8 + i2 * 2;
+                        const float p0 = fast_exp2(fmaf(v[i], scale_log2, neg)), p1 = fast_exp2(fmaf(v[i + 1], scale_log2, neg));
+                        sum0 += p0;
+                        sum1 += p1;
+                        split2x2_trunc(p0, p1, hw[i2], lw[i2]);
+                    }
+                    const int piece16 = ((((kq & 63) >> 3) + i8) ^ (row & 7)) << 4;   // 16-byte piece index xor row bits (128-byte swizzle)
+                    *reinterpret_cast<uint4 *>(prow_hi + piece16) = hi;
+                    *reinterpret_cast<uint4 *>(prow_lo + piece16) = lo;
                 }
             }
             l_run = l_run * alpha + (sum0 + sum1);
-            if (j >= 2) {                    // the P buffer's previous block has been multiplied
-                ok = warp_wait(&p_empty[j & 1], ((j >> 1) - 1) & 1);
-                if (!ok) break;
-            }
-            uint8_t *prow_hi = sp + (j & 1) * C::P_BYTES + row * 128, *prow_lo = prow_hi + AT_BM * 128;
-#pragma unroll
-            for (int i8 = 0; i8 < KP / 8; ++i8) {   // into the A-operand layout: 16-byte piece index xor row bits (128-byte swizzle)
-                const int piece16 = ((part * (KP / 8) + i8) ^ (row & 7)) << 4;
-                *reinterpret_cast<uint4 *>(prow_hi + piece16) = hi[i8];
-                *reinterpret_cast<uint4 *>(prow_lo + piece16) = lo[i8];
-            }
+            tc_fence_before();
+            warp_arrive(&s_empty[j & 1]);    // this part of S_j has been read twice
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P: generic-proxy writes before the tensor core's reads
-            warp_arrive(&p_full[j & 1]);
+            warp_arrive(&p_full[j % AT_PB]);
             if (j >= 1) { add_block(j - 1); if (!ok) break; }
             alpha_prev = alpha;
         }
