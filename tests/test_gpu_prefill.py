@@ -88,6 +88,12 @@ def test_prompt_on_the_1_5b_shape():
     run_case(CONFIGS["qwen2.5-1.5b"], 32, 200, 5, follow=False)
 
 
+def test_prompt_behind_a_long_prefix():
+    """8200 prefix rows (the context then runs the long-context build of the step kernel for the prompt's last token): the
+    queries attend to 65 key blocks, the first 64 of them wholly inside the prefix."""
+    run_case(CONFIGS["tiny"].with_(qkv_bias=True), 8200, 150, 9)
+
+
 def test_prompt_on_the_0_5b_shape():
     """head_dim 64, 14 query heads on 2 kv heads, tied output layer; two query tiles and a ragged third."""
     run_case(CONFIGS["qwen2.5-0.5b"], 10, 300, 6, follow=False)
