@@ -270,7 +270,7 @@ def run_prefill(args, cfg):
     T = args.prefill
     weights = make_weights(cfg)
     ptrs, keep = upload_weights(weights, dev)
-    ctx = DecodeContext(cfg, ptrs, T + 2, dev)
+    ctx = DecodeContext(cfg, ptrs, T + 2, dev, kv_format=None if args.kv_format == "bf16" else args.kv_format)
     toks = np.random.default_rng(1).integers(0, cfg.vocab, T).tolist()
     for _ in range(max(args.warmup_sequences, 3)):
         ctx.reset()
@@ -307,8 +307,8 @@ def run_prefill(args, cfg):
     tf = flops / (ms * 1e-3) / 1e12
     line = {"metric": "prefill_ms_per_prompt", "value": ms, "unit": "ms", "n_gpus": 1, "steps": len(times), "warmup": max(args.warmup_sequences, 3),
             "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16 weights/KV, activations as two bf16 pieces, fp32 accumulate (tcgen05)", "data": "synthetic",
-            "config": {"workload": f"{cfg.name}: prefill of {T} prompt tokens into an empty cache (edgefm_prefill; {n} tokens as dense contractions + one decode step)",
+            "dtype": "bf16 weights/KV, activations as two bf16 pieces, fp32 accumulate (tcgen05)" + (", 8-bit KV cache" if args.kv_format == "int8" else ""), "data": "synthetic",
+            "config": {"workload": f"{cfg.name}: prefill of {T} prompt tokens into an empty " + ("compressed (8-bit) " if args.kv_format == "int8" else "") + f"cache (edgefm_prefill; {n} tokens as dense contractions + one decode step)",
                        "l2": "weights (> 2.6 GB) and activations exceed L2; nothing flushed"},
             "ms_min": times[0], "prompt_tokens_per_s": T / (ms * 1e-3),
             "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak, "traffic": None,

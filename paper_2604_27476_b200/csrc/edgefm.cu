@@ -815,8 +815,6 @@ edgefm_status edgefm_prefill(edgefm_ctx *ctx, const int32_t *tokens, int32_t n, 
     if (position < 0) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "position %d out of range", position);
     for (int i = 0; i < n; ++i)
         if (tokens[i] < 0 || tokens[i] >= ctx->shape.vocab) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "tokens[%d] = %d out of range", i, tokens[i]);
-    if (ctx->kv_format != EDGEFM_KV_BF16)
-        return fail(ctx, EDGEFM_ERR_INVALID_ARG, "edgefm_prefill writes bf16 cache rows: use edgefm_prefill_tokens on a compressed cache");
     if (ctx->cur_len + n > ctx->max_context)
         return fail(ctx, EDGEFM_ERR_CONTEXT_FULL, "%d tokens do not fit behind %d of %d cache slots", n, ctx->cur_len, ctx->max_context);
     DeviceGuard guard(ctx->device);
@@ -824,7 +822,7 @@ edgefm_status edgefm_prefill(edgefm_ctx *ctx, const int32_t *tokens, int32_t n, 
     const int n_dense = n - 1;   // the last token takes the decode step, which also yields the logits
     if (n_dense > 0 && ctx->pf.chunk == 0) {
         const int chunk = std::min(PF_CHUNK_MAX, ctx->max_context);
-        if (prefill_alloc(&ctx->pf, ctx->shape, chunk) != cudaSuccess) {
+        if (prefill_alloc(&ctx->pf, ctx->shape, chunk, ctx->kv_format == EDGEFM_KV_INT8) != cudaSuccess) {
             cudaGetLastError();
             prefill_free(&ctx->pf);
             return fail(ctx, EDGEFM_ERR_OUT_OF_MEMORY, "work buffers of edgefm_prefill (%zu bytes)", prefill_buffer_bytes(ctx->shape, chunk));
@@ -832,7 +830,9 @@ edgefm_status edgefm_prefill(edgefm_ctx *ctx, const int32_t *tokens, int32_t n, 
     }
     ctx->pf.wait_limit = ctx->pf_wait_limit;
     ctx->pf.extra_arrivals = ctx->pf_extra_arrivals;
-    PrefillModel pm{ctx->shape, ctx->layers.data(), ctx->embed, ctx->k_cache, ctx->v_cache, ctx->max_context, ctx->state, ctx->num_sms};
+    PrefillModel pm{ctx->shape, ctx->layers.data(), ctx->embed, ctx->k_cache, ctx->v_cache,
+                    ctx->kv_format == EDGEFM_KV_INT8 ? ctx->k_scale : nullptr, ctx->kv_format == EDGEFM_KV_INT8 ? ctx->v_scale : nullptr,
+                    ctx->max_context, ctx->state, ctx->num_sms};
     ctx->prefill_launches = 0;
     for (int i = 0; i < n_dense;) {
         const int c = std::min(ctx->pf.chunk, n_dense - i);

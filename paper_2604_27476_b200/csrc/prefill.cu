@@ -229,6 +229,36 @@ __global__ void __launch_bounds__(128) prefill_norm_kernel(float *resid, uint16_
     }
 }
 
+// Compressed cache (Sec. 3.9): one warp per new row (k rows, then v rows) of the fp32 staging buffers [nkv][stride / d][d];
+// scale = amax / 127, code = clamp(rint(x * (127 / amax))) in fp32 -- the arithmetic of the decode step's own row.
+__global__ void __launch_bounds__(256) prefill_quantize_rows_kernel(const float *k, const float *v, long long stage_stride, signed char *kc,
+                                                                    signed char *vc, float *ks, float *vs, int nkv, int n, int d,
+                                                                    int max_context, int slot0) {
+    const int lane = threadIdx.x & 31;
+    const long long r = (blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x) >> 5, rows = static_cast<long long>(nkv) * n;
+    if (r >= 2 * rows) return;
+    const bool is_v = r >= rows;
+    const long long rr = is_v ? r - rows : r;
+    const int t = static_cast<int>(rr % n), g = static_cast<int>(rr / n);
+    const float *src = (is_v ? v : k) + g * stage_stride + static_cast<long long>(t) * d;
+    const long long row = static_cast<long long>(g) * max_context + slot0 + t;
+    float x[4];                                                              // d <= 128: at most 4 values per lane
+    float amax = 0.f;
+    for (int e = 0; e < 4; ++e) {
+        const int j = lane + 32 * e;
+        x[e] = j < d ? src[j] : 0.f;
+        amax = fmaxf(amax, fabsf(x[e]));
+    }
+    amax = warp_max(amax);
+    const float inv = amax > 0.f ? __fdiv_rn(127.0f, amax) : 0.f;
+    signed char *dst = (is_v ? vc : kc) + row * d;
+    for (int e = 0; e < 4; ++e) {
+        const int j = lane + 32 * e;
+        if (j < d) dst[j] = static_cast<signed char>(static_cast<int>(fminf(fmaxf(rintf(__fmul_rn(x[e], inv)), -127.f), 127.f)));
+    }
+    if (lane == 0) (is_v ? vs : ks)[row] = amax > 0.f ? __fdiv_rn(amax, 127.0f) : 0.f;
+}
+
 // ---- the contraction -------------------------------------------------------------------------------------------------------
 enum { EPI_QKV = 0, EPI_RESID = 1, EPI_SWIGLU = 2 };
 
@@ -243,6 +273,8 @@ struct GemmArgs {
     uint16_t *q_out;          // [2][..][nq d]: hi and lo planes
     size_t q_plane;           // elements between the planes
     uint16_t *k_rows, *v_rows;  // the layer's cache at the first new slot: + head * head_stride + row * d
+    float *k_stage, *v_stage;   // compressed cache: the rows go here in fp32 instead ([nkv][stage_stride / d rows][d]) and are
+    long long stage_stride;     // compressed by prefill_quantize_rows_kernel
     int nq, nkv, d;
     long long head_stride;
     // O / down
@@ -465,6 +497,14 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
                                     split2x2(a[4], a[5], ah.z, al.z); split2x2(a[6], a[7], ah.w, al.w);
                                     split2x2(b[0], b[1], bh.x, bl.x); split2x2(b[2], b[3], bh.y, bl.y);
                                     split2x2(b[4], b[5], bh.z, bl.z); split2x2(b[6], b[7], bh.w, bl.w);
+                                    if (!is_q && g.k_stage) {                                  // compressed cache: k in fp32 for the quantiser
+                                        float *f = g.k_stage + (head - g.nq) * g.stage_stride + static_cast<size_t>(row) * g.d + j0 + 8 * i;
+                                        *reinterpret_cast<float4 *>(f) = make_float4(a[0], a[1], a[2], a[3]);
+                                        *reinterpret_cast<float4 *>(f + 4) = make_float4(a[4], a[5], a[6], a[7]);
+                                        *reinterpret_cast<float4 *>(f + half) = make_float4(b[0], b[1], b[2], b[3]);
+                                        *reinterpret_cast<float4 *>(f + half + 4) = make_float4(b[4], b[5], b[6], b[7]);
+                                        continue;
+                                    }
                                     *reinterpret_cast<uint4 *>(dst + j0 + 8 * i) = ah;          // k rows: the hi piece IS the bf16 row
                                     *reinterpret_cast<uint4 *>(dst + half + j0 + 8 * i) = bh;
                                     if (is_q) {                                                // queries keep both pieces
@@ -487,6 +527,12 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
 #pragma unroll
                                     for (int j = 0; j < 8; ++j)
                                         o[j] = v[8 * i + j] + (g.bias ? bf16_bits_to_f32(g.bias[col0 + j0 + 8 * i + j]) : 0.f);
+                                    if (g.v_stage) {
+                                        float *f = g.v_stage + (head - g.nq - g.nkv) * g.stage_stride + static_cast<size_t>(row) * g.d + j0 + 8 * i;
+                                        *reinterpret_cast<float4 *>(f) = make_float4(o[0], o[1], o[2], o[3]);
+                                        *reinterpret_cast<float4 *>(f + 4) = make_float4(o[4], o[5], o[6], o[7]);
+                                        continue;
+                                    }
                                     *reinterpret_cast<uint4 *>(dst + j0 + 8 * i) =
                                         make_uint4(pack2_bf16(o[0], o[1]), pack2_bf16(o[2], o[3]), pack2_bf16(o[4], o[5]), pack2_bf16(o[6], o[7]));
                                 }
@@ -542,18 +588,28 @@ template <int D> struct AttnCfg {
     static constexpr int P_PIECE = (AT_BN / 64) * AT_BM * 128; // one piece: AT_BN / 64 blocks of [128 rows][64 keys]
     static constexpr int P_BYTES = 2 * P_PIECE;
     static constexpr int SMEM = Q_BYTES + AT_KVS * (K_BYTES + V_BYTES) + AT_PB * P_BYTES + 1024;
+    // compressed cache: the 8-bit tiles land in the first half of their bf16 tile's own place when a row of codes is as long as
+    // a 128-byte operand row (D = 128: every row is then expanded in place); D = 64 gets a landing area of its own
+    static constexpr int RAW_BYTES = AT_BN * D;
+    static constexpr int SMEM_Q8 = SMEM + (D == 128 ? 0 : 2 * RAW_BYTES);
     static constexpr int TMEM_COLS = 2 * AT_BN + 2 * D <= 256 ? 256 : 512;   // S0, S1, O0, O1
 };
 
-template <int D>
-__global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q_hi,
+template <int D, bool Q8>
+__global__ void __launch_bounds__(AT_THREADS + (Q8 ? 64 : 0)) prefill_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q_hi,
                                                                    const __grid_constant__ CUtensorMap map_q_lo,
                                                                    const __grid_constant__ CUtensorMap map_k,
                                                                    const __grid_constant__ CUtensorMap map_v, uint16_t *out, size_t plane,
                                                                    int T, int slot0, int nq, int group, int max_context,
-                                                                   float scale_log2, uint32_t wait_limit, int *error) {
+                                                                   float scale_log2, uint32_t wait_limit, int *error, const float *k_scale,
+                                                                   const float *v_scale) {
+    // Q8: the cache holds 8-bit codes and a scale per row (k_scale, v_scale: this layer's [nkv][max_context]); map_k / map_v then
+    // describe byte matrices; two more warps expand the codes to bf16 (exactly) into the operand layout, the softmax multiplies
+    // the scores by the keys' scales and folds the values' scales into the probabilities.
     using C = AttnCfg<D>;
     extern __shared__ uint8_t at_tc_dyn[];
+    __shared__ uint64_t kraw_full, vraw_full;
+    __shared__ float sc_k[Q8 ? 4 : 1][AT_BN], sc_v[Q8 ? 4 : 1][AT_BN];   // scales of the last four key blocks
     __shared__ uint64_t q_full, k_full[AT_KVS], k_empty[AT_KVS], v_full[AT_KVS], v_empty[AT_KVS], s_full[2], s_empty[2], p_full[AT_PB], p_empty[AT_PB], o_full[2], o_empty[2], drain_bar[2], pair_bar[4];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
@@ -569,7 +625,8 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
 
     if (threadIdx.x == 0) {
         mbar_init(&q_full, 1);
-        for (int i = 0; i < AT_KVS; ++i) { mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1); mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1); }
+        for (int i = 0; i < AT_KVS; ++i) { mbar_init(&k_full[i], Q8 ? 2 : 1); mbar_init(&k_empty[i], 1); mbar_init(&v_full[i], Q8 ? 2 : 1); mbar_init(&v_empty[i], 1); }
+        mbar_init(&kraw_full, 1); mbar_init(&vraw_full, 1);
         for (int i = 0; i < AT_PB; ++i) { mbar_init(&p_full[i], 4 * AT_PARTS); mbar_init(&p_empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 4 * AT_PARTS); mbar_init(&o_full[i], 1); mbar_init(&o_empty[i], 4 * AT_PARTS); }
         mbar_init(&drain_bar[0], 1); mbar_init(&drain_bar[1], 1);
@@ -599,19 +656,29 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
             const int st = j % AT_KVS;
             uint8_t *k = skv + st * (C::K_BYTES + C::V_BYTES), *v = k + C::K_BYTES;
             if (j >= AT_KVS && !mbar_wait(&k_empty[st], ((j / AT_KVS) - 1) & 1, &abort_flag, wait_limit)) break;
-            mbar_expect_tx(&k_full[st], C::K_BYTES);
-            for (int kb = 0; kb < C::KBLK; ++kb) tma_load_2d(k + kb * AT_BN * 128, &map_k, kb * 64, hk * max_context + j * AT_BN, &k_full[st]);
+            if constexpr (Q8) {
+                mbar_expect_tx(&kraw_full, C::RAW_BYTES);
+                tma_load_2d(D == 128 ? k : sp + AT_PB * C::P_BYTES, &map_k, 0, hk * max_context + j * AT_BN, &kraw_full);
+            } else {
+                mbar_expect_tx(&k_full[st], C::K_BYTES);
+                for (int kb = 0; kb < C::KBLK; ++kb) tma_load_2d(k + kb * AT_BN * 128, &map_k, kb * 64, hk * max_context + j * AT_BN, &k_full[st]);
+            }
             if (j >= AT_KVS && !mbar_wait(&v_empty[st], ((j / AT_KVS) - 1) & 1, &abort_flag, wait_limit)) { issued = -(j + 1); break; }
-            mbar_expect_tx(&v_full[st], C::V_BYTES);
-            for (int kb = 0; kb < C::KBLK; ++kb) tma_load_2d(v + kb * AT_BN * 128, &map_v, kb * 64, hk * max_context + j * AT_BN, &v_full[st]);
+            if constexpr (Q8) {
+                mbar_expect_tx(&vraw_full, C::RAW_BYTES);
+                tma_load_2d(D == 128 ? v : sp + AT_PB * C::P_BYTES + C::RAW_BYTES, &map_v, 0, hk * max_context + j * AT_BN, &vraw_full);
+            } else {
+                mbar_expect_tx(&v_full[st], C::V_BYTES);
+                for (int kb = 0; kb < C::KBLK; ++kb) tma_load_2d(v + kb * AT_BN * 128, &map_v, kb * 64, hk * max_context + j * AT_BN, &v_full[st]);
+            }
             issued = j + 1;
         }
         if (abort_flag) {   // giving up: the copies in flight must land before the shared memory is released
             int dummy = 0;
             mbar_wait(&q_full, 0, &dummy, wait_limit);
             const int nk = issued < 0 ? -issued : issued, nv = issued < 0 ? -issued - 1 : issued;
-            for (int j = nk > AT_KVS ? nk - AT_KVS : 0; j < nk; ++j) mbar_wait(&k_full[j % AT_KVS], (j / AT_KVS) & 1, &dummy, wait_limit);
-            for (int j = nv > AT_KVS ? nv - AT_KVS : 0; j < nv; ++j) mbar_wait(&v_full[j % AT_KVS], (j / AT_KVS) & 1, &dummy, wait_limit);
+            for (int j = nk > AT_KVS ? nk - AT_KVS : 0; j < nk; ++j) mbar_wait(Q8 ? &kraw_full : &k_full[j % AT_KVS], (j / AT_KVS) & 1, &dummy, wait_limit);
+            for (int j = nv > AT_KVS ? nv - AT_KVS : 0; j < nv; ++j) mbar_wait(Q8 ? &vraw_full : &v_full[j % AT_KVS], (j / AT_KVS) & 1, &dummy, wait_limit);
         }
     } else if (warp == 1 && lane == 0) {     // issuer of the scores: S_j = Q K_j^T, hi pieces then lo pieces
         // (two issuing threads, scores here and P V in warp 2: a tcgen05.mma takes about 40 ns to issue, and one thread issuing
@@ -671,6 +738,66 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
             mbar_wait(&drain_bar[1], 0, &dummy, wait_limit);
         }
     }
+    else if (Q8 && warp >= AT_THREADS / 32) {   // compressed cache: expand the 8-bit tiles to bf16 operand tiles (two warps, 64 rows each)
+        static_assert(!Q8 || AT_KVS == 1, "one raw tile of K and of V in flight");
+        const int cw = warp - AT_THREADS / 32;
+        constexpr int LPR = D / 16, RPS = 32 / LPR;       // lanes per row of codes (16 codes each), rows per step
+        auto warp_wait = [&](uint64_t *bar, int parity) {
+            int r = 1;
+            if (lane == 0) r = mbar_wait(bar, parity, &abort_flag, wait_limit) ? 1 : 0;
+            return __shfl_sync(0xffffffffu, r, 0) != 0;
+        };
+        // 16 codes -> 16 bf16, exactly: byte b of (code + 128) under the exponent of 2^23 is the float 8388608 + code + 128
+        auto expand = [&](uint4 c, uint4 &lo8, uint4 &hi8) {
+            uint32_t w[4] = {c.x ^ 0x80808080u, c.y ^ 0x80808080u, c.z ^ 0x80808080u, c.w ^ 0x80808080u};
+            uint32_t o[8];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float f0 = __uint_as_float(__byte_perm(w[i], 0x4B000000u, 0x7650)) - 8388736.f;
+                const float f1 = __uint_as_float(__byte_perm(w[i], 0x4B000000u, 0x7651)) - 8388736.f;
+                const float f2 = __uint_as_float(__byte_perm(w[i], 0x4B000000u, 0x7652)) - 8388736.f;
+                const float f3 = __uint_as_float(__byte_perm(w[i], 0x4B000000u, 0x7653)) - 8388736.f;
+                o[2 * i] = __byte_perm(__float_as_uint(f0), __float_as_uint(f1), 0x7632);
+                o[2 * i + 1] = __byte_perm(__float_as_uint(f2), __float_as_uint(f3), 0x7632);
+            }
+            lo8 = make_uint4(o[0], o[1], o[2], o[3]);
+            hi8 = make_uint4(o[4], o[5], o[6], o[7]);
+        };
+        auto expand_tile = [&](uint8_t *tile, const uint8_t *raw) {
+            // a lane takes 16 codes of a row; the lanes of a row all load before any of them stores (D = 128: in place)
+            for (int step = 0; step < 64 / RPS; ++step) {
+                const int row = cw * 64 + step * RPS + lane / LPR, c = lane % LPR;
+                const uint4 codes = *reinterpret_cast<const uint4 *>(raw + row * D + c * 16);
+                __syncwarp();
+                uint4 a, b;
+                expand(codes, a, b);
+                uint8_t *dst = tile + (c >> 2) * AT_BN * 128 + row * 128;
+                *reinterpret_cast<uint4 *>(dst + (((2 * (c & 3)) ^ (row & 7)) << 4)) = a;
+                *reinterpret_cast<uint4 *>(dst + (((2 * (c & 3) + 1) ^ (row & 7)) << 4)) = b;
+            }
+        };
+        bool ok = true;
+        for (int j = 0; j < nb && ok; ++j) {
+            uint8_t *k = skv, *v = k + C::K_BYTES;
+            ok = warp_wait(&kraw_full, j & 1);
+            if (!ok) break;
+            expand_tile(k, D == 128 ? k : sp + AT_PB * C::P_BYTES);
+            for (int i = lane; i < 64; i += 32) {          // the scales of this block's keys (both kinds: they are in memory already)
+                const int key = min(j * AT_BN + cw * 64 + i, last_key);
+                sc_k[j & 3][cw * 64 + i] = k_scale[static_cast<size_t>(hk) * max_context + key];
+                sc_v[j & 3][cw * 64 + i] = v_scale[static_cast<size_t>(hk) * max_context + key];
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&k_full[0]);
+            ok = warp_wait(&vraw_full, j & 1);
+            if (!ok) break;
+            expand_tile(v, D == 128 ? v : sp + AT_PB * C::P_BYTES + C::RAW_BYTES);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&v_full[0]);
+        }
+    }
     else if (warp >= 3) {                    // softmax: AT_PARTS threads per query row (= lane of tensor memory), AT_BN / AT_PARTS keys of a block each
         const int quarter = warp & 3, part = (warp - 3) >> 2, row = quarter * 32 + lane;
         const uint32_t trow = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
@@ -721,6 +848,10 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
                 float v[32];
                 tmem_ld32(srow + c * 32, v);
                 tmem_ld_wait();
+                if constexpr (Q8) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] *= sc_k[j & 3][part * KP + c * 32 + i];
+                }
                 if (diagonal) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
@@ -748,6 +879,10 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
                 float v[32];
                 tmem_ld32(srow + c * 32, v);
                 tmem_ld_wait();
+                if constexpr (Q8) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] *= sc_k[j & 3][part * KP + c * 32 + i];
+                }
                 if (diagonal) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
@@ -765,7 +900,8 @@ __global__ void __launch_bounds__(AT_THREADS) prefill_attention_tc_kernel(const 
                         const float p0 = fast_exp2(fmaf(v[i], scale_log2, neg)), p1 = fast_exp2(fmaf(v[i + 1], scale_log2, neg));
                         sum0 += p0;
                         sum1 += p1;
-                        split2x2_trunc(p0, p1, hw[i2], lw[i2]);
+                        if constexpr (Q8) split2x2_trunc(p0 * sc_v[j & 3][kq + i], p1 * sc_v[j & 3][kq + i + 1], hw[i2], lw[i2]);
+                        else split2x2_trunc(p0, p1, hw[i2], lw[i2]);
                     }
                     const int piece16 = ((((kq & 63) >> 3) + i8) ^ (row & 7)) << 4;   // 16-byte piece index xor row bits (128-byte swizzle)
                     *reinterpret_cast<uint4 *>(prow_hi + piece16) = hi;
@@ -856,19 +992,43 @@ const char *launch_gemm(const uint16_t *a, size_t a_plane, const void *w, long l
     }
 }
 
+// Map of a byte matrix [rows][row_bytes] (the codes of a compressed cache); a box is box_rows whole rows, unswizzled.
+bool encode_bytes_map(CUtensorMap *m, const void *base, long long rows, int row_bytes, int box_rows) {
+    TensorMapEncodeFn enc = tensor_map_encoder();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(row_bytes), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(row_bytes)};
+    const cuuint32_t box[2] = {static_cast<cuuint32_t>(row_bytes), static_cast<cuuint32_t>(box_rows)};
+    const cuuint32_t es[2] = {1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// kc / vc: this layer's cache, bf16 rows or (k_scale != nullptr) rows of 8-bit codes with their scales.
 template <int D>
-const char *launch_attention_tc(const uint16_t *q, const uint16_t *kc, const uint16_t *vc, uint16_t *out, size_t plane, int T, int slot0,
-                                int nq, int nkv, int max_context, uint32_t wait_limit, int *error, cudaStream_t s) {
+const char *launch_attention_tc(const uint16_t *q, const void *kc, const void *vc, const float *k_scale, const float *v_scale, uint16_t *out,
+                                size_t plane, int T, int slot0, int nq, int nkv, int max_context, uint32_t wait_limit, int *error,
+                                cudaStream_t s) {
     CUtensorMap mqh, mql, mk, mv;
     const long long kv_rows = static_cast<long long>(nkv) * max_context;
-    if (!encode_operand_map(&mqh, q, T, nq * D) || !encode_operand_map(&mql, q + plane, T, nq * D) ||
-        !encode_operand_map(&mk, kc, kv_rows, D, AT_BN) || !encode_operand_map(&mv, vc, kv_rows, D, AT_BN))
+    const bool q8 = k_scale != nullptr;
+    if (!encode_operand_map(&mqh, q, T, nq * D) || !encode_operand_map(&mql, q + plane, T, nq * D)) return "cuTensorMapEncodeTiled failed";
+    if (q8 ? (!encode_bytes_map(&mk, kc, kv_rows, D, AT_BN) || !encode_bytes_map(&mv, vc, kv_rows, D, AT_BN))
+           : (!encode_operand_map(&mk, kc, kv_rows, D, AT_BN) || !encode_operand_map(&mv, vc, kv_rows, D, AT_BN)))
         return "cuTensorMapEncodeTiled failed";
-    if (cudaFuncSetAttribute(prefill_attention_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<D>::SMEM) != cudaSuccess)
-        return "cudaFuncSetAttribute failed";
     const float scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(D)));
-    prefill_attention_tc_kernel<D><<<dim3(nq, (T + AT_BM - 1) / AT_BM), AT_THREADS, AttnCfg<D>::SMEM, s>>>(
-        mqh, mql, mk, mv, out, plane, T, slot0, nq, nq / nkv, max_context, scale_log2, wait_limit, error);
+    const dim3 grid(nq, (T + AT_BM - 1) / AT_BM);
+    if (q8) {
+        if (cudaFuncSetAttribute(prefill_attention_tc_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<D>::SMEM_Q8) != cudaSuccess)
+            return "cudaFuncSetAttribute failed";
+        prefill_attention_tc_kernel<D, true><<<grid, AT_THREADS + 64, AttnCfg<D>::SMEM_Q8, s>>>(
+            mqh, mql, mk, mv, out, plane, T, slot0, nq, nq / nkv, max_context, scale_log2, wait_limit, error, k_scale, v_scale);
+    } else {
+        if (cudaFuncSetAttribute(prefill_attention_tc_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<D>::SMEM) != cudaSuccess)
+            return "cudaFuncSetAttribute failed";
+        prefill_attention_tc_kernel<D, false><<<grid, AT_THREADS, AttnCfg<D>::SMEM, s>>>(
+            mqh, mql, mk, mv, out, plane, T, slot0, nq, nq / nkv, max_context, scale_log2, wait_limit, error, nullptr, nullptr);
+    }
     return cudaGetLastError() == cudaSuccess ? nullptr : "prefill attention launch failed";
 }
 
@@ -899,7 +1059,7 @@ size_t prefill_buffer_bytes(const edgefm_shape &sh, int chunk) {
     return c * sh.hidden * 4 * (1 + PF_SPLIT_MAX) + c * sh.hidden * 4 + 2 * c * qd * 4 + c * sh.ffn * 4 + c * (sh.head_dim / 2) * 8 + c * 4 + 256;
 }
 
-cudaError_t prefill_alloc(PrefillBuffers *b, const edgefm_shape &sh, int chunk) {
+cudaError_t prefill_alloc(PrefillBuffers *b, const edgefm_shape &sh, int chunk, bool kv8) {
     const size_t c = static_cast<size_t>(chunk), qd = static_cast<size_t>(sh.n_q_heads) * sh.head_dim;
     cudaError_t e;
     if ((e = cudaMalloc(&b->resid, c * sh.hidden * 4)) != cudaSuccess) return e;
@@ -909,6 +1069,7 @@ cudaError_t prefill_alloc(PrefillBuffers *b, const edgefm_shape &sh, int chunk) 
     if ((e = cudaMalloc(&b->attn, c * qd * 4)) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->act, c * sh.ffn * 4)) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->rope, c * (sh.head_dim / 2) * sizeof(float2))) != cudaSuccess) return e;
+    if (kv8 && (e = cudaMalloc(&b->kv_stage, 2 * c * sh.n_kv_heads * sh.head_dim * sizeof(float))) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->tokens, c * 4)) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->error, 4)) != cudaSuccess) return e;
     if ((e = cudaMemset(b->error, 0, 4)) != cudaSuccess) return e;
@@ -917,7 +1078,7 @@ cudaError_t prefill_alloc(PrefillBuffers *b, const edgefm_shape &sh, int chunk) 
 }
 
 void prefill_free(PrefillBuffers *b) {
-    cudaFree(b->resid); cudaFree(b->xn); cudaFree(b->part); cudaFree(b->q); cudaFree(b->attn); cudaFree(b->act); cudaFree(b->rope);
+    cudaFree(b->resid); cudaFree(b->xn); cudaFree(b->part); cudaFree(b->kv_stage); cudaFree(b->q); cudaFree(b->attn); cudaFree(b->act); cudaFree(b->rope);
     cudaFree(b->tokens); cudaFree(b->error);
     *b = PrefillBuffers{};
 }
@@ -939,7 +1100,10 @@ const char *prefill_run(const PrefillModel &m, PrefillBuffers *b, const int32_t 
     count += 2;
     for (int l = 0; l < sh.n_layers; ++l) {
         const edgefm_layer_weights &w = m.layers[l];
+        const bool kv8 = m.k_scale != nullptr;   // compressed cache: one byte per element and a scale per row
+        const size_t layer_rows = static_cast<size_t>(l) * nkv * m.max_context;
         uint16_t *kc = m.k_cache + static_cast<size_t>(l) * nkv * head_stride, *vc = m.v_cache + static_cast<size_t>(l) * nkv * head_stride;
+        signed char *kc8 = reinterpret_cast<signed char *>(m.k_cache) + layer_rows * d, *vc8 = reinterpret_cast<signed char *>(m.v_cache) + layer_rows * d;
         GemmArgs g{};
         g.M = n; g.error = b->error; g.wait_limit = b->wait_limit; g.extra_arrivals = b->extra_arrivals;
         g.N = n_qkv; g.K = H;
@@ -947,11 +1111,19 @@ const char *prefill_run(const PrefillModel &m, PrefillBuffers *b, const int32_t 
         g.rope = b->rope; g.q_out = b->q; g.q_plane = q_plane;
         g.k_rows = kc + static_cast<size_t>(slot0) * d; g.v_rows = vc + static_cast<size_t>(slot0) * d;
         g.nq = nq; g.nkv = nkv; g.d = d; g.head_stride = head_stride;
+        if (kv8) { g.k_stage = b->kv_stage; g.v_stage = b->kv_stage + cap * nkv * d; g.stage_stride = static_cast<long long>(cap) * d; }
         if (const char *e = launch_gemm<EPI_QKV>(b->xn, x_plane, w.wqkv, n_qkv, g, m.num_sms, s)) return e;
         ++count;
+        if (kv8) {   // the new rows, compressed into their cache slots (attention reads them from there, like every other row)
+            prefill_quantize_rows_kernel<<<(2 * nkv * n + 7) / 8, 256, 0, s>>>(g.k_stage, g.v_stage, g.stage_stride, kc8, vc8, m.k_scale + layer_rows,
+                                                                              m.v_scale + layer_rows, nkv, n, d, m.max_context, slot0);
+            ++count;
+        }
         if (l == sh.n_layers - 1) break;   // the rest of the last layer feeds nothing that is kept
-        const char *e = d == 64 ? launch_attention_tc<64>(b->q, kc, vc, b->attn, q_plane, n, slot0, nq, nkv, m.max_context, b->wait_limit, b->error, s)
-                                : launch_attention_tc<128>(b->q, kc, vc, b->attn, q_plane, n, slot0, nq, nkv, m.max_context, b->wait_limit, b->error, s);
+        const void *ka = kv8 ? static_cast<const void *>(kc8) : kc, *va = kv8 ? static_cast<const void *>(vc8) : vc;
+        const float *ksc = kv8 ? m.k_scale + layer_rows : nullptr, *vsc = kv8 ? m.v_scale + layer_rows : nullptr;
+        const char *e = d == 64 ? launch_attention_tc<64>(b->q, ka, va, ksc, vsc, b->attn, q_plane, n, slot0, nq, nkv, m.max_context, b->wait_limit, b->error, s)
+                                : launch_attention_tc<128>(b->q, ka, va, ksc, vsc, b->attn, q_plane, n, slot0, nq, nkv, m.max_context, b->wait_limit, b->error, s);
         if (e) return e;
         g.N = H; g.K = qd; g.resid = b->resid; g.part = b->part; g.part_plane = x_plane;
         if ((e = launch_gemm<EPI_RESID>(b->attn, q_plane, w.wo, H, g, m.num_sms, s))) return e;

@@ -21,6 +21,7 @@ struct PrefillBuffers {
     uint16_t *q = nullptr;       // rotated queries [2][chunk][nq d]
     uint16_t *attn = nullptr;    // attention output [2][chunk][nq d]
     uint16_t *act = nullptr;     // SwiGLU output [2][chunk][F]
+    float *kv_stage = nullptr;   // compressed cache only: fp32 k and v rows of the pass [2][nkv][chunk][d], before compression
     float2 *rope = nullptr;      // (cos, sin) of the chunk's positions, [chunk][d/2]
     int *tokens = nullptr;       // device copy of the chunk's token ids
     int *error = nullptr;        // device word: non-zero when a bounded wait of a GEMM ran out
@@ -32,7 +33,8 @@ struct PrefillModel {
     edgefm_shape shape;
     const edgefm_layer_weights *layers;   // host array
     const void *embed;
-    uint16_t *k_cache, *v_cache;          // bf16 [L][nkv][max_context][d]
+    uint16_t *k_cache, *v_cache;          // bf16 [L][nkv][max_context][d], or one signed byte per element (k_scale != nullptr)
+    float *k_scale, *v_scale;             // compressed cache: [L][nkv][max_context], else nullptr
     int max_context;
     StepState *state;
     int num_sms;
@@ -45,7 +47,7 @@ void prefill_plan_contraction(int epilogue, int M, int N, int K, int num_sms, in
 // Bytes the work buffers of a pass over `chunk` tokens take.
 size_t prefill_buffer_bytes(const edgefm_shape &sh, int chunk);
 // Allocate / free.  Returns a CUDA error.
-cudaError_t prefill_alloc(PrefillBuffers *b, const edgefm_shape &sh, int chunk);
+cudaError_t prefill_alloc(PrefillBuffers *b, const edgefm_shape &sh, int chunk, bool kv8);
 void prefill_free(PrefillBuffers *b);
 
 // Enqueue the layers for `n` tokens (host ids) whose cache rows go to slots [slot0, slot0 + n) at rotary positions
