@@ -571,6 +571,7 @@ constexpr int AT_BM = 128, AT_BN = 128, AT_PARTS = 2;
 constexpr int AT_KVS = 1;      // stages of the K / V tiles (one: the next K tile loads under this block's softmax, the next V
                                // tile under the next block's)
 constexpr int AT_PB = 1;       // buffers of the probabilities
+constexpr int AT_CW = 4;       // compressed cache: warps that expand the codes (AT_BN / AT_CW rows of a tile each)
 constexpr int AT_THREADS = 96 + 128 * AT_PARTS;   // producer, two issuers, softmax warps
 
 // B operand in MN-major form for P V: the V tile is D/64 blocks of [64 keys][64 d] (128-byte rows, 128-byte swizzle).  N (= d)
@@ -596,7 +597,7 @@ template <int D> struct AttnCfg {
 };
 
 template <int D, bool Q8>
-__global__ void __launch_bounds__(AT_THREADS + (Q8 ? 64 : 0)) prefill_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q_hi,
+__global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_attention_tc_kernel(const __grid_constant__ CUtensorMap map_q_hi,
                                                                    const __grid_constant__ CUtensorMap map_q_lo,
                                                                    const __grid_constant__ CUtensorMap map_k,
                                                                    const __grid_constant__ CUtensorMap map_v, uint16_t *out, size_t plane,
@@ -625,7 +626,7 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 64 : 0)) prefill_attention_
 
     if (threadIdx.x == 0) {
         mbar_init(&q_full, 1);
-        for (int i = 0; i < AT_KVS; ++i) { mbar_init(&k_full[i], Q8 ? 2 : 1); mbar_init(&k_empty[i], 1); mbar_init(&v_full[i], Q8 ? 2 : 1); mbar_init(&v_empty[i], 1); }
+        for (int i = 0; i < AT_KVS; ++i) { mbar_init(&k_full[i], Q8 ? AT_CW : 1); mbar_init(&k_empty[i], 1); mbar_init(&v_full[i], Q8 ? AT_CW : 1); mbar_init(&v_empty[i], 1); }
         mbar_init(&kraw_full, 1); mbar_init(&vraw_full, 1);
         for (int i = 0; i < AT_PB; ++i) { mbar_init(&p_full[i], 4 * AT_PARTS); mbar_init(&p_empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 4 * AT_PARTS); mbar_init(&o_full[i], 1); mbar_init(&o_empty[i], 4 * AT_PARTS); }
@@ -738,10 +739,11 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 64 : 0)) prefill_attention_
             mbar_wait(&drain_bar[1], 0, &dummy, wait_limit);
         }
     }
-    else if (Q8 && warp >= AT_THREADS / 32) {   // compressed cache: expand the 8-bit tiles to bf16 operand tiles (two warps, 64 rows each)
+    else if (Q8 && warp >= AT_THREADS / 32) {   // compressed cache: expand the 8-bit tiles to bf16 operand tiles (AT_CW warps, AT_BN / AT_CW rows each)
         static_assert(!Q8 || AT_KVS == 1, "one raw tile of K and of V in flight");
         const int cw = warp - AT_THREADS / 32;
         constexpr int LPR = D / 16, RPS = 32 / LPR;       // lanes per row of codes (16 codes each), rows per step
+        constexpr int ROWS = AT_BN / AT_CW;               // rows of a tile this warp expands
         auto warp_wait = [&](uint64_t *bar, int parity) {
             int r = 1;
             if (lane == 0) r = mbar_wait(bar, parity, &abort_flag, wait_limit) ? 1 : 0;
@@ -765,8 +767,8 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 64 : 0)) prefill_attention_
         };
         auto expand_tile = [&](uint8_t *tile, const uint8_t *raw) {
             // a lane takes 16 codes of a row; the lanes of a row all load before any of them stores (D = 128: in place)
-            for (int step = 0; step < 64 / RPS; ++step) {
-                const int row = cw * 64 + step * RPS + lane / LPR, c = lane % LPR;
+            for (int step = 0; step < ROWS / RPS; ++step) {
+                const int row = cw * ROWS + step * RPS + lane / LPR, c = lane % LPR;
                 const uint4 codes = *reinterpret_cast<const uint4 *>(raw + row * D + c * 16);
                 __syncwarp();
                 uint4 a, b;
@@ -782,10 +784,10 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 64 : 0)) prefill_attention_
             ok = warp_wait(&kraw_full, j & 1);
             if (!ok) break;
             expand_tile(k, D == 128 ? k : sp + AT_PB * C::P_BYTES);
-            for (int i = lane; i < 64; i += 32) {          // the scales of this block's keys (both kinds: they are in memory already)
-                const int key = min(j * AT_BN + cw * 64 + i, last_key);
-                sc_k[j & 3][cw * 64 + i] = k_scale[static_cast<size_t>(hk) * max_context + key];
-                sc_v[j & 3][cw * 64 + i] = v_scale[static_cast<size_t>(hk) * max_context + key];
+            for (int i = lane; i < ROWS; i += 32) {        // the scales of this block's keys (both kinds: they are in memory already)
+                const int key = min(j * AT_BN + cw * ROWS + i, last_key);
+                sc_k[j & 3][cw * ROWS + i] = k_scale[static_cast<size_t>(hk) * max_context + key];
+                sc_v[j & 3][cw * ROWS + i] = v_scale[static_cast<size_t>(hk) * max_context + key];
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
@@ -1021,7 +1023,7 @@ const char *launch_attention_tc(const uint16_t *q, const void *kc, const void *v
     if (q8) {
         if (cudaFuncSetAttribute(prefill_attention_tc_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<D>::SMEM_Q8) != cudaSuccess)
             return "cudaFuncSetAttribute failed";
-        prefill_attention_tc_kernel<D, true><<<grid, AT_THREADS + 64, AttnCfg<D>::SMEM_Q8, s>>>(
+        prefill_attention_tc_kernel<D, true><<<grid, AT_THREADS + 32 * AT_CW, AttnCfg<D>::SMEM_Q8, s>>>(
             mqh, mql, mk, mv, out, plane, T, slot0, nq, nq / nkv, max_context, scale_log2, wait_limit, error, k_scale, v_scale);
     } else {
         if (cudaFuncSetAttribute(prefill_attention_tc_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<D>::SMEM) != cudaSuccess)
