@@ -589,10 +589,12 @@ template <int D> struct AttnCfg {
     static constexpr int P_PIECE = (AT_BN / 64) * AT_BM * 128; // one piece: AT_BN / 64 blocks of [128 rows][64 keys]
     static constexpr int P_BYTES = 2 * P_PIECE;
     static constexpr int SMEM = Q_BYTES + AT_KVS * (K_BYTES + V_BYTES) + AT_PB * P_BYTES + 1024;
-    // compressed cache: the 8-bit tiles land in the first half of their bf16 tile's own place when a row of codes is as long as
-    // a 128-byte operand row (D = 128: every row is then expanded in place); D = 64 gets a landing area of its own
+    // compressed cache: the 8-bit K tile has a landing area of its own, so that it can load while the scores of the block
+    // before still read the operand tile; the V tile lands in the first half of its operand tile's own place when a row of
+    // codes is as long as a 128-byte operand row (D = 128: every row is then expanded in place; there is no room for a second
+    // landing area), D = 64 gets one
     static constexpr int RAW_BYTES = AT_BN * D;
-    static constexpr int SMEM_Q8 = SMEM + (D == 128 ? 0 : 2 * RAW_BYTES);
+    static constexpr int SMEM_Q8 = SMEM + (D == 128 ? 1 : 2) * RAW_BYTES;
     static constexpr int TMEM_COLS = 2 * AT_BN + 2 * D <= 256 ? 256 : 512;   // S0, S1, O0, O1
 };
 
@@ -609,8 +611,8 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
     // the scores by the keys' scales and folds the values' scales into the probabilities.
     using C = AttnCfg<D>;
     extern __shared__ uint8_t at_tc_dyn[];
-    __shared__ uint64_t kraw_full, vraw_full;
-    __shared__ float sc_k[Q8 ? 4 : 1][AT_BN], sc_v[Q8 ? 4 : 1][AT_BN];   // scales of the last four key blocks
+    __shared__ uint64_t kraw_full, kraw_empty, vraw_full;
+    __shared__ __align__(16) float sc_k[Q8 ? 4 : 1][AT_BN], sc_v[Q8 ? 4 : 1][AT_BN];   // scales of the last four key blocks
     __shared__ uint64_t q_full, k_full[AT_KVS], k_empty[AT_KVS], v_full[AT_KVS], v_empty[AT_KVS], s_full[2], s_empty[2], p_full[AT_PB], p_empty[AT_PB], o_full[2], o_empty[2], drain_bar[2], pair_bar[4];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
@@ -627,7 +629,7 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
     if (threadIdx.x == 0) {
         mbar_init(&q_full, 1);
         for (int i = 0; i < AT_KVS; ++i) { mbar_init(&k_full[i], Q8 ? AT_CW : 1); mbar_init(&k_empty[i], 1); mbar_init(&v_full[i], Q8 ? AT_CW : 1); mbar_init(&v_empty[i], 1); }
-        mbar_init(&kraw_full, 1); mbar_init(&vraw_full, 1);
+        mbar_init(&kraw_full, 1); mbar_init(&kraw_empty, AT_CW); mbar_init(&vraw_full, 1);
         for (int i = 0; i < AT_PB; ++i) { mbar_init(&p_full[i], 4 * AT_PARTS); mbar_init(&p_empty[i], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&s_full[i], 1); mbar_init(&s_empty[i], 4 * AT_PARTS); mbar_init(&o_full[i], 1); mbar_init(&o_empty[i], 4 * AT_PARTS); }
         mbar_init(&drain_bar[0], 1); mbar_init(&drain_bar[1], 1);
@@ -650,21 +652,28 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
             tma_load_2d(sq + kb * AT_BM * 128, &map_q_hi, h * D + kb * 64, t0, &q_full);
             tma_load_2d(sq + (C::KBLK + kb) * AT_BM * 128, &map_q_lo, h * D + kb * 64, t0, &q_full);
         }
-        // K and V of a block have barriers of their own: the K half of a stage is free again as soon as S_j is done, a block
-        // earlier than the V half, and the next scores need only K
-        int issued = 0;
-        for (int j = 0; j < nb; ++j) {
+        // K and V of a block have barriers of their own: the K tile is free again as soon as S_j is done, a block earlier than
+        // the V tile, and the next scores need only K.  Order of issue: K_0, then K_{j+1} before V_j, so that the wait for V's
+        // tile (P V of the block before) never holds the next K tile back.
+        int nk = 0, nv = 0;
+        auto load_k = [&](int j) {
             const int st = j % AT_KVS;
-            uint8_t *k = skv + st * (C::K_BYTES + C::V_BYTES), *v = k + C::K_BYTES;
-            if (j >= AT_KVS && !mbar_wait(&k_empty[st], ((j / AT_KVS) - 1) & 1, &abort_flag, wait_limit)) break;
+            uint8_t *k = skv + st * (C::K_BYTES + C::V_BYTES);
+            if (j >= AT_KVS && !mbar_wait(Q8 ? &kraw_empty : &k_empty[st], ((j / AT_KVS) - 1) & 1, &abort_flag, wait_limit)) return false;
             if constexpr (Q8) {
                 mbar_expect_tx(&kraw_full, C::RAW_BYTES);
-                tma_load_2d(D == 128 ? k : sp + AT_PB * C::P_BYTES, &map_k, 0, hk * max_context + j * AT_BN, &kraw_full);
+                tma_load_2d(sp + AT_PB * C::P_BYTES, &map_k, 0, hk * max_context + j * AT_BN, &kraw_full);
             } else {
                 mbar_expect_tx(&k_full[st], C::K_BYTES);
                 for (int kb = 0; kb < C::KBLK; ++kb) tma_load_2d(k + kb * AT_BN * 128, &map_k, kb * 64, hk * max_context + j * AT_BN, &k_full[st]);
             }
-            if (j >= AT_KVS && !mbar_wait(&v_empty[st], ((j / AT_KVS) - 1) & 1, &abort_flag, wait_limit)) { issued = -(j + 1); break; }
+            nk = j + 1;
+            return true;
+        };
+        auto load_v = [&](int j) {
+            const int st = j % AT_KVS;
+            uint8_t *v = skv + st * (C::K_BYTES + C::V_BYTES) + C::K_BYTES;
+            if (j >= AT_KVS && !mbar_wait(&v_empty[st], ((j / AT_KVS) - 1) & 1, &abort_flag, wait_limit)) return false;
             if constexpr (Q8) {
                 mbar_expect_tx(&vraw_full, C::RAW_BYTES);
                 tma_load_2d(D == 128 ? v : sp + AT_PB * C::P_BYTES + C::RAW_BYTES, &map_v, 0, hk * max_context + j * AT_BN, &vraw_full);
@@ -672,12 +681,17 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
                 mbar_expect_tx(&v_full[st], C::V_BYTES);
                 for (int kb = 0; kb < C::KBLK; ++kb) tma_load_2d(v + kb * AT_BN * 128, &map_v, kb * 64, hk * max_context + j * AT_BN, &v_full[st]);
             }
-            issued = j + 1;
+            nv = j + 1;
+            return true;
+        };
+        bool ok = load_k(0);
+        for (int j = 0; j < nb && ok; ++j) {
+            if (j + 1 < nb) ok = load_k(j + 1);
+            if (ok) ok = load_v(j);
         }
         if (abort_flag) {   // giving up: the copies in flight must land before the shared memory is released
             int dummy = 0;
             mbar_wait(&q_full, 0, &dummy, wait_limit);
-            const int nk = issued < 0 ? -issued : issued, nv = issued < 0 ? -issued - 1 : issued;
             for (int j = nk > AT_KVS ? nk - AT_KVS : 0; j < nk; ++j) mbar_wait(Q8 ? &kraw_full : &k_full[j % AT_KVS], (j / AT_KVS) & 1, &dummy, wait_limit);
             for (int j = nv > AT_KVS ? nv - AT_KVS : 0; j < nv; ++j) mbar_wait(Q8 ? &vraw_full : &v_full[j % AT_KVS], (j / AT_KVS) & 1, &dummy, wait_limit);
         }
@@ -766,24 +780,29 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
             hi8 = make_uint4(o[4], o[5], o[6], o[7]);
         };
         auto expand_tile = [&](uint8_t *tile, const uint8_t *raw) {
-            // a lane takes 16 codes of a row; the lanes of a row all load before any of them stores (D = 128: in place)
+            // a lane takes 16 codes of a row per step; the warp loads the codes of ALL its rows before it stores anything (D = 128:
+            // the operand rows overwrite the codes they came from), which also lets the loads overlap
+            uint4 codes[ROWS / RPS];
+#pragma unroll
+            for (int step = 0; step < ROWS / RPS; ++step)
+                codes[step] = *reinterpret_cast<const uint4 *>(raw + (cw * ROWS + step * RPS + lane / LPR) * D + (lane % LPR) * 16);
+            __syncwarp();
+#pragma unroll
             for (int step = 0; step < ROWS / RPS; ++step) {
                 const int row = cw * ROWS + step * RPS + lane / LPR, c = lane % LPR;
-                const uint4 codes = *reinterpret_cast<const uint4 *>(raw + row * D + c * 16);
-                __syncwarp();
                 uint4 a, b;
-                expand(codes, a, b);
+                expand(codes[step], a, b);
                 uint8_t *dst = tile + (c >> 2) * AT_BN * 128 + row * 128;
                 *reinterpret_cast<uint4 *>(dst + (((2 * (c & 3)) ^ (row & 7)) << 4)) = a;
                 *reinterpret_cast<uint4 *>(dst + (((2 * (c & 3) + 1) ^ (row & 7)) << 4)) = b;
             }
         };
-        bool ok = true;
-        for (int j = 0; j < nb && ok; ++j) {
-            uint8_t *k = skv, *v = k + C::K_BYTES;
-            ok = warp_wait(&kraw_full, j & 1);
-            if (!ok) break;
-            expand_tile(k, D == 128 ? k : sp + AT_PB * C::P_BYTES);
+        uint8_t *k = skv, *v = k + C::K_BYTES;
+        auto expand_k = [&](int j) {
+            if (!(warp_wait(&kraw_full, j & 1) && (j == 0 || warp_wait(&k_empty[0], (j - 1) & 1)))) return false;   // the codes are here, the operand tile is free
+            expand_tile(k, sp + AT_PB * C::P_BYTES);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&kraw_empty);       // the next K tile may land
             for (int i = lane; i < ROWS; i += 32) {        // the scales of this block's keys (both kinds: they are in memory already)
                 const int key = min(j * AT_BN + cw * ROWS + i, last_key);
                 sc_k[j & 3][cw * ROWS + i] = k_scale[static_cast<size_t>(hk) * max_context + key];
@@ -792,6 +811,12 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(&k_full[0]);
+            return true;
+        };
+        bool ok = expand_k(0);
+        for (int j = 0; j < nb && ok; ++j) {              // like the producer: the next K tile before this block's V tile
+            if (j + 1 < nb) ok = expand_k(j + 1);
+            if (!ok) break;
             ok = warp_wait(&vraw_full, j & 1);
             if (!ok) break;
             expand_tile(v, D == 128 ? v : sp + AT_PB * C::P_BYTES + C::RAW_BYTES);
@@ -850,9 +875,13 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
                 float v[32];
                 tmem_ld32(srow + c * 32, v);
                 tmem_ld_wait();
-                if constexpr (Q8) {
+                if constexpr (Q8) {                   // scores of codes -> scores: the keys' scales (16-byte shared-memory reads)
+                    const float4 *sk = reinterpret_cast<const float4 *>(&sc_k[j & 3][part * KP + c * 32]);
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] *= sc_k[j & 3][part * KP + c * 32 + i];
+                    for (int i = 0; i < 8; ++i) {
+                        const float4 f = sk[i];
+                        v[4 * i] *= f.x; v[4 * i + 1] *= f.y; v[4 * i + 2] *= f.z; v[4 * i + 3] *= f.w;
+                    }
                 }
                 if (diagonal) {
 #pragma unroll
@@ -881,9 +910,13 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
                 float v[32];
                 tmem_ld32(srow + c * 32, v);
                 tmem_ld_wait();
-                if constexpr (Q8) {
+                if constexpr (Q8) {                   // scores of codes -> scores: the keys' scales (16-byte shared-memory reads)
+                    const float4 *sk = reinterpret_cast<const float4 *>(&sc_k[j & 3][part * KP + c * 32]);
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] *= sc_k[j & 3][part * KP + c * 32 + i];
+                    for (int i = 0; i < 8; ++i) {
+                        const float4 f = sk[i];
+                        v[4 * i] *= f.x; v[4 * i + 1] *= f.y; v[4 * i + 2] *= f.z; v[4 * i + 3] *= f.w;
+                    }
                 }
                 if (diagonal) {
 #pragma unroll
@@ -902,8 +935,12 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
                         const float p0 = fast_exp2(fmaf(v[i], scale_log2, neg)), p1 = fast_exp2(fmaf(v[i + 1], scale_log2, neg));
                         sum0 += p0;
                         sum1 += p1;
-                        if constexpr (Q8) split2x2_trunc(p0 * sc_v[j & 3][kq + i], p1 * sc_v[j & 3][kq + i + 1], hw[i2], lw[i2]);
-                        else split2x2_trunc(p0, p1, hw[i2], lw[i2]);
+                        if constexpr (Q8) {           // the values' scales ride on the probabilities
+                            const float2 f = *reinterpret_cast<const float2 *>(&sc_v[j & 3][kq + i]);
+                            split2x2_trunc(p0 * f.x, p1 * f.y, hw[i2], lw[i2]);
+                        } else {
+                            split2x2_trunc(p0, p1, hw[i2], lw[i2]);
+                        }
                     }
                     const int piece16 = ((((kq & 63) >> 3) + i8) ^ (row & 7)) << 4;   // 16-byte piece index xor row bits (128-byte swizzle)
                     *reinterpret_cast<uint4 *>(prow_hi + piece16) = hi;
