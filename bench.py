@@ -261,8 +261,8 @@ def run_block(args, cfg):
 def run_prefill(args, cfg):
     """The prefill phase (edgefm_prefill) for a prompt of --prefill tokens into an empty cache: ms per prompt (median over
     --sequences calls, each between its own CUDA events), prompt tokens/s and the contraction rate.  Not the headline
-    workload.  Flops counted: 2 * tokens * (weights of the four projections of every layer that runs) + causal attention
-    (4 * d * n_q * sum over queries of the keys seen); the last prompt token is a decode step inside the same call."""
+    workload.  Flops counted: 2 * tokens * (weights of the four projections of every layer) + causal attention (4 * d * n_q * sum over
+    queries of the keys seen) + the output layer for the last token."""
     import torch
     from paper_2604_27476_b200 import DecodeContext, build as cuda_build, upload_weights
     cuda_build.build()
@@ -294,10 +294,10 @@ def run_prefill(args, cfg):
     times.sort()
     ms = statistics.median(times)
     H, F, d, nq, nkv, L = cfg.hidden, cfg.ffn, cfg.head_dim, cfg.n_q_heads, cfg.n_kv_heads, cfg.n_layers
-    n = T - 1
+    n = T
     qkv = (nq + 2 * nkv) * d * H
     rest = nq * d * H + 3 * H * F
-    flops = 2.0 * n * (L * qkv + (L - 1) * rest) + (L - 1) * 4.0 * d * nq * (n * (n + 1) / 2)
+    flops = 2.0 * n * L * (qkv + rest) + L * 4.0 * d * nq * (n * (n + 1) / 2) + 2.0 * cfg.vocab * H
     peaks = {}
     try:
         peaks = json.loads((ROOT / "MEASURED_PEAKS.json").read_text())
@@ -308,19 +308,20 @@ def run_prefill(args, cfg):
     line = {"metric": "prefill_ms_per_prompt", "value": ms, "unit": "ms", "n_gpus": 1, "steps": len(times), "warmup": max(args.warmup_sequences, 3),
             "ms_per_step": ms, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16 weights/KV, activations as two bf16 pieces, fp32 accumulate (tcgen05)" + (", 8-bit KV cache" if args.kv_format == "int8" else ""), "data": "synthetic",
-            "config": {"workload": f"{cfg.name}: prefill of {T} prompt tokens into an empty " + ("compressed (8-bit) " if args.kv_format == "int8" else "") + f"cache (edgefm_prefill; {n} tokens as dense contractions + one decode step)",
+            "config": {"workload": f"{cfg.name}: prefill of {T} prompt tokens into an empty " + ("compressed (8-bit) " if args.kv_format == "int8" else "") + f"cache (edgefm_prefill: dense contractions for all tokens, the output layer for the last one)",
                        "l2": "weights (> 2.6 GB) and activations exceed L2; nothing flushed"},
             "ms_min": times[0], "prompt_tokens_per_s": T / (ms * 1e-3),
             "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak, "traffic": None,
                          "note": "achieved counts the method's flops; the tensor cores execute twice that (two bf16 pieces per activation); peak = measured sustained cuBLAS bf16 rate" + ("" if peaks.get("bf16_tflops_sustained") else " (fallback)")},
-            "gpu_launches": len(times) * ctx_prefill_launches(cfg), "clocks": clocks}
+            "gpu_launches": len(times) * ctx_prefill_launches(cfg, args.kv_format == "int8"), "clocks": clocks}
     print(json.dumps(line), flush=True)
     ctx.close()
 
 
-def ctx_prefill_launches(cfg):
-    """Kernels one edgefm_prefill call enqueues: rope table + embedding/norm, 7 per layer but the last (QKV only), one step."""
-    return 2 + 7 * (cfg.n_layers - 1) + 1 + 1
+def ctx_prefill_launches(cfg, kv_int8=False):
+    """Kernels one edgefm_prefill call (8 tokens or more) enqueues: rope table + embedding/norm, 7 per layer (QKV, attention, O,
+    norm, gate/up, down, norm; one more per layer compresses the new rows of an 8-bit cache), the output layer."""
+    return 2 + (8 if kv_int8 else 7) * cfg.n_layers + 1
 
 
 def main():

@@ -188,12 +188,13 @@ edgefm_status edgefm_prefill_tokens(edgefm_ctx *ctx, const int32_t *tokens, int3
 
 /*
  * edgefm_prefill -- the prefill phase (Eq. 3 of the paper, KV <- Prefill(x_1:T; theta_p); with a prefix already in the cache,
- * Eq. 5: KV = Concat(KV_p, KV_u)) as dense contractions.  The first n - 1 tokens pass through the layers TOGETHER (at most
- * 2048 per pass): every projection is one [tokens x K] x [K x N] product on the tensor cores (tcgen05, fp32 accumulation in
+ * Eq. 5: KV = Concat(KV_p, KV_u)) as dense contractions.  The prompt's tokens pass through the layers TOGETHER (at most 2048
+ * per pass): every projection is one [tokens x K] x [K x N] product on the tensor cores (tcgen05, fp32 accumulation in
  * tensor memory; every activation enters as two bf16 pieces, hi + lo = 16 mantissa bits, the weights are bf16 exactly; fp32
  * residual stream), attention is causal over the cache rows 0 .. cur_len + t; the K and V rows go to cache slots cur_len ..
- * Token n - 1 then takes an ordinary decode step, so that logits_out / next_token_out and the device state are what
- * edgefm_decode_step leaves behind; decoding continues with edgefm_decode_step(ctx, -1, -1, ...).
+ * The output layer then runs for the last token alone (final norm, one matrix-vector pass, greedy token), and the device
+ * state is what a decode step of that token leaves behind: decoding continues with edgefm_decode_step(ctx, -1, -1, ...).
+ * (Prompts of fewer than 8 tokens: all but the last token dense, the last one an ordinary decode step.)
  * The cache rows agree with those of n decode steps up to the last bf16 step of a value.
  *   tokens     : HOST int32 [n], n >= 1, read during the call.
  *   position   : rotary position of tokens[0] (>= 0); token i has position + i.

@@ -259,6 +259,85 @@ __global__ void __launch_bounds__(256) prefill_quantize_rows_kernel(const float 
     if (lane == 0) (is_v ? vs : ks)[row] = amax > 0.f ? __fdiv_rn(amax, 127.0f) : 0.f;
 }
 
+// Output layer for ONE row (the prompt's last token): final RMSNorm, logits = W x over `rows` rows of the output matrix (bf16
+// weights, fp32 x and sums), greedy token (larger value wins, equal values -> lower row), and the device state a decode step
+// would leave.  A matrix-vector product: bound by the one pass over W.  grid: any; 256 threads; dynamic shared memory H floats.
+__global__ void __launch_bounds__(256) prefill_head_kernel(const float *x, const uint16_t *wnorm, const uint16_t *lm, const int *ids, int rows,
+                                                           int H, float eps, float *logits_out, int *next_token_out, float *part_val,
+                                                           int *part_idx, unsigned *ticket, StepState *st, int token, int pos) {
+    extern __shared__ __align__(16) float pf_xs[];
+    __shared__ float red[8], bvs[8];
+    __shared__ int bis[8], is_last;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    float ss = 0.f;
+    for (int j = tid; j < H; j += 256) ss = fmaf(x[j], x[j], ss);
+    ss = warp_sum(ss);
+    if (lane == 0) red[warp] = ss;
+    __syncthreads();
+    ss = ((red[0] + red[1]) + (red[2] + red[3])) + ((red[4] + red[5]) + (red[6] + red[7]));
+    const float r = rsqrtf(ss / static_cast<float>(H) + eps);
+    for (int j = tid; j < H; j += 256) pf_xs[j] = x[j] * r * bf16_bits_to_f32(wnorm[j]);
+    __syncthreads();
+    float bv = -INFINITY;
+    int bi = 0x7fffffff;
+    const int stride = gridDim.x * 8;
+    for (int row = blockIdx.x * 8 + warp; row < rows; row += 2 * stride) {   // two rows per round: more loads in flight
+        const int row2 = row + stride;
+        const uint16_t *w0 = lm + static_cast<size_t>(row) * H, *w1 = lm + static_cast<size_t>(row2 < rows ? row2 : row) * H;
+        float a0 = 0.f, a1 = 0.f;
+        for (int j = lane * 8; j < H; j += 256) {
+            const uint4 u0 = *reinterpret_cast<const uint4 *>(w0 + j), u1 = *reinterpret_cast<const uint4 *>(w1 + j);
+            const float4 x0 = *reinterpret_cast<const float4 *>(pf_xs + j), x1 = *reinterpret_cast<const float4 *>(pf_xs + j + 4);
+            a0 = dot8(u0, x0, x1, a0);
+            a1 = dot8(u1, x0, x1, a1);
+        }
+        a0 = warp_sum(a0);
+        a1 = warp_sum(a1);
+        if (lane == 0) {
+            if (logits_out) { logits_out[row] = a0; if (row2 < rows) logits_out[row2] = a1; }
+            if (arg_better(a0, row, bv, bi)) { bv = a0; bi = row; }
+            if (row2 < rows && arg_better(a1, row2, bv, bi)) { bv = a1; bi = row2; }
+        }
+    }
+    if (lane == 0) { bvs[warp] = bv; bis[warp] = bi; }
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < 8; ++w)
+            if (arg_better(bvs[w], bis[w], bv, bi)) { bv = bvs[w]; bi = bis[w]; }
+        part_val[blockIdx.x] = bv;
+        part_idx[blockIdx.x] = bi;
+        __threadfence();
+        is_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (is_last && warp == 0) {      // the last CTA to finish merges the CTAs' candidates
+        __threadfence();
+        bv = -INFINITY; bi = 0x7fffffff;
+        for (int i = lane; i < static_cast<int>(gridDim.x); i += 32) {
+            const float v = __ldcg(part_val + i);
+            const int ix = __ldcg(part_idx + i);
+            if (arg_better(v, ix, bv, bi)) { bv = v; bi = ix; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (arg_better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+        }
+        if (lane == 0) {
+            if (bi == 0x7fffffff) bi = 0;
+            if (ids) bi = ids[bi];   // pruned vocabulary: row index -> token id
+            if (next_token_out) *next_token_out = bi;
+            st->token = token;
+            st->position = pos;
+            st->next_token = bi;
+            st->next_position = pos + 1;
+            st->n_accepted = 1;
+            *ticket = 0u;
+        }
+    }
+}
+
 // ---- the contraction -------------------------------------------------------------------------------------------------------
 enum { EPI_QKV = 0, EPI_RESID = 1, EPI_SWIGLU = 2 };
 
@@ -1111,6 +1190,10 @@ cudaError_t prefill_alloc(PrefillBuffers *b, const edgefm_shape &sh, int chunk, 
     if (kv8 && (e = cudaMalloc(&b->kv_stage, 2 * c * sh.n_kv_heads * sh.head_dim * sizeof(float))) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->tokens, c * 4)) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->error, 4)) != cudaSuccess) return e;
+    if ((e = cudaMalloc(&b->head_val, PF_HEAD_GRID_MAX * 4)) != cudaSuccess) return e;
+    if ((e = cudaMalloc(&b->head_idx, PF_HEAD_GRID_MAX * 4)) != cudaSuccess) return e;
+    if ((e = cudaMalloc(&b->head_ticket, 4)) != cudaSuccess) return e;
+    if ((e = cudaMemset(b->head_ticket, 0, 4)) != cudaSuccess) return e;
     if ((e = cudaMemset(b->error, 0, 4)) != cudaSuccess) return e;
     b->chunk = chunk;
     return cudaSuccess;
@@ -1118,12 +1201,12 @@ cudaError_t prefill_alloc(PrefillBuffers *b, const edgefm_shape &sh, int chunk, 
 
 void prefill_free(PrefillBuffers *b) {
     cudaFree(b->resid); cudaFree(b->xn); cudaFree(b->part); cudaFree(b->kv_stage); cudaFree(b->q); cudaFree(b->attn); cudaFree(b->act); cudaFree(b->rope);
-    cudaFree(b->tokens); cudaFree(b->error);
+    cudaFree(b->tokens); cudaFree(b->error); cudaFree(b->head_val); cudaFree(b->head_idx); cudaFree(b->head_ticket);
     *b = PrefillBuffers{};
 }
 
-const char *prefill_run(const PrefillModel &m, PrefillBuffers *b, const int32_t *tokens, int n, int slot0, int position, cudaStream_t s,
-                        int *launches) {
+const char *prefill_run(const PrefillModel &m, PrefillBuffers *b, const int32_t *tokens, int n, int slot0, int position, bool whole_last_layer,
+                        cudaStream_t s, int *launches) {
     const edgefm_shape &sh = m.shape;
     const int H = sh.hidden, F = sh.ffn, d = sh.head_dim, nq = sh.n_q_heads, nkv = sh.n_kv_heads, qd = nq * d;
     const int n_qkv = (nq + 2 * nkv) * d;
@@ -1158,7 +1241,7 @@ const char *prefill_run(const PrefillModel &m, PrefillBuffers *b, const int32_t 
                                                                               m.v_scale + layer_rows, nkv, n, d, m.max_context, slot0);
             ++count;
         }
-        if (l == sh.n_layers - 1) break;   // the rest of the last layer feeds nothing that is kept
+        if (l == sh.n_layers - 1 && !whole_last_layer) break;   // the rest of the last layer feeds nothing that is kept
         const void *ka = kv8 ? static_cast<const void *>(kc8) : kc, *va = kv8 ? static_cast<const void *>(vc8) : vc;
         const float *ksc = kv8 ? m.k_scale + layer_rows : nullptr, *vsc = kv8 ? m.v_scale + layer_rows : nullptr;
         const char *e = d == 64 ? launch_attention_tc<64>(b->q, ka, va, ksc, vsc, b->attn, q_plane, n, slot0, nq, nkv, m.max_context, b->wait_limit, b->error, s)
@@ -1172,13 +1255,29 @@ const char *prefill_run(const PrefillModel &m, PrefillBuffers *b, const int32_t 
         if ((e = launch_gemm<EPI_SWIGLU>(b->xn, x_plane, w.w_gate_up, 2LL * F, g, m.num_sms, s))) return e;
         g.N = H; g.K = F;
         if ((e = launch_gemm<EPI_RESID>(b->act, f_plane, w.w_down, H, g, m.num_sms, s))) return e;
-        prefill_norm_kernel<<<norm_grid, 128, 0, s>>>(b->resid, b->xn, x_plane, static_cast<const uint16_t *>(m.layers[l + 1].input_norm), nullptr,
-                                                      nullptr, n, H, sh.rms_eps, nullptr, 0, 0, b->part, g.splits, x_plane);
+        // (behind the last layer the norm weights do not matter: the kernel runs for the K-split partial sums of the down projection)
+        prefill_norm_kernel<<<norm_grid, 128, 0, s>>>(b->resid, b->xn, x_plane, static_cast<const uint16_t *>(m.layers[l + 1 < sh.n_layers ? l + 1 : l].input_norm),
+                                                      nullptr, nullptr, n, H, sh.rms_eps, nullptr, 0, 0, b->part, g.splits, x_plane);
         count += 6;
     }
     if (cudaGetLastError() != cudaSuccess) return "prefill kernel launch failed";
     if (launches) *launches = count;
     return nullptr;
+}
+
+const char *prefill_head(const PrefillModel &m, PrefillBuffers *b, int row, const void *final_norm, const void *lm, const int *ids, int rows,
+                         float *logits_out, int *next_token_out, int token, int pos, cudaStream_t s) {
+    const int H = m.shape.hidden;
+    int grid = 2 * m.num_sms;
+    if (grid > PF_HEAD_GRID_MAX) grid = PF_HEAD_GRID_MAX;
+    if (grid * 8 > rows) grid = (rows + 7) / 8;
+    if (H * 4 > 48 * 1024 &&
+        cudaFuncSetAttribute(prefill_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, H * 4) != cudaSuccess)
+        return "cudaFuncSetAttribute failed";
+    prefill_head_kernel<<<grid, 256, static_cast<size_t>(H) * 4, s>>>(b->resid + static_cast<size_t>(row) * H, static_cast<const uint16_t *>(final_norm),
+                                                                     static_cast<const uint16_t *>(lm), ids, rows, H, m.shape.rms_eps, logits_out,
+                                                                     next_token_out, b->head_val, b->head_idx, b->head_ticket, m.state, token, pos);
+    return cudaGetLastError() == cudaSuccess ? nullptr : "prefill output layer launch failed";
 }
 
 }  // namespace edgefm

@@ -9,6 +9,7 @@
 
 namespace edgefm {
 
+constexpr int PF_HEAD_GRID_MAX = 1024;   // CTAs of the output-layer kernel
 constexpr int PF_CHUNK_MAX = 2048;   // tokens per pass over the layers (longer prompts take several passes)
 
 // Work buffers of one pass, owned by the context, allocated at the first prefill call.
@@ -25,6 +26,9 @@ struct PrefillBuffers {
     float2 *rope = nullptr;      // (cos, sin) of the chunk's positions, [chunk][d/2]
     int *tokens = nullptr;       // device copy of the chunk's token ids
     int *error = nullptr;        // device word: non-zero when a bounded wait of a GEMM ran out
+    float *head_val = nullptr;   // output layer: the CTAs' greedy candidates
+    int *head_idx = nullptr;
+    unsigned *head_ticket = nullptr;
     uint32_t wait_limit = 1u << 24;   // polls per wait (far beyond any legitimate wait of a tile)
     uint32_t extra_arrivals = 0;      // tests only: 1 makes the first wait of every contraction run out
 };
@@ -51,10 +55,17 @@ cudaError_t prefill_alloc(PrefillBuffers *b, const edgefm_shape &sh, int chunk, 
 void prefill_free(PrefillBuffers *b);
 
 // Enqueue the layers for `n` tokens (host ids) whose cache rows go to slots [slot0, slot0 + n) at rotary positions
-// position .. position + n - 1.  Every layer's K and V rows are written; the last layer's attention and MLP are skipped
-// (their result would only feed an output layer nobody reads).  Sets the device state to cache length slot0 + n.
+// position .. position + n - 1.  Every layer's K and V rows are written.  whole_last_layer = false: the last layer's attention
+// and MLP are skipped (their result would only feed an output layer nobody reads); true: they run, and the residual stream
+// behind the last layer is left in PrefillBuffers::resid for prefill_head.  Sets the device state to cache length slot0 + n.
 // Returns nullptr or a message.
-const char *prefill_run(const PrefillModel &m, PrefillBuffers *b, const int32_t *tokens, int n, int slot0, int position,
+const char *prefill_run(const PrefillModel &m, PrefillBuffers *b, const int32_t *tokens, int n, int slot0, int position, bool whole_last_layer,
                         cudaStream_t stream, int *launches);
+
+// The output layer for row `row` of the residual stream of the last pass: final norm, logits over `rows` rows of `lm` (ids:
+// their token ids when the vocabulary is pruned, else nullptr), greedy token; leaves the device state as a decode step of
+// `token` at `pos` would.  logits_out / next_token_out: device pointers or nullptr.
+const char *prefill_head(const PrefillModel &m, PrefillBuffers *b, int row, const void *final_norm, const void *lm, const int *ids, int rows,
+                         float *logits_out, int *next_token_out, int token, int pos, cudaStream_t stream);
 
 }  // namespace edgefm
