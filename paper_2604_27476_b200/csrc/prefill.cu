@@ -558,18 +558,25 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
                                 const float2 *cs = g.rope + static_cast<size_t>(row) * half + j0;
 #pragma unroll
                                 for (int i = 0; i < 4; ++i) {
-                                    float a[8], b[8];
+                                    float a[8], b[8], bx[8], by[8];
+                                    if (g.bias) {                        // eight biases per 16-byte load
+                                        const uint4 u = *reinterpret_cast<const uint4 *>(g.bias + col0 + j0 + 8 * i);
+                                        const uint4 w = *reinterpret_cast<const uint4 *>(g.bias + col0 + half + j0 + 8 * i);
+                                        bx[0] = bf16lo(u.x); bx[1] = bf16hi(u.x); bx[2] = bf16lo(u.y); bx[3] = bf16hi(u.y);
+                                        bx[4] = bf16lo(u.z); bx[5] = bf16hi(u.z); bx[6] = bf16lo(u.w); bx[7] = bf16hi(u.w);
+                                        by[0] = bf16lo(w.x); by[1] = bf16hi(w.x); by[2] = bf16lo(w.y); by[3] = bf16hi(w.y);
+                                        by[4] = bf16lo(w.z); by[5] = bf16hi(w.z); by[6] = bf16lo(w.w); by[7] = bf16hi(w.w);
+                                    }
 #pragma unroll
-                                    for (int j = 0; j < 8; ++j) {
+                                    for (int j = 0; j < 8; j += 2) {
                                         const int e = 8 * i + j;
-                                        float x = lo[e], y = hi[e];
-                                        if (g.bias) {
-                                            x += bf16_bits_to_f32(g.bias[col0 + j0 + e]);
-                                            y += bf16_bits_to_f32(g.bias[col0 + half + j0 + e]);
-                                        }
-                                        const float2 t = cs[e];
-                                        a[j] = x * t.x - y * t.y;
-                                        b[j] = y * t.x + x * t.y;
+                                        const float4 t = *reinterpret_cast<const float4 *>(cs + e);   // (cos, sin) of two pairs
+                                        float x0 = lo[e], y0 = hi[e], x1 = lo[e + 1], y1 = hi[e + 1];
+                                        if (g.bias) { x0 += bx[j]; y0 += by[j]; x1 += bx[j + 1]; y1 += by[j + 1]; }
+                                        a[j] = x0 * t.x - y0 * t.y;
+                                        b[j] = y0 * t.x + x0 * t.y;
+                                        a[j + 1] = x1 * t.z - y1 * t.w;
+                                        b[j + 1] = y1 * t.z + x1 * t.w;
                                     }
                                     uint4 ah, al, bh, bl;
                                     split2x2(a[0], a[1], ah.x, al.x); split2x2(a[2], a[3], ah.y, al.y);
@@ -1230,6 +1237,7 @@ const char *prefill_run(const PrefillModel &m, PrefillBuffers *b, const int32_t 
         g.M = n; g.error = b->error; g.wait_limit = b->wait_limit; g.extra_arrivals = b->extra_arrivals;
         g.N = n_qkv; g.K = H;
         g.bias = sh.qkv_bias ? static_cast<const uint16_t *>(w.bqkv) : nullptr;
+        if (g.bias && (reinterpret_cast<uintptr_t>(g.bias) & 15u)) return "edgefm_prefill reads bqkv in 16-byte pieces: the vector must be 16-byte aligned";
         g.rope = b->rope; g.q_out = b->q; g.q_plane = q_plane;
         g.k_rows = kc + static_cast<size_t>(slot0) * d; g.v_rows = vc + static_cast<size_t>(slot0) * d;
         g.nq = nq; g.nkv = nkv; g.d = d; g.head_stride = head_stride;
