@@ -75,7 +75,7 @@ def run_case(cfg, T0, n, seed, follow=True):
         pair.close()
 
 
-@pytest.mark.parametrize("T0,n", [(0, 2), (0, 9), (20, 200), (37, 130), (64, 1), (3, 65)])
+@pytest.mark.parametrize("T0,n", [(0, 2), (0, 7), (0, 8), (0, 9), (20, 200), (37, 130), (64, 1), (3, 65), (0, 128), (5, 257), (123, 384)])
 def test_prompt_as_dense_contractions_tiny(T0, n):
     run_case(CONFIGS["tiny"].with_(qkv_bias=True), T0, n, 300 + n)
 
