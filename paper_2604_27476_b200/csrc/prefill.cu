@@ -111,6 +111,17 @@ template <int N> __device__ __forceinline__ void tmem_ld(uint32_t taddr, float *
         for (int c = 0; c < N / 32; ++c) tmem_ld32(taddr + c * 32, v + c * 32);
     }
 }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float *v) {
+    const uint32_t *r = reinterpret_cast<const uint32_t *>(v);
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, "
+        "%19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]),
+        "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]),
+        "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Shared-memory matrix descriptor of a K-major bf16 tile written by TMA with the 128-byte swizzle: rows of 64 elements
@@ -648,10 +659,11 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
 // tensor memory;  the softmax warps read their part of the row twice (tcgen05.ld; once for the maximum, once for the
 // exponentials), mask on diagonal blocks, update the running maximum and sum, and write the probabilities as two bf16 pieces
 // into shared memory in the swizzled K-major layout of an A operand;  O_j = P_j V_j (M 128, N = D, K = 128 keys; V straight
-// from its cache rows as an MN-major B operand) into one of two O buffers;  the softmax warps add O_j to their fp32 row in
-// registers, o = o * alpha_j + O_j, one block late so that the multiply hides under the next block's softmax.  The scores
-// and P V are issued by two threads (warps 1 and 2), the K and V tiles have barriers of their own.
-//   tensor memory: S0 [0, 128), S1 [128, 256), O0 [256, 256 + D), O1 [256 + D, 256 + 2 D)      (512 columns allocated)
+// from its cache rows as an MN-major B operand), accumulated over the blocks in tensor memory;  the exponentials are taken
+// against a reference maximum that moves only when a row's maximum has grown by more than 2^8 (then the row of O and the row
+// sum are rescaled once, tcgen05.ld / tcgen05.st).  The scores and P V are issued by two threads (warps 1 and 2), the K and V
+// tiles have barriers of their own.
+//   tensor memory: S0 [0, 128), S1 [128, 256), O [256, 256 + D)      (512 columns allocated)
 //   shared memory: Q 2 x D/64 x 16 KB | K D/64 x 16 KB | V D/64 x 16 KB | P 2 x 2 x 16 KB
 constexpr int AT_BM = 128, AT_BN = 128, AT_PARTS = 2;
 constexpr int AT_KVS = 1;      // stages of the K / V tiles (one: the next K tile loads under this block's softmax, the next V
@@ -814,9 +826,8 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
         constexpr uint32_t idesc_o = umma_idesc_bf16(AT_BM, D) | (1u << 16);   // B (= V) is MN-major
         bool ok = true;
         for (int j = 0; j < nb && ok; ++j) {
-            const int st = j % AT_KVS, pb = j % AT_PB, ob = j & 1;
+            const int st = j % AT_KVS, pb = j % AT_PB;
             ok = mbar_wait(&v_full[st], (j / AT_KVS) & 1, &abort_flag, wait_limit);
-            if (ok && j >= 2) ok = mbar_wait(&o_empty[ob], ((j >> 1) - 1) & 1, &abort_flag, wait_limit);   // O_{j-2} has been added
             if (ok) ok = mbar_wait(&p_full[pb], (j / AT_PB) & 1, &abort_flag, wait_limit);
             if (!ok) break;
             tc_fence_after();
@@ -826,10 +837,10 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
                 const uint32_t pa = smem_u32(sp) + pb * C::P_BYTES + piece * C::P_PIECE;
 #pragma unroll
                 for (int kk = 0; kk < AT_BN / 16; ++kk)   // 16 keys: 32 bytes along a P row (64-key blocks 16 KB apart), 2048 bytes of the V tile
-                    umma_bf16(tmem + 2 * AT_BN + ob * D, umma_desc_sw128(pa + (kk >> 2) * AT_BM * 128) + 2 * (kk & 3),
-                              umma_desc_sw128_mn(v + kk * 2048, AT_BN * 128), idesc_o, (piece | kk) != 0);
+                    umma_bf16(tmem + 2 * AT_BN, umma_desc_sw128(pa + (kk >> 2) * AT_BM * 128) + 2 * (kk & 3),
+                              umma_desc_sw128_mn(v + kk * 2048, AT_BN * 128), idesc_o, (j | piece | kk) != 0);   // O accumulates over the blocks
             }
-            umma_commit(&o_full[ob]);
+            umma_commit(&o_full[0]);
             umma_commit(&p_empty[pb]);
             umma_commit(&v_empty[st]);
         }
@@ -917,10 +928,11 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
         const int qi = slot0 + t0 + row;     // cache slot of this query: it sees the keys 0 .. qi
         constexpr int KP = AT_BN / AT_PARTS; // keys of a block per thread
         constexpr int DP = D / AT_PARTS;     // this thread's columns of the output row
-        float o[DP];
-#pragma unroll
-        for (int i = 0; i < DP; ++i) o[i] = 0.f;
-        float m_run = -INFINITY, l_run = 0.f, alpha_prev = 1.f;
+        // The output row accumulates in tensor memory over the blocks (P V with accumulation).  The exponentials are taken
+        // against a reference maximum m_ref that moves only when the row's maximum has grown by more than 2^8 in the
+        // exponent (or at the first block); then the row of O and the row sum are rescaled once.  In between the
+        // probabilities may reach 2^8, which fp32 sums and the two bf16 pieces carry without loss.
+        float m_ref = -INFINITY, l_run = 0.f;
         bool ok = true;
         // one lane waits / arrives for its warp (an mbarrier operation per thread would cost more than the arithmetic)
         auto warp_wait = [&](uint64_t *bar, int parity) {
@@ -935,18 +947,6 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
         auto row_sync = [&](int round) {     // the AT_PARTS warps of a quarter meet (bounded like every other wait)
             warp_arrive(&pair_bar[quarter]);
             return warp_wait(&pair_bar[quarter], round & 1);
-        };
-        auto add_block = [&](int j) {        // o = o * alpha_j + O_j
-            ok = warp_wait(&o_full[j & 1], (j >> 1) & 1);
-            if (!ok) return;
-            tc_fence_after();
-            float v[DP];
-            tmem_ld<DP>(trow + 2 * AT_BN + (j & 1) * D + part * DP, v);
-            tmem_ld_wait();
-            tc_fence_before();
-            warp_arrive(&o_empty[j & 1]);
-#pragma unroll
-            for (int i = 0; i < DP; ++i) o[i] = fmaf(o[i], alpha_prev, v[i]);
         };
         for (int j = 0; j < nb; ++j) {
             ok = warp_wait(&s_full[j & 1], (j >> 1) & 1);
@@ -980,12 +980,35 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
             xchg[j & 1][part][row] = mx;     // the row maximum needs the other threads' keys
             ok = row_sync(j);
             if (!ok) break;
-            mx = m_run;
+            mx = m_ref;
 #pragma unroll
             for (int q = 0; q < AT_PARTS; ++q) mx = fmaxf(mx, xchg[j & 1][q][row]);
-            const float alpha = fast_exp2((m_run - mx) * scale_log2);   // first block: exp2(-inf) = 0
-            m_run = mx;
-            const float neg = -mx * scale_log2;
+            if (j == 0) {
+                m_ref = mx;                  // nothing accumulated yet
+            } else if (__any_sync(0xffffffffu, (mx - m_ref) * scale_log2 > 8.f)) {
+                // some row of this warp has outgrown its reference (both warps of a quarter see the same rows and maxima, so they
+                // decide alike): every row moves its reference to its maximum and rescales its sum and its part of O, once the
+                // multiplies of the blocks before are done (the next one waits for this block's probabilities)
+                ok = warp_wait(&o_full[0], (j - 1) & 1);
+                if (!ok) break;
+                tc_fence_after();
+                const float f = fast_exp2((m_ref - mx) * scale_log2);
+                l_run *= f;
+#pragma unroll
+                for (int c = 0; c < DP / 32; ++c) {
+                    static_assert(DP % 32 == 0, "32 columns per tensor-memory access");
+                    float v[32];
+                    tmem_ld32(trow + 2 * AT_BN + part * DP + c * 32, v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] *= f;
+                    tmem_st32(trow + 2 * AT_BN + part * DP + c * 32, v);
+                }
+                tmem_st_wait();
+                tc_fence_before();
+                m_ref = mx;
+            }
+            const float neg = -m_ref * scale_log2;
             if (j >= AT_PB) {                // the P buffer's previous block has been multiplied
                 ok = warp_wait(&p_empty[j % AT_PB], ((j / AT_PB) - 1) & 1);
                 if (!ok) break;
@@ -1033,15 +1056,19 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
                     *reinterpret_cast<uint4 *>(prow_lo + piece16) = lo;
                 }
             }
-            l_run = l_run * alpha + (sum0 + sum1);
+            l_run += sum0 + sum1;
             tc_fence_before();
             warp_arrive(&s_empty[j & 1]);    // this part of S_j has been read twice
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P: generic-proxy writes before the tensor core's reads
             warp_arrive(&p_full[j % AT_PB]);
-            if (j >= 1) { add_block(j - 1); if (!ok) break; }
-            alpha_prev = alpha;
         }
-        if (ok) add_block(nb - 1);
+        float o[DP];
+        if (ok) ok = warp_wait(&o_full[0], (nb - 1) & 1);   // the last block's multiply
+        if (ok) {
+            tc_fence_after();
+            tmem_ld<DP>(trow + 2 * AT_BN + part * DP, o);
+            tmem_ld_wait();
+        }
         if (ok) {
             xchg[nb & 1][part][row] = l_run; // the parts of the row sum
             ok = row_sync(nb);
