@@ -76,6 +76,15 @@ __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint
         "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// The same with the A operand in tensor memory (lane = row, 16-bit elements packed two per column, K along the columns).
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
 // The mbarrier receives one arrival when every tcgen05.mma issued so far by this thread has finished.
 __device__ __forceinline__ void umma_commit(uint64_t *bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
@@ -657,18 +666,18 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
 // One CTA = 128 queries of one head (a query = a lane of tensor memory, two softmax threads per query); keys in blocks of 128.
 // Per block j:  S_j = Q K_j^T (tcgen05.mma, M 128, N 128, K = D; queries as two bf16 pieces) into one of two S buffers in
 // tensor memory;  the softmax warps read their part of the row twice (tcgen05.ld; once for the maximum, once for the
-// exponentials), mask on diagonal blocks, update the running maximum and sum, and write the probabilities as two bf16 pieces
-// into shared memory in the swizzled K-major layout of an A operand;  O_j = P_j V_j (M 128, N = D, K = 128 keys; V straight
+// exponentials), mask on diagonal blocks, update the running maximum and sum, and store the probabilities as two bf16 pieces
+// into tensor memory (tcgen05.st, two keys per column);  O_j = P_j V_j (M 128, N = D, K = 128 keys; P from tensor memory, V straight
 // from its cache rows as an MN-major B operand), accumulated over the blocks in tensor memory;  the exponentials are taken
 // against a reference maximum that moves only when a row's maximum has grown by more than 2^8 (then the row of O and the row
 // sum are rescaled once, tcgen05.ld / tcgen05.st).  The scores and P V are issued by two threads (warps 1 and 2), the K and V
 // tiles have barriers of their own.
-//   tensor memory: S0 [0, 128), S1 [128, 256), O [256, 256 + D)      (512 columns allocated)
-//   shared memory: Q 2 x D/64 x 16 KB | K D/64 x 16 KB | V D/64 x 16 KB | P 2 x 2 x 16 KB
+//   tensor memory: S0 [0, 128), S1 [128, 256), O [256, 256 + D), P hi [384, 448), P lo [448, 512)
+//   shared memory: Q 2 x D/64 x 16 KB | 2 stages x (K D/64 x 16 KB, V D/64 x 16 KB)   (compressed cache: one stage + landing areas)
 constexpr int AT_BM = 128, AT_BN = 128, AT_PARTS = 2;
-constexpr int AT_KVS = 1;      // stages of the K / V tiles (one: the next K tile loads under this block's softmax, the next V
-                               // tile under the next block's)
-constexpr int AT_PB = 1;       // buffers of the probabilities
+constexpr int AT_KVS_MAX = 2;  // stages of the K / V tiles: two on the bf16 cache, one on the compressed cache (whose tiles are
+                               // expanded in place)
+constexpr int AT_PB = 1;       // buffers of the probabilities (in tensor memory)
 constexpr int AT_CW = 4;       // compressed cache: warps that expand the codes (AT_BN / AT_CW rows of a tile each)
 constexpr int AT_THREADS = 96 + 128 * AT_PARTS;   // producer, two issuers, softmax warps
 
@@ -684,15 +693,13 @@ template <int D> struct AttnCfg {
     static constexpr int KBLK = D / 64;                        // 64-column blocks of a row of q, k, v
     static constexpr int Q_BYTES = 2 * KBLK * AT_BM * 128;     // two pieces
     static constexpr int K_BYTES = KBLK * AT_BN * 128, V_BYTES = K_BYTES;
-    static constexpr int P_PIECE = (AT_BN / 64) * AT_BM * 128; // one piece: AT_BN / 64 blocks of [128 rows][64 keys]
-    static constexpr int P_BYTES = 2 * P_PIECE;
-    static constexpr int SMEM = Q_BYTES + AT_KVS * (K_BYTES + V_BYTES) + AT_PB * P_BYTES + 1024;
+    static constexpr int SMEM = Q_BYTES + 2 * (K_BYTES + V_BYTES) + 1024;     // bf16 cache: two stages of K and V
     // compressed cache: the 8-bit K tile has a landing area of its own, so that it can load while the scores of the block
     // before still read the operand tile; the V tile lands in the first half of its operand tile's own place when a row of
     // codes is as long as a 128-byte operand row (D = 128: every row is then expanded in place; there is no room for a second
     // landing area), D = 64 gets one
     static constexpr int RAW_BYTES = AT_BN * D;
-    static constexpr int SMEM_Q8 = SMEM + (D == 128 ? 1 : 2) * RAW_BYTES;
+    static constexpr int SMEM_Q8 = Q_BYTES + (K_BYTES + V_BYTES) + (D == 128 ? 1 : 2) * RAW_BYTES + 1024;
     static constexpr int TMEM_COLS = 2 * AT_BN + 2 * D <= 256 ? 256 : 512;   // S0, S1, O0, O1
 };
 
@@ -711,12 +718,14 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
     extern __shared__ uint8_t at_tc_dyn[];
     __shared__ uint64_t kraw_full, kraw_empty, vraw_full;
     __shared__ __align__(16) float sc_k[Q8 ? 4 : 1][AT_BN], sc_v[Q8 ? 4 : 1][AT_BN];   // scales of the last four key blocks
-    __shared__ uint64_t q_full, k_full[AT_KVS], k_empty[AT_KVS], v_full[AT_KVS], v_empty[AT_KVS], s_full[2], s_empty[2], p_full[AT_PB], p_empty[AT_PB], o_full[2], o_empty[2], drain_bar[2], pair_bar[4];
+    constexpr int AT_KVS = Q8 ? 1 : 2;
+    __shared__ uint64_t q_full, k_full[AT_KVS_MAX], k_empty[AT_KVS_MAX], v_full[AT_KVS_MAX], v_empty[AT_KVS_MAX], s_full[2], s_empty[2], p_full[AT_PB], p_empty[AT_PB], o_full[2], o_empty[2], drain_bar[2], pair_bar[4];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     __shared__ float xchg[2][AT_PARTS][AT_BM];      // row maxima / sums passed between the two threads of a row
     uint8_t *base = at_tc_dyn + ((1024u - (smem_u32(at_tc_dyn) & 1023u)) & 1023u);
-    uint8_t *sq = base, *skv = sq + C::Q_BYTES, *sp = skv + AT_KVS * (C::K_BYTES + C::V_BYTES);
+    uint8_t *sq = base, *skv = sq + C::Q_BYTES, *sraw = skv + AT_KVS * (C::K_BYTES + C::V_BYTES);   // sraw: landing area of the codes (Q8)
+    const uint32_t tmem_p_off = 2 * AT_BN + 128;             // P in tensor memory: hi piece 64 columns (128 keys, two per column), then lo
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // grid (heads, query tiles): CTAs start in linear order, so every head's longest tile (the last queries) starts first
     const int t0 = (gridDim.y - 1 - blockIdx.y) * AT_BM;
@@ -760,7 +769,7 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
             if (j >= AT_KVS && !mbar_wait(Q8 ? &kraw_empty : &k_empty[st], ((j / AT_KVS) - 1) & 1, &abort_flag, wait_limit)) return false;
             if constexpr (Q8) {
                 mbar_expect_tx(&kraw_full, C::RAW_BYTES);
-                tma_load_2d(sp + AT_PB * C::P_BYTES, &map_k, 0, hk * max_context + j * AT_BN, &kraw_full);
+                tma_load_2d(sraw, &map_k, 0, hk * max_context + j * AT_BN, &kraw_full);
             } else {
                 mbar_expect_tx(&k_full[st], C::K_BYTES);
                 for (int kb = 0; kb < C::KBLK; ++kb) tma_load_2d(k + kb * AT_BN * 128, &map_k, kb * 64, hk * max_context + j * AT_BN, &k_full[st]);
@@ -774,7 +783,7 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
             if (j >= AT_KVS && !mbar_wait(&v_empty[st], ((j / AT_KVS) - 1) & 1, &abort_flag, wait_limit)) return false;
             if constexpr (Q8) {
                 mbar_expect_tx(&vraw_full, C::RAW_BYTES);
-                tma_load_2d(D == 128 ? v : sp + AT_PB * C::P_BYTES + C::RAW_BYTES, &map_v, 0, hk * max_context + j * AT_BN, &vraw_full);
+                tma_load_2d(D == 128 ? v : sraw + C::RAW_BYTES, &map_v, 0, hk * max_context + j * AT_BN, &vraw_full);
             } else {
                 mbar_expect_tx(&v_full[st], C::V_BYTES);
                 for (int kb = 0; kb < C::KBLK; ++kb) tma_load_2d(v + kb * AT_BN * 128, &map_v, kb * 64, hk * max_context + j * AT_BN, &v_full[st]);
@@ -834,11 +843,10 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
             const uint32_t v = smem_u32(skv + st * (C::K_BYTES + C::V_BYTES) + C::K_BYTES);
 #pragma unroll
             for (int piece = 0; piece < 2; ++piece) {
-                const uint32_t pa = smem_u32(sp) + pb * C::P_BYTES + piece * C::P_PIECE;
 #pragma unroll
-                for (int kk = 0; kk < AT_BN / 16; ++kk)   // 16 keys: 32 bytes along a P row (64-key blocks 16 KB apart), 2048 bytes of the V tile
-                    umma_bf16(tmem + 2 * AT_BN, umma_desc_sw128(pa + (kk >> 2) * AT_BM * 128) + 2 * (kk & 3),
-                              umma_desc_sw128_mn(v + kk * 2048, AT_BN * 128), idesc_o, (j | piece | kk) != 0);   // O accumulates over the blocks
+                for (int kk = 0; kk < AT_BN / 16; ++kk)   // 16 keys: 8 columns of P in tensor memory, 2048 bytes of the V tile
+                    umma_bf16_ts(tmem + 2 * AT_BN, tmem + tmem_p_off + piece * (AT_BN / 2) + kk * 8,
+                                 umma_desc_sw128_mn(v + kk * 2048, AT_BN * 128), idesc_o, (j | piece | kk) != 0);   // O accumulates over the blocks
             }
             umma_commit(&o_full[0]);
             umma_commit(&p_empty[pb]);
@@ -897,7 +905,7 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
         uint8_t *k = skv, *v = k + C::K_BYTES;
         auto expand_k = [&](int j) {
             if (!(warp_wait(&kraw_full, j & 1) && (j == 0 || warp_wait(&k_empty[0], (j - 1) & 1)))) return false;   // the codes are here, the operand tile is free
-            expand_tile(k, sp + AT_PB * C::P_BYTES);
+            expand_tile(k, sraw);
             __syncwarp();
             if (lane == 0) mbar_arrive(&kraw_empty);       // the next K tile may land
             for (int i = lane; i < ROWS; i += 32) {        // the scales of this block's keys (both kinds: they are in memory already)
@@ -916,7 +924,7 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
             if (!ok) break;
             ok = warp_wait(&vraw_full, j & 1);
             if (!ok) break;
-            expand_tile(v, D == 128 ? v : sp + AT_PB * C::P_BYTES + C::RAW_BYTES);
+            expand_tile(v, D == 128 ? v : sraw + C::RAW_BYTES);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(&v_full[0]);
@@ -1014,8 +1022,9 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
                 if (!ok) break;
             }
             float sum0 = 0.f, sum1 = 0.f;
+            uint32_t phi[KP / 2], plo[KP / 2];    // this thread's probabilities, two keys per word
 #pragma unroll
-            for (int c = 0; c < KP / 32; ++c) {   // pass 2: probabilities as two bf16 pieces, into the A-operand layout
+            for (int c = 0; c < KP / 32; ++c) {   // pass 2: probabilities as two bf16 pieces
                 float v[32];
                 tmem_ld32(srow + c * 32, v);
                 tmem_ld_wait();
@@ -1033,34 +1042,28 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
                         if (key0 + c * 32 + i > qi) v[i] = -INFINITY;
                 }
                 const int kq = part * KP + c * 32;            // first key of this chunk within the block
-                uint8_t *prow_hi = sp + (j % AT_PB) * C::P_BYTES + (kq >> 6) * AT_BM * 128 + row * 128, *prow_lo = prow_hi + C::P_PIECE;
 #pragma unroll
-                for (int i8 = 0; i8 < 4; ++i8) {
-                    uint4 hi, lo;
-                    uint32_t *hw = &hi.x, *lw = &lo.x;
-#pragma unroll
-                    for (int i2 = 0; i2 < 4; ++i2) {
-                        const int i = i8 * 8 + i2 * 2;
-                        const float p0 = fast_exp2(fmaf(v[i], scale_log2, neg)), p1 = fast_exp2(fmaf(v[i + 1], scale_log2, neg));
-                        sum0 += p0;
-                        sum1 += p1;
-                        if constexpr (Q8) {           // the values' scales ride on the probabilities
-                            const float2 f = *reinterpret_cast<const float2 *>(&sc_v[j & 3][kq + i]);
-                            split2x2_trunc(p0 * f.x, p1 * f.y, hw[i2], lw[i2]);
-                        } else {
-                            split2x2_trunc(p0, p1, hw[i2], lw[i2]);
-                        }
+                for (int i = 0; i < 32; i += 2) {
+                    const float p0 = fast_exp2(fmaf(v[i], scale_log2, neg)), p1 = fast_exp2(fmaf(v[i + 1], scale_log2, neg));
+                    sum0 += p0;
+                    sum1 += p1;
+                    if constexpr (Q8) {               // the values' scales ride on the probabilities
+                        const float2 f = *reinterpret_cast<const float2 *>(&sc_v[j & 3][kq + i]);
+                        split2x2_trunc(p0 * f.x, p1 * f.y, phi[c * 16 + i / 2], plo[c * 16 + i / 2]);
+                    } else {
+                        split2x2_trunc(p0, p1, phi[c * 16 + i / 2], plo[c * 16 + i / 2]);
                     }
-                    const int piece16 = ((((kq & 63) >> 3) + i8) ^ (row & 7)) << 4;   // 16-byte piece index xor row bits (128-byte swizzle)
-                    *reinterpret_cast<uint4 *>(prow_hi + piece16) = hi;
-                    *reinterpret_cast<uint4 *>(prow_lo + piece16) = lo;
                 }
             }
+            // P as the A operand in tensor memory: lane = query row, a column holds two consecutive keys (bf16)
+            static_assert(KP == 64, "32 packed columns per thread and piece");
+            tmem_st32(trow + tmem_p_off + part * (KP / 2), reinterpret_cast<const float *>(phi));
+            tmem_st32(trow + tmem_p_off + AT_BN / 2 + part * (KP / 2), reinterpret_cast<const float *>(plo));
+            tmem_st_wait();
             l_run += sum0 + sum1;
             tc_fence_before();
             warp_arrive(&s_empty[j & 1]);    // this part of S_j has been read twice
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P: generic-proxy writes before the tensor core's reads
-            warp_arrive(&p_full[j % AT_PB]);
+            warp_arrive(&p_full[j % AT_PB]);   // (after tc_fence_before above: the stores to tensor memory are ordered before the multiply)
         }
         float o[DP];
         if (ok) ok = warp_wait(&o_full[0], (nb - 1) & 1);   // the last block's multiply
