@@ -130,6 +130,23 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const float *v) {
         "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
 }
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float *v) {
+    const uint32_t *r = reinterpret_cast<const uint32_t *>(v);
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]),
+        "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+template <int N> __device__ __forceinline__ void tmem_st(uint32_t taddr, const float *v) {
+    static_assert(N == 16 || N % 32 == 0, "16 columns or a multiple of 32");
+    if constexpr (N == 16) {
+        tmem_st16(taddr, v);
+    } else {
+#pragma unroll
+        for (int c = 0; c < N / 32; ++c) tmem_st32(taddr + c * 32, v + c * 32);
+    }
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
@@ -674,10 +691,14 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
 // tiles have barriers of their own.
 //   tensor memory: S0 [0, 128), S1 [128, 256), O [256, 256 + D), P hi [384, 448), P lo [448, 512)
 //   shared memory: Q 2 x D/64 x 16 KB | 2 stages x (K D/64 x 16 KB, V D/64 x 16 KB)   (compressed cache: one stage + landing areas)
-constexpr int AT_BM = 128, AT_BN = 128, AT_PARTS = 2;
+#ifndef AT_PARTS_VALUE
+#define AT_PARTS_VALUE 2
+#endif
+constexpr int AT_BM = 128, AT_BN = 128, AT_PARTS = AT_PARTS_VALUE;
 constexpr int AT_KVS_MAX = 2;  // stages of the K / V tiles: two on the bf16 cache, one on the compressed cache (whose tiles are
                                // expanded in place)
-constexpr int AT_PB = 1;       // buffers of the probabilities (in tensor memory)
+constexpr int AT_PB = 2;       // the probabilities of a block live in tensor memory as two halves of 64 keys with barriers of their own:
+                               // P V of the first half runs while the softmax still works on the second
 constexpr int AT_CW = 4;       // compressed cache: warps that expand the codes (AT_BN / AT_CW rows of a tile each)
 constexpr int AT_THREADS = 96 + 128 * AT_PARTS;   // producer, two issuers, softmax warps
 
@@ -835,21 +856,24 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
         constexpr uint32_t idesc_o = umma_idesc_bf16(AT_BM, D) | (1u << 16);   // B (= V) is MN-major
         bool ok = true;
         for (int j = 0; j < nb && ok; ++j) {
-            const int st = j % AT_KVS, pb = j % AT_PB;
+            const int st = j % AT_KVS;
             ok = mbar_wait(&v_full[st], (j / AT_KVS) & 1, &abort_flag, wait_limit);
-            if (ok) ok = mbar_wait(&p_full[pb], (j / AT_PB) & 1, &abort_flag, wait_limit);
-            if (!ok) break;
-            tc_fence_after();
             const uint32_t v = smem_u32(skv + st * (C::K_BYTES + C::V_BYTES) + C::K_BYTES);
 #pragma unroll
-            for (int piece = 0; piece < 2; ++piece) {
+            for (int h = 0; h < 2 && ok; ++h) {          // the two 64-key halves of the block
+                ok = mbar_wait(&p_full[h], j & 1, &abort_flag, wait_limit);
+                if (!ok) break;
+                tc_fence_after();
 #pragma unroll
-                for (int kk = 0; kk < AT_BN / 16; ++kk)   // 16 keys: 8 columns of P in tensor memory, 2048 bytes of the V tile
-                    umma_bf16_ts(tmem + 2 * AT_BN, tmem + tmem_p_off + piece * (AT_BN / 2) + kk * 8,
-                                 umma_desc_sw128_mn(v + kk * 2048, AT_BN * 128), idesc_o, (j | piece | kk) != 0);   // O accumulates over the blocks
+                for (int piece = 0; piece < 2; ++piece)
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)       // 16 keys: 8 columns of P in tensor memory, 2048 bytes of the V tile
+                        umma_bf16_ts(tmem + 2 * AT_BN, tmem + tmem_p_off + h * 64 + piece * 32 + kk * 8,
+                                     umma_desc_sw128_mn(v + (h * 4 + kk) * 2048, AT_BN * 128), idesc_o, (j | h | piece | kk) != 0);   // O accumulates
+                umma_commit(&p_empty[h]);
             }
+            if (!ok) break;
             umma_commit(&o_full[0]);
-            umma_commit(&p_empty[pb]);
             umma_commit(&v_empty[st]);
         }
         if (!ok) {
@@ -934,7 +958,6 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
         const int quarter = warp & 3, part = (warp - 3) >> 2, row = quarter * 32 + lane;
         const uint32_t trow = tmem + (static_cast<uint32_t>(quarter * 32) << 16);
         const int qi = slot0 + t0 + row;     // cache slot of this query: it sees the keys 0 .. qi
-        constexpr int KP = AT_BN / AT_PARTS; // keys of a block per thread
         constexpr int DP = D / AT_PARTS;     // this thread's columns of the output row
         // The output row accumulates in tensor memory over the blocks (P V with accumulation).  The exponentials are taken
         // against a reference maximum m_ref that moves only when the row's maximum has grown by more than 2^8 in the
@@ -960,17 +983,15 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
             ok = warp_wait(&s_full[j & 1], (j >> 1) & 1);
             if (!ok) break;
             tc_fence_after();
-            const int key0 = j * AT_BN + part * KP;
             const bool diagonal = j * AT_BN + AT_BN - 1 > slot0 + t0;   // some query of the tile does not see the whole block
-            const uint32_t srow = trow + (j & 1) * AT_BN + part * KP;
-            float mx = -INFINITY;
-#pragma unroll
-            for (int c = 0; c < KP / 32; ++c) {   // pass 1: the maximum over this thread's keys the query sees
-                float v[32];
-                tmem_ld32(srow + c * 32, v);
+            // this thread's keys: 32 of the block's first half (chunk 0), 32 of its second half (chunk 1)
+            static_assert(AT_PARTS == 2 && AT_BN == 128, "two threads per row, 2 x 32 keys each");
+            const uint32_t srow = trow + (j & 1) * AT_BN + part * 32;
+            auto load_chunk = [&](int c, float *v) {    // scores of chunk c, scaled (Q8) and masked
+                tmem_ld32(srow + c * 64, v);
                 tmem_ld_wait();
                 if constexpr (Q8) {                   // scores of codes -> scores: the keys' scales (16-byte shared-memory reads)
-                    const float4 *sk = reinterpret_cast<const float4 *>(&sc_k[j & 3][part * KP + c * 32]);
+                    const float4 *sk = reinterpret_cast<const float4 *>(&sc_k[j & 3][c * 64 + part * 32]);
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
                         const float4 f = sk[i];
@@ -980,8 +1001,14 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
                 if (diagonal) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
-                        if (key0 + c * 32 + i > qi) v[i] = -INFINITY;
+                        if (j * AT_BN + c * 64 + part * 32 + i > qi) v[i] = -INFINITY;
                 }
+            };
+            float mx = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {         // pass 1: the maximum over this thread's keys the query sees
+                float v[32];
+                load_chunk(c, v);
 #pragma unroll
                 for (int i = 0; i < 32; i += 4) mx = fmaxf(mx, fmaxf(fmaxf(v[i], v[i + 1]), fmaxf(v[i + 2], v[i + 3])));
             }
@@ -1002,68 +1029,54 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
                 tc_fence_after();
                 const float f = fast_exp2((m_ref - mx) * scale_log2);
                 l_run *= f;
-#pragma unroll
-                for (int c = 0; c < DP / 32; ++c) {
-                    static_assert(DP % 32 == 0, "32 columns per tensor-memory access");
-                    float v[32];
-                    tmem_ld32(trow + 2 * AT_BN + part * DP + c * 32, v);
+                {
+                    float v[DP];
+                    tmem_ld<DP>(trow + 2 * AT_BN + part * DP, v);
                     tmem_ld_wait();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] *= f;
-                    tmem_st32(trow + 2 * AT_BN + part * DP + c * 32, v);
+                    for (int i = 0; i < DP; ++i) v[i] *= f;
+                    tmem_st<DP>(trow + 2 * AT_BN + part * DP, v);
                 }
                 tmem_st_wait();
                 tc_fence_before();
                 m_ref = mx;
             }
             const float neg = -m_ref * scale_log2;
-            if (j >= AT_PB) {                // the P buffer's previous block has been multiplied
-                ok = warp_wait(&p_empty[j % AT_PB], ((j / AT_PB) - 1) & 1);
-                if (!ok) break;
-            }
             float sum0 = 0.f, sum1 = 0.f;
-            uint32_t phi[KP / 2], plo[KP / 2];    // this thread's probabilities, two keys per word
 #pragma unroll
-            for (int c = 0; c < KP / 32; ++c) {   // pass 2: probabilities as two bf16 pieces
+            for (int c = 0; c < 2; ++c) {         // pass 2: probabilities as two bf16 pieces, half by half
                 float v[32];
-                tmem_ld32(srow + c * 32, v);
-                tmem_ld_wait();
-                if constexpr (Q8) {                   // scores of codes -> scores: the keys' scales (16-byte shared-memory reads)
-                    const float4 *sk = reinterpret_cast<const float4 *>(&sc_k[j & 3][part * KP + c * 32]);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const float4 f = sk[i];
-                        v[4 * i] *= f.x; v[4 * i + 1] *= f.y; v[4 * i + 2] *= f.z; v[4 * i + 3] *= f.w;
-                    }
+                load_chunk(c, v);
+                if (c == 1) {
+                    tc_fence_before();
+                    warp_arrive(&s_empty[j & 1]);     // S_j has been read for the last time
                 }
-                if (diagonal) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (key0 + c * 32 + i > qi) v[i] = -INFINITY;
-                }
-                const int kq = part * KP + c * 32;            // first key of this chunk within the block
+                uint32_t phi[16], plo[16];        // two keys per word
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
                     const float p0 = fast_exp2(fmaf(v[i], scale_log2, neg)), p1 = fast_exp2(fmaf(v[i + 1], scale_log2, neg));
                     sum0 += p0;
                     sum1 += p1;
                     if constexpr (Q8) {               // the values' scales ride on the probabilities
-                        const float2 f = *reinterpret_cast<const float2 *>(&sc_v[j & 3][kq + i]);
-                        split2x2_trunc(p0 * f.x, p1 * f.y, phi[c * 16 + i / 2], plo[c * 16 + i / 2]);
+                        const float2 f = *reinterpret_cast<const float2 *>(&sc_v[j & 3][c * 64 + part * 32 + i]);
+                        split2x2_trunc(p0 * f.x, p1 * f.y, phi[i / 2], plo[i / 2]);
                     } else {
-                        split2x2_trunc(p0, p1, phi[c * 16 + i / 2], plo[c * 16 + i / 2]);
+                        split2x2_trunc(p0, p1, phi[i / 2], plo[i / 2]);
                     }
                 }
+                if (j >= 1) {                     // this half's multiply of the block before is done
+                    ok = warp_wait(&p_empty[c], (j - 1) & 1);
+                    if (!ok) break;
+                }
+                // P as the A operand in tensor memory: lane = query row, a column holds two consecutive keys (bf16)
+                tmem_st16(trow + tmem_p_off + c * 64 + part * 16, reinterpret_cast<const float *>(phi));
+                tmem_st16(trow + tmem_p_off + c * 64 + 32 + part * 16, reinterpret_cast<const float *>(plo));
+                tmem_st_wait();
+                tc_fence_before();
+                warp_arrive(&p_full[c]);
             }
-            // P as the A operand in tensor memory: lane = query row, a column holds two consecutive keys (bf16)
-            static_assert(KP == 64, "32 packed columns per thread and piece");
-            tmem_st32(trow + tmem_p_off + part * (KP / 2), reinterpret_cast<const float *>(phi));
-            tmem_st32(trow + tmem_p_off + AT_BN / 2 + part * (KP / 2), reinterpret_cast<const float *>(plo));
-            tmem_st_wait();
+            if (!ok) break;
             l_run += sum0 + sum1;
-            tc_fence_before();
-            warp_arrive(&s_empty[j & 1]);    // this part of S_j has been read twice
-            warp_arrive(&p_full[j % AT_PB]);   // (after tc_fence_before above: the stores to tensor memory are ordered before the multiply)
         }
         float o[DP];
         if (ok) ok = warp_wait(&o_full[0], (nb - 1) & 1);   // the last block's multiply
