@@ -64,6 +64,10 @@ __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, i
                  : "memory");
 }
 
+// Descriptor fetch ahead of the first copy that uses the map (the map is a kernel parameter).
+__device__ __forceinline__ void prefetch_map(const CUtensorMap *map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -448,6 +452,7 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
     };
 
     if (threadIdx.x == 0) {
+        prefetch_map(&map_a_hi); prefetch_map(&map_a_lo); prefetch_map(&map_b);
         for (int s = 0; s < C::STAGES; ++s) { mbar_init(&full_bar[s], 1 + g.extra_arrivals); mbar_init(&empty_bar[s], 1); }
         for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], 4); }
         mbar_init(&drain_bar, 1);
@@ -755,6 +760,7 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
     const int nb = last_key / AT_BN + 1;
 
     if (threadIdx.x == 0) {
+        prefetch_map(&map_q_hi); prefetch_map(&map_q_lo); prefetch_map(&map_k); prefetch_map(&map_v);
         mbar_init(&q_full, 1);
         for (int i = 0; i < AT_KVS; ++i) { mbar_init(&k_full[i], Q8 ? AT_CW : 1); mbar_init(&k_empty[i], 1); mbar_init(&v_full[i], Q8 ? AT_CW : 1); mbar_init(&v_empty[i], 1); }
         mbar_init(&kraw_full, 1); mbar_init(&kraw_empty, AT_CW); mbar_init(&vraw_full, 1);
