@@ -160,7 +160,11 @@ edgefm_status edgefm_decode_step(edgefm_ctx *ctx, int32_t token_id, int32_t posi
  * first mismatch.  n_accepted = 1 + accepted proposals (>= 1: tokens[0] itself always enters the cache); the cache length
  * grows by n_accepted (the rows of rejected tokens stay behind it and are overwritten later); the next token is
  * g_{n_accepted - 1}.  The result is what n_accepted plain decode steps would have produced.
- *   tokens          : HOST int32 [m], read during the call.  m = 1 .. block_tokens of the context (m = 1 is a decode step).
+ *   tokens          : HOST int32 [m], read during the call.  m = 1 .. block_tokens of the context (m = 1 is a decode step)
+ *                     through the step kernel.  Longer blocks, up to 8 tokens (on any context, also block_tokens = 0), take the
+ *                     DENSE path: the prefill kernels of edgefm_prefill for the m tokens, one pass over the output matrix for
+ *                     all m rows, the same acceptance rule on the device.  That path needs tokens[0] and position given (no
+ *                     -1) and an exact host-side cache length: after a verified block, edgefm_sync_length comes first.
  *   logits_out      : DEVICE fp32 [m][vocab] (row t: the logits after token t; rows >= n_accepted belong to rejected
  *                     tokens) or NULL.  With a vocabulary subset of n ids (edgefm_set_vocab_subset) the rows are n long,
  *                     [m][n], and the greedy tokens -- hence the acceptance -- are taken over the subset.

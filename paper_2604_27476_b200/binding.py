@@ -365,7 +365,8 @@ class DecodeContext:
         with torch.cuda.device(self.device):
             self.handle = edgefm_create(shape, device_weight_ptrs, max_context, kv_format, block_tokens=block_tokens)
         self.block_tokens = max(1, block_tokens)
-        self.block_logits = torch.empty((self.block_tokens, cfg.vocab), dtype=torch.float32, device=self.device)
+        # rows for the longest block a call may carry: block_tokens through the step kernel, up to 8 through the dense path
+        self.block_logits = torch.empty((max(self.block_tokens, 8), cfg.vocab), dtype=torch.float32, device=self.device)
         self.logits = self.block_logits[0]
         self.next_token = torch.zeros(1, dtype=torch.int32, device=self.device)
         self.n_accepted = torch.zeros(1, dtype=torch.int32, device=self.device)

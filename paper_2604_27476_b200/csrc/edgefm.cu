@@ -381,6 +381,7 @@ struct edgefm_ctx {
     // host mirrors
     int cur_len = 0;
     bool have_token = false;
+    bool len_exact = true;       // false between a verified block (the device decides how far the cache grows) and edgefm_sync_length
     bool req_valid = false;
     StepRequest last_req{};
     std::string err;
@@ -432,6 +433,9 @@ void free_all(edgefm_ctx *c) {
     for (void *b : bufs) if (b) cudaFree(b);
     if (c->pf.chunk) prefill_free(&c->pf);
 }
+
+edgefm_status ensure_prefill_buffers(edgefm_ctx *ctx);
+PrefillModel prefill_model(edgefm_ctx *ctx);
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -691,6 +695,7 @@ edgefm_status copy_kv_in(edgefm_ctx *ctx, const void *k, const void *v, int32_t 
             ctx->max_context, stride_layer, stride_head, stride_pos, ctx->state, slot0);
         CUDA_TRY(ctx, cudaGetLastError());
         ctx->cur_len = slot0 + n_positions;
+        ctx->len_exact = true;
         ctx->err.clear();
         return EDGEFM_OK;
     }
@@ -705,6 +710,7 @@ edgefm_status copy_kv_in(edgefm_ctx *ctx, const void *k, const void *v, int32_t 
         sh.n_kv_heads, n_positions, sh.head_dim, ctx->max_context, stride_layer, stride_head, stride_pos, vec_ok, ctx->state, slot0);
     CUDA_TRY(ctx, cudaGetLastError());
     ctx->cur_len = slot0 + n_positions;
+    ctx->len_exact = true;
     ctx->err.clear();
     return EDGEFM_OK;
 }
@@ -753,8 +759,13 @@ edgefm_status edgefm_verify_block(edgefm_ctx *ctx, const int32_t *tokens, int32_
                                   int32_t *n_accepted_out, int32_t *next_token_out) {
     if (!ctx) return EDGEFM_ERR_INVALID_ARG;
     if (!tokens) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "null tokens");
-    if (m < 1 || m > ctx->block_tokens)
-        return fail(ctx, EDGEFM_ERR_INVALID_ARG, "m = %d: this context verifies blocks of 1 .. %d tokens (edgefm_options::block_tokens)", m, ctx->block_tokens);
+    const bool dense = m > ctx->block_tokens;   // longer blocks go through the dense path (the prefill kernels)
+    if (m < 1 || m > std::max(ctx->block_tokens, PF_VERIFY_MAX))
+        return fail(ctx, EDGEFM_ERR_INVALID_ARG, "m = %d: blocks of 1 .. %d tokens", m, std::max(ctx->block_tokens, PF_VERIFY_MAX));
+    if (dense && (tokens[0] < 0 || position < 0))
+        return fail(ctx, EDGEFM_ERR_INVALID_ARG, "a block of %d tokens on this context (block_tokens = %d) takes the dense path, which needs tokens[0] and position given", m, ctx->block_tokens);
+    if (dense && !ctx->len_exact)
+        return fail(ctx, EDGEFM_ERR_INVALID_ARG, "the dense path places the block behind the host's cache length: call edgefm_sync_length after the previous block first");
     if (tokens[0] < -1 || tokens[0] >= ctx->shape.vocab) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "tokens[0] = %d out of range", tokens[0]);
     for (int t = 1; t < m; ++t)
         if (tokens[t] < 0 || tokens[t] >= ctx->shape.vocab) return fail(ctx, EDGEFM_ERR_INVALID_ARG, "tokens[%d] = %d out of range", t, tokens[t]);
@@ -764,6 +775,29 @@ edgefm_status edgefm_verify_block(edgefm_ctx *ctx, const int32_t *tokens, int32_
         return fail(ctx, EDGEFM_ERR_CONTEXT_FULL, "%d tokens do not fit behind %d of %d cache slots", m, ctx->cur_len, ctx->max_context);
     DeviceGuard guard(ctx->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (dense) {
+        if (const edgefm_status st = ensure_prefill_buffers(ctx)) return st;
+        PrefillModel pm = prefill_model(ctx);
+        int launches = 0;
+        const int slot0 = ctx->cur_len;
+        if (const char *e = prefill_run(pm, &ctx->pf, tokens, m, slot0, position, true, s, &launches)) {
+            cudaGetLastError();
+            return fail(ctx, EDGEFM_ERR_CUDA, "%s", e);
+        }
+        const bool sub = ctx->vocab_subset > 0;
+        if (const char *e = prefill_verify_head(pm, &ctx->pf, m, ctx->final_norm, sub ? static_cast<const void *>(ctx->sub_lm) : ctx->lm_head,
+                                                sub ? ctx->vocab_ids : nullptr, sub ? ctx->vocab_subset : ctx->shape.vocab, logits_out, n_accepted_out,
+                                                next_token_out, slot0, position, s)) {
+            cudaGetLastError();
+            return fail(ctx, EDGEFM_ERR_CUDA, "%s", e);
+        }
+        ctx->prefill_launches = launches + 1;
+        ctx->cur_len += m;     // an upper bound until edgefm_sync_length
+        ctx->len_exact = false;
+        ctx->have_token = true;
+        ctx->err.clear();
+        return EDGEFM_OK;
+    }
     StepRequest r{tokens[0], position, logits_out, next_token_out};
     r.m = m;
     for (int t = 1; t < m && t <= 3; ++t) r.draft[t - 1] = tokens[t];
@@ -775,6 +809,7 @@ edgefm_status edgefm_verify_block(edgefm_ctx *ctx, const int32_t *tokens, int32_
     }
     CUDA_TRY(ctx, cudaGraphLaunch(ctx->exec, s));
     ctx->cur_len += m;     // an upper bound until edgefm_sync_length: the device decides how many tokens are accepted
+    if (m > 1) ctx->len_exact = false;
     ctx->have_token = true;
     ctx->err.clear();
     return EDGEFM_OK;
@@ -808,6 +843,35 @@ edgefm_status edgefm_prefill_tokens(edgefm_ctx *ctx, const int32_t *tokens, int3
     return EDGEFM_OK;
 }
 
+}  // extern "C" (helpers of the dense path follow)
+
+namespace {
+
+// Work buffers of the dense path (prefill, long verified blocks): allocated at the first use, kept.
+edgefm_status ensure_prefill_buffers(edgefm_ctx *ctx) {
+    if (ctx->pf.chunk == 0) {
+        const int chunk = std::min(PF_CHUNK_MAX, ctx->max_context);
+        if (prefill_alloc(&ctx->pf, ctx->shape, chunk, ctx->kv_format == EDGEFM_KV_INT8) != cudaSuccess) {
+            cudaGetLastError();
+            prefill_free(&ctx->pf);
+            return fail(ctx, EDGEFM_ERR_OUT_OF_MEMORY, "work buffers of the dense path (%zu bytes)", prefill_buffer_bytes(ctx->shape, chunk));
+        }
+    }
+    ctx->pf.wait_limit = ctx->pf_wait_limit;
+    ctx->pf.extra_arrivals = ctx->pf_extra_arrivals;
+    return EDGEFM_OK;
+}
+
+PrefillModel prefill_model(edgefm_ctx *ctx) {
+    return PrefillModel{ctx->shape, ctx->layers.data(), ctx->embed, ctx->k_cache, ctx->v_cache,
+                        ctx->kv_format == EDGEFM_KV_INT8 ? ctx->k_scale : nullptr, ctx->kv_format == EDGEFM_KV_INT8 ? ctx->v_scale : nullptr,
+                        ctx->max_context, ctx->state, ctx->num_sms};
+}
+
+}  // namespace
+
+extern "C" {
+
 edgefm_status edgefm_prefill(edgefm_ctx *ctx, const int32_t *tokens, int32_t n, int32_t position, void *stream, float *logits_out,
                              int32_t *next_token_out) {
     if (!ctx) return EDGEFM_ERR_INVALID_ARG;
@@ -822,21 +886,13 @@ edgefm_status edgefm_prefill(edgefm_ctx *ctx, const int32_t *tokens, int32_t n, 
     // Prompts of at least 8 tokens go through the dense path whole, and the output layer runs for the last row alone (one pass
     // over its matrix); shorter ones leave their last token to a decode step (which streams all weights again: 1.1 ms at the
     // 1.5B shape, against one more layer for a handful of rows).
+    if (!ctx->len_exact)
+        return fail(ctx, EDGEFM_ERR_INVALID_ARG, "the prompt is placed behind the host's cache length: call edgefm_sync_length after a verified block first");
     const bool dense_all = n >= 8;
     const int n_dense = dense_all ? n : n - 1;
-    if (n_dense > 0 && ctx->pf.chunk == 0) {
-        const int chunk = std::min(PF_CHUNK_MAX, ctx->max_context);
-        if (prefill_alloc(&ctx->pf, ctx->shape, chunk, ctx->kv_format == EDGEFM_KV_INT8) != cudaSuccess) {
-            cudaGetLastError();
-            prefill_free(&ctx->pf);
-            return fail(ctx, EDGEFM_ERR_OUT_OF_MEMORY, "work buffers of edgefm_prefill (%zu bytes)", prefill_buffer_bytes(ctx->shape, chunk));
-        }
-    }
-    ctx->pf.wait_limit = ctx->pf_wait_limit;
-    ctx->pf.extra_arrivals = ctx->pf_extra_arrivals;
-    PrefillModel pm{ctx->shape, ctx->layers.data(), ctx->embed, ctx->k_cache, ctx->v_cache,
-                    ctx->kv_format == EDGEFM_KV_INT8 ? ctx->k_scale : nullptr, ctx->kv_format == EDGEFM_KV_INT8 ? ctx->v_scale : nullptr,
-                    ctx->max_context, ctx->state, ctx->num_sms};
+    if (n_dense > 0)
+        if (const edgefm_status st = ensure_prefill_buffers(ctx)) return st;
+    PrefillModel pm = prefill_model(ctx);
     ctx->prefill_launches = 0;
     for (int i = 0; i < n_dense;) {
         const int c = std::min(ctx->pf.chunk, n_dense - i);
@@ -874,6 +930,7 @@ edgefm_status edgefm_sync_length(edgefm_ctx *ctx, void *stream, int32_t *cur_len
     StepState st{};
     CUDA_TRY(ctx, cudaMemcpy(&st, ctx->state, sizeof st, cudaMemcpyDeviceToHost));
     ctx->cur_len = st.cur_len;
+    ctx->len_exact = true;
     *cur_len_host = st.cur_len;
     return EDGEFM_OK;
 }

@@ -393,6 +393,109 @@ __global__ void __launch_bounds__(256) prefill_head_kernel(const float *x, const
     }
 }
 
+// Output layer for the m <= PF_VERIFY_MAX rows of a verified block (Sec. 3.11): final RMSNorm of every row, logits of all rows
+// in ONE pass over the output matrix, the rows' greedy tokens, and the acceptance rule on the device: proposal t + 1 is
+// accepted if tokens[t + 1] equals the greedy token after token t, verification stops at the first mismatch; the cache
+// length becomes slot0 + n_accepted (the rows behind it are overwritten later), the next token is the greedy token after the
+// last accepted one.  256 threads; dynamic shared memory m * H floats.
+__global__ void __launch_bounds__(256) prefill_verify_head_kernel(const float *x, const uint16_t *wnorm, const uint16_t *lm, const int *ids, int rows,
+                                                                  int H, float eps, float *logits_out, int m, const int *tokens,
+                                                                  float *part_val, int *part_idx, unsigned *ticket, StepState *st, int slot0,
+                                                                  int pos, int *n_accepted_out, int *next_token_out) {
+    pdl_trigger();
+    pdl_wait();
+    extern __shared__ __align__(16) float pf_xs[];
+    __shared__ float red[8], bvs[8][PF_VERIFY_MAX];
+    __shared__ int bis[8][PF_VERIFY_MAX], is_last;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    for (int t = 0; t < m; ++t) {
+        const float *xr = x + static_cast<size_t>(t) * H;
+        float ss = 0.f;
+        for (int j = tid; j < H; j += 256) ss = fmaf(xr[j], xr[j], ss);
+        ss = warp_sum(ss);
+        if (lane == 0) red[warp] = ss;
+        __syncthreads();
+        ss = ((red[0] + red[1]) + (red[2] + red[3])) + ((red[4] + red[5]) + (red[6] + red[7]));
+        const float r = rsqrtf(ss / static_cast<float>(H) + eps);
+        for (int j = tid; j < H; j += 256) pf_xs[t * H + j] = xr[j] * r * bf16_bits_to_f32(wnorm[j]);
+        __syncthreads();
+    }
+    float bv[PF_VERIFY_MAX];
+    int bi[PF_VERIFY_MAX];
+#pragma unroll
+    for (int t = 0; t < PF_VERIFY_MAX; ++t) { bv[t] = -INFINITY; bi[t] = 0x7fffffff; }
+    for (int row = blockIdx.x * 8 + warp; row < rows; row += gridDim.x * 8) {
+        const uint16_t *w = lm + static_cast<size_t>(row) * H;
+        float a[PF_VERIFY_MAX];
+#pragma unroll
+        for (int t = 0; t < PF_VERIFY_MAX; ++t) a[t] = 0.f;
+        for (int j = lane * 8; j < H; j += 256) {
+            const uint4 u = *reinterpret_cast<const uint4 *>(w + j);
+#pragma unroll
+            for (int t = 0; t < PF_VERIFY_MAX; ++t)
+                if (t < m) {
+                    const float4 x0 = *reinterpret_cast<const float4 *>(pf_xs + t * H + j), x1 = *reinterpret_cast<const float4 *>(pf_xs + t * H + j + 4);
+                    a[t] = dot8(u, x0, x1, a[t]);
+                }
+        }
+#pragma unroll
+        for (int t = 0; t < PF_VERIFY_MAX; ++t)
+            if (t < m) {
+                a[t] = warp_sum(a[t]);
+                if (lane == 0) {
+                    if (logits_out) logits_out[static_cast<size_t>(t) * rows + row] = a[t];
+                    if (arg_better(a[t], row, bv[t], bi[t])) { bv[t] = a[t]; bi[t] = row; }
+                }
+            }
+    }
+    if (lane == 0)
+        for (int t = 0; t < PF_VERIFY_MAX; ++t) { bvs[warp][t] = bv[t]; bis[warp][t] = bi[t]; }
+    __syncthreads();
+    if (tid < m) {                   // thread t: row t's candidate of this CTA
+        float v = bvs[0][tid];
+        int ix = bis[0][tid];
+        for (int w = 1; w < 8; ++w)
+            if (arg_better(bvs[w][tid], bis[w][tid], v, ix)) { v = bvs[w][tid]; ix = bis[w][tid]; }
+        part_val[blockIdx.x * PF_VERIFY_MAX + tid] = v;
+        part_idx[blockIdx.x * PF_VERIFY_MAX + tid] = ix;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) is_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (is_last && warp == 0) {      // the last CTA to finish merges the candidates and applies the acceptance rule
+        __threadfence();
+        int greedy = 0;
+        if (lane < m) {
+            float v = -INFINITY;
+            int ix = 0x7fffffff;
+            for (int i = 0; i < static_cast<int>(gridDim.x); ++i) {
+                const float pv = __ldcg(part_val + i * PF_VERIFY_MAX + lane);
+                const int pi = __ldcg(part_idx + i * PF_VERIFY_MAX + lane);
+                if (arg_better(pv, pi, v, ix)) { v = pv; ix = pi; }
+            }
+            if (ix == 0x7fffffff) ix = 0;
+            greedy = ids ? ids[ix] : ix;   // pruned vocabulary: row index -> token id
+        }
+        int n_acc = 1, next = __shfl_sync(0xffffffffu, greedy, 0);
+        for (int t = 1; t < m; ++t) {
+            const int g_prev = __shfl_sync(0xffffffffu, greedy, t - 1), g_t = __shfl_sync(0xffffffffu, greedy, t);
+            if (n_acc == t && tokens[t] == g_prev) { n_acc = t + 1; next = g_t; }
+        }
+        if (lane == 0) {
+            if (next_token_out) *next_token_out = next;
+            if (n_accepted_out) *n_accepted_out = n_acc;
+            st->token = tokens[0];
+            st->position = pos;
+            st->next_token = next;
+            st->next_position = pos + n_acc;
+            st->cur_len = slot0 + n_acc;
+            st->n_accepted = n_acc;
+            *ticket = 0u;
+        }
+    }
+}
+
 // ---- the contraction -------------------------------------------------------------------------------------------------------
 enum { EPI_QKV = 0, EPI_RESID = 1, EPI_SWIGLU = 2 };
 
@@ -1367,13 +1470,28 @@ const char *prefill_head(const PrefillModel &m, PrefillBuffers *b, int row, cons
     int grid = 2 * m.num_sms;
     if (grid > PF_HEAD_GRID_MAX) grid = PF_HEAD_GRID_MAX;
     if (grid * 8 > rows) grid = (rows + 7) / 8;
-    if (H * 4 > 48 * 1024 &&
+    if (H * 4 > 40 * 1024 &&
         cudaFuncSetAttribute(prefill_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, H * 4) != cudaSuccess)
         return "cudaFuncSetAttribute failed";
     launch_pdl(prefill_head_kernel, dim3(grid), dim3(256), static_cast<size_t>(H) * 4, s, b->resid + static_cast<size_t>(row) * H, static_cast<const uint16_t *>(final_norm),
                                                                      static_cast<const uint16_t *>(lm), ids, rows, H, m.shape.rms_eps, logits_out,
                                                                      next_token_out, b->head_val, b->head_idx, b->head_ticket, m.state, token, pos);
     return cudaGetLastError() == cudaSuccess ? nullptr : "prefill output layer launch failed";
+}
+
+const char *prefill_verify_head(const PrefillModel &m, PrefillBuffers *b, int n, const void *final_norm, const void *lm, const int *ids, int rows,
+                                float *logits_out, int *n_accepted_out, int *next_token_out, int slot0, int pos, cudaStream_t s) {
+    const int H = m.shape.hidden;
+    int grid = 2 * m.num_sms;
+    if (grid > PF_HEAD_GRID_MAX / PF_VERIFY_MAX) grid = PF_HEAD_GRID_MAX / PF_VERIFY_MAX;
+    if (grid * 8 > rows) grid = (rows + 7) / 8;
+    const size_t smem = static_cast<size_t>(n) * H * 4;
+    if (smem > 40 * 1024 && cudaFuncSetAttribute(prefill_verify_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)   // (the 48 KB default includes the static part)
+        return "cudaFuncSetAttribute failed";
+    launch_pdl(prefill_verify_head_kernel, dim3(grid), dim3(256), smem, s, b->resid, static_cast<const uint16_t *>(final_norm),
+               static_cast<const uint16_t *>(lm), ids, rows, H, m.shape.rms_eps, logits_out, n, b->tokens, b->head_val, b->head_idx, b->head_ticket,
+               m.state, slot0, pos, n_accepted_out, next_token_out);
+    return cudaGetLastError() == cudaSuccess ? nullptr : "block verification output layer launch failed";
 }
 
 }  // namespace edgefm

@@ -9,7 +9,8 @@
 
 namespace edgefm {
 
-constexpr int PF_HEAD_GRID_MAX = 1024;   // CTAs of the output-layer kernel
+constexpr int PF_HEAD_GRID_MAX = 1024;   // CTAs of the output-layer kernel (candidate slots: PF_HEAD_GRID_MAX)
+constexpr int PF_VERIFY_MAX = 8;         // tokens of a block verified through the dense path
 constexpr int PF_CHUNK_MAX = 2048;   // tokens per pass over the layers (longer prompts take several passes)
 
 // Work buffers of one pass, owned by the context, allocated at the first prefill call.
@@ -67,5 +68,10 @@ const char *prefill_run(const PrefillModel &m, PrefillBuffers *b, const int32_t 
 // `token` at `pos` would.  logits_out / next_token_out: device pointers or nullptr.
 const char *prefill_head(const PrefillModel &m, PrefillBuffers *b, int row, const void *final_norm, const void *lm, const int *ids, int rows,
                          float *logits_out, int *next_token_out, int token, int pos, cudaStream_t stream);
+
+// Block verification through the dense path (Sec. 3.11): after prefill_run(..., n tokens, whole_last_layer = true), the logits of
+// all n rows ([n][rows], or nullptr), the greedy acceptance on the device and the state update (cache length slot0 + accepted).
+const char *prefill_verify_head(const PrefillModel &m, PrefillBuffers *b, int n, const void *final_norm, const void *lm, const int *ids, int rows,
+                                float *logits_out, int *n_accepted_out, int *next_token_out, int slot0, int pos, cudaStream_t stream);
 
 }  // namespace edgefm

@@ -95,11 +95,14 @@ def test_block_calls_are_validated():
     block = Pair(cfg, cache_len=3, max_context=4, block_tokens=2)
     try:
         with pytest.raises(EdgefmError) as ei:
-            plain.ctx.verify_block([1, 2], 0)                      # context not built for blocks
+            plain.ctx.verify_block([-1, 2], -1)                    # a plain context verifies through the dense path: tokens must be given
         assert ei.value.status == Status.ERR_INVALID_ARG
         with pytest.raises(EdgefmError) as ei:
-            block.ctx.verify_block([1, 2, 3], 3)                   # more tokens than the build carries
+            block.ctx.verify_block(list(range(1, 10)), 3)          # more than eight tokens
         assert ei.value.status == Status.ERR_INVALID_ARG
+        with pytest.raises(EdgefmError) as ei:
+            block.ctx.verify_block([1, 2, 3], 3)                   # the dense path for three tokens, one free slot
+        assert ei.value.status == Status.ERR_CONTEXT_FULL
         with pytest.raises(EdgefmError) as ei:
             block.ctx.verify_block([1, cfg.vocab], 3)
         assert ei.value.status == Status.ERR_INVALID_ARG
@@ -204,5 +207,58 @@ def test_blocks_of_four_match_the_oracle_verification(name):
         if n > T0:
             assert_appended_rows_close(kg[:, :, T0:n], ko[:, :, T0:n])
             assert_appended_rows_close(vg[:, :, T0:n], vo[:, :, T0:n])
+    finally:
+        pair.close()
+
+
+@pytest.mark.parametrize("name,kv_format", [("tiny", None), ("tiny", "int8"), ("qwen2.5-1.5b", None)])
+def test_blocks_of_up_to_eight_tokens_through_the_dense_path(name, kv_format):
+    """Blocks longer than the context's block_tokens (here a plain context) are verified by the prefill kernels: all m tokens
+    through the layers together, one pass over the output matrix for all rows, the acceptance rule on the device."""
+    import torch
+    cfg = CONFIGS[name] if name != "tiny" else CONFIGS[name].with_(qkv_bias=True)
+    T0 = 40
+    pair = Pair(cfg, cache_len=T0, max_context=T0 + 64, kv_format=kv_format)
+    try:
+        rng = np.random.default_rng(17)
+        tok, pos = int(rng.integers(0, cfg.vocab)), T0 + 5
+        for rnd, (m, wrong_at) in enumerate([(8, None), (8, 3), (5, 1), (7, 6), (6, None)]):
+            # proposals: the oracle's own greedy continuation (found on a scratch pass, then rolled back), one of them spoiled
+            start = pair.oracle.cur_len
+            block, t = [tok], tok
+            for i in range(m - 1):
+                _, t = pair.oracle.step(t, pos + i)
+                block.append(t)
+            pair.oracle.truncate(start)
+            if wrong_at is not None:
+                block[wrong_at] = (block[wrong_at] + 1) % cfg.vocab
+            ref_rows, ref_acc, ref_next = pair.oracle.verify_block(block, pos)
+            pair.ctx.verify_block(block, pos)
+            torch.cuda.synchronize()
+            pair.ctx.sync_status()
+            got = pair.ctx.block_logits.cpu().numpy()
+            margins_ok = all(top2_margin(ref_rows[i]) > TOKEN_MARGIN for i in range(ref_acc))
+            for i in range(ref_acc):
+                assert_logits_close(got[i], ref_rows[i], f"round {rnd} row {i}")
+            length = pair.ctx.sync_length()            # the host learns how far the cache grew (needed before the next long block)
+            if not margins_ok:
+                break                                  # a near-tie among the accepted rows: the two sides may decide differently
+            assert int(pair.ctx.n_accepted.item()) == ref_acc, (rnd, int(pair.ctx.n_accepted.item()), ref_acc)
+            assert length == pair.oracle.cur_len == start + ref_acc
+            assert int(pair.ctx.next_token.item()) == ref_next
+            tok, pos = ref_next, pos + ref_acc
+        # without edgefm_sync_length the next long block is refused; -1 tokens are refused on this path
+        from paper_2604_27476_b200 import EdgefmError, Status
+        pair.ctx.verify_block([1, 2, 3, 4, 5], pos)
+        with pytest.raises(EdgefmError) as ei:
+            pair.ctx.verify_block([1, 2, 3, 4, 5], pos)
+        assert ei.value.status == Status.ERR_INVALID_ARG
+        pair.ctx.sync_length()
+        with pytest.raises(EdgefmError) as ei:
+            pair.ctx.verify_block([-1, 2, 3, 4, 5], pos)
+        assert ei.value.status == Status.ERR_INVALID_ARG
+        with pytest.raises(EdgefmError) as ei:
+            pair.ctx.verify_block(list(range(1, 10)), pos)
+        assert ei.value.status == Status.ERR_INVALID_ARG
     finally:
         pair.close()
