@@ -200,7 +200,9 @@ def run_block(args, cfg):
     k, v = make_kv(cfg)
     ptrs, keep = upload_weights(weights, dev)
     B = args.block_tokens
-    ctx = DecodeContext(cfg, ptrs, cfg.cache_len + B * steps + B + 2, dev, block_tokens=B)
+    dense = B > 4          # blocks of more than four tokens take the dense path (prefill kernels) on a plain context; every call then
+                           # reads the accepted length and the next token back to the host (part of the timed loop)
+    ctx = DecodeContext(cfg, ptrs, cfg.cache_len + B * steps + B + 2, dev, block_tokens=0 if dense else B)
     kd = torch.from_numpy(k.view(np.int16)).to(dev)
     vd = torch.from_numpy(v.view(np.int16)).to(dev)
     tok0, pos0 = first_token(cfg), cfg.first_position
@@ -223,7 +225,11 @@ def run_block(args, cfg):
             props = [seq[idx + t] for t in range(1, B)]
             if spoil:
                 props[-1] = (props[-1] + 1) % cfg.vocab
-            ctx.verify_block([tok0 if c == 0 else -1] + props, pos0 if c == 0 else -1, want_logits=False)
+            if dense:
+                ctx.verify_block([seq[idx]] + props, pos0 + idx, want_logits=False)
+                ctx.sync_length()
+            else:
+                ctx.verify_block([tok0 if c == 0 else -1] + props, pos0 if c == 0 else -1, want_logits=False)
             idx += B - 1 if spoil else B
         return idx
 
@@ -340,7 +346,7 @@ def main():
                     help="prune the output layer to this many evenly spaced token ids (0 = full vocabulary, the headline workload)")
     ap.add_argument("--kv-format", default="bf16", choices=["bf16", "int8"],
                     help="cache format: int8 = the compressed cache (edgefm_create_with_options); not the headline configuration")
-    ap.add_argument("--block-tokens", type=int, default=1, choices=[1, 2, 4],
+    ap.add_argument("--block-tokens", type=int, default=1, choices=[1, 2, 4, 8],
                     help="2 / 4: generate through edgefm_verify_block, that many tokens per call (not the headline configuration)")
     ap.add_argument("--reject-every", type=int, default=0, help="with --block-tokens 2: spoil every n-th proposal (0 = none)")
     ap.add_argument("--prefill", type=int, default=0,
