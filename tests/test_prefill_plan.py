@@ -1,5 +1,5 @@
 """Host logic of edgefm_prefill's contraction planner (tile shape and K split), checked without a GPU: invariants the kernels
-rely on and the choices the design doc quotes for the benchmark shapes."""
+rely on and its choices for the benchmark shapes."""
 import itertools
 
 from edgefm_synth import CONFIGS
