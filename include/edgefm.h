@@ -192,7 +192,7 @@ edgefm_status edgefm_prefill_tokens(edgefm_ctx *ctx, const int32_t *tokens, int3
 
 /*
  * edgefm_prefill -- the prefill phase (Eq. 3 of the paper, KV <- Prefill(x_1:T; theta_p); with a prefix already in the cache,
- * Eq. 5: KV = Concat(KV_p, KV_u)) as dense contractions.  The prompt's tokens pass through the layers TOGETHER (at most 2048
+ * Eq. 5: KV = Concat(KV_p, KV_u)) as dense contractions.  The prompt's tokens pass through the layers TOGETHER (at most 4096
  * per pass): every projection is one [tokens x K] x [K x N] product on the tensor cores (tcgen05, fp32 accumulation in
  * tensor memory; every activation enters as two bf16 pieces, hi + lo = 16 mantissa bits, the weights are bf16 exactly; fp32
  * residual stream), attention is causal over the cache rows 0 .. cur_len + t; the K and V rows go to cache slots cur_len ..

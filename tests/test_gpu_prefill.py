@@ -81,7 +81,7 @@ def test_prompt_as_dense_contractions_tiny(T0, n):
 
 
 def test_prompt_longer_than_one_pass():
-    run_case(CONFIGS["tiny"], 5, 2100, 77, follow=False)
+    run_case(CONFIGS["tiny"], 5, 4200, 77, follow=False)
 
 
 def test_prompt_on_the_1_5b_shape():
@@ -168,7 +168,7 @@ def test_prefill_then_block_verification_and_pruned_vocabulary():
         pair.close()
 
 
-@pytest.mark.parametrize("name,T0,n", [("tiny", 0, 9), ("tiny", 20, 300), ("tiny", 5, 2100), ("qwen2.5-1.5b", 32, 200)])
+@pytest.mark.parametrize("name,T0,n", [("tiny", 0, 9), ("tiny", 20, 300), ("tiny", 5, 4200), ("qwen2.5-1.5b", 32, 200)])
 def test_prompt_into_the_compressed_cache(name, T0, n):
     """The same prefill on a context with the 8-bit cache (Sec. 3.9): the new rows are compressed from their fp32 values (k
     after RoPE, v) exactly as the decode step compresses its own row, and attention reads codes x scales for every row, the
