@@ -203,7 +203,7 @@ edgefm_status edgefm_prefill_tokens(edgefm_ctx *ctx, const int32_t *tokens, int3
  *   tokens     : HOST int32 [n], n >= 1, read during the call.
  *   position   : rotary position of tokens[0] (>= 0); token i has position + i.
  *   logits_out : DEVICE fp32 [vocab] (or the subset's length) or NULL;  next_token_out : DEVICE int32 [1] or NULL.
- * The work buffers (about (24 H + 8 n_q d + 4 F) bytes per token of a pass) are allocated at the first call and kept.
+ * The work buffers (about (40 H + 8 n_q d + 4 F) bytes per token of a pass) are allocated at the first call and kept.
  * After edgefm_verify_block call edgefm_sync_length first: the rows are placed behind the host's cache length (the call is
  * refused with INVALID_ARG while that length is only an upper bound).
  * On a context with the compressed cache (EDGEFM_KV_INT8) the new K and V rows are compressed from their fp32 values (k after

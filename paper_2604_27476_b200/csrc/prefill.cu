@@ -525,7 +525,8 @@ struct GemmArgs {
 };
 
 constexpr int PF_BM = 128, PF_BK = 64;
-constexpr int PF_SPLIT_MAX = 4;               // K splits of a contraction that adds to the residual stream
+constexpr int PF_SPLIT_MAX = 8;               // K splits of a contraction that adds to the residual stream: up to 4, up to 8 when the
+                                             // tokens fit one row tile (short prompts, verified blocks: the grids are smallest there)
 
 // Tile shapes.  PF_NARROW: 128 output columns, 4 stages of 48 KB.  PF_WIDE: 256 output columns, 3 stages of 64 KB: per k-block
 // 64 KB of operands feed twice the multiplies of a narrow tile's 48 KB, which matters because operand delivery from L2, not
@@ -1359,7 +1360,7 @@ void prefill_plan_contraction(int epilogue, int M, int N, int K, int num_sms, in
     int best_shape = 0, best_split = 1;
     double best = 1e30;
     for (int shape = 0; shape < 2; ++shape)
-        for (int sp = 1; sp <= (epilogue == EPI_RESID ? PF_SPLIT_MAX : 1); ++sp) {
+        for (int sp = 1; sp <= (epilogue == EPI_RESID ? (m_tiles == 1 ? PF_SPLIT_MAX : 4) : 1); ++sp) {
             if (sp > 1 && (kb / sp < 12 || tiles[shape] > num_sms)) break;   // split only grids that leave SMs idle in their one round
             const int units = tiles[shape] * sp;
             const double t = ((units + num_sms - 1) / num_sms) * cost[shape] / sp * (sp > 1 ? 1.05 : 1.0);

@@ -21,7 +21,7 @@ constexpr int PF_CHUNK_MAX = PF_CHUNK_MAX_VALUE;   // tokens per pass over the l
 struct PrefillBuffers {
     int chunk = 0;               // rows the buffers hold
     float *resid = nullptr;      // residual stream fp32 [chunk][H]
-    float *part = nullptr;       // K-split partial sums of the O / down contraction, fp32 [4][chunk][H]
+    float *part = nullptr;       // K-split partial sums of the O / down contraction, fp32 [8][chunk][H]
     // activations as two bf16 planes each (hi = bf16(x), lo = bf16(x - hi)):
     uint16_t *xn = nullptr;      // normalised activations [2][chunk][H]
     uint16_t *q = nullptr;       // rotated queries [2][chunk][nq d]
