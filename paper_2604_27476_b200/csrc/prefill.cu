@@ -824,6 +824,7 @@ constexpr int AT_KVS_MAX = 2;  // stages of the K / V tiles: two on the bf16 cac
                                // expanded in place)
 constexpr int AT_PB = 2;       // the probabilities of a block live in tensor memory as two halves of 64 keys with barriers of their own:
                                // P V of the first half runs while the softmax still works on the second
+constexpr int AT_SPLIT_MAX = 8; // CTAs that share the key blocks of a lone query tile
 constexpr int AT_CW = 4;       // compressed cache: warps that expand the codes (AT_BN / AT_CW rows of a tile each)
 constexpr int AT_THREADS = 96 + 128 * AT_PARTS;   // producer, two issuers, softmax warps
 
@@ -856,7 +857,7 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
                                                                    const __grid_constant__ CUtensorMap map_v, uint16_t *out, size_t plane,
                                                                    int T, int slot0, int nq, int group, int max_context,
                                                                    float scale_log2, uint32_t wait_limit, int *error, const float *k_scale,
-                                                                   const float *v_scale) {
+                                                                   const float *v_scale, float *part_o, float *part_ml) {
     // Q8: the cache holds 8-bit codes and a scale per row (k_scale, v_scale: this layer's [nkv][max_context]); map_k / map_v then
     // describe byte matrices; two more warps expand the codes to bf16 (exactly) into the operand layout, the softmax multiplies
     // the scores by the keys' scales and folds the values' scales into the probabilities.
@@ -878,7 +879,11 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
     const int t0 = (gridDim.y - 1 - blockIdx.y) * AT_BM;
     const int h = blockIdx.x, hk = h / group;
     const int last_key = slot0 + min(t0 + AT_BM - 1, T - 1);
-    const int nb = last_key / AT_BN + 1;
+    // gridDim.z > 1 (few queries behind a long cache): the key blocks are shared out among gridDim.z CTAs; each leaves its
+    // unnormalised row of O, its reference maximum and its row sum in part_o / part_ml, prefill_attention_merge_kernel adds them
+    const int nb_total = last_key / AT_BN + 1, splits = gridDim.z;
+    const int j0 = static_cast<int>(blockIdx.z) * nb_total / splits;          // first key block of this CTA
+    const int nb = (static_cast<int>(blockIdx.z) + 1) * nb_total / splits - j0;   // its key blocks (indices below are local)
 
     if (threadIdx.x == 0) {
         prefetch_map(&map_q_hi); prefetch_map(&map_q_lo); prefetch_map(&map_k); prefetch_map(&map_v);
@@ -918,10 +923,10 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
             if (j >= AT_KVS && !mbar_wait(Q8 ? &kraw_empty : &k_empty[st], ((j / AT_KVS) - 1) & 1, &abort_flag, wait_limit)) return false;
             if constexpr (Q8) {
                 mbar_expect_tx(&kraw_full, C::RAW_BYTES);
-                tma_load_2d(sraw, &map_k, 0, hk * max_context + j * AT_BN, &kraw_full);
+                tma_load_2d(sraw, &map_k, 0, hk * max_context + (j0 + j) * AT_BN, &kraw_full);
             } else {
                 mbar_expect_tx(&k_full[st], C::K_BYTES);
-                for (int kb = 0; kb < C::KBLK; ++kb) tma_load_2d(k + kb * AT_BN * 128, &map_k, kb * 64, hk * max_context + j * AT_BN, &k_full[st]);
+                for (int kb = 0; kb < C::KBLK; ++kb) tma_load_2d(k + kb * AT_BN * 128, &map_k, kb * 64, hk * max_context + (j0 + j) * AT_BN, &k_full[st]);
             }
             nk = j + 1;
             return true;
@@ -932,10 +937,10 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
             if (j >= AT_KVS && !mbar_wait(&v_empty[st], ((j / AT_KVS) - 1) & 1, &abort_flag, wait_limit)) return false;
             if constexpr (Q8) {
                 mbar_expect_tx(&vraw_full, C::RAW_BYTES);
-                tma_load_2d(D == 128 ? v : sraw + C::RAW_BYTES, &map_v, 0, hk * max_context + j * AT_BN, &vraw_full);
+                tma_load_2d(D == 128 ? v : sraw + C::RAW_BYTES, &map_v, 0, hk * max_context + (j0 + j) * AT_BN, &vraw_full);
             } else {
                 mbar_expect_tx(&v_full[st], C::V_BYTES);
-                for (int kb = 0; kb < C::KBLK; ++kb) tma_load_2d(v + kb * AT_BN * 128, &map_v, kb * 64, hk * max_context + j * AT_BN, &v_full[st]);
+                for (int kb = 0; kb < C::KBLK; ++kb) tma_load_2d(v + kb * AT_BN * 128, &map_v, kb * 64, hk * max_context + (j0 + j) * AT_BN, &v_full[st]);
             }
             nv = j + 1;
             return true;
@@ -1061,7 +1066,7 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
             __syncwarp();
             if (lane == 0) mbar_arrive(&kraw_empty);       // the next K tile may land
             for (int i = lane; i < ROWS; i += 32) {        // the scales of this block's keys (both kinds: they are in memory already)
-                const int key = min(j * AT_BN + cw * ROWS + i, last_key);
+                const int key = min((j0 + j) * AT_BN + cw * ROWS + i, last_key);
                 sc_k[j & 3][cw * ROWS + i] = k_scale[static_cast<size_t>(hk) * max_context + key];
                 sc_v[j & 3][cw * ROWS + i] = v_scale[static_cast<size_t>(hk) * max_context + key];
             }
@@ -1111,7 +1116,7 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
             ok = warp_wait(&s_full[j & 1], (j >> 1) & 1);
             if (!ok) break;
             tc_fence_after();
-            const bool diagonal = j * AT_BN + AT_BN - 1 > slot0 + t0;   // some query of the tile does not see the whole block
+            const bool diagonal = (j0 + j) * AT_BN + AT_BN - 1 > slot0 + t0;   // some query of the tile does not see the whole block
             // this thread's keys: 32 of the block's first half (chunk 0), 32 of its second half (chunk 1)
             static_assert(AT_PARTS == 2 && AT_BN == 128, "two threads per row, 2 x 32 keys each");
             const uint32_t srow = trow + (j & 1) * AT_BN + part * 32;
@@ -1129,7 +1134,7 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
                 if (diagonal) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
-                        if (j * AT_BN + c * 64 + part * 32 + i > qi) v[i] = -INFINITY;
+                        if ((j0 + j) * AT_BN + c * 64 + part * 32 + i > qi) v[i] = -INFINITY;
                 }
             };
             float mx = -INFINITY;
@@ -1147,7 +1152,7 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
 #pragma unroll
             for (int q = 0; q < AT_PARTS; ++q) mx = fmaxf(mx, xchg[j & 1][q][row]);
             if (j == 0) {
-                m_ref = mx;                  // nothing accumulated yet
+                m_ref = fmaxf(mx, -1e30f);   // nothing accumulated yet (a row that sees none of this CTA's keys keeps a finite reference)
             } else if (__any_sync(0xffffffffu, (mx - m_ref) * scale_log2 > 8.f)) {
                 // some row of this warp has outgrown its reference (both warps of a quarter see the same rows and maxima, so they
                 // decide alike): every row moves its reference to its maximum and rescales its sum and its part of O, once the
@@ -1221,7 +1226,13 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
             for (int q = 0; q < AT_PARTS; ++q) l_run += xchg[nb & 1][q][row];
         }
         const int t = t0 + row;
-        if (ok && t < T) {
+        if (ok && t < T && splits > 1) {     // partial result of this CTA's key blocks
+            const size_t slot = (static_cast<size_t>(blockIdx.z) * AT_BM + row) * nq + h;
+            float *dst = part_o + slot * D + part * DP;
+#pragma unroll
+            for (int i = 0; i < DP; i += 4) *reinterpret_cast<float4 *>(dst + i) = make_float4(o[i], o[i + 1], o[i + 2], o[i + 3]);
+            if (part == 0) { part_ml[slot * 2] = m_ref; part_ml[slot * 2 + 1] = l_run; }
+        } else if (ok && t < T) {
             const float inv = 1.f / l_run;
             uint16_t *dst = out + static_cast<size_t>(t) * nq * D + static_cast<size_t>(h) * D + part * DP;
 #pragma unroll
@@ -1241,6 +1252,34 @@ __global__ void __launch_bounds__(AT_THREADS + (Q8 ? 32 * AT_CW : 0)) prefill_at
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(AttnCfg<D>::TMEM_COLS) : "memory");
     }
     if (threadIdx.x == 0 && abort_flag) atomicExch(error, 1);
+}
+
+// Adds the partial results of a query tile whose key blocks were shared out among `splits` CTAs: for row t and head h,
+// M = max m_s, O = sum O_s 2^((m_s - M) c), L = sum l_s 2^((m_s - M) c), out = O / L as two bf16 planes.  grid (T, nq), D / 4 threads.
+template <int D>
+__global__ void __launch_bounds__(D / 4) prefill_attention_merge_kernel(const float *part_o, const float *part_ml, int splits, uint16_t *out,
+                                                                        size_t plane, int nq, float scale_log2) {
+    pdl_trigger();
+    pdl_wait();
+    const int t = blockIdx.x, h = blockIdx.y, i = threadIdx.x * 4;
+    float mmax = -INFINITY;
+    for (int s = 0; s < splits; ++s) mmax = fmaxf(mmax, part_ml[((static_cast<size_t>(s) * AT_BM + t) * nq + h) * 2]);
+    float l = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s = 0; s < splits; ++s) {
+        const size_t slot = (static_cast<size_t>(s) * AT_BM + t) * nq + h;
+        const float w = fast_exp2((part_ml[slot * 2] - mmax) * scale_log2);
+        const float4 o = *reinterpret_cast<const float4 *>(part_o + slot * D + i);
+        l = fmaf(part_ml[slot * 2 + 1], w, l);
+        acc.x = fmaf(o.x, w, acc.x); acc.y = fmaf(o.y, w, acc.y); acc.z = fmaf(o.z, w, acc.z); acc.w = fmaf(o.w, w, acc.w);
+    }
+    const float inv = 1.f / l;
+    uint2 hi, lo;
+    split2x2(acc.x * inv, acc.y * inv, hi.x, lo.x);
+    split2x2(acc.z * inv, acc.w * inv, hi.y, lo.y);
+    uint16_t *dst = out + static_cast<size_t>(t) * nq * D + static_cast<size_t>(h) * D + i;
+    *reinterpret_cast<uint2 *>(dst) = hi;
+    *reinterpret_cast<uint2 *>(dst + plane) = lo;
 }
 
 // Launch with the programmatic-stream-serialization attribute (see pdl_trigger / pdl_wait) for passes of up to 1024 tokens:
@@ -1321,10 +1360,13 @@ bool encode_bytes_map(CUtensorMap *m, const void *base, long long rows, int row_
 }
 
 // kc / vc: this layer's cache, bf16 rows or (k_scale != nullptr) rows of 8-bit codes with their scales.
+// A single query tile behind a long cache (a short suffix behind a prefix, a verified block) would run on n_q CTAs only: its key
+// blocks are then shared out among up to AT_SPLIT_MAX CTAs per head and the partial results merged (part_o / part_ml: room for
+// AT_SPLIT_MAX x 128 rows).
 template <int D>
 const char *launch_attention_tc(const uint16_t *q, const void *kc, const void *vc, const float *k_scale, const float *v_scale, uint16_t *out,
                                 size_t plane, int T, int slot0, int nq, int nkv, int max_context, uint32_t wait_limit, int *error,
-                                cudaStream_t s) {
+                                float *part_o, float *part_ml, int num_sms, cudaStream_t s) {
     CUtensorMap mqh, mql, mk, mv;
     const long long kv_rows = static_cast<long long>(nkv) * max_context;
     const bool q8 = k_scale != nullptr;
@@ -1333,18 +1375,30 @@ const char *launch_attention_tc(const uint16_t *q, const void *kc, const void *v
            : (!encode_operand_map(&mk, kc, kv_rows, D, AT_BN) || !encode_operand_map(&mv, vc, kv_rows, D, AT_BN)))
         return "cuTensorMapEncodeTiled failed";
     const float scale_log2 = static_cast<float>(1.4426950408889634 / sqrt(static_cast<double>(D)));
-    const dim3 grid(nq, (T + AT_BM - 1) / AT_BM);
+    int splits = 1;
+    if (T <= AT_BM) {
+        const int blocks = (slot0 + T - 1) / AT_BN + 1;
+        splits = num_sms / nq;                       // CTAs per head that still fit the SMs once
+        if (splits > AT_SPLIT_MAX) splits = AT_SPLIT_MAX;
+        if (splits > blocks / 2) splits = blocks / 2;   // at least two key blocks per CTA
+        if (splits < 1) splits = 1;
+    }
+    const dim3 grid(nq, (T + AT_BM - 1) / AT_BM, splits);
     if (q8) {
         if (cudaFuncSetAttribute(prefill_attention_tc_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<D>::SMEM_Q8) != cudaSuccess)
             return "cudaFuncSetAttribute failed";
-        launch_pdl(prefill_attention_tc_kernel<D, true>, dim3(grid), dim3(AT_THREADS + 32 * AT_CW), AttnCfg<D>::SMEM_Q8, s, 
-            mqh, mql, mk, mv, out, plane, T, slot0, nq, nq / nkv, max_context, scale_log2, wait_limit, error, k_scale, v_scale);
+        launch_pdl(prefill_attention_tc_kernel<D, true>, grid, dim3(AT_THREADS + 32 * AT_CW), AttnCfg<D>::SMEM_Q8, s, mqh, mql, mk, mv, out, plane, T,
+                   slot0, nq, nq / nkv, max_context, scale_log2, wait_limit, error, k_scale, v_scale, part_o, part_ml);
     } else {
         if (cudaFuncSetAttribute(prefill_attention_tc_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnCfg<D>::SMEM) != cudaSuccess)
             return "cudaFuncSetAttribute failed";
-        launch_pdl(prefill_attention_tc_kernel<D, false>, dim3(grid), dim3(AT_THREADS), AttnCfg<D>::SMEM, s, 
-            mqh, mql, mk, mv, out, plane, T, slot0, nq, nq / nkv, max_context, scale_log2, wait_limit, error, nullptr, nullptr);
+        launch_pdl(prefill_attention_tc_kernel<D, false>, grid, dim3(AT_THREADS), AttnCfg<D>::SMEM, s, mqh, mql, mk, mv, out, plane, T, slot0, nq,
+                   nq / nkv, max_context, scale_log2, wait_limit, error, static_cast<const float *>(nullptr), static_cast<const float *>(nullptr), part_o,
+                   part_ml);
     }
+    if (splits > 1)
+        launch_pdl(prefill_attention_merge_kernel<D>, dim3(T, nq), dim3(D / 4), 0, s, static_cast<const float *>(part_o),
+                   static_cast<const float *>(part_ml), splits, out, plane, nq, scale_log2);
     return cudaGetLastError() == cudaSuccess ? nullptr : "prefill attention launch failed";
 }
 
@@ -1388,6 +1442,8 @@ cudaError_t prefill_alloc(PrefillBuffers *b, const edgefm_shape &sh, int chunk, 
     if (kv8 && (e = cudaMalloc(&b->kv_stage, 2 * c * sh.n_kv_heads * sh.head_dim * sizeof(float))) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->tokens, c * 4)) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->error, 4)) != cudaSuccess) return e;
+    if ((e = cudaMalloc(&b->att_o, static_cast<size_t>(AT_SPLIT_MAX) * AT_BM * qd * 4)) != cudaSuccess) return e;
+    if ((e = cudaMalloc(&b->att_ml, static_cast<size_t>(AT_SPLIT_MAX) * AT_BM * sh.n_q_heads * 2 * 4)) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->head_val, PF_HEAD_GRID_MAX * 4)) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->head_idx, PF_HEAD_GRID_MAX * 4)) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->head_ticket, 4)) != cudaSuccess) return e;
@@ -1399,7 +1455,7 @@ cudaError_t prefill_alloc(PrefillBuffers *b, const edgefm_shape &sh, int chunk, 
 
 void prefill_free(PrefillBuffers *b) {
     cudaFree(b->resid); cudaFree(b->xn); cudaFree(b->part); cudaFree(b->kv_stage); cudaFree(b->q); cudaFree(b->attn); cudaFree(b->act); cudaFree(b->rope);
-    cudaFree(b->tokens); cudaFree(b->error); cudaFree(b->head_val); cudaFree(b->head_idx); cudaFree(b->head_ticket);
+    cudaFree(b->tokens); cudaFree(b->error); cudaFree(b->att_o); cudaFree(b->att_ml); cudaFree(b->head_val); cudaFree(b->head_idx); cudaFree(b->head_ticket);
     *b = PrefillBuffers{};
 }
 
@@ -1444,8 +1500,8 @@ const char *prefill_run(const PrefillModel &m, PrefillBuffers *b, const int32_t 
         if (l == sh.n_layers - 1 && !whole_last_layer) break;   // the rest of the last layer feeds nothing that is kept
         const void *ka = kv8 ? static_cast<const void *>(kc8) : kc, *va = kv8 ? static_cast<const void *>(vc8) : vc;
         const float *ksc = kv8 ? m.k_scale + layer_rows : nullptr, *vsc = kv8 ? m.v_scale + layer_rows : nullptr;
-        const char *e = d == 64 ? launch_attention_tc<64>(b->q, ka, va, ksc, vsc, b->attn, q_plane, n, slot0, nq, nkv, m.max_context, b->wait_limit, b->error, s)
-                                : launch_attention_tc<128>(b->q, ka, va, ksc, vsc, b->attn, q_plane, n, slot0, nq, nkv, m.max_context, b->wait_limit, b->error, s);
+        const char *e = d == 64 ? launch_attention_tc<64>(b->q, ka, va, ksc, vsc, b->attn, q_plane, n, slot0, nq, nkv, m.max_context, b->wait_limit, b->error, b->att_o, b->att_ml, m.num_sms, s)
+                                : launch_attention_tc<128>(b->q, ka, va, ksc, vsc, b->attn, q_plane, n, slot0, nq, nkv, m.max_context, b->wait_limit, b->error, b->att_o, b->att_ml, m.num_sms, s);
         if (e) return e;
         g.N = H; g.K = qd; g.resid = b->resid; g.part = b->part; g.part_plane = x_plane;
         if ((e = launch_gemm<EPI_RESID>(b->attn, q_plane, w.wo, H, g, m.num_sms, s))) return e;

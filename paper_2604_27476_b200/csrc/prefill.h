@@ -31,6 +31,8 @@ struct PrefillBuffers {
     float2 *rope = nullptr;      // (cos, sin) of the chunk's positions, [chunk][d/2]
     int *tokens = nullptr;       // device copy of the chunk's token ids
     int *error = nullptr;        // device word: non-zero when a bounded wait of a GEMM ran out
+    float *att_o = nullptr;      // attention of a lone query tile shared out among CTAs: partial rows fp32 [8][128][nq d]
+    float *att_ml = nullptr;     // ... and their (reference maximum, row sum) [8][128][nq][2]
     float *head_val = nullptr;   // output layer: the CTAs' greedy candidates
     int *head_idx = nullptr;
     unsigned *head_ticket = nullptr;

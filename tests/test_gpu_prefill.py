@@ -94,6 +94,13 @@ def test_prompt_behind_a_long_prefix():
     run_case(CONFIGS["tiny"].with_(qkv_bias=True), 8200, 150, 9)
 
 
+@pytest.mark.parametrize("name,T0,n", [("tiny", 8200, 60), ("tiny", 1000, 128), ("qwen2.5-1.5b", 2048, 40)])
+def test_short_suffix_behind_a_long_prefix(name, T0, n):
+    """Sec. 3.9, Eq. 5: a request's own short suffix behind a long fixed prefix.  One query tile then faces dozens of key
+    blocks: they are shared out among several CTAs per head and the partial results merged."""
+    run_case(CONFIGS[name] if name != "tiny" else CONFIGS[name].with_(qkv_bias=True), T0, n, 31)
+
+
 def test_prompt_on_the_0_5b_shape():
     """head_dim 64, 14 query heads on 2 kv heads, tied output layer; two query tiles and a ragged third."""
     run_case(CONFIGS["qwen2.5-0.5b"], 10, 300, 6, follow=False)
@@ -168,7 +175,7 @@ def test_prefill_then_block_verification_and_pruned_vocabulary():
         pair.close()
 
 
-@pytest.mark.parametrize("name,T0,n", [("tiny", 0, 9), ("tiny", 20, 300), ("tiny", 5, 4200), ("qwen2.5-1.5b", 32, 200)])
+@pytest.mark.parametrize("name,T0,n", [("tiny", 0, 9), ("tiny", 20, 300), ("tiny", 5, 4200), ("tiny", 3000, 50), ("qwen2.5-1.5b", 32, 200)])
 def test_prompt_into_the_compressed_cache(name, T0, n):
     """The same prefill on a context with the 8-bit cache (Sec. 3.9): the new rows are compressed from their fp32 values (k
     after RoPE, v) exactly as the decode step compresses its own row, and attention reads codes x scales for every row, the
