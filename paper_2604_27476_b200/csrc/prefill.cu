@@ -424,27 +424,35 @@ __global__ void __launch_bounds__(256) prefill_verify_head_kernel(const float *x
     int bi[PF_VERIFY_MAX];
 #pragma unroll
     for (int t = 0; t < PF_VERIFY_MAX; ++t) { bv[t] = -INFINITY; bi[t] = 0x7fffffff; }
-    for (int row = blockIdx.x * 8 + warp; row < rows; row += gridDim.x * 8) {
-        const uint16_t *w = lm + static_cast<size_t>(row) * H;
-        float a[PF_VERIFY_MAX];
+    const int stride = gridDim.x * 8;
+    for (int row = blockIdx.x * 8 + warp; row < rows; row += 2 * stride) {   // two weight rows per round share the reads of x
+        const int row2 = row + stride;
+        const uint16_t *w0 = lm + static_cast<size_t>(row) * H, *w1 = lm + static_cast<size_t>(row2 < rows ? row2 : row) * H;
+        float a[PF_VERIFY_MAX], c[PF_VERIFY_MAX];
 #pragma unroll
-        for (int t = 0; t < PF_VERIFY_MAX; ++t) a[t] = 0.f;
+        for (int t = 0; t < PF_VERIFY_MAX; ++t) a[t] = c[t] = 0.f;
         for (int j = lane * 8; j < H; j += 256) {
-            const uint4 u = *reinterpret_cast<const uint4 *>(w + j);
+            const uint4 u0 = *reinterpret_cast<const uint4 *>(w0 + j), u1 = *reinterpret_cast<const uint4 *>(w1 + j);
 #pragma unroll
             for (int t = 0; t < PF_VERIFY_MAX; ++t)
                 if (t < m) {
                     const float4 x0 = *reinterpret_cast<const float4 *>(pf_xs + t * H + j), x1 = *reinterpret_cast<const float4 *>(pf_xs + t * H + j + 4);
-                    a[t] = dot8(u, x0, x1, a[t]);
+                    a[t] = dot8(u0, x0, x1, a[t]);
+                    c[t] = dot8(u1, x0, x1, c[t]);
                 }
         }
 #pragma unroll
         for (int t = 0; t < PF_VERIFY_MAX; ++t)
             if (t < m) {
                 a[t] = warp_sum(a[t]);
+                c[t] = warp_sum(c[t]);
                 if (lane == 0) {
-                    if (logits_out) logits_out[static_cast<size_t>(t) * rows + row] = a[t];
+                    if (logits_out) {
+                        logits_out[static_cast<size_t>(t) * rows + row] = a[t];
+                        if (row2 < rows) logits_out[static_cast<size_t>(t) * rows + row2] = c[t];
+                    }
                     if (arg_better(a[t], row, bv[t], bi[t])) { bv[t] = a[t]; bi[t] = row; }
+                    if (row2 < rows && arg_better(c[t], row2, bv[t], bi[t])) { bv[t] = c[t]; bi[t] = row2; }
                 }
             }
     }
@@ -1444,8 +1452,8 @@ cudaError_t prefill_alloc(PrefillBuffers *b, const edgefm_shape &sh, int chunk, 
     if ((e = cudaMalloc(&b->error, 4)) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->att_o, static_cast<size_t>(AT_SPLIT_MAX) * AT_BM * qd * 4)) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->att_ml, static_cast<size_t>(AT_SPLIT_MAX) * AT_BM * sh.n_q_heads * 2 * 4)) != cudaSuccess) return e;
-    if ((e = cudaMalloc(&b->head_val, PF_HEAD_GRID_MAX * 4)) != cudaSuccess) return e;
-    if ((e = cudaMalloc(&b->head_idx, PF_HEAD_GRID_MAX * 4)) != cudaSuccess) return e;
+    if ((e = cudaMalloc(&b->head_val, PF_HEAD_GRID_MAX * PF_VERIFY_MAX * 4)) != cudaSuccess) return e;
+    if ((e = cudaMalloc(&b->head_idx, PF_HEAD_GRID_MAX * PF_VERIFY_MAX * 4)) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->head_ticket, 4)) != cudaSuccess) return e;
     if ((e = cudaMemset(b->head_ticket, 0, 4)) != cudaSuccess) return e;
     if ((e = cudaMemset(b->error, 0, 4)) != cudaSuccess) return e;
@@ -1539,8 +1547,8 @@ const char *prefill_head(const PrefillModel &m, PrefillBuffers *b, int row, cons
 const char *prefill_verify_head(const PrefillModel &m, PrefillBuffers *b, int n, const void *final_norm, const void *lm, const int *ids, int rows,
                                 float *logits_out, int *n_accepted_out, int *next_token_out, int slot0, int pos, cudaStream_t s) {
     const int H = m.shape.hidden;
-    int grid = 2 * m.num_sms;
-    if (grid > PF_HEAD_GRID_MAX / PF_VERIFY_MAX) grid = PF_HEAD_GRID_MAX / PF_VERIFY_MAX;
+    int grid = 4 * m.num_sms;   // (48 KB of rows at the 1.5B shape: four CTAs per SM)
+    if (grid > PF_HEAD_GRID_MAX) grid = PF_HEAD_GRID_MAX;
     if (grid * 8 > rows) grid = (rows + 7) / 8;
     const size_t smem = static_cast<size_t>(n) * H * 4;
     if (smem > 40 * 1024 && cudaFuncSetAttribute(prefill_verify_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)   // (the 48 KB default includes the static part)

@@ -9,7 +9,7 @@
 
 namespace edgefm {
 
-constexpr int PF_HEAD_GRID_MAX = 1024;   // CTAs of the output-layer kernel (candidate slots: PF_HEAD_GRID_MAX)
+constexpr int PF_HEAD_GRID_MAX = 1024;   // CTAs of the output-layer kernels (candidate slots: PF_HEAD_GRID_MAX x PF_VERIFY_MAX)
 constexpr int PF_VERIFY_MAX = 8;         // tokens of a block verified through the dense path
 #ifndef PF_CHUNK_MAX_VALUE
 #define PF_CHUNK_MAX_VALUE 4096
