@@ -393,73 +393,35 @@ __global__ void __launch_bounds__(256) prefill_head_kernel(const float *x, const
     }
 }
 
-// Output layer for the m <= PF_VERIFY_MAX rows of a verified block (Sec. 3.11): final RMSNorm of every row, logits of all rows
-// in ONE pass over the output matrix, the rows' greedy tokens, and the acceptance rule on the device: proposal t + 1 is
-// accepted if tokens[t + 1] equals the greedy token after token t, verification stops at the first mismatch; the cache
-// length becomes slot0 + n_accepted (the rows behind it are overwritten later), the next token is the greedy token after the
-// last accepted one.  256 threads; dynamic shared memory m * H floats.
-__global__ void __launch_bounds__(256) prefill_verify_head_kernel(const float *x, const uint16_t *wnorm, const uint16_t *lm, const int *ids, int rows,
-                                                                  int H, float eps, float *logits_out, int m, const int *tokens,
+// Greedy tokens of the m <= PF_VERIFY_MAX rows of a logits matrix [m][rows] and the acceptance rule of a verified block (Sec. 3.11)
+// on the device: proposal t + 1 is accepted if tokens[t + 1] equals the greedy token after token t, verification stops at the
+// first mismatch; the cache length becomes slot0 + n_accepted (the rows behind it are overwritten later), the next token is the
+// greedy token after the last accepted one.  The logits come from a contraction over the output matrix (EPI_LOGITS).
+__global__ void __launch_bounds__(256) prefill_verify_pick_kernel(const float *logits, const int *ids, int rows, int m, const int *tokens,
                                                                   float *part_val, int *part_idx, unsigned *ticket, StepState *st, int slot0,
                                                                   int pos, int *n_accepted_out, int *next_token_out) {
     pdl_trigger();
     pdl_wait();
-    extern __shared__ __align__(16) float pf_xs[];
-    __shared__ float red[8], bvs[8][PF_VERIFY_MAX];
+    __shared__ float bvs[8][PF_VERIFY_MAX];
     __shared__ int bis[8][PF_VERIFY_MAX], is_last;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     for (int t = 0; t < m; ++t) {
-        const float *xr = x + static_cast<size_t>(t) * H;
-        float ss = 0.f;
-        for (int j = tid; j < H; j += 256) ss = fmaf(xr[j], xr[j], ss);
-        ss = warp_sum(ss);
-        if (lane == 0) red[warp] = ss;
-        __syncthreads();
-        ss = ((red[0] + red[1]) + (red[2] + red[3])) + ((red[4] + red[5]) + (red[6] + red[7]));
-        const float r = rsqrtf(ss / static_cast<float>(H) + eps);
-        for (int j = tid; j < H; j += 256) pf_xs[t * H + j] = xr[j] * r * bf16_bits_to_f32(wnorm[j]);
-        __syncthreads();
-    }
-    float bv[PF_VERIFY_MAX];
-    int bi[PF_VERIFY_MAX];
-#pragma unroll
-    for (int t = 0; t < PF_VERIFY_MAX; ++t) { bv[t] = -INFINITY; bi[t] = 0x7fffffff; }
-    const int stride = gridDim.x * 8;
-    for (int row = blockIdx.x * 8 + warp; row < rows; row += 2 * stride) {   // two weight rows per round share the reads of x
-        const int row2 = row + stride;
-        const uint16_t *w0 = lm + static_cast<size_t>(row) * H, *w1 = lm + static_cast<size_t>(row2 < rows ? row2 : row) * H;
-        float a[PF_VERIFY_MAX], c[PF_VERIFY_MAX];
-#pragma unroll
-        for (int t = 0; t < PF_VERIFY_MAX; ++t) a[t] = c[t] = 0.f;
-        for (int j = lane * 8; j < H; j += 256) {
-            const uint4 u0 = *reinterpret_cast<const uint4 *>(w0 + j), u1 = *reinterpret_cast<const uint4 *>(w1 + j);
-#pragma unroll
-            for (int t = 0; t < PF_VERIFY_MAX; ++t)
-                if (t < m) {
-                    const float4 x0 = *reinterpret_cast<const float4 *>(pf_xs + t * H + j), x1 = *reinterpret_cast<const float4 *>(pf_xs + t * H + j + 4);
-                    a[t] = dot8(u0, x0, x1, a[t]);
-                    c[t] = dot8(u1, x0, x1, c[t]);
-                }
+        float bv = -INFINITY;
+        int bi = 0x7fffffff;
+        for (int r = blockIdx.x * 256 + tid; r < rows; r += gridDim.x * 256) {
+            const float v = logits[static_cast<size_t>(t) * rows + r];
+            if (arg_better(v, r, bv, bi)) { bv = v; bi = r; }
         }
 #pragma unroll
-        for (int t = 0; t < PF_VERIFY_MAX; ++t)
-            if (t < m) {
-                a[t] = warp_sum(a[t]);
-                c[t] = warp_sum(c[t]);
-                if (lane == 0) {
-                    if (logits_out) {
-                        logits_out[static_cast<size_t>(t) * rows + row] = a[t];
-                        if (row2 < rows) logits_out[static_cast<size_t>(t) * rows + row2] = c[t];
-                    }
-                    if (arg_better(a[t], row, bv[t], bi[t])) { bv[t] = a[t]; bi[t] = row; }
-                    if (row2 < rows && arg_better(c[t], row2, bv[t], bi[t])) { bv[t] = c[t]; bi[t] = row2; }
-                }
-            }
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (arg_better(ov, oi, bv, bi)) { bv = ov; bi = oi; }
+        }
+        if (lane == 0) { bvs[warp][t] = bv; bis[warp][t] = bi; }
     }
-    if (lane == 0)
-        for (int t = 0; t < PF_VERIFY_MAX; ++t) { bvs[warp][t] = bv[t]; bis[warp][t] = bi[t]; }
     __syncthreads();
-    if (tid < m) {                   // thread t: row t's candidate of this CTA
+    if (tid < m) {
         float v = bvs[0][tid];
         int ix = bis[0][tid];
         for (int w = 1; w < 8; ++w)
@@ -471,7 +433,7 @@ __global__ void __launch_bounds__(256) prefill_verify_head_kernel(const float *x
     __syncthreads();
     if (tid == 0) is_last = atomicAdd(ticket, 1u) == gridDim.x - 1;
     __syncthreads();
-    if (is_last && warp == 0) {      // the last CTA to finish merges the candidates and applies the acceptance rule
+    if (is_last && warp == 0) {
         __threadfence();
         int greedy = 0;
         if (lane < m) {
@@ -483,7 +445,7 @@ __global__ void __launch_bounds__(256) prefill_verify_head_kernel(const float *x
                 if (arg_better(pv, pi, v, ix)) { v = pv; ix = pi; }
             }
             if (ix == 0x7fffffff) ix = 0;
-            greedy = ids ? ids[ix] : ix;   // pruned vocabulary: row index -> token id
+            greedy = ids ? ids[ix] : ix;
         }
         int n_acc = 1, next = __shfl_sync(0xffffffffu, greedy, 0);
         for (int t = 1; t < m; ++t) {
@@ -505,7 +467,7 @@ __global__ void __launch_bounds__(256) prefill_verify_head_kernel(const float *x
 }
 
 // ---- the contraction -------------------------------------------------------------------------------------------------------
-enum { EPI_QKV = 0, EPI_RESID = 1, EPI_SWIGLU = 2 };
+enum { EPI_QKV = 0, EPI_RESID = 1, EPI_SWIGLU = 2, EPI_LOGITS = 3 };   // EPI_LOGITS: plain fp32 store to g.resid [M][N] (output layer)
 
 struct GemmArgs {
     int M, N, K;              // rows (tokens), output features (gate/up: F, each of gate and up), reduction length
@@ -683,6 +645,20 @@ __global__ void __launch_bounds__(192) prefill_gemm_kernel(const __grid_constant
                                 o.x += v[4 * i]; o.y += v[4 * i + 1]; o.z += v[4 * i + 2]; o.w += v[4 * i + 3];
                                 p[i] = o;
                             }
+                    }
+                }
+            } else if (EPI == EPI_LOGITS) {
+                for (int c = 0; c < N_STEP / 32; ++c) {
+                    const int n = n0 + c * 32;
+                    if (n >= g.N) break;
+                    float v[32];
+                    tmem_ld32(trow + c * 32, v);
+                    tmem_ld_wait();
+                    if (live) {                      // N need not be a multiple of 4 (a pruned vocabulary): scalar stores
+                        float *p = g.resid + static_cast<size_t>(row) * g.N + n;
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (n + i < g.N) p[i] = v[i];
                     }
                 }
             } else if (EPI == EPI_SWIGLU) {
@@ -1450,6 +1426,8 @@ cudaError_t prefill_alloc(PrefillBuffers *b, const edgefm_shape &sh, int chunk, 
     if (kv8 && (e = cudaMalloc(&b->kv_stage, 2 * c * sh.n_kv_heads * sh.head_dim * sizeof(float))) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->tokens, c * 4)) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->error, 4)) != cudaSuccess) return e;
+    b->logits_rows = sh.vocab;
+    if ((e = cudaMalloc(&b->logits, static_cast<size_t>(PF_VERIFY_MAX) * sh.vocab * 4)) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->att_o, static_cast<size_t>(AT_SPLIT_MAX) * AT_BM * qd * 4)) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->att_ml, static_cast<size_t>(AT_SPLIT_MAX) * AT_BM * sh.n_q_heads * 2 * 4)) != cudaSuccess) return e;
     if ((e = cudaMalloc(&b->head_val, PF_HEAD_GRID_MAX * PF_VERIFY_MAX * 4)) != cudaSuccess) return e;
@@ -1463,7 +1441,7 @@ cudaError_t prefill_alloc(PrefillBuffers *b, const edgefm_shape &sh, int chunk, 
 
 void prefill_free(PrefillBuffers *b) {
     cudaFree(b->resid); cudaFree(b->xn); cudaFree(b->part); cudaFree(b->kv_stage); cudaFree(b->q); cudaFree(b->attn); cudaFree(b->act); cudaFree(b->rope);
-    cudaFree(b->tokens); cudaFree(b->error); cudaFree(b->att_o); cudaFree(b->att_ml); cudaFree(b->head_val); cudaFree(b->head_idx); cudaFree(b->head_ticket);
+    cudaFree(b->tokens); cudaFree(b->error); cudaFree(b->logits); cudaFree(b->att_o); cudaFree(b->att_ml); cudaFree(b->head_val); cudaFree(b->head_idx); cudaFree(b->head_ticket);
     *b = PrefillBuffers{};
 }
 
@@ -1546,16 +1524,24 @@ const char *prefill_head(const PrefillModel &m, PrefillBuffers *b, int row, cons
 
 const char *prefill_verify_head(const PrefillModel &m, PrefillBuffers *b, int n, const void *final_norm, const void *lm, const int *ids, int rows,
                                 float *logits_out, int *n_accepted_out, int *next_token_out, int slot0, int pos, cudaStream_t s) {
+    // final norm of the block's rows (two bf16 planes), the logits of all rows as ONE contraction over the output matrix on the
+    // tensor cores (into the caller's buffer or the work buffer), then the greedy tokens and the acceptance rule
     const int H = m.shape.hidden;
-    int grid = 4 * m.num_sms;   // (48 KB of rows at the 1.5B shape: four CTAs per SM)
+    const size_t x_plane = static_cast<size_t>(b->chunk) * H;
+    float *logits = logits_out ? logits_out : b->logits;
+    if (!logits_out && rows > b->logits_rows) return "block verification: the work buffer for the logits is too small";
+    launch_pdl(prefill_norm_kernel, dim3(n), dim3(128), 0, s, b->resid, b->xn, x_plane, static_cast<const uint16_t *>(final_norm),
+               static_cast<const uint16_t *>(nullptr), static_cast<const int *>(nullptr), n, H, m.shape.rms_eps, static_cast<StepState *>(nullptr), 0, 0,
+               static_cast<const float *>(nullptr), 0, static_cast<size_t>(0));
+    GemmArgs g{};
+    g.M = n; g.N = rows; g.K = H; g.error = b->error; g.wait_limit = b->wait_limit; g.extra_arrivals = b->extra_arrivals;
+    g.resid = logits;
+    if (const char *e = launch_gemm<EPI_LOGITS>(b->xn, x_plane, lm, rows, g, m.num_sms, s)) return e;
+    int grid = m.num_sms;
     if (grid > PF_HEAD_GRID_MAX) grid = PF_HEAD_GRID_MAX;
-    if (grid * 8 > rows) grid = (rows + 7) / 8;
-    const size_t smem = static_cast<size_t>(n) * H * 4;
-    if (smem > 40 * 1024 && cudaFuncSetAttribute(prefill_verify_head_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)   // (the 48 KB default includes the static part)
-        return "cudaFuncSetAttribute failed";
-    launch_pdl(prefill_verify_head_kernel, dim3(grid), dim3(256), smem, s, b->resid, static_cast<const uint16_t *>(final_norm),
-               static_cast<const uint16_t *>(lm), ids, rows, H, m.shape.rms_eps, logits_out, n, b->tokens, b->head_val, b->head_idx, b->head_ticket,
-               m.state, slot0, pos, n_accepted_out, next_token_out);
+    if (grid * 256 > rows) grid = (rows + 255) / 256;
+    launch_pdl(prefill_verify_pick_kernel, dim3(grid), dim3(256), 0, s, static_cast<const float *>(logits), ids, rows, n, static_cast<const int *>(b->tokens),
+               b->head_val, b->head_idx, b->head_ticket, m.state, slot0, pos, n_accepted_out, next_token_out);
     return cudaGetLastError() == cudaSuccess ? nullptr : "block verification output layer launch failed";
 }
 

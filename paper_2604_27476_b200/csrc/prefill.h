@@ -33,6 +33,8 @@ struct PrefillBuffers {
     int *error = nullptr;        // device word: non-zero when a bounded wait of a GEMM ran out
     float *att_o = nullptr;      // attention of a lone query tile shared out among CTAs: partial rows fp32 [8][128][nq d]
     float *att_ml = nullptr;     // ... and their (reference maximum, row sum) [8][128][nq][2]
+    float *logits = nullptr;     // verified blocks: logits of the block's rows when the caller wants none, fp32 [8][vocab]
+    int logits_rows = 0;
     float *head_val = nullptr;   // output layer: the CTAs' greedy candidates
     int *head_idx = nullptr;
     unsigned *head_ticket = nullptr;
