@@ -262,3 +262,37 @@ def test_blocks_of_up_to_eight_tokens_through_the_dense_path(name, kv_format):
         assert ei.value.status == Status.ERR_INVALID_ARG
     finally:
         pair.close()
+
+
+def test_dense_block_with_a_pruned_output_layer():
+    """The dense path on a context whose output layer is pruned: greedy tokens and acceptance are taken over the subset (here every
+    second id plus the oracle's own choices, so that the oracle's unrestricted verification stays the reference)."""
+    import torch
+    cfg = CONFIGS["tiny"].with_(qkv_bias=True)
+    T0 = 24
+    pair = Pair(cfg, cache_len=T0, max_context=T0 + 16)
+    try:
+        tok, pos, m = 17, T0 + 2, 6
+        start = pair.oracle.cur_len
+        block, t = [tok], tok
+        for i in range(m - 1):
+            _, t = pair.oracle.step(t, pos + i)
+            block.append(t)
+        pair.oracle.truncate(start)
+        block[4] = (block[4] + 1) % cfg.vocab                       # the fifth token is a wrong proposal
+        ref_rows, ref_acc, ref_next = pair.oracle.verify_block(block, pos)
+        greedy = [int(np.argmax(ref_rows[i])) for i in range(m)]
+        ids = sorted(set(range(0, cfg.vocab, 2)) | set(greedy) | set(block))
+        pair.ctx.set_vocab_subset(ids)
+        pair.ctx.verify_block(block, pos)
+        torch.cuda.synchronize()
+        pair.ctx.sync_status()
+        got = pair.ctx.block_logits.cpu().numpy().reshape(-1)[:m * len(ids)].reshape(m, len(ids))
+        for i in range(ref_acc):
+            assert_logits_close(got[i], ref_rows[i][ids], f"row {i}, pruned")
+        if all(top2_margin(ref_rows[i]) > TOKEN_MARGIN for i in range(ref_acc)):
+            assert int(pair.ctx.n_accepted.item()) == ref_acc == 4
+            assert int(pair.ctx.next_token.item()) == ref_next
+            assert pair.ctx.sync_length() == start + ref_acc
+    finally:
+        pair.close()
